@@ -1,0 +1,237 @@
+"""CPU oracle for the SAR graph-attention aggregation (arXiv 2111.06483).
+
+TEST INFRASTRUCTURE ONLY: a plain float64 restatement of Eq. 2, Eq. 3, Algorithm 1
+(with the running max of Sec. 3.4) and the chain rule behind Algorithm 2, compiled from
+``sar_oracle.c`` with gcc and called through ctypes.  It imports nothing from the CUDA
+package and the CUDA package imports nothing from here.  Only tests, the smoke check
+and the benchmark's CPU-baseline / reference arm may use it.
+
+All array arguments are numpy arrays; floating inputs are float32 storage (bf16 cases pass
+bf16-rounded values held in float32), every result is float64.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "sar_oracle.c")
+_LIB = os.path.join(_HERE, "libsar_oracle.so")
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile sar_oracle.c into libsar_oracle.so next to it (gcc -O2 -fopenmp)."""
+    if force or (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", tmp, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+    return _lib
+
+
+def _p(a: np.ndarray, dtype):
+    assert a.dtype == dtype and a.flags["C_CONTIGUOUS"], (a.dtype, dtype)
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _i64(a):
+    return np.ascontiguousarray(a, dtype=np.int64)
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _f32(a):
+    return np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise RuntimeError(f"oracle {what} failed with code {rc}")
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def set_num_threads(n: int) -> None:
+    _load().oracle_set_num_threads(ctypes.c_int(int(n)))
+
+
+# --------------------------------------------------------------------------------------
+# integer side (Sec. 3.2, subgraphs G_{p,q})
+# --------------------------------------------------------------------------------------
+
+def csr_from_coo(n_dst: int, n_src: int, src, dst):
+    """CSR by destination of the edge list src[t] -> dst[t]; sources ascend within a row."""
+    src, dst = _i32(src), _i32(dst)
+    nnz = src.shape[0]
+    indptr = np.empty(n_dst + 1, dtype=np.int64)
+    indices = np.empty(nnz, dtype=np.int32)
+    rc = _load().oracle_csr_from_coo(ctypes.c_int64(n_dst), ctypes.c_int64(n_src), ctypes.c_int64(nnz),
+                                     _p(src, np.int32), _p(dst, np.int32), _p(indptr, np.int64),
+                                     _p(indices, np.int32))
+    _check(rc, "csr_from_coo")
+    return indptr, indices
+
+
+def csr_transpose(n_rows: int, n_cols: int, indptr, indices):
+    indptr, indices = _i64(indptr), _i32(indices)
+    t_indptr = np.empty(n_cols + 1, dtype=np.int64)
+    t_indices = np.empty(indices.shape[0], dtype=np.int32)
+    rc = _load().oracle_csr_transpose(ctypes.c_int64(n_rows), ctypes.c_int64(n_cols), _p(indptr, np.int64),
+                                      _p(indices, np.int32), _p(t_indptr, np.int64), _p(t_indices, np.int32))
+    _check(rc, "csr_transpose")
+    return t_indptr, t_indices
+
+
+def partition_bounds(n: int, k: int) -> np.ndarray:
+    bounds = np.empty(k + 1, dtype=np.int64)
+    _check(_load().oracle_partition_bounds(ctypes.c_int64(n), ctypes.c_int32(k), _p(bounds, np.int64)),
+           "partition_bounds")
+    return bounds
+
+
+@dataclass
+class SplitCSR:
+    """K per-partition CSRs in one block: partition q is indptr_all[q], indices_all[nnz_off[q]:nnz_off[q+1]]."""
+    n_dst: int
+    k: int
+    bounds: np.ndarray       # int64[k+1]
+    indptr_all: np.ndarray   # int64[k, n_dst+1]
+    indices_all: np.ndarray  # int32[nnz], local source ids
+    nnz_off: np.ndarray      # int64[k+1]
+
+    def part(self, q: int):
+        return self.indptr_all[q], self.indices_all[self.nnz_off[q]:self.nnz_off[q + 1]]
+
+
+def csr_split(n_dst: int, indptr, indices, bounds) -> SplitCSR:
+    indptr, indices, bounds = _i64(indptr), _i32(indices), _i64(bounds)
+    k = bounds.shape[0] - 1
+    indptr_all = np.empty((k, n_dst + 1), dtype=np.int64)
+    indices_all = np.empty(indices.shape[0], dtype=np.int32)
+    nnz_off = np.empty(k + 1, dtype=np.int64)
+    rc = _load().oracle_csr_split(ctypes.c_int64(n_dst), _p(indptr, np.int64), _p(indices, np.int32),
+                                  ctypes.c_int32(k), _p(bounds, np.int64), _p(indptr_all, np.int64),
+                                  _p(indices_all, np.int32), _p(nnz_off, np.int64))
+    _check(rc, "csr_split")
+    return SplitCSR(n_dst, k, bounds, indptr_all, indices_all, nnz_off)
+
+
+# --------------------------------------------------------------------------------------
+# floating side
+# --------------------------------------------------------------------------------------
+
+@dataclass
+class GatForward:
+    e: np.ndarray      # [nnz,H]  LeakyReLU(el_i + er_j)
+    alpha: np.ndarray  # [nnz,H]  softmax over each destination's in-edges
+    out: np.ndarray    # [n_dst,H,F]
+    m: np.ndarray      # [n_dst,H] row max of e (-inf for empty rows)
+    d: np.ndarray      # [n_dst,H] sum of exp(e - m) (0 for empty rows)
+
+
+def gat_fwd(indptr, indices, feat, el, er, slope: float) -> GatForward:
+    """Eq. 3 as written: per-edge scores, softmax over each in-neighbourhood, weighted sum."""
+    indptr, indices = _i64(indptr), _i32(indices)
+    feat, el, er = _f32(feat), _f32(el), _f32(er)
+    n_dst = indptr.shape[0] - 1
+    _, H, F = feat.shape
+    assert el.shape == (n_dst, H) and er.shape == (feat.shape[0], H)
+    nnz = indices.shape[0]
+    assert int(indptr[-1]) == nnz
+    if nnz:
+        assert indices.min() >= 0 and indices.max() < feat.shape[0]
+    e = np.empty((nnz, H), dtype=np.float64)
+    alpha = np.empty((nnz, H), dtype=np.float64)
+    out = np.empty((n_dst, H, F), dtype=np.float64)
+    m = np.empty((n_dst, H), dtype=np.float64)
+    d = np.empty((n_dst, H), dtype=np.float64)
+    rc = _load().oracle_gat_fwd(ctypes.c_int64(n_dst), _p(indptr, np.int64), _p(indices, np.int32),
+                                _p(feat, np.float32), _p(el, np.float32), _p(er, np.float32),
+                                ctypes.c_int32(H), ctypes.c_int32(F), ctypes.c_double(slope),
+                                _p(e, np.float64), _p(alpha, np.float64), _p(out, np.float64),
+                                _p(m, np.float64), _p(d, np.float64))
+    _check(rc, "gat_fwd")
+    return GatForward(e, alpha, out, m, d)
+
+
+@dataclass
+class GatBackward:
+    D: np.ndarray      # [n_dst,H]  sum_t alpha*dalpha
+    dfeat: np.ndarray  # [n_src,H,F]
+    del_: np.ndarray   # [n_dst,H]
+    der: np.ndarray    # [n_src,H]
+
+
+def gat_bwd(indptr, indices, feat, el, er, alpha, gout, slope: float) -> GatBackward:
+    """Chain rule on Eq. 3 with the per-edge alpha of gat_fwd."""
+    indptr, indices = _i64(indptr), _i32(indices)
+    feat, el, er, gout = _f32(feat), _f32(el), _f32(er), _f32(gout)
+    alpha = np.ascontiguousarray(alpha, dtype=np.float64)
+    n_dst = indptr.shape[0] - 1
+    n_src, H, F = feat.shape
+    assert gout.shape == (n_dst, H, F) and alpha.shape == (indices.shape[0], H)
+    D = np.empty((n_dst, H), dtype=np.float64)
+    dfeat = np.empty((n_src, H, F), dtype=np.float64)
+    del_ = np.empty((n_dst, H), dtype=np.float64)
+    der = np.empty((n_src, H), dtype=np.float64)
+    rc = _load().oracle_gat_bwd(ctypes.c_int64(n_dst), ctypes.c_int64(n_src), _p(indptr, np.int64),
+                                _p(indices, np.int32), _p(feat, np.float32), _p(el, np.float32),
+                                _p(er, np.float32), _p(alpha, np.float64), _p(gout, np.float32),
+                                ctypes.c_int32(H), ctypes.c_int32(F), ctypes.c_double(slope),
+                                _p(D, np.float64), _p(dfeat, np.float64), _p(del_, np.float64),
+                                _p(der, np.float64))
+    _check(rc, "gat_bwd")
+    return GatBackward(D, dfeat, del_, der)
+
+
+def gat_fwd_seq(split: SplitCSR, feat, el, er, slope: float, order=None):
+    """Algorithm 1 + running max (Sec. 3.4): partitions visited one by one. Returns (out, m, d)."""
+    feat, el, er = _f32(feat), _f32(el), _f32(er)
+    n_dst, k = split.n_dst, split.k
+    _, H, F = feat.shape
+    order = _i32(np.arange(k) if order is None else order)
+    assert sorted(order.tolist()) == list(range(k))
+    out = np.empty((n_dst, H, F), dtype=np.float64)
+    m = np.empty((n_dst, H), dtype=np.float64)
+    d = np.empty((n_dst, H), dtype=np.float64)
+    rc = _load().oracle_gat_fwd_seq(ctypes.c_int64(n_dst), ctypes.c_int32(k), _p(split.bounds, np.int64),
+                                    _p(order, np.int32), _p(split.indptr_all, np.int64),
+                                    _p(split.indices_all, np.int32), _p(split.nnz_off, np.int64),
+                                    _p(feat, np.float32), _p(el, np.float32), _p(er, np.float32),
+                                    ctypes.c_int32(H), ctypes.c_int32(F), ctypes.c_double(slope),
+                                    _p(out, np.float64), _p(m, np.float64), _p(d, np.float64))
+    _check(rc, "gat_fwd_seq")
+    return out, m, d
+
+
+def spmm(indptr, indices, feat, mean: bool = False) -> np.ndarray:
+    """Eq. 2's neighbour sum (mean=True divides by the in-degree)."""
+    indptr, indices = _i64(indptr), _i32(indices)
+    feat = _f32(feat)
+    n_dst = indptr.shape[0] - 1
+    F = feat.shape[1]
+    if indices.shape[0]:
+        assert indices.min() >= 0 and indices.max() < feat.shape[0]
+    out = np.empty((n_dst, F), dtype=np.float64)
+    rc = _load().oracle_spmm(ctypes.c_int64(n_dst), _p(indptr, np.int64), _p(indices, np.int32),
+                             _p(feat, np.float32), ctypes.c_int32(F), ctypes.c_int32(1 if mean else 0),
+                             _p(out, np.float64))
+    _check(rc, "spmm")
+    return out
