@@ -1,0 +1,244 @@
+/*
+ * libsar — fused graph-attention aggregation with attention rematerialisation for one
+ * NVIDIA B200 (sm_100a), after "Sequential Aggregation and Rematerialization" (SAR,
+ * arXiv 2111.06483).
+ *
+ * What the library computes
+ *   Forward (Eq. 3 of the paper, fused as Sec. 3.3 describes): for every destination node i
+ *   and head h, edge scores e = LeakyReLU(el[i,h] + er[j,h]) over the in-edges j -> i, a softmax
+ *   over them and the weighted sum of the neighbours' feature rows, WITHOUT writing the E x H
+ *   attention matrix; only the row max m[i,h] and the normaliser d[i,h] are kept.
+ *   Sequential aggregation (Sec. 3.2, Algorithm 1, "Stable softmax" in Sec. 3.4): the sources
+ *   are split into K partitions that are visited one after the other; the un-normalised
+ *   numerator and the normaliser are accumulated separately under a running max, corrected by
+ *   exp(old_max - new_max) whenever the max moves, and divided at the end.
+ *   Backward (Algorithm 2 with the rematerialisation of Sec. 3.3): the attention is rebuilt from
+ *   (el, er, m, d) per partition to produce dFeat, dEl and dEr.
+ *   Sum aggregation (Eq. 2, "case 1" of Sec. 3.2).
+ *
+ * Conventions
+ *   - Every function returns a sar_status; nothing throws, aborts or prints.
+ *   - Unless a parameter is marked HOST, every pointer is a DEVICE pointer BORROWED from the
+ *     caller for the duration of the enqueued work; the library never allocates or frees
+ *     device memory (except where an entry point documents otherwise) and keeps no state
+ *     between calls.  Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream) and the call returns without synchronising.
+ *   - Argument errors are detected on the host before anything is launched.
+ *   - Arrays are dense, row-major, contiguous.  A graph is a CSR by DESTINATION: row i of
+ *     (indptr, indices) lists the sources j of the edges j -> i in ascending order, duplicate
+ *     edges kept.  indptr is int64, indices int32; every element offset is computed in 64 bits.
+ *   - el[i,h] is the DESTINATION term of the score and er[j,h] the SOURCE term (the two halves of
+ *     a^T (z_i || z_j) in Eq. 3).
+ *   - A destination without in-edges gets out = 0, d = 0, m = -inf and no gradient.  The
+ *     derivative of LeakyReLU at 0 is `slope`.  The running max is a constant in the backward
+ *     pass (the softmax is shift invariant).
+ *   - sar_dtype is the STORAGE type of feat / out / gout / dfeat.  el, er, m, d, D, del, der, the
+ *     running numerator `acc` and every accumulation are float32.
+ *   - The fast kernels need 16-byte aligned feature arrays and F * sizeof(element) a multiple of
+ *     16 bytes; other shapes run on slower scalar kernels with the same results.
+ */
+#ifndef SAR_H_
+#define SAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define SAR_API __attribute__((visibility("default")))
+#else
+#define SAR_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SAR_OK = 0,
+    SAR_ERR_INVALID_ARG = -1, /* null pointer, negative size, bad flag combination          */
+    SAR_ERR_UNSUPPORTED = -2, /* shape outside what the kernels cover (see SAR_MAX_*)       */
+    SAR_ERR_ALIGNMENT = -3,   /* a pointer is not aligned to its element type               */
+    SAR_ERR_WORKSPACE = -4,   /* workspace missing or smaller than *_workspace_bytes says   */
+    SAR_ERR_CUDA = -5,        /* a CUDA runtime call or launch failed                       */
+    SAR_ERR_BAD_GRAPH = -6    /* sar_validate_part found an inconsistent graph              */
+} sar_status;
+
+typedef enum { SAR_F32 = 0, SAR_BF16 = 1 } sar_dtype;
+
+/* flags */
+#define SAR_FIRST 1u /* first partition: ignore incoming running state / overwrite outputs   */
+#define SAR_LAST 2u  /* last partition: normalise and write the final result                 */
+#define SAR_MEAN 4u  /* sar_spmm_agg with SAR_LAST: divide by `deg_total`                    */
+
+#define SAR_MAX_HEADS 16
+#define SAR_MAX_PARTS 64
+#define SAR_MAX_ROW_BYTES 4096 /* H*F*sizeof(element) handled by the fast kernels             */
+
+/* Optional split of long rows into segments, built once per graph by sar_plan_build.  Rows
+ * with more than `threshold` edges are cut into segments of at most `threshold` edges that
+ * are processed in parallel and merged by a second launch (no atomics).  All arrays DEVICE. */
+typedef struct {
+    int32_t threshold;        /* rows with degree > threshold are split                       */
+    int32_t n_long;           /* number of such rows                                          */
+    int64_t n_seg;            /* total number of segments over all long rows                  */
+    const int32_t *long_row;  /* [n_long]   row ids, ascending                                */
+    const int64_t *long_seg;  /* [n_long+1] first segment of each long row                    */
+} sar_split;
+
+/* One source partition q of the graph as worker p sees it (the subgraph G_{p,q} of Sec. 3.2).
+ * On one GPU p owns every destination, so n_dst is the node count. */
+typedef struct {
+    int64_t n_dst;             /* destination rows                                            */
+    int64_t n_src;             /* sources in this partition                                   */
+    int64_t nnz;               /* edges from this partition's sources                         */
+    const int64_t *indptr;     /* [n_dst+1] CSR by destination                                */
+    const int32_t *indices;    /* [nnz] LOCAL source id in [0,n_src), ascending within a row  */
+    const int64_t *t_indptr;   /* [n_src+1] the same edges grouped by local source (CSC);     */
+    const int32_t *t_indices;  /* [nnz] destination id, ascending within a source; both may   */
+                               /* be NULL when only forward calls are made                    */
+    const sar_split *split;    /* HOST pointer or NULL: long-row split of (indptr, indices)   */
+    const sar_split *t_split;  /* HOST pointer or NULL: long-row split of the CSC             */
+} sar_part;
+
+SAR_API const char *sar_status_string(sar_status s);
+/* Compile-time facts: returns the SM architecture the kernels were built for (100). */
+SAR_API int32_t sar_built_for_sm(void);
+
+/* ---------------------------------------------------------------------------------------------
+ * Graph preparation (construction of the subgraphs G_{p,q}, Sec. 3.2).  Integer work; results
+ * are unique and therefore bit-reproducible.
+ * ------------------------------------------------------------------------------------------- */
+
+/* Bytes of scratch the graph-preparation calls below need for a graph of `nnz` edges and `n_rows`
+ * rows (an upper bound that covers every one of them). */
+SAR_API size_t sar_graph_workspace_bytes(int64_t nnz, int64_t n_rows);
+
+/* Edge list -> CSR.  Edge t goes from column col[t] to row row[t]; output row r lists its
+ * columns in ascending order (duplicates adjacent).  For the CSR by destination pass
+ * row = dst, col = src; for the CSC pass row = src, col = dst.
+ * indptr: [n_rows+1] written; indices: [nnz] written.  Ids must lie in range (not checked). */
+SAR_API sar_status sar_csr_from_coo(int64_t n_rows, int64_t n_cols, int64_t nnz, const int32_t *row,
+                            const int32_t *col, int64_t *indptr, int32_t *indices, void *workspace,
+                            size_t workspace_bytes, void *stream);
+
+/* CSR (n_rows x n_cols) -> its transpose (n_cols x n_rows), same ordering rule. */
+SAR_API sar_status sar_csr_transpose(int64_t n_rows, int64_t n_cols, const int64_t *indptr, const int32_t *indices,
+                             int64_t *t_indptr, int32_t *t_indices, void *workspace, size_t workspace_bytes,
+                             void *stream);
+
+/* Contiguous source ranges s_q = floor(q*n/k); bounds is a HOST array of k+1 entries. */
+SAR_API sar_status sar_partition_bounds(int64_t n, int32_t k, int64_t *bounds);
+
+/* Split a CSR by source range in two steps (the caller sizes the index array in between).
+ * Step 1 writes indptr_all: k arrays of n_dst+1 entries, array q being the indptr of the
+ * sub-graph that keeps only sources bounds[q] <= j < bounds[q+1] (HOST bounds, k <= SAR_MAX_PARTS).
+ * The caller then reads nnz_q = indptr_all[q*(n_dst+1) + n_dst], forms the HOST prefix sums
+ * nnz_off[0..k] and calls step 2, which writes partition q's LOCAL ids j - bounds[q] to
+ * indices_all[nnz_off[q] .. nnz_off[q+1]). */
+SAR_API sar_status sar_csr_split_indptr(int64_t n_dst, const int64_t *indptr, const int32_t *indices, int32_t k,
+                                const int64_t *bounds, int64_t *indptr_all, void *workspace,
+                                size_t workspace_bytes, void *stream);
+SAR_API sar_status sar_csr_split_indices(int64_t n_dst, const int64_t *indptr, const int32_t *indices, int32_t k,
+                                 const int64_t *bounds, const int64_t *indptr_all, const int64_t *nnz_off,
+                                 int32_t *indices_all, void *stream);
+
+/* Debug scan of one partition: indptr monotone from 0 to nnz, ids in range and ascending within a
+ * row (both orientations when the CSC is present).  `flag` is 4 bytes of DEVICE scratch.
+ * Synchronises the stream.  The hot calls never scan the graph. */
+SAR_API sar_status sar_validate_part(const sar_part *g, int32_t *flag, void *stream);
+
+/* Long-row plan (see sar_split).  Step 1 counts the rows with more than `threshold` edges and their
+ * segments into the HOST variables n_long / n_seg, using 16 bytes of DEVICE scratch `counts`
+ * (synchronises the stream).  Step 2 fills the DEVICE arrays long_row[n_long], long_seg[n_long+1]. */
+SAR_API sar_status sar_plan_count(int64_t n_rows, const int64_t *indptr, int32_t threshold, int64_t *counts,
+                          int32_t *n_long, int64_t *n_seg, void *stream);
+SAR_API sar_status sar_plan_fill(int64_t n_rows, const int64_t *indptr, int32_t threshold, int32_t n_long,
+                         int32_t *long_row, int64_t *long_seg, void *workspace, size_t workspace_bytes,
+                         void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Fused GAT aggregation, forward (Eq. 3; Algorithm 1; Sec. 3.3; running max of Sec. 3.4).
+ * ------------------------------------------------------------------------------------------- */
+
+/* Scratch bytes the forward / backward calls need for this partition (long-row partials and, for
+ * the backward pass, 16 bytes per (destination, head)). */
+SAR_API size_t sar_gat_workspace_bytes(const sar_part *g, int32_t H, int32_t F, sar_dtype t);
+
+/* One step of Algorithm 1's loop: fold partition q into the running state.
+ *   feat_q [n_src,H,F] (storage type t), el [n_dst,H], er_q [n_src,H].
+ *   acc [n_dst,H,F] float32 running numerator, m [n_dst,H] running max, d [n_dst,H] running
+ *   normaliser: read unless SAR_FIRST, written unless SAR_LAST (m, d are always written).
+ *   With SAR_LAST, out [n_dst,H,F] (type t) = acc/d is written (0 where d == 0) and m, d hold the
+ *   final statistics the backward pass needs.  With SAR_FIRST|SAR_LAST (one partition holding all
+ *   sources) acc may be NULL: the numerator never leaves the registers.
+ *   Destinations without edges in this partition are skipped unless a flag forces a write. */
+SAR_API sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, const float *er_q, int32_t H,
+                       int32_t F, sar_dtype t, float slope, uint32_t flags, float *acc, float *m, float *d,
+                       void *out, void *workspace, size_t workspace_bytes, void *stream);
+
+/* The whole loop of Algorithm 1 in one launch, row-stationary: `g` is the UN-split graph (global
+ * source ids, n_src = all sources); partition q owns the sources bounds[q] <= j < bounds[q+1]
+ * (HOST bounds) whose rows live at feat_q[q] / er_q[q] (HOST arrays of k DEVICE pointers, e.g.
+ * buffers fetched from k different owners).  Each destination walks its in-edges in ascending
+ * source order, i.e. partition after partition, carrying (running max, normaliser, numerator) in
+ * registers with the same correction rule, so nothing of size n_dst*H*F is re-read between
+ * partitions.  Writes out, m, d as sar_gat_fwd does with SAR_LAST. */
+SAR_API sar_status sar_gat_fwd_fused(const sar_part *g, int32_t k, const int64_t *bounds, const void *const *feat_q,
+                             const float *el, const float *const *er_q, int32_t H, int32_t F, sar_dtype t,
+                             float slope, float *m, float *d, void *out, void *workspace,
+                             size_t workspace_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Fused GAT aggregation, backward (Algorithm 2 restricted to the aggregation; attention rebuilt
+ * from (el, er, m, d) as Sec. 3.3 describes).  With alpha = exp(e - m)/d, dalpha = <gout_i, feat_j>,
+ * D_i = sum_j alpha*dalpha (= <gout_i, out_i>), ds = alpha*(dalpha - D_i)*LeakyReLU'(s):
+ *   dfeat[j] = sum_i alpha*gout[i],  der[j] = sum_i ds,  del[i] = sum_j ds.
+ * ------------------------------------------------------------------------------------------- */
+
+/* Row dot D[i,h] = <gout[i,h,:], out[i,h,:]> and the packed per-destination record
+ * {el, m, 1/d, D} (16 bytes per (i,h), written to the start of `workspace`) that lets each
+ * partition's backward step run independently of the others.  `out` may be given as the float32
+ * numerator `acc` with acc_is_numerator != 0 (then out = acc/d is formed on the fly), which avoids
+ * the rounding of a bf16 `out`.  D may be NULL. */
+SAR_API sar_status sar_gat_bwd_prepare(int64_t n_dst, int32_t H, int32_t F, sar_dtype t, const void *out_or_acc,
+                               int32_t acc_is_numerator, const void *gout, const float *el, const float *m,
+                               const float *d, float *D, void *workspace, size_t workspace_bytes,
+                               void *stream);
+
+/* One step of Algorithm 2's loop for partition q.  m, d are the FINAL statistics.
+ *   dfeat_q [n_src,H,F] (type t) and der_q [n_src,H] are written (this partition's sources receive
+ *   all their gradient here, since every destination is local); del [n_dst,H] is written with
+ *   SAR_FIRST and accumulated otherwise.
+ *   With SAR_FIRST|SAR_LAST (one partition holding all sources) D is rebuilt from the edges and
+ *   sar_gat_bwd_prepare is not needed; otherwise `workspace` must hold what sar_gat_bwd_prepare
+ *   wrote for these (gout, m, d).  Needs g->t_indptr / g->t_indices. */
+SAR_API sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, const float *er_q,
+                       const float *m, const float *d, const void *gout, int32_t H, int32_t F, sar_dtype t,
+                       float slope, uint32_t flags, void *dfeat_q, float *del, float *der_q, void *workspace,
+                       size_t workspace_bytes, void *stream);
+
+/* The whole loop of Algorithm 2 on the un-split graph (see sar_gat_fwd_fused for the argument
+ * conventions): dfeat_q[q], der_q[q] are HOST arrays of k DEVICE pointers to each partition's
+ * gradient buffers. */
+SAR_API sar_status sar_gat_bwd_fused(const sar_part *g, int32_t k, const int64_t *bounds, const void *const *feat_q,
+                             const float *el, const float *const *er_q, const float *m, const float *d,
+                             const void *gout, int32_t H, int32_t F, sar_dtype t, float slope,
+                             void *const *dfeat_q, float *del, float *const *der_q, void *workspace,
+                             size_t workspace_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Sum aggregation (Eq. 2; Sec. 3.2 "case 1").  out[i,:] (+)= sum over this partition's in-edges of
+ * feat_q[j,:]; feat_q [n_src,F], out [n_dst,F], both of type t, float32 accumulation within the
+ * call.  SAR_FIRST overwrites out, otherwise the partition's sum is added to it.  SAR_MEAN with
+ * SAR_LAST divides the result by deg_total[i] (int64 [n_dst] total in-degree over all partitions;
+ * rows with degree 0 stay 0).  The backward pass of the sum is this same call on the transposed
+ * partition applied to gout. */
+SAR_API sar_status sar_spmm_agg(const sar_part *g, const void *feat_q, int32_t F, sar_dtype t, uint32_t flags,
+                        const int64_t *deg_total, void *out, void *workspace, size_t workspace_bytes,
+                        void *stream);
+SAR_API size_t sar_spmm_workspace_bytes(const sar_part *g, int32_t F, sar_dtype t);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SAR_H_ */

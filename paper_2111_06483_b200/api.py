@@ -1,0 +1,165 @@
+"""Convenience layer over the binding: allocates device tensors with torch and calls libsar.
+
+Nothing is computed here; every step (graph build, transpose, split, long-row plan, forward,
+backward, sum aggregation) is a call into the C-ABI library.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import List, Optional
+
+import torch
+
+from . import binding as B
+
+DEFAULT_THRESHOLD = 512  # rows with more edges are cut into segments of this many edges
+
+
+def _workspace(nbytes: int, device) -> torch.Tensor:
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+def build_plan(n_rows: int, indptr: torch.Tensor, threshold: int) -> Optional[B.Split]:
+    """Long-row plan of one CSR (None when no row is longer than `threshold`)."""
+    dev = indptr.device
+    counts = torch.zeros(2, dtype=torch.int64, device=dev)
+    n_long, n_seg = B.sar_plan_count(n_rows, indptr, threshold, counts)
+    if n_long == 0:
+        return None
+    long_row = torch.empty(n_long, dtype=torch.int32, device=dev)
+    long_seg = torch.empty(n_long + 1, dtype=torch.int64, device=dev)
+    ws = _workspace(B.sar_graph_workspace_bytes(0, n_rows), dev)
+    B.sar_plan_fill(n_rows, indptr, threshold, n_long, long_row, long_seg, ws)
+    return B.Split(threshold, n_long, n_seg, long_row, long_seg)
+
+
+@dataclass
+class Graph:
+    """A graph on the device: the un-split CSR/CSC (`whole`) and, optionally, its K source partitions."""
+    n: int
+    nnz: int
+    whole: B.Part
+    k: int = 1
+    bounds: List[int] = field(default_factory=list)
+    parts: List[B.Part] = field(default_factory=list)
+
+    @staticmethod
+    def from_coo(n: int, src: torch.Tensor, dst: torch.Tensor, k: int = 1, threshold: int = DEFAULT_THRESHOLD,
+                 build_parts: bool = False) -> "Graph":
+        """src[t] -> dst[t] int32 CUDA tensors.  Builds CSR by destination, its transpose, the long-row
+        plans and (build_parts) the K per-partition sub-graphs with local source ids."""
+        dev = src.device
+        nnz = src.numel()
+        ws = _workspace(B.sar_graph_workspace_bytes(nnz, n), dev)
+        indptr = torch.empty(n + 1, dtype=torch.int64, device=dev)
+        indices = torch.empty(nnz, dtype=torch.int32, device=dev)
+        B.sar_csr_from_coo(n, n, dst, src, indptr, indices, ws)
+        t_indptr = torch.empty(n + 1, dtype=torch.int64, device=dev)
+        t_indices = torch.empty(nnz, dtype=torch.int32, device=dev)
+        B.sar_csr_from_coo(n, n, src, dst, t_indptr, t_indices, ws)
+        split = build_plan(n, indptr, threshold) if threshold else None
+        t_split = build_plan(n, t_indptr, threshold) if threshold else None
+        whole = B.Part(n, n, indptr, indices, t_indptr, t_indices, split, t_split)
+        g = Graph(n=n, nnz=nnz, whole=whole, k=k, bounds=B.sar_partition_bounds(n, k))
+        if build_parts:
+            g.parts = split_parts(whole, g.bounds, threshold, ws)
+        return g
+
+
+def split_parts(whole: B.Part, bounds: List[int], threshold: int, ws: Optional[torch.Tensor] = None) -> List[B.Part]:
+    """The K sub-graphs G_{p,q}: CSR with local source ids (split on the device) and CSC slices."""
+    dev = whole.indptr.device
+    n, k = whole.n_dst, len(bounds) - 1
+    if ws is None:
+        ws = _workspace(B.sar_graph_workspace_bytes(whole.nnz, n), dev)
+    indptr_all = torch.empty((k, n + 1), dtype=torch.int64, device=dev)
+    B.sar_csr_split_indptr(n, whole.indptr, whole.indices, bounds, indptr_all, ws)
+    nnz_q = indptr_all[:, n].tolist()
+    nnz_off = [0]
+    for c in nnz_q:
+        nnz_off.append(nnz_off[-1] + int(c))
+    indices_all = torch.empty(max(nnz_off[-1], 1), dtype=torch.int32, device=dev)
+    B.sar_csr_split_indices(n, whole.indptr, whole.indices, bounds, indptr_all, nnz_off, indices_all)
+    parts = []
+    for q in range(k):
+        s0, s1 = bounds[q], bounds[q + 1]
+        ip = indptr_all[q]
+        idx = indices_all[nnz_off[q]:nnz_off[q + 1]]
+        # CSC of partition q: the sources s0..s1 of the whole CSC, offsets rebased to 0
+        t_ip = (whole.t_indptr[s0:s1 + 1] - whole.t_indptr[s0]).contiguous()
+        e0 = int(whole.t_indptr[s0])
+        t_idx = whole.t_indices[e0:e0 + nnz_q[q]]
+        split = build_plan(n, ip, threshold) if threshold else None
+        t_split = build_plan(s1 - s0, t_ip, threshold) if threshold else None
+        parts.append(B.Part(n, s1 - s0, ip, idx, t_ip, t_idx, split, t_split, nnz=nnz_q[q]))
+    return parts
+
+
+# ----------------------------------------------------------------------------------------------
+
+def gat_workspace(part: B.Part, H: int, F: int, dtype: torch.dtype) -> torch.Tensor:
+    code = B.SAR_BF16 if dtype == torch.bfloat16 else B.SAR_F32
+    return _workspace(B.sar_gat_workspace_bytes(part, H, F, code), part.indptr.device)
+
+
+def gat_forward(g: Graph, feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor, slope: float,
+                workspace: Optional[torch.Tensor] = None, mode: str = "fused"):
+    """Forward over the K partitions.  mode "fused": one row-stationary launch (sar_gat_fwd_fused);
+    mode "stateful": K calls of sar_gat_fwd with the running state in global memory (Algorithm 1)."""
+    n, H, F = feat.shape
+    dev = feat.device
+    m = torch.empty((g.n, H), dtype=torch.float32, device=dev)
+    d = torch.empty((g.n, H), dtype=torch.float32, device=dev)
+    out = torch.empty((g.n, H, F), dtype=feat.dtype, device=dev)
+    if mode == "fused":
+        ws = workspace if workspace is not None else gat_workspace(g.whole, H, F, feat.dtype)
+        feat_q = [feat[g.bounds[q]:] for q in range(g.k)]
+        er_q = [er[g.bounds[q]:] for q in range(g.k)]
+        B.sar_gat_fwd_fused(g.whole, g.bounds, feat_q, el, er_q, H, F, slope, m, d, out, ws)
+        return out, m, d
+    assert g.parts, "stateful mode needs Graph.from_coo(..., build_parts=True)"
+    acc = torch.empty((g.n, H, F), dtype=torch.float32, device=dev) if g.k > 1 else None
+    for q, part in enumerate(g.parts):
+        flags = (B.SAR_FIRST if q == 0 else 0) | (B.SAR_LAST if q == g.k - 1 else 0)
+        ws = gat_workspace(part, H, F, feat.dtype)
+        s0, s1 = g.bounds[q], g.bounds[q + 1]
+        B.sar_gat_fwd(part, feat[s0:s1], el, er[s0:s1], H, F, slope, flags, acc, m, d, out, ws)
+    return out, m, d
+
+
+def gat_backward(g: Graph, feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor, m: torch.Tensor,
+                 d: torch.Tensor, gout: torch.Tensor, slope: float, out: Optional[torch.Tensor] = None,
+                 workspace: Optional[torch.Tensor] = None, mode: str = "fused"):
+    """Backward over the K partitions; returns (dfeat, del, der).  "stateful" needs `out` (for the
+    row dot) and runs sar_gat_bwd_prepare followed by K calls of sar_gat_bwd."""
+    n, H, F = feat.shape
+    dev = feat.device
+    dfeat = torch.empty_like(feat)
+    del_ = torch.empty((g.n, H), dtype=torch.float32, device=dev)
+    der = torch.empty((g.n, H), dtype=torch.float32, device=dev)
+    if mode == "fused":
+        ws = workspace if workspace is not None else gat_workspace(g.whole, H, F, feat.dtype)
+        sl = lambda t: [t[g.bounds[q]:] for q in range(g.k)]
+        B.sar_gat_bwd_fused(g.whole, g.bounds, sl(feat), el, sl(er), m, d, gout, H, F, slope, sl(dfeat), del_,
+                            sl(der), ws)
+        return dfeat, del_, der
+    assert g.parts and out is not None
+    nbytes = max(B.sar_gat_workspace_bytes(p, H, F, B._dtype(feat)) for p in g.parts)
+    ws = _workspace(nbytes, dev)
+    B.sar_gat_bwd_prepare(g.n, H, F, out, False, gout, el, m, d, None, ws)
+    for q, part in enumerate(g.parts):
+        flags = (B.SAR_FIRST if q == 0 else 0) | (B.SAR_LAST if q == g.k - 1 else 0)
+        s0, s1 = g.bounds[q], g.bounds[q + 1]
+        B.sar_gat_bwd(part, feat[s0:s1], el, er[s0:s1], m, d, gout, H, F, slope, flags, dfeat[s0:s1], del_,
+                      der[s0:s1], ws)
+    return dfeat, del_, der
+
+
+def spmm_sum(part: B.Part, feat: torch.Tensor, mean: bool = False, deg_total: Optional[torch.Tensor] = None):
+    """out[i,:] = sum (or mean) of feat over the in-edges of i for one partition holding all sources."""
+    F = feat.shape[1]
+    out = torch.empty((part.n_dst, F), dtype=feat.dtype, device=feat.device)
+    ws = _workspace(B.sar_spmm_workspace_bytes(part, F, B._dtype(feat)), feat.device)
+    flags = B.SAR_FIRST | B.SAR_LAST | (B.SAR_MEAN if mean else 0)
+    B.sar_spmm_agg(part, feat, F, flags, deg_total, out, ws)
+    return out

@@ -1,0 +1,282 @@
+"""ctypes binding of libsar.so (include/sar.h): argument marshalling only.
+
+Every function here has the name of the C entry point it calls and does nothing but turn
+torch CUDA tensors into pointers (PyTorch supplies device memory and the current stream) and
+check the returned status.  There is no Python or CPU fallback: if the library cannot be loaded
+the import of this module's functions fails loudly.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, Structure, byref, c_char_p, c_float, c_int32, c_int64, c_size_t, c_uint32, c_void_p
+from typing import Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libsar.so")
+
+SAR_OK = 0
+SAR_F32, SAR_BF16 = 0, 1
+SAR_FIRST, SAR_LAST, SAR_MEAN = 1, 2, 4
+SAR_MAX_PARTS = 64
+
+EXPORTS = [
+    "sar_status_string", "sar_built_for_sm", "sar_graph_workspace_bytes", "sar_csr_from_coo", "sar_csr_transpose",
+    "sar_partition_bounds", "sar_csr_split_indptr", "sar_csr_split_indices", "sar_validate_part", "sar_plan_count",
+    "sar_plan_fill", "sar_gat_workspace_bytes", "sar_gat_fwd", "sar_gat_fwd_fused", "sar_gat_bwd_prepare",
+    "sar_gat_bwd", "sar_gat_bwd_fused", "sar_spmm_agg", "sar_spmm_workspace_bytes",
+]
+
+
+class SarError(RuntimeError):
+    def __init__(self, fn: str, code: int, text: str):
+        super().__init__(f"{fn} failed: {text} (status {code})")
+        self.code = code
+
+
+class sar_split(Structure):
+    _fields_ = [("threshold", c_int32), ("n_long", c_int32), ("n_seg", c_int64), ("long_row", c_void_p),
+                ("long_seg", c_void_p)]
+
+
+class sar_part(Structure):
+    _fields_ = [("n_dst", c_int64), ("n_src", c_int64), ("nnz", c_int64), ("indptr", c_void_p),
+                ("indices", c_void_p), ("t_indptr", c_void_p), ("t_indices", c_void_p),
+                ("split", POINTER(sar_split)), ("t_split", POINTER(sar_split))]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded library.  Raises if libsar.so is missing: build it with
+    `python -m paper_2111_06483_b200.build` (there is no other code path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(f"{LIB_PATH} not found: run `python -m paper_2111_06483_b200.build` "
+                               "(libsar has no CPU or PyTorch fallback)")
+        L = ctypes.CDLL(LIB_PATH)
+        L.sar_status_string.restype = c_char_p
+        L.sar_status_string.argtypes = [ctypes.c_int]
+        L.sar_built_for_sm.restype = c_int32
+        for name in ("sar_graph_workspace_bytes", "sar_gat_workspace_bytes", "sar_spmm_workspace_bytes"):
+            getattr(L, name).restype = c_size_t
+        _lib = L
+    return _lib
+
+
+def _check(fn: str, code: int) -> None:
+    if code != SAR_OK:
+        raise SarError(fn, code, lib().sar_status_string(code).decode())
+
+
+def _ptr(t: Optional[torch.Tensor]) -> c_void_p:
+    if t is None:
+        return c_void_p(0)
+    assert t.is_cuda and t.is_contiguous(), "libsar takes contiguous CUDA tensors"
+    return c_void_p(t.data_ptr())
+
+
+def _stream() -> c_void_p:
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _dtype(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return SAR_F32
+    if t.dtype == torch.bfloat16:
+        return SAR_BF16
+    raise TypeError(f"unsupported storage dtype {t.dtype}")
+
+
+def _ws(workspace: Optional[torch.Tensor]):
+    if workspace is None:
+        return c_void_p(0), c_size_t(0)
+    return _ptr(workspace), c_size_t(workspace.numel() * workspace.element_size())
+
+
+class Split:
+    """Device arrays of a long-row plan plus the C struct that points at them."""
+
+    def __init__(self, threshold: int, n_long: int, n_seg: int, long_row: torch.Tensor, long_seg: torch.Tensor):
+        self.threshold, self.n_long, self.n_seg = threshold, n_long, n_seg
+        self.long_row, self.long_seg = long_row, long_seg
+        self.c = sar_split(threshold, n_long, n_seg, long_row.data_ptr(), long_seg.data_ptr())
+
+
+class Part:
+    """One source partition (or the whole graph): owns the index tensors and the C struct."""
+
+    def __init__(self, n_dst: int, n_src: int, indptr: torch.Tensor, indices: torch.Tensor,
+                 t_indptr: Optional[torch.Tensor] = None, t_indices: Optional[torch.Tensor] = None,
+                 split: Optional[Split] = None, t_split: Optional[Split] = None, nnz: Optional[int] = None):
+        assert indptr.dtype == torch.int64 and indices.dtype == torch.int32
+        self.n_dst, self.n_src = int(n_dst), int(n_src)
+        self.nnz = int(indices.numel() if nnz is None else nnz)
+        self.indptr, self.indices, self.t_indptr, self.t_indices = indptr, indices, t_indptr, t_indices
+        self.split, self.t_split = split, t_split
+        self.c = sar_part(self.n_dst, self.n_src, self.nnz, indptr.data_ptr(), indices.data_ptr(),
+                          t_indptr.data_ptr() if t_indptr is not None else None,
+                          t_indices.data_ptr() if t_indices is not None else None,
+                          ctypes.pointer(split.c) if split is not None else None,
+                          ctypes.pointer(t_split.c) if t_split is not None else None)
+
+    def transposed(self) -> "Part":
+        """The same edges with the roles of rows and columns swapped (for the backward of the sum)."""
+        assert self.t_indptr is not None
+        return Part(self.n_src, self.n_dst, self.t_indptr, self.t_indices, self.indptr, self.indices,
+                    self.t_split, self.split, nnz=self.nnz)
+
+
+# ----------------------------------------------------------------------------------------------
+# graph preparation
+# ----------------------------------------------------------------------------------------------
+
+def sar_built_for_sm() -> int:
+    return int(lib().sar_built_for_sm())
+
+
+def sar_graph_workspace_bytes(nnz: int, n_rows: int) -> int:
+    return int(lib().sar_graph_workspace_bytes(c_int64(nnz), c_int64(n_rows)))
+
+
+def sar_csr_from_coo(n_rows: int, n_cols: int, row: torch.Tensor, col: torch.Tensor, indptr: torch.Tensor,
+                     indices: torch.Tensor, workspace: torch.Tensor) -> None:
+    assert row.dtype == torch.int32 and col.dtype == torch.int32 and row.numel() == col.numel()
+    w, wb = _ws(workspace)
+    _check("sar_csr_from_coo", lib().sar_csr_from_coo(c_int64(n_rows), c_int64(n_cols), c_int64(row.numel()),
+                                                      _ptr(row), _ptr(col), _ptr(indptr), _ptr(indices), w, wb,
+                                                      _stream()))
+
+
+def sar_csr_transpose(n_rows: int, n_cols: int, indptr: torch.Tensor, indices: torch.Tensor,
+                      t_indptr: torch.Tensor, t_indices: torch.Tensor, workspace: torch.Tensor) -> None:
+    w, wb = _ws(workspace)
+    _check("sar_csr_transpose", lib().sar_csr_transpose(c_int64(n_rows), c_int64(n_cols), _ptr(indptr),
+                                                        _ptr(indices), _ptr(t_indptr), _ptr(t_indices), w, wb,
+                                                        _stream()))
+
+
+def sar_partition_bounds(n: int, k: int) -> list:
+    arr = (c_int64 * (k + 1))()
+    _check("sar_partition_bounds", lib().sar_partition_bounds(c_int64(n), c_int32(k), arr))
+    return list(arr)
+
+
+def _host_i64(xs: Sequence[int]):
+    return (c_int64 * len(xs))(*[int(x) for x in xs])
+
+
+def sar_csr_split_indptr(n_dst: int, indptr: torch.Tensor, indices: torch.Tensor, bounds: Sequence[int],
+                         indptr_all: torch.Tensor, workspace: torch.Tensor) -> None:
+    k = len(bounds) - 1
+    w, wb = _ws(workspace)
+    _check("sar_csr_split_indptr", lib().sar_csr_split_indptr(c_int64(n_dst), _ptr(indptr), _ptr(indices),
+                                                              c_int32(k), _host_i64(bounds), _ptr(indptr_all), w, wb,
+                                                              _stream()))
+
+
+def sar_csr_split_indices(n_dst: int, indptr: torch.Tensor, indices: torch.Tensor, bounds: Sequence[int],
+                          indptr_all: torch.Tensor, nnz_off: Sequence[int], indices_all: torch.Tensor) -> None:
+    k = len(bounds) - 1
+    _check("sar_csr_split_indices", lib().sar_csr_split_indices(c_int64(n_dst), _ptr(indptr), _ptr(indices),
+                                                                c_int32(k), _host_i64(bounds), _ptr(indptr_all),
+                                                                _host_i64(nnz_off), _ptr(indices_all), _stream()))
+
+
+def sar_validate_part(part: Part, flag: torch.Tensor) -> None:
+    _check("sar_validate_part", lib().sar_validate_part(byref(part.c), _ptr(flag), _stream()))
+
+
+def sar_plan_count(n_rows: int, indptr: torch.Tensor, threshold: int, counts: torch.Tensor):
+    n_long, n_seg = c_int32(0), c_int64(0)
+    _check("sar_plan_count", lib().sar_plan_count(c_int64(n_rows), _ptr(indptr), c_int32(threshold), _ptr(counts),
+                                                  byref(n_long), byref(n_seg), _stream()))
+    return n_long.value, n_seg.value
+
+
+def sar_plan_fill(n_rows: int, indptr: torch.Tensor, threshold: int, n_long: int, long_row: torch.Tensor,
+                  long_seg: torch.Tensor, workspace: torch.Tensor) -> None:
+    w, wb = _ws(workspace)
+    _check("sar_plan_fill", lib().sar_plan_fill(c_int64(n_rows), _ptr(indptr), c_int32(threshold), c_int32(n_long),
+                                                _ptr(long_row), _ptr(long_seg), w, wb, _stream()))
+
+
+# ----------------------------------------------------------------------------------------------
+# aggregation
+# ----------------------------------------------------------------------------------------------
+
+def sar_gat_workspace_bytes(part: Part, H: int, F: int, dtype: int) -> int:
+    return int(lib().sar_gat_workspace_bytes(byref(part.c), c_int32(H), c_int32(F), ctypes.c_int(dtype)))
+
+
+def sar_spmm_workspace_bytes(part: Part, F: int, dtype: int) -> int:
+    return int(lib().sar_spmm_workspace_bytes(byref(part.c), c_int32(F), ctypes.c_int(dtype)))
+
+
+def sar_gat_fwd(part: Part, feat_q: torch.Tensor, el: torch.Tensor, er_q: torch.Tensor, H: int, F: int,
+                slope: float, flags: int, acc: Optional[torch.Tensor], m: torch.Tensor, d: torch.Tensor,
+                out: Optional[torch.Tensor], workspace: Optional[torch.Tensor]) -> None:
+    w, wb = _ws(workspace)
+    _check("sar_gat_fwd", lib().sar_gat_fwd(byref(part.c), _ptr(feat_q), _ptr(el), _ptr(er_q), c_int32(H), c_int32(F),
+                                            ctypes.c_int(_dtype(feat_q)), c_float(slope), c_uint32(flags), _ptr(acc),
+                                            _ptr(m), _ptr(d), _ptr(out), w, wb, _stream()))
+
+
+def _ptr_array(ts: Sequence[torch.Tensor]):
+    return (c_void_p * len(ts))(*[t.data_ptr() for t in ts])
+
+
+def sar_gat_fwd_fused(part: Part, bounds: Sequence[int], feat_q: Sequence[torch.Tensor], el: torch.Tensor,
+                      er_q: Sequence[torch.Tensor], H: int, F: int, slope: float, m: torch.Tensor, d: torch.Tensor,
+                      out: torch.Tensor, workspace: Optional[torch.Tensor]) -> None:
+    k = len(bounds) - 1
+    w, wb = _ws(workspace)
+    _check("sar_gat_fwd_fused", lib().sar_gat_fwd_fused(byref(part.c), c_int32(k), _host_i64(bounds),
+                                                        _ptr_array(feat_q), _ptr(el), _ptr_array(er_q), c_int32(H),
+                                                        c_int32(F), ctypes.c_int(_dtype(feat_q[0])), c_float(slope),
+                                                        _ptr(m), _ptr(d), _ptr(out), w, wb, _stream()))
+
+
+def sar_gat_bwd_prepare(n_dst: int, H: int, F: int, out_or_acc: torch.Tensor, acc_is_numerator: bool,
+                        gout: torch.Tensor, el: torch.Tensor, m: torch.Tensor, d: torch.Tensor,
+                        D: Optional[torch.Tensor], workspace: torch.Tensor) -> None:
+    w, wb = _ws(workspace)
+    _check("sar_gat_bwd_prepare", lib().sar_gat_bwd_prepare(c_int64(n_dst), c_int32(H), c_int32(F),
+                                                            ctypes.c_int(_dtype(gout)), _ptr(out_or_acc),
+                                                            c_int32(1 if acc_is_numerator else 0), _ptr(gout),
+                                                            _ptr(el), _ptr(m), _ptr(d), _ptr(D), w, wb, _stream()))
+
+
+def sar_gat_bwd(part: Part, feat_q: torch.Tensor, el: torch.Tensor, er_q: torch.Tensor, m: torch.Tensor,
+                d: torch.Tensor, gout: torch.Tensor, H: int, F: int, slope: float, flags: int,
+                dfeat_q: torch.Tensor, del_: torch.Tensor, der_q: torch.Tensor, workspace: torch.Tensor) -> None:
+    w, wb = _ws(workspace)
+    _check("sar_gat_bwd", lib().sar_gat_bwd(byref(part.c), _ptr(feat_q), _ptr(el), _ptr(er_q), _ptr(m), _ptr(d),
+                                            _ptr(gout), c_int32(H), c_int32(F), ctypes.c_int(_dtype(feat_q)),
+                                            c_float(slope), c_uint32(flags), _ptr(dfeat_q), _ptr(del_), _ptr(der_q),
+                                            w, wb, _stream()))
+
+
+def sar_gat_bwd_fused(part: Part, bounds: Sequence[int], feat_q: Sequence[torch.Tensor], el: torch.Tensor,
+                      er_q: Sequence[torch.Tensor], m: torch.Tensor, d: torch.Tensor, gout: torch.Tensor, H: int,
+                      F: int, slope: float, dfeat_q: Sequence[torch.Tensor], del_: torch.Tensor,
+                      der_q: Sequence[torch.Tensor], workspace: torch.Tensor) -> None:
+    k = len(bounds) - 1
+    w, wb = _ws(workspace)
+    _check("sar_gat_bwd_fused", lib().sar_gat_bwd_fused(byref(part.c), c_int32(k), _host_i64(bounds),
+                                                        _ptr_array(feat_q), _ptr(el), _ptr_array(er_q), _ptr(m),
+                                                        _ptr(d), _ptr(gout), c_int32(H), c_int32(F),
+                                                        ctypes.c_int(_dtype(gout)), c_float(slope),
+                                                        _ptr_array(dfeat_q), _ptr(del_), _ptr_array(der_q), w, wb,
+                                                        _stream()))
+
+
+def sar_spmm_agg(part: Part, feat_q: torch.Tensor, F: int, flags: int, deg_total: Optional[torch.Tensor],
+                 out: torch.Tensor, workspace: Optional[torch.Tensor]) -> None:
+    w, wb = _ws(workspace)
+    _check("sar_spmm_agg", lib().sar_spmm_agg(byref(part.c), _ptr(feat_q), c_int32(F), ctypes.c_int(_dtype(feat_q)),
+                                              c_uint32(flags), _ptr(deg_total), _ptr(out), w, wb, _stream()))

@@ -1,0 +1,577 @@
+// C-ABI entry points of the fused GAT aggregation and of the sum aggregation: argument checks,
+// kernel selection and launches.  Declarations and contracts are in include/sar.h.
+#include "sar_gat_kernels.cuh"
+#include "sar_generic_kernels.cuh"
+
+namespace sar {
+
+sar_status make_shape(int32_t H, int32_t F, sar_dtype t, bool ptrs_16B_aligned, Shape *out) {
+    if (H < 1 || F < 1) return SAR_ERR_INVALID_ARG;
+    if (t != SAR_F32 && t != SAR_BF16) return SAR_ERR_INVALID_ARG;
+    if ((long long)H * F > (1 << 20)) return SAR_ERR_UNSUPPORTED;
+    Shape s;
+    s.H = H;
+    s.F = F;
+    s.t = t;
+    const size_t es = sar_elem_size(t);
+    s.row_bytes = (size_t)H * F * es;
+    const size_t head_bytes = (size_t)F * es;
+    s.fast = ptrs_16B_aligned && (head_bytes % 16 == 0) && H <= SAR_MAX_HEADS && s.row_bytes <= SAR_MAX_ROW_BYTES;
+    s.G = s.V = 0;
+    s.geom = RowGeom{H, 1, 0, 1, 1};
+    if (s.fast) {
+        const int n_vec = (int)(s.row_bytes / 16);
+        const int Hp = sar_pow2_ceil(H);
+        int G = sar_pow2_ceil(n_vec);
+        if (G > 32) G = 32;
+        if (G < 4) G = 4;
+        if (G < Hp) G = Hp;
+        int V = sar_pow2_ceil((n_vec + G - 1) / G);
+        s.G = G;
+        s.V = V;
+        s.geom = RowGeom{H, Hp, sar_log2(Hp), (int)(head_bytes / 16), n_vec};
+    }
+    *out = s;
+    return SAR_OK;
+}
+
+template <typename T, int G, int V, int U>
+struct Cfg {
+    using type = T;
+    static constexpr int g = G, v = V, u = U;
+};
+
+// Calls f(Cfg<T,G,V,U>{}) for the instantiation matching the shape.
+template <typename Fn>
+static sar_status dispatch(const Shape &s, Fn &&f) {
+#define SAR_CASE(GG, VV, UU)                                                   \
+    if (s.G == GG && s.V == VV) {                                              \
+        if (s.t == SAR_F32) return f(Cfg<float, GG, VV, UU>{});                \
+        return f(Cfg<__nv_bfloat16, GG, VV, UU>{});                            \
+    }
+    SAR_CASE(4, 1, 4)
+    SAR_CASE(8, 1, 4)
+    SAR_CASE(16, 1, 4)
+    SAR_CASE(32, 1, 4)
+    SAR_CASE(32, 2, 2)
+    SAR_CASE(32, 4, 1)
+    SAR_CASE(32, 8, 1)
+#undef SAR_CASE
+    return SAR_ERR_UNSUPPORTED;
+}
+
+static inline unsigned blocks_for(long long items, int G) {
+    const long long per_block = (long long)kWarpsPerBlock * (32 / G);
+    return (unsigned)((items + per_block - 1) / per_block);
+}
+
+template <typename K>
+static sar_status ensure_smem(K kernel, size_t bytes) {
+    if (bytes > 48 * 1024)
+        SAR_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
+    return SAR_OK;
+}
+
+// ---- workspace layout ---------------------------------------------------------------------------
+// [ destination records: n_dst*H float4 ][ long-row partials of the CSR ][ long-row partials of the CSC ]
+static size_t rec_bytes(long long n_dst, int H) { return sar_round_up((size_t)n_dst * H * 16, 256); }
+static long long part_stride(int H, int F) {  // floats per segment, a multiple of 4 (float4 rows)
+    return (2LL * H * F + 2LL * H + 3) & ~3LL;
+}
+static size_t part_bytes(const sar_split *sp, int H, int F) {
+    return sp ? sar_round_up((size_t)sp->n_seg * part_stride(H, F) * 4, 256) : 0;
+}
+
+static SplitArgs split_args(const sar_split *sp, float *part, int H, int F, bool fast) {
+    SplitArgs a;
+    a.threshold = 0;
+    a.n_long = 0;
+    a.n_seg = 0;
+    a.long_row = nullptr;
+    a.long_seg = nullptr;
+    a.part = part;
+    a.pstride = part_stride(H, F);
+    if (sp && fast && sp->n_long > 0 && sp->threshold > 0) {
+        a.threshold = sp->threshold;
+        a.n_long = sp->n_long;
+        a.n_seg = sp->n_seg;
+        a.long_row = sp->long_row;
+        a.long_seg = sp->long_seg;
+    }
+    return a;
+}
+
+static sar_status check_split(const sar_split *sp) {
+    if (!sp) return SAR_OK;
+    if (sp->threshold < 1 || sp->n_long < 0 || sp->n_seg < 0) return SAR_ERR_INVALID_ARG;
+    if (sp->n_long > 0 && (!sp->long_row || !sp->long_seg)) return SAR_ERR_INVALID_ARG;
+    return SAR_OK;
+}
+
+static sar_status check_part(const sar_part *g, bool need_csc) {
+    if (!g) return SAR_ERR_INVALID_ARG;
+    if (g->n_dst < 0 || g->n_src < 0 || g->nnz < 0) return SAR_ERR_INVALID_ARG;
+    if (g->n_src > INT32_MAX) return SAR_ERR_UNSUPPORTED;
+    if (!g->indptr || (g->nnz > 0 && !g->indices)) return SAR_ERR_INVALID_ARG;
+    if (!sar_aligned(g->indptr, 8) || !sar_aligned(g->indices, 4)) return SAR_ERR_ALIGNMENT;
+    if (need_csc) {
+        if (!g->t_indptr || (g->nnz > 0 && !g->t_indices)) return SAR_ERR_INVALID_ARG;
+        if (!sar_aligned(g->t_indptr, 8) || !sar_aligned(g->t_indices, 4)) return SAR_ERR_ALIGNMENT;
+    }
+    SAR_TRY(check_split(g->split));
+    SAR_TRY(check_split(g->t_split));
+    return SAR_OK;
+}
+
+static bool all16(std::initializer_list<const void *> ps) {
+    for (const void *p : ps)
+        if (p && !sar_aligned(p, 16)) return false;
+    return true;
+}
+
+static sar_status check_elem_align(std::initializer_list<const void *> ps, size_t a) {
+    for (const void *p : ps)
+        if (p && !sar_aligned(p, a)) return SAR_ERR_ALIGNMENT;
+    return SAR_OK;
+}
+
+}  // namespace sar
+
+using namespace sar;
+
+extern "C" {
+
+const char *sar_status_string(sar_status s) {
+    switch (s) {
+        case SAR_OK: return "ok";
+        case SAR_ERR_INVALID_ARG: return "invalid argument";
+        case SAR_ERR_UNSUPPORTED: return "unsupported shape";
+        case SAR_ERR_ALIGNMENT: return "misaligned pointer";
+        case SAR_ERR_WORKSPACE: return "workspace missing or too small";
+        case SAR_ERR_CUDA: return "CUDA error";
+        case SAR_ERR_BAD_GRAPH: return "inconsistent graph";
+    }
+    return "unknown status";
+}
+
+int32_t sar_built_for_sm(void) {
+#ifdef SAR_BUILT_FOR_SM
+    return SAR_BUILT_FOR_SM;
+#else
+    return 0;
+#endif
+}
+
+size_t sar_gat_workspace_bytes(const sar_part *g, int32_t H, int32_t F, sar_dtype t) {
+    (void)t;
+    if (!g || H < 1 || F < 1) return 0;
+    return rec_bytes(g->n_dst, H) + part_bytes(g->split, H, F) + part_bytes(g->t_split, H, F) + 256;
+}
+
+size_t sar_spmm_workspace_bytes(const sar_part *g, int32_t F, sar_dtype t) {
+    (void)t;
+    if (!g || F < 1) return 0;
+    return part_bytes(g->split, 1, F) + 256;
+}
+
+// ---------------------------------------------------------------------------------------------
+sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, const float *er_q, int32_t H,
+                       int32_t F, sar_dtype t, float slope, uint32_t flags, float *acc, float *m, float *d,
+                       void *out, void *workspace, size_t workspace_bytes, void *stream) {
+    SAR_TRY(check_part(g, false));
+    if (flags & ~(SAR_FIRST | SAR_LAST)) return SAR_ERR_INVALID_ARG;
+    const bool first = flags & SAR_FIRST, last = flags & SAR_LAST;
+    if (!el || !m || !d) return SAR_ERR_INVALID_ARG;
+    if (g->n_src > 0 && (!feat_q || !er_q)) return SAR_ERR_INVALID_ARG;
+    if (last && !out) return SAR_ERR_INVALID_ARG;
+    if (!(first && last) && !acc) return SAR_ERR_INVALID_ARG;
+    SAR_TRY(check_elem_align({el, er_q, m, d, acc}, 4));
+    SAR_TRY(check_elem_align({feat_q, out}, sar_elem_size(t)));
+    Shape s;
+    SAR_TRY(make_shape(H, F, t, all16({feat_q, out, acc}), &s));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (g->n_dst == 0) return SAR_OK;
+
+    if (!s.fast) {
+        GenericArgs a{};
+        a.n_dst = g->n_dst;
+        a.indptr = g->indptr;
+        a.indices = g->indices;
+        a.feat = feat_q;
+        a.el = el;
+        a.er = er_q;
+        a.acc = acc;
+        a.m = m;
+        a.d = d;
+        a.out = out;
+        a.H = H;
+        a.F = F;
+        a.slope = slope;
+        a.flags = flags;
+        const long long n = g->n_dst * H;
+        const unsigned blocks = (unsigned)((n + 255) / 256);
+        if (t == SAR_F32)
+            gat_fwd_generic<float><<<blocks, 256, 0, st>>>(a);
+        else
+            gat_fwd_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a);
+        return sar_after_launch();
+    }
+
+    const bool use_split = g->split && g->split->n_long > 0;
+    float *part = nullptr;
+    if (use_split) {
+        const size_t need = rec_bytes(g->n_dst, H) + part_bytes(g->split, H, F);
+        if (!workspace || workspace_bytes < need || !sar_aligned(workspace, 16)) return SAR_ERR_WORKSPACE;
+        part = reinterpret_cast<float *>(static_cast<char *>(workspace) + rec_bytes(g->n_dst, H));
+    }
+    FwdArgs a;
+    a.n_dst = g->n_dst;
+    a.indptr = g->indptr;
+    a.indices = g->indices;
+    a.feat = feat_q;
+    a.el = el;
+    a.er = er_q;
+    a.acc = acc;
+    a.m = m;
+    a.d = d;
+    a.out = out;
+    a.slope = slope;
+    a.flags = flags;
+    a.g = s.geom;
+    a.sp = split_args(g->split, part, H, F, true);
+    a.mode = 0;
+    return dispatch(s, [&](auto cfg) -> sar_status {
+        using C = decltype(cfg);
+        using T = typename C::type;
+        const size_t smem = (size_t)kWarpsPerBlock * warp_smem_floats(s.geom.Hp, C::v, 1) * 4;
+        auto kern = gat_fwd_kernel<T, C::g, C::v, C::u>;
+        SAR_TRY(ensure_smem(kern, smem));
+        FwdArgs b = a;
+        kern<<<blocks_for(g->n_dst, C::g), kThreads, smem, st>>>(b);
+        SAR_TRY(sar_after_launch());
+        if (b.sp.threshold > 0) {
+            b.mode = 1;
+            kern<<<blocks_for(b.sp.n_seg, C::g), kThreads, smem, st>>>(b);
+            SAR_TRY(sar_after_launch());
+            b.mode = 0;
+            gat_fwd_merge_kernel<T, C::g, C::v><<<blocks_for(b.sp.n_long, C::g), kThreads, 0, st>>>(b);
+            SAR_TRY(sar_after_launch());
+        }
+        return SAR_OK;
+    });
+}
+
+// Are the k per-partition buffers one contiguous array cut at `bounds`?
+static bool contiguous(const void *const *ptrs, int32_t k, const int64_t *bounds, size_t row_bytes) {
+    for (int32_t q = 0; q < k; ++q)
+        if (static_cast<const char *>(ptrs[q]) != static_cast<const char *>(ptrs[0]) + (size_t)bounds[q] * row_bytes)
+            return false;
+    return true;
+}
+
+static sar_status check_fused(const sar_part *g, int32_t k, const int64_t *bounds) {
+    if (!g || !bounds || k < 1) return SAR_ERR_INVALID_ARG;
+    if (k > SAR_MAX_PARTS) return SAR_ERR_UNSUPPORTED;
+    if (bounds[0] != 0 || bounds[k] != g->n_src) return SAR_ERR_INVALID_ARG;
+    for (int32_t q = 0; q < k; ++q)
+        if (bounds[q + 1] < bounds[q]) return SAR_ERR_INVALID_ARG;
+    return SAR_OK;
+}
+
+sar_status sar_gat_fwd_fused(const sar_part *g, int32_t k, const int64_t *bounds, const void *const *feat_q,
+                             const float *el, const float *const *er_q, int32_t H, int32_t F, sar_dtype t,
+                             float slope, float *m, float *d, void *out, void *workspace,
+                             size_t workspace_bytes, void *stream) {
+    SAR_TRY(check_fused(g, k, bounds));
+    if (!feat_q || !er_q || H < 1 || F < 1) return SAR_ERR_INVALID_ARG;
+    for (int32_t q = 0; q < k; ++q)
+        if (!feat_q[q] || !er_q[q]) return SAR_ERR_INVALID_ARG;
+    // Sources ascend within a row, so walking a row once IS the partition-after-partition visit.
+    // Buffers that form one array need no per-edge partition lookup.
+    if (!contiguous(feat_q, k, bounds, (size_t)H * F * sar_elem_size(t)) ||
+        !contiguous(reinterpret_cast<const void *const *>(er_q), k, bounds, (size_t)H * 4))
+        return SAR_ERR_UNSUPPORTED;
+    return sar_gat_fwd(g, feat_q[0], el, er_q[0], H, F, t, slope, SAR_FIRST | SAR_LAST, nullptr, m, d, out,
+                       workspace, workspace_bytes, stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+sar_status sar_gat_bwd_prepare(int64_t n_dst, int32_t H, int32_t F, sar_dtype t, const void *out_or_acc,
+                               int32_t acc_is_numerator, const void *gout, const float *el, const float *m,
+                               const float *d, float *D, void *workspace, size_t workspace_bytes, void *stream) {
+    if (n_dst < 0 || !out_or_acc || !gout || !el || !m || !d) return SAR_ERR_INVALID_ARG;
+    if (!workspace || !sar_aligned(workspace, 16) || workspace_bytes < (size_t)n_dst * H * 16) return SAR_ERR_WORKSPACE;
+    SAR_TRY(check_elem_align({el, m, d, D}, 4));
+    SAR_TRY(check_elem_align({gout}, sar_elem_size(t)));
+    SAR_TRY(check_elem_align({out_or_acc}, acc_is_numerator ? 4 : sar_elem_size(t)));
+    Shape s;
+    SAR_TRY(make_shape(H, F, t, all16({out_or_acc, gout}), &s));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (n_dst == 0) return SAR_OK;
+    if (!s.fast) {
+        GenericArgs a{};
+        a.n_dst = n_dst;
+        a.out_in = out_or_acc;
+        a.gout = gout;
+        a.el = el;
+        a.m_in = m;
+        a.d_in = d;
+        a.D = D;
+        a.rec = static_cast<float4 *>(workspace);
+        a.H = H;
+        a.F = F;
+        a.acc_is_numerator = acc_is_numerator;
+        const unsigned blocks = (unsigned)((n_dst * H + 255) / 256);
+        if (t == SAR_F32)
+            gat_bwd_prepare_generic<float><<<blocks, 256, 0, st>>>(a);
+        else
+            gat_bwd_prepare_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a);
+        return sar_after_launch();
+    }
+    PrepArgs a;
+    a.n_dst = n_dst;
+    a.out = out_or_acc;
+    a.gout = gout;
+    a.el = el;
+    a.m = m;
+    a.d = d;
+    a.D = D;
+    a.rec = static_cast<float4 *>(workspace);
+    a.acc_is_numerator = acc_is_numerator;
+    a.g = s.geom;
+    return dispatch(s, [&](auto cfg) -> sar_status {
+        using C = decltype(cfg);
+        using T = typename C::type;
+        const size_t smem = (size_t)kWarpsPerBlock * 32 * C::v * 4;
+        gat_bwd_prepare_kernel<T, C::g, C::v><<<blocks_for(n_dst, C::g), kThreads, smem, st>>>(a);
+        return sar_after_launch();
+    });
+}
+
+sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, const float *er_q, const float *m,
+                       const float *d, const void *gout, int32_t H, int32_t F, sar_dtype t, float slope,
+                       uint32_t flags, void *dfeat_q, float *del, float *der_q, void *workspace,
+                       size_t workspace_bytes, void *stream) {
+    SAR_TRY(check_part(g, true));
+    if (flags & ~(SAR_FIRST | SAR_LAST)) return SAR_ERR_INVALID_ARG;
+    if (!el || !m || !d || !gout || !del) return SAR_ERR_INVALID_ARG;
+    if (g->n_src > 0 && (!feat_q || !er_q || !dfeat_q || !der_q)) return SAR_ERR_INVALID_ARG;
+    SAR_TRY(check_elem_align({el, er_q, m, d, del, der_q}, 4));
+    SAR_TRY(check_elem_align({feat_q, gout, dfeat_q}, sar_elem_size(t)));
+    Shape s;
+    SAR_TRY(make_shape(H, F, t, all16({feat_q, gout, dfeat_q}), &s));
+    const size_t need = rec_bytes(g->n_dst, H) + (s.fast ? part_bytes(g->split, H, F) + part_bytes(g->t_split, H, F) : 0);
+    if (!workspace || !sar_aligned(workspace, 16) || workspace_bytes < need) return SAR_ERR_WORKSPACE;
+    const bool whole = (flags & SAR_FIRST) && (flags & SAR_LAST);  // D rebuilt from the edges
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    float4 *rec = static_cast<float4 *>(workspace);
+    char *wsb = static_cast<char *>(workspace);
+    float *part_csr = reinterpret_cast<float *>(wsb + rec_bytes(g->n_dst, H));
+    float *part_csc = reinterpret_cast<float *>(wsb + rec_bytes(g->n_dst, H) + part_bytes(g->split, H, F));
+
+    if (!s.fast) {
+        GenericArgs a{};
+        a.n_dst = g->n_dst;
+        a.n_src = g->n_src;
+        a.indptr = g->indptr;
+        a.indices = g->indices;
+        a.t_indptr = g->t_indptr;
+        a.t_indices = g->t_indices;
+        a.feat = feat_q;
+        a.gout = gout;
+        a.el = el;
+        a.er = er_q;
+        a.m_in = m;
+        a.d_in = d;
+        a.dfeat = dfeat_q;
+        a.del = del;
+        a.der = der_q;
+        a.rec = rec;
+        a.H = H;
+        a.F = F;
+        a.slope = slope;
+        a.flags = flags;
+        a.given_d = whole ? 0 : 1;
+        if (g->n_dst > 0) {
+            const unsigned blocks = (unsigned)((g->n_dst * H + 255) / 256);
+            if (t == SAR_F32)
+                gat_bwd_dst_generic<float><<<blocks, 256, 0, st>>>(a);
+            else
+                gat_bwd_dst_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a);
+            SAR_TRY(sar_after_launch());
+        }
+        if (g->n_src > 0) {
+            const unsigned blocks = (unsigned)((g->n_src * H + 255) / 256);
+            if (t == SAR_F32)
+                gat_bwd_src_generic<float><<<blocks, 256, 0, st>>>(a);
+            else
+                gat_bwd_src_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a);
+            SAR_TRY(sar_after_launch());
+        }
+        return SAR_OK;
+    }
+
+    BwdDstArgs da;
+    da.n_dst = g->n_dst;
+    da.indptr = g->indptr;
+    da.indices = g->indices;
+    da.feat = feat_q;
+    da.gout = gout;
+    da.el = el;
+    da.er = er_q;
+    da.m = m;
+    da.d = d;
+    da.rec = rec;
+    da.del = del;
+    da.slope = slope;
+    da.flags = flags;
+    da.g = s.geom;
+    da.sp = split_args(g->split, part_csr, H, F, true);
+    da.mode = 0;
+    BwdSrcArgs sa;
+    sa.n_src = g->n_src;
+    sa.t_indptr = g->t_indptr;
+    sa.t_indices = g->t_indices;
+    sa.gout = gout;
+    sa.feat = feat_q;
+    sa.er = er_q;
+    sa.rec = rec;
+    sa.dfeat = dfeat_q;
+    sa.der = der_q;
+    sa.slope = slope;
+    sa.g = s.geom;
+    sa.sp = split_args(g->t_split, part_csc, H, F, true);
+    sa.mode = 0;
+
+    return dispatch(s, [&](auto cfg) -> sar_status {
+        using C = decltype(cfg);
+        using T = typename C::type;
+        if (g->n_dst > 0) {
+            const size_t smem = (size_t)kWarpsPerBlock * warp_smem_floats(s.geom.Hp, C::v, 2) * 4;
+            auto run = [&](auto kern, auto merge) -> sar_status {
+                SAR_TRY(ensure_smem(kern, smem));
+                SAR_TRY(ensure_smem(merge, smem));
+                BwdDstArgs b = da;
+                kern<<<blocks_for(g->n_dst, C::g), kThreads, smem, st>>>(b);
+                SAR_TRY(sar_after_launch());
+                if (b.sp.threshold > 0) {
+                    b.mode = 1;
+                    kern<<<blocks_for(b.sp.n_seg, C::g), kThreads, smem, st>>>(b);
+                    SAR_TRY(sar_after_launch());
+                    b.mode = 0;
+                    merge<<<blocks_for(b.sp.n_long, C::g), kThreads, smem, st>>>(b);
+                    SAR_TRY(sar_after_launch());
+                }
+                return SAR_OK;
+            };
+            if (whole)
+                SAR_TRY(run(gat_bwd_dst_kernel<T, C::g, C::v, C::u, false>, gat_bwd_dst_merge_kernel<T, C::g, C::v, false>));
+            else
+                SAR_TRY(run(gat_bwd_dst_kernel<T, C::g, C::v, C::u, true>, gat_bwd_dst_merge_kernel<T, C::g, C::v, true>));
+        }
+        if (g->n_src > 0) {
+            const size_t smem = (size_t)kWarpsPerBlock * warp_smem_floats(s.geom.Hp, C::v, 4) * 4;
+            auto kern = gat_bwd_src_kernel<T, C::g, C::v, C::u>;
+            auto merge = gat_bwd_src_merge_kernel<T, C::g, C::v>;
+            SAR_TRY(ensure_smem(kern, smem));
+            SAR_TRY(ensure_smem(merge, smem));
+            BwdSrcArgs b = sa;
+            kern<<<blocks_for(g->n_src, C::g), kThreads, smem, st>>>(b);
+            SAR_TRY(sar_after_launch());
+            if (b.sp.threshold > 0) {
+                b.mode = 1;
+                kern<<<blocks_for(b.sp.n_seg, C::g), kThreads, smem, st>>>(b);
+                SAR_TRY(sar_after_launch());
+                b.mode = 0;
+                merge<<<blocks_for(b.sp.n_long, C::g), kThreads, smem, st>>>(b);
+                SAR_TRY(sar_after_launch());
+            }
+        }
+        return SAR_OK;
+    });
+}
+
+sar_status sar_gat_bwd_fused(const sar_part *g, int32_t k, const int64_t *bounds, const void *const *feat_q,
+                             const float *el, const float *const *er_q, const float *m, const float *d,
+                             const void *gout, int32_t H, int32_t F, sar_dtype t, float slope,
+                             void *const *dfeat_q, float *del, float *const *der_q, void *workspace,
+                             size_t workspace_bytes, void *stream) {
+    SAR_TRY(check_fused(g, k, bounds));
+    if (!feat_q || !er_q || !dfeat_q || !der_q || H < 1 || F < 1) return SAR_ERR_INVALID_ARG;
+    for (int32_t q = 0; q < k; ++q)
+        if (!feat_q[q] || !er_q[q] || !dfeat_q[q] || !der_q[q]) return SAR_ERR_INVALID_ARG;
+    const size_t rb = (size_t)H * F * sar_elem_size(t);
+    if (!contiguous(feat_q, k, bounds, rb) || !contiguous(reinterpret_cast<const void *const *>(dfeat_q), k, bounds, rb) ||
+        !contiguous(reinterpret_cast<const void *const *>(er_q), k, bounds, (size_t)H * 4) ||
+        !contiguous(reinterpret_cast<const void *const *>(der_q), k, bounds, (size_t)H * 4))
+        return SAR_ERR_UNSUPPORTED;
+    return sar_gat_bwd(g, feat_q[0], el, er_q[0], m, d, gout, H, F, t, slope, SAR_FIRST | SAR_LAST, dfeat_q[0], del,
+                       der_q[0], workspace, workspace_bytes, stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+sar_status sar_spmm_agg(const sar_part *g, const void *feat_q, int32_t F, sar_dtype t, uint32_t flags,
+                        const int64_t *deg_total, void *out, void *workspace, size_t workspace_bytes,
+                        void *stream) {
+    SAR_TRY(check_part(g, false));
+    if (flags & ~(SAR_FIRST | SAR_LAST | SAR_MEAN)) return SAR_ERR_INVALID_ARG;
+    if (!out || (g->n_src > 0 && !feat_q)) return SAR_ERR_INVALID_ARG;
+    if ((flags & SAR_MEAN) && (flags & SAR_LAST) && !deg_total) return SAR_ERR_INVALID_ARG;
+    SAR_TRY(check_elem_align({feat_q, out}, sar_elem_size(t)));
+    SAR_TRY(check_elem_align({deg_total}, 8));
+    Shape s;
+    SAR_TRY(make_shape(1, F, t, all16({feat_q, out}), &s));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (g->n_dst == 0) return SAR_OK;
+    if (!s.fast) {
+        GenericArgs a{};
+        a.n_dst = g->n_dst;
+        a.indptr = g->indptr;
+        a.indices = g->indices;
+        a.feat = feat_q;
+        a.out = out;
+        a.deg_total = deg_total;
+        a.H = 1;
+        a.F = F;
+        a.flags = flags;
+        const unsigned blocks = (unsigned)((g->n_dst * F + 255) / 256);
+        if (t == SAR_F32)
+            spmm_generic<float><<<blocks, 256, 0, st>>>(a);
+        else
+            spmm_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a);
+        return sar_after_launch();
+    }
+    const bool use_split = g->split && g->split->n_long > 0;
+    if (use_split && (!workspace || !sar_aligned(workspace, 16) || workspace_bytes < part_bytes(g->split, 1, F)))
+        return SAR_ERR_WORKSPACE;
+    SumArgs a;
+    a.n_dst = g->n_dst;
+    a.indptr = g->indptr;
+    a.indices = g->indices;
+    a.feat = feat_q;
+    a.out = out;
+    a.deg_total = deg_total;
+    a.flags = flags;
+    a.g = s.geom;
+    a.sp = split_args(g->split, static_cast<float *>(workspace), 1, F, true);
+    a.mode = 0;
+    return dispatch(s, [&](auto cfg) -> sar_status {
+        using C = decltype(cfg);
+        using T = typename C::type;
+        const size_t smem = (size_t)kWarpsPerBlock * 32 * 4;
+        SumArgs b = a;
+        spmm_kernel<T, C::g, C::v, C::u><<<blocks_for(g->n_dst, C::g), kThreads, smem, st>>>(b);
+        SAR_TRY(sar_after_launch());
+        if (b.sp.threshold > 0) {
+            b.mode = 1;
+            spmm_kernel<T, C::g, C::v, C::u><<<blocks_for(b.sp.n_seg, C::g), kThreads, smem, st>>>(b);
+            SAR_TRY(sar_after_launch());
+            b.mode = 0;
+            spmm_merge_kernel<T, C::g, C::v><<<blocks_for(b.sp.n_long, C::g), kThreads, 0, st>>>(b);
+            SAR_TRY(sar_after_launch());
+        }
+        return SAR_OK;
+    });
+}
+
+}  // extern "C"

@@ -1,0 +1,686 @@
+// Fused GAT aggregation kernels (forward, destination-major backward, source-major backward,
+// row-dot preparation) built on the row-stationary skeleton of sar_rowkernels.cuh (internal).
+#pragma once
+
+#include "sar_rowkernels.cuh"
+
+namespace sar {
+
+// ------------------------------------------------------------------------------------------------
+// Forward: scores, online softmax and weighted neighbour sum in one pass (Eq. 3, Sec. 3.3), with
+// the running-max correction of Sec. 3.4 applied batch by batch (and partition by partition when
+// the state comes from / goes to global memory, Algorithm 1).
+// ------------------------------------------------------------------------------------------------
+struct FwdArgs {
+    long long n_dst;
+    const int64_t *indptr;
+    const int32_t *indices;
+    const void *feat;   // [n_src, n_vec] 16-byte vectors
+    const float *el;    // [n_dst,H]
+    const float *er;    // [n_src,H]
+    float *acc;         // [n_dst,H*F] running numerator (float32) or null
+    float *m;           // [n_dst,H]
+    float *d;           // [n_dst,H]
+    void *out;          // [n_dst, n_vec] or null
+    float slope;
+    unsigned flags;
+    RowGeom g;
+    SplitArgs sp;
+    int mode;           // 0: one group per row; 1: one group per long-row segment
+};
+
+// Partial record of a forward segment in the workspace: [rowf floats numerator][H max][H norm].
+template <typename T, int G, int V, int U>
+__global__ void __launch_bounds__(kThreads) gat_fwd_kernel(const FwdArgs a) {
+    constexpr int EPV = Elem<T>::EPV;
+    constexpr int RPW = 32 / G;
+    extern __shared__ __align__(16) float smem[];
+    const LaneId<G> id;
+    const int H = a.g.H, Hp = a.g.Hp;
+    float *wbase = smem + (size_t)id.warp * warp_smem_floats(Hp, V, 1);
+    int *sj = reinterpret_cast<int *>(wbase) + id.gid * G;
+    float *sc = wbase + 32 + id.gid * Hp;
+    float *sw = wbase + 64 + (size_t)id.gid * G * Hp;
+
+    const long long item = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
+    WorkItem w = locate_work(item, a.n_dst, a.indptr, a.sp, a.mode);
+    const bool first = (a.flags & SAR_FIRST) || a.mode == 1;
+    const bool last = (a.flags & SAR_LAST) && a.mode == 0;
+    if (a.mode == 0 && w.active && !(a.flags & SAR_FIRST) && !(a.flags & SAR_LAST) && w.beg == w.end)
+        w.active = false;  // nothing to fold in, state stays as it is
+
+    const VecGeom<G, V> vg(a.g, id.gl);
+    const int sh = id.gl & (Hp - 1);        // head this lane scores
+    const int se0 = id.gl >> a.g.lgHp;      // first edge of the batch this lane scores
+    const int epi = G >> a.g.lgHp;          // edges scored per sweep of the group
+    const bool sh_ok = sh < H;
+
+    float el_i = 0.f, Mrun = SAR_NEG_INF;
+    float dv[V];
+    float acc[V][EPV];
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        dv[v] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) acc[v][e] = 0.f;
+    }
+    if (w.active) {
+        if (sh_ok) el_i = __ldg(a.el + w.row * H + sh);
+        if (!first) {
+            if (sh_ok) Mrun = a.m[w.row * H + sh];
+#pragma unroll
+            for (int v = 0; v < V; ++v)
+                if (vg.vok[v]) dv[v] = a.d[w.row * H + vg.hv[v]];
+            load_acc_row<G, V, EPV>(a.acc + w.row * (long long)(a.g.n_vec * EPV), id.gl, vg.vok, acc);
+        }
+    }
+
+    const int nbatch = (int)((w.end - w.beg + G - 1) / G);
+    const int wmax = __reduce_max_sync(0xffffffffu, nbatch);
+    const uint4 *featv = reinterpret_cast<const uint4 *>(a.feat);
+    for (int it = 0; it < wmax; ++it) {
+        const long long b0 = w.beg + (long long)it * G;
+        const long long rem = w.end - b0;
+        const int nb = rem <= 0 ? 0 : (rem < G ? (int)rem : G);
+        sj[id.gl] = id.gl < nb ? ld_stream_i32(a.indices + b0 + id.gl) : 0;
+        __syncwarp();
+        // SCORE, sweep 1: e = LeakyReLU(el_i + er_j) per (edge, head); batch max per head
+        float lm = SAR_NEG_INF;
+        if (sh_ok)
+            for (int k = se0; k < nb; k += epi) {
+                float gr;
+                const float e = leaky(el_i + __ldg(a.er + (long long)sj[k] * H + sh), a.slope, gr);
+                sw[k * Hp + sh] = e;
+                lm = fmaxf(lm, e);
+            }
+        for (int off = Hp; off < G; off <<= 1) lm = fmaxf(lm, __shfl_xor_sync(0xffffffffu, lm, off));
+        const float Mn = fmaxf(Mrun, lm);
+        const float c = (Mn == SAR_NEG_INF) ? 1.f : fast_exp(Mrun - Mn);  // exp(old_max - new_max)
+        Mrun = Mn;
+        if (id.gl < Hp) sc[id.gl] = c;
+        // SCORE, sweep 2: un-normalised weights exp(e - running max)
+        if (sh_ok)
+            for (int k = se0; k < nb; k += epi) sw[k * Hp + sh] = fast_exp(sw[k * Hp + sh] - Mn);
+        __syncwarp();
+        // correct what has been accumulated so far, then GATHER
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const float cv = sc[vg.hv[v]];
+            dv[v] *= cv;
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) acc[v][e] *= cv;
+        }
+        gather_batch<T, G, V, U, kFwd>(featv, a.g.n_vec, sj, sw, Hp, nb, id.gl, vg.hv, vg.vok, acc, acc, dv);
+        __syncwarp();
+    }
+
+    if (!w.active) return;
+    const long long rowf = (long long)a.g.n_vec * EPV;
+    if (a.mode == 1) {
+        float *rec = a.sp.part + w.seg * a.sp.pstride;
+        store_acc_row<G, V, EPV>(rec, id.gl, vg.vok, acc);
+        if (id.gl < H) rec[rowf + id.gl] = Mrun;
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+            if (vg.vok[v] && ((v * G + id.gl) % a.g.vph) == 0) rec[rowf + H + vg.hv[v]] = dv[v];
+        return;
+    }
+    if (last) {
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const float inv = dv[v] > 0.f ? 1.f / dv[v] : 0.f;
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) acc[v][e] *= inv;
+        }
+        store_row_vec<T, G, V>(a.out, w.row, a.g.n_vec, id.gl, vg.vok, acc);
+    } else {
+        store_acc_row<G, V, EPV>(a.acc + w.row * rowf, id.gl, vg.vok, acc);
+    }
+    if (id.gl < H) a.m[w.row * H + id.gl] = Mrun;
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+        if (vg.vok[v] && ((v * G + id.gl) % a.g.vph) == 0) a.d[w.row * H + vg.hv[v]] = dv[v];
+}
+
+// Merge of the forward partials of the long rows: one group per long row folds its segments in
+// order with the same running-max rule, starting from the incoming state unless SAR_FIRST.
+template <typename T, int G, int V>
+__global__ void __launch_bounds__(kThreads) gat_fwd_merge_kernel(const FwdArgs a) {
+    constexpr int EPV = Elem<T>::EPV;
+    constexpr int RPW = 32 / G;
+    const LaneId<G> id;
+    const int H = a.g.H;
+    const long long lr = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
+    if (lr >= a.sp.n_long) return;
+    const long long row = a.sp.long_row[lr];
+    const long long s0 = a.sp.long_seg[lr], s1 = a.sp.long_seg[lr + 1];
+    const VecGeom<G, V> vg(a.g, id.gl);
+    const long long rowf = (long long)a.g.n_vec * EPV;
+    const bool first = a.flags & SAR_FIRST, last = a.flags & SAR_LAST;
+
+    float Mv[V], dv[V], acc[V][EPV];
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        Mv[v] = SAR_NEG_INF;
+        dv[v] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) acc[v][e] = 0.f;
+    }
+    if (!first) {
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+            if (vg.vok[v]) {
+                Mv[v] = a.m[row * H + vg.hv[v]];
+                dv[v] = a.d[row * H + vg.hv[v]];
+            }
+        load_acc_row<G, V, EPV>(a.acc + row * rowf, id.gl, vg.vok, acc);
+    }
+    for (long long s = s0; s < s1; ++s) {
+        const float *rec = a.sp.part + s * a.sp.pstride;
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+            if (vg.vok[v]) {
+                const float Ms = rec[rowf + vg.hv[v]], ds = rec[rowf + H + vg.hv[v]];
+                const float Mn = fmaxf(Mv[v], Ms);
+                const float c_old = (Mn == SAR_NEG_INF) ? 1.f : fast_exp(Mv[v] - Mn);
+                const float c_new = (Mn == SAR_NEG_INF) ? 1.f : fast_exp(Ms - Mn);
+                const float4 *p = reinterpret_cast<const float4 *>(rec + (size_t)(v * G + id.gl) * EPV);
+#pragma unroll
+                for (int q = 0; q < EPV / 4; ++q) {
+                    const float4 x = p[q];
+                    acc[v][4 * q] = acc[v][4 * q] * c_old + x.x * c_new;
+                    acc[v][4 * q + 1] = acc[v][4 * q + 1] * c_old + x.y * c_new;
+                    acc[v][4 * q + 2] = acc[v][4 * q + 2] * c_old + x.z * c_new;
+                    acc[v][4 * q + 3] = acc[v][4 * q + 3] * c_old + x.w * c_new;
+                }
+                dv[v] = dv[v] * c_old + ds * c_new;
+                Mv[v] = Mn;
+            }
+    }
+    if (last) {
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const float inv = dv[v] > 0.f ? 1.f / dv[v] : 0.f;
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) acc[v][e] *= inv;
+        }
+        store_row_vec<T, G, V>(a.out, row, a.g.n_vec, id.gl, vg.vok, acc);
+    } else {
+        store_acc_row<G, V, EPV>(a.acc + row * rowf, id.gl, vg.vok, acc);
+    }
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+        if (vg.vok[v] && ((v * G + id.gl) % a.g.vph) == 0) {
+            a.m[row * H + vg.hv[v]] = Mv[v];
+            a.d[row * H + vg.hv[v]] = dv[v];
+        }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Backward, destination-major pass over the CSR (Algorithm 2's per-edge loop, rematerialised):
+// with alpha = exp(e - m)/d and g' = LeakyReLU'(s),
+//     A = sum_j alpha * feat_j            (= out, rebuilt so that bf16 rounding of `out` never enters)
+//     B = sum_j alpha * g' * feat_j,      S = sum_j alpha * g'
+//     D = <gout_i, A>,   del_i = <gout_i, B> - D * S     (= sum_j alpha (dalpha - D) g')
+// and the packed record {el, m, 1/d, D} per (i,h) for the source-major pass.
+// With GIVEN_D the record already exists (sar_gat_bwd_prepare) and only B, S are accumulated over
+// this partition's edges.
+// ------------------------------------------------------------------------------------------------
+struct BwdDstArgs {
+    long long n_dst;
+    const int64_t *indptr;
+    const int32_t *indices;
+    const void *feat;   // gathered rows
+    const void *gout;   // row-stationary vector
+    const float *el, *er, *m, *d;
+    float4 *rec;        // [n_dst,H] {el, m, 1/d, D}: written (full) or read (GIVEN_D)
+    float *del;         // [n_dst,H]
+    float slope;
+    unsigned flags;
+    RowGeom g;
+    SplitArgs sp;
+    int mode;
+};
+
+template <typename T, int G, int V, bool GIVEN_D>
+__device__ __forceinline__ void bwd_dst_epilogue(const BwdDstArgs &a, const LaneId<G> &id, const VecGeom<G, V> &vg,
+                                                 float *scratch, long long row, const float (&gv)[V][Elem<T>::EPV],
+                                                 const float (&accA)[V][Elem<T>::EPV],
+                                                 const float (&accB)[V][Elem<T>::EPV], const float (&S)[V]) {
+    constexpr int EPV = Elem<T>::EPV;
+    const int H = a.g.H;
+    float pA[V], pB[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        pA[v] = pB[v] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) {
+            pA[v] = fmaf(gv[v][e], accA[v][e], pA[v]);
+            pB[v] = fmaf(gv[v][e], accB[v][e], pB[v]);
+        }
+    }
+    const float DB = head_sum<G, V>(scratch, pB, vg.vok, id.gl, a.g);
+    const float Sh = head_scalar<G, V>(scratch, S, vg.hv, vg.vok, id.gl, a.g);
+    float D;
+    if constexpr (GIVEN_D) {
+        D = (id.gl < H && row >= 0) ? a.rec[row * H + id.gl].w : 0.f;
+    } else {
+        D = head_sum<G, V>(scratch, pA, vg.vok, id.gl, a.g);
+    }
+    if (row >= 0 && id.gl < H) {
+        const float v = DB - D * Sh;
+        float *p = a.del + row * H + id.gl;
+        *p = (a.flags & SAR_FIRST) ? v : *p + v;
+        if constexpr (!GIVEN_D) {
+            const float dd = a.d[row * H + id.gl];
+            a.rec[row * H + id.gl] =
+                make_float4(a.el[row * H + id.gl], a.m[row * H + id.gl], dd > 0.f ? 1.f / dd : 0.f, D);
+        }
+    }
+}
+
+template <typename T, int G, int V, int U, bool GIVEN_D>
+__global__ void __launch_bounds__(kThreads) gat_bwd_dst_kernel(const BwdDstArgs a) {
+    constexpr int EPV = Elem<T>::EPV;
+    constexpr int RPW = 32 / G;
+    constexpr int MODE = GIVEN_D ? kBwdDstGivenD : kBwdDst;
+    extern __shared__ __align__(16) float smem[];
+    const LaneId<G> id;
+    const int H = a.g.H, Hp = a.g.Hp;
+    float *wbase = smem + (size_t)id.warp * warp_smem_floats(Hp, V, 2);
+    int *sj = reinterpret_cast<int *>(wbase) + id.gid * G;
+    float2 *sw = reinterpret_cast<float2 *>(wbase + 64) + (size_t)id.gid * G * Hp;
+    float *scratch = wbase + 64 + id.gid * (G * V);
+
+    const long long item = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
+    WorkItem w = locate_work(item, a.n_dst, a.indptr, a.sp, a.mode);
+    if (a.mode == 0 && w.active && !(a.flags & SAR_FIRST) && GIVEN_D && w.beg == w.end) w.active = false;
+
+    const VecGeom<G, V> vg(a.g, id.gl);
+    const int sh = id.gl & (Hp - 1), se0 = id.gl >> a.g.lgHp, epi = G >> a.g.lgHp;
+    const bool sh_ok = sh < H;
+
+    float el_i = 0.f, m_i = 0.f, invd_i = 0.f;
+    float gv[V][EPV], accA[V][EPV], accB[V][EPV], S[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        S[v] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) gv[v][e] = accA[v][e] = accB[v][e] = 0.f;
+    }
+    if (w.active && sh_ok && w.end > w.beg) {
+        el_i = __ldg(a.el + w.row * H + sh);
+        m_i = __ldg(a.m + w.row * H + sh);
+        const float dd = __ldg(a.d + w.row * H + sh);
+        invd_i = dd > 0.f ? 1.f / dd : 0.f;
+    }
+
+    const int nbatch = (int)((w.end - w.beg + G - 1) / G);
+    const int wmax = __reduce_max_sync(0xffffffffu, nbatch);
+    const uint4 *featv = reinterpret_cast<const uint4 *>(a.feat);
+    for (int it = 0; it < wmax; ++it) {
+        const long long b0 = w.beg + (long long)it * G;
+        const long long rem = w.end - b0;
+        const int nb = rem <= 0 ? 0 : (rem < G ? (int)rem : G);
+        sj[id.gl] = id.gl < nb ? ld_stream_i32(a.indices + b0 + id.gl) : 0;
+        __syncwarp();
+        if (sh_ok)
+            for (int k = se0; k < nb; k += epi) {
+                float gr;
+                const float e = leaky(el_i + __ldg(a.er + (long long)sj[k] * H + sh), a.slope, gr);
+                const float al = fast_exp(e - m_i) * invd_i;  // rematerialised attention coefficient
+                sw[k * Hp + sh] = make_float2(al, al * gr);
+            }
+        __syncwarp();
+        gather_batch<T, G, V, U, MODE>(featv, a.g.n_vec, sj, sw, Hp, nb, id.gl, vg.hv, vg.vok, accA, accB, S);
+        __syncwarp();
+    }
+
+    if (a.mode == 1) {
+        if (!w.active) return;
+        const long long rowf = (long long)a.g.n_vec * EPV;
+        float *recp = a.sp.part + w.seg * a.sp.pstride;
+        store_acc_row<G, V, EPV>(recp, id.gl, vg.vok, accB);
+        if constexpr (!GIVEN_D) store_acc_row<G, V, EPV>(recp + rowf, id.gl, vg.vok, accA);
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+            if (vg.vok[v] && ((v * G + id.gl) % a.g.vph) == 0) recp[2 * rowf + vg.hv[v]] = S[v];
+        return;
+    }
+    if (w.active) load_row_vec<T, G, V>(a.gout, w.row, a.g.n_vec, id.gl, vg.vok, gv);
+    bwd_dst_epilogue<T, G, V, GIVEN_D>(a, id, vg, scratch, w.active ? w.row : -1, gv, accA, accB, S);
+}
+
+template <typename T, int G, int V, bool GIVEN_D>
+__global__ void __launch_bounds__(kThreads) gat_bwd_dst_merge_kernel(const BwdDstArgs a) {
+    constexpr int EPV = Elem<T>::EPV;
+    constexpr int RPW = 32 / G;
+    extern __shared__ __align__(16) float smem[];
+    const LaneId<G> id;
+    float *wbase = smem + (size_t)id.warp * warp_smem_floats(a.g.Hp, V, 2);
+    float *scratch = wbase + 64 + id.gid * (G * V);
+    const long long lr = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
+    const bool active = lr < a.sp.n_long;
+    const VecGeom<G, V> vg(a.g, id.gl);
+    const long long rowf = (long long)a.g.n_vec * EPV;
+    float gv[V][EPV], accA[V][EPV], accB[V][EPV], S[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        S[v] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) gv[v][e] = accA[v][e] = accB[v][e] = 0.f;
+    }
+    long long row = -1;
+    if (active) {
+        row = a.sp.long_row[lr];
+        for (long long s = a.sp.long_seg[lr]; s < a.sp.long_seg[lr + 1]; ++s) {
+            const float *recp = a.sp.part + s * a.sp.pstride;
+            add_acc_row<G, V, EPV>(recp, id.gl, vg.vok, accB, 1.f, 1.f);
+            if constexpr (!GIVEN_D) add_acc_row<G, V, EPV>(recp + rowf, id.gl, vg.vok, accA, 1.f, 1.f);
+#pragma unroll
+            for (int v = 0; v < V; ++v)
+                if (vg.vok[v]) S[v] += recp[2 * rowf + vg.hv[v]];
+        }
+        load_row_vec<T, G, V>(a.gout, row, a.g.n_vec, id.gl, vg.vok, gv);
+    }
+    bwd_dst_epilogue<T, G, V, GIVEN_D>(a, id, vg, scratch, row, gv, accA, accB, S);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Backward, source-major pass over the CSC (the error E_{p->q} Algorithm 2 returns to the owner of
+// the features, and the source half of the score gradient), no atomics: one group per source j,
+//     dfeat_j = sum_i alpha * gout_i
+//     C = sum_i alpha * g' * gout_i,   S = sum_i alpha * g' * D_i
+//     der_j = <feat_j, C> - S           (= sum_i alpha (dalpha - D_i) g')
+// alpha is rebuilt from the destination record {el, m, 1/d, D} and er_j.
+// ------------------------------------------------------------------------------------------------
+struct BwdSrcArgs {
+    long long n_src;
+    const int64_t *t_indptr;
+    const int32_t *t_indices;
+    const void *gout;   // gathered rows
+    const void *feat;   // row-stationary vector [n_src]
+    const float *er;    // [n_src,H]
+    const float4 *rec;  // [n_dst,H]
+    void *dfeat;        // [n_src, n_vec]
+    float *der;         // [n_src,H]
+    float slope;
+    RowGeom g;
+    SplitArgs sp;
+    int mode;
+};
+
+template <typename T, int G, int V>
+__device__ __forceinline__ void bwd_src_epilogue(const BwdSrcArgs &a, const LaneId<G> &id, const VecGeom<G, V> &vg,
+                                                 float *scratch, long long row, const float (&accD)[V][Elem<T>::EPV],
+                                                 const float (&accC)[V][Elem<T>::EPV], const float (&S)[V]) {
+    constexpr int EPV = Elem<T>::EPV;
+    float fv[V][EPV], pC[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) fv[v][e] = 0.f;
+    if (row >= 0) {
+        load_row_vec<T, G, V>(a.feat, row, a.g.n_vec, id.gl, vg.vok, fv);
+        store_row_vec<T, G, V>(a.dfeat, row, a.g.n_vec, id.gl, vg.vok, accD);
+    }
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        pC[v] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) pC[v] = fmaf(fv[v][e], accC[v][e], pC[v]);
+    }
+    const float DC = head_sum<G, V>(scratch, pC, vg.vok, id.gl, a.g);
+    const float Sh = head_scalar<G, V>(scratch, S, vg.hv, vg.vok, id.gl, a.g);
+    if (row >= 0 && id.gl < a.g.H) a.der[row * a.g.H + id.gl] = DC - Sh;
+}
+
+template <typename T, int G, int V, int U>
+__global__ void __launch_bounds__(kThreads) gat_bwd_src_kernel(const BwdSrcArgs a) {
+    constexpr int EPV = Elem<T>::EPV;
+    constexpr int RPW = 32 / G;
+    extern __shared__ __align__(16) float smem[];
+    const LaneId<G> id;
+    const int H = a.g.H, Hp = a.g.Hp;
+    float *wbase = smem + (size_t)id.warp * warp_smem_floats(Hp, V, 4);
+    int *si = reinterpret_cast<int *>(wbase) + id.gid * G;
+    float4 *sw = reinterpret_cast<float4 *>(wbase + 64) + (size_t)id.gid * G * Hp;
+    float *scratch = wbase + 64 + id.gid * (G * V);
+
+    const long long item = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
+    const WorkItem w = locate_work(item, a.n_src, a.t_indptr, a.sp, a.mode);
+    const VecGeom<G, V> vg(a.g, id.gl);
+    const int sh = id.gl & (Hp - 1), se0 = id.gl >> a.g.lgHp, epi = G >> a.g.lgHp;
+    const bool sh_ok = sh < H;
+
+    float er_j = 0.f;
+    float accD[V][EPV], accC[V][EPV], S[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        S[v] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) accD[v][e] = accC[v][e] = 0.f;
+    }
+    if (w.active && sh_ok) er_j = __ldg(a.er + w.row * H + sh);
+
+    const int nbatch = (int)((w.end - w.beg + G - 1) / G);
+    const int wmax = __reduce_max_sync(0xffffffffu, nbatch);
+    const uint4 *goutv = reinterpret_cast<const uint4 *>(a.gout);
+    for (int it = 0; it < wmax; ++it) {
+        const long long b0 = w.beg + (long long)it * G;
+        const long long rem = w.end - b0;
+        const int nb = rem <= 0 ? 0 : (rem < G ? (int)rem : G);
+        si[id.gl] = id.gl < nb ? ld_stream_i32(a.t_indices + b0 + id.gl) : 0;
+        __syncwarp();
+        if (sh_ok)
+            for (int k = se0; k < nb; k += epi) {
+                const float4 r = __ldg(a.rec + (long long)si[k] * H + sh);  // {el_i, m_i, 1/d_i, D_i}
+                float gr;
+                const float e = leaky(r.x + er_j, a.slope, gr);
+                const float al = fast_exp(e - r.y) * r.z;
+                const float w2 = al * gr;
+                sw[k * Hp + sh] = make_float4(al, w2, w2 * r.w, 0.f);
+            }
+        __syncwarp();
+        gather_batch<T, G, V, U, kBwdSrc>(goutv, a.g.n_vec, si, sw, Hp, nb, id.gl, vg.hv, vg.vok, accD, accC, S);
+        __syncwarp();
+    }
+
+    if (a.mode == 1) {
+        if (!w.active) return;
+        const long long rowf = (long long)a.g.n_vec * EPV;
+        float *recp = a.sp.part + w.seg * a.sp.pstride;
+        store_acc_row<G, V, EPV>(recp, id.gl, vg.vok, accD);
+        store_acc_row<G, V, EPV>(recp + rowf, id.gl, vg.vok, accC);
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+            if (vg.vok[v] && ((v * G + id.gl) % a.g.vph) == 0) recp[2 * rowf + vg.hv[v]] = S[v];
+        return;
+    }
+    bwd_src_epilogue<T, G, V>(a, id, vg, scratch, w.active ? w.row : -1, accD, accC, S);
+}
+
+template <typename T, int G, int V>
+__global__ void __launch_bounds__(kThreads) gat_bwd_src_merge_kernel(const BwdSrcArgs a) {
+    constexpr int EPV = Elem<T>::EPV;
+    constexpr int RPW = 32 / G;
+    extern __shared__ __align__(16) float smem[];
+    const LaneId<G> id;
+    float *wbase = smem + (size_t)id.warp * warp_smem_floats(a.g.Hp, V, 4);
+    float *scratch = wbase + 64 + id.gid * (G * V);
+    const long long lr = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
+    const VecGeom<G, V> vg(a.g, id.gl);
+    const long long rowf = (long long)a.g.n_vec * EPV;
+    float accD[V][EPV], accC[V][EPV], S[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        S[v] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) accD[v][e] = accC[v][e] = 0.f;
+    }
+    long long row = -1;
+    if (lr < a.sp.n_long) {
+        row = a.sp.long_row[lr];
+        for (long long s = a.sp.long_seg[lr]; s < a.sp.long_seg[lr + 1]; ++s) {
+            const float *recp = a.sp.part + s * a.sp.pstride;
+            add_acc_row<G, V, EPV>(recp, id.gl, vg.vok, accD, 1.f, 1.f);
+            add_acc_row<G, V, EPV>(recp + rowf, id.gl, vg.vok, accC, 1.f, 1.f);
+#pragma unroll
+            for (int v = 0; v < V; ++v)
+                if (vg.vok[v]) S[v] += recp[2 * rowf + vg.hv[v]];
+        }
+    }
+    bwd_src_epilogue<T, G, V>(a, id, vg, scratch, row, accD, accC, S);
+}
+
+// ------------------------------------------------------------------------------------------------
+// Row dot D[i,h] = <gout_i, out_i> and the packed destination record (streaming, one group per row).
+// ------------------------------------------------------------------------------------------------
+struct PrepArgs {
+    long long n_dst;
+    const void *out;     // type T, or float32 numerator when acc_is_numerator
+    const void *gout;
+    const float *el, *m, *d;
+    float *D;            // may be null
+    float4 *rec;
+    int acc_is_numerator;
+    RowGeom g;
+};
+
+template <typename T, int G, int V>
+__global__ void __launch_bounds__(kThreads) gat_bwd_prepare_kernel(const PrepArgs a) {
+    constexpr int EPV = Elem<T>::EPV;
+    constexpr int RPW = 32 / G;
+    extern __shared__ __align__(16) float smem[];
+    const LaneId<G> id;
+    float *scratch = smem + (size_t)id.warp * (32 * V) + id.gid * (G * V);
+    const long long row = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
+    const bool active = row < a.n_dst;
+    const VecGeom<G, V> vg(a.g, id.gl);
+    const int H = a.g.H;
+    float gv[V][EPV], ov[V][EPV], p[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) gv[v][e] = ov[v][e] = 0.f;
+    if (active) {
+        load_row_vec<T, G, V>(a.gout, row, a.g.n_vec, id.gl, vg.vok, gv);
+        if (a.acc_is_numerator)
+            load_acc_row<G, V, EPV>(reinterpret_cast<const float *>(a.out) + row * (long long)(a.g.n_vec * EPV), id.gl,
+                                    vg.vok, ov);
+        else
+            load_row_vec<T, G, V>(a.out, row, a.g.n_vec, id.gl, vg.vok, ov);
+    }
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        p[v] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) p[v] = fmaf(gv[v][e], ov[v][e], p[v]);
+    }
+    float D = head_sum<G, V>(scratch, p, vg.vok, id.gl, a.g);
+    if (active && id.gl < H) {
+        const float dd = a.d[row * H + id.gl];
+        const float inv = dd > 0.f ? 1.f / dd : 0.f;
+        if (a.acc_is_numerator) D *= inv;
+        if (a.D) a.D[row * H + id.gl] = D;
+        a.rec[row * H + id.gl] = make_float4(a.el[row * H + id.gl], a.m[row * H + id.gl], inv, D);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Sum aggregation (Eq. 2): the gather phase alone.
+// ------------------------------------------------------------------------------------------------
+struct SumArgs {
+    long long n_dst;
+    const int64_t *indptr;
+    const int32_t *indices;
+    const void *feat;
+    void *out;
+    const int64_t *deg_total;  // for SAR_MEAN
+    unsigned flags;
+    RowGeom g;                 // H = 1, vph = n_vec
+    SplitArgs sp;
+    int mode;
+};
+
+template <typename T, int G, int V>
+__device__ __forceinline__ void sum_epilogue(const SumArgs &a, int gl, const VecGeom<G, V> &vg, long long row,
+                                             float (&acc)[V][Elem<T>::EPV]) {
+    constexpr int EPV = Elem<T>::EPV;
+    if (!(a.flags & SAR_FIRST)) {
+        float old[V][EPV];
+        load_row_vec<T, G, V, false>(a.out, row, a.g.n_vec, gl, vg.vok, old);
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) acc[v][e] += old[v][e];
+    }
+    if ((a.flags & SAR_MEAN) && (a.flags & SAR_LAST)) {
+        const long long dg = a.deg_total[row];
+        const float inv = dg > 0 ? 1.f / (float)dg : 0.f;
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) acc[v][e] *= inv;
+    }
+    store_row_vec<T, G, V>(a.out, row, a.g.n_vec, gl, vg.vok, acc);
+}
+
+template <typename T, int G, int V, int U>
+__global__ void __launch_bounds__(kThreads) spmm_kernel(const SumArgs a) {
+    constexpr int EPV = Elem<T>::EPV;
+    constexpr int RPW = 32 / G;
+    extern __shared__ __align__(16) float smem[];
+    const LaneId<G> id;
+    int *sj = reinterpret_cast<int *>(smem) + id.warp * 32 + id.gid * G;
+    const long long item = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
+    WorkItem w = locate_work(item, a.n_dst, a.indptr, a.sp, a.mode);
+    const bool must_write = (a.flags & SAR_FIRST) || ((a.flags & SAR_MEAN) && (a.flags & SAR_LAST));
+    if (a.mode == 0 && w.active && !must_write && w.beg == w.end) w.active = false;
+    const VecGeom<G, V> vg(a.g, id.gl);
+    float acc[V][EPV], dummy[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        dummy[v] = 0.f;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) acc[v][e] = 0.f;
+    }
+    const int nbatch = (int)((w.end - w.beg + G - 1) / G);
+    const int wmax = __reduce_max_sync(0xffffffffu, nbatch);
+    const uint4 *featv = reinterpret_cast<const uint4 *>(a.feat);
+    for (int it = 0; it < wmax; ++it) {
+        const long long b0 = w.beg + (long long)it * G;
+        const long long rem = w.end - b0;
+        const int nb = rem <= 0 ? 0 : (rem < G ? (int)rem : G);
+        sj[id.gl] = id.gl < nb ? ld_stream_i32(a.indices + b0 + id.gl) : 0;
+        __syncwarp();
+        gather_batch<T, G, V, U, kSum>(featv, a.g.n_vec, sj, nullptr, 1, nb, id.gl, vg.hv, vg.vok, acc, acc, dummy);
+        __syncwarp();
+    }
+    if (!w.active) return;
+    if (a.mode == 1) {
+        store_acc_row<G, V, EPV>(a.sp.part + w.seg * a.sp.pstride, id.gl, vg.vok, acc);
+        return;
+    }
+    sum_epilogue<T, G, V>(a, id.gl, vg, w.row, acc);
+}
+
+template <typename T, int G, int V>
+__global__ void __launch_bounds__(kThreads) spmm_merge_kernel(const SumArgs a) {
+    constexpr int EPV = Elem<T>::EPV;
+    constexpr int RPW = 32 / G;
+    const LaneId<G> id;
+    const long long lr = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
+    if (lr >= a.sp.n_long) return;
+    const VecGeom<G, V> vg(a.g, id.gl);
+    float acc[V][EPV];
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) acc[v][e] = 0.f;
+    for (long long s = a.sp.long_seg[lr]; s < a.sp.long_seg[lr + 1]; ++s)
+        add_acc_row<G, V, EPV>(a.sp.part + s * a.sp.pstride, id.gl, vg.vok, acc, 1.f, 1.f);
+    sum_epilogue<T, G, V>(a, id.gl, vg, a.sp.long_row[lr], acc);
+}
+
+}  // namespace sar

@@ -1,0 +1,367 @@
+"""GPU parity tests: the CUDA library (through its C-ABI binding) against the CPU oracle on the
+same seeded inputs, element by element.
+
+Tolerances (|got - want| <= atol + rtol*|want|, want = float64 oracle on the same rounded inputs):
+  float32 outputs        rtol 1e-5, atol 1e-6
+  float32 gradients      rtol 1e-4, atol 1e-5 * scale   (scale = RMS of the oracle's array: the
+                         sums cancel, so a floor proportional to the operand scale is needed)
+  bf16 storage variants  rtol 2e-2, atol 2e-2 * scale   (outputs are rounded to bf16 once)
+Integer outputs (CSR, CSC, partition split, plans) are compared bit for bit.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+from helpers import allclose_report
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from paper_2111_06483_b200 import api, binding as B
+
+DEV = "cuda"
+
+
+def rms(x):
+    x = np.asarray(x, dtype=np.float64)
+    x = x[np.isfinite(x)]
+    return float(np.sqrt(np.mean(x * x))) if x.size else 0.0
+
+
+def check_out(got, want, dtype, what):
+    got = got.float().cpu().numpy()
+    if dtype == "bf16":
+        allclose_report(got, want, 2e-2, 2e-2 * rms(want), what)
+    else:
+        allclose_report(got, want, 1e-5, 1e-6, what)
+
+
+def check_grad(got, want, dtype, what):
+    got = got.float().cpu().numpy()
+    if dtype == "bf16":
+        allclose_report(got, want, 2e-2, 2e-2 * rms(want), what)
+    else:
+        allclose_report(got, want, 1e-4, 1e-5 * rms(want), what)
+
+
+class Problem:
+    """Seeded inputs on the host (for the oracle) and on the device (for the library)."""
+
+    def __init__(self, n, src, dst, H, F, seed, dtype="f32", k=1, threshold=api.DEFAULT_THRESHOLD if torch.cuda.is_available() else 0,
+                 build_parts=False, scale=1.0):
+        self.n, self.H, self.F, self.dtype, self.k = n, H, F, dtype, k
+        self.src, self.dst = src.cpu(), dst.cpu()
+        t = workloads.make_node_inputs(n, H, F, seed, dtype=dtype)
+        if scale != 1.0:
+            t["el"] = t["el"] * scale
+            t["er"] = t["er"] * scale
+        self.host = {k_: v.float().numpy() for k_, v in t.items()}
+        self.dev = {k_: v.to(DEV) for k_, v in t.items()}
+        self.indptr, self.indices = oracle.csr_from_coo(n, n, self.src.numpy(), self.dst.numpy())
+        self.graph = api.Graph.from_coo(n, self.src.to(DEV), self.dst.to(DEV), k=k, threshold=threshold,
+                                        build_parts=build_parts)
+
+    def oracle_fwd(self, slope=0.2):
+        h = self.host
+        return oracle.gat_fwd(self.indptr, self.indices, h["feat"], h["el"], h["er"], slope)
+
+    def oracle_bwd(self, fwd, slope=0.2):
+        h = self.host
+        return oracle.gat_bwd(self.indptr, self.indices, h["feat"], h["el"], h["er"], fwd.alpha, h["gout"], slope)
+
+    def gpu_fwd(self, mode="fused", slope=0.2):
+        d = self.dev
+        return api.gat_forward(self.graph, d["feat"], d["el"], d["er"], slope, mode=mode)
+
+    def gpu_bwd(self, m, dd, out=None, mode="fused", slope=0.2):
+        d = self.dev
+        return api.gat_backward(self.graph, d["feat"], d["el"], d["er"], m, dd, d["gout"], slope, out=out, mode=mode)
+
+
+def uniform_problem(n, e, H, F, seed, loops=False, **kw):
+    src, dst = workloads.uniform_edges(n, e, seed, loops)
+    return Problem(n, src, dst, H, F, seed, **kw)
+
+
+def config_problem(name, scale=None, **kw):
+    cfg = workloads.CONFIGS[name]
+    if scale:
+        cfg = cfg.scaled(scale)
+    src, dst = workloads.make_graph(cfg)
+    n = cfg.n
+    return cfg, Problem(n, src, dst, cfg.heads, cfg.feat, cfg.seed, k=cfg.k, **kw)
+
+
+# ------------------------------------------------------------------------------------------------
+# integer side
+# ------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n,e,k", [(2000, 20000, 1), (5000, 100000, 8), (257, 3000, 16), (64, 0, 3), (1, 5, 1)])
+def test_graph_preparation_is_bit_exact(n, e, k):
+    if n == 1:
+        src = torch.zeros(e, dtype=torch.int32)
+        dst = torch.zeros(e, dtype=torch.int32)
+    elif e == 0:
+        src = torch.zeros(0, dtype=torch.int32)
+        dst = torch.zeros(0, dtype=torch.int32)
+    else:
+        src, dst = workloads.uniform_edges(n, e, 40 + k, self_loops=True)
+        src = torch.cat([src, src[:50]])           # duplicates
+        dst = torch.cat([dst, dst[:50]])
+    g = api.Graph.from_coo(n, src.to(DEV), dst.to(DEV), k=k, threshold=8, build_parts=True)
+    indptr, indices = oracle.csr_from_coo(n, n, src.numpy(), dst.numpy())
+    t_indptr, t_indices = oracle.csr_transpose(n, n, indptr, indices)
+    assert np.array_equal(g.whole.indptr.cpu().numpy(), indptr)
+    assert np.array_equal(g.whole.indices.cpu().numpy(), indices)
+    assert np.array_equal(g.whole.t_indptr.cpu().numpy(), t_indptr)
+    assert np.array_equal(g.whole.t_indices.cpu().numpy(), t_indices)
+    # the library's own transpose call agrees too
+    ws = torch.empty(B.sar_graph_workspace_bytes(len(indices), n), dtype=torch.uint8, device=DEV)
+    tp = torch.empty(n + 1, dtype=torch.int64, device=DEV)
+    ti = torch.empty(max(len(indices), 1), dtype=torch.int32, device=DEV)
+    B.sar_csr_transpose(n, n, g.whole.indptr, g.whole.indices, tp, ti, ws)
+    assert np.array_equal(tp.cpu().numpy(), t_indptr) and np.array_equal(ti.cpu().numpy()[:len(indices)], t_indices)
+    bounds = oracle.partition_bounds(n, k)
+    assert list(bounds) == g.bounds
+    sp = oracle.csr_split(n, indptr, indices, bounds)
+    for q, part in enumerate(g.parts):
+        ip, idx = sp.part(q)
+        assert np.array_equal(part.indptr.cpu().numpy(), ip)
+        assert np.array_equal(part.indices.cpu().numpy()[:part.nnz], idx)
+        # CSC slice of the partition == transpose of the partition's CSR
+        tq_ip, tq_idx = oracle.csr_transpose(n, int(bounds[q + 1] - bounds[q]), ip, idx)
+        assert np.array_equal(part.t_indptr.cpu().numpy(), tq_ip)
+        assert np.array_equal(part.t_indices.cpu().numpy()[:part.nnz], tq_idx)
+        flag = torch.zeros(1, dtype=torch.int32, device=DEV)
+        B.sar_validate_part(part, flag)
+    # long-row plan: rows with more than 8 edges, ceil(deg/8) segments each
+    deg = np.diff(indptr)
+    long_rows = np.nonzero(deg > 8)[0]
+    if len(long_rows):
+        s = g.whole.split
+        assert s.n_long == len(long_rows) and np.array_equal(s.long_row.cpu().numpy(), long_rows)
+        segs = -(-deg[long_rows] // 8)
+        assert np.array_equal(s.long_seg.cpu().numpy(), np.concatenate([[0], np.cumsum(segs)]))
+        assert s.n_seg == segs.sum()
+    else:
+        assert g.whole.split is None
+
+
+def test_validate_part_flags_a_broken_graph():
+    src, dst = workloads.uniform_edges(100, 1000, 3, False)
+    g = api.Graph.from_coo(100, src.to(DEV), dst.to(DEV))
+    flag = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.sar_validate_part(g.whole, flag)
+    bad_idx = g.whole.indices.clone()
+    bad_idx[5] = 100                                   # out of range
+    bad = B.Part(100, 100, g.whole.indptr, bad_idx)
+    with pytest.raises(B.SarError) as ei:
+        B.sar_validate_part(bad, flag)
+    assert ei.value.code == -6
+
+
+# ------------------------------------------------------------------------------------------------
+# forward + backward, float32
+# ------------------------------------------------------------------------------------------------
+
+def _full_check(p, dtype="f32", modes=("fused",), slope=0.2):
+    f = p.oracle_fwd(slope)
+    b = p.oracle_bwd(f, slope)
+    results = {}
+    for mode in modes:
+        out, m, d = p.gpu_fwd(mode, slope)
+        check_out(out, f.out, dtype, f"out[{mode}]")
+        allclose_report(m.cpu().numpy(), f.m, 1e-6, 1e-6, f"m[{mode}]")
+        allclose_report(d.cpu().numpy(), f.d, 1e-5, 1e-6, f"d[{mode}]")
+        dfeat, del_, der = p.gpu_bwd(m, d, out=out, mode=mode, slope=slope)
+        check_grad(dfeat, b.dfeat, dtype, f"dfeat[{mode}]")
+        if mode == "stateful" and dtype == "bf16" and p.k > 1:
+            # the row dot is taken from the bf16-rounded `out` here: a looser floor applies
+            allclose_report(del_.cpu().numpy(), b.del_, 2e-2, 0.1 * rms(b.del_), f"del[{mode}]")
+            allclose_report(der.cpu().numpy(), b.der, 2e-2, 0.1 * rms(b.der), f"der[{mode}]")
+        else:
+            check_grad(del_, b.del_, dtype, f"del[{mode}]")
+            check_grad(der, b.der, dtype, f"der[{mode}]")
+        results[mode] = (out, m, d, dfeat, del_, der)
+    return f, b, results
+
+
+def test_tiny_config_forward_backward_fp32():
+    cfg, p = config_problem("tiny")
+    assert p.graph.nnz == 22000
+    _full_check(p)
+
+
+@pytest.mark.parametrize("threshold", [0, 16])
+def test_sequential_partitions_equal_single_pass(threshold):
+    """K = 8 partitions, stateful (Algorithm 1 call by call) and fused, against K = 1 and the oracle."""
+    cfg, p = config_problem("seqpart", scale=0.2, build_parts=True, threshold=threshold)
+    assert p.k == 8
+    f, b, res = _full_check(p, modes=("fused", "stateful"))
+    out_f, m_f, d_f = res["fused"][:3]
+    out_s, m_s, d_s = res["stateful"][:3]
+    assert torch.equal(m_f, m_s)                        # the running max ends exact in any schedule
+    # K = 1 through the per-partition entry point
+    g1 = api.Graph.from_coo(p.n, p.src.to(DEV), p.dst.to(DEV), k=1, threshold=threshold, build_parts=True)
+    d = p.dev
+    out_1, m_1, d_1 = api.gat_forward(g1, d["feat"], d["el"], d["er"], 0.2, mode="stateful")
+    assert torch.equal(m_1, m_s)
+    allclose_report(out_s.cpu().numpy(), out_1.cpu().numpy(), 1e-5, 1e-6, "K=8 vs K=1")
+    # oracle's sequential form agrees with the GPU's statistics as well
+    sp = oracle.csr_split(p.n, p.indptr, p.indices, oracle.partition_bounds(p.n, 8))
+    o_out, o_m, o_d = oracle.gat_fwd_seq(sp, p.host["feat"], p.host["el"], p.host["er"], 0.2)
+    allclose_report(out_s.cpu().numpy(), o_out, 1e-5, 1e-6, "stateful vs sequential oracle")
+    allclose_report(d_s.cpu().numpy(), o_d, 1e-5, 1e-6, "d vs sequential oracle")
+
+
+@pytest.mark.parametrize("H,F,dtype", [(4, 64, "f32"), (4, 64, "bf16"), (8, 32, "bf16"), (4, 32, "bf16"), (1, 8, "f32"),
+                                       (2, 128, "f32"), (3, 12, "f32"), (16, 8, "bf16"), (4, 256, "bf16")])
+@pytest.mark.parametrize("threshold", [0, 24])
+def test_shapes_of_the_vector_kernels(H, F, dtype, threshold):
+    """Power-law graph with hubs in both directions, empty rows, several tiles and a ragged tail."""
+    cfg = workloads.CONFIGS["medium"].scaled(0.002)
+    src, dst = workloads.make_graph(cfg)
+    p = Problem(cfg.n, src, dst, H, F, 50 + H + F, dtype=dtype, k=4, threshold=threshold, build_parts=True)
+    deg = np.diff(p.indptr)
+    assert deg.max() > 24 and (deg == 0).any()
+    _full_check(p, dtype=dtype, modes=("fused", "stateful"))
+
+
+@pytest.mark.parametrize("H,F,dtype", [(3, 5, "f32"), (1, 1, "f32"), (2, 7, "bf16"), (5, 3, "bf16")])
+def test_odd_shapes_run_on_the_scalar_kernels(H, F, dtype):
+    p = uniform_problem(300, 3000, H, F, 60 + H, loops=True, dtype=dtype, k=3, build_parts=True)
+    _full_check(p, dtype=dtype, modes=("fused", "stateful"))
+
+
+def test_misaligned_feature_pointer_falls_back_to_scalar_kernels():
+    p = uniform_problem(200, 2000, 2, 4, 61)
+    d = p.dev
+    pad = torch.zeros(p.n * 8 + 1, dtype=torch.float32, device=DEV)
+    feat = pad[1:].view(p.n, 2, 4)
+    feat.copy_(d["feat"])
+    assert feat.data_ptr() % 16 != 0
+    out, m, dd = api.gat_forward(p.graph, feat, d["el"], d["er"], 0.2)
+    check_out(out, p.oracle_fwd().out, "f32", "misaligned")
+
+
+def test_large_logits_stay_finite_and_match():
+    p = uniform_problem(500, 6000, 4, 16, 62, scale=300.0, k=4, build_parts=True)
+    f = p.oracle_fwd()
+    for mode in ("fused", "stateful"):
+        out, m, d = p.gpu_fwd(mode)
+        assert torch.isfinite(out).all()
+        # scores of magnitude ~1e3 carry float32 input rounding of ~1e-4 in the exponent
+        allclose_report(out.cpu().numpy(), f.out, 2e-3, 1e-4, f"large logits [{mode}]")
+        allclose_report(m.cpu().numpy(), f.m, 1e-6, 1e-6, "m")
+
+
+def test_degenerate_graphs():
+    # no edges at all
+    n = 37
+    empty = torch.zeros(0, dtype=torch.int32, device=DEV)
+    g = api.Graph.from_coo(n, empty, empty)
+    t = {k: v.to(DEV) for k, v in workloads.make_node_inputs(n, 4, 8, 1).items()}
+    out, m, d = api.gat_forward(g, t["feat"], t["el"], t["er"], 0.2)
+    assert (out == 0).all() and (d == 0).all() and torch.isneginf(m).all()
+    dfeat, del_, der = api.gat_backward(g, t["feat"], t["el"], t["er"], m, d, t["gout"], 0.2)
+    assert (dfeat == 0).all() and (del_ == 0).all() and (der == 0).all()
+    # one node, many self-loops (duplicates): out = feat, gradients flow back to the same row
+    loops = torch.zeros(40, dtype=torch.int32)
+    p = Problem(1, loops, loops, 2, 8, 2, threshold=16)
+    _full_check(p)
+    # a single hub: every node points at node 0 (one giant row, split into segments)
+    n = 3000
+    src = torch.arange(n, dtype=torch.int32)
+    dst = torch.zeros(n, dtype=torch.int32)
+    p = Problem(n, src, dst, 4, 16, 3, threshold=64)
+    assert p.graph.whole.split.n_long == 1
+    _full_check(p)
+    # and the transpose: node 0 points at everyone (one giant CSC row)
+    p = Problem(n, dst, src, 4, 16, 4, threshold=64)
+    assert p.graph.whole.t_split.n_long == 1
+    _full_check(p)
+
+
+def test_row_dot_identity_and_prepare():
+    """D = <gout, out> (what lets each partition's backward run on its own)."""
+    p = uniform_problem(400, 5000, 4, 8, 63)
+    f = p.oracle_fwd()
+    b = p.oracle_bwd(f)
+    out, m, d = p.gpu_fwd()
+    D = torch.empty((p.n, 4), dtype=torch.float32, device=DEV)
+    ws = api.gat_workspace(p.graph.whole, 4, 8, torch.float32)
+    B.sar_gat_bwd_prepare(p.n, 4, 8, out, False, p.dev["gout"], p.dev["el"], m, d, D, ws)
+    allclose_report(D.cpu().numpy(), b.D, 1e-4, 1e-5 * rms(b.D), "D")
+
+
+# ------------------------------------------------------------------------------------------------
+# sum aggregation
+# ------------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("F,dtype", [(256, "f32"), (256, "bf16"), (64, "f32"), (8, "bf16"), (5, "f32"), (1000, "f32")])
+@pytest.mark.parametrize("threshold", [0, 24])
+def test_spmm_sum_forward_backward_mean_and_partitions(F, dtype, threshold):
+    cfg = workloads.CONFIGS["medium"].scaled(0.002)
+    src, dst = workloads.make_graph(cfg)
+    n = cfg.n
+    g = api.Graph.from_coo(n, src.to(DEV), dst.to(DEV), k=4, threshold=threshold, build_parts=True)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    feat = workloads.normal_tensor((n, F), 7, 1, dtype=tdt)
+    gout = workloads.normal_tensor((n, F), 7, 2, dtype=tdt)
+    indptr, indices = oracle.csr_from_coo(n, n, src.numpy(), dst.numpy())
+    t_indptr, t_indices = oracle.csr_transpose(n, n, indptr, indices)
+    want = oracle.spmm(indptr, indices, feat.float().numpy())
+    got = api.spmm_sum(g.whole, feat.to(DEV))
+    tol = dict(rtol=2e-2, atol=2e-2 * rms(want)) if dtype == "bf16" else dict(rtol=1e-5, atol=1e-5)
+    allclose_report(got.float().cpu().numpy(), want, what="spmm", **tol)
+    # backward = the same call on the transposed partition
+    want_b = oracle.spmm(t_indptr, t_indices, gout.float().numpy())
+    got_b = api.spmm_sum(g.whole.transposed(), gout.to(DEV))
+    allclose_report(got_b.float().cpu().numpy(), want_b, what="spmm bwd", **tol)
+    # mean
+    deg = torch.from_numpy(np.diff(indptr)).to(DEV)
+    got_m = api.spmm_sum(g.whole, feat.to(DEV), mean=True, deg_total=deg)
+    allclose_report(got_m.float().cpu().numpy(), oracle.spmm(indptr, indices, feat.float().numpy(), mean=True),
+                    what="spmm mean", **tol)
+    # K partitions accumulated one after the other
+    out = torch.empty((n, F), dtype=tdt, device=DEV)
+    fd = feat.to(DEV)
+    for q, part in enumerate(g.parts):
+        flags = (B.SAR_FIRST if q == 0 else 0) | (B.SAR_LAST if q == 3 else 0)
+        ws = torch.empty(B.sar_spmm_workspace_bytes(part, F, B._dtype(fd)), dtype=torch.uint8, device=DEV)
+        B.sar_spmm_agg(part, fd[g.bounds[q]:g.bounds[q + 1]], F, flags, None, out, ws)
+    tol_k = dict(rtol=4e-2, atol=4e-2 * rms(want)) if dtype == "bf16" else tol  # re-rounded once per partition
+    allclose_report(out.float().cpu().numpy(), want, what="spmm K=4", **tol_k)
+
+
+# ------------------------------------------------------------------------------------------------
+# argument errors: status codes, nothing launched
+# ------------------------------------------------------------------------------------------------
+
+def test_argument_errors_return_status_codes():
+    p = uniform_problem(100, 500, 2, 8, 64)
+    d = p.dev
+    m = torch.empty((p.n, 2), device=DEV)
+    dd = torch.empty((p.n, 2), device=DEV)
+    out = torch.empty((p.n, 2, 8), device=DEV)
+    with pytest.raises(B.SarError) as ei:       # partial pass without a numerator buffer
+        B.sar_gat_fwd(p.graph.whole, d["feat"], d["el"], d["er"], 2, 8, 0.2, B.SAR_FIRST, None, m, dd, out, None)
+    assert ei.value.code == -1
+    with pytest.raises(B.SarError) as ei:       # unknown flag
+        B.sar_gat_fwd(p.graph.whole, d["feat"], d["el"], d["er"], 2, 8, 0.2, 64, None, m, dd, out, None)
+    assert ei.value.code == -1
+    with pytest.raises(B.SarError) as ei:       # backward without workspace
+        B.sar_gat_bwd(p.graph.whole, d["feat"], d["el"], d["er"], m, dd, d["gout"], 2, 8, 0.2, 3, out, m, dd, None)
+    assert ei.value.code == -4
+    with pytest.raises(B.SarError) as ei:       # partition buffers that are not one array
+        B.sar_gat_fwd_fused(p.graph.whole, [0, 50, 100], [d["feat"], d["feat"]], d["el"], [d["er"], d["er"]], 2, 8, 0.2,
+                            m, dd, out, None)
+    assert ei.value.code == -2
+    fwd_only = B.Part(p.n, p.n, p.graph.whole.indptr, p.graph.whole.indices)
+    ws = api.gat_workspace(p.graph.whole, 2, 8, torch.float32)
+    with pytest.raises(B.SarError) as ei:       # backward needs the CSC
+        B.sar_gat_bwd(fwd_only, d["feat"], d["el"], d["er"], m, dd, d["gout"], 2, 8, 0.2, 3, out, m, dd, ws)
+    assert ei.value.code == -1
+    torch.cuda.synchronize()
