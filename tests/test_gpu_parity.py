@@ -3,8 +3,9 @@ same seeded inputs, element by element.
 
 Tolerances (|got - want| <= atol + rtol*|want|, want = float64 oracle on the same rounded inputs):
   float32 outputs        rtol 1e-5, atol 1e-6
-  float32 gradients      rtol 1e-4, atol 1e-5 * scale   (scale = RMS of the oracle's array: the
-                         sums cancel, so a floor proportional to the operand scale is needed)
+  float32 gradients      rtol 1e-4, atol 1e-5 * scale   (scale = max(RMS of the oracle's array, 1):
+                         the sums cancel, so a floor proportional to the operand scale, which is
+                         O(1) for N(0,1) inputs, is needed)
   bf16 storage variants  rtol 2e-2, atol 2e-2 * scale   (outputs are rounded to bf16 once)
 Integer outputs (CSR, CSC, partition split, plans) are compared bit for bit.
 """
@@ -38,12 +39,13 @@ def check_out(got, want, dtype, what):
         allclose_report(got, want, 1e-5, 1e-6, what)
 
 
-def check_grad(got, want, dtype, what):
+def check_grad(got, want, dtype, what, floor=1.0):
     got = got.float().cpu().numpy()
+    scale = max(rms(want), floor)    # inputs are N(0,1): sums of O(1) terms that cancel
     if dtype == "bf16":
-        allclose_report(got, want, 2e-2, 2e-2 * rms(want), what)
+        allclose_report(got, want, 2e-2, 2e-2 * scale, what)
     else:
-        allclose_report(got, want, 1e-4, 1e-5 * rms(want), what)
+        allclose_report(got, want, 1e-4, 1e-5 * scale, what)
 
 
 class Problem:
@@ -83,6 +85,13 @@ class Problem:
 def uniform_problem(n, e, H, F, seed, loops=False, **kw):
     src, dst = workloads.uniform_edges(n, e, seed, loops)
     return Problem(n, src, dst, H, F, seed, **kw)
+
+
+def hub_graph(n=6000, e=60000, d_max=600.0, seed=9):
+    """Small power-law graph (exponent 2.1) with hubs in both directions and isolated rows."""
+    spec = workloads.ChungLuSpec(n=n, e=e, gamma=2.1, d_max=d_max, seed=seed)
+    src, dst = workloads.chung_lu_edges(spec)
+    return n, src, dst
 
 
 def config_problem(name, scale=None, **kw):
@@ -166,7 +175,7 @@ def test_validate_part_flags_a_broken_graph():
 # forward + backward, float32
 # ------------------------------------------------------------------------------------------------
 
-def _full_check(p, dtype="f32", modes=("fused",), slope=0.2):
+def _full_check(p, dtype="f32", modes=("fused",), slope=0.2, grad_floor=1.0):
     f = p.oracle_fwd(slope)
     b = p.oracle_bwd(f, slope)
     results = {}
@@ -182,8 +191,8 @@ def _full_check(p, dtype="f32", modes=("fused",), slope=0.2):
             allclose_report(del_.cpu().numpy(), b.del_, 2e-2, 0.1 * rms(b.del_), f"del[{mode}]")
             allclose_report(der.cpu().numpy(), b.der, 2e-2, 0.1 * rms(b.der), f"der[{mode}]")
         else:
-            check_grad(del_, b.del_, dtype, f"del[{mode}]")
-            check_grad(der, b.der, dtype, f"der[{mode}]")
+            check_grad(del_, b.del_, dtype, f"del[{mode}]", grad_floor)
+            check_grad(der, b.der, dtype, f"der[{mode}]", grad_floor)
         results[mode] = (out, m, d, dfeat, del_, der)
     return f, b, results
 
@@ -221,9 +230,8 @@ def test_sequential_partitions_equal_single_pass(threshold):
 @pytest.mark.parametrize("threshold", [0, 24])
 def test_shapes_of_the_vector_kernels(H, F, dtype, threshold):
     """Power-law graph with hubs in both directions, empty rows, several tiles and a ragged tail."""
-    cfg = workloads.CONFIGS["medium"].scaled(0.002)
-    src, dst = workloads.make_graph(cfg)
-    p = Problem(cfg.n, src, dst, H, F, 50 + H + F, dtype=dtype, k=4, threshold=threshold, build_parts=True)
+    n, src, dst = hub_graph()
+    p = Problem(n, src, dst, H, F, 50 + H + F, dtype=dtype, k=4, threshold=threshold, build_parts=True)
     deg = np.diff(p.indptr)
     assert deg.max() > 24 and (deg == 0).any()
     _full_check(p, dtype=dtype, modes=("fused", "stateful"))
@@ -279,9 +287,12 @@ def test_degenerate_graphs():
     assert p.graph.whole.split.n_long == 1
     _full_check(p)
     # and the transpose: node 0 points at everyone (one giant CSC row)
+    # Every destination has ONE in-edge here, so each edge's softmax gradient is exactly 0 in exact
+    # arithmetic; the source-major pass forms it as <feat_0, sum_i w_i gout_i> - sum_i w_i D_i over
+    # 3000 edges with |dalpha| ~ 5, which float32 leaves at ~eps*sqrt(3000)*5*few = 1e-4.
     p = Problem(n, dst, src, 4, 16, 4, threshold=64)
     assert p.graph.whole.t_split.n_long == 1
-    _full_check(p)
+    _full_check(p, grad_floor=30.0)
 
 
 def test_row_dot_identity_and_prepare():
@@ -303,9 +314,7 @@ def test_row_dot_identity_and_prepare():
 @pytest.mark.parametrize("F,dtype", [(256, "f32"), (256, "bf16"), (64, "f32"), (8, "bf16"), (5, "f32"), (1000, "f32")])
 @pytest.mark.parametrize("threshold", [0, 24])
 def test_spmm_sum_forward_backward_mean_and_partitions(F, dtype, threshold):
-    cfg = workloads.CONFIGS["medium"].scaled(0.002)
-    src, dst = workloads.make_graph(cfg)
-    n = cfg.n
+    n, src, dst = hub_graph()
     g = api.Graph.from_coo(n, src.to(DEV), dst.to(DEV), k=4, threshold=threshold, build_parts=True)
     tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
     feat = workloads.normal_tensor((n, F), 7, 1, dtype=tdt)
@@ -314,7 +323,11 @@ def test_spmm_sum_forward_backward_mean_and_partitions(F, dtype, threshold):
     t_indptr, t_indices = oracle.csr_transpose(n, n, indptr, indices)
     want = oracle.spmm(indptr, indices, feat.float().numpy())
     got = api.spmm_sum(g.whole, feat.to(DEV))
-    tol = dict(rtol=2e-2, atol=2e-2 * rms(want)) if dtype == "bf16" else dict(rtol=1e-5, atol=1e-5)
+    # plain sums of N(0,1) rows cancel: sequential float32 accumulation of deg unit-scale terms
+    # leaves up to ~2^-24 * deg * |x| (typically eps*sqrt(deg)*|partial sum|), so the floor follows
+    # the longest row: 2^-23 * max degree
+    max_deg = int(max(np.diff(indptr).max(), np.diff(t_indptr).max()))
+    tol = dict(rtol=2e-2, atol=2e-2 * rms(want)) if dtype == "bf16" else dict(rtol=1e-5, atol=2.0 ** -23 * max_deg)
     allclose_report(got.float().cpu().numpy(), want, what="spmm", **tol)
     # backward = the same call on the transposed partition
     want_b = oracle.spmm(t_indptr, t_indices, gout.float().numpy())
@@ -332,7 +345,8 @@ def test_spmm_sum_forward_backward_mean_and_partitions(F, dtype, threshold):
         flags = (B.SAR_FIRST if q == 0 else 0) | (B.SAR_LAST if q == 3 else 0)
         ws = torch.empty(B.sar_spmm_workspace_bytes(part, F, B._dtype(fd)), dtype=torch.uint8, device=DEV)
         B.sar_spmm_agg(part, fd[g.bounds[q]:g.bounds[q + 1]], F, flags, None, out, ws)
-    tol_k = dict(rtol=4e-2, atol=4e-2 * rms(want)) if dtype == "bf16" else tol  # re-rounded once per partition
+    # bf16 `out` is re-rounded after every partition: up to one bf16 ulp of the running sum per step
+    tol_k = dict(rtol=4e-2, atol=4 * 2.0 ** -8 * float(np.abs(want).max())) if dtype == "bf16" else tol
     allclose_report(out.float().cpu().numpy(), want, what="spmm K=4", **tol_k)
 
 
