@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the fused GAT aggregation (forward + backward with attention rematerialisation).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+One STEP is one pass of the whole hot path over one batch of synthetic node tensors: for each of
+the workload's layers the fused forward over the K source partitions, then for each layer the
+rematerialising backward (destination-major and source-major passes).  The graph (CSR, CSC,
+long-row plan) is prepared once by the library before the timed region and its time is reported
+as `prep_ms`; a graph is fixed across the training steps the paper times (its partitioning is an
+offline step).
+
+Prints ONE JSON line (rank 0).  `value` = edges x layers processed per second by all ranks (each
+rank runs an independent replica: the path does not shard, so scaling is "weak" with no
+collective on the data path).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "gat_fwd_bwd_edges_per_sec"
+UNIT = "edges/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large", help="tiny | seqpart | medium | dense | large")
+    ap.add_argument("--dtype", default=None, help="f32 | bf16 (default: the workload's last listed dtype)")
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (debugging only)")
+    ap.add_argument("--threshold", type=int, default=None, help="long-row split threshold")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample", type=float, default=0.05, help="fraction of the workload the oracle is timed on")
+    return ap.parse_args()
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+# --------------------------------------------------------------------------------------------------
+# algorithmic (compulsory) bytes: every distinct input byte read once, every output byte written once
+# --------------------------------------------------------------------------------------------------
+
+def idx_bytes(n, e):
+    return 8 * (n + 1) + 4 * e
+
+
+def bytes_fwd(n, e, H, F, b):
+    return idx_bytes(n, e) + 2 * n * H * F * b + 4 * n * H * 4          # feat, out; el, er, m, d
+
+
+def bytes_bwd_dst(n, e, H, F, b):
+    # CSR, gathered feat, gout row; el, er, m, d read; del and the 16-byte record written
+    return idx_bytes(n, e) + 2 * n * H * F * b + 4 * n * H * 4 + n * H * 4 + n * H * 16
+
+
+def bytes_bwd_src(n, e, H, F, b):
+    # CSC, gathered gout, feat row, dfeat written; er and the record read; der written
+    return idx_bytes(n, e) + 3 * n * H * F * b + n * H * 4 + n * H * 16 + n * H * 4
+
+
+def bytes_layer_fwd_bwd(n, e, H, F, b):
+    # the whole layer, each array once: 3x index (CSR fwd, CSR + CSC bwd), feat, out, gout, dfeat,
+    # el, er, m, d (written then read), del, der
+    return 3 * idx_bytes(n, e) + 4 * n * H * F * b + 10 * n * H * 4
+
+
+KERNEL_BYTES = {"gat_fwd": bytes_fwd, "gat_bwd_dst": bytes_bwd_dst, "gat_bwd_src": bytes_bwd_src}
+
+
+# --------------------------------------------------------------------------------------------------
+# clocks
+# --------------------------------------------------------------------------------------------------
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.mktemp(prefix="clocks_", suffix=".csv")
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(gpu_index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()       # the exact child started above
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 7:
+                    continue
+                try:
+                    sm.append(float(f[0]))
+                    mx.append(float(f[1]))
+                except ValueError:
+                    continue
+                for nme, val in zip(names, f[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(nme)
+            os.unlink(self.path)
+        except OSError:
+            pass
+        if sm:
+            sm.sort()
+            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+# --------------------------------------------------------------------------------------------------
+# the CPU oracle as a timed baseline (reference arm and cpu_baseline leg)
+# --------------------------------------------------------------------------------------------------
+
+def oracle_sample(cfg, dtype, fraction):
+    """Inputs of a bounded sample of the workload for the oracle: the same recipe with node and edge
+    counts multiplied by `fraction`, one layer."""
+    import workloads
+    small = cfg.scaled(fraction) if fraction < 1.0 else cfg
+    src, dst = workloads.make_graph(small)
+    t = workloads.make_node_inputs(small.n, small.heads, small.feat, small.seed, dtype=dtype)
+    return small, src.numpy(), dst.numpy(), {k: v.float().numpy() for k, v in t.items()}
+
+
+def oracle_step(small, src, dst, h, slope):
+    """One layer forward + backward of the oracle as it stands (CSR given); returns seconds."""
+    import oracle
+    indptr, indices = oracle.csr_from_coo(small.n, small.n, src, dst)
+    t0 = time.perf_counter()
+    f = oracle.gat_fwd(indptr, indices, h["feat"], h["el"], h["er"], slope)
+    oracle.gat_bwd(indptr, indices, h["feat"], h["el"], h["er"], f.alpha, h["gout"], slope)
+    return time.perf_counter() - t0
+
+
+def run_reference(args, rank):
+    """--impl reference: the oracle, as it stands, on the host cores, on a bounded sample."""
+    if rank != 0:
+        return
+    import oracle
+    import workloads
+    cfg = workloads.CONFIGS[args.workload]
+    dtype = args.dtype or cfg.dtypes[-1]
+    # a smaller sample than the cpu_baseline leg: warmup + steps passes must end within minutes
+    small, src, dst, h = oracle_sample(cfg, dtype, min(1.0, 0.4 * args.cpu_sample * args.scale))
+    for _ in range(args.warmup):
+        oracle_step(small, src, dst, h, cfg.slope)
+    secs = [oracle_step(small, src, dst, h, cfg.slope) for _ in range(args.steps)]
+    total = sum(secs)
+    value = small.e * args.steps / total
+    sample = f"{small.name}: n={small.n} e={small.e} H={small.heads} F={small.feat}, one layer fwd+bwd per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, "sample": sample, "storage_dtype": dtype},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# --------------------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------------------
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import workloads
+    from paper_2111_06483_b200 import api, binding as B
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    dev = torch.device(f"cuda:{local_rank}")
+    torch.cuda.set_device(dev)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = workloads.CONFIGS[args.workload]
+    if args.scale != 1.0:
+        cfg = cfg.scaled(args.scale)
+    dtype = args.dtype or cfg.dtypes[-1]
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    b = 2 if dtype == "bf16" else 4
+    n, H, F, L, K = cfg.n, cfg.heads, cfg.feat, cfg.layers, cfg.k
+    threshold = args.threshold if args.threshold is not None else api.DEFAULT_THRESHOLD
+
+    # ---- inputs (seeded, generated on the device; same recipe as the parity tests) --------------
+    src, dst = workloads.make_graph(cfg, device=dev)
+    e = src.numel()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    g = api.Graph.from_coo(n, src, dst, k=K, threshold=threshold)
+    torch.cuda.synchronize()
+    prep_ms = 1e3 * (time.perf_counter() - t0)
+    del src, dst
+    feats = [workloads.normal_tensor((n, H, F), cfg.seed, 10, device=dev, dtype=tdt)]
+    feats += [torch.empty((n, H, F), dtype=tdt, device=dev) for _ in range(L)]
+    els = [workloads.normal_tensor((n, H), cfg.seed, 16 * l + 12, device=dev) for l in range(L)]
+    ers = [workloads.normal_tensor((n, H), cfg.seed, 16 * l + 13, device=dev) for l in range(L)]
+    gout = workloads.normal_tensor((n, H, F), cfg.seed, 11, device=dev, dtype=tdt)
+    gbuf = [torch.empty((n, H, F), dtype=tdt, device=dev) for _ in range(2)]
+    ms = [torch.empty((n, H), dtype=torch.float32, device=dev) for _ in range(L)]
+    ds = [torch.empty((n, H), dtype=torch.float32, device=dev) for _ in range(L)]
+    dels = [torch.empty((n, H), dtype=torch.float32, device=dev) for _ in range(L)]
+    ders = [torch.empty((n, H), dtype=torch.float32, device=dev) for _ in range(L)]
+    ws = api.gat_workspace(g.whole, H, F, tdt)
+    cut = lambda t: [t[g.bounds[q]:] for q in range(K)]
+    feat_q = [cut(f) for f in feats]
+    er_q = [cut(x) for x in ers]
+    der_q = [cut(x) for x in ders]
+    gbuf_q = [cut(x) for x in gbuf]
+
+    def step():
+        for l in range(L):
+            B.sar_gat_fwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], H, F, cfg.slope, ms[l], ds[l],
+                                feats[l + 1], ws)
+        gin = gout
+        for i, l in enumerate(reversed(range(L))):
+            B.sar_gat_bwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], ms[l], ds[l], gin, H, F, cfg.slope,
+                                gbuf_q[i % 2], dels[l], der_q[l], ws)
+            gin = gbuf[i % 2]
+
+    torch.cuda.reset_peak_memory_stats()
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    peak_mem = torch.cuda.max_memory_allocated()
+
+    # ---- timed region ----------------------------------------------------------------------------
+    gpu_index = int(os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",")[local_rank]) \
+        if os.environ.get("CUDA_VISIBLE_DEVICES", "").replace(",", "").isdigit() else local_rank
+    sampler = ClockSampler(gpu_index) if rank == 0 else None
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with B.LaunchTimer() as lt:
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    elapsed_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else {}
+    if dist:
+        tmax = torch.tensor([elapsed_ms], device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(tmax.item())
+    kernels = lt.summary()
+    launches = sum(v["launches"] for v in kernels.values())
+    ms_per_step = elapsed_ms / args.steps
+    value = world * L * e / (ms_per_step * 1e-3)
+
+    # ---- roofline of the dominant kernel -----------------------------------------------------------
+    peak, peak_src = load_peaks()
+    dom = max(kernels, key=lambda k_: kernels[k_]["total_ms"])
+    fn = KERNEL_BYTES.get(dom)
+    roofline = None
+    if fn:
+        alg = fn(n, e, H, F, b)
+        achieved = alg / (kernels[dom]["avg_ms"] * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
+                    "algorithmic_bytes_per_launch": alg, "avg_launch_ms": kernels[dom]["avg_ms"]}
+    step_bytes = L * bytes_layer_fwd_bwd(n, e, H, F, b)
+    step_frac = step_bytes / (ms_per_step * 1e-3) / 1e9 / peak
+
+    # ---- end to end through the host-buffer entry point ---------------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        del feats, gbuf, feat_q, gbuf_q, gout
+        torch.cuda.empty_cache()
+        pin = lambda shape, dt: torch.empty(shape, dtype=dt).pin_memory()
+        h_feat0 = pin((n, H, F), tdt)
+        h_gout = pin((n, H, F), tdt)
+        h_out, h_dfeat = pin((n, H, F), tdt), pin((n, H, F), tdt)
+        h_el = [pin((n, H), torch.float32) for _ in range(L)]
+        h_er = [pin((n, H), torch.float32) for _ in range(L)]
+        h_del = [pin((n, H), torch.float32) for _ in range(L)]
+        h_der = [pin((n, H), torch.float32) for _ in range(L)]
+        h_feat0.copy_(workloads.normal_tensor((n, H, F), cfg.seed, 10, device=dev, dtype=tdt))
+        h_gout.copy_(workloads.normal_tensor((n, H, F), cfg.seed, 11, device=dev, dtype=tdt))
+        for l in range(L):
+            h_el[l].copy_(els[l])
+            h_er[l].copy_(ers[l])
+        arena = torch.empty(B.sar_gat_stack_arena_bytes(g.whole, L, H, F, B._dtype(h_feat0)), dtype=torch.uint8,
+                            device=dev)
+
+        def host_step():
+            B.sar_gat_stack_host(g.whole, g.bounds, H, F, cfg.slope, h_feat0, h_el, h_er, h_gout, h_out, h_dfeat,
+                                 h_del, h_der, arena)
+
+        host_step()
+        torch.cuda.synchronize()
+        n_e2e = max(1, min(args.steps, 3))
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            host_step()
+        torch.cuda.synchronize()
+        dt = time.perf_counter() - t0
+        if dist:
+            tmax = torch.tensor([dt], device=dev)
+            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+            dt = float(tmax.item())
+        h2d = 2 * n * H * F * b + 2 * L * n * H * 4
+        d2h = 2 * n * H * F * b + 2 * L * n * H * 4
+        e2e = {"value": world * L * e * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+               "ms_per_step": 1e3 * dt / n_e2e, "steps": n_e2e, "entry_point": "sar_gat_stack_host"}
+
+    # ---- the oracle on the host cores, bounded sample ------------------------------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        small, s_src, s_dst, h = oracle_sample(workloads.CONFIGS[args.workload], dtype,
+                                               min(1.0, args.cpu_sample * args.scale))
+        secs = oracle_step(small, s_src, s_dst, h, cfg.slope)
+        cpu = {"value": small.e / secs, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": f"{small.name}: n={small.n} e={small.e} H={small.heads} F={small.feat}, one layer fwd+bwd, "
+                         f"{secs:.1f} s"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {
+                "workload": cfg.name, "n": n, "e": e, "heads": H, "feat_per_head": F, "layers": L, "partitions": K,
+                "storage_dtype": dtype, "schedule": "fused row-stationary (sar_gat_fwd_fused / sar_gat_bwd_fused)",
+                "l2": "inputs_exceed_l2", "long_row_threshold": threshold, "parallelism": f"replicas x{world}",
+                "edges_x_heads_x_feat_per_sec": value * H * F,
+            },
+            "roofline": roofline,
+            "step_roofline": {"compulsory_bytes_per_step": step_bytes, "frac_of_peak": step_frac, "peak": peak,
+                              "peak_source": peak_src},
+            "kernels": kernels, "gpu_launches": launches, "prep_ms": prep_ms,
+            "peak_mem_bytes": peak_mem, "attention_bytes_if_stored": L * e * H * 4,
+            "stats_bytes_kept": L * 2 * n * H * 4,
+            "clocks": clocks, "e2e": e2e, "cpu_baseline": cpu,
+        }
+        print(json.dumps(line), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()

@@ -104,6 +104,14 @@ SAR_API const char *sar_status_string(sar_status s);
 /* Compile-time facts: returns the SM architecture the kernels were built for (100). */
 SAR_API int32_t sar_built_for_sm(void);
 
+/* Optional observer of the library's kernel launches, for profiling: when set, `hook` is called on
+ * the launching host thread right before (phase 0) and right after (phase 1) each kernel launch
+ * of the aggregation entry points, with the kernel's name and the stream, so that a caller can
+ * record events around individual kernels.  Process-global and not thread-safe; NULL disables
+ * it (the default).  The paper has no counterpart; this is measurement plumbing. */
+typedef void (*sar_launch_hook_fn)(const char *kernel, int32_t phase, void *stream, void *user);
+SAR_API void sar_set_launch_hook(sar_launch_hook_fn hook, void *user);
+
 /* ---------------------------------------------------------------------------------------------
  * Graph preparation (construction of the subgraphs G_{p,q}, Sec. 3.2).  Integer work; results
  * are unique and therefore bit-reproducible.
@@ -237,6 +245,39 @@ SAR_API sar_status sar_spmm_agg(const sar_part *g, const void *feat_q, int32_t F
                         const int64_t *deg_total, void *out, void *workspace, size_t workspace_bytes,
                         void *stream);
 SAR_API size_t sar_spmm_workspace_bytes(const sar_part *g, int32_t F, sar_dtype t);
+
+/* ---------------------------------------------------------------------------------------------
+ * A stack of L aggregation layers with HOST buffers (the 3-layer GAT of the paper's Sec. 4.2 reduced
+ * to its aggregation steps): layer l computes out^l from feat^l = out^(l-1) (feat^0 given) with its
+ * own el^l, er^l; the backward pass feeds dfeat^(l+1) as gout of layer l.  All copies and kernels
+ * are enqueued on `stream` in order: host->device of the inputs, L fused forwards, L fused
+ * backwards, device->host of the results.  Returns without synchronising; use pinned host memory
+ * for the copies to be asynchronous.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    int32_t L, H, F;
+    sar_dtype t;
+    float slope;
+    /* HOST inputs */
+    const void *feat0;        /* [n,H,F] type t                                          */
+    const float *const *el;   /* HOST array of L HOST pointers, each [n,H]               */
+    const float *const *er;   /* idem                                                    */
+    const void *gout;         /* [n,H,F] type t: gradient w.r.t. the last layer's output */
+    /* HOST outputs (any may be NULL to skip its copy) */
+    void *out_last;           /* [n,H,F] type t                                          */
+    void *dfeat0;             /* [n,H,F] type t                                          */
+    float *const *del;        /* HOST array of L HOST pointers, each [n,H], or NULL      */
+    float *const *der;        /* idem                                                    */
+} sar_stack_host_io;
+
+/* DEVICE bytes sar_gat_stack_host needs in `arena` for this graph and shape. */
+SAR_API size_t sar_gat_stack_arena_bytes(const sar_part *g, int32_t L, int32_t H, int32_t F, sar_dtype t);
+
+/* `g` is the un-split graph (DEVICE arrays), partitions as in sar_gat_fwd_fused; `arena` is DEVICE
+ * scratch of at least sar_gat_stack_arena_bytes, 256-byte aligned. */
+SAR_API sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bounds,
+                                      const sar_stack_host_io *io, void *arena, size_t arena_bytes,
+                                      void *stream);
 
 #ifdef __cplusplus
 }

@@ -26,7 +26,8 @@ EXPORTS = [
     "sar_status_string", "sar_built_for_sm", "sar_graph_workspace_bytes", "sar_csr_from_coo", "sar_csr_transpose",
     "sar_partition_bounds", "sar_csr_split_indptr", "sar_csr_split_indices", "sar_validate_part", "sar_plan_count",
     "sar_plan_fill", "sar_gat_workspace_bytes", "sar_gat_fwd", "sar_gat_fwd_fused", "sar_gat_bwd_prepare",
-    "sar_gat_bwd", "sar_gat_bwd_fused", "sar_spmm_agg", "sar_spmm_workspace_bytes",
+    "sar_gat_bwd", "sar_gat_bwd_fused", "sar_spmm_agg", "sar_spmm_workspace_bytes", "sar_set_launch_hook",
+    "sar_gat_stack_arena_bytes", "sar_gat_stack_host",
 ]
 
 
@@ -62,7 +63,8 @@ def lib() -> ctypes.CDLL:
         L.sar_status_string.restype = c_char_p
         L.sar_status_string.argtypes = [ctypes.c_int]
         L.sar_built_for_sm.restype = c_int32
-        for name in ("sar_graph_workspace_bytes", "sar_gat_workspace_bytes", "sar_spmm_workspace_bytes"):
+        for name in ("sar_graph_workspace_bytes", "sar_gat_workspace_bytes", "sar_spmm_workspace_bytes",
+                     "sar_gat_stack_arena_bytes"):
             getattr(L, name).restype = c_size_t
         _lib = L
     return _lib
@@ -129,6 +131,61 @@ class Part:
         assert self.t_indptr is not None
         return Part(self.n_src, self.n_dst, self.t_indptr, self.t_indices, self.indptr, self.indices,
                     self.t_split, self.split, nnz=self.nnz)
+
+
+# ----------------------------------------------------------------------------------------------
+# launch observer
+# ----------------------------------------------------------------------------------------------
+
+_HOOK_T = ctypes.CFUNCTYPE(None, c_char_p, c_int32, c_void_p, c_void_p)
+_hook_keepalive = None
+
+
+def sar_set_launch_hook(fn) -> None:
+    """fn(kernel_name: str, phase: int) is called before (0) and after (1) every kernel launch of the
+    aggregation entry points; None removes the observer."""
+    global _hook_keepalive
+    if fn is None:
+        lib().sar_set_launch_hook(None, None)
+        _hook_keepalive = None
+        return
+    cb = _HOOK_T(lambda name, phase, stream, user: fn(name.decode(), int(phase)))
+    lib().sar_set_launch_hook(cb, None)
+    _hook_keepalive = cb
+
+
+class LaunchTimer:
+    """Context manager: CUDA events around every kernel launch inside the block, on the current
+    stream.  After the block (and a synchronize) `summary()` gives per-kernel launch counts and
+    device times."""
+
+    def __init__(self):
+        self.records = []   # (name, start_event, end_event)
+        self._open = {}
+
+    def _hook(self, name, phase):
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record()
+        if phase == 0:
+            self._open[name] = ev
+        else:
+            self.records.append((name, self._open.pop(name), ev))
+
+    def __enter__(self):
+        sar_set_launch_hook(self._hook)
+        return self
+
+    def __exit__(self, *exc):
+        sar_set_launch_hook(None)
+        return False
+
+    def summary(self):
+        torch.cuda.synchronize()
+        agg = {}
+        for name, e0, e1 in self.records:
+            n, ms = agg.get(name, (0, 0.0))
+            agg[name] = (n + 1, ms + e0.elapsed_time(e1))
+        return {k: {"launches": n, "total_ms": ms, "avg_ms": ms / n} for k, (n, ms) in agg.items()}
 
 
 # ----------------------------------------------------------------------------------------------
@@ -280,3 +337,45 @@ def sar_spmm_agg(part: Part, feat_q: torch.Tensor, F: int, flags: int, deg_total
     w, wb = _ws(workspace)
     _check("sar_spmm_agg", lib().sar_spmm_agg(byref(part.c), _ptr(feat_q), c_int32(F), ctypes.c_int(_dtype(feat_q)),
                                               c_uint32(flags), _ptr(deg_total), _ptr(out), w, wb, _stream()))
+
+
+# ----------------------------------------------------------------------------------------------
+# host-buffer stack
+# ----------------------------------------------------------------------------------------------
+
+class sar_stack_host_io(Structure):
+    _fields_ = [("L", c_int32), ("H", c_int32), ("F", c_int32), ("t", ctypes.c_int), ("slope", c_float),
+                ("feat0", c_void_p), ("el", POINTER(c_void_p)), ("er", POINTER(c_void_p)), ("gout", c_void_p),
+                ("out_last", c_void_p), ("dfeat0", c_void_p), ("del_", POINTER(c_void_p)), ("der", POINTER(c_void_p))]
+
+
+def sar_gat_stack_arena_bytes(part: Part, L: int, H: int, F: int, dtype: int) -> int:
+    return int(lib().sar_gat_stack_arena_bytes(byref(part.c), c_int32(L), c_int32(H), c_int32(F), ctypes.c_int(dtype)))
+
+
+def _host_ptr(t: Optional[torch.Tensor]):
+    if t is None:
+        return None
+    assert (not t.is_cuda) and t.is_contiguous(), "host buffers are contiguous CPU tensors (pin them for async copies)"
+    return t.data_ptr()
+
+
+def _host_ptr_array(ts):
+    if ts is None:
+        return None
+    return (c_void_p * len(ts))(*[_host_ptr(t) for t in ts])
+
+
+def sar_gat_stack_host(part: Part, bounds: Sequence[int], H: int, F: int, slope: float, feat0: torch.Tensor,
+                       el: Sequence[torch.Tensor], er: Sequence[torch.Tensor], gout: torch.Tensor,
+                       out_last: Optional[torch.Tensor], dfeat0: Optional[torch.Tensor],
+                       del_: Optional[Sequence[torch.Tensor]], der: Optional[Sequence[torch.Tensor]],
+                       arena: torch.Tensor) -> None:
+    """L = len(el) chained aggregation layers, fwd + bwd, all node tensors in HOST memory."""
+    L = len(el)
+    io = sar_stack_host_io(L, H, F, _dtype(feat0), slope, _host_ptr(feat0), _host_ptr_array(el), _host_ptr_array(er),
+                           _host_ptr(gout), _host_ptr(out_last), _host_ptr(dfeat0), _host_ptr_array(del_),
+                           _host_ptr_array(der))
+    w, wb = _ws(arena)
+    _check("sar_gat_stack_host", lib().sar_gat_stack_host(byref(part.c), c_int32(len(bounds) - 1), _host_i64(bounds),
+                                                          byref(io), w, wb, _stream()))

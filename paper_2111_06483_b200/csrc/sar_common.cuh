@@ -42,6 +42,28 @@ static inline size_t sar_elem_size(sar_dtype t) { return t == SAR_BF16 ? 2 : 4; 
 
 #define SAR_NEG_INF (-INFINITY)
 
+// launch observer (sar_set_launch_hook)
+namespace sar {
+extern sar_launch_hook_fn g_launch_hook;
+extern void *g_launch_hook_user;
+struct LaunchScope {
+    const char *name;
+    cudaStream_t st;
+    LaunchScope(const char *n, cudaStream_t s) : name(n), st(s) {
+        if (g_launch_hook) g_launch_hook(name, 0, st, g_launch_hook_user);
+    }
+    ~LaunchScope() {
+        if (g_launch_hook) g_launch_hook(name, 1, st, g_launch_hook_user);
+    }
+};
+}  // namespace sar
+// SAR_LAUNCH("name", stream, kernel<<<...>>>(args));
+#define SAR_LAUNCH(name, st, ...)            \
+    do {                                     \
+        sar::LaunchScope scope__(name, st);  \
+        __VA_ARGS__;                         \
+    } while (0)
+
 namespace sar {
 
 constexpr int kWarpsPerBlock = 8;

@@ -1,9 +1,13 @@
 // C-ABI entry points of the fused GAT aggregation and of the sum aggregation: argument checks,
 // kernel selection and launches.  Declarations and contracts are in include/sar.h.
 #include "sar_gat_kernels.cuh"
+#include "sar_span_kernels.cuh"
 #include "sar_generic_kernels.cuh"
 
 namespace sar {
+
+sar_launch_hook_fn g_launch_hook = nullptr;
+void *g_launch_hook_user = nullptr;
 
 sar_status make_shape(int32_t H, int32_t F, sar_dtype t, bool ptrs_16B_aligned, Shape *out) {
     if (H < 1 || F < 1) return SAR_ERR_INVALID_ARG;
@@ -135,6 +139,44 @@ static sar_status check_elem_align(std::initializer_list<const void *> ps, size_
     return SAR_OK;
 }
 
+// ---- span kernels ---------------------------------------------------------------------------------
+constexpr int kCapFwd = 128, kCapDst = 128, kCapSrc = 128, kCapSum = 128;
+constexpr int kMinBlocksFwd = 4, kMinBlocksBwd = 3;  // resident blocks per SM the register budget is cut for
+
+static int rows_per_span(long long n_rows, long long nnz, int cap) {
+    const double avg = n_rows > 0 ? (double)nnz / (double)n_rows : 0.0;
+    int R = avg > 0.5 ? (int)(0.75 * cap / avg + 0.5) : kMaxSpanRows;  // about 3/4 cap edges per span
+    if (R < 1) R = 1;
+    if (R > kMaxSpanRows) R = kMaxSpanRows;
+    return R;
+}
+
+// Launches span_kernel<MODE> over the rows (mode 0) and, with a long-row plan, over the segments
+// (mode 1).  The merge launch is the caller's.
+template <typename T, int G, int V, int S, int MODE, int CAP, int MINB>
+static sar_status launch_span(SpanArgs a, long long nnz, const char *name, const char *seg_name, cudaStream_t st) {
+    auto kern = span_kernel<T, G, V, S, MODE, CAP, MINB>;
+    const size_t smem = (size_t)kSpanWarps * span_layout<MODE>(a.g.Hp, V, CAP, S, 32 / G).total;
+    SAR_TRY(ensure_smem(kern, smem));
+    a.mode = 0;
+    a.R = rows_per_span(a.n_rows, nnz, CAP);
+    const long long spans = (a.n_rows + a.R - 1) / a.R;
+    if (spans > 0) {
+        SAR_LAUNCH(name, st, kern<<<(unsigned)((spans + kSpanWarps - 1) / kSpanWarps), kSpanThreads, smem, st>>>(a));
+        SAR_TRY(sar_after_launch());
+    }
+    if (a.sp.threshold > 0 && a.sp.n_seg > 0) {
+        a.mode = 1;
+        SAR_LAUNCH(seg_name, st, kern<<<(unsigned)((a.sp.n_seg + kSpanWarps - 1) / kSpanWarps), kSpanThreads, smem, st>>>(a));
+        SAR_TRY(sar_after_launch());
+    }
+    return SAR_OK;
+}
+
+// stages of the gather ring: 16 x 512 bytes in flight per warp for one-vector rows
+template <int V> struct UFwd { static constexpr int u = V == 1 ? 16 : (V == 2 ? 8 : (V == 4 ? 4 : 2)); };
+template <int V> struct UBwd { static constexpr int u = V == 1 ? 16 : (V == 2 ? 8 : (V == 4 ? 4 : 2)); };
+
 }  // namespace sar
 
 using namespace sar;
@@ -152,6 +194,11 @@ const char *sar_status_string(sar_status s) {
         case SAR_ERR_BAD_GRAPH: return "inconsistent graph";
     }
     return "unknown status";
+}
+
+void sar_set_launch_hook(sar_launch_hook_fn hook, void *user) {
+    g_launch_hook = hook;
+    g_launch_hook_user = user;
 }
 
 int32_t sar_built_for_sm(void) {
@@ -211,9 +258,9 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
         const long long n = g->n_dst * H;
         const unsigned blocks = (unsigned)((n + 255) / 256);
         if (t == SAR_F32)
-            gat_fwd_generic<float><<<blocks, 256, 0, st>>>(a);
+            SAR_LAUNCH("gat_fwd_generic", st, gat_fwd_generic<float><<<blocks, 256, 0, st>>>(a));
         else
-            gat_fwd_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a);
+            SAR_LAUNCH("gat_fwd_generic", st, gat_fwd_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a));
         return sar_after_launch();
     }
 
@@ -224,37 +271,43 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
         if (!workspace || workspace_bytes < need || !sar_aligned(workspace, 16)) return SAR_ERR_WORKSPACE;
         part = reinterpret_cast<float *>(static_cast<char *>(workspace) + rec_bytes(g->n_dst, H));
     }
-    FwdArgs a;
-    a.n_dst = g->n_dst;
+    FwdArgs ma;  // arguments of the merge launch
+    ma.n_dst = g->n_dst;
+    ma.indptr = g->indptr;
+    ma.indices = g->indices;
+    ma.feat = feat_q;
+    ma.el = el;
+    ma.er = er_q;
+    ma.acc = acc;
+    ma.m = m;
+    ma.d = d;
+    ma.out = out;
+    ma.slope = slope;
+    ma.flags = flags;
+    ma.g = s.geom;
+    ma.sp = split_args(g->split, part, H, F, true);
+    ma.mode = 0;
+    SpanArgs a{};
+    a.n_rows = g->n_dst;
     a.indptr = g->indptr;
     a.indices = g->indices;
-    a.feat = feat_q;
+    a.gather = feat_q;
     a.el = el;
     a.er = er_q;
-    a.acc = acc;
-    a.m = m;
-    a.d = d;
+    a.acc_state = acc;
+    a.m_state = m;
+    a.d_state = d;
     a.out = out;
     a.slope = slope;
     a.flags = flags;
     a.g = s.geom;
-    a.sp = split_args(g->split, part, H, F, true);
-    a.mode = 0;
+    a.sp = ma.sp;
     return dispatch(s, [&](auto cfg) -> sar_status {
         using C = decltype(cfg);
         using T = typename C::type;
-        const size_t smem = (size_t)kWarpsPerBlock * warp_smem_floats(s.geom.Hp, C::v, 1) * 4;
-        auto kern = gat_fwd_kernel<T, C::g, C::v, C::u>;
-        SAR_TRY(ensure_smem(kern, smem));
-        FwdArgs b = a;
-        kern<<<blocks_for(g->n_dst, C::g), kThreads, smem, st>>>(b);
-        SAR_TRY(sar_after_launch());
-        if (b.sp.threshold > 0) {
-            b.mode = 1;
-            kern<<<blocks_for(b.sp.n_seg, C::g), kThreads, smem, st>>>(b);
-            SAR_TRY(sar_after_launch());
-            b.mode = 0;
-            gat_fwd_merge_kernel<T, C::g, C::v><<<blocks_for(b.sp.n_long, C::g), kThreads, 0, st>>>(b);
+        SAR_TRY((launch_span<T, C::g, C::v, UFwd<C::v>::u, kFwd, kCapFwd, kMinBlocksFwd>(a, g->nnz, "gat_fwd", "gat_fwd_seg", st)));
+        if (ma.sp.threshold > 0) {
+            SAR_LAUNCH("gat_fwd_merge", st, gat_fwd_merge_kernel<T, C::g, C::v><<<blocks_for(ma.sp.n_long, C::g), kThreads, 0, st>>>(ma));
             SAR_TRY(sar_after_launch());
         }
         return SAR_OK;
@@ -323,9 +376,9 @@ sar_status sar_gat_bwd_prepare(int64_t n_dst, int32_t H, int32_t F, sar_dtype t,
         a.acc_is_numerator = acc_is_numerator;
         const unsigned blocks = (unsigned)((n_dst * H + 255) / 256);
         if (t == SAR_F32)
-            gat_bwd_prepare_generic<float><<<blocks, 256, 0, st>>>(a);
+            SAR_LAUNCH("gat_bwd_prepare_generic", st, gat_bwd_prepare_generic<float><<<blocks, 256, 0, st>>>(a));
         else
-            gat_bwd_prepare_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a);
+            SAR_LAUNCH("gat_bwd_prepare_generic", st, gat_bwd_prepare_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a));
         return sar_after_launch();
     }
     PrepArgs a;
@@ -343,7 +396,7 @@ sar_status sar_gat_bwd_prepare(int64_t n_dst, int32_t H, int32_t F, sar_dtype t,
         using C = decltype(cfg);
         using T = typename C::type;
         const size_t smem = (size_t)kWarpsPerBlock * 32 * C::v * 4;
-        gat_bwd_prepare_kernel<T, C::g, C::v><<<blocks_for(n_dst, C::g), kThreads, smem, st>>>(a);
+        SAR_LAUNCH("gat_bwd_prepare", st, gat_bwd_prepare_kernel<T, C::g, C::v><<<blocks_for(n_dst, C::g), kThreads, smem, st>>>(a));
         return sar_after_launch();
     });
 }
@@ -395,23 +448,23 @@ sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, c
         if (g->n_dst > 0) {
             const unsigned blocks = (unsigned)((g->n_dst * H + 255) / 256);
             if (t == SAR_F32)
-                gat_bwd_dst_generic<float><<<blocks, 256, 0, st>>>(a);
+                SAR_LAUNCH("gat_bwd_dst_generic", st, gat_bwd_dst_generic<float><<<blocks, 256, 0, st>>>(a));
             else
-                gat_bwd_dst_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a);
+                SAR_LAUNCH("gat_bwd_dst_generic", st, gat_bwd_dst_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a));
             SAR_TRY(sar_after_launch());
         }
         if (g->n_src > 0) {
             const unsigned blocks = (unsigned)((g->n_src * H + 255) / 256);
             if (t == SAR_F32)
-                gat_bwd_src_generic<float><<<blocks, 256, 0, st>>>(a);
+                SAR_LAUNCH("gat_bwd_src_generic", st, gat_bwd_src_generic<float><<<blocks, 256, 0, st>>>(a));
             else
-                gat_bwd_src_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a);
+                SAR_LAUNCH("gat_bwd_src_generic", st, gat_bwd_src_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a));
             SAR_TRY(sar_after_launch());
         }
         return SAR_OK;
     }
 
-    BwdDstArgs da;
+    BwdDstArgs da;  // merge launches
     da.n_dst = g->n_dst;
     da.indptr = g->indptr;
     da.indices = g->indices;
@@ -442,48 +495,68 @@ sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, c
     sa.g = s.geom;
     sa.sp = split_args(g->t_split, part_csc, H, F, true);
     sa.mode = 0;
+    SpanArgs d1{};  // destination-major pass over the CSR
+    d1.n_rows = g->n_dst;
+    d1.indptr = g->indptr;
+    d1.indices = g->indices;
+    d1.gather = feat_q;
+    d1.rowvec = gout;
+    d1.el = el;
+    d1.er = er_q;
+    d1.m = m;
+    d1.d = d;
+    d1.rec_in = rec;
+    d1.rec_out = rec;
+    d1.del = del;
+    d1.slope = slope;
+    d1.flags = flags;
+    d1.g = s.geom;
+    d1.sp = da.sp;
+    SpanArgs s1{};  // source-major pass over the CSC
+    s1.n_rows = g->n_src;
+    s1.indptr = g->t_indptr;
+    s1.indices = g->t_indices;
+    s1.gather = gout;
+    s1.rowvec = feat_q;
+    s1.er = er_q;
+    s1.rec_in = rec;
+    s1.out = dfeat_q;
+    s1.der = der_q;
+    s1.slope = slope;
+    s1.flags = flags;
+    s1.g = s.geom;
+    s1.sp = sa.sp;
 
     return dispatch(s, [&](auto cfg) -> sar_status {
         using C = decltype(cfg);
         using T = typename C::type;
+        constexpr int U = UBwd<C::v>::u;
+        const size_t msmem = (size_t)kWarpsPerBlock * warp_smem_floats(s.geom.Hp, C::v, 4) * 4;
         if (g->n_dst > 0) {
-            const size_t smem = (size_t)kWarpsPerBlock * warp_smem_floats(s.geom.Hp, C::v, 2) * 4;
-            auto run = [&](auto kern, auto merge) -> sar_status {
-                SAR_TRY(ensure_smem(kern, smem));
-                SAR_TRY(ensure_smem(merge, smem));
-                BwdDstArgs b = da;
-                kern<<<blocks_for(g->n_dst, C::g), kThreads, smem, st>>>(b);
-                SAR_TRY(sar_after_launch());
-                if (b.sp.threshold > 0) {
-                    b.mode = 1;
-                    kern<<<blocks_for(b.sp.n_seg, C::g), kThreads, smem, st>>>(b);
-                    SAR_TRY(sar_after_launch());
-                    b.mode = 0;
-                    merge<<<blocks_for(b.sp.n_long, C::g), kThreads, smem, st>>>(b);
+            if (whole) {
+                SAR_TRY((launch_span<T, C::g, C::v, U, kBwdDst, kCapDst, kMinBlocksBwd>(d1, g->nnz, "gat_bwd_dst", "gat_bwd_dst_seg", st)));
+                if (da.sp.threshold > 0) {
+                    auto merge = gat_bwd_dst_merge_kernel<T, C::g, C::v, false>;
+                    SAR_TRY(ensure_smem(merge, msmem));
+                    SAR_LAUNCH("gat_bwd_dst_merge", st, merge<<<blocks_for(da.sp.n_long, C::g), kThreads, msmem, st>>>(da));
                     SAR_TRY(sar_after_launch());
                 }
-                return SAR_OK;
-            };
-            if (whole)
-                SAR_TRY(run(gat_bwd_dst_kernel<T, C::g, C::v, C::u, false>, gat_bwd_dst_merge_kernel<T, C::g, C::v, false>));
-            else
-                SAR_TRY(run(gat_bwd_dst_kernel<T, C::g, C::v, C::u, true>, gat_bwd_dst_merge_kernel<T, C::g, C::v, true>));
+            } else {
+                SAR_TRY((launch_span<T, C::g, C::v, U, kBwdDstGivenD, kCapDst, kMinBlocksBwd>(d1, g->nnz, "gat_bwd_dst", "gat_bwd_dst_seg", st)));
+                if (da.sp.threshold > 0) {
+                    auto merge = gat_bwd_dst_merge_kernel<T, C::g, C::v, true>;
+                    SAR_TRY(ensure_smem(merge, msmem));
+                    SAR_LAUNCH("gat_bwd_dst_merge", st, merge<<<blocks_for(da.sp.n_long, C::g), kThreads, msmem, st>>>(da));
+                    SAR_TRY(sar_after_launch());
+                }
+            }
         }
         if (g->n_src > 0) {
-            const size_t smem = (size_t)kWarpsPerBlock * warp_smem_floats(s.geom.Hp, C::v, 4) * 4;
-            auto kern = gat_bwd_src_kernel<T, C::g, C::v, C::u>;
-            auto merge = gat_bwd_src_merge_kernel<T, C::g, C::v>;
-            SAR_TRY(ensure_smem(kern, smem));
-            SAR_TRY(ensure_smem(merge, smem));
-            BwdSrcArgs b = sa;
-            kern<<<blocks_for(g->n_src, C::g), kThreads, smem, st>>>(b);
-            SAR_TRY(sar_after_launch());
-            if (b.sp.threshold > 0) {
-                b.mode = 1;
-                kern<<<blocks_for(b.sp.n_seg, C::g), kThreads, smem, st>>>(b);
-                SAR_TRY(sar_after_launch());
-                b.mode = 0;
-                merge<<<blocks_for(b.sp.n_long, C::g), kThreads, smem, st>>>(b);
+            SAR_TRY((launch_span<T, C::g, C::v, U, kBwdSrc, kCapSrc, kMinBlocksBwd>(s1, g->nnz, "gat_bwd_src", "gat_bwd_src_seg", st)));
+            if (sa.sp.threshold > 0) {
+                auto merge = gat_bwd_src_merge_kernel<T, C::g, C::v>;
+                SAR_TRY(ensure_smem(merge, msmem));
+                SAR_LAUNCH("gat_bwd_src_merge", st, merge<<<blocks_for(sa.sp.n_long, C::g), kThreads, msmem, st>>>(sa));
                 SAR_TRY(sar_after_launch());
             }
         }
@@ -536,38 +609,41 @@ sar_status sar_spmm_agg(const sar_part *g, const void *feat_q, int32_t F, sar_dt
         a.flags = flags;
         const unsigned blocks = (unsigned)((g->n_dst * F + 255) / 256);
         if (t == SAR_F32)
-            spmm_generic<float><<<blocks, 256, 0, st>>>(a);
+            SAR_LAUNCH("spmm_generic", st, spmm_generic<float><<<blocks, 256, 0, st>>>(a));
         else
-            spmm_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a);
+            SAR_LAUNCH("spmm_generic", st, spmm_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a));
         return sar_after_launch();
     }
     const bool use_split = g->split && g->split->n_long > 0;
     if (use_split && (!workspace || !sar_aligned(workspace, 16) || workspace_bytes < part_bytes(g->split, 1, F)))
         return SAR_ERR_WORKSPACE;
-    SumArgs a;
-    a.n_dst = g->n_dst;
+    SumArgs ma;  // merge launch
+    ma.n_dst = g->n_dst;
+    ma.indptr = g->indptr;
+    ma.indices = g->indices;
+    ma.feat = feat_q;
+    ma.out = out;
+    ma.deg_total = deg_total;
+    ma.flags = flags;
+    ma.g = s.geom;
+    ma.sp = split_args(g->split, static_cast<float *>(workspace), 1, F, true);
+    ma.mode = 0;
+    SpanArgs a{};
+    a.n_rows = g->n_dst;
     a.indptr = g->indptr;
     a.indices = g->indices;
-    a.feat = feat_q;
+    a.gather = feat_q;
     a.out = out;
     a.deg_total = deg_total;
     a.flags = flags;
     a.g = s.geom;
-    a.sp = split_args(g->split, static_cast<float *>(workspace), 1, F, true);
-    a.mode = 0;
+    a.sp = ma.sp;
     return dispatch(s, [&](auto cfg) -> sar_status {
         using C = decltype(cfg);
         using T = typename C::type;
-        const size_t smem = (size_t)kWarpsPerBlock * 32 * 4;
-        SumArgs b = a;
-        spmm_kernel<T, C::g, C::v, C::u><<<blocks_for(g->n_dst, C::g), kThreads, smem, st>>>(b);
-        SAR_TRY(sar_after_launch());
-        if (b.sp.threshold > 0) {
-            b.mode = 1;
-            spmm_kernel<T, C::g, C::v, C::u><<<blocks_for(b.sp.n_seg, C::g), kThreads, smem, st>>>(b);
-            SAR_TRY(sar_after_launch());
-            b.mode = 0;
-            spmm_merge_kernel<T, C::g, C::v><<<blocks_for(b.sp.n_long, C::g), kThreads, 0, st>>>(b);
+        SAR_TRY((launch_span<T, C::g, C::v, UFwd<C::v>::u, kSum, kCapSum, kMinBlocksFwd>(a, g->nnz, "spmm", "spmm_seg", st)));
+        if (ma.sp.threshold > 0) {
+            SAR_LAUNCH("spmm_merge", st, spmm_merge_kernel<T, C::g, C::v><<<blocks_for(ma.sp.n_long, C::g), kThreads, 0, st>>>(ma));
             SAR_TRY(sar_after_launch());
         }
         return SAR_OK;

@@ -1,0 +1,117 @@
+// Host-buffer entry point: a stack of aggregation layers with the copies inside the call.
+// Contracts are in include/sar.h.
+#include <vector>
+
+#include "sar_common.cuh"
+
+namespace {
+
+struct Arena {
+    char *base;
+    size_t used, cap;
+    void *take(size_t bytes) {
+        const size_t b = sar_round_up(bytes, 256);
+        if (used + b > cap) return nullptr;
+        void *p = base + used;
+        used += b;
+        return p;
+    }
+};
+
+size_t stack_bytes(const sar_part *g, int32_t L, int32_t H, int32_t F, sar_dtype t) {
+    const size_t n = (size_t)g->n_dst;
+    const size_t row = sar_round_up(n * H * F * sar_elem_size(t), 256);
+    const size_t nh = sar_round_up(n * H * 4, 256);
+    return (size_t)(L + 1) * row + 2 * row + (size_t)L * 6 * nh + sar_round_up(sar_gat_workspace_bytes(g, H, F, t), 256) + 256;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t sar_gat_stack_arena_bytes(const sar_part *g, int32_t L, int32_t H, int32_t F, sar_dtype t) {
+    if (!g || L < 1 || H < 1 || F < 1) return 0;
+    return stack_bytes(g, L, H, F, t);
+}
+
+sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bounds, const sar_stack_host_io *io,
+                              void *arena, size_t arena_bytes, void *stream) {
+    if (!g || !io || !bounds || k < 1) return SAR_ERR_INVALID_ARG;
+    const int32_t L = io->L, H = io->H, F = io->F;
+    if (L < 1 || L > 64 || H < 1 || F < 1) return SAR_ERR_INVALID_ARG;
+    if (g->n_dst != g->n_src) return SAR_ERR_INVALID_ARG;  // layers chain: outputs become inputs
+    if (!io->feat0 || !io->el || !io->er || !io->gout) return SAR_ERR_INVALID_ARG;
+    for (int l = 0; l < L; ++l)
+        if (!io->el[l] || !io->er[l] || (io->del && !io->del[l]) || (io->der && !io->der[l])) return SAR_ERR_INVALID_ARG;
+    if (!arena || !sar_aligned(arena, 256) || arena_bytes < stack_bytes(g, L, H, F, io->t)) return SAR_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t n = (size_t)g->n_dst;
+    const size_t row_b = n * H * F * sar_elem_size(io->t), nh_b = n * H * 4;
+
+    Arena a{static_cast<char *>(arena), 0, arena_bytes};
+    std::vector<void *> feat(L + 1);
+    std::vector<float *> el(L), er(L), m(L), d(L), del(L), der(L);
+    for (int l = 0; l <= L; ++l) feat[l] = a.take(row_b);
+    void *ga = a.take(row_b), *gb = a.take(row_b);
+    for (int l = 0; l < L; ++l) {
+        el[l] = static_cast<float *>(a.take(nh_b));
+        er[l] = static_cast<float *>(a.take(nh_b));
+        m[l] = static_cast<float *>(a.take(nh_b));
+        d[l] = static_cast<float *>(a.take(nh_b));
+        del[l] = static_cast<float *>(a.take(nh_b));
+        der[l] = static_cast<float *>(a.take(nh_b));
+    }
+    const size_t ws_bytes = sar_gat_workspace_bytes(g, H, F, io->t);
+    void *ws = a.take(ws_bytes);
+    if (!ws || !gb) return SAR_ERR_WORKSPACE;
+
+    // host -> device
+    SAR_CUDA_TRY(cudaMemcpyAsync(feat[0], io->feat0, row_b, cudaMemcpyHostToDevice, st));
+    SAR_CUDA_TRY(cudaMemcpyAsync(ga, io->gout, row_b, cudaMemcpyHostToDevice, st));
+    for (int l = 0; l < L; ++l) {
+        SAR_CUDA_TRY(cudaMemcpyAsync(el[l], io->el[l], nh_b, cudaMemcpyHostToDevice, st));
+        SAR_CUDA_TRY(cudaMemcpyAsync(er[l], io->er[l], nh_b, cudaMemcpyHostToDevice, st));
+    }
+
+    // per-partition pointer lists (one array cut at `bounds`)
+    std::vector<const void *> fq(k);
+    std::vector<void *> dfq(k);
+    std::vector<const float *> erq(k);
+    std::vector<float *> derq(k);
+    const size_t rb = (size_t)H * F * sar_elem_size(io->t);
+    auto cut = [&](const void *base, size_t stride, int q) {
+        return static_cast<const char *>(base) + (size_t)bounds[q] * stride;
+    };
+    for (int l = 0; l < L; ++l) {
+        for (int q = 0; q < k; ++q) {
+            fq[q] = cut(feat[l], rb, q);
+            erq[q] = reinterpret_cast<const float *>(cut(er[l], (size_t)H * 4, q));
+        }
+        SAR_TRY(sar_gat_fwd_fused(g, k, bounds, fq.data(), el[l], erq.data(), H, F, io->t, io->slope, m[l], d[l],
+                                  feat[l + 1], ws, ws_bytes, st));
+    }
+    void *gin = ga, *gout = gb;
+    for (int l = L - 1; l >= 0; --l) {
+        for (int q = 0; q < k; ++q) {
+            fq[q] = cut(feat[l], rb, q);
+            erq[q] = reinterpret_cast<const float *>(cut(er[l], (size_t)H * 4, q));
+            dfq[q] = const_cast<char *>(cut(gout, rb, q));
+            derq[q] = reinterpret_cast<float *>(const_cast<char *>(cut(der[l], (size_t)H * 4, q)));
+        }
+        SAR_TRY(sar_gat_bwd_fused(g, k, bounds, fq.data(), el[l], erq.data(), m[l], d[l], gin, H, F, io->t, io->slope,
+                                  dfq.data(), del[l], derq.data(), ws, ws_bytes, st));
+        void *tmp = gin;
+        gin = gout;
+        gout = tmp;
+    }
+    // device -> host (gin now holds dfeat of layer 0)
+    if (io->out_last) SAR_CUDA_TRY(cudaMemcpyAsync(io->out_last, feat[L], row_b, cudaMemcpyDeviceToHost, st));
+    if (io->dfeat0) SAR_CUDA_TRY(cudaMemcpyAsync(io->dfeat0, gin, row_b, cudaMemcpyDeviceToHost, st));
+    for (int l = 0; l < L; ++l) {
+        if (io->del) SAR_CUDA_TRY(cudaMemcpyAsync(io->del[l], del[l], nh_b, cudaMemcpyDeviceToHost, st));
+        if (io->der) SAR_CUDA_TRY(cudaMemcpyAsync(io->der[l], der[l], nh_b, cudaMemcpyDeviceToHost, st));
+    }
+    return SAR_OK;
+}
+
+}  // extern "C"

@@ -38,16 +38,8 @@ struct WeightOf {
     using type = float;
 };
 template <>
-struct WeightOf<kBwdDst> {
-    using type = float2;
-};
-template <>
-struct WeightOf<kBwdDstGivenD> {
-    using type = float2;
-};
-template <>
 struct WeightOf<kBwdSrc> {
-    using type = float4;
+    using type = float2;
 };
 
 // Floats of shared memory one warp needs: 32 column ids, 32 rescale factors, then the larger of

@@ -1,0 +1,642 @@
+// Span kernels of libsar (internal): forward, both backward passes and the sum aggregation.
+//
+// A WARP owns a SPAN of R consecutive rows of the traversal (destinations for the CSR passes,
+// sources for the CSC pass).  Rows are short on average (a power-law graph's median degree is a
+// handful of edges), so walking them one by one leaves a chain of dependent loads per row
+// (indptr -> indices -> scores -> feature rows) and almost nothing in flight.  Instead the warp
+//   1. cuts the span into CHUNKS of whole rows holding at most CAP edges (a row longer than CAP is
+//      taken alone, CAP edges at a time, its accumulators staying in registers in between);
+//   2. stages the chunk in shared memory, SLOT-major: a slot is 32/G consecutive edges of one row
+//      (G lanes x 16 bytes cover one feature row), rows are padded to whole slots.  Column ids are
+//      loaded coalesced; the score phase computes one weight record per (edge, head) - spread evenly
+//      over the 32 lanes whatever the row lengths, one exponential per pair, many independent
+//      gathers of er / destination records in flight;
+//   3. streams the chunk's feature rows through a ring of S stages in shared memory filled by
+//      cp.async (16 bytes per lane, bypassing L1): the copies of slot s+S are issued when slot s has
+//      been accumulated, so S x 512 bytes per warp are in flight without holding registers, and no
+//      load of this phase depends on another load.  A row is finalised when its last slot has been
+//      consumed: the 32/G edge lanes are folded with shuffles and one of them writes the result.
+// Nothing per edge is written to global memory.  No floating-point atomics: every output element
+// has one writer (the per-(row, head) max of the forward pass is a shared-memory atomicMax on an
+// order-preserving integer key, whose result does not depend on the order).
+// Rows above the plan's threshold are skipped here and processed as independent segments by a second
+// launch (mode 1) that writes partial accumulators; the merge kernels of sar_gat_kernels.cuh fold them.
+#pragma once
+
+#include "sar_rowkernels.cuh"
+
+namespace sar {
+
+constexpr int kSpanWarps = 4;             // warps per block
+constexpr int kSpanThreads = kSpanWarps * 32;
+constexpr int kMaxSpanRows = 16;          // rows per span
+
+struct SpanArgs {
+    long long n_rows;
+    const int64_t *indptr;
+    const int32_t *indices;
+    const void *gather;      // rows fetched per edge: feat (forward, bwd-dst, sum) or gout (bwd-src)
+    const void *rowvec;      // row-stationary vector: gout (bwd-dst) or feat (bwd-src)
+    const float *el, *er;    // forward / bwd-dst: el[row], er[col];  bwd-src: er[row]
+    const float *m, *d;      // bwd-dst: final statistics of the row
+    const float4 *rec_in;    // bwd-src: {el, m, 1/d, D} of the column; bwd-dst GIVEN_D: of the row
+    float4 *rec_out;         // bwd-dst (D rebuilt): record written per row
+    float *acc_state;        // forward: running numerator [n_rows, H*F] or null
+    float *m_state, *d_state;
+    void *out;               // forward: out; bwd-src: dfeat; sum: out
+    float *del, *der;
+    const int64_t *deg_total;
+    float slope;
+    unsigned flags;
+    RowGeom g;
+    SplitArgs sp;
+    int mode;                // 0: spans of R rows; 1: one long-row segment per warp
+    int R;                   // rows per span (<= kMaxSpanRows)
+};
+
+// order-preserving float -> unsigned key (for shared-memory atomicMax)
+__device__ __forceinline__ unsigned fkey(float x) {
+    const unsigned b = __float_as_uint(x);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ __forceinline__ float fkey_inv(unsigned k) {
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7fffffffu) : ~k);
+}
+constexpr unsigned kKeyNegInf = 0x007fffffu;  // fkey(-inf)
+
+// 16-byte asynchronous copy global -> shared that bypasses L1; src_bytes = 0 writes zeros.
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc, int src_bytes) {
+    const unsigned s = (unsigned)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(s), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
+}
+
+// Shared-memory layout of one warp (byte offsets).
+struct SpanSmem {
+    size_t stage, sj, w, rowc, srb, sso, mrun, fac, scratch, total;
+};
+__host__ __device__ inline size_t span_align16(size_t x) { return (x + 15) & ~(size_t)15; }
+template <int MODE>
+__host__ __device__ inline SpanSmem span_layout(int Hp, int V, int cap, int stages, int epw) {
+    const size_t wbytes = MODE == kSum ? 0 : sizeof(typename WeightOf<MODE>::type);
+    const size_t pos = (size_t)cap + (size_t)kMaxSpanRows * (epw - 1);  // padded edge positions
+    SpanSmem L;
+    size_t o = 0;
+    L.stage = o;   o += (size_t)stages * V * 512;                // ring of gathered slots
+    L.sj = o;      o += span_align16(pos * 4);                   // column id per padded position (-1: padding)
+    L.w = o;       o += span_align16(pos * Hp * wbytes);         // weight record per (position, head)
+    L.rowc = o;    o += (size_t)kMaxSpanRows * Hp * 16;          // per-(row, head) constants
+    L.srb = o;     o += (size_t)(kMaxSpanRows + 1) * 4;          // local first edge of each row
+    L.sso = o;     o += (size_t)(kMaxSpanRows + 1) * 4;          // first slot of each row
+    L.mrun = o;    o += (size_t)Hp * 4;                          // running max of a continued row
+    L.fac = o;     o += (size_t)Hp * 4;                          // its rescale factors
+    o = span_align16(o);
+    L.scratch = o; o += (size_t)(64 * V + 32) * 4;               // epilogue scratch
+    L.total = span_align16(o);
+    return L;
+}
+
+template <typename T, int G, int V, int S, int MODE, int CAP, int MINB>
+__global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs a) {
+    constexpr int EPV = Elem<T>::EPV;
+    constexpr int EPW = 32 / G;  // edges per slot
+    using W = typename WeightOf<MODE>::type;
+    constexpr bool kFwdMode = MODE == kFwd;
+    constexpr bool kDst = MODE == kBwdDst || MODE == kBwdDstGivenD;
+    constexpr bool kSrc = MODE == kBwdSrc;
+    constexpr bool kAcc0 = MODE != kBwdDstGivenD;                  // accumulator 0 live
+    constexpr bool kAcc1 = kDst || kSrc;                           // accumulator 1 live
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int gl = lane & (G - 1), half = lane / G;
+    const int H = a.g.H, Hp = a.g.Hp, lgHp = a.g.lgHp, n_vec = a.g.n_vec;
+    const long long rowf = (long long)n_vec * EPV;
+
+    // ---- shared memory carve-up (per warp) ----------------------------------------------------
+    const SpanSmem L = span_layout<MODE>(Hp, V, CAP, S, EPW);
+    unsigned char *wb = smem_raw + (size_t)warp * L.total;
+    uint4 *stage = reinterpret_cast<uint4 *>(wb + L.stage);  // [S][V][32]
+    int *sj = reinterpret_cast<int *>(wb + L.sj);
+    W *sw = reinterpret_cast<W *>(wb + L.w);
+    float4 *srowc = reinterpret_cast<float4 *>(wb + L.rowc);
+    int *srb = reinterpret_cast<int *>(wb + L.srb);
+    int *sso = reinterpret_cast<int *>(wb + L.sso);
+    float *smrun = reinterpret_cast<float *>(wb + L.mrun);
+    float *sfac = reinterpret_cast<float *>(wb + L.fac);
+    float *scratch = reinterpret_cast<float *>(wb + L.scratch);
+    float *srowf = reinterpret_cast<float *>(srowc);         // forward: {el, key, ref, -} per (row, head)
+    unsigned *skey = reinterpret_cast<unsigned *>(srowc);
+
+    // ---- which rows ---------------------------------------------------------------------------
+    const long long item = (long long)blockIdx.x * kSpanWarps + warp;
+    long long row0, eb = 0, ee = 0;   // lane r: edge range of row row0 + r
+    int nrows;
+    bool excluded = false;            // long row left to the segment launch
+    long long seg = -1;
+    if (a.mode == 0) {
+        row0 = item * a.R;
+        if (row0 >= a.n_rows) return;
+        nrows = (int)((a.n_rows - row0) < a.R ? (a.n_rows - row0) : a.R);
+        long long p = 0;
+        if (lane <= nrows) p = __ldg(a.indptr + row0 + lane);  // nrows <= 16 < 32 lanes
+        const long long pn = __shfl_down_sync(0xffffffffu, p, 1);
+        if (lane < nrows) {
+            eb = p;
+            ee = pn;
+            excluded = a.sp.threshold > 0 && ee - eb > a.sp.threshold;
+        }
+    } else {
+        if (item >= a.sp.n_seg) return;
+        int lo = 0, hi = a.sp.n_long;
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (__ldg(a.sp.long_seg + mid) <= item) lo = mid; else hi = mid;
+        }
+        row0 = __ldg(a.sp.long_row + lo);
+        nrows = 1;
+        seg = item;
+        if (lane == 0) {
+            const long long c = item - __ldg(a.sp.long_seg + lo);
+            const long long rb_ = __ldg(a.indptr + row0), re_ = __ldg(a.indptr + row0 + 1);
+            eb = rb_ + c * a.sp.threshold;
+            ee = eb + a.sp.threshold < re_ ? eb + a.sp.threshold : re_;
+        }
+    }
+    const bool first_part = (a.flags & SAR_FIRST) || a.mode == 1;
+    const bool last_part = (a.flags & SAR_LAST) && a.mode == 0;
+    const bool mean_now = (a.flags & SAR_MEAN) && (a.flags & SAR_LAST);
+    // does a row without edges (in this partition) still have to be written?
+    bool write_empty;
+    if (kFwdMode) write_empty = (a.flags & SAR_FIRST) || (a.flags & SAR_LAST);
+    else if (MODE == kBwdDst) write_empty = true;
+    else if (MODE == kBwdDstGivenD) write_empty = a.flags & SAR_FIRST;
+    else if (kSrc) write_empty = true;
+    else write_empty = (a.flags & SAR_FIRST) || mean_now;
+    if (a.mode == 1) write_empty = false;
+
+    // ---- lane geometry ------------------------------------------------------------------------
+    int hv[V];
+    bool vok[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        const int vi = v * G + gl;
+        vok[v] = vi < n_vec;
+        hv[v] = vok[v] ? vi / a.g.vph : 0;
+    }
+    const uint4 *gbase = reinterpret_cast<const uint4 *>(a.gather) + gl;
+
+    // ---- per-row accumulators (persist across the chunks of a row longer than CAP) --------------
+    float acc0[V][EPV], acc1[V][EPV], sv[V], mrun[V];
+    float rv[V][EPV];  // row-stationary vector (bwd)
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        sv[v] = 0.f;
+        mrun[v] = SAR_NEG_INF;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) acc0[v][e] = acc1[v][e] = rv[v][e] = 0.f;
+    }
+
+    const int deg_l = (lane < nrows && !excluded) ? (int)((ee - eb) > 0x3fffffff ? 0x3fffffff : (ee - eb)) : 0;
+    const unsigned excl_all = __ballot_sync(0xffffffffu, excluded);
+
+    int r = 0;           // next row of the span to process
+    int piece_off = 0;   // edges of row r already consumed (row longer than CAP)
+    while (r < nrows) {
+        // ---- choose the chunk: rows [r, r2) --------------------------------------------------
+        if ((excl_all >> r) & 1u) {
+            ++r;
+            continue;
+        }
+        const int deg_r = __shfl_sync(0xffffffffu, deg_l, r);
+        int r2, ne;                       // chunk rows [r, r2), edges in chunk
+        const bool cont = piece_off > 0;  // first row continues from the previous chunk
+        bool unfinished = false;          // the row goes on in the next chunk
+        const long long cb = __shfl_sync(0xffffffffu, eb, r) + piece_off;  // global index of the chunk's first edge
+        if (deg_r - piece_off > CAP) {
+            r2 = r + 1;
+            ne = CAP;
+            unfinished = true;
+        } else if (cont) {
+            r2 = r + 1;
+            ne = deg_r - piece_off;
+        } else {
+            // greedy run of whole rows: none excluded, total <= CAP
+            int pre = (lane >= r && lane < nrows) ? deg_l : 0;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, pre, o);
+                if (lane >= o) pre = (pre > 0x3fffffff - t) ? 0x3fffffff : pre + t;
+            }
+            const unsigned later = excl_all & ~((1u << r) - 1u);
+            const int stop = later ? __ffs(later) - 1 : nrows;  // first excluded row after r
+            const unsigned fits = __ballot_sync(0xffffffffu, lane >= r && lane < stop && pre <= CAP);
+            r2 = r + __popc(fits);  // `fits` is a run of lanes starting at r (prefix sums ascend)
+            ne = __shfl_sync(0xffffffffu, pre, r2 - 1);
+        }
+        const int nr = r2 - r;
+        const bool piece = cont || unfinished;
+
+        // ---- stage A: row tables and per-row constants ---------------------------------------
+        {
+            const int i = lane - r;
+            int ns = 0;
+            if (i >= 0 && i < nr) {
+                const int dg = piece ? ne : deg_l;
+                srb[i] = piece ? 0 : (int)(eb - cb);
+                if (i == nr - 1) srb[nr] = ne;
+                ns = (dg + EPW - 1) / EPW;
+            }
+            int inc = ns;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const int t = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += t;
+            }
+            if (i >= 0 && i < nr) sso[i] = inc - ns;
+            if (i == nr - 1) sso[nr] = inc;
+        }
+        if constexpr (MODE != kSum) {
+            for (int x = lane; x < nr * Hp; x += 32) {
+                const int i = x >> lgHp, h = x & (Hp - 1);
+                const long long row = row0 + r + i;
+                float4 c = make_float4(0.f, __uint_as_float(kKeyNegInf), 0.f, 0.f);
+                if (h < H) {
+                    if constexpr (kFwdMode) {
+                        c.x = __ldg(a.el + row * H + h);
+                    } else if constexpr (kDst) {
+                        const float dd = __ldg(a.d + row * H + h);
+                        c = make_float4(__ldg(a.el + row * H + h), __ldg(a.m + row * H + h), dd > 0.f ? 1.f / dd : 0.f, 0.f);
+                    } else {
+                        c.x = __ldg(a.er + row * H + h);
+                    }
+                }
+                srowc[x] = c;
+            }
+        }
+        __syncwarp();
+        // ---- stage B: column ids, slot-major (row i's edges start at position sso[i]*EPW) --------
+        const int nslots = sso[nr];
+        const int npos = nslots * EPW;
+        {
+            int i = 0;
+            for (int q = lane; q < npos; q += 32) {
+                while (q >= sso[i + 1] * EPW) ++i;
+                const int t = srb[i] + (q - sso[i] * EPW);
+                sj[q] = t < srb[i + 1] ? ld_stream_i32(a.indices + cb + t) : -1;
+            }
+        }
+        __syncwarp();
+
+        // ---- stage C: one weight record per (position, head) ---------------------------------------
+        if constexpr (MODE != kSum) {
+            int i = 0;
+#pragma unroll 2
+            for (int x = lane; x < (npos << lgHp); x += 32) {
+                const int q = x >> lgHp, h = x & (Hp - 1);
+                while (q >= sso[i + 1] * EPW) ++i;
+                const int col = sj[q];
+                const bool live = col >= 0 && h < H;
+                const float4 c = srowc[i * Hp + h];
+                float gr;
+                if constexpr (kFwdMode) {
+                    float e = SAR_NEG_INF;  // padding: weight exp(-inf - max) = 0
+                    if (live) {
+                        e = leaky(c.x + __ldg(a.er + (long long)col * H + h), a.slope, gr);
+                        atomicMax(&skey[(i * Hp + h) * 4 + 1], fkey(e));
+                    }
+                    sw[x] = e;
+                } else if constexpr (kDst) {
+                    // rematerialised attention coefficient alpha >= 0; its sign bit carries
+                    // "score <= 0" (LeakyReLU' = slope), so one float holds both weights
+                    float wrec = 0.f;
+                    if (live) {
+                        const float s_ = c.x + __ldg(a.er + (long long)col * H + h);
+                        const float al = fast_exp(leaky(s_, a.slope, gr) - c.y) * c.z;
+                        wrec = s_ > 0.f ? al : -al;
+                    }
+                    sw[x] = wrec;
+                } else {
+                    float2 wrec = make_float2(0.f, 0.f);
+                    if (live) {
+                        const float4 rec = __ldg(a.rec_in + (long long)col * H + h);  // {el_i, m_i, 1/d_i, D_i}
+                        const float s_ = rec.x + c.x;
+                        const float al = fast_exp(leaky(s_, a.slope, gr) - rec.y) * rec.z;
+                        wrec = make_float2(s_ > 0.f ? al : -al, al * gr * rec.w);
+                    }
+                    sw[x] = wrec;
+                }
+            }
+            __syncwarp();
+        }
+        if constexpr (kFwdMode) {
+            // reference max per (row, head): the chunk's max, joined with the running max of a
+            // continued row; rescale factor exp(old_max - new_max) for what is already accumulated
+            for (int x = lane; x < nr * Hp; x += 32) {
+                float ref = fkey_inv(skey[x * 4 + 1]);
+                if (cont) {  // then nr == 1 and x is the head
+                    const float old = smrun[x];
+                    ref = fmaxf(ref, old);
+                    sfac[x] = (ref == SAR_NEG_INF) ? 1.f : fast_exp(old - ref);
+                }
+                srowf[x * 4 + 2] = ref;
+            }
+            __syncwarp();
+            int i = 0;
+#pragma unroll 2
+            for (int x = lane; x < (npos << lgHp); x += 32) {
+                const int q = x >> lgHp, h = x & (Hp - 1);
+                while (q >= sso[i + 1] * EPW) ++i;
+                const float ref = srowf[(i * Hp + h) * 4 + 2];
+                sw[x] = (ref == SAR_NEG_INF) ? 0.f : fast_exp(sw[x] - ref);
+            }
+            __syncwarp();
+            if (cont) {
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    const float c = sfac[hv[v]];
+                    sv[v] *= c;
+                    mrun[v] = srowf[hv[v] * 4 + 2];
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) acc0[v][e] *= c;
+                }
+            }
+        }
+
+        // ---- stage D: gather through the cp.async ring ---------------------------------------------
+        auto issue = [&](int s) {
+            const int col = s < nslots ? sj[s * EPW + half] : -1;
+            const uint4 *src = gbase + (long long)(col < 0 ? 0 : col) * n_vec;
+            uint4 *dst = stage + (size_t)(s % S) * V * 32 + lane;
+#pragma unroll
+            for (int v = 0; v < V; ++v)
+                cp_async16(dst + v * 32, src + v * G, (col >= 0 && vok[v]) ? 16 : 0);
+            cp_async_commit();
+        };
+#pragma unroll
+        for (int s = 0; s < S; ++s) issue(s);
+
+        int s = 0;
+        for (int ri = 0; ri < nr; ++ri) {
+            const int s_end = sso[ri + 1];
+            const long long row = row0 + r + ri;
+            const bool row_starts = !(cont && ri == 0);
+            const bool row_ends = !(unfinished && ri == nr - 1);
+            if (s_end == s && !(write_empty && row_starts)) continue;  // no edges here, nothing to write
+            if (row_starts) {
+                if constexpr (kFwdMode) {
+#pragma unroll
+                    for (int v = 0; v < V; ++v) mrun[v] = srowf[(ri * Hp + hv[v]) * 4 + 2];
+                }
+                if constexpr (kDst || kSrc) load_row_vec<T, G, V>(a.rowvec, row, n_vec, gl, vok, rv);
+            }
+            for (; s < s_end; ++s) {
+                cp_async_wait<S - 1>();  // this lane's copies of slot s have landed
+                const uint4 *src = stage + (size_t)(s % S) * V * 32 + lane;
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    float x[EPV];
+                    Elem<T>::unpack(src[v * 32], x);
+                    if constexpr (MODE == kSum) {
+#pragma unroll
+                        for (int e = 0; e < EPV; ++e) acc0[v][e] += x[e];
+                    } else {
+                        const int wi = ((s * EPW + half) << lgHp) + hv[v];
+                        if constexpr (kFwdMode) {
+                            const float w = sw[wi];
+                            sv[v] += w;
+#pragma unroll
+                            for (int e = 0; e < EPV; ++e) acc0[v][e] = fmaf(w, x[e], acc0[v][e]);
+                        } else if constexpr (kDst) {
+                            const float ws = sw[wi];
+                            const float al = fabsf(ws);
+                            const float w2 = ws < 0.f ? al * a.slope : al;  // alpha * LeakyReLU'
+                            sv[v] += w2;
+#pragma unroll
+                            for (int e = 0; e < EPV; ++e) {
+                                if constexpr (kAcc0) acc0[v][e] = fmaf(al, x[e], acc0[v][e]);
+                                acc1[v][e] = fmaf(w2, x[e], acc1[v][e]);
+                            }
+                        } else {
+                            const float2 w = sw[wi];
+                            const float al = fabsf(w.x);
+                            const float w2 = w.x < 0.f ? al * a.slope : al;
+                            sv[v] += w.y;
+#pragma unroll
+                            for (int e = 0; e < EPV; ++e) {
+                                acc0[v][e] = fmaf(al, x[e], acc0[v][e]);
+                                acc1[v][e] = fmaf(w2, x[e], acc1[v][e]);
+                            }
+                        }
+                    }
+                }
+                issue(s + S);  // refill the stage just consumed (each lane re-uses its own 16 bytes)
+            }
+            if (!row_ends) continue;
+
+            // ---- the row is complete: fold the 32/G edge lanes, finalise, reset --------------------
+#pragma unroll
+            for (int off = G; off < 32; off <<= 1) {
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    sv[v] += __shfl_xor_sync(0xffffffffu, sv[v], off);
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) {
+                        if constexpr (kAcc0) acc0[v][e] += __shfl_xor_sync(0xffffffffu, acc0[v][e], off);
+                        if constexpr (kAcc1) acc1[v][e] += __shfl_xor_sync(0xffffffffu, acc1[v][e], off);
+                    }
+                }
+            }
+            const bool writer = half == 0;  // every edge lane now holds the full sums; one writes
+            if constexpr (kFwdMode) {
+                if (a.mode == 1) {
+                    if (writer) {
+                        float *rec = a.sp.part + seg * a.sp.pstride;
+                        store_acc_row<G, V, EPV>(rec, gl, vok, acc0);
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+                            if (vok[v] && ((v * G + gl) % a.g.vph) == 0) {
+                                rec[rowf + hv[v]] = mrun[v];
+                                rec[rowf + H + hv[v]] = sv[v];
+                            }
+                    }
+                } else {
+                    if (!first_part) {  // fold the state left by the earlier partitions (Algorithm 1)
+                        float old[V][EPV];
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+#pragma unroll
+                            for (int e = 0; e < EPV; ++e) old[v][e] = 0.f;
+                        load_acc_row<G, V, EPV>(a.acc_state + row * rowf, gl, vok, old);
+#pragma unroll
+                        for (int v = 0; v < V; ++v) {
+                            const float mo = vok[v] ? a.m_state[row * H + hv[v]] : SAR_NEG_INF;
+                            const float dd = vok[v] ? a.d_state[row * H + hv[v]] : 0.f;
+                            const float mn = fmaxf(mo, mrun[v]);
+                            const float c_old = (mn == SAR_NEG_INF) ? 1.f : fast_exp(mo - mn);
+                            const float c_new = (mn == SAR_NEG_INF) ? 1.f : fast_exp(mrun[v] - mn);
+                            sv[v] = dd * c_old + sv[v] * c_new;
+                            mrun[v] = mn;
+#pragma unroll
+                            for (int e = 0; e < EPV; ++e) acc0[v][e] = old[v][e] * c_old + acc0[v][e] * c_new;
+                        }
+                        __syncwarp();  // every edge lane has read the old state before one overwrites it
+                    }
+                    if (writer) {
+                        if (last_part) {
+#pragma unroll
+                            for (int v = 0; v < V; ++v) {
+                                const float inv = sv[v] > 0.f ? 1.f / sv[v] : 0.f;
+#pragma unroll
+                                for (int e = 0; e < EPV; ++e) acc0[v][e] *= inv;
+                            }
+                            store_row_vec<T, G, V>(a.out, row, n_vec, gl, vok, acc0);
+                        } else {
+                            store_acc_row<G, V, EPV>(a.acc_state + row * rowf, gl, vok, acc0);
+                        }
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+                            if (vok[v] && ((v * G + gl) % a.g.vph) == 0) {
+                                a.m_state[row * H + hv[v]] = mrun[v];
+                                a.d_state[row * H + hv[v]] = sv[v];
+                            }
+                    }
+                }
+            } else if constexpr (kDst) {
+                if (a.mode == 1) {
+                    if (writer) {
+                        float *rec = a.sp.part + seg * a.sp.pstride;
+                        store_acc_row<G, V, EPV>(rec, gl, vok, acc1);
+                        if constexpr (MODE == kBwdDst) store_acc_row<G, V, EPV>(rec + rowf, gl, vok, acc0);
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+                            if (vok[v] && ((v * G + gl) % a.g.vph) == 0) rec[2 * rowf + hv[v]] = sv[v];
+                    }
+                } else {
+                    float pA[V], pB[V];
+#pragma unroll
+                    for (int v = 0; v < V; ++v) {
+                        pA[v] = pB[v] = 0.f;
+#pragma unroll
+                        for (int e = 0; e < EPV; ++e) {
+                            if constexpr (kAcc0) pA[v] = fmaf(rv[v][e], acc0[v][e], pA[v]);
+                            pB[v] = fmaf(rv[v][e], acc1[v][e], pB[v]);
+                        }
+                    }
+                    // per-head sums through shared memory (edge lane 0 deposits, lanes < H add up)
+                    if (writer) {
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+                            if (vok[v]) {
+                                scratch[v * G + gl] = pB[v];
+                                scratch[32 * V + v * G + gl] = pA[v];
+                                if (((v * G + gl) % a.g.vph) == 0) scratch[64 * V + hv[v]] = sv[v];
+                            }
+                    }
+                    __syncwarp();
+                    if (lane < H) {
+                        float DB = 0.f, DA = 0.f;
+                        for (int k = 0; k < a.g.vph; ++k) {
+                            DB += scratch[lane * a.g.vph + k];
+                            DA += scratch[32 * V + lane * a.g.vph + k];
+                        }
+                        const float Sh = scratch[64 * V + lane];
+                        const float4 c = srowc[ri * Hp + lane];
+                        const float D = MODE == kBwdDstGivenD ? a.rec_in[row * H + lane].w : DA;
+                        const float val = DB - D * Sh;
+                        float *p = a.del + row * H + lane;
+                        *p = (a.flags & SAR_FIRST) ? val : *p + val;
+                        if constexpr (MODE == kBwdDst) a.rec_out[row * H + lane] = make_float4(c.x, c.y, c.z, D);
+                    }
+                    __syncwarp();
+                }
+            } else if constexpr (kSrc) {
+                if (a.mode == 1) {
+                    if (writer) {
+                        float *rec = a.sp.part + seg * a.sp.pstride;
+                        store_acc_row<G, V, EPV>(rec, gl, vok, acc0);
+                        store_acc_row<G, V, EPV>(rec + rowf, gl, vok, acc1);
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+                            if (vok[v] && ((v * G + gl) % a.g.vph) == 0) rec[2 * rowf + hv[v]] = sv[v];
+                    }
+                } else {
+                    float pC[V];
+#pragma unroll
+                    for (int v = 0; v < V; ++v) {
+                        pC[v] = 0.f;
+#pragma unroll
+                        for (int e = 0; e < EPV; ++e) pC[v] = fmaf(rv[v][e], acc1[v][e], pC[v]);
+                    }
+                    if (writer) {
+                        store_row_vec<T, G, V>(a.out, row, n_vec, gl, vok, acc0);
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+                            if (vok[v]) {
+                                scratch[v * G + gl] = pC[v];
+                                if (((v * G + gl) % a.g.vph) == 0) scratch[64 * V + hv[v]] = sv[v];
+                            }
+                    }
+                    __syncwarp();
+                    if (lane < H) {
+                        float DC = 0.f;
+                        for (int k = 0; k < a.g.vph; ++k) DC += scratch[lane * a.g.vph + k];
+                        a.der[row * H + lane] = DC - scratch[64 * V + lane];
+                    }
+                    __syncwarp();
+                }
+            } else {  // sum aggregation
+                if (a.mode == 1) {
+                    if (writer) store_acc_row<G, V, EPV>(a.sp.part + seg * a.sp.pstride, gl, vok, acc0);
+                } else if (writer) {
+                    if (!(a.flags & SAR_FIRST)) {
+                        float old[V][EPV];
+                        load_row_vec<T, G, V, false>(a.out, row, n_vec, gl, vok, old);
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+#pragma unroll
+                            for (int e = 0; e < EPV; ++e) acc0[v][e] += old[v][e];
+                    }
+                    if (mean_now) {
+                        const long long dg = a.deg_total[row];
+                        const float inv = dg > 0 ? 1.f / (float)dg : 0.f;
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+#pragma unroll
+                            for (int e = 0; e < EPV; ++e) acc0[v][e] *= inv;
+                    }
+                    store_row_vec<T, G, V>(a.out, row, n_vec, gl, vok, acc0);
+                }
+            }
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                sv[v] = 0.f;
+                mrun[v] = SAR_NEG_INF;
+#pragma unroll
+                for (int e = 0; e < EPV; ++e) acc0[v][e] = acc1[v][e] = 0.f;
+            }
+        }
+        cp_async_wait<0>();  // drain the (zero-size) refills issued past the last slot
+        // ---- a row that goes on: publish its running max for the next chunk's score phase -------
+        if constexpr (kFwdMode) {
+            if (unfinished && half == 0) {
+#pragma unroll
+                for (int v = 0; v < V; ++v)
+                    if (vok[v] && ((v * G + gl) % a.g.vph) == 0) smrun[hv[v]] = mrun[v];
+            }
+        }
+        __syncwarp();
+        if (unfinished) {
+            piece_off += CAP;
+        } else {
+            piece_off = 0;
+            r = r2;
+        }
+    }
+}
+
+}  // namespace sar
