@@ -141,7 +141,7 @@ static sar_status check_elem_align(std::initializer_list<const void *> ps, size_
 
 // ---- span kernels ---------------------------------------------------------------------------------
 constexpr int kCapFwd = 128, kCapDst = 128, kCapSrc = 128, kCapSum = 128;
-constexpr int kMinBlocksFwd = 4, kMinBlocksBwd = 3;  // resident blocks per SM the register budget is cut for
+constexpr int kMinBlocksFwd = 6, kMinBlocksBwd = 5;  // resident blocks per SM the register budget is cut for
 
 static int rows_per_span(long long n_rows, long long nnz, int cap) {
     const double avg = n_rows > 0 ? (double)nnz / (double)n_rows : 0.0;
@@ -173,9 +173,9 @@ static sar_status launch_span(SpanArgs a, long long nnz, const char *name, const
     return SAR_OK;
 }
 
-// stages of the gather ring: 16 x 512 bytes in flight per warp for one-vector rows
-template <int V> struct UFwd { static constexpr int u = V == 1 ? 16 : (V == 2 ? 8 : (V == 4 ? 4 : 2)); };
-template <int V> struct UBwd { static constexpr int u = V == 1 ? 16 : (V == 2 ? 8 : (V == 4 ? 4 : 2)); };
+// stages of the gather ring: 8 x 512 bytes in flight per warp for one-vector rows
+template <int V> struct UFwd { static constexpr int u = V == 1 ? 8 : (V == 2 ? 4 : 2); };
+template <int V> struct UBwd { static constexpr int u = V == 1 ? 8 : (V == 2 ? 4 : 2); };
 
 }  // namespace sar
 
@@ -302,6 +302,7 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
     a.flags = flags;
     a.g = s.geom;
     a.sp = ma.sp;
+    a.hvec = (H % 4 == 0) && sar_aligned(er_q, 16);
     return dispatch(s, [&](auto cfg) -> sar_status {
         using C = decltype(cfg);
         using T = typename C::type;
@@ -512,6 +513,7 @@ sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, c
     d1.flags = flags;
     d1.g = s.geom;
     d1.sp = da.sp;
+    d1.hvec = (H % 4 == 0) && sar_aligned(er_q, 16);
     SpanArgs s1{};  // source-major pass over the CSC
     s1.n_rows = g->n_src;
     s1.indptr = g->t_indptr;
@@ -526,6 +528,7 @@ sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, c
     s1.flags = flags;
     s1.g = s.geom;
     s1.sp = sa.sp;
+    s1.hvec = (H % 4 == 0);
 
     return dispatch(s, [&](auto cfg) -> sar_status {
         using C = decltype(cfg);

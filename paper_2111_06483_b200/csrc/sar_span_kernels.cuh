@@ -52,6 +52,7 @@ struct SpanArgs {
     SplitArgs sp;
     int mode;                // 0: spans of R rows; 1: one long-row segment per warp
     int R;                   // rows per span (<= kMaxSpanRows)
+    int hvec;                // heads are scored four at a time (H % 4 == 0 and er is 16-byte aligned)
 };
 
 // order-preserving float -> unsigned key (for shared-memory atomicMax)
@@ -83,13 +84,13 @@ __host__ __device__ inline size_t span_align16(size_t x) { return (x + 15) & ~(s
 template <int MODE>
 __host__ __device__ inline SpanSmem span_layout(int Hp, int V, int cap, int stages, int epw) {
     const size_t wbytes = MODE == kSum ? 0 : sizeof(typename WeightOf<MODE>::type);
-    const size_t pos = (size_t)cap + (size_t)kMaxSpanRows * (epw - 1);  // padded edge positions
+    const size_t pos = (size_t)cap + (size_t)kMaxSpanRows * (epw - 1) + (size_t)stages * epw;  // padded positions
     SpanSmem L;
     size_t o = 0;
     L.stage = o;   o += (size_t)stages * V * 512;                // ring of gathered slots
     L.sj = o;      o += span_align16(pos * 4);                   // column id per padded position (-1: padding)
     L.w = o;       o += span_align16(pos * Hp * wbytes);         // weight record per (position, head)
-    L.rowc = o;    o += (size_t)kMaxSpanRows * Hp * 16;          // per-(row, head) constants
+    L.rowc = o;    o += span_align16((size_t)kMaxSpanRows * Hp * 4) * 3;  // three planes of per-(row, head) constants
     L.srb = o;     o += (size_t)(kMaxSpanRows + 1) * 4;          // local first edge of each row
     L.sso = o;     o += (size_t)(kMaxSpanRows + 1) * 4;          // first slot of each row
     L.mrun = o;    o += (size_t)Hp * 4;                          // running max of a continued row
@@ -123,14 +124,16 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
     uint4 *stage = reinterpret_cast<uint4 *>(wb + L.stage);  // [S][V][32]
     int *sj = reinterpret_cast<int *>(wb + L.sj);
     W *sw = reinterpret_cast<W *>(wb + L.w);
-    float4 *srowc = reinterpret_cast<float4 *>(wb + L.rowc);
+    const int plane = (int)(span_align16((size_t)kMaxSpanRows * Hp * 4) / 4);
+    float *sc0 = reinterpret_cast<float *>(wb + L.rowc);  // el of the row (CSR passes) / er of the row (CSC pass)
+    float *sc1 = sc0 + plane;                             // forward: max key; bwd-dst: m
+    float *sc2 = sc1 + plane;                             // forward: reference max; bwd-dst: 1/d
     int *srb = reinterpret_cast<int *>(wb + L.srb);
     int *sso = reinterpret_cast<int *>(wb + L.sso);
     float *smrun = reinterpret_cast<float *>(wb + L.mrun);
     float *sfac = reinterpret_cast<float *>(wb + L.fac);
     float *scratch = reinterpret_cast<float *>(wb + L.scratch);
-    float *srowf = reinterpret_cast<float *>(srowc);         // forward: {el, key, ref, -} per (row, head)
-    unsigned *skey = reinterpret_cast<unsigned *>(srowc);
+    unsigned *skey = reinterpret_cast<unsigned *>(sc1);
 
     // ---- which rows ---------------------------------------------------------------------------
     const long long item = (long long)blockIdx.x * kSpanWarps + warp;
@@ -264,18 +267,22 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
             for (int x = lane; x < nr * Hp; x += 32) {
                 const int i = x >> lgHp, h = x & (Hp - 1);
                 const long long row = row0 + r + i;
-                float4 c = make_float4(0.f, __uint_as_float(kKeyNegInf), 0.f, 0.f);
+                float c0 = 0.f, c1 = __uint_as_float(kKeyNegInf), c2 = 0.f;
                 if (h < H) {
                     if constexpr (kFwdMode) {
-                        c.x = __ldg(a.el + row * H + h);
+                        c0 = __ldg(a.el + row * H + h);
                     } else if constexpr (kDst) {
                         const float dd = __ldg(a.d + row * H + h);
-                        c = make_float4(__ldg(a.el + row * H + h), __ldg(a.m + row * H + h), dd > 0.f ? 1.f / dd : 0.f, 0.f);
+                        c0 = __ldg(a.el + row * H + h);
+                        c1 = __ldg(a.m + row * H + h);
+                        c2 = dd > 0.f ? 1.f / dd : 0.f;
                     } else {
-                        c.x = __ldg(a.er + row * H + h);
+                        c0 = __ldg(a.er + row * H + h);
                     }
                 }
-                srowc[x] = c;
+                sc0[x] = c0;
+                sc1[x] = c1;
+                sc2[x] = c2;
             }
         }
         __syncwarp();
@@ -289,46 +296,102 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                 const int t = srb[i] + (q - sso[i] * EPW);
                 sj[q] = t < srb[i + 1] ? ld_stream_i32(a.indices + cb + t) : -1;
             }
+            for (int q = npos + lane; q < npos + S * EPW; q += 32) sj[q] = -1;  // the ring's run-out
         }
         __syncwarp();
 
-        // ---- stage C: one weight record per (position, head) ---------------------------------------
+        // ---- stage C: weight records, one padded position per lane and sweep, all its heads ------
         if constexpr (MODE != kSum) {
+            const bool vec4 = a.hvec != 0;  // heads handled four at a time with 16-byte accesses
             int i = 0;
-#pragma unroll 2
-            for (int x = lane; x < (npos << lgHp); x += 32) {
-                const int q = x >> lgHp, h = x & (Hp - 1);
+            for (int q = lane; q < npos; q += 32) {
                 while (q >= sso[i + 1] * EPW) ++i;
                 const int col = sj[q];
-                const bool live = col >= 0 && h < H;
-                const float4 c = srowc[i * Hp + h];
-                float gr;
-                if constexpr (kFwdMode) {
-                    float e = SAR_NEG_INF;  // padding: weight exp(-inf - max) = 0
-                    if (live) {
-                        e = leaky(c.x + __ldg(a.er + (long long)col * H + h), a.slope, gr);
-                        atomicMax(&skey[(i * Hp + h) * 4 + 1], fkey(e));
+                const int rb = i * Hp, wb_ = q << lgHp;
+                if (vec4) {
+                    for (int h = 0; h < H; h += 4) {
+                        const float4 c0 = *reinterpret_cast<const float4 *>(sc0 + rb + h);
+                        float s4[4], g4[4];
+                        if constexpr (kFwdMode || kDst) {
+                            float4 e4 = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (col >= 0) e4 = __ldg(reinterpret_cast<const float4 *>(a.er + (long long)col * H + h));
+                            s4[0] = c0.x + e4.x; s4[1] = c0.y + e4.y; s4[2] = c0.z + e4.z; s4[3] = c0.w + e4.w;
+                        }
+                        if constexpr (kFwdMode) {
+                            float4 o;
+                            float *op = reinterpret_cast<float *>(&o);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                op[k] = SAR_NEG_INF;  // padding: weight exp(-inf - max) = 0
+                                if (col >= 0) {
+                                    op[k] = leaky(s4[k], a.slope, g4[k]);
+                                    atomicMax(&skey[rb + h + k], fkey(op[k]));
+                                }
+                            }
+                            *reinterpret_cast<float4 *>(reinterpret_cast<float *>(sw) + wb_ + h) = o;
+                        } else if constexpr (kDst) {
+                            // rematerialised attention coefficient alpha >= 0; its sign bit carries
+                            // "score <= 0" (LeakyReLU' = slope), so one float holds both weights
+                            const float4 m4 = *reinterpret_cast<const float4 *>(sc1 + rb + h);
+                            const float4 i4 = *reinterpret_cast<const float4 *>(sc2 + rb + h);
+                            const float *mp = reinterpret_cast<const float *>(&m4), *ip = reinterpret_cast<const float *>(&i4);
+                            float4 o;
+                            float *op = reinterpret_cast<float *>(&o);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const float al = fast_exp(leaky(s4[k], a.slope, g4[k]) - mp[k]) * ip[k];
+                                op[k] = col >= 0 ? (s4[k] > 0.f ? al : -al) : 0.f;
+                            }
+                            *reinterpret_cast<float4 *>(reinterpret_cast<float *>(sw) + wb_ + h) = o;
+                        } else {
+                            const float *cp0 = reinterpret_cast<const float *>(&c0);
+                            float2 o[4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                o[k] = make_float2(0.f, 0.f);
+                                if (col >= 0) {
+                                    const float4 rec = __ldg(a.rec_in + (long long)col * H + h + k);  // {el_i, m_i, 1/d_i, D_i}
+                                    const float s_ = rec.x + cp0[k];
+                                    float gr;
+                                    const float al = fast_exp(leaky(s_, a.slope, gr) - rec.y) * rec.z;
+                                    o[k] = make_float2(s_ > 0.f ? al : -al, al * gr * rec.w);
+                                }
+                            }
+                            float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float2 *>(sw) + wb_ + h);
+                            dst[0] = make_float4(o[0].x, o[0].y, o[1].x, o[1].y);
+                            dst[1] = make_float4(o[2].x, o[2].y, o[3].x, o[3].y);
+                        }
                     }
-                    sw[x] = e;
-                } else if constexpr (kDst) {
-                    // rematerialised attention coefficient alpha >= 0; its sign bit carries
-                    // "score <= 0" (LeakyReLU' = slope), so one float holds both weights
-                    float wrec = 0.f;
-                    if (live) {
-                        const float s_ = c.x + __ldg(a.er + (long long)col * H + h);
-                        const float al = fast_exp(leaky(s_, a.slope, gr) - c.y) * c.z;
-                        wrec = s_ > 0.f ? al : -al;
-                    }
-                    sw[x] = wrec;
                 } else {
-                    float2 wrec = make_float2(0.f, 0.f);
-                    if (live) {
-                        const float4 rec = __ldg(a.rec_in + (long long)col * H + h);  // {el_i, m_i, 1/d_i, D_i}
-                        const float s_ = rec.x + c.x;
-                        const float al = fast_exp(leaky(s_, a.slope, gr) - rec.y) * rec.z;
-                        wrec = make_float2(s_ > 0.f ? al : -al, al * gr * rec.w);
+                    for (int h = 0; h < H; ++h) {
+                        const float c0 = sc0[rb + h];
+                        float gr;
+                        if constexpr (kFwdMode) {
+                            float e = SAR_NEG_INF;
+                            if (col >= 0) {
+                                e = leaky(c0 + __ldg(a.er + (long long)col * H + h), a.slope, gr);
+                                atomicMax(&skey[rb + h], fkey(e));
+                            }
+                            reinterpret_cast<float *>(sw)[wb_ + h] = e;
+                        } else if constexpr (kDst) {
+                            float wrec = 0.f;
+                            if (col >= 0) {
+                                const float s_ = c0 + __ldg(a.er + (long long)col * H + h);
+                                const float al = fast_exp(leaky(s_, a.slope, gr) - sc1[rb + h]) * sc2[rb + h];
+                                wrec = s_ > 0.f ? al : -al;
+                            }
+                            reinterpret_cast<float *>(sw)[wb_ + h] = wrec;
+                        } else {
+                            float2 wrec = make_float2(0.f, 0.f);
+                            if (col >= 0) {
+                                const float4 rec = __ldg(a.rec_in + (long long)col * H + h);
+                                const float s_ = rec.x + c0;
+                                const float al = fast_exp(leaky(s_, a.slope, gr) - rec.y) * rec.z;
+                                wrec = make_float2(s_ > 0.f ? al : -al, al * gr * rec.w);
+                            }
+                            reinterpret_cast<float2 *>(sw)[wb_ + h] = wrec;
+                        }
                     }
-                    sw[x] = wrec;
                 }
             }
             __syncwarp();
@@ -337,22 +400,34 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
             // reference max per (row, head): the chunk's max, joined with the running max of a
             // continued row; rescale factor exp(old_max - new_max) for what is already accumulated
             for (int x = lane; x < nr * Hp; x += 32) {
-                float ref = fkey_inv(skey[x * 4 + 1]);
+                float ref = fkey_inv(skey[x]);
                 if (cont) {  // then nr == 1 and x is the head
                     const float old = smrun[x];
                     ref = fmaxf(ref, old);
                     sfac[x] = (ref == SAR_NEG_INF) ? 1.f : fast_exp(old - ref);
                 }
-                srowf[x * 4 + 2] = ref;
+                sc2[x] = ref;
             }
             __syncwarp();
+            const bool vec4 = a.hvec != 0;
             int i = 0;
-#pragma unroll 2
-            for (int x = lane; x < (npos << lgHp); x += 32) {
-                const int q = x >> lgHp, h = x & (Hp - 1);
+            for (int q = lane; q < npos; q += 32) {
                 while (q >= sso[i + 1] * EPW) ++i;
-                const float ref = srowf[(i * Hp + h) * 4 + 2];
-                sw[x] = (ref == SAR_NEG_INF) ? 0.f : fast_exp(sw[x] - ref);
+                float *wp = reinterpret_cast<float *>(sw) + (q << lgHp);
+                const float *rp = sc2 + i * Hp;
+                if (vec4) {
+                    for (int h = 0; h < H; h += 4) {
+                        float4 e4 = *reinterpret_cast<const float4 *>(wp + h);
+                        const float4 r4 = *reinterpret_cast<const float4 *>(rp + h);
+                        e4.x = fast_exp(e4.x - r4.x);  // rows with edges have a finite reference
+                        e4.y = fast_exp(e4.y - r4.y);
+                        e4.z = fast_exp(e4.z - r4.z);
+                        e4.w = fast_exp(e4.w - r4.w);
+                        *reinterpret_cast<float4 *>(wp + h) = e4;
+                    }
+                } else {
+                    for (int h = 0; h < H; ++h) wp[h] = fast_exp(wp[h] - rp[h]);
+                }
             }
             __syncwarp();
             if (cont) {
@@ -360,7 +435,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                 for (int v = 0; v < V; ++v) {
                     const float c = sfac[hv[v]];
                     sv[v] *= c;
-                    mrun[v] = srowf[hv[v] * 4 + 2];
+                    mrun[v] = sc2[hv[v]];
 #pragma unroll
                     for (int e = 0; e < EPV; ++e) acc0[v][e] *= c;
                 }
@@ -368,17 +443,18 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
         }
 
         // ---- stage D: gather through the cp.async ring ---------------------------------------------
-        auto issue = [&](int s) {
-            const int col = s < nslots ? sj[s * EPW + half] : -1;
+        // Slot s lives in ring stage s % S; lane (half, gl) copies and later reads back its own 16
+        // bytes of edge s*EPW + half, so no cross-lane synchronisation is needed around the ring.
+        auto issue = [&](int s_, uint4 *dst) {
+            const int col = sj[s_ * EPW + half];  // -1 past the row's / chunk's end: zero fill
             const uint4 *src = gbase + (long long)(col < 0 ? 0 : col) * n_vec;
-            uint4 *dst = stage + (size_t)(s % S) * V * 32 + lane;
 #pragma unroll
             for (int v = 0; v < V; ++v)
                 cp_async16(dst + v * 32, src + v * G, (col >= 0 && vok[v]) ? 16 : 0);
             cp_async_commit();
         };
 #pragma unroll
-        for (int s = 0; s < S; ++s) issue(s);
+        for (int s_ = 0; s_ < S; ++s_) issue(s_, stage + (size_t)s_ * V * 32 + lane);
 
         int s = 0;
         for (int ri = 0; ri < nr; ++ri) {
@@ -390,13 +466,14 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
             if (row_starts) {
                 if constexpr (kFwdMode) {
 #pragma unroll
-                    for (int v = 0; v < V; ++v) mrun[v] = srowf[(ri * Hp + hv[v]) * 4 + 2];
+                    for (int v = 0; v < V; ++v) mrun[v] = sc2[ri * Hp + hv[v]];
                 }
                 if constexpr (kDst || kSrc) load_row_vec<T, G, V>(a.rowvec, row, n_vec, gl, vok, rv);
             }
             for (; s < s_end; ++s) {
                 cp_async_wait<S - 1>();  // this lane's copies of slot s have landed
-                const uint4 *src = stage + (size_t)(s % S) * V * 32 + lane;
+                uint4 *src = stage + (size_t)(s % S) * V * 32 + lane;
+                const int wbase = (s * EPW + half) << lgHp;
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
                     float x[EPV];
@@ -404,37 +481,34 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                     if constexpr (MODE == kSum) {
 #pragma unroll
                         for (int e = 0; e < EPV; ++e) acc0[v][e] += x[e];
+                    } else if constexpr (kFwdMode) {
+                        const float w = reinterpret_cast<const float *>(sw)[wbase + hv[v]];
+                        sv[v] += w;
+#pragma unroll
+                        for (int e = 0; e < EPV; ++e) acc0[v][e] = fmaf(w, x[e], acc0[v][e]);
+                    } else if constexpr (kDst) {
+                        const float ws = reinterpret_cast<const float *>(sw)[wbase + hv[v]];
+                        const float al = fabsf(ws);
+                        const float w2 = ws < 0.f ? al * a.slope : al;  // alpha * LeakyReLU'
+                        sv[v] += w2;
+#pragma unroll
+                        for (int e = 0; e < EPV; ++e) {
+                            if constexpr (kAcc0) acc0[v][e] = fmaf(al, x[e], acc0[v][e]);
+                            acc1[v][e] = fmaf(w2, x[e], acc1[v][e]);
+                        }
                     } else {
-                        const int wi = ((s * EPW + half) << lgHp) + hv[v];
-                        if constexpr (kFwdMode) {
-                            const float w = sw[wi];
-                            sv[v] += w;
+                        const float2 w = reinterpret_cast<const float2 *>(sw)[wbase + hv[v]];
+                        const float al = fabsf(w.x);
+                        const float w2 = w.x < 0.f ? al * a.slope : al;
+                        sv[v] += w.y;
 #pragma unroll
-                            for (int e = 0; e < EPV; ++e) acc0[v][e] = fmaf(w, x[e], acc0[v][e]);
-                        } else if constexpr (kDst) {
-                            const float ws = sw[wi];
-                            const float al = fabsf(ws);
-                            const float w2 = ws < 0.f ? al * a.slope : al;  // alpha * LeakyReLU'
-                            sv[v] += w2;
-#pragma unroll
-                            for (int e = 0; e < EPV; ++e) {
-                                if constexpr (kAcc0) acc0[v][e] = fmaf(al, x[e], acc0[v][e]);
-                                acc1[v][e] = fmaf(w2, x[e], acc1[v][e]);
-                            }
-                        } else {
-                            const float2 w = sw[wi];
-                            const float al = fabsf(w.x);
-                            const float w2 = w.x < 0.f ? al * a.slope : al;
-                            sv[v] += w.y;
-#pragma unroll
-                            for (int e = 0; e < EPV; ++e) {
-                                acc0[v][e] = fmaf(al, x[e], acc0[v][e]);
-                                acc1[v][e] = fmaf(w2, x[e], acc1[v][e]);
-                            }
+                        for (int e = 0; e < EPV; ++e) {
+                            acc0[v][e] = fmaf(al, x[e], acc0[v][e]);
+                            acc1[v][e] = fmaf(w2, x[e], acc1[v][e]);
                         }
                     }
                 }
-                issue(s + S);  // refill the stage just consumed (each lane re-uses its own 16 bytes)
+                issue(s + S, src);  // refill the stage just consumed
             }
             if (!row_ends) continue;
 
@@ -545,12 +619,12 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                             DA += scratch[32 * V + lane * a.g.vph + k];
                         }
                         const float Sh = scratch[64 * V + lane];
-                        const float4 c = srowc[ri * Hp + lane];
                         const float D = MODE == kBwdDstGivenD ? a.rec_in[row * H + lane].w : DA;
                         const float val = DB - D * Sh;
                         float *p = a.del + row * H + lane;
                         *p = (a.flags & SAR_FIRST) ? val : *p + val;
-                        if constexpr (MODE == kBwdDst) a.rec_out[row * H + lane] = make_float4(c.x, c.y, c.z, D);
+                        if constexpr (MODE == kBwdDst)
+                            a.rec_out[row * H + lane] = make_float4(sc0[ri * Hp + lane], sc1[ri * Hp + lane], sc2[ri * Hp + lane], D);
                     }
                     __syncwarp();
                 }
