@@ -76,6 +76,66 @@ __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory");
 }
 
+// shared-memory accesses through 32-bit shared-window addresses (no 64-bit pointer arithmetic)
+__device__ __forceinline__ uint4 lds128(unsigned addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float lds_f32(unsigned addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];\n" : "=f"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float2 lds_f32x2(unsigned addr) {
+    float2 v;
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2];\n" : "=f"(v.x), "=f"(v.y) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ int lds_s32(unsigned addr) {
+    int v;
+    asm volatile("ld.shared.s32 %0, [%1];\n" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ void cp_async16_s(unsigned smem_addr, const void *gsrc, int src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(smem_addr), "l"(gsrc), "r"(src_bytes) : "memory");
+}
+
+// packed pairs of float32 (Blackwell's two-wide FP32 pipe: one instruction, two fused multiply-adds)
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};\n" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 p, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;\n" : "=f"(lo), "=f"(hi) : "l"(p));
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {  // a*b + c, element-wise
+    f32x2 r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+// 16 bytes of storage type T -> EPV/2 packed float32 pairs
+template <typename T>
+struct Pairs;
+template <>
+struct Pairs<float> {
+    __device__ __forceinline__ static void get(const uint4 &d, f32x2 (&p)[2]) {
+        p[0] = pack2(__uint_as_float(d.x), __uint_as_float(d.y));
+        p[1] = pack2(__uint_as_float(d.z), __uint_as_float(d.w));
+    }
+};
+template <>
+struct Pairs<__nv_bfloat16> {
+    __device__ __forceinline__ static void get(const uint4 &d, f32x2 (&p)[4]) {
+        p[0] = pack2(__uint_as_float(d.x << 16), __uint_as_float(d.x & 0xffff0000u));
+        p[1] = pack2(__uint_as_float(d.y << 16), __uint_as_float(d.y & 0xffff0000u));
+        p[2] = pack2(__uint_as_float(d.z << 16), __uint_as_float(d.z & 0xffff0000u));
+        p[3] = pack2(__uint_as_float(d.w << 16), __uint_as_float(d.w & 0xffff0000u));
+    }
+};
+
 // Shared-memory layout of one warp (byte offsets).
 struct SpanSmem {
     size_t stage, sj, w, rowc, srb, sso, mrun, fac, scratch, total;
@@ -184,24 +244,35 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
 
     // ---- lane geometry ------------------------------------------------------------------------
     int hv[V];
-    bool vok[V];
+    bool vok[V], lead[V];  // lead: this lane's vector is the first of its head (writes the head's scalars)
 #pragma unroll
     for (int v = 0; v < V; ++v) {
         const int vi = v * G + gl;
         vok[v] = vi < n_vec;
         hv[v] = vok[v] ? vi / a.g.vph : 0;
+        lead[v] = vok[v] && (vi - hv[v] * a.g.vph) == 0;
     }
+    const unsigned stage_s = (unsigned)__cvta_generic_to_shared(stage) + lane * 16;
+    const unsigned sj_s = (unsigned)__cvta_generic_to_shared(sj) + half * 4;
+    unsigned w_s[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+        w_s[v] = (unsigned)__cvta_generic_to_shared(sw) + (((half << lgHp) + hv[v]) * (unsigned)sizeof(W));
     const uint4 *gbase = reinterpret_cast<const uint4 *>(a.gather) + gl;
 
     // ---- per-row accumulators (persist across the chunks of a row longer than CAP) --------------
-    float acc0[V][EPV], acc1[V][EPV], sv[V], mrun[V];
+    constexpr int NP = EPV / 2;
+    f32x2 pacc0[V][NP], pacc1[V][NP];  // packed float32 pairs
+    float sv[V], mrun[V];
     float rv[V][EPV];  // row-stationary vector (bwd)
 #pragma unroll
     for (int v = 0; v < V; ++v) {
         sv[v] = 0.f;
         mrun[v] = SAR_NEG_INF;
 #pragma unroll
-        for (int e = 0; e < EPV; ++e) acc0[v][e] = acc1[v][e] = rv[v][e] = 0.f;
+        for (int k = 0; k < NP; ++k) pacc0[v][k] = pacc1[v][k] = 0ull;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) rv[v][e] = 0.f;
     }
 
     const int deg_l = (lane < nrows && !excluded) ? (int)((ee - eb) > 0x3fffffff ? 0x3fffffff : (ee - eb)) : 0;
@@ -436,8 +507,9 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                     const float c = sfac[hv[v]];
                     sv[v] *= c;
                     mrun[v] = sc2[hv[v]];
+                    const f32x2 c2 = pack2(c, c);
 #pragma unroll
-                    for (int e = 0; e < EPV; ++e) acc0[v][e] *= c;
+                    for (int k = 0; k < NP; ++k) pacc0[v][k] = fma2(pacc0[v][k], c2, 0ull);
                 }
             }
         }
@@ -445,16 +517,15 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
         // ---- stage D: gather through the cp.async ring ---------------------------------------------
         // Slot s lives in ring stage s % S; lane (half, gl) copies and later reads back its own 16
         // bytes of edge s*EPW + half, so no cross-lane synchronisation is needed around the ring.
-        auto issue = [&](int s_, uint4 *dst) {
-            const int col = sj[s_ * EPW + half];  // -1 past the row's / chunk's end: zero fill
+        auto issue = [&](int s_, unsigned dst_s) {
+            const int col = lds_s32(sj_s + s_ * (EPW * 4));  // -1 past the row's / chunk's end: zero fill
             const uint4 *src = gbase + (long long)(col < 0 ? 0 : col) * n_vec;
 #pragma unroll
-            for (int v = 0; v < V; ++v)
-                cp_async16(dst + v * 32, src + v * G, (col >= 0 && vok[v]) ? 16 : 0);
+            for (int v = 0; v < V; ++v) cp_async16_s(dst_s + v * 512, src + v * G, (col >= 0 && vok[v]) ? 16 : 0);
             cp_async_commit();
         };
 #pragma unroll
-        for (int s_ = 0; s_ < S; ++s_) issue(s_, stage + (size_t)s_ * V * 32 + lane);
+        for (int s_ = 0; s_ < S; ++s_) issue(s_, stage_s + s_ * (V * 512));
 
         int s = 0;
         for (int ri = 0; ri < nr; ++ri) {
@@ -472,47 +543,59 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
             }
             for (; s < s_end; ++s) {
                 cp_async_wait<S - 1>();  // this lane's copies of slot s have landed
-                uint4 *src = stage + (size_t)(s % S) * V * 32 + lane;
-                const int wbase = (s * EPW + half) << lgHp;
+                const unsigned src_s = stage_s + (s & (S - 1)) * (V * 512);
+                const unsigned woff = (unsigned)s * (unsigned)((EPW << lgHp) * sizeof(W));
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
-                    float x[EPV];
-                    Elem<T>::unpack(src[v * 32], x);
+                    f32x2 x[NP];
+                    Pairs<T>::get(lds128(src_s + v * 512), x);
                     if constexpr (MODE == kSum) {
+                        const f32x2 one = pack2(1.f, 1.f);
 #pragma unroll
-                        for (int e = 0; e < EPV; ++e) acc0[v][e] += x[e];
+                        for (int k = 0; k < NP; ++k) pacc0[v][k] = fma2(x[k], one, pacc0[v][k]);
                     } else if constexpr (kFwdMode) {
-                        const float w = reinterpret_cast<const float *>(sw)[wbase + hv[v]];
+                        const float w = lds_f32(w_s[v] + woff);
                         sv[v] += w;
+                        const f32x2 w2 = pack2(w, w);
 #pragma unroll
-                        for (int e = 0; e < EPV; ++e) acc0[v][e] = fmaf(w, x[e], acc0[v][e]);
+                        for (int k = 0; k < NP; ++k) pacc0[v][k] = fma2(w2, x[k], pacc0[v][k]);
                     } else if constexpr (kDst) {
-                        const float ws = reinterpret_cast<const float *>(sw)[wbase + hv[v]];
+                        const float ws = lds_f32(w_s[v] + woff);
                         const float al = fabsf(ws);
-                        const float w2 = ws < 0.f ? al * a.slope : al;  // alpha * LeakyReLU'
-                        sv[v] += w2;
+                        const float wg = ws < 0.f ? al * a.slope : al;  // alpha * LeakyReLU'
+                        sv[v] += wg;
+                        const f32x2 a2 = pack2(al, al), g2 = pack2(wg, wg);
 #pragma unroll
-                        for (int e = 0; e < EPV; ++e) {
-                            if constexpr (kAcc0) acc0[v][e] = fmaf(al, x[e], acc0[v][e]);
-                            acc1[v][e] = fmaf(w2, x[e], acc1[v][e]);
+                        for (int k = 0; k < NP; ++k) {
+                            if constexpr (kAcc0) pacc0[v][k] = fma2(a2, x[k], pacc0[v][k]);
+                            pacc1[v][k] = fma2(g2, x[k], pacc1[v][k]);
                         }
                     } else {
-                        const float2 w = reinterpret_cast<const float2 *>(sw)[wbase + hv[v]];
+                        const float2 w = lds_f32x2(w_s[v] + woff);
                         const float al = fabsf(w.x);
-                        const float w2 = w.x < 0.f ? al * a.slope : al;
+                        const float wg = w.x < 0.f ? al * a.slope : al;
                         sv[v] += w.y;
+                        const f32x2 a2 = pack2(al, al), g2 = pack2(wg, wg);
 #pragma unroll
-                        for (int e = 0; e < EPV; ++e) {
-                            acc0[v][e] = fmaf(al, x[e], acc0[v][e]);
-                            acc1[v][e] = fmaf(w2, x[e], acc1[v][e]);
+                        for (int k = 0; k < NP; ++k) {
+                            pacc0[v][k] = fma2(a2, x[k], pacc0[v][k]);
+                            pacc1[v][k] = fma2(g2, x[k], pacc1[v][k]);
                         }
                     }
                 }
-                issue(s + S, src);  // refill the stage just consumed
+                issue(s + S, src_s);  // refill the stage just consumed
             }
             if (!row_ends) continue;
 
             // ---- the row is complete: fold the 32/G edge lanes, finalise, reset --------------------
+            float acc0[V][EPV], acc1[V][EPV];
+#pragma unroll
+            for (int v = 0; v < V; ++v)
+#pragma unroll
+                for (int k = 0; k < NP; ++k) {
+                    unpack2(pacc0[v][k], acc0[v][2 * k], acc0[v][2 * k + 1]);
+                    unpack2(pacc1[v][k], acc1[v][2 * k], acc1[v][2 * k + 1]);
+                }
 #pragma unroll
             for (int off = G; off < 32; off <<= 1) {
 #pragma unroll
@@ -533,7 +616,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                         store_acc_row<G, V, EPV>(rec, gl, vok, acc0);
 #pragma unroll
                         for (int v = 0; v < V; ++v)
-                            if (vok[v] && ((v * G + gl) % a.g.vph) == 0) {
+                            if (lead[v]) {
                                 rec[rowf + hv[v]] = mrun[v];
                                 rec[rowf + H + hv[v]] = sv[v];
                             }
@@ -564,7 +647,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                         if (last_part) {
 #pragma unroll
                             for (int v = 0; v < V; ++v) {
-                                const float inv = sv[v] > 0.f ? 1.f / sv[v] : 0.f;
+                                const float inv = sv[v] > 0.f ? __fdividef(1.f, sv[v]) : 0.f;
 #pragma unroll
                                 for (int e = 0; e < EPV; ++e) acc0[v][e] *= inv;
                             }
@@ -574,7 +657,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                         }
 #pragma unroll
                         for (int v = 0; v < V; ++v)
-                            if (vok[v] && ((v * G + gl) % a.g.vph) == 0) {
+                            if (lead[v]) {
                                 a.m_state[row * H + hv[v]] = mrun[v];
                                 a.d_state[row * H + hv[v]] = sv[v];
                             }
@@ -588,7 +671,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                         if constexpr (MODE == kBwdDst) store_acc_row<G, V, EPV>(rec + rowf, gl, vok, acc0);
 #pragma unroll
                         for (int v = 0; v < V; ++v)
-                            if (vok[v] && ((v * G + gl) % a.g.vph) == 0) rec[2 * rowf + hv[v]] = sv[v];
+                            if (lead[v]) rec[2 * rowf + hv[v]] = sv[v];
                     }
                 } else {
                     float pA[V], pB[V];
@@ -608,7 +691,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                             if (vok[v]) {
                                 scratch[v * G + gl] = pB[v];
                                 scratch[32 * V + v * G + gl] = pA[v];
-                                if (((v * G + gl) % a.g.vph) == 0) scratch[64 * V + hv[v]] = sv[v];
+                                if (lead[v]) scratch[64 * V + hv[v]] = sv[v];
                             }
                     }
                     __syncwarp();
@@ -636,7 +719,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                         store_acc_row<G, V, EPV>(rec + rowf, gl, vok, acc1);
 #pragma unroll
                         for (int v = 0; v < V; ++v)
-                            if (vok[v] && ((v * G + gl) % a.g.vph) == 0) rec[2 * rowf + hv[v]] = sv[v];
+                            if (lead[v]) rec[2 * rowf + hv[v]] = sv[v];
                     }
                 } else {
                     float pC[V];
@@ -652,7 +735,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                         for (int v = 0; v < V; ++v)
                             if (vok[v]) {
                                 scratch[v * G + gl] = pC[v];
-                                if (((v * G + gl) % a.g.vph) == 0) scratch[64 * V + hv[v]] = sv[v];
+                                if (lead[v]) scratch[64 * V + hv[v]] = sv[v];
                             }
                     }
                     __syncwarp();
@@ -691,7 +774,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                 sv[v] = 0.f;
                 mrun[v] = SAR_NEG_INF;
 #pragma unroll
-                for (int e = 0; e < EPV; ++e) acc0[v][e] = acc1[v][e] = 0.f;
+                for (int k = 0; k < NP; ++k) pacc0[v][k] = pacc1[v][k] = 0ull;
             }
         }
         cp_async_wait<0>();  // drain the (zero-size) refills issued past the last slot
@@ -700,7 +783,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
             if (unfinished && half == 0) {
 #pragma unroll
                 for (int v = 0; v < V; ++v)
-                    if (vok[v] && ((v * G + gl) % a.g.vph) == 0) smrun[hv[v]] = mrun[v];
+                    if (lead[v]) smrun[hv[v]] = mrun[v];
             }
         }
         __syncwarp();
