@@ -1,5 +1,7 @@
-// Fused GAT aggregation kernels (forward, destination-major backward, source-major backward,
-// row-dot preparation) built on the row-stationary skeleton of sar_rowkernels.cuh (internal).
+// Kernels around the span kernels of sar_span_kernels.cuh (internal): the merges of the long-row
+// segments (forward, destination-major backward, source-major backward, sum) and the row-dot
+// preparation of the per-partition backward.  One group of G lanes per row, lane gl / slot v holding
+// the 16-byte vector v*G + gl of the row.
 #pragma once
 
 #include "sar_rowkernels.cuh"
@@ -7,9 +9,10 @@
 namespace sar {
 
 // ------------------------------------------------------------------------------------------------
-// Forward: scores, online softmax and weighted neighbour sum in one pass (Eq. 3, Sec. 3.3), with
-// the running-max correction of Sec. 3.4 applied batch by batch (and partition by partition when
-// the state comes from / goes to global memory, Algorithm 1).
+// Forward merge: the segments of a long row are folded with the running-max correction of Sec. 3.4
+// (exp(old_max - new_max) on numerator and normaliser), starting from the state left by earlier
+// partitions unless SAR_FIRST (Algorithm 1).
+// Partial record of a segment in the workspace: [rowf floats numerator][H max][H normaliser].
 // ------------------------------------------------------------------------------------------------
 struct FwdArgs {
     long long n_dst;
@@ -28,119 +31,6 @@ struct FwdArgs {
     SplitArgs sp;
     int mode;           // 0: one group per row; 1: one group per long-row segment
 };
-
-// Partial record of a forward segment in the workspace: [rowf floats numerator][H max][H norm].
-template <typename T, int G, int V, int U>
-__global__ void __launch_bounds__(kThreads) gat_fwd_kernel(const FwdArgs a) {
-    constexpr int EPV = Elem<T>::EPV;
-    constexpr int RPW = 32 / G;
-    extern __shared__ __align__(16) float smem[];
-    const LaneId<G> id;
-    const int H = a.g.H, Hp = a.g.Hp;
-    float *wbase = smem + (size_t)id.warp * warp_smem_floats(Hp, V, 1);
-    int *sj = reinterpret_cast<int *>(wbase) + id.gid * G;
-    float *sc = wbase + 32 + id.gid * Hp;
-    float *sw = wbase + 64 + (size_t)id.gid * G * Hp;
-
-    const long long item = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
-    WorkItem w = locate_work(item, a.n_dst, a.indptr, a.sp, a.mode);
-    const bool first = (a.flags & SAR_FIRST) || a.mode == 1;
-    const bool last = (a.flags & SAR_LAST) && a.mode == 0;
-    if (a.mode == 0 && w.active && !(a.flags & SAR_FIRST) && !(a.flags & SAR_LAST) && w.beg == w.end)
-        w.active = false;  // nothing to fold in, state stays as it is
-
-    const VecGeom<G, V> vg(a.g, id.gl);
-    const int sh = id.gl & (Hp - 1);        // head this lane scores
-    const int se0 = id.gl >> a.g.lgHp;      // first edge of the batch this lane scores
-    const int epi = G >> a.g.lgHp;          // edges scored per sweep of the group
-    const bool sh_ok = sh < H;
-
-    float el_i = 0.f, Mrun = SAR_NEG_INF;
-    float dv[V];
-    float acc[V][EPV];
-#pragma unroll
-    for (int v = 0; v < V; ++v) {
-        dv[v] = 0.f;
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) acc[v][e] = 0.f;
-    }
-    if (w.active) {
-        if (sh_ok) el_i = __ldg(a.el + w.row * H + sh);
-        if (!first) {
-            if (sh_ok) Mrun = a.m[w.row * H + sh];
-#pragma unroll
-            for (int v = 0; v < V; ++v)
-                if (vg.vok[v]) dv[v] = a.d[w.row * H + vg.hv[v]];
-            load_acc_row<G, V, EPV>(a.acc + w.row * (long long)(a.g.n_vec * EPV), id.gl, vg.vok, acc);
-        }
-    }
-
-    const int nbatch = (int)((w.end - w.beg + G - 1) / G);
-    const int wmax = __reduce_max_sync(0xffffffffu, nbatch);
-    const uint4 *featv = reinterpret_cast<const uint4 *>(a.feat);
-    for (int it = 0; it < wmax; ++it) {
-        const long long b0 = w.beg + (long long)it * G;
-        const long long rem = w.end - b0;
-        const int nb = rem <= 0 ? 0 : (rem < G ? (int)rem : G);
-        sj[id.gl] = id.gl < nb ? ld_stream_i32(a.indices + b0 + id.gl) : 0;
-        __syncwarp();
-        // SCORE, sweep 1: e = LeakyReLU(el_i + er_j) per (edge, head); batch max per head
-        float lm = SAR_NEG_INF;
-        if (sh_ok)
-            for (int k = se0; k < nb; k += epi) {
-                float gr;
-                const float e = leaky(el_i + __ldg(a.er + (long long)sj[k] * H + sh), a.slope, gr);
-                sw[k * Hp + sh] = e;
-                lm = fmaxf(lm, e);
-            }
-        for (int off = Hp; off < G; off <<= 1) lm = fmaxf(lm, __shfl_xor_sync(0xffffffffu, lm, off));
-        const float Mn = fmaxf(Mrun, lm);
-        const float c = (Mn == SAR_NEG_INF) ? 1.f : fast_exp(Mrun - Mn);  // exp(old_max - new_max)
-        Mrun = Mn;
-        if (id.gl < Hp) sc[id.gl] = c;
-        // SCORE, sweep 2: un-normalised weights exp(e - running max)
-        if (sh_ok)
-            for (int k = se0; k < nb; k += epi) sw[k * Hp + sh] = fast_exp(sw[k * Hp + sh] - Mn);
-        __syncwarp();
-        // correct what has been accumulated so far, then GATHER
-#pragma unroll
-        for (int v = 0; v < V; ++v) {
-            const float cv = sc[vg.hv[v]];
-            dv[v] *= cv;
-#pragma unroll
-            for (int e = 0; e < EPV; ++e) acc[v][e] *= cv;
-        }
-        gather_batch<T, G, V, U, kFwd>(featv, a.g.n_vec, sj, sw, Hp, nb, id.gl, vg.hv, vg.vok, acc, acc, dv);
-        __syncwarp();
-    }
-
-    if (!w.active) return;
-    const long long rowf = (long long)a.g.n_vec * EPV;
-    if (a.mode == 1) {
-        float *rec = a.sp.part + w.seg * a.sp.pstride;
-        store_acc_row<G, V, EPV>(rec, id.gl, vg.vok, acc);
-        if (id.gl < H) rec[rowf + id.gl] = Mrun;
-#pragma unroll
-        for (int v = 0; v < V; ++v)
-            if (vg.vok[v] && ((v * G + id.gl) % a.g.vph) == 0) rec[rowf + H + vg.hv[v]] = dv[v];
-        return;
-    }
-    if (last) {
-#pragma unroll
-        for (int v = 0; v < V; ++v) {
-            const float inv = dv[v] > 0.f ? 1.f / dv[v] : 0.f;
-#pragma unroll
-            for (int e = 0; e < EPV; ++e) acc[v][e] *= inv;
-        }
-        store_row_vec<T, G, V>(a.out, w.row, a.g.n_vec, id.gl, vg.vok, acc);
-    } else {
-        store_acc_row<G, V, EPV>(a.acc + w.row * rowf, id.gl, vg.vok, acc);
-    }
-    if (id.gl < H) a.m[w.row * H + id.gl] = Mrun;
-#pragma unroll
-    for (int v = 0; v < V; ++v)
-        if (vg.vok[v] && ((v * G + id.gl) % a.g.vph) == 0) a.d[w.row * H + vg.hv[v]] = dv[v];
-}
 
 // Merge of the forward partials of the long rows: one group per long row folds its segments in
 // order with the same running-max rule, starting from the incoming state unless SAR_FIRST.
@@ -279,78 +169,6 @@ __device__ __forceinline__ void bwd_dst_epilogue(const BwdDstArgs &a, const Lane
     }
 }
 
-template <typename T, int G, int V, int U, bool GIVEN_D>
-__global__ void __launch_bounds__(kThreads) gat_bwd_dst_kernel(const BwdDstArgs a) {
-    constexpr int EPV = Elem<T>::EPV;
-    constexpr int RPW = 32 / G;
-    constexpr int MODE = GIVEN_D ? kBwdDstGivenD : kBwdDst;
-    extern __shared__ __align__(16) float smem[];
-    const LaneId<G> id;
-    const int H = a.g.H, Hp = a.g.Hp;
-    float *wbase = smem + (size_t)id.warp * warp_smem_floats(Hp, V, 2);
-    int *sj = reinterpret_cast<int *>(wbase) + id.gid * G;
-    float2 *sw = reinterpret_cast<float2 *>(wbase + 64) + (size_t)id.gid * G * Hp;
-    float *scratch = wbase + 64 + id.gid * (G * V);
-
-    const long long item = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
-    WorkItem w = locate_work(item, a.n_dst, a.indptr, a.sp, a.mode);
-    if (a.mode == 0 && w.active && !(a.flags & SAR_FIRST) && GIVEN_D && w.beg == w.end) w.active = false;
-
-    const VecGeom<G, V> vg(a.g, id.gl);
-    const int sh = id.gl & (Hp - 1), se0 = id.gl >> a.g.lgHp, epi = G >> a.g.lgHp;
-    const bool sh_ok = sh < H;
-
-    float el_i = 0.f, m_i = 0.f, invd_i = 0.f;
-    float gv[V][EPV], accA[V][EPV], accB[V][EPV], S[V];
-#pragma unroll
-    for (int v = 0; v < V; ++v) {
-        S[v] = 0.f;
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) gv[v][e] = accA[v][e] = accB[v][e] = 0.f;
-    }
-    if (w.active && sh_ok && w.end > w.beg) {
-        el_i = __ldg(a.el + w.row * H + sh);
-        m_i = __ldg(a.m + w.row * H + sh);
-        const float dd = __ldg(a.d + w.row * H + sh);
-        invd_i = dd > 0.f ? 1.f / dd : 0.f;
-    }
-
-    const int nbatch = (int)((w.end - w.beg + G - 1) / G);
-    const int wmax = __reduce_max_sync(0xffffffffu, nbatch);
-    const uint4 *featv = reinterpret_cast<const uint4 *>(a.feat);
-    for (int it = 0; it < wmax; ++it) {
-        const long long b0 = w.beg + (long long)it * G;
-        const long long rem = w.end - b0;
-        const int nb = rem <= 0 ? 0 : (rem < G ? (int)rem : G);
-        sj[id.gl] = id.gl < nb ? ld_stream_i32(a.indices + b0 + id.gl) : 0;
-        __syncwarp();
-        if (sh_ok)
-            for (int k = se0; k < nb; k += epi) {
-                float gr;
-                const float e = leaky(el_i + __ldg(a.er + (long long)sj[k] * H + sh), a.slope, gr);
-                const float al = fast_exp(e - m_i) * invd_i;  // rematerialised attention coefficient
-                sw[k * Hp + sh] = make_float2(al, al * gr);
-            }
-        __syncwarp();
-        gather_batch<T, G, V, U, MODE>(featv, a.g.n_vec, sj, sw, Hp, nb, id.gl, vg.hv, vg.vok, accA, accB, S);
-        __syncwarp();
-    }
-
-    if (a.mode == 1) {
-        if (!w.active) return;
-        const long long rowf = (long long)a.g.n_vec * EPV;
-        float *recp = a.sp.part + w.seg * a.sp.pstride;
-        store_acc_row<G, V, EPV>(recp, id.gl, vg.vok, accB);
-        if constexpr (!GIVEN_D) store_acc_row<G, V, EPV>(recp + rowf, id.gl, vg.vok, accA);
-#pragma unroll
-        for (int v = 0; v < V; ++v)
-            if (vg.vok[v] && ((v * G + id.gl) % a.g.vph) == 0) recp[2 * rowf + vg.hv[v]] = S[v];
-        return;
-    }
-    if (w.active) load_row_vec<T, G, V>(a.gout, w.row, a.g.n_vec, id.gl, vg.vok, gv);
-    bwd_dst_epilogue<T, G, V, GIVEN_D>(a, id, vg, scratch, w.active ? w.row : -1, gv, accA, accB, S);
-}
-
 template <typename T, int G, int V, bool GIVEN_D>
 __global__ void __launch_bounds__(kThreads) gat_bwd_dst_merge_kernel(const BwdDstArgs a) {
     constexpr int EPV = Elem<T>::EPV;
@@ -433,71 +251,6 @@ __device__ __forceinline__ void bwd_src_epilogue(const BwdSrcArgs &a, const Lane
     const float DC = head_sum<G, V>(scratch, pC, vg.vok, id.gl, a.g);
     const float Sh = head_scalar<G, V>(scratch, S, vg.hv, vg.vok, id.gl, a.g);
     if (row >= 0 && id.gl < a.g.H) a.der[row * a.g.H + id.gl] = DC - Sh;
-}
-
-template <typename T, int G, int V, int U>
-__global__ void __launch_bounds__(kThreads) gat_bwd_src_kernel(const BwdSrcArgs a) {
-    constexpr int EPV = Elem<T>::EPV;
-    constexpr int RPW = 32 / G;
-    extern __shared__ __align__(16) float smem[];
-    const LaneId<G> id;
-    const int H = a.g.H, Hp = a.g.Hp;
-    float *wbase = smem + (size_t)id.warp * warp_smem_floats(Hp, V, 4);
-    int *si = reinterpret_cast<int *>(wbase) + id.gid * G;
-    float4 *sw = reinterpret_cast<float4 *>(wbase + 64) + (size_t)id.gid * G * Hp;
-    float *scratch = wbase + 64 + id.gid * (G * V);
-
-    const long long item = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
-    const WorkItem w = locate_work(item, a.n_src, a.t_indptr, a.sp, a.mode);
-    const VecGeom<G, V> vg(a.g, id.gl);
-    const int sh = id.gl & (Hp - 1), se0 = id.gl >> a.g.lgHp, epi = G >> a.g.lgHp;
-    const bool sh_ok = sh < H;
-
-    float er_j = 0.f;
-    float accD[V][EPV], accC[V][EPV], S[V];
-#pragma unroll
-    for (int v = 0; v < V; ++v) {
-        S[v] = 0.f;
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) accD[v][e] = accC[v][e] = 0.f;
-    }
-    if (w.active && sh_ok) er_j = __ldg(a.er + w.row * H + sh);
-
-    const int nbatch = (int)((w.end - w.beg + G - 1) / G);
-    const int wmax = __reduce_max_sync(0xffffffffu, nbatch);
-    const uint4 *goutv = reinterpret_cast<const uint4 *>(a.gout);
-    for (int it = 0; it < wmax; ++it) {
-        const long long b0 = w.beg + (long long)it * G;
-        const long long rem = w.end - b0;
-        const int nb = rem <= 0 ? 0 : (rem < G ? (int)rem : G);
-        si[id.gl] = id.gl < nb ? ld_stream_i32(a.t_indices + b0 + id.gl) : 0;
-        __syncwarp();
-        if (sh_ok)
-            for (int k = se0; k < nb; k += epi) {
-                const float4 r = __ldg(a.rec + (long long)si[k] * H + sh);  // {el_i, m_i, 1/d_i, D_i}
-                float gr;
-                const float e = leaky(r.x + er_j, a.slope, gr);
-                const float al = fast_exp(e - r.y) * r.z;
-                const float w2 = al * gr;
-                sw[k * Hp + sh] = make_float4(al, w2, w2 * r.w, 0.f);
-            }
-        __syncwarp();
-        gather_batch<T, G, V, U, kBwdSrc>(goutv, a.g.n_vec, si, sw, Hp, nb, id.gl, vg.hv, vg.vok, accD, accC, S);
-        __syncwarp();
-    }
-
-    if (a.mode == 1) {
-        if (!w.active) return;
-        const long long rowf = (long long)a.g.n_vec * EPV;
-        float *recp = a.sp.part + w.seg * a.sp.pstride;
-        store_acc_row<G, V, EPV>(recp, id.gl, vg.vok, accD);
-        store_acc_row<G, V, EPV>(recp + rowf, id.gl, vg.vok, accC);
-#pragma unroll
-        for (int v = 0; v < V; ++v)
-            if (vg.vok[v] && ((v * G + id.gl) % a.g.vph) == 0) recp[2 * rowf + vg.hv[v]] = S[v];
-        return;
-    }
-    bwd_src_epilogue<T, G, V>(a, id, vg, scratch, w.active ? w.row : -1, accD, accC, S);
 }
 
 template <typename T, int G, int V>
@@ -624,45 +377,6 @@ __device__ __forceinline__ void sum_epilogue(const SumArgs &a, int gl, const Vec
             for (int e = 0; e < EPV; ++e) acc[v][e] *= inv;
     }
     store_row_vec<T, G, V>(a.out, row, a.g.n_vec, gl, vg.vok, acc);
-}
-
-template <typename T, int G, int V, int U>
-__global__ void __launch_bounds__(kThreads) spmm_kernel(const SumArgs a) {
-    constexpr int EPV = Elem<T>::EPV;
-    constexpr int RPW = 32 / G;
-    extern __shared__ __align__(16) float smem[];
-    const LaneId<G> id;
-    int *sj = reinterpret_cast<int *>(smem) + id.warp * 32 + id.gid * G;
-    const long long item = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
-    WorkItem w = locate_work(item, a.n_dst, a.indptr, a.sp, a.mode);
-    const bool must_write = (a.flags & SAR_FIRST) || ((a.flags & SAR_MEAN) && (a.flags & SAR_LAST));
-    if (a.mode == 0 && w.active && !must_write && w.beg == w.end) w.active = false;
-    const VecGeom<G, V> vg(a.g, id.gl);
-    float acc[V][EPV], dummy[V];
-#pragma unroll
-    for (int v = 0; v < V; ++v) {
-        dummy[v] = 0.f;
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) acc[v][e] = 0.f;
-    }
-    const int nbatch = (int)((w.end - w.beg + G - 1) / G);
-    const int wmax = __reduce_max_sync(0xffffffffu, nbatch);
-    const uint4 *featv = reinterpret_cast<const uint4 *>(a.feat);
-    for (int it = 0; it < wmax; ++it) {
-        const long long b0 = w.beg + (long long)it * G;
-        const long long rem = w.end - b0;
-        const int nb = rem <= 0 ? 0 : (rem < G ? (int)rem : G);
-        sj[id.gl] = id.gl < nb ? ld_stream_i32(a.indices + b0 + id.gl) : 0;
-        __syncwarp();
-        gather_batch<T, G, V, U, kSum>(featv, a.g.n_vec, sj, nullptr, 1, nb, id.gl, vg.hv, vg.vok, acc, acc, dummy);
-        __syncwarp();
-    }
-    if (!w.active) return;
-    if (a.mode == 1) {
-        store_acc_row<G, V, EPV>(a.sp.part + w.seg * a.sp.pstride, id.gl, vg.vok, acc);
-        return;
-    }
-    sum_epilogue<T, G, V>(a, id.gl, vg, w.row, acc);
 }
 
 template <typename T, int G, int V>

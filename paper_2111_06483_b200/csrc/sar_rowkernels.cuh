@@ -1,20 +1,10 @@
-// Row-stationary gather kernels of libsar (internal).
+// Row geometry shared by the kernels of libsar (internal).
 //
-// One skeleton serves the forward pass, both backward passes and the sum aggregation:
-//   a GROUP of G lanes (G = 4..32, a power of two) owns one row of the traversal (a destination
-//   for the CSR passes, a source for the CSC pass); lane gl, slot v holds the 16-byte vector
-//   vi = v*G + gl of the H*F-wide row, so that one warp instruction fetches G consecutive
-//   vectors (coalesced 128-bit gathers) of 32/G different neighbour rows.
-//   The row's edges are consumed in batches of G:
-//     1. each lane loads one column index of the batch (coalesced) into shared memory;
-//     2. SCORE phase: the (edge, head) pairs of the batch are spread over the lanes, each pair's
-//        weight(s) are computed ONCE (one exponential per pair) and parked in shared memory;
-//     3. GATHER phase: every lane walks the batch, fetches its vectors of each neighbour row and
-//        accumulates them, scaled by the weight of the vector's head, in float32 registers.
-//   Nothing per edge is ever written to global memory.
-//   Rows longer than `threshold` edges are cut into segments processed by other groups in a
-//   second launch of the same kernel (mode 1), which parks partial accumulators in a workspace; a
-//   third launch merges them.  No atomics anywhere: every output element has one writer.
+// A feature row of H*F elements is n_vec 16-byte vectors.  A GROUP of G lanes (G = 4..32, a power of
+// two) covers one row: lane gl, slot v holds the vector vi = v*G + gl, so that one warp instruction
+// moves G consecutive vectors (coalesced 128-bit accesses) of 32/G different rows.  Vector vi belongs
+// to head vi / vph.  Float32 accumulator rows in global memory (running numerator, long-row partials)
+// use the same mapping with EPV floats per vector.
 #pragma once
 
 #include "sar_common.cuh"
@@ -74,47 +64,6 @@ struct VecGeom {
         }
     }
 };
-
-// Which (row, edge range) does this group work on?  mode 0: row = item, whole row unless it is
-// long (then skipped, the segment launch covers it); mode 1: item is a segment of a long row.
-struct WorkItem {
-    bool active;
-    long long row;
-    long long beg, end;
-    long long seg;
-};
-
-__device__ __forceinline__ WorkItem locate_work(long long item, long long n_rows, const int64_t *__restrict__ indptr,
-                                                const SplitArgs &sp, int mode) {
-    WorkItem w;
-    w.active = false;
-    w.row = 0;
-    w.beg = w.end = 0;
-    w.seg = -1;
-    if (mode == 0) {
-        if (item < n_rows) {
-            w.row = item;
-            w.beg = __ldg(indptr + item);
-            w.end = __ldg(indptr + item + 1);
-            w.active = !(sp.threshold > 0 && w.end - w.beg > sp.threshold);
-        }
-    } else if (item < sp.n_seg) {
-        int lo = 0, hi = sp.n_long;  // last lr with long_seg[lr] <= item
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (__ldg(sp.long_seg + mid) <= item) lo = mid; else hi = mid;
-        }
-        w.row = __ldg(sp.long_row + lo);
-        const long long c = item - __ldg(sp.long_seg + lo);
-        const long long rb = __ldg(indptr + w.row), re = __ldg(indptr + w.row + 1);
-        w.beg = rb + c * sp.threshold;
-        w.end = w.beg + sp.threshold < re ? w.beg + sp.threshold : re;
-        w.seg = item;
-        w.active = true;
-    }
-    if (!w.active) w.beg = w.end = 0;
-    return w;
-}
 
 // float32 accumulator rows in global memory (running numerator, partials): lane's slot v covers
 // floats [(v*G+gl)*EPV, +EPV).
@@ -191,86 +140,6 @@ __device__ __forceinline__ void store_row_vec(void *base, long long row, int n_v
 #pragma unroll
     for (int v = 0; v < V; ++v)
         if (vok[v]) rp[v * G + gl] = Elem<T>::pack(r[v]);
-}
-
-// GATHER phase over one batch of nb (<= G) edges of this group.
-//   sjg: the batch's column ids; swg: the batch's weights, [edge][Hp].
-//   kFwd:           acc0 += w * x,                    s += w
-//   kBwdDst:        acc0 += w.x * x, acc1 += w.y * x, s += w.y
-//   kBwdDstGivenD:                   acc1 += w.y * x, s += w.y
-//   kBwdSrc:        acc0 += w.x * x, acc1 += w.y * x, s += w.z
-//   kSum:           acc0 += x
-template <typename T, int G, int V, int U, int MODE>
-__device__ __forceinline__ void gather_batch(const uint4 *__restrict__ base, int n_vec, const int *sjg,
-                                             const typename WeightOf<MODE>::type *swg, int Hp, int nb, int gl,
-                                             const int (&hv)[V], const bool (&vok)[V],
-                                             float (&acc0)[V][Elem<T>::EPV], float (&acc1)[V][Elem<T>::EPV],
-                                             float (&s)[V]) {
-    constexpr int EPV = Elem<T>::EPV;
-    using W = typename WeightOf<MODE>::type;
-    for (int k0 = 0; k0 < nb; k0 += U) {
-        uint4 buf[U][V];
-        W w[U][V];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int kk = k0 + u;
-            const bool ok = kk < nb;
-            const int jj = sjg[ok ? kk : k0];
-            const uint4 *rp = base + (long long)jj * n_vec + gl;
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                buf[u][v] = make_uint4(0, 0, 0, 0);
-                if (ok && vok[v]) buf[u][v] = ldg16(rp + v * G);
-            }
-            if constexpr (MODE != kSum) {
-#pragma unroll
-                for (int v = 0; v < V; ++v) {
-                    const W ww = swg[(ok ? kk : k0) * Hp + hv[v]];
-                    if constexpr (MODE == kFwd) {
-                        w[u][v] = ok ? ww : 0.f;
-                    } else if constexpr (MODE == kBwdSrc) {
-                        w[u][v] = ok ? ww : make_float4(0.f, 0.f, 0.f, 0.f);
-                    } else {
-                        w[u][v] = ok ? ww : make_float2(0.f, 0.f);
-                    }
-                }
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-#pragma unroll
-            for (int v = 0; v < V; ++v) {
-                float x[EPV];
-                Elem<T>::unpack(buf[u][v], x);
-                if constexpr (MODE == kFwd) {
-                    s[v] += w[u][v];
-#pragma unroll
-                    for (int e = 0; e < EPV; ++e) acc0[v][e] = fmaf(w[u][v], x[e], acc0[v][e]);
-                } else if constexpr (MODE == kBwdDst) {
-                    s[v] += w[u][v].y;
-#pragma unroll
-                    for (int e = 0; e < EPV; ++e) {
-                        acc0[v][e] = fmaf(w[u][v].x, x[e], acc0[v][e]);
-                        acc1[v][e] = fmaf(w[u][v].y, x[e], acc1[v][e]);
-                    }
-                } else if constexpr (MODE == kBwdDstGivenD) {
-                    s[v] += w[u][v].y;
-#pragma unroll
-                    for (int e = 0; e < EPV; ++e) acc1[v][e] = fmaf(w[u][v].y, x[e], acc1[v][e]);
-                } else if constexpr (MODE == kBwdSrc) {
-                    s[v] += w[u][v].z;
-#pragma unroll
-                    for (int e = 0; e < EPV; ++e) {
-                        acc0[v][e] = fmaf(w[u][v].x, x[e], acc0[v][e]);
-                        acc1[v][e] = fmaf(w[u][v].y, x[e], acc1[v][e]);
-                    }
-                } else {
-#pragma unroll
-                    for (int e = 0; e < EPV; ++e) acc0[v][e] += x[e];
-                }
-            }
-        }
-    }
 }
 
 // Per-head sum of per-lane partial dot products, through shared memory: lane (gl, v) deposits its

@@ -1,0 +1,158 @@
+"""GPU parity at the full sizes of the named workloads, in the launch configuration bench.py times
+(fused calls over the K partitions of the un-split graph, long-row plan with the default threshold).
+
+The oracle cannot run 300 M edges in test time, so outputs are SAMPLED: a sub-problem that contains
+every edge the sampled outputs depend on is cut out with torch indexing, handed to the oracle, and
+compared element by element; invariants that hold at any size cover the rest.
+  forward / del : sampled destinations with ALL their in-edges (out, m, d, del depend on nothing else)
+  dfeat / der   : sampled sources with all their out-edges, plus, for every destination those edges
+                  reach, ALL of its in-edges (so that the softmax statistics of the sub-problem are exact)
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import workloads
+from helpers import allclose_report
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from paper_2111_06483_b200 import api
+
+DEV = "cuda"
+
+
+def _rows_subgraph(indptr, indices, rows):
+    """CSR restricted to `rows` (device tensors): returns (sub_indptr[len(rows)+1], cols) on the device."""
+    deg = indptr[rows + 1] - indptr[rows]
+    sub_indptr = torch.zeros(rows.numel() + 1, dtype=torch.int64, device=rows.device)
+    sub_indptr[1:] = torch.cumsum(deg, 0)
+    total = int(sub_indptr[-1])
+    owner = torch.repeat_interleave(torch.arange(rows.numel(), device=rows.device), deg)
+    pos = torch.arange(total, device=rows.device) - sub_indptr[owner] + indptr[rows][owner]
+    return sub_indptr, indices[pos].long()
+
+
+def _tol(dtype, want, grad=False):
+    x = np.asarray(want, dtype=np.float64)
+    scale = max(float(np.sqrt(np.mean(x * x))) if x.size else 0.0, 1.0)
+    if dtype == "bf16":
+        return dict(rtol=2e-2, atol=2e-2 * scale)
+    return dict(rtol=1e-4, atol=1e-5 * scale) if grad else dict(rtol=1e-5, atol=1e-6)
+
+
+@pytest.mark.parametrize("name,dtype", [("seqpart", "f32"), ("medium", "f32"), ("medium", "bf16"), ("dense", "bf16"),
+                                        ("large", "bf16")])
+def test_sampled_rows_at_full_size(name, dtype):
+    cfg = workloads.CONFIGS[name]
+    n, H, F = cfg.n, cfg.heads, cfg.feat
+    need = (4 * n * H * F * (2 if dtype == "bf16" else 4) + 24 * cfg.e) * 1.5
+    if torch.cuda.get_device_properties(0).total_memory < need:
+        pytest.skip("not enough device memory for this workload")
+    src, dst = workloads.make_graph(cfg, device=DEV)
+    g = api.Graph.from_coo(n, src, dst, k=cfg.k)
+    del src, dst
+    t = workloads.make_node_inputs(n, H, F, cfg.seed, dtype=dtype, device=DEV)
+    feat, gout, el, er = t["feat"], t["gout"], t["el"], t["er"]
+    out, m, d = api.gat_forward(g, feat, el, er, cfg.slope)
+    dfeat, del_, der = api.gat_backward(g, feat, el, er, m, d, gout, cfg.slope)
+    torch.cuda.synchronize()
+    W = g.whole
+    in_deg = W.indptr[1:] - W.indptr[:-1]
+    out_deg = W.t_indptr[1:] - W.t_indptr[:-1]
+
+    # ---- invariants over the whole arrays ----------------------------------------------------------
+    assert torch.isfinite(out.float()).all() and torch.isfinite(dfeat.float()).all()
+    empty = in_deg == 0
+    assert (d[empty] == 0).all() and torch.isneginf(m[empty]).all() and (out[empty] == 0).all()
+    assert (d[~empty] >= 1.0 - 1e-5).all()                      # the max term contributes exp(0) = 1
+    s_del, s_der = del_.double().sum(0), der.double().sum(0)      # two groupings of the same per-edge terms
+    scale = float(del_.double().abs().sum(0).max())
+    assert float((s_del - s_der).abs().max()) <= (2e-2 if dtype == "bf16" else 1e-4) * max(scale, 1.0) ** 0.5 * 50
+    want_sum = gout[~empty].double().sum(0)                       # every edge hands alpha*gout to its source
+    got_sum = dfeat.double().sum(0)
+    tol = (2e-2 if dtype == "bf16" else 1e-4) * float(gout.double().abs().sum(0).max()) ** 0.5 * 50
+    assert float((got_sum - want_sum).abs().max()) <= tol
+
+    # ---- sampled destinations: out, m, d, del --------------------------------------------------------
+    gen = torch.Generator(device="cpu").manual_seed(cfg.seed + 100)
+    rows = torch.randperm(n, generator=gen)[:3000].to(DEV)
+    hubs = torch.topk(in_deg, 3).indices                          # the longest rows go through the segment path
+    rows = torch.unique(torch.cat([rows, hubs]))
+    sub_indptr, cols = _rows_subgraph(W.indptr, W.indices, rows)
+    ucols, inv = torch.unique(cols, return_inverse=True)
+    f_sub = feat[ucols].float().cpu().numpy()
+    fwd = oracle.gat_fwd(sub_indptr.cpu().numpy(), inv.cpu().numpy().astype(np.int32), f_sub,
+                         el[rows].cpu().numpy(), er[ucols].cpu().numpy(), cfg.slope)
+    allclose_report(out[rows].float().cpu().numpy(), fwd.out, what="out", **_tol(dtype, fwd.out))
+    allclose_report(m[rows].cpu().numpy(), fwd.m, 1e-6, 1e-6, "m")
+    allclose_report(d[rows].cpu().numpy(), fwd.d, 1e-5, 1e-6, "d")
+    bwd = oracle.gat_bwd(sub_indptr.cpu().numpy(), inv.cpu().numpy().astype(np.int32), f_sub,
+                         el[rows].cpu().numpy(), er[ucols].cpu().numpy(), fwd.alpha,
+                         gout[rows].float().cpu().numpy(), cfg.slope)
+    allclose_report(del_[rows].cpu().numpy(), bwd.del_, what="del", **_tol(dtype, bwd.del_, grad=True))
+
+    # ---- sampled sources: dfeat, der (two-hop sub-problem) -------------------------------------------
+    avg_deg = cfg.e / n
+    srcs = torch.randperm(n, generator=gen)[:max(3, int(2000 / avg_deg))].to(DEV)
+    if avg_deg < 50:                                             # and a couple of busy sources
+        mid = torch.nonzero((out_deg > 200) & (out_deg < 3000)).flatten()[:2]
+        srcs = torch.cat([srcs, mid])
+    srcs = torch.unique(srcs)
+    _, reached = _rows_subgraph(W.t_indptr, W.t_indices, srcs)
+    drows = torch.unique(reached)
+    sub_indptr, cols = _rows_subgraph(W.indptr, W.indices, drows)
+    assert sub_indptr[-1] < 40_000_000, "sample grew too large for the oracle"
+    ucols, inv = torch.unique(cols, return_inverse=True)
+    f_sub = feat[ucols].float().cpu().numpy()
+    ip, ix = sub_indptr.cpu().numpy(), inv.cpu().numpy().astype(np.int32)
+    fwd = oracle.gat_fwd(ip, ix, f_sub, el[drows].cpu().numpy(), er[ucols].cpu().numpy(), cfg.slope)
+    bwd = oracle.gat_bwd(ip, ix, f_sub, el[drows].cpu().numpy(), er[ucols].cpu().numpy(), fwd.alpha,
+                         gout[drows].float().cpu().numpy(), cfg.slope)
+    where = torch.searchsorted(ucols, srcs)                      # sampled sources inside the sub-problem
+    has_out = out_deg[srcs] > 0
+    where_np, srcs_ok = where[has_out].cpu().numpy(), srcs[has_out]
+    allclose_report(dfeat[srcs_ok].float().cpu().numpy(), bwd.dfeat[where_np], what="dfeat",
+                    **_tol(dtype, bwd.dfeat[where_np], grad=True))
+    allclose_report(der[srcs_ok].cpu().numpy(), bwd.der[where_np], what="der", **_tol(dtype, bwd.der[where_np], grad=True))
+    no_out = srcs[~has_out]
+    assert (dfeat[no_out] == 0).all() and (der[no_out] == 0).all()
+
+
+def test_stack_host_entry_point_matches_device_calls():
+    """sar_gat_stack_host (host buffers in, host buffers out) == the same layers run call by call."""
+    from paper_2111_06483_b200 import binding as B
+    cfg = workloads.CONFIGS["seqpart"].scaled(0.1)
+    n, H, F, L = cfg.n, cfg.heads, cfg.feat, 3
+    src, dst = workloads.make_graph(cfg, device=DEV)
+    g = api.Graph.from_coo(n, src, dst, k=cfg.k)
+    for dtype in ("f32", "bf16"):
+        tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+        feat0 = workloads.normal_tensor((n, H, F), 5, 10, dtype=tdt)
+        gout = workloads.normal_tensor((n, H, F), 5, 11, dtype=tdt)
+        els = [workloads.normal_tensor((n, H), 5, 16 * l + 12) for l in range(L)]
+        ers = [workloads.normal_tensor((n, H), 5, 16 * l + 13) for l in range(L)]
+        pin = lambda x: x.pin_memory()
+        h_out, h_dfeat = pin(torch.empty_like(feat0)), pin(torch.empty_like(feat0))
+        h_del = [pin(torch.empty((n, H))) for _ in range(L)]
+        h_der = [pin(torch.empty((n, H))) for _ in range(L)]
+        arena = torch.empty(B.sar_gat_stack_arena_bytes(g.whole, L, H, F, B._dtype(feat0)), dtype=torch.uint8, device=DEV)
+        B.sar_gat_stack_host(g.whole, g.bounds, H, F, cfg.slope, pin(feat0), [pin(x) for x in els],
+                             [pin(x) for x in ers], pin(gout), h_out, h_dfeat, h_del, h_der, arena)
+        torch.cuda.synchronize()
+        # the same chain with device tensors
+        x = feat0.to(DEV)
+        saved = []
+        for l in range(L):
+            o, m, d = api.gat_forward(g, x, els[l].to(DEV), ers[l].to(DEV), cfg.slope)
+            saved.append((x, m, d))
+            x = o
+        assert torch.equal(x.cpu(), h_out)
+        gr = gout.to(DEV)
+        for l in reversed(range(L)):
+            xin, m, d = saved[l]
+            gr, dl, dr = api.gat_backward(g, xin, els[l].to(DEV), ers[l].to(DEV), m, d, gr, cfg.slope)
+            assert torch.equal(dl.cpu(), h_del[l]) and torch.equal(dr.cpu(), h_der[l])
+        assert torch.equal(gr.cpu(), h_dfeat)
