@@ -247,6 +247,35 @@ SAR_API sar_status sar_spmm_agg(const sar_part *g, const void *feat_q, int32_t F
 SAR_API size_t sar_spmm_workspace_bytes(const sar_part *g, int32_t F, sar_dtype t);
 
 /* ---------------------------------------------------------------------------------------------
+ * Backward pass without any caller-provided scratch.  (The paper has no counterpart: this is a
+ * convenience of this library.)
+ *
+ * Some callers have no way to give the library working memory: code that runs where cudaMalloc is off
+ * limits (inside a latency-critical loop, because cudaMalloc synchronises the whole device; in a plug-in
+ * whose host owns the allocator and hands out only the input and output buffers; in a process that has
+ * pinned its memory budget at start-up).  For them this entry point runs the whole-graph backward pass of
+ * sar_gat_bwd (one partition holding all sources, D rebuilt from the edges) with its scratch taken from a
+ * fixed array of SAR_NOALLOC_SCRATCH_BYTES that is part of the library's device image.  It calls no
+ * cudaMalloc / cudaFree and no allocating library routine; inputs and outputs are the caller's, exactly
+ * as for sar_gat_bwd.
+ *
+ *   - Limit: sar_gat_workspace_bytes(g, H, F, t) must not exceed SAR_NOALLOC_SCRATCH_BYTES (16 bytes per
+ *     (destination, head) plus the long-row partials); larger problems return SAR_ERR_WORKSPACE and launch
+ *     nothing.  Every GPU that loads the library carries the array until the process exits.
+ *   - The first call on each device looks up the array's device address (with that device current) and
+ *     remembers it; make that first call before any stream capture begins.
+ *   - All calls on a device share the one array, which keeps whatever the previous call left in it.  The
+ *     pass writes every byte of it that it later reads, so nothing needs clearing between calls; but two
+ *     calls whose kernels overlap on the GPU (different streams, no dependency) race on it: keep calls to
+ *     this entry point ordered.
+ * ------------------------------------------------------------------------------------------- */
+#define SAR_NOALLOC_SCRATCH_BYTES (16u << 20)
+SAR_API size_t sar_gat_bwd_noalloc_limit(void); /* = SAR_NOALLOC_SCRATCH_BYTES */
+SAR_API sar_status sar_gat_bwd_noalloc(const sar_part *g, const void *feat, const float *el, const float *er,
+                                       const float *m, const float *d, const void *gout, int32_t H, int32_t F,
+                                       sar_dtype t, float slope, void *dfeat, float *del, float *der, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * A stack of L aggregation layers with HOST buffers (the 3-layer GAT of the paper's Sec. 4.2 reduced
  * to its aggregation steps): layer l computes out^l from feat^l = out^(l-1) (feat^0 given) with its
  * own el^l, er^l; the backward pass feeds dfeat^(l+1) as gout of layer l.  All copies and kernels

@@ -27,7 +27,7 @@ EXPORTS = [
     "sar_partition_bounds", "sar_csr_split_indptr", "sar_csr_split_indices", "sar_validate_part", "sar_plan_count",
     "sar_plan_fill", "sar_gat_workspace_bytes", "sar_gat_fwd", "sar_gat_fwd_fused", "sar_gat_bwd_prepare",
     "sar_gat_bwd", "sar_gat_bwd_fused", "sar_spmm_agg", "sar_spmm_workspace_bytes", "sar_set_launch_hook",
-    "sar_gat_stack_arena_bytes", "sar_gat_stack_host",
+    "sar_gat_stack_arena_bytes", "sar_gat_stack_host", "sar_gat_bwd_noalloc", "sar_gat_bwd_noalloc_limit",
 ]
 
 
@@ -64,7 +64,7 @@ def lib() -> ctypes.CDLL:
         L.sar_status_string.argtypes = [ctypes.c_int]
         L.sar_built_for_sm.restype = c_int32
         for name in ("sar_graph_workspace_bytes", "sar_gat_workspace_bytes", "sar_spmm_workspace_bytes",
-                     "sar_gat_stack_arena_bytes"):
+                     "sar_gat_stack_arena_bytes", "sar_gat_bwd_noalloc_limit"):
             getattr(L, name).restype = c_size_t
         _lib = L
     return _lib
@@ -379,3 +379,23 @@ def sar_gat_stack_host(part: Part, bounds: Sequence[int], H: int, F: int, slope:
     w, wb = _ws(arena)
     _check("sar_gat_stack_host", lib().sar_gat_stack_host(byref(part.c), c_int32(len(bounds) - 1), _host_i64(bounds),
                                                           byref(io), w, wb, _stream()))
+
+
+# ----------------------------------------------------------------------------------------------
+# backward pass with the library's built-in scratch
+# ----------------------------------------------------------------------------------------------
+
+def sar_gat_bwd_noalloc_limit() -> int:
+    return int(lib().sar_gat_bwd_noalloc_limit())
+
+
+def sar_gat_bwd_noalloc(part: Part, feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor, m: torch.Tensor,
+                        d: torch.Tensor, gout: torch.Tensor, H: int, F: int, slope: float, dfeat: torch.Tensor,
+                        del_: torch.Tensor, der: torch.Tensor) -> None:
+    """Whole-graph backward pass for callers that cannot provide scratch memory: the library uses a fixed
+    array inside its own device image (problems whose scratch need exceeds it are refused).  Calls on
+    one device must not overlap on the GPU; make the first call on a device outside stream capture."""
+    _check("sar_gat_bwd_noalloc", lib().sar_gat_bwd_noalloc(byref(part.c), _ptr(feat), _ptr(el), _ptr(er), _ptr(m),
+                                                            _ptr(d), _ptr(gout), c_int32(H), c_int32(F),
+                                                            ctypes.c_int(_dtype(feat)), c_float(slope), _ptr(dfeat),
+                                                            _ptr(del_), _ptr(der), _stream()))
