@@ -334,133 +334,223 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
             if (i >= 0 && i < nr) sso[i] = inc - ns;
             if (i == nr - 1) sso[nr] = inc;
         }
-        if constexpr (MODE != kSum) {
-            for (int x = lane; x < nr * Hp; x += 32) {
-                const int i = x >> lgHp, h = x & (Hp - 1);
-                const long long row = row0 + r + i;
-                float c0 = 0.f, c1 = __uint_as_float(kKeyNegInf), c2 = 0.f;
-                if (h < H) {
-                    if constexpr (kFwdMode) {
-                        c0 = __ldg(a.el + row * H + h);
-                    } else if constexpr (kDst) {
-                        const float dd = __ldg(a.d + row * H + h);
-                        c0 = __ldg(a.el + row * H + h);
-                        c1 = __ldg(a.m + row * H + h);
-                        c2 = dd > 0.f ? 1.f / dd : 0.f;
-                    } else {
-                        c0 = __ldg(a.er + row * H + h);
-                    }
+        __syncwarp();
+        const int nslots = sso[nr];
+        const int npos = nslots * EPW;
+
+        // Every stage below first ISSUES all of its global loads into registers and only then
+        // consumes them: a warp executes in order, so a load followed by its use inside a loop body
+        // would expose one full memory latency per sweep.
+        // ---- stage B: per-(row, head) constants and column ids (slot-major) -----------------------
+        auto load_consts = [&](int x, float &c0, float &c1, float &c2) {
+            c0 = 0.f;
+            c1 = __uint_as_float(kKeyNegInf);
+            c2 = 0.f;
+            const int i = x >> lgHp, h = x & (Hp - 1);
+            if (x < nr * Hp && h < H) {
+                const long long o = (row0 + r + i) * H + h;
+                if constexpr (kFwdMode) {
+                    c0 = __ldg(a.el + o);
+                } else if constexpr (kDst) {
+                    c0 = __ldg(a.el + o);
+                    c1 = __ldg(a.m + o);
+                    c2 = __ldg(a.d + o);
+                } else {
+                    c0 = __ldg(a.er + o);
                 }
+            }
+        };
+        auto store_consts = [&](int x, float c0, float c1, float c2) {
+            if (x < nr * Hp) {
+                if constexpr (kDst) c2 = c2 > 0.f ? __fdividef(1.f, c2) : 0.f;  // 1/d
                 sc0[x] = c0;
                 sc1[x] = c1;
                 sc2[x] = c2;
             }
+        };
+        float ca[2][3];
+        if constexpr (MODE != kSum) {
+            load_consts(lane, ca[0][0], ca[0][1], ca[0][2]);
+            load_consts(lane + 32, ca[1][0], ca[1][1], ca[1][2]);
         }
-        __syncwarp();
-        // ---- stage B: column ids, slot-major (row i's edges start at position sso[i]*EPW) --------
-        const int nslots = sso[nr];
-        const int npos = nslots * EPW;
-        {
+        {   // two positions per lane and sweep: both loads are issued before either is stored
             int i = 0;
-            for (int q = lane; q < npos; q += 32) {
-                while (q >= sso[i + 1] * EPW) ++i;
-                const int t = srb[i] + (q - sso[i] * EPW);
-                sj[q] = t < srb[i + 1] ? ld_stream_i32(a.indices + cb + t) : -1;
+            for (int q0 = lane; q0 < npos; q0 += 64) {
+                int c[2] = {-1, -1};
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int q = q0 + 32 * u;
+                    if (q < npos) {
+                        while (q >= sso[i + 1] * EPW) ++i;
+                        const int t = srb[i] + (q - sso[i] * EPW);
+                        if (t < srb[i + 1]) c[u] = ld_stream_i32(a.indices + cb + t);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 2; ++u)
+                    if (q0 + 32 * u < npos) sj[q0 + 32 * u] = c[u];
             }
             for (int q = npos + lane; q < npos + S * EPW; q += 32) sj[q] = -1;  // the ring's run-out
         }
+        if constexpr (MODE != kSum) {
+            store_consts(lane, ca[0][0], ca[0][1], ca[0][2]);
+            store_consts(lane + 32, ca[1][0], ca[1][1], ca[1][2]);
+            for (int x = lane + 64; x < nr * Hp; x += 32) {  // many heads x many rows: the rest, plainly
+                float c0, c1, c2;
+                load_consts(x, c0, c1, c2);
+                store_consts(x, c0, c1, c2);
+            }
+        }
         __syncwarp();
 
-        // ---- stage C: weight records, one padded position per lane and sweep, all its heads ------
+        // ---- start the gather ring now: the first S slots need only the column ids ----------------
+        auto issue = [&](int s_, unsigned dst_s) {
+            const int col = lds_s32(sj_s + s_ * (EPW * 4));  // -1 past the row's / chunk's end: zero fill
+            const uint4 *src = gbase + (long long)(col < 0 ? 0 : col) * n_vec;
+#pragma unroll
+            for (int v = 0; v < V; ++v) cp_async16_s(dst_s + v * 512, src + v * G, (col >= 0 && vok[v]) ? 16 : 0);
+            cp_async_commit();
+        };
+#pragma unroll
+        for (int s_ = 0; s_ < S; ++s_) issue(s_, stage_s + s_ * (V * 512));
+
+        // ---- stage C: weight records, two positions per lane and sweep, all their heads -----------
         if constexpr (MODE != kSum) {
             const bool vec4 = a.hvec != 0;  // heads handled four at a time with 16-byte accesses
             int i = 0;
-            for (int q = lane; q < npos; q += 32) {
-                while (q >= sso[i + 1] * EPW) ++i;
-                const int col = sj[q];
-                const int rb = i * Hp, wb_ = q << lgHp;
+            for (int q0 = lane; q0 < npos; q0 += 64) {
+                int col[2], rbase[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int q = q0 + 32 * u;
+                    col[u] = -1;
+                    rbase[u] = 0;
+                    if (q < npos) {
+                        while (q >= sso[i + 1] * EPW) ++i;
+                        col[u] = sj[q];
+                        rbase[u] = i * Hp;
+                    }
+                }
                 if (vec4) {
                     for (int h = 0; h < H; h += 4) {
-                        const float4 c0 = *reinterpret_cast<const float4 *>(sc0 + rb + h);
-                        float s4[4], g4[4];
                         if constexpr (kFwdMode || kDst) {
-                            float4 e4 = make_float4(0.f, 0.f, 0.f, 0.f);
-                            if (col >= 0) e4 = __ldg(reinterpret_cast<const float4 *>(a.er + (long long)col * H + h));
-                            s4[0] = c0.x + e4.x; s4[1] = c0.y + e4.y; s4[2] = c0.z + e4.z; s4[3] = c0.w + e4.w;
-                        }
-                        if constexpr (kFwdMode) {
-                            float4 o;
-                            float *op = reinterpret_cast<float *>(&o);
+                            float4 e4[2];
 #pragma unroll
-                            for (int k = 0; k < 4; ++k) {
-                                op[k] = SAR_NEG_INF;  // padding: weight exp(-inf - max) = 0
-                                if (col >= 0) {
-                                    op[k] = leaky(s4[k], a.slope, g4[k]);
-                                    atomicMax(&skey[rb + h + k], fkey(op[k]));
+                            for (int u = 0; u < 2; ++u) {
+                                e4[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                if (col[u] >= 0) e4[u] = __ldg(reinterpret_cast<const float4 *>(a.er + (long long)col[u] * H + h));
+                            }
+#pragma unroll
+                            for (int u = 0; u < 2; ++u) {
+                                const int q = q0 + 32 * u;
+                                if (q >= npos) continue;
+                                const int rb = rbase[u] + h;
+                                const float4 c0 = *reinterpret_cast<const float4 *>(sc0 + rb);
+                                const float s4[4] = {c0.x + e4[u].x, c0.y + e4[u].y, c0.z + e4[u].z, c0.w + e4[u].w};
+                                float4 o;
+                                float *op = reinterpret_cast<float *>(&o);
+                                if constexpr (kFwdMode) {
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j) {
+                                        float gr;
+                                        op[j] = SAR_NEG_INF;  // padding: weight exp(-inf - max) = 0
+                                        if (col[u] >= 0) {
+                                            op[j] = leaky(s4[j], a.slope, gr);
+                                            atomicMax(&skey[rb + j], fkey(op[j]));
+                                        }
+                                    }
+                                } else {
+                                    // rematerialised attention coefficient alpha >= 0; its sign bit carries
+                                    // "score <= 0" (LeakyReLU' = slope), so one float holds both weights
+                                    const float4 m4 = *reinterpret_cast<const float4 *>(sc1 + rb);
+                                    const float4 i4 = *reinterpret_cast<const float4 *>(sc2 + rb);
+                                    const float *mp = reinterpret_cast<const float *>(&m4);
+                                    const float *ip = reinterpret_cast<const float *>(&i4);
+#pragma unroll
+                                    for (int j = 0; j < 4; ++j) {
+                                        float gr;
+                                        const float al = fast_exp(leaky(s4[j], a.slope, gr) - mp[j]) * ip[j];
+                                        op[j] = col[u] >= 0 ? (s4[j] > 0.f ? al : -al) : 0.f;
+                                    }
                                 }
+                                *reinterpret_cast<float4 *>(reinterpret_cast<float *>(sw) + (q << lgHp) + h) = o;
                             }
-                            *reinterpret_cast<float4 *>(reinterpret_cast<float *>(sw) + wb_ + h) = o;
-                        } else if constexpr (kDst) {
-                            // rematerialised attention coefficient alpha >= 0; its sign bit carries
-                            // "score <= 0" (LeakyReLU' = slope), so one float holds both weights
-                            const float4 m4 = *reinterpret_cast<const float4 *>(sc1 + rb + h);
-                            const float4 i4 = *reinterpret_cast<const float4 *>(sc2 + rb + h);
-                            const float *mp = reinterpret_cast<const float *>(&m4), *ip = reinterpret_cast<const float *>(&i4);
-                            float4 o;
-                            float *op = reinterpret_cast<float *>(&o);
-#pragma unroll
-                            for (int k = 0; k < 4; ++k) {
-                                const float al = fast_exp(leaky(s4[k], a.slope, g4[k]) - mp[k]) * ip[k];
-                                op[k] = col >= 0 ? (s4[k] > 0.f ? al : -al) : 0.f;
-                            }
-                            *reinterpret_cast<float4 *>(reinterpret_cast<float *>(sw) + wb_ + h) = o;
                         } else {
-                            const float *cp0 = reinterpret_cast<const float *>(&c0);
-                            float2 o[4];
+                            // source-major pass: one 16-byte record {el_i, m_i, 1/d_i, D_i} per (column, head)
+                            float4 rec[2][4];
 #pragma unroll
-                            for (int k = 0; k < 4; ++k) {
-                                o[k] = make_float2(0.f, 0.f);
-                                if (col >= 0) {
-                                    const float4 rec = __ldg(a.rec_in + (long long)col * H + h + k);  // {el_i, m_i, 1/d_i, D_i}
-                                    const float s_ = rec.x + cp0[k];
-                                    float gr;
-                                    const float al = fast_exp(leaky(s_, a.slope, gr) - rec.y) * rec.z;
-                                    o[k] = make_float2(s_ > 0.f ? al : -al, al * gr * rec.w);
+                            for (int u = 0; u < 2; ++u)
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    rec[u][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                                    if (col[u] >= 0) rec[u][j] = __ldg(a.rec_in + (long long)col[u] * H + h + j);
                                 }
+#pragma unroll
+                            for (int u = 0; u < 2; ++u) {
+                                const int q = q0 + 32 * u;
+                                if (q >= npos) continue;
+                                const float4 c0 = *reinterpret_cast<const float4 *>(sc0 + rbase[u] + h);
+                                const float *cp0 = reinterpret_cast<const float *>(&c0);
+                                float2 o[4];
+#pragma unroll
+                                for (int j = 0; j < 4; ++j) {
+                                    o[j] = make_float2(0.f, 0.f);
+                                    if (col[u] >= 0) {
+                                        const float s_ = rec[u][j].x + cp0[j];
+                                        float gr;
+                                        const float al = fast_exp(leaky(s_, a.slope, gr) - rec[u][j].y) * rec[u][j].z;
+                                        o[j] = make_float2(s_ > 0.f ? al : -al, al * gr * rec[u][j].w);
+                                    }
+                                }
+                                float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float2 *>(sw) + (q << lgHp) + h);
+                                dst[0] = make_float4(o[0].x, o[0].y, o[1].x, o[1].y);
+                                dst[1] = make_float4(o[2].x, o[2].y, o[3].x, o[3].y);
                             }
-                            float4 *dst = reinterpret_cast<float4 *>(reinterpret_cast<float2 *>(sw) + wb_ + h);
-                            dst[0] = make_float4(o[0].x, o[0].y, o[1].x, o[1].y);
-                            dst[1] = make_float4(o[2].x, o[2].y, o[3].x, o[3].y);
                         }
                     }
                 } else {
                     for (int h = 0; h < H; ++h) {
-                        const float c0 = sc0[rb + h];
-                        float gr;
-                        if constexpr (kFwdMode) {
-                            float e = SAR_NEG_INF;
-                            if (col >= 0) {
-                                e = leaky(c0 + __ldg(a.er + (long long)col * H + h), a.slope, gr);
-                                atomicMax(&skey[rb + h], fkey(e));
+                        float ev[2] = {0.f, 0.f};
+                        float4 rec[2];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            rec[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (col[u] >= 0) {
+                                if constexpr (kSrc) rec[u] = __ldg(a.rec_in + (long long)col[u] * H + h);
+                                else ev[u] = __ldg(a.er + (long long)col[u] * H + h);
                             }
-                            reinterpret_cast<float *>(sw)[wb_ + h] = e;
-                        } else if constexpr (kDst) {
-                            float wrec = 0.f;
-                            if (col >= 0) {
-                                const float s_ = c0 + __ldg(a.er + (long long)col * H + h);
-                                const float al = fast_exp(leaky(s_, a.slope, gr) - sc1[rb + h]) * sc2[rb + h];
-                                wrec = s_ > 0.f ? al : -al;
+                        }
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const int q = q0 + 32 * u;
+                            if (q >= npos) continue;
+                            const int rb = rbase[u] + h;
+                            const bool live = col[u] >= 0;
+                            float gr;
+                            if constexpr (kFwdMode) {
+                                float e = SAR_NEG_INF;
+                                if (live) {
+                                    e = leaky(sc0[rb] + ev[u], a.slope, gr);
+                                    atomicMax(&skey[rb], fkey(e));
+                                }
+                                reinterpret_cast<float *>(sw)[(q << lgHp) + h] = e;
+                            } else if constexpr (kDst) {
+                                float wrec = 0.f;
+                                if (live) {
+                                    const float s_ = sc0[rb] + ev[u];
+                                    const float al = fast_exp(leaky(s_, a.slope, gr) - sc1[rb]) * sc2[rb];
+                                    wrec = s_ > 0.f ? al : -al;
+                                }
+                                reinterpret_cast<float *>(sw)[(q << lgHp) + h] = wrec;
+                            } else {
+                                float2 wrec = make_float2(0.f, 0.f);
+                                if (live) {
+                                    const float s_ = rec[u].x + sc0[rb];
+                                    const float al = fast_exp(leaky(s_, a.slope, gr) - rec[u].y) * rec[u].z;
+                                    wrec = make_float2(s_ > 0.f ? al : -al, al * gr * rec[u].w);
+                                }
+                                reinterpret_cast<float2 *>(sw)[(q << lgHp) + h] = wrec;
                             }
-                            reinterpret_cast<float *>(sw)[wb_ + h] = wrec;
-                        } else {
-                            float2 wrec = make_float2(0.f, 0.f);
-                            if (col >= 0) {
-                                const float4 rec = __ldg(a.rec_in + (long long)col * H + h);
-                                const float s_ = rec.x + c0;
-                                const float al = fast_exp(leaky(s_, a.slope, gr) - rec.y) * rec.z;
-                                wrec = make_float2(s_ > 0.f ? al : -al, al * gr * rec.w);
-                            }
-                            reinterpret_cast<float2 *>(sw)[wb_ + h] = wrec;
                         }
                     }
                 }
@@ -517,16 +607,6 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
         // ---- stage D: gather through the cp.async ring ---------------------------------------------
         // Slot s lives in ring stage s % S; lane (half, gl) copies and later reads back its own 16
         // bytes of edge s*EPW + half, so no cross-lane synchronisation is needed around the ring.
-        auto issue = [&](int s_, unsigned dst_s) {
-            const int col = lds_s32(sj_s + s_ * (EPW * 4));  // -1 past the row's / chunk's end: zero fill
-            const uint4 *src = gbase + (long long)(col < 0 ? 0 : col) * n_vec;
-#pragma unroll
-            for (int v = 0; v < V; ++v) cp_async16_s(dst_s + v * 512, src + v * G, (col >= 0 && vok[v]) ? 16 : 0);
-            cp_async_commit();
-        };
-#pragma unroll
-        for (int s_ = 0; s_ < S; ++s_) issue(s_, stage_s + s_ * (V * 512));
-
         int s = 0;
         for (int ri = 0; ri < nr; ++ri) {
             const int s_end = sso[ri + 1];
