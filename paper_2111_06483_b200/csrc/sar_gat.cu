@@ -140,8 +140,8 @@ static sar_status check_elem_align(std::initializer_list<const void *> ps, size_
 }
 
 // ---- span kernels ---------------------------------------------------------------------------------
-constexpr int kCapFwd = 128, kCapDst = 128, kCapSrc = 128, kCapSum = 128;
-constexpr int kMinBlocksFwd = 6, kMinBlocksBwd = 5;  // resident blocks per SM the register budget is cut for
+constexpr int kCapFwd = 256, kCapDst = 256, kCapSrc = 128, kCapSum = 256;
+constexpr int kMinBlocksFwd = 24, kMinBlocksBwd = 20;  // resident blocks per SM the register budget is cut for
 
 static int rows_per_span(long long n_rows, long long nnz, int cap) {
     const double avg = n_rows > 0 ? (double)nnz / (double)n_rows : 0.0;

@@ -27,7 +27,7 @@
 
 namespace sar {
 
-constexpr int kSpanWarps = 4;             // warps per block
+constexpr int kSpanWarps = 1;             // warps per block
 constexpr int kSpanThreads = kSpanWarps * 32;
 constexpr int kMaxSpanRows = 16;          // rows per span
 
