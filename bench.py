@@ -96,6 +96,30 @@ NCU_TRAFFIC_BYTES = {
 }
 
 
+def max_over_ranks(value: float, dist=None, device="cpu") -> float:
+    """Largest `value` over all ranks (the job is as slow as its slowest replica); identity without dist."""
+    if dist is None:
+        return float(value)
+    import torch
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def group_passes(kernels: dict) -> dict:
+    """Launch names -> passes: 'gat_fwd', 'gat_fwd_seg', 'gat_fwd_merge' together are one pass over the edges."""
+    passes = {}
+    for name, v in kernels.items():
+        base = name
+        for suffix in ("_seg", "_merge"):
+            if name.endswith(suffix):
+                base = name[:-len(suffix)]
+        p_ = passes.setdefault(base, {"ms": 0.0, "launches": []})
+        p_["ms"] += v["avg_ms"]
+        p_["launches"].append(name)
+    return passes
+
+
 # --------------------------------------------------------------------------------------------------
 # clocks
 # --------------------------------------------------------------------------------------------------
@@ -124,24 +148,31 @@ class ClockSampler:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         try:
-            for line in open(self.path):
-                f = [x.strip() for x in line.split(",")]
-                if len(f) < 7:
-                    continue
-                try:
-                    sm.append(float(f[0]))
-                    mx.append(float(f[1]))
-                except ValueError:
-                    continue
-                for nme, val in zip(names, f[3:7]):
-                    if val.lower().startswith("active"):
-                        reasons.add(nme)
+            out = self.parse(open(self.path).read().splitlines())
             os.unlink(self.path)
         except OSError:
             pass
+        return out
+
+    @staticmethod
+    def parse(lines):
+        """nvidia-smi CSV lines -> median SM clock under load, max clock, throttle reasons seen Active."""
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in lines:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nme, val in zip(names, f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nme)
         if sm:
             sm.sort()
             out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
@@ -287,10 +318,7 @@ def run_ours(args, rank, world, local_rank):
         dist.barrier()
     elapsed_ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if sampler else {}
-    if dist:
-        tmax = torch.tensor([elapsed_ms], device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(tmax.item())
+    elapsed_ms = max_over_ranks(elapsed_ms, dist, dev)
     kernels = lt.summary()
     launches = sum(v["launches"] for v in kernels.values())
     ms_per_step = elapsed_ms / args.steps
@@ -300,12 +328,7 @@ def run_ours(args, rank, world, local_rank):
     # A pass over the E edges is up to three launches of the library (rows, long-row segments, merge);
     # its algorithmic bytes are divided by the sum of their average CUDA-event durations.
     peak, peak_src = load_peaks()
-    passes = {}
-    for name, v in kernels.items():
-        base = name[:-4] if name.endswith("_seg") else (name[:-6] if name.endswith("_merge") else name)
-        p_ = passes.setdefault(base, {"ms": 0.0, "launches": []})
-        p_["ms"] += v["avg_ms"]
-        p_["launches"].append(name)
+    passes = group_passes(kernels)
     dom = max(passes, key=lambda k_: passes[k_]["ms"])
     roofline = None
     if dom in KERNEL_BYTES:
@@ -354,10 +377,7 @@ def run_ours(args, rank, world, local_rank):
             host_step()
         torch.cuda.synchronize()
         dt = time.perf_counter() - t0
-        if dist:
-            tmax = torch.tensor([dt], device=dev)
-            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-            dt = float(tmax.item())
+        dt = max_over_ranks(dt, dist, dev)
         h2d = 2 * n * H * F * b + 2 * L * n * H * 4
         d2h = 2 * n * H * F * b + 2 * L * n * H * 4
         e2e = {"value": world * L * e * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,

@@ -379,3 +379,27 @@ def test_argument_errors_return_status_codes():
         B.sar_gat_bwd(fwd_only, d["feat"], d["el"], d["er"], m, dd, d["gout"], 2, 8, 0.2, 3, out, m, dd, ws)
     assert ei.value.code == -1
     torch.cuda.synchronize()
+
+
+def test_memory_kept_for_backward_does_not_grow_with_the_edge_count():
+    """The attention coefficients are never stored (Sec. 3.3): what forward + backward allocate beyond
+    the graph itself depends on N*H*F and N*H, not on E*H."""
+    n, H, F = 50_000, 4, 32
+    peaks = []
+    for e in (500_000, 2_000_000):
+        src, dst = workloads.uniform_edges(n, e, 70, self_loops=False)
+        g = api.Graph.from_coo(n, src.to(DEV), dst.to(DEV), threshold=0)
+        t = {k: v.to(DEV) for k, v in workloads.make_node_inputs(n, H, F, 70).items()}
+        torch.cuda.synchronize()
+        torch.cuda.reset_peak_memory_stats()
+        base = torch.cuda.memory_allocated()
+        out, m, d = api.gat_forward(g, t["feat"], t["el"], t["er"], 0.2)
+        grads = api.gat_backward(g, t["feat"], t["el"], t["er"], m, d, t["gout"], 0.2)
+        torch.cuda.synchronize()
+        peaks.append(torch.cuda.max_memory_allocated() - base)
+        del out, m, d, grads, g, t
+    node_bytes = n * H * F * 4
+    assert peaks[1] <= peaks[0] + 4096                       # 4x the edges, same extra memory
+    assert peaks[0] <= 2 * node_bytes + 64 * n * H + (1 << 20)   # out + dfeat + [N,H] vectors and records
+    # a storing implementation would add 4*E*H bytes per kept copy of the coefficients: +24 MB between the two graphs
+    assert 4 * (2_000_000 - 500_000) * H > 1000 * (peaks[1] - peaks[0] + 1)
