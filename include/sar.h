@@ -278,10 +278,13 @@ SAR_API sar_status sar_gat_bwd_noalloc(const sar_part *g, const void *feat, cons
 /* ---------------------------------------------------------------------------------------------
  * A stack of L aggregation layers with HOST buffers (the 3-layer GAT of the paper's Sec. 4.2 reduced
  * to its aggregation steps): layer l computes out^l from feat^l = out^(l-1) (feat^0 given) with its
- * own el^l, er^l; the backward pass feeds dfeat^(l+1) as gout of layer l.  All copies and kernels
- * are enqueued on `stream` in order: host->device of the inputs, L fused forwards, L fused
- * backwards, device->host of the results.  Returns without synchronising; use pinned host memory
- * for the copies to be asynchronous.
+ * own el^l, er^l; the backward pass feeds dfeat^(l+1) as gout of layer l.  The kernels are enqueued on
+ * `stream`; the host->device copies of the inputs and the device->host copies of the results run on two
+ * side streams of the library (created on first use, one pair per device) so that they overlap with the
+ * kernels, ordered after the work already queued on `stream`, and `stream` waits for the last copy:
+ * once `stream` has completed, every output is in host memory.  Returns without synchronising; use
+ * pinned host memory for the copies to be asynchronous.  The host inputs must stay unchanged, and
+ * `arena` untouched, until then.
  * ------------------------------------------------------------------------------------------- */
 typedef struct {
     int32_t L, H, F;

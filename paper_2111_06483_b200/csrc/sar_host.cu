@@ -1,5 +1,6 @@
 // Host-buffer entry point: a stack of aggregation layers with the copies inside the call.
 // Contracts are in include/sar.h.
+#include <mutex>
 #include <vector>
 
 #include "sar_common.cuh"
@@ -17,6 +18,26 @@ struct Arena {
         return p;
     }
 };
+
+// Two non-blocking side streams per device for the copies, created on first use and kept.
+struct Copies {
+    cudaStream_t up = nullptr, down = nullptr;
+};
+constexpr int kMaxDevices = 64;
+Copies g_copies[kMaxDevices];
+std::mutex g_copies_mutex;
+
+sar_status copies_for_current_device(Copies **out) {
+    int dev = -1;
+    SAR_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return SAR_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_copies_mutex);
+    Copies &c = g_copies[dev];
+    if (!c.up) SAR_CUDA_TRY(cudaStreamCreateWithFlags(&c.up, cudaStreamNonBlocking));
+    if (!c.down) SAR_CUDA_TRY(cudaStreamCreateWithFlags(&c.down, cudaStreamNonBlocking));
+    *out = &c;
+    return SAR_OK;
+}
 
 size_t stack_bytes(const sar_part *g, int32_t L, int32_t H, int32_t F, sar_dtype t) {
     const size_t n = (size_t)g->n_dst;
@@ -65,13 +86,54 @@ sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bound
     void *ws = a.take(ws_bytes);
     if (!ws || !gb) return SAR_ERR_WORKSPACE;
 
-    // host -> device
-    SAR_CUDA_TRY(cudaMemcpyAsync(feat[0], io->feat0, row_b, cudaMemcpyHostToDevice, st));
-    SAR_CUDA_TRY(cudaMemcpyAsync(ga, io->gout, row_b, cudaMemcpyHostToDevice, st));
+    // Copies run on two side streams of the library so that they overlap with the kernels (PCIe is full
+    // duplex): `up` brings the inputs in layer order, `down` returns each result as soon as it exists.
+    // Everything is ordered after the work already queued on `st`, and `st` finally waits for the last
+    // copy, so that completion of `st` still means "all done".
+    Copies *cp = nullptr;
+    SAR_TRY(copies_for_current_device(&cp));
+    cudaStream_t up = cp->up, down = cp->down;
+    std::vector<cudaEvent_t> ev;
+    auto new_event = [&](cudaEvent_t *e) -> sar_status {
+        SAR_CUDA_TRY(cudaEventCreateWithFlags(e, cudaEventDisableTiming));
+        ev.push_back(*e);
+        return SAR_OK;
+    };
+    auto cleanup = [&]() {
+        for (cudaEvent_t e : ev) cudaEventDestroy(e);  // released by the runtime once the work that uses them is done
+    };
+#define SAR_STEP(expr)                    \
+    do {                                  \
+        sar_status st__ = (expr);         \
+        if (st__ != SAR_OK) {             \
+            cleanup();                    \
+            return st__;                  \
+        }                                 \
+    } while (0)
+#define SAR_CUDA_STEP(expr) SAR_STEP((expr) == cudaSuccess ? SAR_OK : SAR_ERR_CUDA)
+
+    cudaEvent_t e_start, e_gout, e_done;
+    std::vector<cudaEvent_t> e_in(L), e_bwd(L);
+    SAR_STEP(new_event(&e_start));
+    SAR_STEP(new_event(&e_gout));
+    SAR_STEP(new_event(&e_done));
     for (int l = 0; l < L; ++l) {
-        SAR_CUDA_TRY(cudaMemcpyAsync(el[l], io->el[l], nh_b, cudaMemcpyHostToDevice, st));
-        SAR_CUDA_TRY(cudaMemcpyAsync(er[l], io->er[l], nh_b, cudaMemcpyHostToDevice, st));
+        SAR_STEP(new_event(&e_in[l]));
+        SAR_STEP(new_event(&e_bwd[l]));
     }
+    SAR_CUDA_STEP(cudaEventRecord(e_start, st));
+    SAR_CUDA_STEP(cudaStreamWaitEvent(up, e_start, 0));
+    SAR_CUDA_STEP(cudaStreamWaitEvent(down, e_start, 0));
+
+    // host -> device, in the order the layers need them
+    SAR_CUDA_STEP(cudaMemcpyAsync(feat[0], io->feat0, row_b, cudaMemcpyHostToDevice, up));
+    for (int l = 0; l < L; ++l) {
+        SAR_CUDA_STEP(cudaMemcpyAsync(el[l], io->el[l], nh_b, cudaMemcpyHostToDevice, up));
+        SAR_CUDA_STEP(cudaMemcpyAsync(er[l], io->er[l], nh_b, cudaMemcpyHostToDevice, up));
+        SAR_CUDA_STEP(cudaEventRecord(e_in[l], up));
+    }
+    SAR_CUDA_STEP(cudaMemcpyAsync(ga, io->gout, row_b, cudaMemcpyHostToDevice, up));
+    SAR_CUDA_STEP(cudaEventRecord(e_gout, up));
 
     // per-partition pointer lists (one array cut at `bounds`)
     std::vector<const void *> fq(k);
@@ -87,9 +149,18 @@ sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bound
             fq[q] = cut(feat[l], rb, q);
             erq[q] = reinterpret_cast<const float *>(cut(er[l], (size_t)H * 4, q));
         }
-        SAR_TRY(sar_gat_fwd_fused(g, k, bounds, fq.data(), el[l], erq.data(), H, F, io->t, io->slope, m[l], d[l],
-                                  feat[l + 1], ws, ws_bytes, st));
+        SAR_CUDA_STEP(cudaStreamWaitEvent(st, e_in[l], 0));
+        SAR_STEP(sar_gat_fwd_fused(g, k, bounds, fq.data(), el[l], erq.data(), H, F, io->t, io->slope, m[l], d[l],
+                                   feat[l + 1], ws, ws_bytes, st));
     }
+    if (io->out_last) {
+        cudaEvent_t e_out;
+        SAR_STEP(new_event(&e_out));
+        SAR_CUDA_STEP(cudaEventRecord(e_out, st));
+        SAR_CUDA_STEP(cudaStreamWaitEvent(down, e_out, 0));
+        SAR_CUDA_STEP(cudaMemcpyAsync(io->out_last, feat[L], row_b, cudaMemcpyDeviceToHost, down));
+    }
+    SAR_CUDA_STEP(cudaStreamWaitEvent(st, e_gout, 0));
     void *gin = ga, *gout = gb;
     for (int l = L - 1; l >= 0; --l) {
         for (int q = 0; q < k; ++q) {
@@ -98,19 +169,23 @@ sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bound
             dfq[q] = const_cast<char *>(cut(gout, rb, q));
             derq[q] = reinterpret_cast<float *>(const_cast<char *>(cut(der[l], (size_t)H * 4, q)));
         }
-        SAR_TRY(sar_gat_bwd_fused(g, k, bounds, fq.data(), el[l], erq.data(), m[l], d[l], gin, H, F, io->t, io->slope,
-                                  dfq.data(), del[l], derq.data(), ws, ws_bytes, st));
+        SAR_STEP(sar_gat_bwd_fused(g, k, bounds, fq.data(), el[l], erq.data(), m[l], d[l], gin, H, F, io->t, io->slope,
+                                   dfq.data(), del[l], derq.data(), ws, ws_bytes, st));
+        SAR_CUDA_STEP(cudaEventRecord(e_bwd[l], st));
+        SAR_CUDA_STEP(cudaStreamWaitEvent(down, e_bwd[l], 0));
+        if (io->del) SAR_CUDA_STEP(cudaMemcpyAsync(io->del[l], del[l], nh_b, cudaMemcpyDeviceToHost, down));
+        if (io->der) SAR_CUDA_STEP(cudaMemcpyAsync(io->der[l], der[l], nh_b, cudaMemcpyDeviceToHost, down));
         void *tmp = gin;
         gin = gout;
         gout = tmp;
     }
-    // device -> host (gin now holds dfeat of layer 0)
-    if (io->out_last) SAR_CUDA_TRY(cudaMemcpyAsync(io->out_last, feat[L], row_b, cudaMemcpyDeviceToHost, st));
-    if (io->dfeat0) SAR_CUDA_TRY(cudaMemcpyAsync(io->dfeat0, gin, row_b, cudaMemcpyDeviceToHost, st));
-    for (int l = 0; l < L; ++l) {
-        if (io->del) SAR_CUDA_TRY(cudaMemcpyAsync(io->del[l], del[l], nh_b, cudaMemcpyDeviceToHost, st));
-        if (io->der) SAR_CUDA_TRY(cudaMemcpyAsync(io->der[l], der[l], nh_b, cudaMemcpyDeviceToHost, st));
-    }
+    // gin now holds dfeat of layer 0 (the last backward call has been waited for by `down` above)
+    if (io->dfeat0) SAR_CUDA_STEP(cudaMemcpyAsync(io->dfeat0, gin, row_b, cudaMemcpyDeviceToHost, down));
+    SAR_CUDA_STEP(cudaEventRecord(e_done, down));
+    SAR_CUDA_STEP(cudaStreamWaitEvent(st, e_done, 0));
+    cleanup();
+#undef SAR_STEP
+#undef SAR_CUDA_STEP
     return SAR_OK;
 }
 
