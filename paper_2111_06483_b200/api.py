@@ -12,7 +12,7 @@ import torch
 
 from . import binding as B
 
-DEFAULT_THRESHOLD = 128  # rows with more edges are cut into segments of this many edges
+DEFAULT_THRESHOLD = 384  # rows with more edges are cut into segments of this many edges
 
 
 def _workspace(nbytes: int, device) -> torch.Tensor:

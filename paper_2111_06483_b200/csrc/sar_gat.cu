@@ -141,6 +141,7 @@ static sar_status check_elem_align(std::initializer_list<const void *> ps, size_
 
 // ---- span kernels ---------------------------------------------------------------------------------
 constexpr int kCapFwd = 256, kCapDst = 256, kCapSrc = 128, kCapSum = 256;
+constexpr int kCapSeg = 128;  // capacity of the segment launches (segments hold at most the plan threshold)
 constexpr int kMinBlocksFwd = 24, kMinBlocksBwd = 20;  // resident blocks per SM the register budget is cut for
 
 static int rows_per_span(long long n_rows, long long nnz, int cap) {
@@ -155,6 +156,9 @@ static int rows_per_span(long long n_rows, long long nnz, int cap) {
 // (mode 1).  The merge launch is the caller's.
 template <typename T, int G, int V, int S, int MODE, int CAP, int MINB>
 static sar_status launch_span(SpanArgs a, long long nnz, const char *name, const char *seg_name, cudaStream_t st) {
+    // The segment launch never stages more than `threshold` edges at a time: when that fits the small
+    // capacity it runs the instantiation with the smaller shared-memory footprint (more resident warps).
+    constexpr int CAP_SEG = CAP < kCapSeg ? CAP : kCapSeg;
     auto kern = span_kernel<T, G, V, S, MODE, CAP, MINB>;
     const size_t smem = (size_t)kSpanWarps * span_layout<MODE>(a.g.Hp, V, CAP, S, 32 / G).total;
     SAR_TRY(ensure_smem(kern, smem));
@@ -167,7 +171,15 @@ static sar_status launch_span(SpanArgs a, long long nnz, const char *name, const
     }
     if (a.sp.threshold > 0 && a.sp.n_seg > 0) {
         a.mode = 1;
-        SAR_LAUNCH(seg_name, st, kern<<<(unsigned)((a.sp.n_seg + kSpanWarps - 1) / kSpanWarps), kSpanThreads, smem, st>>>(a));
+        const unsigned blocks = (unsigned)((a.sp.n_seg + kSpanWarps - 1) / kSpanWarps);
+        if (a.sp.threshold <= CAP_SEG) {
+            auto seg_kern = span_kernel<T, G, V, S, MODE, CAP_SEG, MINB>;
+            const size_t seg_smem = (size_t)kSpanWarps * span_layout<MODE>(a.g.Hp, V, CAP_SEG, S, 32 / G).total;
+            SAR_TRY(ensure_smem(seg_kern, seg_smem));
+            SAR_LAUNCH(seg_name, st, seg_kern<<<blocks, kSpanThreads, seg_smem, st>>>(a));
+        } else {
+            SAR_LAUNCH(seg_name, st, kern<<<blocks, kSpanThreads, smem, st>>>(a));
+        }
         SAR_TRY(sar_after_launch());
     }
     return SAR_OK;
