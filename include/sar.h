@@ -247,6 +247,31 @@ SAR_API sar_status sar_spmm_agg(const sar_part *g, const void *feat_q, int32_t F
 SAR_API size_t sar_spmm_workspace_bytes(const sar_part *g, int32_t F, sar_dtype t);
 
 /* ---------------------------------------------------------------------------------------------
+ * The rest of a GAT layer around the aggregation (Eq. 3; Eq. 1's f_node reduced to a ReLU).
+ *   sar_gat_project      el[i,h] = <z[i,h,:], a_l[h,:]>, er[i,h] = <z[i,h,:], a_r[h,:]>: the two halves of
+ *                        a^T (z_i || z_j) in Eq. 3.  z [n,H,F] (type t); a_l, a_r [H,F] float32.
+ *   sar_gat_project_bwd  chain rule through the projection: dz[i,h,:] += a_l[h,:]*del[i,h] + a_r[h,:]*der[i,h]
+ *                        (dz is the dfeat the aggregation's backward pass wrote, updated in place) and
+ *                        da_l[h,:] = sum_i del[i,h]*z[i,h,:], da_r likewise (written; fixed summation order,
+ *                        no atomics).  Needs sar_gat_project_workspace_bytes(H, F) bytes of scratch.
+ *   sar_relu             x = max(x, 0) in place (NaN -> 0).   sar_relu_bwd: g = 0 where y <= 0, y being the
+ *                        layer's output after the ReLU.
+ * All pointers are DEVICE memory owned by the caller.  n = 0 is allowed (node buffers may then be NULL;
+ * da_l, da_r are still written, as zeros).  Rows whose head slice F*sizeof(t) is a multiple of 16 bytes
+ * with 16-byte aligned z / dz take the vector kernels, everything else a scalar path.
+ * Errors: SAR_ERR_INVALID_ARG (NULL pointer with n > 0, H or F < 1, unknown t), SAR_ERR_ALIGNMENT
+ * (float arrays not 4-byte aligned), SAR_ERR_WORKSPACE (scratch missing, misaligned or too small).
+ * ------------------------------------------------------------------------------------------- */
+SAR_API size_t sar_gat_project_workspace_bytes(int32_t H, int32_t F);
+SAR_API sar_status sar_gat_project(int64_t n, int32_t H, int32_t F, sar_dtype t, const void *z, const float *a_l,
+                                   const float *a_r, float *el, float *er, void *stream);
+SAR_API sar_status sar_gat_project_bwd(int64_t n, int32_t H, int32_t F, sar_dtype t, const void *z, const float *a_l,
+                                       const float *a_r, const float *del, const float *der, void *dz, float *da_l,
+                                       float *da_r, void *workspace, size_t workspace_bytes, void *stream);
+SAR_API sar_status sar_relu(int64_t n_elems, sar_dtype t, void *x, void *stream);
+SAR_API sar_status sar_relu_bwd(int64_t n_elems, sar_dtype t, const void *y, void *g, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Backward pass without any caller-provided scratch.  (The paper has no counterpart: this is a
  * convenience of this library.)
  *

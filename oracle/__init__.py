@@ -235,3 +235,47 @@ def spmm(indptr, indices, feat, mean: bool = False) -> np.ndarray:
                              _p(out, np.float64))
     _check(rc, "spmm")
     return out
+
+
+# --------------------------------------------------------------------------------------
+# the layer around the aggregation (Eq. 3's a^T(z_i || z_j); f_node of Eq. 1 taken as a ReLU)
+# plain numpy, float64
+# --------------------------------------------------------------------------------------
+
+def project(z, a_l, a_r):
+    """el[i,h] = <z[i,h,:], a_l[h,:]>, er[i,h] = <z[i,h,:], a_r[h,:]>."""
+    z = np.asarray(z, dtype=np.float64)
+    return np.einsum("nhf,hf->nh", z, np.asarray(a_l, np.float64)), np.einsum("nhf,hf->nh", z, np.asarray(a_r, np.float64))
+
+
+def project_bwd(z, a_l, a_r, del_, der):
+    """Returns (dz_add[n,H,F], da_l[H,F], da_r[H,F]) of the projection for upstream del, der."""
+    z, a_l, a_r = (np.asarray(x, np.float64) for x in (z, a_l, a_r))
+    del_, der = np.asarray(del_, np.float64), np.asarray(der, np.float64)
+    dz = del_[:, :, None] * a_l[None] + der[:, :, None] * a_r[None]
+    return dz, np.einsum("nh,nhf->hf", del_, z), np.einsum("nh,nhf->hf", der, z)
+
+
+def gat_stack(indptr, indices, feat0, a_l, a_r, gout, slope: float, storage=np.float32):
+    """L layers z^{l+1} = ReLU(GAT(z^l, <z^l,a_l^l>, <z^l,a_r^l>)) and the gradient of <gout, z^L>.
+
+    The aggregation functions take float32 storage, so activations are rounded to `storage` between
+    layers exactly where the library stores them (z, el, er and the upstream gradient)."""
+    L = len(a_l)
+    z = [np.asarray(feat0, dtype=storage)]
+    saved = []
+    for l in range(L):
+        el, er = project(z[l], a_l[l], a_r[l])
+        el, er = el.astype(np.float32), er.astype(np.float32)
+        f = gat_fwd(indptr, indices, z[l].astype(np.float32), el, er, slope)
+        saved.append((el, er, f))
+        z.append(np.maximum(f.out, 0.0).astype(storage))
+    g = np.asarray(gout, dtype=np.float64)
+    da_l, da_r = [None] * L, [None] * L
+    for l in reversed(range(L)):
+        el, er, f = saved[l]
+        g = np.where(z[l + 1].astype(np.float64) > 0, g, 0.0).astype(storage)
+        b = gat_bwd(indptr, indices, z[l].astype(np.float32), el, er, f.alpha, g.astype(np.float32), slope)
+        dz_add, da_l[l], da_r[l] = project_bwd(z[l], a_l[l], a_r[l], b.del_.astype(np.float32), b.der.astype(np.float32))
+        g = (b.dfeat.astype(storage).astype(np.float64) + dz_add)
+    return dict(out=z[L].astype(np.float64), dfeat0=g, da_l=da_l, da_r=da_r)

@@ -28,6 +28,7 @@ EXPORTS = [
     "sar_plan_fill", "sar_gat_workspace_bytes", "sar_gat_fwd", "sar_gat_fwd_fused", "sar_gat_bwd_prepare",
     "sar_gat_bwd", "sar_gat_bwd_fused", "sar_spmm_agg", "sar_spmm_workspace_bytes", "sar_set_launch_hook",
     "sar_gat_stack_arena_bytes", "sar_gat_stack_host", "sar_gat_bwd_noalloc", "sar_gat_bwd_noalloc_limit",
+    "sar_gat_project_workspace_bytes", "sar_gat_project", "sar_gat_project_bwd", "sar_relu", "sar_relu_bwd",
 ]
 
 
@@ -64,7 +65,7 @@ def lib() -> ctypes.CDLL:
         L.sar_status_string.argtypes = [ctypes.c_int]
         L.sar_built_for_sm.restype = c_int32
         for name in ("sar_graph_workspace_bytes", "sar_gat_workspace_bytes", "sar_spmm_workspace_bytes",
-                     "sar_gat_stack_arena_bytes", "sar_gat_bwd_noalloc_limit"):
+                     "sar_gat_stack_arena_bytes", "sar_gat_bwd_noalloc_limit", "sar_gat_project_workspace_bytes"):
             getattr(L, name).restype = c_size_t
         _lib = L
     return _lib
@@ -399,3 +400,34 @@ def sar_gat_bwd_noalloc(part: Part, feat: torch.Tensor, el: torch.Tensor, er: to
                                                             _ptr(d), _ptr(gout), c_int32(H), c_int32(F),
                                                             ctypes.c_int(_dtype(feat)), c_float(slope), _ptr(dfeat),
                                                             _ptr(del_), _ptr(der), _stream()))
+
+
+# ----------------------------------------------------------------------------------------------
+# the layer around the aggregation
+# ----------------------------------------------------------------------------------------------
+
+def sar_gat_project_workspace_bytes(H: int, F: int) -> int:
+    return int(lib().sar_gat_project_workspace_bytes(c_int32(H), c_int32(F)))
+
+
+def sar_gat_project(z: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, el: torch.Tensor, er: torch.Tensor) -> None:
+    n, H, F = z.shape
+    _check("sar_gat_project", lib().sar_gat_project(c_int64(n), c_int32(H), c_int32(F), ctypes.c_int(_dtype(z)), _ptr(z),
+                                                    _ptr(a_l), _ptr(a_r), _ptr(el), _ptr(er), _stream()))
+
+
+def sar_gat_project_bwd(z: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, del_: torch.Tensor, der: torch.Tensor,
+                        dz: torch.Tensor, da_l: torch.Tensor, da_r: torch.Tensor, workspace: torch.Tensor) -> None:
+    n, H, F = z.shape
+    w, wb = _ws(workspace)
+    _check("sar_gat_project_bwd", lib().sar_gat_project_bwd(c_int64(n), c_int32(H), c_int32(F), ctypes.c_int(_dtype(z)),
+                                                            _ptr(z), _ptr(a_l), _ptr(a_r), _ptr(del_), _ptr(der), _ptr(dz),
+                                                            _ptr(da_l), _ptr(da_r), w, wb, _stream()))
+
+
+def sar_relu(x: torch.Tensor) -> None:
+    _check("sar_relu", lib().sar_relu(c_int64(x.numel()), ctypes.c_int(_dtype(x)), _ptr(x), _stream()))
+
+
+def sar_relu_bwd(y: torch.Tensor, g: torch.Tensor) -> None:
+    _check("sar_relu_bwd", lib().sar_relu_bwd(c_int64(y.numel()), ctypes.c_int(_dtype(y)), _ptr(y), _ptr(g), _stream()))

@@ -2,6 +2,7 @@
 // kernel selection and launches.  Declarations and contracts are in include/sar.h.
 #include "sar_gat_kernels.cuh"
 #include "sar_span_kernels.cuh"
+#include "sar_dispatch.cuh"
 #include "sar_generic_kernels.cuh"
 
 namespace sar {
@@ -36,43 +37,6 @@ sar_status make_shape(int32_t H, int32_t F, sar_dtype t, bool ptrs_16B_aligned, 
         s.geom = RowGeom{H, Hp, sar_log2(Hp), (int)(head_bytes / 16), n_vec};
     }
     *out = s;
-    return SAR_OK;
-}
-
-template <typename T, int G, int V, int U>
-struct Cfg {
-    using type = T;
-    static constexpr int g = G, v = V, u = U;
-};
-
-// Calls f(Cfg<T,G,V,U>{}) for the instantiation matching the shape.
-template <typename Fn>
-static sar_status dispatch(const Shape &s, Fn &&f) {
-#define SAR_CASE(GG, VV, UU)                                                   \
-    if (s.G == GG && s.V == VV) {                                              \
-        if (s.t == SAR_F32) return f(Cfg<float, GG, VV, UU>{});                \
-        return f(Cfg<__nv_bfloat16, GG, VV, UU>{});                            \
-    }
-    SAR_CASE(4, 1, 4)
-    SAR_CASE(8, 1, 4)
-    SAR_CASE(16, 1, 4)
-    SAR_CASE(32, 1, 4)
-    SAR_CASE(32, 2, 2)
-    SAR_CASE(32, 4, 1)
-    SAR_CASE(32, 8, 1)
-#undef SAR_CASE
-    return SAR_ERR_UNSUPPORTED;
-}
-
-static inline unsigned blocks_for(long long items, int G) {
-    const long long per_block = (long long)kWarpsPerBlock * (32 / G);
-    return (unsigned)((items + per_block - 1) / per_block);
-}
-
-template <typename K>
-static sar_status ensure_smem(K kernel, size_t bytes) {
-    if (bytes > 48 * 1024)
-        SAR_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes));
     return SAR_OK;
 }
 
@@ -127,17 +91,6 @@ static sar_status check_part(const sar_part *g, bool need_csc) {
     return SAR_OK;
 }
 
-static bool all16(std::initializer_list<const void *> ps) {
-    for (const void *p : ps)
-        if (p && !sar_aligned(p, 16)) return false;
-    return true;
-}
-
-static sar_status check_elem_align(std::initializer_list<const void *> ps, size_t a) {
-    for (const void *p : ps)
-        if (p && !sar_aligned(p, a)) return SAR_ERR_ALIGNMENT;
-    return SAR_OK;
-}
 
 // ---- span kernels ---------------------------------------------------------------------------------
 constexpr int kCapFwd = 256, kCapDst = 256, kCapSrc = 128, kCapSum = 256;

@@ -1,0 +1,328 @@
+// The GAT layer around the aggregation (Eq. 3): score projections el = <z, a_left>, er = <z, a_right>
+// per head, their backward pass (chain-rule add into dz, gradients of a), and the element-wise ReLU
+// between layers.  Streaming kernels; contracts are in include/sar.h.
+#include "sar_dispatch.cuh"
+#include "sar_rowkernels.cuh"
+
+namespace sar {
+
+constexpr int kGlueBlocks = 148 * 8;  // fixed grid of the reducing kernel: a fixed summation order
+
+struct ProjArgs {
+    long long n;
+    const void *feat;
+    const float *a_l, *a_r;  // [H,F]
+    float *el, *er;          // forward: written
+    const float *del, *der;  // backward: read
+    void *dfeat;             // backward: dfeat += a_l*del + a_r*der (in place)
+    float *partial;          // backward: [blocks][2][H*F]
+    int H, F;
+    RowGeom g;
+};
+
+// lane (gl, v) -> the EPV coefficients of a[h, :] that meet its vector
+template <int G, int V, int EPV>
+__device__ __forceinline__ void load_coeffs(const float *__restrict__ a, const RowGeom &g, int F, int gl,
+                                            float (&c)[V][EPV]) {
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        const int vi = v * G + gl;
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) c[v][e] = 0.f;
+        if (vi < g.n_vec) {
+            const int h = vi / g.vph, f0 = (vi - h * g.vph) * EPV;
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) c[v][e] = __ldg(a + h * F + f0 + e);
+        }
+    }
+}
+
+template <typename T, int G, int V>
+__global__ void __launch_bounds__(kThreads) project_kernel(const ProjArgs a) {
+    constexpr int EPV = Elem<T>::EPV;
+    constexpr int RPW = 32 / G;
+    extern __shared__ __align__(16) float smem[];
+    const LaneId<G> id;
+    float *scratch = smem + (size_t)id.warp * (32 * V) + id.gid * (G * V);
+    const VecGeom<G, V> vg(a.g, id.gl);
+    float cl[V][EPV], cr[V][EPV];
+    load_coeffs<G, V, EPV>(a.a_l, a.g, a.F, id.gl, cl);
+    load_coeffs<G, V, EPV>(a.a_r, a.g, a.F, id.gl, cr);
+    const long long stride = (long long)gridDim.x * kWarpsPerBlock * RPW;
+    const long long first = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
+    // every lane of the warp runs the same number of sweeps (head_sum synchronises the warp)
+    const long long sweeps = (a.n + stride - 1) / stride;
+    for (long long s = 0; s < sweeps; ++s) {
+        const long long row = first + s * stride;
+        const bool active = row < a.n;
+        float fv[V][EPV], pl[V], pr[V];
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) fv[v][e] = 0.f;
+        if (active) load_row_vec<T, G, V>(a.feat, row, a.g.n_vec, id.gl, vg.vok, fv);
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            pl[v] = pr[v] = 0.f;
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) {
+                pl[v] = fmaf(fv[v][e], cl[v][e], pl[v]);
+                pr[v] = fmaf(fv[v][e], cr[v][e], pr[v]);
+            }
+        }
+        const float L = head_sum<G, V>(scratch, pl, vg.vok, id.gl, a.g);
+        const float R = head_sum<G, V>(scratch, pr, vg.vok, id.gl, a.g);
+        if (active && id.gl < a.H) {
+            a.el[row * a.H + id.gl] = L;
+            a.er[row * a.H + id.gl] = R;
+        }
+    }
+}
+
+// dfeat += a_l*del + a_r*der; per-block partial sums of del*feat and der*feat over the block's rows
+template <typename T, int G, int V>
+__global__ void __launch_bounds__(kThreads) project_bwd_kernel(const ProjArgs a) {
+    constexpr int EPV = Elem<T>::EPV;
+    constexpr int RPW = 32 / G;
+    constexpr int GPB = kWarpsPerBlock * RPW;  // groups per block
+    extern __shared__ __align__(16) float smem[];  // [GPB][2][G*V*EPV]
+    const LaneId<G> id;
+    const VecGeom<G, V> vg(a.g, id.gl);
+    float cl[V][EPV], cr[V][EPV], sl[V][EPV], sr[V][EPV];
+    load_coeffs<G, V, EPV>(a.a_l, a.g, a.F, id.gl, cl);
+    load_coeffs<G, V, EPV>(a.a_r, a.g, a.F, id.gl, cr);
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) sl[v][e] = sr[v][e] = 0.f;
+    const long long stride = (long long)gridDim.x * GPB;
+    const int group = id.warp * RPW + id.gid;
+    for (long long row = (long long)blockIdx.x * GPB + group; row < a.n; row += stride) {
+        float fv[V][EPV], gv[V][EPV];
+        load_row_vec<T, G, V>(a.feat, row, a.g.n_vec, id.gl, vg.vok, fv);
+        load_row_vec<T, G, V, false>(a.dfeat, row, a.g.n_vec, id.gl, vg.vok, gv);
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            float dl = 0.f, dr = 0.f;
+            if (vg.vok[v]) {
+                dl = __ldg(a.del + row * a.H + vg.hv[v]);
+                dr = __ldg(a.der + row * a.H + vg.hv[v]);
+            }
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) {
+                gv[v][e] += cl[v][e] * dl + cr[v][e] * dr;
+                sl[v][e] = fmaf(dl, fv[v][e], sl[v][e]);
+                sr[v][e] = fmaf(dr, fv[v][e], sr[v][e]);
+            }
+        }
+        store_row_vec<T, G, V>(a.dfeat, row, a.g.n_vec, id.gl, vg.vok, gv);
+    }
+    // block reduction in a fixed order: group 0 adds the other groups' sums
+    const int rowf = G * V * EPV;
+    float *mine = smem + (size_t)group * 2 * rowf;
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) {
+            mine[(v * G + id.gl) * EPV + e] = sl[v][e];
+            mine[rowf + (v * G + id.gl) * EPV + e] = sr[v][e];
+        }
+    __syncthreads();
+    const int HF = a.H * a.F;
+    for (int x = threadIdx.x; x < 2 * HF; x += blockDim.x) {
+        const int which = x / HF, o = x - which * HF;  // o < H*F <= rowf
+        float acc = 0.f;
+        for (int gq = 0; gq < GPB; ++gq) acc += smem[(size_t)gq * 2 * rowf + which * rowf + o];
+        a.partial[(size_t)blockIdx.x * 2 * HF + x] = acc;
+    }
+}
+
+__global__ void project_reduce_kernel(int blocks, int HF, const float *__restrict__ partial, float *__restrict__ da_l,
+                                      float *__restrict__ da_r) {
+    const int x = blockIdx.x * blockDim.x + threadIdx.x;
+    if (x >= 2 * HF) return;
+    float acc = 0.f;
+    for (int b = 0; b < blocks; ++b) acc += partial[(size_t)b * 2 * HF + x];
+    if (x < HF) da_l[x] = acc; else da_r[x - HF] = acc;
+}
+
+__device__ __forceinline__ float as_float(float x) { return x; }
+__device__ __forceinline__ float as_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+
+// scalar fallbacks
+template <typename T>
+__global__ void project_generic(const ProjArgs a) {
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= a.n * a.H) return;
+    const int h = (int)(idx % a.H);
+    const T *f = reinterpret_cast<const T *>(a.feat) + idx * a.F;
+    float L = 0.f, R = 0.f;
+    for (int k = 0; k < a.F; ++k) {
+        const float x = Elem<T>::load1(f + k);
+        L = fmaf(x, a.a_l[h * a.F + k], L);
+        R = fmaf(x, a.a_r[h * a.F + k], R);
+    }
+    a.el[idx] = L;
+    a.er[idx] = R;
+}
+
+template <typename T>
+__global__ void project_bwd_generic(const ProjArgs a, float *da_l, float *da_r) {
+    const long long HF = (long long)a.H * a.F;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx < HF) {  // one thread per coefficient walks every node in order
+        const int h = (int)(idx / a.F);
+        float L = 0.f, R = 0.f;
+        for (long long i = 0; i < a.n; ++i) {
+            const float x = Elem<T>::load1(reinterpret_cast<const T *>(a.feat) + i * HF + idx);
+            L = fmaf(a.del[i * a.H + h], x, L);
+            R = fmaf(a.der[i * a.H + h], x, R);
+        }
+        da_l[idx] = L;
+        da_r[idx] = R;
+    }
+    for (long long x = idx; x < a.n * HF; x += (long long)gridDim.x * blockDim.x) {
+        const long long i = x / HF;
+        const int o = (int)(x - i * HF), h = o / a.F;
+        T *p = reinterpret_cast<T *>(a.dfeat) + x;
+        Elem<T>::store1(p, as_float(*p) + a.a_l[o] * a.del[i * a.H + h] + a.a_r[o] * a.der[i * a.H + h]);
+    }
+}
+
+// forward: x = max(x, 0) in place; backward: g = 0 where the layer's output y is not positive
+template <typename T, bool BWD>
+__global__ void relu_kernel(long long n, const T *y, T *x) {
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+        const float v = as_float(BWD ? y[i] : x[i]);
+        if (!(v > 0.f)) Elem<T>::store1(x + i, 0.f);
+    }
+}
+
+static sar_status glue_shape(int64_t n, int32_t H, int32_t F, sar_dtype t, std::initializer_list<const void *> ps,
+                             Shape *s) {
+    if (n < 0 || H < 1 || F < 1) return SAR_ERR_INVALID_ARG;
+    return make_shape(H, F, t, all16(ps), s);
+}
+
+}  // namespace sar
+
+using namespace sar;
+
+extern "C" {
+
+size_t sar_gat_project_workspace_bytes(int32_t H, int32_t F) {
+    if (H < 1 || F < 1) return 0;
+    return (size_t)kGlueBlocks * 2 * H * F * 4 + 256;
+}
+
+sar_status sar_gat_project(int64_t n, int32_t H, int32_t F, sar_dtype t, const void *feat, const float *a_l,
+                           const float *a_r, float *el, float *er, void *stream) {
+    if (!a_l || !a_r || (n > 0 && (!feat || !el || !er))) return SAR_ERR_INVALID_ARG;
+    Shape s;
+    SAR_TRY(glue_shape(n, H, F, t, {feat}, &s));
+    SAR_TRY(check_elem_align({a_l, a_r, el, er}, 4));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (n == 0) return SAR_OK;
+    ProjArgs a{};
+    a.n = n;
+    a.feat = feat;
+    a.a_l = a_l;
+    a.a_r = a_r;
+    a.el = el;
+    a.er = er;
+    a.H = H;
+    a.F = F;
+    a.g = s.geom;
+    if (!s.fast) {
+        const unsigned blocks = (unsigned)((n * H + 255) / 256);
+        if (t == SAR_F32)
+            SAR_LAUNCH("gat_project_generic", st, project_generic<float><<<blocks, 256, 0, st>>>(a));
+        else
+            SAR_LAUNCH("gat_project_generic", st, project_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a));
+        return sar_after_launch();
+    }
+    return dispatch(s, [&](auto cfg) -> sar_status {
+        using C = decltype(cfg);
+        using T = typename C::type;
+        const size_t smem = (size_t)kWarpsPerBlock * 32 * C::v * 4;
+        unsigned blocks = blocks_for(n, C::g);
+        if (blocks > (unsigned)kGlueBlocks * 4) blocks = kGlueBlocks * 4;
+        SAR_LAUNCH("gat_project", st, project_kernel<T, C::g, C::v><<<blocks, kThreads, smem, st>>>(a));
+        return sar_after_launch();
+    });
+}
+
+sar_status sar_gat_project_bwd(int64_t n, int32_t H, int32_t F, sar_dtype t, const void *feat, const float *a_l,
+                               const float *a_r, const float *del, const float *der, void *dfeat, float *da_l,
+                               float *da_r, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!a_l || !a_r || !da_l || !da_r || (n > 0 && (!feat || !del || !der || !dfeat))) return SAR_ERR_INVALID_ARG;
+    Shape s;
+    SAR_TRY(glue_shape(n, H, F, t, {feat, dfeat}, &s));
+    SAR_TRY(check_elem_align({a_l, a_r, del, der, da_l, da_r}, 4));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    ProjArgs a{};
+    a.n = n;
+    a.feat = feat;
+    a.a_l = a_l;
+    a.a_r = a_r;
+    a.del = del;
+    a.der = der;
+    a.dfeat = dfeat;
+    a.H = H;
+    a.F = F;
+    a.g = s.geom;
+    const int HF = H * F;
+    if (!s.fast) {
+        long long work = (long long)n * HF > HF ? (long long)n * HF : HF;
+        unsigned blocks = (unsigned)((work + 255) / 256);
+        if (blocks > 65535u * 16) blocks = 65535u * 16;
+        if (t == SAR_F32)
+            SAR_LAUNCH("gat_project_bwd_generic", st, project_bwd_generic<float><<<blocks, 256, 0, st>>>(a, da_l, da_r));
+        else
+            SAR_LAUNCH("gat_project_bwd_generic", st, project_bwd_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a, da_l, da_r));
+        return sar_after_launch();
+    }
+    if (!workspace || !sar_aligned(workspace, 16) || workspace_bytes < (size_t)kGlueBlocks * 2 * HF * 4) return SAR_ERR_WORKSPACE;
+    a.partial = static_cast<float *>(workspace);
+    return dispatch(s, [&](auto cfg) -> sar_status {
+        using C = decltype(cfg);
+        using T = typename C::type;
+        constexpr int EPV = Elem<T>::EPV;
+        const size_t smem = (size_t)kWarpsPerBlock * (32 / C::g) * 2 * (C::g * C::v * EPV) * 4;
+        auto kern = project_bwd_kernel<T, C::g, C::v>;
+        SAR_TRY(ensure_smem(kern, smem));
+        SAR_LAUNCH("gat_project_bwd", st, kern<<<kGlueBlocks, kThreads, smem, st>>>(a));
+        SAR_TRY(sar_after_launch());
+        SAR_LAUNCH("gat_project_reduce", st,
+                   project_reduce_kernel<<<(2 * HF + 255) / 256, 256, 0, st>>>(kGlueBlocks, HF, a.partial, da_l, da_r));
+        return sar_after_launch();
+    });
+}
+
+sar_status sar_relu(int64_t n_elems, sar_dtype t, void *x, void *stream) {
+    if (n_elems < 0 || (n_elems > 0 && !x)) return SAR_ERR_INVALID_ARG;
+    if (t != SAR_F32 && t != SAR_BF16) return SAR_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (n_elems == 0) return SAR_OK;
+    const unsigned blocks = (unsigned)((n_elems / 4 + 255) / 256 < 148 * 32 ? (n_elems / 4 + 255) / 256 + 1 : 148 * 32);
+    if (t == SAR_F32)
+        SAR_LAUNCH("relu", st, relu_kernel<float, false><<<blocks, 256, 0, st>>>(n_elems, nullptr, static_cast<float *>(x)));
+    else
+        SAR_LAUNCH("relu", st, relu_kernel<__nv_bfloat16, false><<<blocks, 256, 0, st>>>(n_elems, nullptr, static_cast<__nv_bfloat16 *>(x)));
+    return sar_after_launch();
+}
+
+sar_status sar_relu_bwd(int64_t n_elems, sar_dtype t, const void *y, void *g, void *stream) {
+    if (n_elems < 0 || (n_elems > 0 && (!y || !g))) return SAR_ERR_INVALID_ARG;
+    if (t != SAR_F32 && t != SAR_BF16) return SAR_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (n_elems == 0) return SAR_OK;
+    const unsigned blocks = (unsigned)((n_elems / 4 + 255) / 256 < 148 * 32 ? (n_elems / 4 + 255) / 256 + 1 : 148 * 32);
+    if (t == SAR_F32)
+        SAR_LAUNCH("relu_bwd", st, relu_kernel<float, true><<<blocks, 256, 0, st>>>(n_elems, static_cast<const float *>(y), static_cast<float *>(g)));
+    else
+        SAR_LAUNCH("relu_bwd", st, relu_kernel<__nv_bfloat16, true><<<blocks, 256, 0, st>>>(n_elems, static_cast<const __nv_bfloat16 *>(y), static_cast<__nv_bfloat16 *>(g)));
+    return sar_after_launch();
+}
+
+}  // extern "C"
