@@ -43,6 +43,9 @@ def parse_args():
     ap.add_argument("--dtype", default=None, help="f32 | bf16 (default: the workload's last listed dtype)")
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (debugging only)")
     ap.add_argument("--threshold", type=int, default=None, help="long-row split threshold")
+    ap.add_argument("--glue", action="store_true",
+                    help="also run the layer glue each step: score projections before every aggregation, "
+                         "ReLU after it, and their backward passes (default: aggregation kernels only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample", type=float, default=0.05, help="fraction of the workload the oracle is timed on")
@@ -284,15 +287,31 @@ def run_ours(args, rank, world, local_rank):
     der_q = [cut(x) for x in ders]
     gbuf_q = [cut(x) for x in gbuf]
 
+    glue = args.glue
+    if glue:
+        a_ls = [workloads.normal_tensor((H, F), cfg.seed, 16 * l + 14, device=dev) / F ** 0.5 for l in range(L)]
+        a_rs = [workloads.normal_tensor((H, F), cfg.seed, 16 * l + 15, device=dev) / F ** 0.5 for l in range(L)]
+        da_l, da_r = torch.empty((H, F), device=dev), torch.empty((H, F), device=dev)
+        pws = torch.empty(B.sar_gat_project_workspace_bytes(H, F), dtype=torch.uint8, device=dev)
+
     def step():
         for l in range(L):
+            if glue:  # the ReLU closing layer l-1 runs inside layer l's projection
+                B.sar_gat_project(feats[l], a_ls[l], a_rs[l], els[l], ers[l], B.SAR_GLUE_RELU if l > 0 else 0)
             B.sar_gat_fwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], H, F, cfg.slope, ms[l], ds[l],
                                 feats[l + 1], ws)
+        if glue:
+            B.sar_relu(feats[L])
         gin = gout
+        if glue:
+            B.sar_relu_bwd(feats[L], gin)  # masks gout in place on the first pass; the same mask every step
         for i, l in enumerate(reversed(range(L))):
             B.sar_gat_bwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], ms[l], ds[l], gin, H, F, cfg.slope,
                                 gbuf_q[i % 2], dels[l], der_q[l], ws)
             gin = gbuf[i % 2]
+            if glue:
+                B.sar_gat_project_bwd(feats[l], a_ls[l], a_rs[l], dels[l], ders[l], gin, da_l, da_r, pws,
+                                      B.SAR_GLUE_RELU if l > 0 else 0)
 
     torch.cuda.reset_peak_memory_stats()
     for _ in range(args.warmup):
@@ -401,7 +420,7 @@ def run_ours(args, rank, world, local_rank):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {
                 "workload": cfg.name, "n": n, "e": e, "heads": H, "feat_per_head": F, "layers": L, "partitions": K,
-                "storage_dtype": dtype, "schedule": "fused row-stationary (sar_gat_fwd_fused / sar_gat_bwd_fused)",
+                "storage_dtype": dtype, "layer_glue": bool(args.glue), "schedule": "fused row-stationary (sar_gat_fwd_fused / sar_gat_bwd_fused)",
                 "l2": "inputs_exceed_l2", "long_row_threshold": threshold, "parallelism": f"replicas x{world}",
                 "edges_x_heads_x_feat_per_sec": value * H * F,
             },

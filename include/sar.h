@@ -256,6 +256,10 @@ SAR_API size_t sar_spmm_workspace_bytes(const sar_part *g, int32_t F, sar_dtype 
  *                        no atomics).  Needs sar_gat_project_workspace_bytes(H, F) bytes of scratch.
  *   sar_relu             x = max(x, 0) in place (NaN -> 0).   sar_relu_bwd: g = 0 where y <= 0, y being the
  *                        layer's output after the ReLU.
+ * flags = SAR_GLUE_RELU folds the ReLU that closes the previous layer into these two calls, saving its own
+ * pass over the node features: sar_gat_project then first writes z = max(z, 0) in place (the only case in
+ * which it writes z) and projects the result; sar_gat_project_bwd, after the update of dz, zeroes dz where
+ * z <= 0 (what sar_relu_bwd(z, dz) would do).  Any other flag bit: SAR_ERR_INVALID_ARG.
  * All pointers are DEVICE memory owned by the caller.  n = 0 is allowed (node buffers may then be NULL;
  * da_l, da_r are still written, as zeros).  Rows whose head slice F*sizeof(t) is a multiple of 16 bytes
  * with 16-byte aligned z / dz take the vector kernels, everything else a scalar path.
@@ -263,11 +267,13 @@ SAR_API size_t sar_spmm_workspace_bytes(const sar_part *g, int32_t F, sar_dtype 
  * (float arrays not 4-byte aligned), SAR_ERR_WORKSPACE (scratch missing, misaligned or too small).
  * ------------------------------------------------------------------------------------------- */
 SAR_API size_t sar_gat_project_workspace_bytes(int32_t H, int32_t F);
-SAR_API sar_status sar_gat_project(int64_t n, int32_t H, int32_t F, sar_dtype t, const void *z, const float *a_l,
-                                   const float *a_r, float *el, float *er, void *stream);
+#define SAR_GLUE_RELU 1u
+SAR_API sar_status sar_gat_project(int64_t n, int32_t H, int32_t F, sar_dtype t, void *z, const float *a_l,
+                                   const float *a_r, float *el, float *er, uint32_t flags, void *stream);
 SAR_API sar_status sar_gat_project_bwd(int64_t n, int32_t H, int32_t F, sar_dtype t, const void *z, const float *a_l,
                                        const float *a_r, const float *del, const float *der, void *dz, float *da_l,
-                                       float *da_r, void *workspace, size_t workspace_bytes, void *stream);
+                                       float *da_r, uint32_t flags, void *workspace, size_t workspace_bytes,
+                                       void *stream);
 SAR_API sar_status sar_relu(int64_t n_elems, sar_dtype t, void *x, void *stream);
 SAR_API sar_status sar_relu_bwd(int64_t n_elems, sar_dtype t, const void *y, void *g, void *stream);
 

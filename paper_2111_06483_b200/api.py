@@ -166,33 +166,32 @@ def spmm_sum(part: B.Part, feat: torch.Tensor, mean: bool = False, deg_total: Op
 
 
 # ----------------------------------------------------------------------------------------------
-# the layer around the aggregation: z' = ReLU(GAT(z, <z,a_l>, <z,a_r>)) (Eq. 3 with f_node of Eq. 1
-# taken as a ReLU); argument marshalling only, every step is a library call.
+# the layer around the aggregation: z' = GAT(z, <z,a_l>, <z,a_r>) with z = ReLU(previous layer's
+# output) (Eq. 3 with f_node of Eq. 1 taken as a ReLU); argument marshalling only, every step is a
+# library call.
 
 def gat_layer_forward(g: Graph, z: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, slope: float,
-                      workspace: Optional[torch.Tensor] = None, relu: bool = True):
-    """Returns (z_next, saved) where saved = (el, er, m, d) is what the backward pass needs besides z."""
+                      workspace: Optional[torch.Tensor] = None, relu_input: bool = False):
+    """Returns (out, saved): out is the layer's aggregation output (before any activation) and
+    saved = (el, er, m, d) is what the backward pass needs besides z.  relu_input=True first applies
+    z = max(z, 0) in place, inside the projection kernel."""
     n, H, F = z.shape
     el = torch.empty((n, H), dtype=torch.float32, device=z.device)
     er = torch.empty_like(el)
-    B.sar_gat_project(z, a_l, a_r, el, er)
+    B.sar_gat_project(z, a_l, a_r, el, er, B.SAR_GLUE_RELU if relu_input else 0)
     out, m, d = gat_forward(g, z, el, er, slope, workspace)
-    if relu:
-        B.sar_relu(out)
     return out, (el, er, m, d)
 
 
-def gat_layer_backward(g: Graph, z: torch.Tensor, z_next: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor,
-                       saved, gout: torch.Tensor, slope: float, workspace: Optional[torch.Tensor] = None,
-                       relu: bool = True):
-    """Returns (dz, da_l, da_r).  `gout` is overwritten by the ReLU mask when relu=True."""
+def gat_layer_backward(g: Graph, z: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, saved, gout: torch.Tensor,
+                       slope: float, workspace: Optional[torch.Tensor] = None, relu_input: bool = False):
+    """Returns (dz, da_l, da_r); with relu_input=True dz is the gradient with respect to the input
+    before its ReLU (zero where z <= 0)."""
     n, H, F = z.shape
     el, er, m, d = saved
-    if relu:
-        B.sar_relu_bwd(z_next, gout)
     dz, del_, der = gat_backward(g, z, el, er, m, d, gout, slope, workspace=workspace)
     da_l = torch.empty((H, F), dtype=torch.float32, device=z.device)
     da_r = torch.empty_like(da_l)
     ws = _workspace(B.sar_gat_project_workspace_bytes(H, F), z.device)
-    B.sar_gat_project_bwd(z, a_l, a_r, del_, der, dz, da_l, da_r, ws)
+    B.sar_gat_project_bwd(z, a_l, a_r, del_, der, dz, da_l, da_r, ws, B.SAR_GLUE_RELU if relu_input else 0)
     return dz, da_l, da_r

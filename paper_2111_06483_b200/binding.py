@@ -410,19 +410,26 @@ def sar_gat_project_workspace_bytes(H: int, F: int) -> int:
     return int(lib().sar_gat_project_workspace_bytes(c_int32(H), c_int32(F)))
 
 
-def sar_gat_project(z: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, el: torch.Tensor, er: torch.Tensor) -> None:
+SAR_GLUE_RELU = 1
+
+
+def sar_gat_project(z: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, el: torch.Tensor, er: torch.Tensor,
+                    flags: int = 0) -> None:
     n, H, F = z.shape
     _check("sar_gat_project", lib().sar_gat_project(c_int64(n), c_int32(H), c_int32(F), ctypes.c_int(_dtype(z)), _ptr(z),
-                                                    _ptr(a_l), _ptr(a_r), _ptr(el), _ptr(er), _stream()))
+                                                    _ptr(a_l), _ptr(a_r), _ptr(el), _ptr(er), c_uint32(flags),
+                                                    _stream()))
 
 
 def sar_gat_project_bwd(z: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, del_: torch.Tensor, der: torch.Tensor,
-                        dz: torch.Tensor, da_l: torch.Tensor, da_r: torch.Tensor, workspace: torch.Tensor) -> None:
+                        dz: torch.Tensor, da_l: torch.Tensor, da_r: torch.Tensor, workspace: torch.Tensor,
+                        flags: int = 0) -> None:
     n, H, F = z.shape
     w, wb = _ws(workspace)
     _check("sar_gat_project_bwd", lib().sar_gat_project_bwd(c_int64(n), c_int32(H), c_int32(F), ctypes.c_int(_dtype(z)),
                                                             _ptr(z), _ptr(a_l), _ptr(a_r), _ptr(del_), _ptr(der), _ptr(dz),
-                                                            _ptr(da_l), _ptr(da_r), w, wb, _stream()))
+                                                            _ptr(da_l), _ptr(da_r), c_uint32(flags), w, wb,
+                                                            _stream()))
 
 
 def sar_relu(x: torch.Tensor) -> None:

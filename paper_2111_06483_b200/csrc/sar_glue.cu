@@ -37,10 +37,12 @@ __device__ __forceinline__ void load_coeffs(const float *__restrict__ a, const R
     }
 }
 
-template <typename T, int G, int V>
+// RELU: z = max(z, 0) is written back before it is projected (the ReLU that closes the previous layer).
+template <typename T, int G, int V, bool RELU>
 __global__ void __launch_bounds__(kThreads) project_kernel(const ProjArgs a) {
     constexpr int EPV = Elem<T>::EPV;
     constexpr int RPW = 32 / G;
+    constexpr int U = V <= 2 ? 2 : 1;  // rows in flight per group
     extern __shared__ __align__(16) float smem[];
     const LaneId<G> id;
     float *scratch = smem + (size_t)id.warp * (32 * V) + id.gid * (G * V);
@@ -51,36 +53,53 @@ __global__ void __launch_bounds__(kThreads) project_kernel(const ProjArgs a) {
     const long long stride = (long long)gridDim.x * kWarpsPerBlock * RPW;
     const long long first = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
     // every lane of the warp runs the same number of sweeps (head_sum synchronises the warp)
-    const long long sweeps = (a.n + stride - 1) / stride;
+    const long long sweeps = (a.n + stride * U - 1) / (stride * U);
     for (long long s = 0; s < sweeps; ++s) {
-        const long long row = first + s * stride;
-        const bool active = row < a.n;
-        float fv[V][EPV], pl[V], pr[V];
+        float fv[U][V][EPV];
+        long long row[U];
 #pragma unroll
-        for (int v = 0; v < V; ++v)
+        for (int u = 0; u < U; ++u) {
+            row[u] = first + (s * U + u) * stride;
 #pragma unroll
-            for (int e = 0; e < EPV; ++e) fv[v][e] = 0.f;
-        if (active) load_row_vec<T, G, V>(a.feat, row, a.g.n_vec, id.gl, vg.vok, fv);
+            for (int v = 0; v < V; ++v)
 #pragma unroll
-        for (int v = 0; v < V; ++v) {
-            pl[v] = pr[v] = 0.f;
-#pragma unroll
-            for (int e = 0; e < EPV; ++e) {
-                pl[v] = fmaf(fv[v][e], cl[v][e], pl[v]);
-                pr[v] = fmaf(fv[v][e], cr[v][e], pr[v]);
-            }
+                for (int e = 0; e < EPV; ++e) fv[u][v][e] = 0.f;
+            if (row[u] < a.n) load_row_vec<T, G, V, !RELU>(a.feat, row[u], a.g.n_vec, id.gl, vg.vok, fv[u]);
         }
-        const float L = head_sum<G, V>(scratch, pl, vg.vok, id.gl, a.g);
-        const float R = head_sum<G, V>(scratch, pr, vg.vok, id.gl, a.g);
-        if (active && id.gl < a.H) {
-            a.el[row * a.H + id.gl] = L;
-            a.er[row * a.H + id.gl] = R;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const bool active = row[u] < a.n;
+            float pl[V], pr[V];
+            if constexpr (RELU) {
+#pragma unroll
+                for (int v = 0; v < V; ++v)
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) fv[u][v][e] = fv[u][v][e] > 0.f ? fv[u][v][e] : 0.f;
+                if (active) store_row_vec<T, G, V>(const_cast<void *>(a.feat), row[u], a.g.n_vec, id.gl, vg.vok, fv[u]);
+            }
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                pl[v] = pr[v] = 0.f;
+#pragma unroll
+                for (int e = 0; e < EPV; ++e) {
+                    pl[v] = fmaf(fv[u][v][e], cl[v][e], pl[v]);
+                    pr[v] = fmaf(fv[u][v][e], cr[v][e], pr[v]);
+                }
+            }
+            const float L = head_sum<G, V>(scratch, pl, vg.vok, id.gl, a.g);
+            const float R = head_sum<G, V>(scratch, pr, vg.vok, id.gl, a.g);
+            if (active && id.gl < a.H) {
+                a.el[row[u] * a.H + id.gl] = L;
+                a.er[row[u] * a.H + id.gl] = R;
+            }
         }
     }
 }
 
-// dfeat += a_l*del + a_r*der; per-block partial sums of del*feat and der*feat over the block's rows
-template <typename T, int G, int V>
+// dfeat += a_l*del + a_r*der; per-block partial sums of del*feat and der*feat over the block's rows.
+// MASK: the updated dfeat is then zeroed where feat <= 0 (feat being a ReLU's output, this is that
+// ReLU's backward pass).
+template <typename T, int G, int V, bool MASK>
 __global__ void __launch_bounds__(kThreads) project_bwd_kernel(const ProjArgs a) {
     constexpr int EPV = Elem<T>::EPV;
     constexpr int RPW = 32 / G;
@@ -111,6 +130,7 @@ __global__ void __launch_bounds__(kThreads) project_bwd_kernel(const ProjArgs a)
 #pragma unroll
             for (int e = 0; e < EPV; ++e) {
                 gv[v][e] += cl[v][e] * dl + cr[v][e] * dr;
+                if constexpr (MASK) gv[v][e] = fv[v][e] > 0.f ? gv[v][e] : 0.f;
                 sl[v][e] = fmaf(dl, fv[v][e], sl[v][e]);
                 sr[v][e] = fmaf(dr, fv[v][e], sr[v][e]);
             }
@@ -151,14 +171,18 @@ __device__ __forceinline__ float as_float(__nv_bfloat16 x) { return __bfloat162f
 
 // scalar fallbacks
 template <typename T>
-__global__ void project_generic(const ProjArgs a) {
+__global__ void project_generic(const ProjArgs a, bool relu) {
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= a.n * a.H) return;
     const int h = (int)(idx % a.H);
-    const T *f = reinterpret_cast<const T *>(a.feat) + idx * a.F;
+    T *f = reinterpret_cast<T *>(const_cast<void *>(a.feat)) + idx * a.F;
     float L = 0.f, R = 0.f;
     for (int k = 0; k < a.F; ++k) {
-        const float x = Elem<T>::load1(f + k);
+        float x = as_float(f[k]);
+        if (relu) {
+            x = x > 0.f ? x : 0.f;
+            Elem<T>::store1(f + k, x);
+        }
         L = fmaf(x, a.a_l[h * a.F + k], L);
         R = fmaf(x, a.a_r[h * a.F + k], R);
     }
@@ -167,7 +191,7 @@ __global__ void project_generic(const ProjArgs a) {
 }
 
 template <typename T>
-__global__ void project_bwd_generic(const ProjArgs a, float *da_l, float *da_r) {
+__global__ void project_bwd_generic(const ProjArgs a, float *da_l, float *da_r, bool mask) {
     const long long HF = (long long)a.H * a.F;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx < HF) {  // one thread per coefficient walks every node in order
@@ -185,17 +209,47 @@ __global__ void project_bwd_generic(const ProjArgs a, float *da_l, float *da_r) 
         const long long i = x / HF;
         const int o = (int)(x - i * HF), h = o / a.F;
         T *p = reinterpret_cast<T *>(a.dfeat) + x;
-        Elem<T>::store1(p, as_float(*p) + a.a_l[o] * a.del[i * a.H + h] + a.a_r[o] * a.der[i * a.H + h]);
+        float v = as_float(*p) + a.a_l[o] * a.del[i * a.H + h] + a.a_r[o] * a.der[i * a.H + h];
+        if (mask && !(Elem<T>::load1(reinterpret_cast<const T *>(a.feat) + x) > 0.f)) v = 0.f;
+        Elem<T>::store1(p, v);
     }
 }
 
-// forward: x = max(x, 0) in place; backward: g = 0 where the layer's output y is not positive
+// forward: x = max(x, 0) in place; backward: g = 0 where the layer's output y is not positive.
+// 16 bytes per thread where both arrays are 16-byte aligned; the ragged tail (and unaligned arrays) one
+// element at a time.
 template <typename T, bool BWD>
-__global__ void relu_kernel(long long n, const T *y, T *x) {
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x) {
+__global__ void relu_kernel(long long n, const T *y, T *x, long long n_vec16) {
+    constexpr int EPV = Elem<T>::EPV;
+    const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long nthreads = (long long)gridDim.x * blockDim.x;
+    for (long long i = tid; i < n_vec16; i += nthreads) {
+        uint4 *xp = reinterpret_cast<uint4 *>(x) + i;
+        float xv[EPV], yv[EPV];
+        Elem<T>::unpack(*xp, xv);
+        if constexpr (BWD) Elem<T>::unpack(__ldg(reinterpret_cast<const uint4 *>(y) + i), yv);
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) {
+            const float v = BWD ? yv[e] : xv[e];
+            if (!(v > 0.f)) xv[e] = 0.f;
+        }
+        *xp = Elem<T>::pack(xv);
+    }
+    for (long long i = n_vec16 * EPV + tid; i < n; i += nthreads) {
         const float v = as_float(BWD ? y[i] : x[i]);
         if (!(v > 0.f)) Elem<T>::store1(x + i, 0.f);
     }
+}
+
+template <typename T, bool BWD>
+static sar_status launch_relu(const char *name, int64_t n, const void *y, void *x, cudaStream_t st) {
+    const bool vec = sar_aligned(x, 16) && (!BWD || sar_aligned(y, 16));
+    const long long n_vec16 = vec ? n / Elem<T>::EPV : 0;
+    const long long work = n_vec16 > 0 ? n_vec16 : n;
+    long long blocks = (work + 255) / 256;
+    if (blocks > 148 * 64) blocks = 148 * 64;
+    SAR_LAUNCH(name, st, (relu_kernel<T, BWD><<<(unsigned)blocks, 256, 0, st>>>(n, static_cast<const T *>(y), static_cast<T *>(x), n_vec16)));
+    return sar_after_launch();
 }
 
 static sar_status glue_shape(int64_t n, int32_t H, int32_t F, sar_dtype t, std::initializer_list<const void *> ps,
@@ -215,8 +269,10 @@ size_t sar_gat_project_workspace_bytes(int32_t H, int32_t F) {
     return (size_t)kGlueBlocks * 2 * H * F * 4 + 256;
 }
 
-sar_status sar_gat_project(int64_t n, int32_t H, int32_t F, sar_dtype t, const void *feat, const float *a_l,
-                           const float *a_r, float *el, float *er, void *stream) {
+sar_status sar_gat_project(int64_t n, int32_t H, int32_t F, sar_dtype t, void *feat, const float *a_l,
+                           const float *a_r, float *el, float *er, uint32_t flags, void *stream) {
+    if (flags & ~(uint32_t)SAR_GLUE_RELU) return SAR_ERR_INVALID_ARG;
+    const bool relu = (flags & SAR_GLUE_RELU) != 0;
     if (!a_l || !a_r || (n > 0 && (!feat || !el || !er))) return SAR_ERR_INVALID_ARG;
     Shape s;
     SAR_TRY(glue_shape(n, H, F, t, {feat}, &s));
@@ -236,9 +292,9 @@ sar_status sar_gat_project(int64_t n, int32_t H, int32_t F, sar_dtype t, const v
     if (!s.fast) {
         const unsigned blocks = (unsigned)((n * H + 255) / 256);
         if (t == SAR_F32)
-            SAR_LAUNCH("gat_project_generic", st, project_generic<float><<<blocks, 256, 0, st>>>(a));
+            SAR_LAUNCH("gat_project_generic", st, project_generic<float><<<blocks, 256, 0, st>>>(a, relu));
         else
-            SAR_LAUNCH("gat_project_generic", st, project_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a));
+            SAR_LAUNCH("gat_project_generic", st, project_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a, relu));
         return sar_after_launch();
     }
     return dispatch(s, [&](auto cfg) -> sar_status {
@@ -247,14 +303,19 @@ sar_status sar_gat_project(int64_t n, int32_t H, int32_t F, sar_dtype t, const v
         const size_t smem = (size_t)kWarpsPerBlock * 32 * C::v * 4;
         unsigned blocks = blocks_for(n, C::g);
         if (blocks > (unsigned)kGlueBlocks * 4) blocks = kGlueBlocks * 4;
-        SAR_LAUNCH("gat_project", st, project_kernel<T, C::g, C::v><<<blocks, kThreads, smem, st>>>(a));
+        if (relu)
+            SAR_LAUNCH("gat_project", st, (project_kernel<T, C::g, C::v, true><<<blocks, kThreads, smem, st>>>(a)));
+        else
+            SAR_LAUNCH("gat_project", st, (project_kernel<T, C::g, C::v, false><<<blocks, kThreads, smem, st>>>(a)));
         return sar_after_launch();
     });
 }
 
 sar_status sar_gat_project_bwd(int64_t n, int32_t H, int32_t F, sar_dtype t, const void *feat, const float *a_l,
                                const float *a_r, const float *del, const float *der, void *dfeat, float *da_l,
-                               float *da_r, void *workspace, size_t workspace_bytes, void *stream) {
+                               float *da_r, uint32_t flags, void *workspace, size_t workspace_bytes, void *stream) {
+    if (flags & ~(uint32_t)SAR_GLUE_RELU) return SAR_ERR_INVALID_ARG;
+    const bool mask = (flags & SAR_GLUE_RELU) != 0;
     if (!a_l || !a_r || !da_l || !da_r || (n > 0 && (!feat || !del || !der || !dfeat))) return SAR_ERR_INVALID_ARG;
     Shape s;
     SAR_TRY(glue_shape(n, H, F, t, {feat, dfeat}, &s));
@@ -277,9 +338,9 @@ sar_status sar_gat_project_bwd(int64_t n, int32_t H, int32_t F, sar_dtype t, con
         unsigned blocks = (unsigned)((work + 255) / 256);
         if (blocks > 65535u * 16) blocks = 65535u * 16;
         if (t == SAR_F32)
-            SAR_LAUNCH("gat_project_bwd_generic", st, project_bwd_generic<float><<<blocks, 256, 0, st>>>(a, da_l, da_r));
+            SAR_LAUNCH("gat_project_bwd_generic", st, project_bwd_generic<float><<<blocks, 256, 0, st>>>(a, da_l, da_r, mask));
         else
-            SAR_LAUNCH("gat_project_bwd_generic", st, project_bwd_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a, da_l, da_r));
+            SAR_LAUNCH("gat_project_bwd_generic", st, project_bwd_generic<__nv_bfloat16><<<blocks, 256, 0, st>>>(a, da_l, da_r, mask));
         return sar_after_launch();
     }
     if (!workspace || !sar_aligned(workspace, 16) || workspace_bytes < (size_t)kGlueBlocks * 2 * HF * 4) return SAR_ERR_WORKSPACE;
@@ -289,8 +350,9 @@ sar_status sar_gat_project_bwd(int64_t n, int32_t H, int32_t F, sar_dtype t, con
         using T = typename C::type;
         constexpr int EPV = Elem<T>::EPV;
         const size_t smem = (size_t)kWarpsPerBlock * (32 / C::g) * 2 * (C::g * C::v * EPV) * 4;
-        auto kern = project_bwd_kernel<T, C::g, C::v>;
-        SAR_TRY(ensure_smem(kern, smem));
+        auto kern = mask ? project_bwd_kernel<T, C::g, C::v, true> : project_bwd_kernel<T, C::g, C::v, false>;
+        SAR_TRY(ensure_smem(project_bwd_kernel<T, C::g, C::v, true>, smem));
+        SAR_TRY(ensure_smem(project_bwd_kernel<T, C::g, C::v, false>, smem));
         SAR_LAUNCH("gat_project_bwd", st, kern<<<kGlueBlocks, kThreads, smem, st>>>(a));
         SAR_TRY(sar_after_launch());
         SAR_LAUNCH("gat_project_reduce", st,
@@ -304,12 +366,8 @@ sar_status sar_relu(int64_t n_elems, sar_dtype t, void *x, void *stream) {
     if (t != SAR_F32 && t != SAR_BF16) return SAR_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (n_elems == 0) return SAR_OK;
-    const unsigned blocks = (unsigned)((n_elems / 4 + 255) / 256 < 148 * 32 ? (n_elems / 4 + 255) / 256 + 1 : 148 * 32);
-    if (t == SAR_F32)
-        SAR_LAUNCH("relu", st, relu_kernel<float, false><<<blocks, 256, 0, st>>>(n_elems, nullptr, static_cast<float *>(x)));
-    else
-        SAR_LAUNCH("relu", st, relu_kernel<__nv_bfloat16, false><<<blocks, 256, 0, st>>>(n_elems, nullptr, static_cast<__nv_bfloat16 *>(x)));
-    return sar_after_launch();
+    if (t == SAR_F32) return launch_relu<float, false>("relu", n_elems, nullptr, x, st);
+    return launch_relu<__nv_bfloat16, false>("relu", n_elems, nullptr, x, st);
 }
 
 sar_status sar_relu_bwd(int64_t n_elems, sar_dtype t, const void *y, void *g, void *stream) {
@@ -317,12 +375,8 @@ sar_status sar_relu_bwd(int64_t n_elems, sar_dtype t, const void *y, void *g, vo
     if (t != SAR_F32 && t != SAR_BF16) return SAR_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (n_elems == 0) return SAR_OK;
-    const unsigned blocks = (unsigned)((n_elems / 4 + 255) / 256 < 148 * 32 ? (n_elems / 4 + 255) / 256 + 1 : 148 * 32);
-    if (t == SAR_F32)
-        SAR_LAUNCH("relu_bwd", st, relu_kernel<float, true><<<blocks, 256, 0, st>>>(n_elems, static_cast<const float *>(y), static_cast<float *>(g)));
-    else
-        SAR_LAUNCH("relu_bwd", st, relu_kernel<__nv_bfloat16, true><<<blocks, 256, 0, st>>>(n_elems, static_cast<const __nv_bfloat16 *>(y), static_cast<__nv_bfloat16 *>(g)));
-    return sar_after_launch();
+    if (t == SAR_F32) return launch_relu<float, true>("relu_bwd", n_elems, y, g, st);
+    return launch_relu<__nv_bfloat16, true>("relu_bwd", n_elems, y, g, st);
 }
 
 }  // extern "C"

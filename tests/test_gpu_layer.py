@@ -32,7 +32,8 @@ SHAPES = [(1, 4), (1, 8), (4, 32), (2, 16), (8, 8), (3, 20), (1, 256), (4, 64), 
 @pytest.mark.parametrize("H,F", SHAPES)
 @pytest.mark.parametrize("dt", ["f32", "bf16"])
 @pytest.mark.parametrize("n", [0, 1, 1237, 40001])
-def test_projection_and_its_backward(H, F, dt, n):
+@pytest.mark.parametrize("flags", [0, 1])
+def test_projection_and_its_backward(H, F, dt, n, flags):
     from paper_2111_06483_b200 import binding as B
     if n == 40001 and H * F > 512:
         n = 9001
@@ -48,7 +49,10 @@ def test_projection_and_its_backward(H, F, dt, n):
     dz_ref = _np(dzt)
     el = torch.full((n, H), float("nan"), device="cuda")
     er = torch.full((n, H), float("nan"), device="cuda")
-    B.sar_gat_project(zt, _dev(a_l), _dev(a_r), el, er)
+    B.sar_gat_project(zt, _dev(a_l), _dev(a_r), el, er, flags)
+    if flags:  # the ReLU of the input is applied in place, exactly
+        z_ref = np.maximum(z_ref, 0.0)
+    assert np.array_equal(_np(zt), z_ref)
     want_el, want_er = oracle.project(z_ref, a_l, a_r)
     # float32 accumulation of F products: error <= F * 2^-24 * sum|terms|; floor from the term magnitudes
     floor = 1e-6 * max(1.0, float(np.sqrt(F)))
@@ -57,9 +61,12 @@ def test_projection_and_its_backward(H, F, dt, n):
     da_l = torch.full((H, F), float("nan"), device="cuda")
     da_r = torch.full((H, F), float("nan"), device="cuda")
     ws = torch.empty(B.sar_gat_project_workspace_bytes(H, F), dtype=torch.uint8, device="cuda")
-    B.sar_gat_project_bwd(zt, _dev(a_l), _dev(a_r), _dev(gl), _dev(gr), dzt, da_l, da_r, ws)
+    B.sar_gat_project_bwd(zt, _dev(a_l), _dev(a_r), _dev(gl), _dev(gr), dzt, da_l, da_r, ws, flags)
     want_dz, want_dal, want_dar = oracle.project_bwd(z_ref, a_l, a_r, gl, gr)
     want_dz = want_dz + dz_ref
+    if flags:
+        want_dz = np.where(z_ref > 0, want_dz, 0.0)
+        assert np.all(_np(dzt)[z_ref <= 0] == 0.0)
     if dt == "bf16":
         allclose_report(_np(dzt), want_dz, 2e-2, 2e-2, "dz")
     else:
@@ -90,7 +97,7 @@ def test_relu_forward_and_backward_are_exact(dt, n):
 
 @pytest.mark.parametrize("k", [1, 3])
 def test_three_layer_stack_matches_oracle_f32(k):
-    from paper_2111_06483_b200 import api
+    from paper_2111_06483_b200 import api, binding as B
     n, H, F, L = 3000, 2, 16, 3
     p = small_problem(n, 40000, H, F, 77, self_loops=True, empty_rows=5)
     rng = np.random.default_rng(5)
@@ -100,15 +107,17 @@ def test_three_layer_stack_matches_oracle_f32(k):
     g = api.Graph.from_coo(n, _dev(p["src"], torch.int32), _dev(p["dst"], torch.int32), k=k)
     z = [_dev(p["feat"])]
     saved = []
-    for l in range(L):
-        zn, s = api.gat_layer_forward(g, z[l], _dev(a_l[l]), _dev(a_r[l]), 0.2)
-        z.append(zn)
-        saved.append(s)
+    for l in range(L):  # z[l + 1] holds layer l's output; the next layer's projection applies its ReLU in place
+        out, sv = api.gat_layer_forward(g, z[l], _dev(a_l[l]), _dev(a_r[l]), 0.2, relu_input=l > 0)
+        z.append(out)
+        saved.append(sv)
+    B.sar_relu(z[L])
     grad = _dev(p["gout"])
+    B.sar_relu_bwd(z[L], grad)
     got_al, got_ar = [None] * L, [None] * L
     for l in reversed(range(L)):
-        grad, got_al[l], got_ar[l] = api.gat_layer_backward(g, z[l], z[l + 1], _dev(a_l[l]), _dev(a_r[l]), saved[l],
-                                                            grad, 0.2)
+        grad, got_al[l], got_ar[l] = api.gat_layer_backward(g, z[l], _dev(a_l[l]), _dev(a_r[l]), saved[l], grad, 0.2,
+                                                            relu_input=l > 0)
     # three layers deep: rounding of each layer's float32 outputs feeds the next, and a unit whose
     # pre-activation is within rounding of zero may flip its ReLU mask; compare in a norm that tolerates that
     out_err = np.abs(_np(z[L]) - want["out"]).max()
