@@ -93,9 +93,9 @@ KERNEL_BYTES = {"gat_fwd": bytes_fwd, "gat_bwd_dst": bytes_bwd_dst, "gat_bwd_src
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one pass (rows + segments + merge launches),
 # from the one-pass ncu capture at full size summarised in profiles/span_kernels_large_launch_list.md.
 NCU_TRAFFIC_BYTES = {
-    ("large", "bf16", "gat_fwd"): 83.09e9,
-    ("large", "bf16", "gat_bwd_dst"): 86.28e9,
-    ("large", "bf16", "gat_bwd_src"): 91.87e9,
+    ("large", "bf16", "gat_fwd"): 81.85e9,
+    ("large", "bf16", "gat_bwd_dst"): 84.07e9,
+    ("large", "bf16", "gat_bwd_src"): 89.10e9,
 }
 
 
