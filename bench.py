@@ -46,6 +46,9 @@ def parse_args():
     ap.add_argument("--glue", action="store_true",
                     help="also run the layer glue each step: score projections before every aggregation, "
                          "ReLU after it, and their backward passes (default: aggregation kernels only)")
+    ap.add_argument("--ids", default="permuted", choices=["permuted", "degree_sorted"],
+                    help="node numbering of the power-law graph: seeded random permutation (the workload) or "
+                         "degree rank = id (locality ablation)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample", type=float, default=0.05, help="fraction of the workload the oracle is timed on")
@@ -262,7 +265,7 @@ def run_ours(args, rank, world, local_rank):
     threshold = args.threshold if args.threshold is not None else api.DEFAULT_THRESHOLD
 
     # ---- inputs (seeded, generated on the device; same recipe as the parity tests) --------------
-    src, dst = workloads.make_graph(cfg, device=dev)
+    src, dst = workloads.make_graph(cfg, device=dev, permute=args.ids == "permuted")
     e = src.numel()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
@@ -357,6 +360,10 @@ def run_ours(args, rank, world, local_rank):
                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                     "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dtype, dom)) if args.scale == 1.0 else None,
                     "algorithmic_bytes_per_launch": alg, "avg_launch_ms": passes[dom]["ms"]}
+    pass_ms = {k_: v["ms"] for k_, v in passes.items() if k_ in KERNEL_BYTES}
+    per_pass = {k_: {"ms": ms_, "edges_per_sec": e / (ms_ * 1e-3),
+                     "frac_of_roofline": KERNEL_BYTES[k_](n, e, H, F, b) / (ms_ * 1e-3) / 1e9 / peak}
+                for k_, ms_ in pass_ms.items()}
     step_bytes = L * bytes_layer_fwd_bwd(n, e, H, F, b)
     step_frac = step_bytes / (ms_per_step * 1e-3) / 1e9 / peak
 
@@ -420,14 +427,14 @@ def run_ours(args, rank, world, local_rank):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {
                 "workload": cfg.name, "n": n, "e": e, "heads": H, "feat_per_head": F, "layers": L, "partitions": K,
-                "storage_dtype": dtype, "layer_glue": bool(args.glue), "schedule": "fused row-stationary (sar_gat_fwd_fused / sar_gat_bwd_fused)",
+                "storage_dtype": dtype, "layer_glue": bool(args.glue), "ids": args.ids, "schedule": "fused row-stationary (sar_gat_fwd_fused / sar_gat_bwd_fused)",
                 "l2": "inputs_exceed_l2", "long_row_threshold": threshold, "parallelism": f"replicas x{world}",
                 "edges_x_heads_x_feat_per_sec": value * H * F,
             },
             "roofline": roofline,
             "step_roofline": {"compulsory_bytes_per_step": step_bytes, "frac_of_peak": step_frac, "peak": peak,
                               "peak_source": peak_src},
-            "kernels": kernels, "gpu_launches": launches, "prep_ms": prep_ms,
+            "passes": per_pass, "kernels": kernels, "gpu_launches": launches, "prep_ms": prep_ms,
             "peak_mem_bytes": peak_mem, "attention_bytes_if_stored": L * e * H * 4,
             "stats_bytes_kept": L * 2 * n * H * 4,
             "clocks": clocks, "e2e": e2e, "cpu_baseline": cpu,

@@ -55,11 +55,12 @@ CONFIGS = {
 }
 
 
-def make_graph(cfg: WorkloadConfig, device="cpu"):
-    """(src, dst) int32 edge list of the workload on `device`."""
+def make_graph(cfg: WorkloadConfig, device="cpu", permute: bool = True):
+    """(src, dst) int32 edge list of the workload on `device`.  permute=False keeps node id = degree
+    rank (hubs first): the locality ablation of the power-law workloads."""
     if cfg.graph == "uniform":
         return uniform_edges(cfg.n, cfg.e, cfg.seed, cfg.self_loops, device=device)
-    spec = ChungLuSpec(n=cfg.n, e=cfg.e, gamma=cfg.gamma, d_max=cfg.d_max, seed=cfg.seed)
+    spec = ChungLuSpec(n=cfg.n, e=cfg.e, gamma=cfg.gamma, d_max=cfg.d_max, seed=cfg.seed, permute=permute)
     return chung_lu_edges(spec, device=device)
 
 
