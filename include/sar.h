@@ -150,6 +150,28 @@ SAR_API sar_status sar_csr_split_indices(int64_t n_dst, const int64_t *indptr, c
                                  const int64_t *bounds, const int64_t *indptr_all, const int64_t *nnz_off,
                                  int32_t *indices_all, void *stream);
 
+/* Message-flow pruning (Appendix B: with few labelled nodes, a layer only has to update the nodes that can
+ * still influence a labelled node's output).  Both masks are DEVICE arrays of n bytes (0 / non-zero).
+ *
+ * sar_mfg_frontier: need_out marks the rows whose output of a layer is needed; need_in (written) marks the
+ * nodes whose INPUT to that layer is then needed: every needed row itself (its own features enter its
+ * score term el) and every source of one of its in-edges.  Apply it layer by layer from the labelled set
+ * backwards: need_out of layer l-1 = need_in of layer l.  The graph is the CSR by destination with n rows
+ * and n columns.
+ *
+ * sar_csr_filter_rows_*: the CSR in which only the rows with keep[i] != 0 keep their edges (the others
+ * become empty, so the aggregation kernels write zeros for them at no gather cost).  Two steps like the
+ * partition split: step 1 writes indptr_out [n+1] (scratch: sar_graph_workspace_bytes(0, n) bytes); the
+ * caller reads nnz_out = indptr_out[n], sizes indices_out, and step 2 copies the kept rows' column ids in
+ * their original order.  Integer work, bit-exact. */
+SAR_API sar_status sar_mfg_frontier(int64_t n, const int64_t *indptr, const int32_t *indices,
+                                    const uint8_t *need_out, uint8_t *need_in, void *stream);
+SAR_API sar_status sar_csr_filter_rows_indptr(int64_t n, const int64_t *indptr, const uint8_t *keep,
+                                              int64_t *indptr_out, void *workspace, size_t workspace_bytes,
+                                              void *stream);
+SAR_API sar_status sar_csr_filter_rows_indices(int64_t n, const int64_t *indptr, const int32_t *indices,
+                                               const int64_t *indptr_out, int32_t *indices_out, void *stream);
+
 /* Debug scan of one partition: indptr monotone from 0 to nnz, ids in range and ascending within a
  * row (both orientations when the CSC is present).  `flag` is 4 bytes of DEVICE scratch.
  * Synchronises the stream.  The hot calls never scan the graph. */

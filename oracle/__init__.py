@@ -279,3 +279,33 @@ def gat_stack(indptr, indices, feat0, a_l, a_r, gout, slope: float, storage=np.f
         dz_add, da_l[l], da_r[l] = project_bwd(z[l], a_l[l], a_r[l], b.del_.astype(np.float32), b.der.astype(np.float32))
         g = (b.dfeat.astype(storage).astype(np.float64) + dz_add)
     return dict(out=z[L].astype(np.float64), dfeat0=g, da_l=da_l, da_r=da_r)
+
+
+# --------------------------------------------------------------------------------------
+# message-flow pruning (Appendix B), plain numpy / Python loops
+# --------------------------------------------------------------------------------------
+
+def mfg_frontier(indptr, indices, need_out):
+    """need_in[j] = 1 if j's input to the layer can reach a needed output: j is a needed row itself
+    (its features enter its own score term) or the source of an in-edge of a needed row."""
+    indptr, indices = _i64(indptr), _i32(indices)
+    need_out = np.asarray(need_out).astype(bool)
+    need_in = need_out.copy()
+    for i in np.flatnonzero(need_out):
+        need_in[indices[indptr[i]:indptr[i + 1]]] = True
+    return need_in.astype(np.uint8)
+
+
+def csr_filter_rows(indptr, indices, keep):
+    """CSR in which the rows with keep[i] == 0 are empty; kept rows keep their column ids in order."""
+    indptr, indices = _i64(indptr), _i32(indices)
+    keep = np.asarray(keep).astype(bool)
+    n = indptr.shape[0] - 1
+    out_ptr = np.zeros(n + 1, dtype=np.int64)
+    rows = []
+    for i in range(n):
+        row = indices[indptr[i]:indptr[i + 1]] if keep[i] else indices[:0]
+        rows.append(row)
+        out_ptr[i + 1] = out_ptr[i] + row.shape[0]
+    out_idx = np.concatenate(rows).astype(np.int32) if rows else np.zeros(0, np.int32)
+    return out_ptr, out_idx

@@ -66,6 +66,49 @@ class Graph:
         return g
 
 
+def graph_from_csr(n: int, indptr: torch.Tensor, indices: torch.Tensor, k: int = 1,
+                   threshold: int = DEFAULT_THRESHOLD) -> Graph:
+    """A Graph from a CSR by destination already on the device (n rows, n columns)."""
+    dev = indptr.device
+    nnz = indices.numel()
+    ws = _workspace(B.sar_graph_workspace_bytes(nnz, n), dev)
+    t_indptr = torch.empty(n + 1, dtype=torch.int64, device=dev)
+    t_indices = torch.empty(nnz, dtype=torch.int32, device=dev)
+    B.sar_csr_transpose(n, n, indptr, indices, t_indptr, t_indices, ws)
+    split = build_plan(n, indptr, threshold) if threshold else None
+    t_split = build_plan(n, t_indptr, threshold) if threshold else None
+    whole = B.Part(n, n, indptr, indices, t_indptr, t_indices, split, t_split)
+    return Graph(n=n, nnz=nnz, whole=whole, k=k, bounds=B.sar_partition_bounds(n, k))
+
+
+def filter_rows(g: Graph, keep: torch.Tensor, threshold: int = DEFAULT_THRESHOLD) -> Graph:
+    """The graph in which only the destinations with keep[i] != 0 keep their in-edges."""
+    dev = keep.device
+    ws = _workspace(B.sar_graph_workspace_bytes(0, g.n), dev)
+    indptr = torch.empty(g.n + 1, dtype=torch.int64, device=dev)
+    B.sar_csr_filter_rows_indptr(g.n, g.whole.indptr, keep, indptr, ws)
+    nnz = int(indptr[-1].item())
+    indices = torch.empty(nnz, dtype=torch.int32, device=dev)
+    if nnz > 0:
+        B.sar_csr_filter_rows_indices(g.n, g.whole.indptr, g.whole.indices, indptr, indices)
+    return graph_from_csr(g.n, indptr, indices, k=g.k, threshold=threshold)
+
+
+def mfg_layers(g: Graph, labelled: torch.Tensor, layers: int, threshold: int = DEFAULT_THRESHOLD):
+    """Message-flow pruning for a stack of `layers` layers whose loss reads only the nodes with
+    labelled[i] != 0 (uint8 [n]).  Returns (graphs, need): graphs[l] is the graph layer l aggregates over
+    (only the rows whose output still matters keep their edges), need[l] marks the nodes whose input to
+    layer l matters (need[layers] = labelled)."""
+    need = [None] * (layers + 1)
+    graphs = [None] * layers
+    need[layers] = labelled.to(torch.uint8).contiguous()
+    for l in reversed(range(layers)):
+        graphs[l] = filter_rows(g, need[l + 1], threshold)
+        need[l] = torch.empty(g.n, dtype=torch.uint8, device=labelled.device)
+        B.sar_mfg_frontier(g.n, g.whole.indptr, g.whole.indices, need[l + 1], need[l])
+    return graphs, need
+
+
 def split_parts(whole: B.Part, bounds: List[int], threshold: int, ws: Optional[torch.Tensor] = None) -> List[B.Part]:
     """The K sub-graphs G_{p,q}: CSR with local source ids (split on the device) and CSC slices."""
     dev = whole.indptr.device

@@ -29,6 +29,7 @@ EXPORTS = [
     "sar_gat_bwd", "sar_gat_bwd_fused", "sar_spmm_agg", "sar_spmm_workspace_bytes", "sar_set_launch_hook",
     "sar_gat_stack_arena_bytes", "sar_gat_stack_host", "sar_gat_bwd_noalloc", "sar_gat_bwd_noalloc_limit",
     "sar_gat_project_workspace_bytes", "sar_gat_project", "sar_gat_project_bwd", "sar_relu", "sar_relu_bwd",
+    "sar_mfg_frontier", "sar_csr_filter_rows_indptr", "sar_csr_filter_rows_indices",
 ]
 
 
@@ -243,6 +244,26 @@ def sar_csr_split_indices(n_dst: int, indptr: torch.Tensor, indices: torch.Tenso
     _check("sar_csr_split_indices", lib().sar_csr_split_indices(c_int64(n_dst), _ptr(indptr), _ptr(indices),
                                                                 c_int32(k), _host_i64(bounds), _ptr(indptr_all),
                                                                 _host_i64(nnz_off), _ptr(indices_all), _stream()))
+
+
+def sar_mfg_frontier(n: int, indptr: torch.Tensor, indices: torch.Tensor, need_out: torch.Tensor,
+                     need_in: torch.Tensor) -> None:
+    _check("sar_mfg_frontier", lib().sar_mfg_frontier(c_int64(n), _ptr(indptr), _ptr(indices), _ptr(need_out),
+                                                      _ptr(need_in), _stream()))
+
+
+def sar_csr_filter_rows_indptr(n: int, indptr: torch.Tensor, keep: torch.Tensor, indptr_out: torch.Tensor,
+                               workspace: torch.Tensor) -> None:
+    w, wb = _ws(workspace)
+    _check("sar_csr_filter_rows_indptr", lib().sar_csr_filter_rows_indptr(c_int64(n), _ptr(indptr), _ptr(keep),
+                                                                          _ptr(indptr_out), w, wb, _stream()))
+
+
+def sar_csr_filter_rows_indices(n: int, indptr: torch.Tensor, indices: torch.Tensor, indptr_out: torch.Tensor,
+                                indices_out: torch.Tensor) -> None:
+    _check("sar_csr_filter_rows_indices", lib().sar_csr_filter_rows_indices(c_int64(n), _ptr(indptr), _ptr(indices),
+                                                                            _ptr(indptr_out), _ptr(indices_out),
+                                                                            _stream()))
 
 
 def sar_validate_part(part: Part, flag: torch.Tensor) -> None:

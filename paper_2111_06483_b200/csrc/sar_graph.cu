@@ -135,6 +135,38 @@ __global__ void validate_kernel(long long n_rows, long long n_cols, long long nn
     if (bad) *flag = 1;  // every writer stores the same value
 }
 
+
+// ---- message-flow pruning (Appendix B) ------------------------------------------------------------
+// One warp per destination row: an active row marks itself and every source it reads.  All writers
+// store the same value 1, so the races are benign and the result does not depend on the schedule.
+__global__ void mfg_frontier_kernel(long long n, const int64_t *__restrict__ indptr, const int32_t *__restrict__ indices,
+                                    const uint8_t *__restrict__ need_out, uint8_t *__restrict__ need_in) {
+    const long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (row >= n || !need_out[row]) return;
+    if (lane == 0) need_in[row] = 1;
+    const long long beg = indptr[row], end = indptr[row + 1];
+    for (long long t = beg + lane; t < end; t += 32) need_in[indices[t]] = 1;
+}
+
+// degrees of the kept rows, one slot to the right (ready for an inclusive scan)
+__global__ void filter_count_kernel(long long n, const int64_t *__restrict__ indptr, const uint8_t *__restrict__ keep,
+                                    int64_t *__restrict__ indptr_out) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    indptr_out[i + 1] = keep[i] ? indptr[i + 1] - indptr[i] : 0;
+    if (i == 0) indptr_out[0] = 0;
+}
+
+__global__ void filter_fill_kernel(long long n, const int64_t *__restrict__ indptr, const int32_t *__restrict__ indices,
+                                   const int64_t *__restrict__ indptr_out, int32_t *__restrict__ indices_out) {
+    const long long row = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (row >= n) return;
+    const long long w = indptr_out[row], cnt = indptr_out[row + 1] - w, beg = indptr[row];
+    for (long long t = lane; t < cnt; t += 32) indices_out[w + t] = indices[beg + t];
+}
+
 static inline unsigned nblk(long long n) { return (unsigned)((n + 255) / 256); }
 
 static size_t sort_temp_bytes(long long nnz) {
@@ -307,6 +339,47 @@ sar_status sar_csr_split_indices(int64_t n_dst, const int64_t *indptr, const int
     if (!indices || !indices_all) return SAR_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     split_fill_kernel<<<nblk(n_dst), 256, 0, st>>>(n_dst, indptr, indices, b, off, indptr_all, indices_all);
+    return sar_after_launch();
+}
+
+sar_status sar_mfg_frontier(int64_t n, const int64_t *indptr, const int32_t *indices, const uint8_t *need_out,
+                            uint8_t *need_in, void *stream) {
+    if (n < 0 || (n > 0 && (!indptr || !need_out || !need_in))) return SAR_ERR_INVALID_ARG;
+    if (n > INT32_MAX) return SAR_ERR_UNSUPPORTED;
+    if (!sar_aligned(indptr, 8) || !sar_aligned(indices, 4)) return SAR_ERR_ALIGNMENT;
+    if (n == 0) return SAR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SAR_CUDA_TRY(cudaMemsetAsync(need_in, 0, (size_t)n, st));
+    mfg_frontier_kernel<<<nblk(n * 32), 256, 0, st>>>(n, indptr, indices, need_out, need_in);
+    return sar_after_launch();
+}
+
+sar_status sar_csr_filter_rows_indptr(int64_t n, const int64_t *indptr, const uint8_t *keep, int64_t *indptr_out,
+                                      void *workspace, size_t workspace_bytes, void *stream) {
+    if (n < 0 || !indptr_out || (n > 0 && (!indptr || !keep))) return SAR_ERR_INVALID_ARG;
+    if (!sar_aligned(indptr, 8) || !sar_aligned(indptr_out, 8)) return SAR_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (n == 0) {
+        SAR_CUDA_TRY(cudaMemsetAsync(indptr_out, 0, 8, st));
+        return SAR_OK;
+    }
+    filter_count_kernel<<<nblk(n), 256, 0, st>>>(n, indptr, keep, indptr_out);
+    SAR_TRY(sar_after_launch());
+    size_t need = 0;
+    SAR_CUDA_TRY(cub::DeviceScan::InclusiveSum(nullptr, need, indptr_out, indptr_out, n + 1, st));
+    if (!workspace || workspace_bytes < need) return SAR_ERR_WORKSPACE;
+    SAR_CUDA_TRY(cub::DeviceScan::InclusiveSum(workspace, need, indptr_out, indptr_out, n + 1, st));
+    return SAR_OK;
+}
+
+sar_status sar_csr_filter_rows_indices(int64_t n, const int64_t *indptr, const int32_t *indices,
+                                       const int64_t *indptr_out, int32_t *indices_out, void *stream) {
+    if (n < 0 || (n > 0 && (!indptr || !indptr_out))) return SAR_ERR_INVALID_ARG;
+    if (n == 0) return SAR_OK;
+    if (!indices || !indices_out) return SAR_ERR_INVALID_ARG;
+    if (!sar_aligned(indices, 4) || !sar_aligned(indices_out, 4)) return SAR_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    filter_fill_kernel<<<nblk(n * 32), 256, 0, st>>>(n, indptr, indices, indptr_out, indices_out);
     return sar_after_launch();
 }
 

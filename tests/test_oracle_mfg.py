@@ -1,0 +1,80 @@
+"""Pins for the oracle's message-flow pruning (Appendix B), CPU only: a dense boolean formulation, the
+definition by reachability, and the invariance it exists for (pruned and full stacks agree on the
+labelled nodes)."""
+import numpy as np
+
+import oracle
+from helpers import count_matrix, small_problem
+
+
+def test_frontier_is_the_boolean_matrix_product():
+    p = small_problem(60, 240, 1, 4, 3)
+    rng = np.random.default_rng(0)
+    C = count_matrix(60, 60, p["src"], p["dst"]) > 0  # C[i, j]: some edge j -> i
+    for density in (0.0, 0.05, 0.3, 1.0):
+        need_out = rng.random(60) < density
+        want = need_out | (C.T.astype(np.int64) @ need_out.astype(np.int64) > 0)
+        got = oracle.mfg_frontier(p["indptr"], p["indices"], need_out)
+        assert np.array_equal(got.astype(bool), want)
+
+
+def test_repeated_frontier_is_bounded_reachability():
+    # nodes whose layer-0 input matters for a 3-layer stack = nodes with a directed walk of length <= 3 to a labelled node
+    p = small_problem(50, 120, 1, 4, 5)
+    A = (count_matrix(50, 50, p["src"], p["dst"]) > 0).astype(np.int64)  # A[i, j]: j -> i
+    labelled = np.zeros(50, dtype=bool)
+    labelled[[3, 17]] = True
+    need = labelled
+    for _ in range(3):
+        need = oracle.mfg_frontier(p["indptr"], p["indices"], need).astype(bool)
+    reach = np.eye(50, dtype=np.int64)
+    total = reach.copy()
+    for _ in range(3):
+        reach = (reach @ A > 0).astype(np.int64)  # reach[i, j]: walk j -> ... -> i of this length
+        total = ((total + reach) > 0).astype(np.int64)
+    want = total[labelled].sum(axis=0) > 0
+    assert np.array_equal(need, want)
+
+
+def test_filter_rows_keeps_slices_and_empties_the_rest():
+    p = small_problem(40, 300, 1, 4, 7, self_loops=True)
+    keep = np.arange(40) % 3 != 0
+    ptr, idx = oracle.csr_filter_rows(p["indptr"], p["indices"], keep)
+    assert ptr[0] == 0 and ptr[-1] == idx.shape[0]
+    for i in range(40):
+        row = idx[ptr[i]:ptr[i + 1]]
+        if keep[i]:
+            assert np.array_equal(row, p["indices"][p["indptr"][i]:p["indptr"][i + 1]])
+        else:
+            assert row.shape[0] == 0
+    # as an edge multiset: exactly the edges whose destination is kept
+    dst_of = np.repeat(np.arange(40), np.diff(p["indptr"]))
+    assert idx.shape[0] == int(keep[dst_of].sum())
+
+
+def test_pruned_stack_agrees_with_the_full_stack_on_the_labelled_nodes():
+    p = small_problem(80, 400, 2, 4, 11)
+    rng = np.random.default_rng(2)
+    L = 2
+    a_l = [rng.standard_normal((2, 4)) * 0.5 for _ in range(L)]
+    a_r = [rng.standard_normal((2, 4)) * 0.5 for _ in range(L)]
+    labelled = np.zeros(80, dtype=bool)
+    labelled[[5, 40, 41]] = True
+
+    def stack(graphs):
+        z = p["feat"].astype(np.float64)
+        for l in range(L):
+            ptr, idx = graphs[l]
+            el, er = oracle.project(z, a_l[l], a_r[l])
+            z = np.maximum(oracle.gat_fwd(ptr, idx, z.astype(np.float32), el.astype(np.float32), er.astype(np.float32), 0.2).out, 0.0)
+        return z
+
+    full = stack([(p["indptr"], p["indices"])] * L)
+    need = labelled
+    graphs = [None] * L
+    for l in reversed(range(L)):
+        graphs[l] = oracle.csr_filter_rows(p["indptr"], p["indices"], need)
+        need = oracle.mfg_frontier(p["indptr"], p["indices"], need).astype(bool)
+    pruned = stack(graphs)
+    assert np.array_equal(pruned[labelled], full[labelled])
+    assert sum(g[1].shape[0] for g in graphs) < L * p["indices"].shape[0]
