@@ -268,6 +268,18 @@ SAR_API sar_status sar_spmm_agg(const sar_part *g, const void *feat_q, int32_t F
                         void *stream);
 SAR_API size_t sar_spmm_workspace_bytes(const sar_part *g, int32_t F, sar_dtype t);
 
+/* Weighted sum aggregation: out[i,:] (+)= dst_scale[i] * sum over this partition's in-edges of
+ * src_scale[j] * feat_q[j,:] - the propagation step X <- S X with S = diag(dst_scale) A diag(src_scale),
+ * e.g. the symmetrically normalised adjacency (both scales = degree^-1/2) of the label-propagation
+ * post-processing the paper combines SAR with (Sec. 4.2).  src_scale [n_src] and dst_scale [n_dst] are
+ * float32 DEVICE arrays; either may be NULL (= all ones).  The factors are applied on the fly, nothing of
+ * size E is stored.  SAR_FIRST overwrites out, otherwise the partition's weighted sum is added; SAR_MEAN is
+ * not accepted (SAR_ERR_INVALID_ARG).  Workspace and other conventions as for sar_spmm_agg.  The backward
+ * pass is this call on the transposed partition with the two scale arrays exchanged. */
+SAR_API sar_status sar_spmm_agg_scaled(const sar_part *g, const void *feat_q, int32_t F, sar_dtype t, uint32_t flags,
+                                       const float *src_scale, const float *dst_scale, void *out, void *workspace,
+                                       size_t workspace_bytes, void *stream);
+
 /* ---------------------------------------------------------------------------------------------
  * The rest of a GAT layer around the aggregation (Eq. 3; Eq. 1's f_node reduced to a ReLU).
  *   sar_gat_project      el[i,h] = <z[i,h,:], a_l[h,:]>, er[i,h] = <z[i,h,:], a_r[h,:]>: the two halves of

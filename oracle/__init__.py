@@ -309,3 +309,20 @@ def csr_filter_rows(indptr, indices, keep):
         out_ptr[i + 1] = out_ptr[i] + row.shape[0]
     out_idx = np.concatenate(rows).astype(np.int32) if rows else np.zeros(0, np.int32)
     return out_ptr, out_idx
+
+
+def spmm_scaled(indptr, indices, feat, src_scale=None, dst_scale=None):
+    """out[i,:] = dst_scale[i] * sum over the in-edges (j -> i) of src_scale[j] * feat[j,:], float64
+    (the propagation X <- diag(dst_scale) A diag(src_scale) X; a missing scale is all ones)."""
+    feat = np.asarray(feat, dtype=np.float64)
+    x = feat if src_scale is None else feat * np.asarray(src_scale, np.float64)[:, None]
+    indptr, indices = _i64(indptr), _i32(indices)
+    n = indptr.shape[0] - 1
+    out = np.zeros((n, feat.shape[1]), dtype=np.float64)
+    for i in range(n):
+        cols = indices[indptr[i]:indptr[i + 1]]
+        if cols.shape[0]:
+            out[i] = x[cols].sum(axis=0)
+    if dst_scale is not None:
+        out *= np.asarray(dst_scale, np.float64)[:, None]
+    return out

@@ -238,3 +238,14 @@ def gat_layer_backward(g: Graph, z: torch.Tensor, a_l: torch.Tensor, a_r: torch.
     ws = _workspace(B.sar_gat_project_workspace_bytes(H, F), z.device)
     B.sar_gat_project_bwd(z, a_l, a_r, del_, der, dz, da_l, da_r, ws, B.SAR_GLUE_RELU if relu_input else 0)
     return dz, da_l, da_r
+
+
+def spmm_scaled(part: B.Part, feat: torch.Tensor, src_scale: Optional[torch.Tensor] = None,
+                dst_scale: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None, first: bool = True):
+    """out[i,:] (+)= dst_scale[i] * sum over the in-edges of i of src_scale[j] * feat[j,:] (one partition)."""
+    F = feat.shape[1]
+    if out is None:
+        out = torch.empty((part.n_dst, F), dtype=feat.dtype, device=feat.device)
+    ws = _workspace(B.sar_spmm_workspace_bytes(part, F, B._dtype(feat)), feat.device)
+    B.sar_spmm_agg_scaled(part, feat, F, (B.SAR_FIRST if first else 0) | B.SAR_LAST, src_scale, dst_scale, out, ws)
+    return out

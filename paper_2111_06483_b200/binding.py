@@ -29,7 +29,7 @@ EXPORTS = [
     "sar_gat_bwd", "sar_gat_bwd_fused", "sar_spmm_agg", "sar_spmm_workspace_bytes", "sar_set_launch_hook",
     "sar_gat_stack_arena_bytes", "sar_gat_stack_host", "sar_gat_bwd_noalloc", "sar_gat_bwd_noalloc_limit",
     "sar_gat_project_workspace_bytes", "sar_gat_project", "sar_gat_project_bwd", "sar_relu", "sar_relu_bwd",
-    "sar_mfg_frontier", "sar_csr_filter_rows_indptr", "sar_csr_filter_rows_indices",
+    "sar_mfg_frontier", "sar_csr_filter_rows_indptr", "sar_csr_filter_rows_indices", "sar_spmm_agg_scaled",
 ]
 
 
@@ -359,6 +359,15 @@ def sar_spmm_agg(part: Part, feat_q: torch.Tensor, F: int, flags: int, deg_total
     w, wb = _ws(workspace)
     _check("sar_spmm_agg", lib().sar_spmm_agg(byref(part.c), _ptr(feat_q), c_int32(F), ctypes.c_int(_dtype(feat_q)),
                                               c_uint32(flags), _ptr(deg_total), _ptr(out), w, wb, _stream()))
+
+
+def sar_spmm_agg_scaled(part: Part, feat_q: torch.Tensor, F: int, flags: int, src_scale: Optional[torch.Tensor],
+                        dst_scale: Optional[torch.Tensor], out: torch.Tensor, workspace: Optional[torch.Tensor]) -> None:
+    w, wb = _ws(workspace)
+    _check("sar_spmm_agg_scaled", lib().sar_spmm_agg_scaled(byref(part.c), _ptr(feat_q), c_int32(F),
+                                                            ctypes.c_int(_dtype(feat_q)), c_uint32(flags),
+                                                            _ptr(src_scale), _ptr(dst_scale), _ptr(out), w, wb,
+                                                            _stream()))
 
 
 # ----------------------------------------------------------------------------------------------

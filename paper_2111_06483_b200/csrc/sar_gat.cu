@@ -551,15 +551,17 @@ sar_status sar_gat_bwd_fused(const sar_part *g, int32_t k, const int64_t *bounds
 }
 
 // ---------------------------------------------------------------------------------------------
-sar_status sar_spmm_agg(const sar_part *g, const void *feat_q, int32_t F, sar_dtype t, uint32_t flags,
-                        const int64_t *deg_total, void *out, void *workspace, size_t workspace_bytes,
-                        void *stream) {
+static sar_status spmm_impl(const sar_part *g, const void *feat_q, int32_t F, sar_dtype t, uint32_t flags,
+                            const int64_t *deg_total, const float *src_scale, const float *dst_scale, void *out,
+                            void *workspace, size_t workspace_bytes, void *stream) {
     SAR_TRY(check_part(g, false));
     if (flags & ~(SAR_FIRST | SAR_LAST | SAR_MEAN)) return SAR_ERR_INVALID_ARG;
     if (!out || (g->n_src > 0 && !feat_q)) return SAR_ERR_INVALID_ARG;
     if ((flags & SAR_MEAN) && (flags & SAR_LAST) && !deg_total) return SAR_ERR_INVALID_ARG;
     SAR_TRY(check_elem_align({feat_q, out}, sar_elem_size(t)));
     SAR_TRY(check_elem_align({deg_total}, 8));
+    SAR_TRY(check_elem_align({src_scale, dst_scale}, 4));
+    const bool weighted = src_scale || dst_scale;
     Shape s;
     SAR_TRY(make_shape(1, F, t, all16({feat_q, out}), &s));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -572,6 +574,8 @@ sar_status sar_spmm_agg(const sar_part *g, const void *feat_q, int32_t F, sar_dt
         a.feat = feat_q;
         a.out = out;
         a.deg_total = deg_total;
+        a.src_scale = src_scale;
+        a.dst_scale = dst_scale;
         a.H = 1;
         a.F = F;
         a.flags = flags;
@@ -592,6 +596,7 @@ sar_status sar_spmm_agg(const sar_part *g, const void *feat_q, int32_t F, sar_dt
     ma.feat = feat_q;
     ma.out = out;
     ma.deg_total = deg_total;
+    ma.dst_scale = dst_scale;
     ma.flags = flags;
     ma.g = s.geom;
     ma.sp = split_args(g->split, static_cast<float *>(workspace), 1, F, true);
@@ -603,19 +608,37 @@ sar_status sar_spmm_agg(const sar_part *g, const void *feat_q, int32_t F, sar_dt
     a.gather = feat_q;
     a.out = out;
     a.deg_total = deg_total;
+    a.src_scale = src_scale;
+    a.dst_scale = dst_scale;
     a.flags = flags;
     a.g = s.geom;
     a.sp = ma.sp;
     return dispatch(s, [&](auto cfg) -> sar_status {
         using C = decltype(cfg);
         using T = typename C::type;
-        SAR_TRY((launch_span<T, C::g, C::v, UFwd<C::v>::u, kSum, kCapSum, kMinBlocksFwd>(a, g->nnz, "spmm", "spmm_seg", st)));
+        if (weighted)
+            SAR_TRY((launch_span<T, C::g, C::v, UFwd<C::v>::u, kSumW, kCapSum, kMinBlocksFwd>(a, g->nnz, "spmm", "spmm_seg", st)));
+        else
+            SAR_TRY((launch_span<T, C::g, C::v, UFwd<C::v>::u, kSum, kCapSum, kMinBlocksFwd>(a, g->nnz, "spmm", "spmm_seg", st)));
         if (ma.sp.threshold > 0) {
             SAR_LAUNCH("spmm_merge", st, spmm_merge_kernel<T, C::g, C::v><<<blocks_for(ma.sp.n_long, C::g), kThreads, 0, st>>>(ma));
             SAR_TRY(sar_after_launch());
         }
         return SAR_OK;
     });
+}
+
+sar_status sar_spmm_agg(const sar_part *g, const void *feat_q, int32_t F, sar_dtype t, uint32_t flags,
+                        const int64_t *deg_total, void *out, void *workspace, size_t workspace_bytes,
+                        void *stream) {
+    return spmm_impl(g, feat_q, F, t, flags, deg_total, nullptr, nullptr, out, workspace, workspace_bytes, stream);
+}
+
+sar_status sar_spmm_agg_scaled(const sar_part *g, const void *feat_q, int32_t F, sar_dtype t, uint32_t flags,
+                               const float *src_scale, const float *dst_scale, void *out, void *workspace,
+                               size_t workspace_bytes, void *stream) {
+    if (flags & SAR_MEAN) return SAR_ERR_INVALID_ARG;
+    return spmm_impl(g, feat_q, F, t, flags, nullptr, src_scale, dst_scale, out, workspace, workspace_bytes, stream);
 }
 
 }  // extern "C"

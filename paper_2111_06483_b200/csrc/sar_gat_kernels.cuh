@@ -350,6 +350,7 @@ struct SumArgs {
     const void *feat;
     void *out;
     const int64_t *deg_total;  // for SAR_MEAN
+    const float *dst_scale;    // per-row factor of the weighted sum, or null
     unsigned flags;
     RowGeom g;                 // H = 1, vph = n_vec
     SplitArgs sp;
@@ -360,6 +361,13 @@ template <typename T, int G, int V>
 __device__ __forceinline__ void sum_epilogue(const SumArgs &a, int gl, const VecGeom<G, V> &vg, long long row,
                                              float (&acc)[V][Elem<T>::EPV]) {
     constexpr int EPV = Elem<T>::EPV;
+    if (a.dst_scale) {
+        const float ds = a.dst_scale[row];
+#pragma unroll
+        for (int v = 0; v < V; ++v)
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) acc[v][e] *= ds;
+    }
     if (!(a.flags & SAR_FIRST)) {
         float old[V][EPV];
         load_row_vec<T, G, V, false>(a.out, row, a.g.n_vec, gl, vg.vok, old);

@@ -24,6 +24,7 @@ struct GenericArgs {
     float *del, *der, *D;
     float4 *rec;
     const int64_t *deg_total;
+    const float *src_scale, *dst_scale;
     int H, F;
     float slope;
     unsigned flags;
@@ -183,7 +184,12 @@ __global__ void spmm_generic(const GenericArgs a) {
     const T *feat = reinterpret_cast<const T *>(a.feat);
     T *out = reinterpret_cast<T *>(a.out);
     float acc = 0.f;
-    for (long long t = beg; t < end; ++t) acc += Elem<T>::load1(feat + (long long)a.indices[t] * a.F + f);
+    for (long long t = beg; t < end; ++t) {
+        const long long j = a.indices[t];
+        const float x = Elem<T>::load1(feat + j * a.F + f);
+        acc = a.src_scale ? fmaf(a.src_scale[j], x, acc) : acc + x;
+    }
+    if (a.dst_scale) acc *= a.dst_scale[row];
     if (!first) acc += Elem<T>::load1(out + idx);
     if (mean) {
         const long long dg = a.deg_total[row];

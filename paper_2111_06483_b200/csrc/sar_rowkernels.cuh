@@ -21,7 +21,7 @@ struct SplitArgs {
     long long pstride;        // floats per segment
 };
 
-enum GatherMode { kFwd = 0, kBwdDst = 1, kBwdDstGivenD = 2, kBwdSrc = 3, kSum = 4 };
+enum GatherMode { kFwd = 0, kBwdDst = 1, kBwdDstGivenD = 2, kBwdSrc = 3, kSum = 4, kSumW = 5 };
 
 template <int MODE>
 struct WeightOf {

@@ -46,6 +46,7 @@ struct SpanArgs {
     void *out;               // forward: out; bwd-src: dfeat; sum: out
     float *del, *der;
     const int64_t *deg_total;
+    const float *src_scale, *dst_scale;  // weighted sum (kSumW): per-source factor, per-row factor (either may be null)
     float slope;
     unsigned flags;
     RowGeom g;
@@ -369,7 +370,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
             }
         };
         float ca[2][3];
-        if constexpr (MODE != kSum) {
+        if constexpr (MODE != kSum && MODE != kSumW) {
             load_consts(lane, ca[0][0], ca[0][1], ca[0][2]);
             load_consts(lane + 32, ca[1][0], ca[1][1], ca[1][2]);
         }
@@ -392,7 +393,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
             }
             for (int q = npos + lane; q < npos + S * EPW; q += 32) sj[q] = -1;  // the ring's run-out
         }
-        if constexpr (MODE != kSum) {
+        if constexpr (MODE != kSum && MODE != kSumW) {
             store_consts(lane, ca[0][0], ca[0][1], ca[0][2]);
             store_consts(lane + 32, ca[1][0], ca[1][1], ca[1][2]);
             for (int x = lane + 64; x < nr * Hp; x += 32) {  // many heads x many rows: the rest, plainly
@@ -415,7 +416,24 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
         for (int s_ = 0; s_ < S; ++s_) issue(s_, stage_s + s_ * (V * 512));
 
         // ---- stage C: weight records, two positions per lane and sweep, all their heads -----------
-        if constexpr (MODE != kSum) {
+        if constexpr (MODE == kSumW) {
+            // weighted sum: one factor per edge, the source's
+            for (int q0 = lane; q0 < npos; q0 += 64) {
+                float w[2] = {0.f, 0.f};
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int q = q0 + 32 * u;
+                    if (q < npos) {
+                        const int col = sj[q];
+                        if (col >= 0) w[u] = a.src_scale ? __ldg(a.src_scale + col) : 1.f;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 2; ++u)
+                    if (q0 + 32 * u < npos) reinterpret_cast<float *>(sw)[q0 + 32 * u] = w[u];
+            }
+            __syncwarp();
+        } else if constexpr (MODE != kSum) {
             const bool vec4 = a.hvec != 0;  // heads handled four at a time with 16-byte accesses
             int i = 0;
             for (int q0 = lane; q0 < npos; q0 += 64) {
@@ -633,7 +651,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                         const f32x2 one = pack2(1.f, 1.f);
 #pragma unroll
                         for (int k = 0; k < NP; ++k) pacc0[v][k] = fma2(x[k], one, pacc0[v][k]);
-                    } else if constexpr (kFwdMode) {
+                    } else if constexpr (kFwdMode || MODE == kSumW) {
                         const float w = lds_f32(w_s[v] + woff);
                         sv[v] += w;
                         const f32x2 w2 = pack2(w, w);
@@ -830,6 +848,13 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                 if (a.mode == 1) {
                     if (writer) store_acc_row<G, V, EPV>(a.sp.part + seg * a.sp.pstride, gl, vok, acc0);
                 } else if (writer) {
+                    if (a.dst_scale) {
+                        const float ds = a.dst_scale[row];
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+#pragma unroll
+                            for (int e = 0; e < EPV; ++e) acc0[v][e] *= ds;
+                    }
                     if (!(a.flags & SAR_FIRST)) {
                         float old[V][EPV];
                         load_row_vec<T, G, V, false>(a.out, row, n_vec, gl, vok, old);

@@ -1,4 +1,4 @@
-"""Pins for the oracle's message-flow pruning (Appendix B), CPU only: a dense boolean formulation, the
+"""Pins for the oracle's message-flow pruning (Appendix B) and weighted propagation, CPU only: dense formulations, the
 definition by reachability, and the invariance it exists for (pruned and full stacks agree on the
 labelled nodes)."""
 import numpy as np
@@ -78,3 +78,23 @@ def test_pruned_stack_agrees_with_the_full_stack_on_the_labelled_nodes():
     pruned = stack(graphs)
     assert np.array_equal(pruned[labelled], full[labelled])
     assert sum(g[1].shape[0] for g in graphs) < L * p["indices"].shape[0]
+
+
+def test_scaled_sum_is_the_sparse_matrix_product():
+    import scipy.sparse as sp
+    p = small_problem(70, 500, 1, 6, 17, self_loops=True, empty_rows=3)
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((70, 6))
+    s_src, s_dst = rng.random(70) + 0.5, rng.random(70) + 0.5
+    A = sp.csr_matrix((np.ones(len(p["indices"])), p["indices"], p["indptr"]), shape=(70, 70))  # duplicates add up
+    want = sp.diags(s_dst) @ (A @ (sp.diags(s_src) @ x))
+    assert np.allclose(oracle.spmm_scaled(p["indptr"], p["indices"], x, s_src, s_dst), want, rtol=1e-13, atol=1e-13)
+    assert np.allclose(oracle.spmm_scaled(p["indptr"], p["indices"], x), A @ x, rtol=1e-13, atol=1e-13)
+    # symmetric normalisation of an undirected graph: the constant vector d^(1/2) is a fixed point
+    src = np.concatenate([p["src"], p["dst"]])
+    dst = np.concatenate([p["dst"], p["src"]])
+    ptr, idx = oracle.csr_from_coo(70, 70, src, dst)
+    deg = np.diff(ptr).astype(np.float64)
+    s = np.where(deg > 0, 1.0 / np.sqrt(np.maximum(deg, 1)), 0.0)
+    v = np.sqrt(deg)[:, None]
+    assert np.allclose(oracle.spmm_scaled(ptr, idx, v, s, s), v, rtol=1e-12, atol=1e-12)
