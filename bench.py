@@ -94,7 +94,7 @@ def bytes_layer_fwd_bwd(n, e, H, F, b):
 KERNEL_BYTES = {"gat_fwd": bytes_fwd, "gat_bwd_dst": bytes_bwd_dst, "gat_bwd_src": bytes_bwd_src}
 
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one pass (rows + segments + merge launches),
-# from the one-pass ncu capture at full size summarised in profiles/span_kernels_large_launch_list.md.
+# from the one-pass ncu capture at full size whose launch list is summarised under profiles/.
 NCU_TRAFFIC_BYTES = {
     ("large", "bf16", "gat_fwd"): 81.85e9,
     ("large", "bf16", "gat_bwd_dst"): 84.07e9,
