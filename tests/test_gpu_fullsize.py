@@ -156,3 +156,51 @@ def test_stack_host_entry_point_matches_device_calls():
             gr, dl, dr = api.gat_backward(g, xin, els[l].to(DEV), ers[l].to(DEV), m, d, gr, cfg.slope)
             assert torch.equal(dl.cpu(), h_del[l]) and torch.equal(dr.cpu(), h_der[l])
         assert torch.equal(gr.cpu(), h_dfeat)
+
+
+def test_more_than_two_to_the_31_edges():
+    """Maximum sizes: an edge count that does not fit 32 bits (edge offsets are 64-bit throughout).  No oracle
+    can visit 2.3 G edges in test time, so the checks are the ones that hold at any size: the CSR's degrees
+    equal a count of the destination ids made with torch, the library's own scan finds it well formed, the
+    sum of an all-ones feature is the degree (exact in float32 below 2^24), and an attention layer over
+    constant features returns that constant with d = degree and m = 0 when all scores are zero."""
+    from paper_2111_06483_b200 import binding as B
+    if torch.cuda.get_device_properties(0).total_memory < 120e9:
+        pytest.skip("needs about 90 GB of device memory")
+    n, e = 2_000_000, (1 << 31) + (1 << 27)
+    spec = workloads.ChungLuSpec(n=n, e=e, gamma=2.1, d_max=100_000.0, seed=31)
+    src, dst = workloads.chung_lu_edges(spec, device=DEV)
+    deg = torch.zeros(n, dtype=torch.int64, device=DEV)
+    for lo in range(0, e, 1 << 28):
+        deg += torch.bincount(dst[lo:lo + (1 << 28)].long(), minlength=n)
+    g = api.Graph.from_coo(n, src, dst, k=1)
+    del src, dst
+    torch.cuda.empty_cache()
+    assert g.nnz == e and int(g.whole.indptr[-1]) == e and e > 2 ** 31
+    assert torch.equal(g.whole.indptr[1:] - g.whole.indptr[:-1], deg)
+    assert int((g.whole.t_indptr[1:] - g.whole.t_indptr[:-1]).sum()) == e
+    flag = torch.zeros(1, dtype=torch.int32, device=DEV)
+    B.sar_validate_part(g.whole, flag)  # raises on a malformed CSR / CSC
+    assert int(deg.max()) < 2 ** 24
+    ones = torch.ones((n, 8), dtype=torch.float32, device=DEV)
+    assert torch.equal(api.spmm_sum(g.whole, ones), deg.float()[:, None].expand(n, 8))
+    # the rows at the far end of the edge array in particular
+    tail = torch.nonzero(g.whole.indptr[:-1] > 2 ** 31).flatten()
+    assert tail.numel() > 1000
+    H, F = 2, 8
+    feat = torch.full((n, H, F), 3.0, dtype=torch.float32, device=DEV)
+    zeros = torch.zeros((n, H), dtype=torch.float32, device=DEV)
+    out, m, d = api.gat_forward(g, feat, zeros, zeros, 0.2)
+    has = deg > 0
+    assert torch.equal(d, deg.float()[:, None].expand(n, H))
+    assert torch.equal(m[has], torch.zeros_like(m[has])) and bool(torch.isinf(m[~has]).all())
+    want = torch.where(has[:, None, None], torch.full_like(out, 3.0), torch.zeros_like(out))
+    assert float((out - want).abs().max()) <= 3.0 * 1e-5
+    # backward: with constant features every d(alpha) equals D, so del = der = 0, and sum_j dfeat[j] = sum_i gout[i] over the rows with edges
+    gout = torch.ones_like(feat)
+    dfeat, del_, der = api.gat_backward(g, feat, zeros, zeros, m, d, gout, 0.2)
+    assert float(del_.abs().max()) <= 1e-3 and float(der.abs().max()) <= 1e-3
+    total = float(dfeat[:, 0, 0].double().sum())
+    assert abs(total - float(has.sum())) <= 1e-4 * float(has.sum())   # sum_j dfeat[j] = number of rows with edges
+    del g, feat, out, dfeat
+    torch.cuda.empty_cache()
