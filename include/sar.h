@@ -350,7 +350,20 @@ SAR_API sar_status sar_gat_bwd_noalloc(const sar_part *g, const void *feat, cons
  * once `stream` has completed, every output is in host memory.  Returns without synchronising; use
  * pinned host memory for the copies to be asynchronous.  The host inputs must stay unchanged, and
  * `arena` untouched, until then.
+ *
+ * Pipelined mode (io->flags = SAR_STACK_PIPELINED) for a sequence of calls, e.g. one per training step:
+ * `arena` holds TWO working sets (2 x sar_gat_stack_arena_bytes) used alternately, so that the input
+ * copies of call t+1 run while the kernels of call t are still busy and its results are still on their
+ * way back.  In this mode
+ *   - the input copies are NOT ordered after earlier work on `stream` (only the kernels are): the host
+ *     inputs must already hold their values when the call is made;
+ *   - `stream` does not wait for the result copies of the call: sar_gat_stack_host_wait(stream) makes it
+ *     wait for everything the pipelined calls on this device have in flight (call it before reading
+ *     results on the host, reusing the host inputs, freeing the arena, or switching mode);
+ *   - results of successive calls arrive in call order (one copy stream), so calls may share their host
+ *     output buffers if only the last result matters.
  * ------------------------------------------------------------------------------------------- */
+#define SAR_STACK_PIPELINED 1u
 typedef struct {
     int32_t L, H, F;
     sar_dtype t;
@@ -365,6 +378,7 @@ typedef struct {
     void *dfeat0;             /* [n,H,F] type t                                          */
     float *const *del;        /* HOST array of L HOST pointers, each [n,H], or NULL      */
     float *const *der;        /* idem                                                    */
+    uint32_t flags;           /* 0 or SAR_STACK_PIPELINED                                */
 } sar_stack_host_io;
 
 /* DEVICE bytes sar_gat_stack_host needs in `arena` for this graph and shape. */
@@ -375,6 +389,10 @@ SAR_API size_t sar_gat_stack_arena_bytes(const sar_part *g, int32_t L, int32_t H
 SAR_API sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bounds,
                                       const sar_stack_host_io *io, void *arena, size_t arena_bytes,
                                       void *stream);
+
+/* Makes `stream` wait for every copy that pipelined calls of sar_gat_stack_host on the current device
+ * still have in flight.  Does not block the host. */
+SAR_API sar_status sar_gat_stack_host_wait(void *stream);
 
 #ifdef __cplusplus
 }

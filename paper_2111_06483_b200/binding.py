@@ -30,6 +30,7 @@ EXPORTS = [
     "sar_gat_stack_arena_bytes", "sar_gat_stack_host", "sar_gat_bwd_noalloc", "sar_gat_bwd_noalloc_limit",
     "sar_gat_project_workspace_bytes", "sar_gat_project", "sar_gat_project_bwd", "sar_relu", "sar_relu_bwd",
     "sar_mfg_frontier", "sar_csr_filter_rows_indptr", "sar_csr_filter_rows_indices", "sar_spmm_agg_scaled",
+    "sar_gat_stack_host_wait",
 ]
 
 
@@ -377,7 +378,11 @@ def sar_spmm_agg_scaled(part: Part, feat_q: torch.Tensor, F: int, flags: int, sr
 class sar_stack_host_io(Structure):
     _fields_ = [("L", c_int32), ("H", c_int32), ("F", c_int32), ("t", ctypes.c_int), ("slope", c_float),
                 ("feat0", c_void_p), ("el", POINTER(c_void_p)), ("er", POINTER(c_void_p)), ("gout", c_void_p),
-                ("out_last", c_void_p), ("dfeat0", c_void_p), ("del_", POINTER(c_void_p)), ("der", POINTER(c_void_p))]
+                ("out_last", c_void_p), ("dfeat0", c_void_p), ("del_", POINTER(c_void_p)), ("der", POINTER(c_void_p)),
+                ("flags", c_uint32)]
+
+
+SAR_STACK_PIPELINED = 1
 
 
 def sar_gat_stack_arena_bytes(part: Part, L: int, H: int, F: int, dtype: int) -> int:
@@ -401,15 +406,20 @@ def sar_gat_stack_host(part: Part, bounds: Sequence[int], H: int, F: int, slope:
                        el: Sequence[torch.Tensor], er: Sequence[torch.Tensor], gout: torch.Tensor,
                        out_last: Optional[torch.Tensor], dfeat0: Optional[torch.Tensor],
                        del_: Optional[Sequence[torch.Tensor]], der: Optional[Sequence[torch.Tensor]],
-                       arena: torch.Tensor) -> None:
-    """L = len(el) chained aggregation layers, fwd + bwd, all node tensors in HOST memory."""
+                       arena: torch.Tensor, pipelined: bool = False) -> None:
+    """L = len(el) chained aggregation layers, fwd + bwd, all node tensors in HOST memory.  pipelined=True:
+    `arena` holds two working sets and successive calls overlap (finish with sar_gat_stack_host_wait)."""
     L = len(el)
     io = sar_stack_host_io(L, H, F, _dtype(feat0), slope, _host_ptr(feat0), _host_ptr_array(el), _host_ptr_array(er),
                            _host_ptr(gout), _host_ptr(out_last), _host_ptr(dfeat0), _host_ptr_array(del_),
-                           _host_ptr_array(der))
+                           _host_ptr_array(der), SAR_STACK_PIPELINED if pipelined else 0)
     w, wb = _ws(arena)
     _check("sar_gat_stack_host", lib().sar_gat_stack_host(byref(part.c), c_int32(len(bounds) - 1), _host_i64(bounds),
                                                           byref(io), w, wb, _stream()))
+
+
+def sar_gat_stack_host_wait() -> None:
+    _check("sar_gat_stack_host_wait", lib().sar_gat_stack_host_wait(_stream()))
 
 
 # ----------------------------------------------------------------------------------------------

@@ -22,6 +22,11 @@ struct Arena {
 // Two non-blocking side streams per device for the copies, created on first use and kept.
 struct Copies {
     cudaStream_t up = nullptr, down = nullptr;
+    // pipelined mode: the two halves of the arena alternate; half_done[i] follows the last result copy of the
+    // latest call that used half i
+    cudaEvent_t half_done[2] = {nullptr, nullptr};
+    bool half_used[2] = {false, false};
+    unsigned long long calls = 0;
 };
 constexpr int kMaxDevices = 64;
 Copies g_copies[kMaxDevices];
@@ -35,6 +40,8 @@ sar_status copies_for_current_device(Copies **out) {
     Copies &c = g_copies[dev];
     if (!c.up) SAR_CUDA_TRY(cudaStreamCreateWithFlags(&c.up, cudaStreamNonBlocking));
     if (!c.down) SAR_CUDA_TRY(cudaStreamCreateWithFlags(&c.down, cudaStreamNonBlocking));
+    for (int i = 0; i < 2; ++i)
+        if (!c.half_done[i]) SAR_CUDA_TRY(cudaEventCreateWithFlags(&c.half_done[i], cudaEventDisableTiming));
     *out = &c;
     return SAR_OK;
 }
@@ -64,12 +71,18 @@ sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bound
     if (!io->feat0 || !io->el || !io->er || !io->gout) return SAR_ERR_INVALID_ARG;
     for (int l = 0; l < L; ++l)
         if (!io->el[l] || !io->er[l] || (io->del && !io->del[l]) || (io->der && !io->der[l])) return SAR_ERR_INVALID_ARG;
-    if (!arena || !sar_aligned(arena, 256) || arena_bytes < stack_bytes(g, L, H, F, io->t)) return SAR_ERR_WORKSPACE;
+    if (io->flags & ~(uint32_t)SAR_STACK_PIPELINED) return SAR_ERR_INVALID_ARG;
+    const bool pipelined = (io->flags & SAR_STACK_PIPELINED) != 0;
+    const size_t one = sar_round_up(stack_bytes(g, L, H, F, io->t), 256);
+    if (!arena || !sar_aligned(arena, 256) || arena_bytes < (pipelined ? 2 * one : one)) return SAR_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const size_t n = (size_t)g->n_dst;
     const size_t row_b = n * H * F * sar_elem_size(io->t), nh_b = n * H * 4;
 
-    Arena a{static_cast<char *>(arena), 0, arena_bytes};
+    Copies *cp = nullptr;
+    SAR_TRY(copies_for_current_device(&cp));
+    const int half = pipelined ? (int)(cp->calls & 1ull) : 0;
+    Arena a{static_cast<char *>(arena) + (size_t)half * one, 0, one};
     std::vector<void *> feat(L + 1);
     std::vector<float *> el(L), er(L), m(L), d(L), del(L), der(L);
     for (int l = 0; l <= L; ++l) feat[l] = a.take(row_b);
@@ -90,8 +103,6 @@ sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bound
     // duplex): `up` brings the inputs in layer order, `down` returns each result as soon as it exists.
     // Everything is ordered after the work already queued on `st`, and `st` finally waits for the last
     // copy, so that completion of `st` still means "all done".
-    Copies *cp = nullptr;
-    SAR_TRY(copies_for_current_device(&cp));
     cudaStream_t up = cp->up, down = cp->down;
     std::vector<cudaEvent_t> ev;
     auto new_event = [&](cudaEvent_t *e) -> sar_status {
@@ -121,9 +132,26 @@ sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bound
         SAR_STEP(new_event(&e_in[l]));
         SAR_STEP(new_event(&e_bwd[l]));
     }
-    SAR_CUDA_STEP(cudaEventRecord(e_start, st));
-    SAR_CUDA_STEP(cudaStreamWaitEvent(up, e_start, 0));
-    SAR_CUDA_STEP(cudaStreamWaitEvent(down, e_start, 0));
+    if (pipelined) {
+        // this half's previous user must be completely done (kernels and result copies) before anything is
+        // written into it; nothing else of the earlier calls is waited for
+        if (cp->half_used[half]) {
+            SAR_CUDA_STEP(cudaStreamWaitEvent(up, cp->half_done[half], 0));
+            SAR_CUDA_STEP(cudaStreamWaitEvent(st, cp->half_done[half], 0));
+        }
+        ++cp->calls;
+    } else {
+        // a plain call after pipelined ones: let those finish first (they may be using this part of the arena)
+        for (int i = 0; i < 2; ++i)
+            if (cp->half_used[i]) {
+                SAR_CUDA_STEP(cudaStreamWaitEvent(st, cp->half_done[i], 0));
+                cp->half_used[i] = false;
+            }
+        cp->calls = 0;
+        SAR_CUDA_STEP(cudaEventRecord(e_start, st));
+        SAR_CUDA_STEP(cudaStreamWaitEvent(up, e_start, 0));
+        SAR_CUDA_STEP(cudaStreamWaitEvent(down, e_start, 0));
+    }
 
     // host -> device, in the order the layers need them
     SAR_CUDA_STEP(cudaMemcpyAsync(feat[0], io->feat0, row_b, cudaMemcpyHostToDevice, up));
@@ -181,12 +209,32 @@ sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bound
     }
     // gin now holds dfeat of layer 0 (the last backward call has been waited for by `down` above)
     if (io->dfeat0) SAR_CUDA_STEP(cudaMemcpyAsync(io->dfeat0, gin, row_b, cudaMemcpyDeviceToHost, down));
-    SAR_CUDA_STEP(cudaEventRecord(e_done, down));
-    SAR_CUDA_STEP(cudaStreamWaitEvent(st, e_done, 0));
+    if (pipelined) {
+        SAR_CUDA_STEP(cudaEventRecord(cp->half_done[half], down));
+        cp->half_used[half] = true;
+    } else {
+        SAR_CUDA_STEP(cudaEventRecord(e_done, down));
+        SAR_CUDA_STEP(cudaStreamWaitEvent(st, e_done, 0));
+    }
     cleanup();
 #undef SAR_STEP
 #undef SAR_CUDA_STEP
     return SAR_OK;
+}
+
+sar_status sar_gat_stack_host_wait(void *stream) {
+    Copies *cp = nullptr;
+    SAR_TRY(copies_for_current_device(&cp));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    cudaEvent_t e = nullptr;
+    SAR_CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    // the copy streams run their work in order, so their current ends cover every call made so far
+    cudaError_t err = cudaEventRecord(e, cp->up);
+    if (err == cudaSuccess) err = cudaStreamWaitEvent(st, e, 0);
+    if (err == cudaSuccess) err = cudaEventRecord(e, cp->down);
+    if (err == cudaSuccess) err = cudaStreamWaitEvent(st, e, 0);
+    cudaEventDestroy(e);
+    return err == cudaSuccess ? SAR_OK : SAR_ERR_CUDA;
 }
 
 }  // extern "C"

@@ -158,6 +158,62 @@ def test_stack_host_entry_point_matches_device_calls():
         assert torch.equal(gr.cpu(), h_dfeat)
 
 
+def test_stack_host_pipelined_calls_equal_plain_calls():
+    """Five pipelined calls with different inputs (two working sets used alternately, copies of one call
+    overlapping the kernels of the previous one) return what five plain calls return, then a plain call
+    after them still works."""
+    from paper_2111_06483_b200 import binding as B
+    cfg = workloads.CONFIGS["seqpart"].scaled(0.5)
+    n, H, F, L, T = cfg.n, cfg.heads, cfg.feat, 2, 5
+    src, dst = workloads.make_graph(cfg, device=DEV)
+    g = api.Graph.from_coo(n, src, dst, k=cfg.k)
+    tdt = torch.bfloat16
+    pin = lambda x: x.pin_memory()
+    ins = []
+    for t in range(T):
+        ins.append(dict(
+            feat0=pin(workloads.normal_tensor((n, H, F), 50 + t, 10, dtype=tdt)),
+            gout=pin(workloads.normal_tensor((n, H, F), 50 + t, 11, dtype=tdt)),
+            el=[pin(workloads.normal_tensor((n, H), 50 + t, 16 * l + 12)) for l in range(L)],
+            er=[pin(workloads.normal_tensor((n, H), 50 + t, 16 * l + 13)) for l in range(L)]))
+
+    def outputs():
+        return dict(out=pin(torch.empty((n, H, F), dtype=tdt)), dfeat=pin(torch.empty((n, H, F), dtype=tdt)),
+                    del_=[pin(torch.empty((n, H))) for _ in range(L)], der=[pin(torch.empty((n, H))) for _ in range(L)])
+
+    one = B.sar_gat_stack_arena_bytes(g.whole, L, H, F, B.SAR_BF16)
+    arena = torch.empty(2 * ((one + 255) // 256 * 256), dtype=torch.uint8, device=DEV)
+
+    def call(i, o, pipelined):
+        B.sar_gat_stack_host(g.whole, g.bounds, H, F, cfg.slope, i["feat0"], i["el"], i["er"], i["gout"], o["out"],
+                             o["dfeat"], o["del_"], o["der"], arena, pipelined=pipelined)
+
+    plain = [outputs() for _ in range(T)]
+    for t in range(T):
+        call(ins[t], plain[t], False)
+    torch.cuda.synchronize()
+    piped = [outputs() for _ in range(T)]
+    for t in range(T):
+        call(ins[t], piped[t], True)
+    B.sar_gat_stack_host_wait()
+    torch.cuda.synchronize()
+    for t in range(T):
+        assert torch.equal(piped[t]["out"], plain[t]["out"]) and torch.equal(piped[t]["dfeat"], plain[t]["dfeat"]), t
+        for l in range(L):
+            assert torch.equal(piped[t]["del_"][l], plain[t]["del_"][l]), (t, l)
+            assert torch.equal(piped[t]["der"][l], plain[t]["der"][l]), (t, l)
+    assert not torch.equal(plain[0]["out"], plain[1]["out"])
+    again = outputs()
+    call(ins[2], again, False)  # switching back to the plain mode
+    torch.cuda.synchronize()
+    assert torch.equal(again["out"], plain[2]["out"]) and torch.equal(again["dfeat"], plain[2]["dfeat"])
+    with pytest.raises(B.SarError) as ei:  # the pipelined mode needs both working sets
+        B.sar_gat_stack_host(g.whole, g.bounds, H, F, cfg.slope, ins[0]["feat0"], ins[0]["el"], ins[0]["er"],
+                             ins[0]["gout"], again["out"], again["dfeat"], again["del_"], again["der"],
+                             arena[:one], pipelined=True)
+    assert ei.value.code == -4
+
+
 def test_more_than_two_to_the_31_edges():
     """Maximum sizes: an edge count that does not fit 32 bits (edge offsets are 64-bit throughout).  No oracle
     can visit 2.3 G edges in test time, so the checks are the ones that hold at any size: the CSR's degrees
