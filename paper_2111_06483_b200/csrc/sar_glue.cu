@@ -50,9 +50,10 @@ __global__ void __launch_bounds__(kThreads) project_kernel(const ProjArgs a) {
     float cl[V][EPV], cr[V][EPV];
     load_coeffs<G, V, EPV>(a.a_l, a.g, a.F, id.gl, cl);
     load_coeffs<G, V, EPV>(a.a_r, a.g, a.F, id.gl, cr);
+    const bool pow2_heads = (a.g.vph & (a.g.vph - 1)) == 0 && a.g.vph <= G;
     const long long stride = (long long)gridDim.x * kWarpsPerBlock * RPW;
     const long long first = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
-    // every lane of the warp runs the same number of sweeps (head_sum synchronises the warp)
+    // every lane of the warp runs the same number of sweeps (the head sums are warp-wide)
     const long long sweeps = (a.n + stride * U - 1) / (stride * U);
     for (long long s = 0; s < sweeps; ++s) {
         float fv[U][V][EPV];
@@ -86,11 +87,24 @@ __global__ void __launch_bounds__(kThreads) project_kernel(const ProjArgs a) {
                     pr[v] = fmaf(fv[u][v][e], cr[v][e], pr[v]);
                 }
             }
-            const float L = head_sum<G, V>(scratch, pl, vg.vok, id.gl, a.g);
-            const float R = head_sum<G, V>(scratch, pr, vg.vok, id.gl, a.g);
-            if (active && id.gl < a.H) {
-                a.el[row[u] * a.H + id.gl] = L;
-                a.er[row[u] * a.H + id.gl] = R;
+            if (V == 1 && pow2_heads) {
+                // a head is vph adjacent lanes: fold them with shuffles, the head's first lane writes
+                float L = pl[0], R = pr[0];
+                for (int o = 1; o < a.g.vph; o <<= 1) {
+                    L += __shfl_xor_sync(0xffffffffu, L, o);
+                    R += __shfl_xor_sync(0xffffffffu, R, o);
+                }
+                if (active && vg.vok[0] && (id.gl & (a.g.vph - 1)) == 0) {
+                    a.el[row[u] * a.H + vg.hv[0]] = L;
+                    a.er[row[u] * a.H + vg.hv[0]] = R;
+                }
+            } else {
+                const float L = head_sum<G, V>(scratch, pl, vg.vok, id.gl, a.g);
+                const float R = head_sum<G, V>(scratch, pr, vg.vok, id.gl, a.g);
+                if (active && id.gl < a.H) {
+                    a.el[row[u] * a.H + id.gl] = L;
+                    a.er[row[u] * a.H + id.gl] = R;
+                }
             }
         }
     }
