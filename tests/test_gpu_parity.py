@@ -107,7 +107,8 @@ def config_problem(name, scale=None, **kw):
 # integer side
 # ------------------------------------------------------------------------------------------------
 
-@pytest.mark.parametrize("n,e,k", [(2000, 20000, 1), (5000, 100000, 8), (257, 3000, 16), (64, 0, 3), (1, 5, 1)])
+@pytest.mark.parametrize("n,e,k", [(2000, 20000, 1), (5000, 100000, 8), (257, 3000, 16), (64, 0, 3), (1, 5, 1),
+                                   (3000, 40000, 64), (40, 500, 64)])  # the last: the maximum partition count, more partitions than nodes
 def test_graph_preparation_is_bit_exact(n, e, k):
     if n == 1:
         src = torch.zeros(e, dtype=torch.int32)
@@ -223,6 +224,16 @@ def test_sequential_partitions_equal_single_pass(threshold):
     o_out, o_m, o_d = oracle.gat_fwd_seq(sp, p.host["feat"], p.host["el"], p.host["er"], 0.2)
     allclose_report(out_s.cpu().numpy(), o_out, 1e-5, 1e-6, "stateful vs sequential oracle")
     allclose_report(d_s.cpu().numpy(), o_d, 1e-5, 1e-6, "d vs sequential oracle")
+
+
+def test_maximum_partition_count_with_empty_partitions():
+    """K = 64 (the most the library accepts) on a graph with fewer edges per partition than rows: most
+    (row, partition) pairs are empty, the running state must pass through them untouched; forward and
+    backward, stateful and fused, against the oracle."""
+    n, src, dst = hub_graph(n=900, e=5000, d_max=200.0, seed=12)
+    p = Problem(n, src, dst, 2, 16, 33, k=64, threshold=16, build_parts=True)
+    assert p.k == 64 and len(p.graph.parts) == 64
+    _full_check(p, modes=("fused", "stateful"))
 
 
 @pytest.mark.parametrize("H,F,dtype", [(4, 64, "f32"), (4, 64, "bf16"), (8, 32, "bf16"), (4, 32, "bf16"), (1, 8, "f32"),
