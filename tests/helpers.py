@@ -64,7 +64,8 @@ def allclose_report(got, want, rtol, atol, what=""):
     want = np.asarray(want, dtype=np.float64)
     assert got.shape == want.shape, (what, got.shape, want.shape)
     both_inf = np.isinf(got) & np.isinf(want) & (np.sign(got) == np.sign(want))
-    err = np.where(both_inf, 0.0, np.abs(got - want))
+    with np.errstate(invalid="ignore"):  # inf - inf where both are the same infinity
+        err = np.where(both_inf, 0.0, np.abs(got - want))
     tol = atol + rtol * np.where(both_inf, 0.0, np.abs(want))
     bad = ~(err <= tol)
     if bad.any():
