@@ -312,6 +312,40 @@ SAR_API sar_status sar_relu(int64_t n_elems, sar_dtype t, void *x, void *stream)
 SAR_API sar_status sar_relu_bwd(int64_t n_elems, sar_dtype t, const void *y, void *g, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Batch normalisation over the node dimension (Sec. 3.4, "Batch normalization"): y[i,c] =
+ * (x[i,c] - mean[c]) * rstd[c] * gamma[c] + beta[c] with mean and variance taken over ALL rows of
+ * x [n, C] (type t).  A worker that holds only some of the rows computes LOCAL statistics, combines them
+ * with the other workers' (a few floats per column: that is all that is communicated), and applies the
+ * global ones; the entry points are split accordingly.  All arrays are DEVICE memory; [C] arrays are
+ * float32; gamma / beta may be NULL (1 / 0); y may be x, gx may be gy.  Scratch for the two *_stats
+ * calls: sar_bn_workspace_bytes(C).  Sums are formed in a fixed order (no atomics), block partials are
+ * added in float64.
+ *   sar_bn_stats      mean[c] = (1/n) sum_i x[i,c] and m2[c] = sum_i (x[i,c] - mean[c])^2 of the n local rows
+ *                     (two passes, no cancellation).  Workers combine (n, mean, m2) triples by the pairwise
+ *                     rule mean = sum n_r mean_r / N, m2 = sum [m2_r + n_r (mean_r - mean)^2]; the variance
+ *                     is m2 / N and rstd = 1 / sqrt(variance + eps).
+ *   sar_bn_apply      the normalisation with given (global) mean and rstd.
+ *   sar_bn_bwd_stats  sum_gy[c] = sum_i gy[i,c] (= d beta) and sum_gy_xhat[c] = sum_i gy[i,c] * xhat[i,c]
+ *                     (= d gamma) over the local rows, xhat = (x - mean) * rstd; workers add these up.
+ *   sar_bn_bwd_apply  gx = gamma * rstd * (gy - sum_gy * inv_count - xhat * sum_gy_xhat * inv_count) with
+ *                     the GLOBAL sums and inv_count = 1 / N, N the global row count: the gradients through
+ *                     the mean and the variance, scaled by the number of rows everywhere, as the paper
+ *                     requires of the distributed backward pass.
+ * n = 0 is allowed (statistics and sums are written as zeros).  Errors as for the other streaming calls.
+ * ------------------------------------------------------------------------------------------- */
+SAR_API size_t sar_bn_workspace_bytes(int32_t C);
+SAR_API sar_status sar_bn_stats(int64_t n, int32_t C, sar_dtype t, const void *x, float *mean, float *m2,
+                                void *workspace, size_t workspace_bytes, void *stream);
+SAR_API sar_status sar_bn_apply(int64_t n, int32_t C, sar_dtype t, const void *x, const float *mean,
+                                const float *rstd, const float *gamma, const float *beta, void *y, void *stream);
+SAR_API sar_status sar_bn_bwd_stats(int64_t n, int32_t C, sar_dtype t, const void *x, const float *mean,
+                                    const float *rstd, const void *gy, float *sum_gy, float *sum_gy_xhat,
+                                    void *workspace, size_t workspace_bytes, void *stream);
+SAR_API sar_status sar_bn_bwd_apply(int64_t n, int32_t C, sar_dtype t, const void *x, const float *mean,
+                                    const float *rstd, const float *gamma, const void *gy, const float *sum_gy,
+                                    const float *sum_gy_xhat, float inv_count, void *gx, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Backward pass without any caller-provided scratch.  (The paper has no counterpart: this is a
  * convenience of this library.)
  *

@@ -326,3 +326,39 @@ def spmm_scaled(indptr, indices, feat, src_scale=None, dst_scale=None):
     if dst_scale is not None:
         out *= np.asarray(dst_scale, np.float64)[:, None]
     return out
+
+
+# --------------------------------------------------------------------------------------
+# batch normalisation over the node dimension (Sec. 3.4), plain numpy float64
+# --------------------------------------------------------------------------------------
+
+def bn_moments(x):
+    """(mean[c], m2[c] = sum_i (x[i,c] - mean[c])^2) over the rows of x."""
+    x = np.asarray(x, dtype=np.float64)
+    mean = x.mean(axis=0) if x.shape[0] else np.zeros(x.shape[1])
+    return mean, ((x - mean) ** 2).sum(axis=0)
+
+
+def bn_forward(x, eps=1e-5, gamma=None, beta=None):
+    x = np.asarray(x, dtype=np.float64)
+    mean, m2 = bn_moments(x)
+    rstd = 1.0 / np.sqrt(m2 / max(x.shape[0], 1) + eps)
+    y = (x - mean) * rstd
+    if gamma is not None:
+        y = y * np.asarray(gamma, np.float64)
+    if beta is not None:
+        y = y + np.asarray(beta, np.float64)
+    return y, mean, rstd
+
+
+def bn_backward(x, gy, eps=1e-5, gamma=None):
+    """(gx, dgamma, dbeta) of y = xhat * gamma + beta for the upstream gradient gy."""
+    x, gy = np.asarray(x, np.float64), np.asarray(gy, np.float64)
+    n = x.shape[0]
+    _, mean, rstd = bn_forward(x, eps)
+    xhat = (x - mean) * rstd
+    dbeta = gy.sum(axis=0)
+    dgamma = (gy * xhat).sum(axis=0)
+    g = 1.0 if gamma is None else np.asarray(gamma, np.float64)
+    gx = g * rstd * (gy - dbeta / n - xhat * dgamma / n)
+    return gx, dgamma, dbeta

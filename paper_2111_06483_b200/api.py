@@ -249,3 +249,68 @@ def spmm_scaled(part: B.Part, feat: torch.Tensor, src_scale: Optional[torch.Tens
     ws = _workspace(B.sar_spmm_workspace_bytes(part, F, B._dtype(feat)), feat.device)
     B.sar_spmm_agg_scaled(part, feat, F, (B.SAR_FIRST if first else 0) | B.SAR_LAST, src_scale, dst_scale, out, ws)
     return out
+
+
+# ----------------------------------------------------------------------------------------------
+# batch normalisation over the node dimension (Sec. 3.4); with `group` the statistics are combined across
+# the workers of a torch.distributed process group (each holds some of the rows): a few floats per column.
+
+def combine_moments(n_local: int, mean: torch.Tensor, m2: torch.Tensor, group=None):
+    """(n, mean, m2 = sum of squared deviations) of the local rows -> the same for all rows of all workers.
+    Pairwise rule: mean = sum n_r mean_r / N;  m2 = sum [m2_r + n_r (mean_r - mean)^2].  float64 on the way."""
+    if group is None:
+        return n_local, mean, m2
+    import torch.distributed as dist
+    acc = torch.cat([torch.tensor([float(n_local)], dtype=torch.float64, device=mean.device),
+                     mean.double() * n_local])
+    dist.all_reduce(acc, group=group)
+    n_all = int(round(float(acc[0])))
+    mean_all = acc[1:] / max(n_all, 1)
+    m2_part = m2.double() + n_local * (mean.double() - mean_all) ** 2
+    dist.all_reduce(m2_part, group=group)
+    return n_all, mean_all.float(), m2_part.float()
+
+
+def combine_sums(tensors, group=None):
+    """Element-wise sums over the workers (the backward statistics)."""
+    if group is None:
+        return tensors
+    import torch.distributed as dist
+    flat = torch.cat([t.double().flatten() for t in tensors])
+    dist.all_reduce(flat, group=group)
+    out, o = [], 0
+    for t in tensors:
+        out.append(flat[o:o + t.numel()].reshape(t.shape).to(t.dtype))
+        o += t.numel()
+    return out
+
+
+def bn_forward(x: torch.Tensor, eps: float = 1e-5, gamma: Optional[torch.Tensor] = None,
+               beta: Optional[torch.Tensor] = None, group=None):
+    """Returns (y, saved) with saved = (mean, rstd, n_all) for bn_backward.  x is [n_local, C]."""
+    n, C = x.shape
+    dev = x.device
+    ws = _workspace(B.sar_bn_workspace_bytes(C), dev)
+    mean = torch.empty(C, dtype=torch.float32, device=dev)
+    m2 = torch.empty(C, dtype=torch.float32, device=dev)
+    B.sar_bn_stats(x, mean, m2, ws)
+    n_all, mean, m2 = combine_moments(n, mean, m2, group)
+    rstd = torch.rsqrt(m2 / max(n_all, 1) + eps)
+    y = torch.empty_like(x)
+    B.sar_bn_apply(x, mean, rstd, gamma, beta, y)
+    return y, (mean, rstd, n_all)
+
+
+def bn_backward(x: torch.Tensor, gy: torch.Tensor, saved, gamma: Optional[torch.Tensor] = None, group=None):
+    """Returns (gx, dgamma, dbeta); dgamma and dbeta are already summed over the workers."""
+    n, C = x.shape
+    dev = x.device
+    mean, rstd, n_all = saved
+    ws = _workspace(B.sar_bn_workspace_bytes(C), dev)
+    s0 = torch.empty(C, dtype=torch.float32, device=dev)
+    s1 = torch.empty(C, dtype=torch.float32, device=dev)
+    B.sar_bn_bwd_stats(x, mean, rstd, gy, s0, s1, ws)
+    s0, s1 = combine_sums([s0, s1], group)
+    gx = torch.empty_like(x)
+    B.sar_bn_bwd_apply(x, mean, rstd, gamma, gy, s0, s1, 1.0 / max(n_all, 1), gx)
+    return gx, s1, s0

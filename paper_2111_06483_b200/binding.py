@@ -30,7 +30,8 @@ EXPORTS = [
     "sar_gat_stack_arena_bytes", "sar_gat_stack_host", "sar_gat_bwd_noalloc", "sar_gat_bwd_noalloc_limit",
     "sar_gat_project_workspace_bytes", "sar_gat_project", "sar_gat_project_bwd", "sar_relu", "sar_relu_bwd",
     "sar_mfg_frontier", "sar_csr_filter_rows_indptr", "sar_csr_filter_rows_indices", "sar_spmm_agg_scaled",
-    "sar_gat_stack_host_wait",
+    "sar_gat_stack_host_wait", "sar_bn_workspace_bytes", "sar_bn_stats", "sar_bn_apply", "sar_bn_bwd_stats",
+    "sar_bn_bwd_apply",
 ]
 
 
@@ -67,7 +68,8 @@ def lib() -> ctypes.CDLL:
         L.sar_status_string.argtypes = [ctypes.c_int]
         L.sar_built_for_sm.restype = c_int32
         for name in ("sar_graph_workspace_bytes", "sar_gat_workspace_bytes", "sar_spmm_workspace_bytes",
-                     "sar_gat_stack_arena_bytes", "sar_gat_bwd_noalloc_limit", "sar_gat_project_workspace_bytes"):
+                     "sar_gat_stack_arena_bytes", "sar_gat_bwd_noalloc_limit", "sar_gat_project_workspace_bytes",
+                     "sar_bn_workspace_bytes"):
             getattr(L, name).restype = c_size_t
         _lib = L
     return _lib
@@ -416,6 +418,42 @@ def sar_gat_stack_host(part: Part, bounds: Sequence[int], H: int, F: int, slope:
     w, wb = _ws(arena)
     _check("sar_gat_stack_host", lib().sar_gat_stack_host(byref(part.c), c_int32(len(bounds) - 1), _host_i64(bounds),
                                                           byref(io), w, wb, _stream()))
+
+
+def sar_bn_workspace_bytes(C: int) -> int:
+    return int(lib().sar_bn_workspace_bytes(c_int32(C)))
+
+
+def sar_bn_stats(x: torch.Tensor, mean: torch.Tensor, m2: torch.Tensor, workspace: torch.Tensor) -> None:
+    n, C = x.shape
+    w, wb = _ws(workspace)
+    _check("sar_bn_stats", lib().sar_bn_stats(c_int64(n), c_int32(C), ctypes.c_int(_dtype(x)), _ptr(x), _ptr(mean),
+                                              _ptr(m2), w, wb, _stream()))
+
+
+def sar_bn_apply(x: torch.Tensor, mean: torch.Tensor, rstd: torch.Tensor, gamma: Optional[torch.Tensor],
+                 beta: Optional[torch.Tensor], y: torch.Tensor) -> None:
+    n, C = x.shape
+    _check("sar_bn_apply", lib().sar_bn_apply(c_int64(n), c_int32(C), ctypes.c_int(_dtype(x)), _ptr(x), _ptr(mean),
+                                              _ptr(rstd), _ptr(gamma), _ptr(beta), _ptr(y), _stream()))
+
+
+def sar_bn_bwd_stats(x: torch.Tensor, mean: torch.Tensor, rstd: torch.Tensor, gy: torch.Tensor, sum_gy: torch.Tensor,
+                     sum_gy_xhat: torch.Tensor, workspace: torch.Tensor) -> None:
+    n, C = x.shape
+    w, wb = _ws(workspace)
+    _check("sar_bn_bwd_stats", lib().sar_bn_bwd_stats(c_int64(n), c_int32(C), ctypes.c_int(_dtype(x)), _ptr(x),
+                                                      _ptr(mean), _ptr(rstd), _ptr(gy), _ptr(sum_gy),
+                                                      _ptr(sum_gy_xhat), w, wb, _stream()))
+
+
+def sar_bn_bwd_apply(x: torch.Tensor, mean: torch.Tensor, rstd: torch.Tensor, gamma: Optional[torch.Tensor],
+                     gy: torch.Tensor, sum_gy: torch.Tensor, sum_gy_xhat: torch.Tensor, inv_count: float,
+                     gx: torch.Tensor) -> None:
+    n, C = x.shape
+    _check("sar_bn_bwd_apply", lib().sar_bn_bwd_apply(c_int64(n), c_int32(C), ctypes.c_int(_dtype(x)), _ptr(x),
+                                                      _ptr(mean), _ptr(rstd), _ptr(gamma), _ptr(gy), _ptr(sum_gy),
+                                                      _ptr(sum_gy_xhat), c_float(inv_count), _ptr(gx), _stream()))
 
 
 def sar_gat_stack_host_wait() -> None:
