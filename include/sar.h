@@ -227,9 +227,11 @@ SAR_API sar_status sar_gat_fwd_fused(const sar_part *g, int32_t k, const int64_t
 
 /* Row dot D[i,h] = <gout[i,h,:], out[i,h,:]> and the packed per-destination record
  * {el, m, 1/d, D} (16 bytes per (i,h), written to the start of `workspace`) that lets each
- * partition's backward step run independently of the others.  `out` may be given as the float32
- * numerator `acc` with acc_is_numerator != 0 (then out = acc/d is formed on the fly), which avoids
- * the rounding of a bf16 `out`.  D may be NULL. */
+ * partition's backward step run independently of the others.  `out` may be given as the COMPLETE float32
+ * numerator with acc_is_numerator != 0 (then out = acc/d is formed on the fly), which avoids the
+ * rounding of a bf16 `out`; note that the forward call with SAR_LAST does not update `acc`, so the
+ * complete numerator exists only for a caller that runs all partitions without SAR_LAST and
+ * normalises itself.  D may be NULL. */
 SAR_API sar_status sar_gat_bwd_prepare(int64_t n_dst, int32_t H, int32_t F, sar_dtype t, const void *out_or_acc,
                                int32_t acc_is_numerator, const void *gout, const float *el, const float *m,
                                const float *d, float *D, void *workspace, size_t workspace_bytes,
