@@ -311,6 +311,13 @@ SAR_API sar_status sar_gat_project_bwd(int64_t n, int32_t H, int32_t F, sar_dtyp
                                        float *da_r, uint32_t flags, void *workspace, size_t workspace_bytes,
                                        void *stream);
 SAR_API sar_status sar_relu(int64_t n_elems, sar_dtype t, void *x, void *stream);
+/* Dropout between layers (Sec. 4.2: "batch normalization and dropout between all layers"), counter-based so
+ * that nothing is kept for the backward pass: element i is KEPT (and multiplied by 1/(1-p)) when the top
+ * 24 bits of the (i+1)-th output of SplitMix64 started at `seed` (z = seed + (i+1)*0x9E3779B97F4A7C15, then
+ * the generator's two multiply-xorshift rounds) are >= floor(p * 2^24); otherwise y[i] = 0.  0 <= p < 1.
+ * y may be x.  The backward pass is the same call on the upstream gradient with the same seed and p. */
+SAR_API sar_status sar_dropout(int64_t n_elems, sar_dtype t, const void *x, float p, uint64_t seed, void *y,
+                               void *stream);
 SAR_API sar_status sar_relu_bwd(int64_t n_elems, sar_dtype t, const void *y, void *g, void *stream);
 
 /* ---------------------------------------------------------------------------------------------

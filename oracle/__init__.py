@@ -362,3 +362,25 @@ def bn_backward(x, gy, eps=1e-5, gamma=None):
     g = 1.0 if gamma is None else np.asarray(gamma, np.float64)
     gx = g * rstd * (gy - dbeta / n - xhat * dgamma / n)
     return gx, dgamma, dbeta
+
+
+# --------------------------------------------------------------------------------------
+# dropout with a counter-based mask (SplitMix64), numpy
+# --------------------------------------------------------------------------------------
+
+def splitmix64(seed: int, count: int) -> np.ndarray:
+    """The first `count` outputs of the SplitMix64 generator started at `seed` (uint64)."""
+    with np.errstate(over="ignore"):
+        k = np.arange(1, count + 1, dtype=np.uint64)
+        z = np.uint64(seed & 0xFFFFFFFFFFFFFFFF) + k * np.uint64(0x9E3779B97F4A7C15)
+        z = (z ^ (z >> np.uint64(30))) * np.uint64(0xBF58476D1CE4E5B9)
+        z = (z ^ (z >> np.uint64(27))) * np.uint64(0x94D049BB133111EB)
+        return z ^ (z >> np.uint64(31))
+
+
+def dropout(x, p: float, seed: int):
+    """y = x / (1 - p) where the element's 24-bit draw reaches floor(p * 2^24), else 0 (flattened order)."""
+    x = np.asarray(x, dtype=np.float64)
+    draws = (splitmix64(seed, x.size) >> np.uint64(40)).astype(np.int64).reshape(x.shape)
+    keep = draws >= int(float(np.float32(p)) * 16777216.0)
+    return np.where(keep, x * float(np.float32(1.0) / (np.float32(1.0) - np.float32(p))), 0.0), keep

@@ -31,7 +31,7 @@ EXPORTS = [
     "sar_gat_project_workspace_bytes", "sar_gat_project", "sar_gat_project_bwd", "sar_relu", "sar_relu_bwd",
     "sar_mfg_frontier", "sar_csr_filter_rows_indptr", "sar_csr_filter_rows_indices", "sar_spmm_agg_scaled",
     "sar_gat_stack_host_wait", "sar_bn_workspace_bytes", "sar_bn_stats", "sar_bn_apply", "sar_bn_bwd_stats",
-    "sar_bn_bwd_apply",
+    "sar_bn_bwd_apply", "sar_dropout",
 ]
 
 
@@ -512,6 +512,11 @@ def sar_gat_project_bwd(z: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, d
 
 def sar_relu(x: torch.Tensor) -> None:
     _check("sar_relu", lib().sar_relu(c_int64(x.numel()), ctypes.c_int(_dtype(x)), _ptr(x), _stream()))
+
+
+def sar_dropout(x: torch.Tensor, p: float, seed: int, y: torch.Tensor) -> None:
+    _check("sar_dropout", lib().sar_dropout(c_int64(x.numel()), ctypes.c_int(_dtype(x)), _ptr(x), c_float(p),
+                                            ctypes.c_uint64(seed & 0xFFFFFFFFFFFFFFFF), _ptr(y), _stream()))
 
 
 def sar_relu_bwd(y: torch.Tensor, g: torch.Tensor) -> None:

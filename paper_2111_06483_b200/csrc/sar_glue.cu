@@ -266,6 +266,39 @@ static sar_status launch_relu(const char *name, int64_t n, const void *y, void *
     return sar_after_launch();
 }
 
+
+// ---- dropout (the paper's networks use batch normalisation and dropout between all layers, Sec. 4.2) ------
+// Counter-based: element i is kept when the top 24 bits of SplitMix64's (i+1)-th output for `seed` reach
+// p * 2^24; nothing is stored, the backward pass draws the same mask again from the seed.
+__device__ __forceinline__ unsigned long long splitmix64_at(unsigned long long seed, unsigned long long i) {
+    unsigned long long z = seed + (i + 1ull) * 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+template <typename T>
+__global__ void dropout_kernel(long long n, const T *x, T *y, unsigned threshold, float scale, unsigned long long seed,
+                               long long n_vec16) {
+    constexpr int EPV = Elem<T>::EPV;
+    const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long nthreads = (long long)gridDim.x * blockDim.x;
+    for (long long v = tid; v < n_vec16; v += nthreads) {
+        float f[EPV];
+        Elem<T>::unpack(reinterpret_cast<const uint4 *>(x)[v], f);  // plain load: y may be x
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) {
+            const unsigned r = (unsigned)(splitmix64_at(seed, (unsigned long long)(v * EPV + e)) >> 40);
+            f[e] = r >= threshold ? f[e] * scale : 0.f;
+        }
+        reinterpret_cast<uint4 *>(y)[v] = Elem<T>::pack(f);
+    }
+    for (long long i = n_vec16 * EPV + tid; i < n; i += nthreads) {
+        const unsigned r = (unsigned)(splitmix64_at(seed, (unsigned long long)i) >> 40);
+        Elem<T>::store1(y + i, r >= threshold ? as_float(x[i]) * scale : 0.f);
+    }
+}
+
 static sar_status glue_shape(int64_t n, int32_t H, int32_t F, sar_dtype t, std::initializer_list<const void *> ps,
                              Shape *s) {
     if (n < 0 || H < 1 || F < 1) return SAR_ERR_INVALID_ARG;
@@ -391,6 +424,28 @@ sar_status sar_relu_bwd(int64_t n_elems, sar_dtype t, const void *y, void *g, vo
     if (n_elems == 0) return SAR_OK;
     if (t == SAR_F32) return launch_relu<float, true>("relu_bwd", n_elems, y, g, st);
     return launch_relu<__nv_bfloat16, true>("relu_bwd", n_elems, y, g, st);
+}
+
+sar_status sar_dropout(int64_t n_elems, sar_dtype t, const void *x, float p, uint64_t seed, void *y, void *stream) {
+    if (n_elems < 0 || (n_elems > 0 && (!x || !y))) return SAR_ERR_INVALID_ARG;
+    if (t != SAR_F32 && t != SAR_BF16) return SAR_ERR_INVALID_ARG;
+    if (!(p >= 0.f && p < 1.f)) return SAR_ERR_INVALID_ARG;
+    SAR_TRY(check_elem_align({x, y}, sar_elem_size(t)));
+    if (n_elems == 0) return SAR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const unsigned threshold = (unsigned)((double)p * 16777216.0);  // floor(p * 2^24)
+    const float scale = 1.f / (1.f - p);
+    const bool vec = sar_aligned(x, 16) && sar_aligned(y, 16);
+    const long long epv = t == SAR_F32 ? 4 : 8;
+    const long long n_vec16 = vec ? n_elems / epv : 0;
+    const long long work = n_vec16 > 0 ? n_vec16 : n_elems;
+    long long blocks = (work + 255) / 256;
+    if (blocks > 148 * 64) blocks = 148 * 64;
+    if (t == SAR_F32)
+        SAR_LAUNCH("dropout", st, (dropout_kernel<float><<<(unsigned)blocks, 256, 0, st>>>(n_elems, static_cast<const float *>(x), static_cast<float *>(y), threshold, scale, seed, n_vec16)));
+    else
+        SAR_LAUNCH("dropout", st, (dropout_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, st>>>(n_elems, static_cast<const __nv_bfloat16 *>(x), static_cast<__nv_bfloat16 *>(y), threshold, scale, seed, n_vec16)));
+    return sar_after_launch();
 }
 
 }  // extern "C"

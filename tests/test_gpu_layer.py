@@ -128,3 +128,29 @@ def test_three_layer_stack_matches_oracle_f32(k):
     for l in range(L):
         assert rel(_np(got_al[l]), want["da_l"][l]) < 1e-3, l
         assert rel(_np(got_ar[l]), want["da_r"][l]) < 1e-3, l
+
+
+@pytest.mark.parametrize("dt", ["f32", "bf16"])
+@pytest.mark.parametrize("n", [0, 1, 7, 4099, (1 << 20) + 5])
+@pytest.mark.parametrize("p", [0.0, 0.25, 0.5])
+def test_dropout_mask_is_the_oracles_mask(dt, n, p):
+    from paper_2111_06483_b200 import binding as B
+    x = _dev(normal_tensor((n,), 8).astype(np.float32), DT[dt])
+    y = torch.full_like(x, float("nan"))
+    B.sar_dropout(x, p, 0xDEADBEEFCAFE, y)
+    want, keep = oracle.dropout(_np(x), p, 0xDEADBEEFCAFE)
+    got = _np(y)
+    assert np.array_equal(got != 0, keep & (_np(x) != 0))          # the same elements survive
+    if dt == "bf16":
+        allclose_report(got, want, 2 ** -8, 0.0, "dropout")           # one rounding to bf16
+    else:
+        allclose_report(got, want, 2e-7, 0.0, "dropout")
+    # the backward pass draws the same mask again; in place
+    g = x.clone()
+    B.sar_dropout(g, p, 0xDEADBEEFCAFE, g)
+    assert torch.equal(g, y)
+    if n > 4 and p > 0:   # an unaligned view takes the scalar path and must agree with the vector path
+        xo = x[1:]
+        yo = torch.empty_like(xo)
+        B.sar_dropout(xo, p, 3, yo)
+        assert np.array_equal(_np(yo) != 0, oracle.dropout(_np(xo), p, 3)[1] & (_np(xo) != 0))

@@ -73,3 +73,23 @@ def test_two_workers_combine_to_the_statistics_of_all_rows():
         assert np.allclose(m2_r.numpy(), m2, rtol=1e-5)
         # each worker's gradient rows are the rows of the gradient computed over all rows at once
         assert np.allclose(gx.numpy(), gx_all[rows], rtol=1e-4, atol=1e-5)
+
+
+def test_splitmix64_known_answers_and_dropout_statistics():
+    # the generator's published first outputs for seed 0
+    assert [hex(int(v)) for v in oracle.splitmix64(0, 4)] == ["0xe220a8397b1dcdaf", "0x6e789e6aa1b965f4",
+                                                              "0x6c45d188009454f", "0xf88bb8a8724c81ec"]
+    x = np.ones((1000, 200))
+    for p in (0.0, 0.1, 0.5, 0.9):
+        y, keep = oracle.dropout(x, p, 12345)
+        n = x.size
+        assert abs(keep.mean() - (1 - p)) <= 4 * np.sqrt(p * (1 - p) / n) + 1e-7   # binomial, 4 sigma
+        assert np.allclose(y[keep], 1 / (1 - p), rtol=1e-6) and np.all(y[~keep] == 0)
+        assert abs(y.mean() - 1.0) <= 4 * np.sqrt(p / (1 - p) / n) + 1e-6            # expectation preserved
+    a, _ = oracle.dropout(x, 0.5, 1)
+    b, _ = oracle.dropout(x, 0.5, 2)
+    c, _ = oracle.dropout(x, 0.5, 1)
+    assert np.array_equal(a, c) and not np.array_equal(a, b)
+    # neighbouring elements are not correlated: the lag-1 agreement rate of the mask is 1/2 at p = 1/2
+    k = oracle.dropout(np.ones(200000), 0.5, 7)[1]
+    assert abs((k[1:] == k[:-1]).mean() - 0.5) < 0.01
