@@ -44,8 +44,8 @@ def parse_args():
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (debugging only)")
     ap.add_argument("--threshold", type=int, default=None, help="long-row split threshold")
     ap.add_argument("--glue", action="store_true",
-                    help="also run the layer glue each step: score projections before every aggregation, "
-                         "ReLU after it, and their backward passes (default: aggregation kernels only)")
+                    help="also run the rest of the layer each step: dense projection z = h W (bf16 workloads), score "
+                         "projections, ReLU, and their backward passes (default: aggregation kernels only)")
     ap.add_argument("--ids", default="permuted", choices=["permuted", "degree_sorted"],
                     help="node numbering of the power-law graph: seeded random permutation (the workload) or "
                          "degree rank = id (locality ablation)")
@@ -297,24 +297,56 @@ def run_ours(args, rank, world, local_rank):
         da_l, da_r = torch.empty((H, F), device=dev), torch.empty((H, F), device=dev)
         pws = torch.empty(B.sar_gat_project_workspace_bytes(H, F), dtype=torch.uint8, device=dev)
 
-    def step():
-        for l in range(L):
-            if glue:  # the ReLU closing layer l-1 runs inside layer l's projection
-                B.sar_gat_project(feats[l], a_ls[l], a_rs[l], els[l], ers[l], B.SAR_GLUE_RELU if l > 0 else 0)
-            B.sar_gat_fwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], H, F, cfg.slope, ms[l], ds[l],
-                                feats[l + 1], ws)
-        if glue:
+    if glue and tdt == torch.bfloat16 and (H * F) % 8 == 0:
+        # the whole layer: dense projection z = h W on the tensor cores, scores, aggregation, ReLU
+        D = H * F
+        Ws = [(workloads.normal_tensor((D, D), cfg.seed, 16 * l + 9, device=dev) / D ** 0.5).to(tdt) for l in range(L)]
+        zs = [torch.empty((n, H, F), dtype=tdt, device=dev) for _ in range(L)]
+        z_q = [cut(z) for z in zs]
+        dW = torch.empty((D, D), dtype=torch.float32, device=dev)
+        lws = torch.empty(B.sar_linear_workspace_bytes(n, D, D), dtype=torch.uint8, device=dev)
+        flat = lambda x: x.view(n, D)
+
+        def step():
+            for l in range(L):
+                if l > 0:
+                    B.sar_relu(feats[l])
+                B.sar_linear(flat(feats[l]), Ws[l], flat(zs[l]), lws)
+                B.sar_gat_project(zs[l], a_ls[l], a_rs[l], els[l], ers[l], 0)
+                B.sar_gat_fwd_fused(g.whole, g.bounds, z_q[l], els[l], er_q[l], H, F, cfg.slope, ms[l], ds[l],
+                                    feats[l + 1], ws)
             B.sar_relu(feats[L])
-        gin = gout
-        if glue:
+            gin = gout
             B.sar_relu_bwd(feats[L], gin)  # masks gout in place on the first pass; the same mask every step
-        for i, l in enumerate(reversed(range(L))):
-            B.sar_gat_bwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], ms[l], ds[l], gin, H, F, cfg.slope,
-                                gbuf_q[i % 2], dels[l], der_q[l], ws)
-            gin = gbuf[i % 2]
+            for l in reversed(range(L)):
+                # gbuf[0]: gradient w.r.t. z of this layer, gbuf[1]: w.r.t. the layer's input
+                B.sar_gat_bwd_fused(g.whole, g.bounds, z_q[l], els[l], er_q[l], ms[l], ds[l], gin, H, F, cfg.slope,
+                                    gbuf_q[0], dels[l], der_q[l], ws)
+                B.sar_gat_project_bwd(zs[l], a_ls[l], a_rs[l], dels[l], ders[l], gbuf[0], da_l, da_r, pws, 0)
+                B.sar_linear_bwd_weight(flat(feats[l]), flat(gbuf[0]), dW, lws)
+                B.sar_linear_bwd_input(flat(gbuf[0]), Ws[l], flat(gbuf[1]), lws)
+                if l > 0:
+                    B.sar_relu_bwd(feats[l], gbuf[1])
+                gin = gbuf[1]
+    else:
+        def step():
+            for l in range(L):
+                if glue:  # the ReLU closing layer l-1 runs inside layer l's projection
+                    B.sar_gat_project(feats[l], a_ls[l], a_rs[l], els[l], ers[l], B.SAR_GLUE_RELU if l > 0 else 0)
+                B.sar_gat_fwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], H, F, cfg.slope, ms[l], ds[l],
+                                    feats[l + 1], ws)
             if glue:
-                B.sar_gat_project_bwd(feats[l], a_ls[l], a_rs[l], dels[l], ders[l], gin, da_l, da_r, pws,
-                                      B.SAR_GLUE_RELU if l > 0 else 0)
+                B.sar_relu(feats[L])
+            gin = gout
+            if glue:
+                B.sar_relu_bwd(feats[L], gin)  # masks gout in place on the first pass; the same mask every step
+            for i, l in enumerate(reversed(range(L))):
+                B.sar_gat_bwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], ms[l], ds[l], gin, H, F, cfg.slope,
+                                    gbuf_q[i % 2], dels[l], der_q[l], ws)
+                gin = gbuf[i % 2]
+                if glue:
+                    B.sar_gat_project_bwd(feats[l], a_ls[l], a_rs[l], dels[l], ders[l], gin, da_l, da_r, pws,
+                                          B.SAR_GLUE_RELU if l > 0 else 0)
 
     torch.cuda.reset_peak_memory_stats()
     for _ in range(args.warmup):

@@ -321,6 +321,29 @@ SAR_API sar_status sar_dropout(int64_t n_elems, sar_dtype t, const void *x, floa
 SAR_API sar_status sar_relu_bwd(int64_t n_elems, sar_dtype t, const void *y, void *g, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * The dense projection of a layer, z = h W (Eq. 1 / Eq. 3 apply a weight matrix to every node's features
+ * before the aggregation), and its backward pass: the one dense contraction around the aggregation.  It
+ * runs on the tensor cores (tcgen05 MMA, accumulators in tensor memory, operands staged by TMA; CUTLASS
+ * sm100 collectives instantiated in the library), bf16 operands with float32 accumulation.
+ *   sar_linear             z[n, d_out]  = h[n, d_in] W[d_in, d_out]          (bf16 out)
+ *   sar_linear_bwd_input   dh[n, d_in]  = dz[n, d_out] W^T                   (bf16 out)
+ *   sar_linear_bwd_weight  dw[d_in, d_out] = h^T dz                          (float32 out; the n-long
+ *                          contraction is cut across the SMs and the partial tiles are reduced in the scratch)
+ * All arrays row-major DEVICE memory, 16-byte aligned; t must be SAR_BF16 and d_in, d_out multiples of 8
+ * (SAR_ERR_UNSUPPORTED otherwise); n <= 2^31-1.  Scratch: sar_linear_workspace_bytes(n, d_in, d_out) covers
+ * the three calls.  n = 0 is allowed (dw is then written as zeros).
+ * ------------------------------------------------------------------------------------------- */
+SAR_API size_t sar_linear_workspace_bytes(int64_t n, int32_t d_in, int32_t d_out);
+SAR_API sar_status sar_linear(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *h, const void *w,
+                              void *z, void *workspace, size_t workspace_bytes, void *stream);
+SAR_API sar_status sar_linear_bwd_input(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *dz,
+                                        const void *w, void *dh, void *workspace, size_t workspace_bytes,
+                                        void *stream);
+SAR_API sar_status sar_linear_bwd_weight(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *h,
+                                         const void *dz, float *dw, void *workspace, size_t workspace_bytes,
+                                         void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Batch normalisation over the node dimension (Sec. 3.4, "Batch normalization"): y[i,c] =
  * (x[i,c] - mean[c]) * rstd[c] * gamma[c] + beta[c] with mean and variance taken over ALL rows of
  * x [n, C] (type t).  A worker that holds only some of the rows computes LOCAL statistics, combines them

@@ -384,3 +384,18 @@ def dropout(x, p: float, seed: int):
     draws = (splitmix64(seed, x.size) >> np.uint64(40)).astype(np.int64).reshape(x.shape)
     keep = draws >= int(float(np.float32(p)) * 16777216.0)
     return np.where(keep, x * float(np.float32(1.0) / (np.float32(1.0) - np.float32(p))), 0.0), keep
+
+
+# --------------------------------------------------------------------------------------
+# the dense projection of a layer, numpy float64
+# --------------------------------------------------------------------------------------
+
+def linear(h, w):
+    """z[i, o] = sum_k h[i, k] * w[k, o]."""
+    return np.asarray(h, np.float64) @ np.asarray(w, np.float64)
+
+
+def linear_bwd(h, w, dz):
+    """(dh, dw) of z = h w for the upstream gradient dz."""
+    h, w, dz = (np.asarray(x, np.float64) for x in (h, w, dz))
+    return dz @ w.T, h.T @ dz

@@ -31,7 +31,8 @@ EXPORTS = [
     "sar_gat_project_workspace_bytes", "sar_gat_project", "sar_gat_project_bwd", "sar_relu", "sar_relu_bwd",
     "sar_mfg_frontier", "sar_csr_filter_rows_indptr", "sar_csr_filter_rows_indices", "sar_spmm_agg_scaled",
     "sar_gat_stack_host_wait", "sar_bn_workspace_bytes", "sar_bn_stats", "sar_bn_apply", "sar_bn_bwd_stats",
-    "sar_bn_bwd_apply", "sar_dropout",
+    "sar_bn_bwd_apply", "sar_dropout", "sar_linear_workspace_bytes", "sar_linear", "sar_linear_bwd_input",
+    "sar_linear_bwd_weight",
 ]
 
 
@@ -69,7 +70,7 @@ def lib() -> ctypes.CDLL:
         L.sar_built_for_sm.restype = c_int32
         for name in ("sar_graph_workspace_bytes", "sar_gat_workspace_bytes", "sar_spmm_workspace_bytes",
                      "sar_gat_stack_arena_bytes", "sar_gat_bwd_noalloc_limit", "sar_gat_project_workspace_bytes",
-                     "sar_bn_workspace_bytes"):
+                     "sar_bn_workspace_bytes", "sar_linear_workspace_bytes"):
             getattr(L, name).restype = c_size_t
         _lib = L
     return _lib
@@ -512,6 +513,36 @@ def sar_gat_project_bwd(z: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, d
 
 def sar_relu(x: torch.Tensor) -> None:
     _check("sar_relu", lib().sar_relu(c_int64(x.numel()), ctypes.c_int(_dtype(x)), _ptr(x), _stream()))
+
+
+def sar_linear_workspace_bytes(n: int, d_in: int, d_out: int) -> int:
+    return int(lib().sar_linear_workspace_bytes(c_int64(n), c_int32(d_in), c_int32(d_out)))
+
+
+def sar_linear(h: torch.Tensor, w: torch.Tensor, z: torch.Tensor, workspace: torch.Tensor) -> None:
+    n, d_in = h.shape
+    d_out = w.shape[1]
+    ws, wb = _ws(workspace)
+    _check("sar_linear", lib().sar_linear(c_int64(n), c_int32(d_in), c_int32(d_out), ctypes.c_int(_dtype(h)), _ptr(h),
+                                          _ptr(w), _ptr(z), ws, wb, _stream()))
+
+
+def sar_linear_bwd_input(dz: torch.Tensor, w: torch.Tensor, dh: torch.Tensor, workspace: torch.Tensor) -> None:
+    n, d_out = dz.shape
+    d_in = w.shape[0]
+    ws, wb = _ws(workspace)
+    _check("sar_linear_bwd_input", lib().sar_linear_bwd_input(c_int64(n), c_int32(d_in), c_int32(d_out),
+                                                              ctypes.c_int(_dtype(dz)), _ptr(dz), _ptr(w), _ptr(dh), ws,
+                                                              wb, _stream()))
+
+
+def sar_linear_bwd_weight(h: torch.Tensor, dz: torch.Tensor, dw: torch.Tensor, workspace: torch.Tensor) -> None:
+    n, d_in = h.shape
+    d_out = dz.shape[1]
+    ws, wb = _ws(workspace)
+    _check("sar_linear_bwd_weight", lib().sar_linear_bwd_weight(c_int64(n), c_int32(d_in), c_int32(d_out),
+                                                                ctypes.c_int(_dtype(h)), _ptr(h), _ptr(dz), _ptr(dw), ws,
+                                                                wb, _stream()))
 
 
 def sar_dropout(x: torch.Tensor, p: float, seed: int, y: torch.Tensor) -> None:

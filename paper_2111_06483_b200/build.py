@@ -18,7 +18,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(CSRC, "build")
 LIB = os.path.join(PKG, "libsar.so")
-SOURCES = ["sar_gat.cu", "sar_graph.cu", "sar_host.cu", "sar_noalloc.cu", "sar_glue.cu", "sar_norm.cu"]
+SOURCES = ["sar_gat.cu", "sar_graph.cu", "sar_host.cu", "sar_noalloc.cu", "sar_glue.cu", "sar_norm.cu", "sar_linear.cu"]
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr",
@@ -31,6 +31,19 @@ def _nvcc() -> str:
         if cand and (os.path.isabs(cand) and os.path.exists(cand) or not os.path.isabs(cand)):
             return cand
     raise RuntimeError("nvcc not found")
+
+
+def _cutlass_includes() -> list:
+    """Include paths of a CUTLASS / CuTe header tree with sm100 support (sar_linear.cu instantiates its
+    collective templates).  The image vendors one inside the flashinfer package."""
+    import site
+    roots = list(site.getsitepackages()) + [os.environ.get("CUTLASS_PATH", "")]
+    for root in roots:
+        for sub in ("flashinfer/data/cutlass", "tilelang/3rdparty/cutlass", ""):
+            base = os.path.join(root, sub) if root else ""
+            if base and os.path.exists(os.path.join(base, "include", "cute", "arch", "mma_sm100_umma.hpp")):
+                return ["-I", os.path.join(base, "include"), "-I", os.path.join(base, "tools", "util", "include")]
+    raise RuntimeError("no CUTLASS header tree with sm100 support found (set CUTLASS_PATH)")
 
 
 def _fingerprint() -> str:
@@ -56,7 +69,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
     def compile_one(src):
         obj = os.path.join(OBJ, src.replace(".cu", ".o"))
-        cmd = [nvcc, *NVCC_FLAGS, *extra, "-c", os.path.join(CSRC, src), "-o", obj]
+        inc = _cutlass_includes() if src == "sar_linear.cu" else []
+        cmd = [nvcc, *NVCC_FLAGS, *inc, *extra, "-c", os.path.join(CSRC, src), "-o", obj]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             raise RuntimeError(f"nvcc failed on {src}:\n{r.stdout}\n{r.stderr}")

@@ -46,3 +46,16 @@ def test_layer_stack_matches_torch_autograd_on_dense_formulation():
     for l in range(L):
         allclose_report(got["da_l"][l], als[l].grad.numpy(), 1e-4, 1e-5, f"da_l[{l}]")
         allclose_report(got["da_r"][l], ars[l].grad.numpy(), 1e-4, 1e-5, f"da_r[{l}]")
+
+
+def test_linear_is_the_definition_and_its_backward_matches_autograd():
+    rng = np.random.default_rng(4)
+    h, w, dz = rng.standard_normal((9, 5)), rng.standard_normal((5, 7)), rng.standard_normal((9, 7))
+    z = oracle.linear(h, w)
+    brute = np.array([[sum(h[i, k] * w[k, o] for k in range(5)) for o in range(7)] for i in range(9)])
+    allclose_report(z, brute, 1e-13, 1e-14, "z")
+    ht, wt = torch.tensor(h, requires_grad=True), torch.tensor(w, requires_grad=True)
+    ((ht @ wt) * torch.tensor(dz)).sum().backward()
+    dh, dw = oracle.linear_bwd(h, w, dz)
+    allclose_report(dh, ht.grad.numpy(), 1e-12, 1e-13, "dh")
+    allclose_report(dw, wt.grad.numpy(), 1e-12, 1e-13, "dw")
