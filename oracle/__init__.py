@@ -281,6 +281,39 @@ def gat_stack(indptr, indices, feat0, a_l, a_r, gout, slope: float, storage=np.f
     return dict(out=z[L].astype(np.float64), dfeat0=g, da_l=da_l, da_r=da_r)
 
 
+def gat_net(indptr, indices, h0, weights, a_l, a_r, gout, slope: float, stored=None):
+    """L whole layers h^{l+1} = ReLU(GAT(z, <z,a_l>, <z,a_r>)) with z = h^l W^l, and the gradient of
+    <gout, h^L> with respect to h^0, every W^l, a_l^l, a_r^l.  float64 except at the aggregation
+    functions' float32 inputs.  `stored(x)` (default: identity) is applied wherever an implementation with
+    narrower storage keeps a node array between two steps (z, the layer outputs, dz, dh), so that a bf16
+    implementation can be compared on equal inputs: the score gradients are differences of nearly equal sums
+    and amplify a rounding of their inputs."""
+    st = (lambda x: x) if stored is None else stored
+    L = len(weights)
+    h = [np.asarray(h0, dtype=np.float64)]
+    saved = []
+    n = h[0].shape[0]
+    H, F = np.asarray(a_l[0]).shape
+    for l in range(L):
+        z = st(linear(h[l], weights[l])).reshape(n, H, F)
+        el, er = project(z, a_l[l], a_r[l])
+        f = gat_fwd(indptr, indices, z.astype(np.float32), el.astype(np.float32), er.astype(np.float32), slope)
+        saved.append((z, el, er, f))
+        h.append(np.maximum(st(f.out), 0.0).reshape(n, H * F))
+    g = np.asarray(gout, dtype=np.float64).reshape(n, H * F)
+    dW, da_l, da_r = [None] * L, [None] * L, [None] * L
+    for l in reversed(range(L)):
+        z, el, er, f = saved[l]
+        g = np.where(h[l + 1] > 0, g, 0.0)
+        b = gat_bwd(indptr, indices, z.astype(np.float32), el.astype(np.float32), er.astype(np.float32), f.alpha,
+                    g.reshape(n, H, F).astype(np.float32), slope)
+        dz_add, da_l[l], da_r[l] = project_bwd(z, a_l[l], a_r[l], b.del_.astype(np.float32), b.der.astype(np.float32))
+        dz = st(st(b.dfeat) + dz_add).reshape(n, H * F)
+        dh, dW[l] = linear_bwd(h[l], weights[l], dz)
+        g = st(dh)
+    return dict(out=h[L], dh0=g, dW=dW, da_l=da_l, da_r=da_r)
+
+
 # --------------------------------------------------------------------------------------
 # message-flow pruning (Appendix B), plain numpy / Python loops
 # --------------------------------------------------------------------------------------

@@ -314,3 +314,46 @@ def bn_backward(x: torch.Tensor, gy: torch.Tensor, saved, gamma: Optional[torch.
     gx = torch.empty_like(x)
     B.sar_bn_bwd_apply(x, mean, rstd, gamma, gy, s0, s1, 1.0 / max(n_all, 1), gx)
     return gx, s1, s0
+
+
+# ----------------------------------------------------------------------------------------------
+# whole layers: h' = GAT(z, <z,a_l>, <z,a_r>) with z = ReLU?(h) W  (bf16; the dense projection runs on the
+# tensor cores).  Marshalling only.
+
+def full_layer_forward(g: Graph, h: torch.Tensor, W: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, slope: float,
+                       relu_input: bool = False):
+    """h [n, D_in], W [D_in, H*F] (bf16), a_l / a_r [H, F] float32.  Returns (out [n,H,F], saved).
+    relu_input=True first applies h = max(h, 0) in place (the activation that closes the previous layer)."""
+    n = h.shape[0]
+    H, F = a_l.shape
+    if relu_input:
+        B.sar_relu(h)
+    z = torch.empty((n, H, F), dtype=h.dtype, device=h.device)
+    ws = _workspace(B.sar_linear_workspace_bytes(n, h.shape[1], H * F), h.device)
+    B.sar_linear(h, W, z.view(n, H * F), ws)
+    el = torch.empty((n, H), dtype=torch.float32, device=h.device)
+    er = torch.empty_like(el)
+    B.sar_gat_project(z, a_l, a_r, el, er, 0)
+    out, m, d = gat_forward(g, z, el, er, slope)
+    return out, (z, el, er, m, d)
+
+
+def full_layer_backward(g: Graph, h: torch.Tensor, W: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, saved,
+                        gout: torch.Tensor, slope: float, relu_input: bool = False):
+    """Returns (dh [n, D_in], dW [D_in, H*F] float32, da_l, da_r); with relu_input=True dh is the gradient
+    before the input's ReLU (h must be the array full_layer_forward left, i.e. already max(h, 0))."""
+    n, d_in = h.shape
+    H, F = a_l.shape
+    z, el, er, m, d = saved
+    dz, del_, der = gat_backward(g, z, el, er, m, d, gout, slope)
+    da_l = torch.empty((H, F), dtype=torch.float32, device=h.device)
+    da_r = torch.empty_like(da_l)
+    B.sar_gat_project_bwd(z, a_l, a_r, del_, der, dz, da_l, da_r, _workspace(B.sar_gat_project_workspace_bytes(H, F), h.device), 0)
+    ws = _workspace(B.sar_linear_workspace_bytes(n, d_in, H * F), h.device)
+    dW = torch.empty((d_in, H * F), dtype=torch.float32, device=h.device)
+    B.sar_linear_bwd_weight(h, dz.view(n, H * F), dW, ws)
+    dh = torch.empty_like(h)
+    B.sar_linear_bwd_input(dz.view(n, H * F), W, dh, ws)
+    if relu_input:
+        B.sar_relu_bwd(h, dh)
+    return dh, dW, da_l, da_r

@@ -51,3 +51,49 @@ def test_projection_rejects_what_it_cannot_do():
     with pytest.raises(B.SarError) as ei:   # float32 storage
         B.sar_linear(hf, torch.zeros((16, 8), device="cuda"), torch.zeros((16, 8), device="cuda"), ws)
     assert ei.value.code == -2
+
+
+def test_two_whole_layers_match_the_oracle_network():
+    """Dense projection -> scores -> aggregation -> ReLU, twice, forward and backward, on bf16 storage, against
+    the float64 network of the oracle, which rounds the node arrays to bf16 where the library stores them (the
+    score gradients amplify a rounding of their inputs).  Compared in relative Frobenius norm."""
+    from paper_2111_06483_b200 import api, binding as B
+    from helpers import small_problem
+    n, H, F, L = 4000, 4, 16, 2
+    D = H * F
+    p = small_problem(n, 50000, H, F, 61, self_loops=True, empty_rows=6)
+    rng = np.random.default_rng(8)
+    bf = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(torch.bfloat16)
+    Ws = [bf(rng.standard_normal((D, D)) / np.sqrt(D)) for _ in range(L)]
+    a_l = [(rng.standard_normal((H, F)) * 0.3).astype(np.float32) for _ in range(L)]
+    a_r = [(rng.standard_normal((H, F)) * 0.3).astype(np.float32) for _ in range(L)]
+    h0 = bf(p["feat"].reshape(n, D))
+    gout = bf(p["gout"])
+    as_bf16 = lambda x: torch.from_numpy(np.ascontiguousarray(x)).to(torch.bfloat16).double().numpy()
+    want = oracle.gat_net(p["indptr"], p["indices"], _np(h0), [_np(w) for w in Ws], a_l, a_r, _np(gout), 0.2,
+                          stored=as_bf16)
+    g = api.Graph.from_coo(n, torch.from_numpy(p["src"]).cuda(), torch.from_numpy(p["dst"]).cuda(), k=2)
+    dev = lambda x: torch.from_numpy(x).cuda()
+    h = [h0.cuda()]
+    saved = []
+    for l in range(L):
+        out, sv = api.full_layer_forward(g, h[l], Ws[l].cuda(), dev(a_l[l]), dev(a_r[l]), 0.2, relu_input=l > 0)
+        h.append(out.view(n, D))
+        saved.append(sv)
+    B.sar_relu(h[L])
+    grad = gout.cuda().clone()
+    B.sar_relu_bwd(h[L].view(n, H, F), grad)
+    got_dW, got_al, got_ar = [None] * L, [None] * L, [None] * L
+    for l in reversed(range(L)):
+        grad, got_dW[l], got_al[l], got_ar[l] = api.full_layer_backward(g, h[l], Ws[l].cuda(), dev(a_l[l]), dev(a_r[l]),
+                                                                        saved[l], grad.view(n, H, F), 0.2, relu_input=l > 0)
+    rel = lambda a, b: np.linalg.norm(a - b) / max(np.linalg.norm(b), 1e-30)
+    assert rel(_np(h[L]), want["out"]) < 2e-2
+    # gradients: a unit whose pre-activation lies within the forward error of zero takes the other branch of its
+    # ReLU; a wrong or missing term would show as an error of tens of percent
+    errs = {"dh0": rel(_np(grad), want["dh0"])}
+    for l in range(L):
+        errs[f"dW{l}"] = rel(_np(got_dW[l]), want["dW"][l])
+        errs[f"da_l{l}"] = rel(_np(got_al[l]), want["da_l"][l])
+        errs[f"da_r{l}"] = rel(_np(got_ar[l]), want["da_r"][l])
+    assert max(errs.values()) < 3e-2, errs

@@ -59,3 +59,30 @@ def test_linear_is_the_definition_and_its_backward_matches_autograd():
     dh, dw = oracle.linear_bwd(h, w, dz)
     allclose_report(dh, ht.grad.numpy(), 1e-12, 1e-13, "dh")
     allclose_report(dw, wt.grad.numpy(), 1e-12, 1e-13, "dw")
+
+
+def test_whole_network_with_weights_matches_torch_autograd():
+    p = small_problem(30, 200, 2, 4, 43, self_loops=True, empty_rows=2)
+    rng = np.random.default_rng(6)
+    L, D = 2, 8
+    Ws = [rng.standard_normal((D, D)) / np.sqrt(D) for _ in range(L)]
+    a_l = [rng.standard_normal((2, 4)) * 0.5 for _ in range(L)]
+    a_r = [rng.standard_normal((2, 4)) * 0.5 for _ in range(L)]
+    h0 = p["feat"].reshape(30, D).astype(np.float64)
+    got = oracle.gat_net(p["indptr"], p["indices"], h0, Ws, a_l, a_r, p["gout"], 0.2)
+    C = torch.from_numpy(count_matrix(30, 30, p["src"], p["dst"]))
+    h = torch.tensor(h0, requires_grad=True)
+    h_in = h
+    Wt = [torch.tensor(x, requires_grad=True) for x in Ws]
+    als = [torch.tensor(x, requires_grad=True) for x in a_l]
+    ars = [torch.tensor(x, requires_grad=True) for x in a_r]
+    for l in range(L):
+        z = (h @ Wt[l]).reshape(30, 2, 4)
+        h = torch.relu(dense_gat_torch(C, z, (z * als[l]).sum(-1), (z * ars[l]).sum(-1), 0.2)).reshape(30, D)
+    (h * torch.tensor(p["gout"], dtype=torch.float64).reshape(30, D)).sum().backward()
+    allclose_report(got["out"], h.detach().numpy(), 1e-5, 1e-6, "net out")
+    allclose_report(got["dh0"], h_in.grad.numpy(), 1e-4, 1e-5, "net dh0")
+    for l in range(L):
+        allclose_report(got["dW"][l], Wt[l].grad.numpy(), 1e-4, 1e-5, f"dW[{l}]")
+        allclose_report(got["da_l"][l], als[l].grad.numpy(), 1e-4, 1e-5, f"da_l[{l}]")
+        allclose_report(got["da_r"][l], ars[l].grad.numpy(), 1e-4, 1e-5, f"da_r[{l}]")
