@@ -119,19 +119,28 @@ static sar_status launch_span(SpanArgs a, long long nnz, const char *name, const
     a.R = rows_per_span(a.n_rows, nnz, CAP);
     const long long spans = (a.n_rows + a.R - 1) / a.R;
     if (spans > 0) {
-        SAR_LAUNCH(name, st, kern<<<(unsigned)((spans + kSpanWarps - 1) / kSpanWarps), kSpanThreads, smem, st>>>(a));
+        const unsigned blocks = (unsigned)((spans + kSpanWarps - 1) / kSpanWarps);
+        if ((a.flags & SAR_FIRST) && (a.flags & SAR_LAST)) {  // the epilogue's flag tests decided at compile time
+            auto whole = span_kernel<T, G, V, S, MODE, CAP, MINB, 1>;
+            SAR_TRY(ensure_smem(whole, smem));
+            SAR_LAUNCH(name, st, whole<<<blocks, kSpanThreads, smem, st>>>(a));
+        } else {
+            SAR_LAUNCH(name, st, kern<<<blocks, kSpanThreads, smem, st>>>(a));
+        }
         SAR_TRY(sar_after_launch());
     }
     if (a.sp.threshold > 0 && a.sp.n_seg > 0) {
         a.mode = 1;
         const unsigned blocks = (unsigned)((a.sp.n_seg + kSpanWarps - 1) / kSpanWarps);
         if (a.sp.threshold <= CAP_SEG) {
-            auto seg_kern = span_kernel<T, G, V, S, MODE, CAP_SEG, MINB>;
+            auto seg_kern = span_kernel<T, G, V, S, MODE, CAP_SEG, MINB, 2>;
             const size_t seg_smem = (size_t)kSpanWarps * span_layout<MODE>(a.g.Hp, V, CAP_SEG, S, 32 / G).total;
             SAR_TRY(ensure_smem(seg_kern, seg_smem));
             SAR_LAUNCH(seg_name, st, seg_kern<<<blocks, kSpanThreads, seg_smem, st>>>(a));
         } else {
-            SAR_LAUNCH(seg_name, st, kern<<<blocks, kSpanThreads, smem, st>>>(a));
+            auto seg_kern = span_kernel<T, G, V, S, MODE, CAP, MINB, 2>;
+            SAR_TRY(ensure_smem(seg_kern, smem));
+            SAR_LAUNCH(seg_name, st, seg_kern<<<blocks, kSpanThreads, smem, st>>>(a));
         }
         SAR_TRY(sar_after_launch());
     }
