@@ -120,10 +120,17 @@ static sar_status launch_span(SpanArgs a, long long nnz, const char *name, const
     const long long spans = (a.n_rows + a.R - 1) / a.R;
     if (spans > 0) {
         const unsigned blocks = (unsigned)((spans + kSpanWarps - 1) / kSpanWarps);
+        const bool geo = G * V >= 4 && a.g.H == 4 && a.g.Hp == 4 && a.g.n_vec == G * V && MODE != kSum && MODE != kSumW;
         if ((a.flags & SAR_FIRST) && (a.flags & SAR_LAST)) {  // the epilogue's flag tests decided at compile time
-            auto whole = span_kernel<T, G, V, S, MODE, CAP, MINB, 1>;
-            SAR_TRY(ensure_smem(whole, smem));
-            SAR_LAUNCH(name, st, whole<<<blocks, kSpanThreads, smem, st>>>(a));
+            if (geo) {
+                auto whole = span_kernel<T, G, V, S, MODE, CAP, MINB, 1, (G * V >= 4 && MODE != kSum && MODE != kSumW) ? 1 : 0>;
+                SAR_TRY(ensure_smem(whole, smem));
+                SAR_LAUNCH(name, st, whole<<<blocks, kSpanThreads, smem, st>>>(a));
+            } else {
+                auto whole = span_kernel<T, G, V, S, MODE, CAP, MINB, 1>;
+                SAR_TRY(ensure_smem(whole, smem));
+                SAR_LAUNCH(name, st, whole<<<blocks, kSpanThreads, smem, st>>>(a));
+            }
         } else {
             SAR_LAUNCH(name, st, kern<<<blocks, kSpanThreads, smem, st>>>(a));
         }

@@ -165,7 +165,9 @@ __host__ __device__ inline SpanSmem span_layout(int Hp, int V, int cap, int stag
 // STATIC decides the launch mode at compile time, so that the flag tests of the row epilogue fold away:
 // 1 = rows (mode 0) of a partition that holds all sources (SAR_FIRST | SAR_LAST), the benchmarked configuration;
 // 2 = long-row segments (mode 1); 0 = whatever SpanArgs says.
-template <typename T, int G, int V, int S, int MODE, int CAP, int MINB, int STATIC = 0>
+// GEO = 1 fixes the row geometry at compile time as well: 4 heads and rows of exactly G*V vectors (the paper's GAT:
+// 4 heads, hidden size 128), so that head arithmetic becomes shifts and the lane predicates vanish.
+template <typename T, int G, int V, int S, int MODE, int CAP, int MINB, int STATIC = 0, int GEO = 0>
 __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs a) {
     constexpr int EPV = Elem<T>::EPV;
     constexpr int EPW = 32 / G;  // edges per slot
@@ -181,7 +183,8 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gl = lane & (G - 1), half = lane / G;
-    const int H = a.g.H, Hp = a.g.Hp, lgHp = a.g.lgHp, n_vec = a.g.n_vec;
+    const int H = GEO ? 4 : a.g.H, Hp = GEO ? 4 : a.g.Hp, lgHp = GEO ? 2 : a.g.lgHp, n_vec = GEO ? G * V : a.g.n_vec;
+    const int vph = GEO ? (G * V) / 4 : a.g.vph;
     const long long rowf = (long long)n_vec * EPV;
 
     // ---- shared memory carve-up (per warp) ----------------------------------------------------
@@ -255,8 +258,8 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
     for (int v = 0; v < V; ++v) {
         const int vi = v * G + gl;
         vok[v] = vi < n_vec;
-        hv[v] = vok[v] ? vi / a.g.vph : 0;
-        lead[v] = vok[v] && (vi - hv[v] * a.g.vph) == 0;
+        hv[v] = vok[v] ? vi / vph : 0;
+        lead[v] = vok[v] && (vi - hv[v] * vph) == 0;
     }
     const unsigned stage_s = (unsigned)__cvta_generic_to_shared(stage) + lane * 16;
     const unsigned sj_s = (unsigned)__cvta_generic_to_shared(sj) + half * 4;
@@ -800,9 +803,9 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                     __syncwarp();
                     if (lane < H) {
                         float DB = 0.f, DA = 0.f;
-                        for (int k = 0; k < a.g.vph; ++k) {
-                            DB += scratch[lane * a.g.vph + k];
-                            DA += scratch[32 * V + lane * a.g.vph + k];
+                        for (int k = 0; k < vph; ++k) {
+                            DB += scratch[lane * vph + k];
+                            DA += scratch[32 * V + lane * vph + k];
                         }
                         const float Sh = scratch[64 * V + lane];
                         const float D = MODE == kBwdDstGivenD ? a.rec_in[row * H + lane].w : DA;
@@ -844,7 +847,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                     __syncwarp();
                     if (lane < H) {
                         float DC = 0.f;
-                        for (int k = 0; k < a.g.vph; ++k) DC += scratch[lane * a.g.vph + k];
+                        for (int k = 0; k < vph; ++k) DC += scratch[lane * vph + k];
                         a.der[row * H + lane] = DC - scratch[64 * V + lane];
                     }
                     __syncwarp();
