@@ -116,14 +116,15 @@ static sar_status launch_span(SpanArgs a, long long nnz, const char *name, const
     const size_t smem = (size_t)kSpanWarps * span_layout<MODE>(a.g.Hp, V, CAP, S, 32 / G).total;
     SAR_TRY(ensure_smem(kern, smem));
     a.mode = 0;
+    constexpr int kGeo = (G * V >= 4 && MODE != kSum && MODE != kSumW) ? 1 : 0;
+    const bool geo = kGeo && a.g.H == 4 && a.g.Hp == 4 && a.g.n_vec == G * V && a.hvec;
     a.R = rows_per_span(a.n_rows, nnz, CAP);
     const long long spans = (a.n_rows + a.R - 1) / a.R;
     if (spans > 0) {
         const unsigned blocks = (unsigned)((spans + kSpanWarps - 1) / kSpanWarps);
-        const bool geo = G * V >= 4 && a.g.H == 4 && a.g.Hp == 4 && a.g.n_vec == G * V && MODE != kSum && MODE != kSumW;
         if ((a.flags & SAR_FIRST) && (a.flags & SAR_LAST)) {  // the epilogue's flag tests decided at compile time
             if (geo) {
-                auto whole = span_kernel<T, G, V, S, MODE, CAP, MINB, 1, (G * V >= 4 && MODE != kSum && MODE != kSumW) ? 1 : 0>;
+                auto whole = span_kernel<T, G, V, S, MODE, CAP, MINB, 1, kGeo>;
                 SAR_TRY(ensure_smem(whole, smem));
                 SAR_LAUNCH(name, st, whole<<<blocks, kSpanThreads, smem, st>>>(a));
             } else {
@@ -140,13 +141,15 @@ static sar_status launch_span(SpanArgs a, long long nnz, const char *name, const
         a.mode = 1;
         const unsigned blocks = (unsigned)((a.sp.n_seg + kSpanWarps - 1) / kSpanWarps);
         if (a.sp.threshold <= CAP_SEG) {
-            auto seg_kern = span_kernel<T, G, V, S, MODE, CAP_SEG, MINB, 2>;
             const size_t seg_smem = (size_t)kSpanWarps * span_layout<MODE>(a.g.Hp, V, CAP_SEG, S, 32 / G).total;
-            SAR_TRY(ensure_smem(seg_kern, seg_smem));
+            auto seg_kern = geo ? span_kernel<T, G, V, S, MODE, CAP_SEG, MINB, 2, kGeo> : span_kernel<T, G, V, S, MODE, CAP_SEG, MINB, 2>;
+            SAR_TRY(ensure_smem(span_kernel<T, G, V, S, MODE, CAP_SEG, MINB, 2, kGeo>, seg_smem));
+            SAR_TRY(ensure_smem(span_kernel<T, G, V, S, MODE, CAP_SEG, MINB, 2>, seg_smem));
             SAR_LAUNCH(seg_name, st, seg_kern<<<blocks, kSpanThreads, seg_smem, st>>>(a));
         } else {
-            auto seg_kern = span_kernel<T, G, V, S, MODE, CAP, MINB, 2>;
-            SAR_TRY(ensure_smem(seg_kern, smem));
+            auto seg_kern = geo ? span_kernel<T, G, V, S, MODE, CAP, MINB, 2, kGeo> : span_kernel<T, G, V, S, MODE, CAP, MINB, 2>;
+            SAR_TRY(ensure_smem(span_kernel<T, G, V, S, MODE, CAP, MINB, 2, kGeo>, smem));
+            SAR_TRY(ensure_smem(span_kernel<T, G, V, S, MODE, CAP, MINB, 2>, smem));
             SAR_LAUNCH(seg_name, st, seg_kern<<<blocks, kSpanThreads, smem, st>>>(a));
         }
         SAR_TRY(sar_after_launch());

@@ -165,8 +165,9 @@ __host__ __device__ inline SpanSmem span_layout(int Hp, int V, int cap, int stag
 // STATIC decides the launch mode at compile time, so that the flag tests of the row epilogue fold away:
 // 1 = rows (mode 0) of a partition that holds all sources (SAR_FIRST | SAR_LAST), the benchmarked configuration;
 // 2 = long-row segments (mode 1); 0 = whatever SpanArgs says.
-// GEO = 1 fixes the row geometry at compile time as well: 4 heads and rows of exactly G*V vectors (the paper's GAT:
-// 4 heads, hidden size 128), so that head arithmetic becomes shifts and the lane predicates vanish.
+// GEO = 1 fixes the row geometry at compile time as well: 4 heads scored four at a time (SpanArgs::hvec set) and rows
+// of exactly G*V vectors (the paper's GAT: 4 heads, hidden size 128), so that head arithmetic becomes shifts and the
+// lane predicates vanish.
 template <typename T, int G, int V, int S, int MODE, int CAP, int MINB, int STATIC = 0, int GEO = 0>
 __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs a) {
     constexpr int EPV = Elem<T>::EPV;
@@ -442,7 +443,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
             }
             __syncwarp();
         } else if constexpr (MODE != kSum) {
-            const bool vec4 = a.hvec != 0;  // heads handled four at a time with 16-byte accesses
+            const bool vec4 = GEO ? true : a.hvec != 0;  // heads handled four at a time with 16-byte accesses
             int i = 0;
             for (int q0 = lane; q0 < npos; q0 += 64) {
                 int col[2], rbase[2];
@@ -596,7 +597,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                 sc2[x] = ref;
             }
             __syncwarp();
-            const bool vec4 = a.hvec != 0;
+            const bool vec4 = GEO ? true : a.hvec != 0;
             int i = 0;
             for (int q = lane; q < npos; q += 32) {
                 while (q >= sso[i + 1] * EPW) ++i;
