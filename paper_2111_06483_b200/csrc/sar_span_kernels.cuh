@@ -103,20 +103,14 @@ __device__ __forceinline__ void cp_async16_s(unsigned smem_addr, const void *gsr
 }
 
 // packed pairs of float32 (Blackwell's two-wide FP32 pipe: one instruction, two fused multiply-adds)
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pack2(float lo, float hi) {
-    f32x2 r;
-    asm("mov.b64 %0, {%1, %2};\n" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
+typedef float2 f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi) { return make_float2(lo, hi); }
 __device__ __forceinline__ void unpack2(f32x2 p, float &lo, float &hi) {
-    asm("mov.b64 {%0, %1}, %2;\n" : "=f"(lo), "=f"(hi) : "l"(p));
+    lo = p.x;
+    hi = p.y;
 }
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) {  // a*b + c, element-wise
-    f32x2 r;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;\n" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-    return r;
-}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c) { return __ffma2_rn(a, b, c); }  // a*b + c, element-wise
+__device__ __forceinline__ f32x2 zero2() { return make_float2(0.f, 0.f); }
 // 16 bytes of storage type T -> EPV/2 packed float32 pairs
 template <typename T>
 struct Pairs;
@@ -280,7 +274,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
         sv[v] = 0.f;
         mrun[v] = SAR_NEG_INF;
 #pragma unroll
-        for (int k = 0; k < NP; ++k) pacc0[v][k] = pacc1[v][k] = 0ull;
+        for (int k = 0; k < NP; ++k) pacc0[v][k] = pacc1[v][k] = zero2();
 #pragma unroll
         for (int e = 0; e < EPV; ++e) rv[v][e] = 0.f;
     }
@@ -626,7 +620,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                     mrun[v] = sc2[hv[v]];
                     const f32x2 c2 = pack2(c, c);
 #pragma unroll
-                    for (int k = 0; k < NP; ++k) pacc0[v][k] = fma2(pacc0[v][k], c2, 0ull);
+                    for (int k = 0; k < NP; ++k) pacc0[v][k] = fma2(pacc0[v][k], c2, zero2());
                 }
             }
         }
@@ -888,7 +882,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                 sv[v] = 0.f;
                 mrun[v] = SAR_NEG_INF;
 #pragma unroll
-                for (int k = 0; k < NP; ++k) pacc0[v][k] = pacc1[v][k] = 0ull;
+                for (int k = 0; k < NP; ++k) pacc0[v][k] = pacc1[v][k] = zero2();
             }
         }
         cp_async_wait<0>();  // drain the (zero-size) refills issued past the last slot
