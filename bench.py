@@ -96,9 +96,9 @@ KERNEL_BYTES = {"gat_fwd": bytes_fwd, "gat_bwd_dst": bytes_bwd_dst, "gat_bwd_src
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one pass (rows + segments + merge launches),
 # from the one-pass ncu capture at full size whose launch list is summarised under profiles/.
 NCU_TRAFFIC_BYTES = {
-    ("large", "bf16", "gat_fwd"): 81.85e9,
+    ("large", "bf16", "gat_fwd"): 81.89e9,
     ("large", "bf16", "gat_bwd_dst"): 84.07e9,
-    ("large", "bf16", "gat_bwd_src"): 89.10e9,
+    ("large", "bf16", "gat_bwd_src"): 89.08e9,
 }
 
 
