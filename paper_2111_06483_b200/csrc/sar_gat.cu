@@ -116,8 +116,9 @@ static sar_status launch_span(SpanArgs a, long long nnz, const char *name, const
     const size_t smem = (size_t)kSpanWarps * span_layout<MODE>(a.g.Hp, V, CAP, S, 32 / G).total;
     SAR_TRY(ensure_smem(kern, smem));
     a.mode = 0;
-    constexpr int kGeo = (G * V >= 4 && MODE != kSum && MODE != kSumW) ? 1 : 0;
-    const bool geo = kGeo && a.g.H == 4 && a.g.Hp == 4 && a.g.n_vec == G * V && a.hvec;
+    constexpr bool kIsSum = MODE == kSum || MODE == kSumW;
+    constexpr int kGeo = (kIsSum || G * V >= 4) ? 1 : 0;
+    const bool geo = kGeo && a.g.n_vec == G * V && (kIsSum ? a.g.H == 1 : (a.g.H == 4 && a.g.Hp == 4 && a.hvec));
     a.R = rows_per_span(a.n_rows, nnz, CAP);
     const long long spans = (a.n_rows + a.R - 1) / a.R;
     if (spans > 0) {

@@ -159,9 +159,9 @@ __host__ __device__ inline SpanSmem span_layout(int Hp, int V, int cap, int stag
 // STATIC decides the launch mode at compile time, so that the flag tests of the row epilogue fold away:
 // 1 = rows (mode 0) of a partition that holds all sources (SAR_FIRST | SAR_LAST), the benchmarked configuration;
 // 2 = long-row segments (mode 1); 0 = whatever SpanArgs says.
-// GEO = 1 fixes the row geometry at compile time as well: 4 heads scored four at a time (SpanArgs::hvec set) and rows
-// of exactly G*V vectors (the paper's GAT: 4 heads, hidden size 128), so that head arithmetic becomes shifts and the
-// lane predicates vanish.
+// GEO = 1 fixes the row geometry at compile time as well: rows of exactly G*V vectors and, for the attention modes,
+// 4 heads scored four at a time (SpanArgs::hvec set; the paper's GAT: 4 heads, hidden size 128), for the sums one
+// head, so that head arithmetic becomes shifts and the lane predicates vanish.
 template <typename T, int G, int V, int S, int MODE, int CAP, int MINB, int STATIC = 0, int GEO = 0>
 __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs a) {
     constexpr int EPV = Elem<T>::EPV;
@@ -178,8 +178,9 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
 
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int gl = lane & (G - 1), half = lane / G;
-    const int H = GEO ? 4 : a.g.H, Hp = GEO ? 4 : a.g.Hp, lgHp = GEO ? 2 : a.g.lgHp, n_vec = GEO ? G * V : a.g.n_vec;
-    const int vph = GEO ? (G * V) / 4 : a.g.vph;
+    constexpr int kGeoH = (MODE == kSum || MODE == kSumW) ? 1 : 4;  // heads of the compile-time geometry
+    const int H = GEO ? kGeoH : a.g.H, Hp = GEO ? kGeoH : a.g.Hp, lgHp = GEO ? (kGeoH == 4 ? 2 : 0) : a.g.lgHp;
+    const int n_vec = GEO ? G * V : a.g.n_vec, vph = GEO ? (G * V) / kGeoH : a.g.vph;
     const long long rowf = (long long)n_vec * EPV;
 
     // ---- shared memory carve-up (per warp) ----------------------------------------------------
