@@ -326,22 +326,50 @@ SAR_API sar_status sar_relu_bwd(int64_t n_elems, sar_dtype t, const void *y, voi
  * runs on the tensor cores (tcgen05 MMA, accumulators in tensor memory, operands staged by TMA; CUTLASS
  * sm100 collectives instantiated in the library), bf16 operands with float32 accumulation.
  *   sar_linear             z[n, d_out]  = h[n, d_in] W[d_in, d_out]          (bf16 out)
+ *   sar_linear_accumulate  z[n, d_out] += h[n, d_in] W[d_in, d_out]          (z read and written, bf16: the sum
+ *                          over relations of Appendix A's layer, one call per relation)
  *   sar_linear_bwd_input   dh[n, d_in]  = dz[n, d_out] W^T                   (bf16 out)
  *   sar_linear_bwd_weight  dw[d_in, d_out] = h^T dz                          (float32 out; the n-long
  *                          contraction is cut across the SMs and the partial tiles are reduced in the scratch)
  * All arrays row-major DEVICE memory, 16-byte aligned; t must be SAR_BF16 and d_in, d_out multiples of 8
  * (SAR_ERR_UNSUPPORTED otherwise); n <= 2^31-1.  Scratch: sar_linear_workspace_bytes(n, d_in, d_out) covers
- * the three calls.  n = 0 is allowed (dw is then written as zeros).
+ * all of these calls.  n = 0 is allowed (dw is then written as zeros).
  * ------------------------------------------------------------------------------------------- */
 SAR_API size_t sar_linear_workspace_bytes(int64_t n, int32_t d_in, int32_t d_out);
 SAR_API sar_status sar_linear(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *h, const void *w,
                               void *z, void *workspace, size_t workspace_bytes, void *stream);
+SAR_API sar_status sar_linear_accumulate(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *h,
+                                         const void *w, void *z, void *workspace, size_t workspace_bytes,
+                                         void *stream);
 SAR_API sar_status sar_linear_bwd_input(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *dz,
                                         const void *w, void *dh, void *workspace, size_t workspace_bytes,
                                         void *stream);
 SAR_API sar_status sar_linear_bwd_weight(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *h,
                                          const void *dz, float *dw, void *workspace, size_t workspace_bytes,
                                          void *stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Relational layer (Appendix A): h'_i = sigma( sum_r sum_{j in N^r_i} W_r h_j / |N^r_i| ), one graph per
+ * relation r.  The layer is a sequence of calls of this library, per relation: the mean aggregation of h over
+ * the relation's graph (sar_spmm_agg with SAR_MEAN, partition by partition), then z += agg_r W_r
+ * (sar_linear / sar_linear_accumulate).  Backward, per relation: the aggregate is rebuilt from h (the
+ * input features are needed again, as the appendix notes - nothing of size R x n is kept), dW_r = agg_r^T dz
+ * (sar_linear_bwd_weight), dagg_r = dz W_r^T (sar_linear_bwd_input), and dh (+)= the sum over the relation's
+ * out-edges of dagg_r[i] / |N^r_i| (sar_spmm_agg_scaled on the transposed partition with src_scale from
+ * sar_degree_scale).  The two helpers below are what is not covered by those calls.
+ *   sar_degree_scale    scale[i] = deg(i)^power with deg(i) = indptr[i+1] - indptr[i], 0 where deg(i) = 0;
+ *                       power <= 0 (-1: the mean's factor, -0.5: the symmetric normalisation of Sec. 4.2's
+ *                       propagation).  indptr [n+1] int64, scale [n] float32.
+ *   sar_rgcn_basis      W[r,:] = sum_b a[r,b] V[b,:] (the appendix's second equation): a [R,B], V [B,size]
+ *                       float32, W [R,size] of type t (bf16 for the contraction), size = d_in*d_out.
+ *   sar_rgcn_basis_bwd  da[r,b] = <dW[r,:], V[b,:]>, dV[b,:] = sum_r a[r,b] dW[r,:]; all float32, written.
+ * All pointers DEVICE memory owned by the caller; n = 0 / size = 0 allowed.
+ * ------------------------------------------------------------------------------------------- */
+SAR_API sar_status sar_degree_scale(int64_t n, const int64_t *indptr, float power, float *scale, void *stream);
+SAR_API sar_status sar_rgcn_basis(int32_t R, int32_t B, int64_t size, sar_dtype t, const float *a, const float *V,
+                                  void *W, void *stream);
+SAR_API sar_status sar_rgcn_basis_bwd(int32_t R, int32_t B, int64_t size, const float *a, const float *V,
+                                      const float *dW, float *da, float *dV, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Batch normalisation over the node dimension (Sec. 3.4, "Batch normalization"): y[i,c] =

@@ -432,3 +432,67 @@ def linear_bwd(h, w, dz):
     """(dh, dw) of z = h w for the upstream gradient dz."""
     h, w, dz = (np.asarray(x, np.float64) for x in (h, w, dz))
     return dz @ w.T, h.T @ dz
+
+
+# --------------------------------------------------------------------------------------
+# relational layer (Appendix A), plain numpy float64 written from the layer's equation:
+# every neighbour's features are transformed by the relation's matrix, then averaged per
+# relation and summed over the relations
+# --------------------------------------------------------------------------------------
+
+def rgcn_layer(graphs, h, weights):
+    """z[i,:] = sum_r (1/|N^r_i|) sum_{j in N^r_i} h[j,:] W_r  (the argument of sigma in the appendix's first
+    equation).  graphs: one (indptr, indices) CSR by destination per relation; weights: [R][d_in, d_out]."""
+    h = np.asarray(h, np.float64)
+    n = _i64(graphs[0][0]).shape[0] - 1
+    d_out = np.asarray(weights[0]).shape[1]
+    z = np.zeros((n, d_out), np.float64)
+    for (indptr, indices), w in zip(graphs, weights):
+        indptr, indices, w = _i64(indptr), _i32(indices), np.asarray(w, np.float64)
+        for i in range(n):
+            nb = indices[indptr[i]:indptr[i + 1]]
+            if nb.shape[0]:
+                z[i] += (h[nb] @ w).sum(axis=0) / nb.shape[0]
+    return z
+
+
+def rgcn_layer_bwd(graphs, h, weights, gz):
+    """(dh, [dW_r]) for the upstream gradient gz of rgcn_layer's result: edge by edge,
+    dW_r += h_j^T gz_i / |N^r_i| and dh_j += gz_i W_r^T / |N^r_i|."""
+    h, gz = np.asarray(h, np.float64), np.asarray(gz, np.float64)
+    dh = np.zeros_like(h)
+    dws = []
+    for (indptr, indices), w in zip(graphs, weights):
+        indptr, indices, w = _i64(indptr), _i32(indices), np.asarray(w, np.float64)
+        dw = np.zeros_like(w)
+        back = gz @ w.T
+        for i in range(indptr.shape[0] - 1):
+            nb = indices[indptr[i]:indptr[i + 1]]
+            if nb.shape[0]:
+                c = 1.0 / nb.shape[0]
+                dw += c * np.outer(h[nb].sum(axis=0), gz[i])
+                np.add.at(dh, nb, c * back[i])
+        dws.append(dw)
+    return dh, dws
+
+
+def rgcn_basis(a, V):
+    """W_r = sum_b a[r,b] V_b (the appendix's second equation); a [R,B], V [B, ...]."""
+    a, V = np.asarray(a, np.float64), np.asarray(V, np.float64)
+    W = np.zeros((a.shape[0],) + V.shape[1:], np.float64)
+    for r in range(a.shape[0]):
+        for b in range(a.shape[1]):
+            W[r] += a[r, b] * V[b]
+    return W
+
+
+def rgcn_basis_bwd(a, V, dW):
+    """(da, dV) for the upstream gradient dW [R, ...] of rgcn_basis's result."""
+    a, V, dW = np.asarray(a, np.float64), np.asarray(V, np.float64), np.asarray(dW, np.float64)
+    da = np.zeros_like(a)
+    dV = np.zeros_like(V)
+    for r in range(a.shape[0]):
+        for b in range(a.shape[1]):
+            da[r, b] = float((dW[r] * V[b]).sum())
+            dV[b] += a[r, b] * dW[r]
+    return da, dV

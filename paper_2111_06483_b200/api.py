@@ -357,3 +357,81 @@ def full_layer_backward(g: Graph, h: torch.Tensor, W: torch.Tensor, a_l: torch.T
     if relu_input:
         B.sar_relu_bwd(h, dh)
     return dh, dW, da_l, da_r
+
+
+# ----------------------------------------------------------------------------------------------
+# relational layer (Appendix A): z_i = sum_r (1/|N^r_i|) sum_{j in N^r_i} h_j W_r, one Graph per relation.
+# Per relation the mean aggregate of h is built partition by partition and multiplied by W_r into z; the
+# backward pass rebuilds the aggregate from h instead of keeping R of them.  Marshalling only.
+
+def rgcn_inv_degrees(graphs: List[Graph]) -> List[torch.Tensor]:
+    """Per relation the factor 1/|N^r_i| of every node (0 without in-edges), float32 [n]."""
+    out = []
+    for g in graphs:
+        inv = torch.empty(g.n, dtype=torch.float32, device=g.whole.indptr.device)
+        B.sar_degree_scale(g.whole.indptr, -1.0, inv)
+        out.append(inv)
+    return out
+
+
+def _pieces(g: Graph):
+    return (g.parts, g.bounds) if g.parts else ([g.whole], [0, g.n])
+
+
+def _rgcn_aggregate(g: Graph, h: torch.Tensor, inv: torch.Tensor, agg: torch.Tensor) -> None:
+    parts, bounds = _pieces(g)
+    for q, part in enumerate(parts):
+        flags = (B.SAR_FIRST if q == 0 else 0) | (B.SAR_LAST if q == len(parts) - 1 else 0)
+        ws = _workspace(B.sar_spmm_workspace_bytes(part, h.shape[1], B._dtype(h)), h.device)
+        B.sar_spmm_agg_scaled(part, h[bounds[q]:bounds[q + 1]], h.shape[1], flags, None, inv, agg, ws)
+
+
+def rgcn_layer_forward(graphs: List[Graph], h: torch.Tensor, W: torch.Tensor, inv: Optional[List[torch.Tensor]] = None):
+    """h [n, d_in] bf16, W [R, d_in, d_out] bf16.  Returns (z [n, d_out] before the activation, inv)."""
+    n, d_in = h.shape
+    d_out = W.shape[2]
+    inv = inv if inv is not None else rgcn_inv_degrees(graphs)
+    agg = torch.empty_like(h)
+    z = torch.empty((n, d_out), dtype=h.dtype, device=h.device)
+    ws = _workspace(B.sar_linear_workspace_bytes(n, d_in, d_out), h.device)
+    for r, g in enumerate(graphs):
+        _rgcn_aggregate(g, h, inv[r], agg)
+        (B.sar_linear if r == 0 else B.sar_linear_accumulate)(agg, W[r], z, ws)
+    return z, inv
+
+
+def rgcn_layer_backward(graphs: List[Graph], h: torch.Tensor, W: torch.Tensor, inv: List[torch.Tensor], gz: torch.Tensor):
+    """Returns (dh [n, d_in], dW [R, d_in, d_out] float32) for the upstream gradient gz [n, d_out]."""
+    n, d_in = h.shape
+    d_out = W.shape[2]
+    agg = torch.empty_like(h)
+    dagg = torch.empty_like(h)
+    dh = torch.empty_like(h)
+    dW = torch.empty((len(graphs), d_in, d_out), dtype=torch.float32, device=h.device)
+    ws = _workspace(B.sar_linear_workspace_bytes(n, d_in, d_out), h.device)
+    for r, g in enumerate(graphs):
+        _rgcn_aggregate(g, h, inv[r], agg)  # rebuilt from the input features
+        B.sar_linear_bwd_weight(agg, gz, dW[r], ws)
+        B.sar_linear_bwd_input(gz, W[r], dagg, ws)
+        parts, bounds = _pieces(g)
+        for q, part in enumerate(parts):  # the partition's sources receive from all destinations
+            tp = part.transposed()
+            sws = _workspace(B.sar_spmm_workspace_bytes(tp, d_in, B._dtype(h)), h.device)
+            B.sar_spmm_agg_scaled(tp, dagg, d_in, (B.SAR_FIRST if r == 0 else 0) | B.SAR_LAST, inv[r], None,
+                                  dh[bounds[q]:bounds[q + 1]], sws)
+    return dh, dW
+
+
+def rgcn_basis_weights(a: torch.Tensor, V: torch.Tensor, dtype: torch.dtype = torch.bfloat16) -> torch.Tensor:
+    """W [R, d_in, d_out] = sum_b a[r,b] V[b] from a [R,B] and V [B, d_in, d_out] (float32)."""
+    W = torch.empty((a.shape[0],) + tuple(V.shape[1:]), dtype=dtype, device=V.device)
+    B.sar_rgcn_basis(a, V, W)
+    return W
+
+
+def rgcn_basis_backward(a: torch.Tensor, V: torch.Tensor, dW: torch.Tensor):
+    """(da [R,B], dV like V) from dW [R, d_in, d_out] float32."""
+    da = torch.empty_like(a)
+    dV = torch.empty_like(V)
+    B.sar_rgcn_basis_bwd(a, V, dW, da, dV)
+    return da, dV

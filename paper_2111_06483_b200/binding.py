@@ -32,7 +32,7 @@ EXPORTS = [
     "sar_mfg_frontier", "sar_csr_filter_rows_indptr", "sar_csr_filter_rows_indices", "sar_spmm_agg_scaled",
     "sar_gat_stack_host_wait", "sar_bn_workspace_bytes", "sar_bn_stats", "sar_bn_apply", "sar_bn_bwd_stats",
     "sar_bn_bwd_apply", "sar_dropout", "sar_linear_workspace_bytes", "sar_linear", "sar_linear_bwd_input",
-    "sar_linear_bwd_weight",
+    "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd",
 ]
 
 
@@ -525,6 +525,35 @@ def sar_linear(h: torch.Tensor, w: torch.Tensor, z: torch.Tensor, workspace: tor
     ws, wb = _ws(workspace)
     _check("sar_linear", lib().sar_linear(c_int64(n), c_int32(d_in), c_int32(d_out), ctypes.c_int(_dtype(h)), _ptr(h),
                                           _ptr(w), _ptr(z), ws, wb, _stream()))
+
+
+def sar_linear_accumulate(h: torch.Tensor, w: torch.Tensor, z: torch.Tensor, workspace: torch.Tensor) -> None:
+    n, d_in = h.shape
+    d_out = w.shape[1]
+    ws, wb = _ws(workspace)
+    _check("sar_linear_accumulate", lib().sar_linear_accumulate(c_int64(n), c_int32(d_in), c_int32(d_out),
+                                                                ctypes.c_int(_dtype(h)), _ptr(h), _ptr(w), _ptr(z), ws,
+                                                                wb, _stream()))
+
+
+def sar_degree_scale(indptr: torch.Tensor, power: float, scale: torch.Tensor) -> None:
+    _check("sar_degree_scale", lib().sar_degree_scale(c_int64(indptr.numel() - 1), _ptr(indptr), c_float(power),
+                                                      _ptr(scale), _stream()))
+
+
+def sar_rgcn_basis(a: torch.Tensor, V: torch.Tensor, W: torch.Tensor) -> None:
+    """a [R,B], V [B,...] float32; W [R,...] bf16 or float32."""
+    R, Bn = a.shape
+    size = V.numel() // Bn
+    _check("sar_rgcn_basis", lib().sar_rgcn_basis(c_int32(R), c_int32(Bn), c_int64(size), ctypes.c_int(_dtype(W)),
+                                                  _ptr(a), _ptr(V), _ptr(W), _stream()))
+
+
+def sar_rgcn_basis_bwd(a: torch.Tensor, V: torch.Tensor, dW: torch.Tensor, da: torch.Tensor, dV: torch.Tensor) -> None:
+    R, Bn = a.shape
+    size = V.numel() // Bn
+    _check("sar_rgcn_basis_bwd", lib().sar_rgcn_basis_bwd(c_int32(R), c_int32(Bn), c_int64(size), _ptr(a), _ptr(V),
+                                                          _ptr(dW), _ptr(da), _ptr(dV), _stream()))
 
 
 def sar_linear_bwd_input(dz: torch.Tensor, w: torch.Tensor, dh: torch.Tensor, workspace: torch.Tensor) -> None:

@@ -18,7 +18,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(CSRC, "build")
 LIB = os.path.join(PKG, "libsar.so")
-SOURCES = ["sar_gat.cu", "sar_graph.cu", "sar_host.cu", "sar_noalloc.cu", "sar_glue.cu", "sar_norm.cu", "sar_linear.cu"]
+SOURCES = ["sar_gat.cu", "sar_graph.cu", "sar_host.cu", "sar_noalloc.cu", "sar_glue.cu", "sar_norm.cu", "sar_linear.cu", "sar_rgcn.cu"]
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr",

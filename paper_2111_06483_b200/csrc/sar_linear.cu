@@ -43,13 +43,13 @@ struct LinearGemm {
     using StrideC = typename Kernel::StrideC;
     using StrideD = typename Kernel::StrideD;
 
-    static typename Gemm::Arguments arguments(int M, int N, int K, const void *a, const void *b, void *d) {
+    static typename Gemm::Arguments arguments(int M, int N, int K, const void *a, const void *b, void *d, float beta = 0.f) {
         typename Gemm::Arguments args{
             cutlass::gemm::GemmUniversalMode::kGemm,
             {M, N, K, 1},
             {static_cast<const ElementA *>(a), cutlass::make_cute_packed_stride(StrideA{}, cute::make_shape(M, K, 1)),
              static_cast<const ElementB *>(b), cutlass::make_cute_packed_stride(StrideB{}, cute::make_shape(N, K, 1))},
-            {{1.f, 0.f},
+            {{1.f, beta},  // D = A B + beta D: with beta = 0 the epilogue does not read D
              static_cast<const ElementOut *>(d), cutlass::make_cute_packed_stride(StrideC{}, cute::make_shape(M, N, 1)),
              static_cast<ElementOut *>(d), cutlass::make_cute_packed_stride(StrideD{}, cute::make_shape(M, N, 1))}};
         return args;
@@ -60,8 +60,8 @@ struct LinearGemm {
     }
 
     static sar_status run(int M, int N, int K, const void *a, const void *b, void *d, void *workspace, size_t workspace_bytes_,
-                          cudaStream_t st, const char *name) {
-        auto args = arguments(M, N, K, a, b, d);
+                          cudaStream_t st, const char *name, float beta = 0.f) {
+        auto args = arguments(M, N, K, a, b, d, beta);
         Gemm gemm;
         if (gemm.can_implement(args) != cutlass::Status::kSuccess) return SAR_ERR_UNSUPPORTED;
         const size_t need = Gemm::get_workspace_size(args);
@@ -117,6 +117,14 @@ sar_status sar_linear(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const
     SAR_TRY(linear_check(n, d_in, d_out, t, {h, w, z}));
     return GemmForward::run((int)n, d_out, d_in, h, w, z, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
                             "linear");
+}
+
+sar_status sar_linear_accumulate(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *h, const void *w, void *z,
+                                 void *workspace, size_t workspace_bytes, void *stream) {
+    if (n == 0 && d_in > 0 && d_out > 0) return t == SAR_BF16 ? SAR_OK : SAR_ERR_UNSUPPORTED;
+    SAR_TRY(linear_check(n, d_in, d_out, t, {h, w, z}));
+    return GemmForward::run((int)n, d_out, d_in, h, w, z, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
+                            "linear_accumulate", 1.f);
 }
 
 sar_status sar_linear_bwd_input(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *dz, const void *w,
