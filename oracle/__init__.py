@@ -496,3 +496,34 @@ def rgcn_basis_bwd(a, V, dW):
             da[r, b] = float((dW[r] * V[b]).sum())
             dV[b] += a[r, b] * dW[r]
     return da, dV
+
+
+# --------------------------------------------------------------------------------------
+# GraphSage layer (Eq. 2), plain numpy float64 in the equation's order: project every
+# node (z = h W), average the neighbours' z, add the residual term h W_res
+# --------------------------------------------------------------------------------------
+
+def sage_layer(indptr, indices, h, w, w_res):
+    """pre[i,:] = h[i,:] W_res + (1/|N(i)|) sum_{j in N(i)} (h W)[j,:]  (the argument of sigma in Eq. 2;
+    the mean of an empty neighbourhood is 0)."""
+    h, w, w_res = (np.asarray(x, np.float64) for x in (h, w, w_res))
+    indptr, indices = _i64(indptr), _i32(indices)
+    z = h @ w
+    pre = h @ w_res
+    for i in range(indptr.shape[0] - 1):
+        nb = indices[indptr[i]:indptr[i + 1]]
+        if nb.shape[0]:
+            pre[i] += z[nb].sum(axis=0) / nb.shape[0]
+    return pre
+
+
+def sage_layer_bwd(indptr, indices, h, w, w_res, g):
+    """(dh, dW, dW_res) for the upstream gradient g of sage_layer's result."""
+    h, w, w_res, g = (np.asarray(x, np.float64) for x in (h, w, w_res, g))
+    indptr, indices = _i64(indptr), _i32(indices)
+    dz = np.zeros((h.shape[0], w.shape[1]), np.float64)  # gradient of z = h W: every in-edge hands back g_i / |N(i)|
+    for i in range(indptr.shape[0] - 1):
+        nb = indices[indptr[i]:indptr[i + 1]]
+        if nb.shape[0]:
+            np.add.at(dz, nb, g[i] / nb.shape[0])
+    return g @ w_res.T + dz @ w.T, h.T @ dz, h.T @ g

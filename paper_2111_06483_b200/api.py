@@ -435,3 +435,46 @@ def rgcn_basis_backward(a: torch.Tensor, V: torch.Tensor, dW: torch.Tensor):
     dV = torch.empty_like(V)
     B.sar_rgcn_basis_bwd(a, V, dW, da, dV)
     return da, dV
+
+
+# ----------------------------------------------------------------------------------------------
+# GraphSage layer (Eq. 2): pre_i = h_i W_res + mean_{j in N(i)} h_j W.  The mean commutes with W, so the
+# neighbours' raw features are averaged first (one aggregation of d_in columns) and the two projections
+# accumulate into one output.  The aggregation has no parameters ("case 1" of Sec. 3.2): the backward pass
+# needs no source features, only the graph.  Marshalling only.
+
+def sage_layer_forward(g: Graph, h: torch.Tensor, W: torch.Tensor, W_res: torch.Tensor, inv: Optional[torch.Tensor] = None):
+    """h [n, d_in], W and W_res [d_in, d_out] (bf16).  Returns (pre [n, d_out] before the activation, saved)."""
+    n, d_in = h.shape
+    d_out = W.shape[1]
+    if inv is None:
+        inv = rgcn_inv_degrees([g])[0]
+    agg = torch.empty_like(h)
+    _rgcn_aggregate(g, h, inv, agg)
+    pre = torch.empty((n, d_out), dtype=h.dtype, device=h.device)
+    ws = _workspace(B.sar_linear_workspace_bytes(n, d_in, d_out), h.device)
+    B.sar_linear(h, W_res, pre, ws)
+    B.sar_linear_accumulate(agg, W, pre, ws)
+    return pre, (agg, inv)
+
+
+def sage_layer_backward(g: Graph, h: torch.Tensor, W: torch.Tensor, W_res: torch.Tensor, saved, gpre: torch.Tensor):
+    """Returns (dh [n, d_in], dW, dW_res [d_in, d_out] float32) for the upstream gradient gpre [n, d_out]."""
+    n, d_in = h.shape
+    d_out = W.shape[1]
+    agg, inv = saved
+    ws = _workspace(B.sar_linear_workspace_bytes(n, d_in, d_out), h.device)
+    dW = torch.empty((d_in, d_out), dtype=torch.float32, device=h.device)
+    dW_res = torch.empty_like(dW)
+    B.sar_linear_bwd_weight(agg, gpre, dW, ws)
+    B.sar_linear_bwd_weight(h, gpre, dW_res, ws)
+    dh = torch.empty_like(h)
+    B.sar_linear_bwd_input(gpre, W_res, dh, ws)       # the residual path
+    dagg = torch.empty_like(h)
+    B.sar_linear_bwd_input(gpre, W, dagg, ws)
+    parts, bounds = _pieces(g)
+    for q, part in enumerate(parts):                  # plus what every out-edge hands back: dagg_i / |N(i)|
+        tp = part.transposed()
+        sws = _workspace(B.sar_spmm_workspace_bytes(tp, d_in, B._dtype(h)), h.device)
+        B.sar_spmm_agg_scaled(tp, dagg, d_in, B.SAR_LAST, inv, None, dh[bounds[q]:bounds[q + 1]], sws)
+    return dh, dW, dW_res
