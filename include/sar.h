@@ -319,6 +319,10 @@ SAR_API sar_status sar_relu(int64_t n_elems, sar_dtype t, void *x, void *stream)
 SAR_API sar_status sar_dropout(int64_t n_elems, sar_dtype t, const void *x, float p, uint64_t seed, void *y,
                                void *stream);
 SAR_API sar_status sar_relu_bwd(int64_t n_elems, sar_dtype t, const void *y, void *g, void *stream);
+/* y = a*x + b*y element-wise (float32 arithmetic; x, y of type t, n_elems each, DEVICE memory, x != y): the mixing
+ * step of an iterated propagation X <- (1-alpha) X0 + alpha S X (Sec. 4.2: label-propagation post-processing), whose
+ * product S X is sar_spmm_agg_scaled. */
+SAR_API sar_status sar_axpby(int64_t n_elems, sar_dtype t, float a, const void *x, float b, void *y, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * The dense projection of a layer, z = h W (Eq. 1 / Eq. 3 apply a weight matrix to every node's features

@@ -527,3 +527,13 @@ def sage_layer_bwd(indptr, indices, h, w, w_res, g):
         if nb.shape[0]:
             np.add.at(dz, nb, g[i] / nb.shape[0])
     return g @ w_res.T + dz @ w.T, h.T @ dz, h.T @ g
+
+
+def propagate(indptr, indices, x0, alpha: float, iters: int, src_scale=None, dst_scale=None):
+    """X_iters of the iteration X_0 = x0, X_{t+1} = (1 - alpha) x0 + alpha S X_t with S = diag(dst_scale) A
+    diag(src_scale) (the propagation of Sec. 4.2's label post-processing), float64."""
+    x0 = np.asarray(x0, np.float64)
+    x = x0.copy()
+    for _ in range(iters):
+        x = (1.0 - alpha) * x0 + alpha * spmm_scaled(indptr, indices, x, src_scale, dst_scale)
+    return x

@@ -478,3 +478,35 @@ def sage_layer_backward(g: Graph, h: torch.Tensor, W: torch.Tensor, W_res: torch
         sws = _workspace(B.sar_spmm_workspace_bytes(tp, d_in, B._dtype(h)), h.device)
         B.sar_spmm_agg_scaled(tp, dagg, d_in, B.SAR_LAST, inv, None, dh[bounds[q]:bounds[q + 1]], sws)
     return dh, dW, dW_res
+
+
+# ----------------------------------------------------------------------------------------------
+# iterated propagation X <- (1 - alpha) X0 + alpha S X with S = diag(dst_scale) A diag(src_scale): the smoothing /
+# error-correction steps of the label-propagation post-processing the paper combines SAR with (Sec. 4.2).
+
+def sym_norm_scales(g: Graph):
+    """(src_scale, dst_scale) = (out-degree^-1/2, in-degree^-1/2), the symmetric normalisation (0 for degree 0)."""
+    dev = g.whole.indptr.device
+    dst = torch.empty(g.n, dtype=torch.float32, device=dev)
+    src = torch.empty(g.n, dtype=torch.float32, device=dev)
+    B.sar_degree_scale(g.whole.indptr, -0.5, dst)
+    B.sar_degree_scale(g.whole.t_indptr, -0.5, src)
+    return src, dst
+
+
+def propagate(g: Graph, x0: torch.Tensor, alpha: float, iters: int, src_scale: Optional[torch.Tensor] = None,
+              dst_scale: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Returns X_iters with X_0 = x0 and X_{t+1} = (1 - alpha) x0 + alpha S X_t; x0 [n, F]."""
+    x = x0.clone()
+    nxt = torch.empty_like(x0)
+    parts, bounds = _pieces(g)
+    F = x0.shape[1]
+    for _ in range(iters):
+        for q, part in enumerate(parts):
+            flags = (B.SAR_FIRST if q == 0 else 0) | (B.SAR_LAST if q == len(parts) - 1 else 0)
+            ws = _workspace(B.sar_spmm_workspace_bytes(part, F, B._dtype(x0)), x0.device)
+            sq = None if src_scale is None else src_scale[bounds[q]:bounds[q + 1]]
+            B.sar_spmm_agg_scaled(part, x[bounds[q]:bounds[q + 1]], F, flags, sq, dst_scale, nxt, ws)
+        B.sar_axpby(1.0 - alpha, x0, alpha, nxt)
+        x, nxt = nxt, x
+    return x

@@ -32,7 +32,7 @@ EXPORTS = [
     "sar_mfg_frontier", "sar_csr_filter_rows_indptr", "sar_csr_filter_rows_indices", "sar_spmm_agg_scaled",
     "sar_gat_stack_host_wait", "sar_bn_workspace_bytes", "sar_bn_stats", "sar_bn_apply", "sar_bn_bwd_stats",
     "sar_bn_bwd_apply", "sar_dropout", "sar_linear_workspace_bytes", "sar_linear", "sar_linear_bwd_input",
-    "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd",
+    "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd", "sar_axpby",
 ]
 
 
@@ -577,6 +577,13 @@ def sar_linear_bwd_weight(h: torch.Tensor, dz: torch.Tensor, dw: torch.Tensor, w
 def sar_dropout(x: torch.Tensor, p: float, seed: int, y: torch.Tensor) -> None:
     _check("sar_dropout", lib().sar_dropout(c_int64(x.numel()), ctypes.c_int(_dtype(x)), _ptr(x), c_float(p),
                                             ctypes.c_uint64(seed & 0xFFFFFFFFFFFFFFFF), _ptr(y), _stream()))
+
+
+def sar_axpby(a: float, x: torch.Tensor, b: float, y: torch.Tensor) -> None:
+    """y = a*x + b*y."""
+    assert x.numel() == y.numel() and x.dtype == y.dtype
+    _check("sar_axpby", lib().sar_axpby(c_int64(x.numel()), ctypes.c_int(_dtype(x)), c_float(a), _ptr(x), c_float(b),
+                                        _ptr(y), _stream()))
 
 
 def sar_relu_bwd(y: torch.Tensor, g: torch.Tensor) -> None:

@@ -267,6 +267,25 @@ static sar_status launch_relu(const char *name, int64_t n, const void *y, void *
 }
 
 
+// y = a*x + b*y, element-wise in float32 (the mixing step X <- (1-alpha) X0 + alpha S X of a propagation, Sec. 4.2)
+template <typename T>
+__global__ void axpby_kernel(long long n, float ca, const T *x, float cb, T *y, long long n_vec16) {
+    constexpr int EPV = Elem<T>::EPV;
+    const long long tid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long nthreads = (long long)gridDim.x * blockDim.x;
+    for (long long i = tid; i < n_vec16; i += nthreads) {
+        uint4 *yp = reinterpret_cast<uint4 *>(y) + i;
+        float xv[EPV], yv[EPV];
+        Elem<T>::unpack(__ldg(reinterpret_cast<const uint4 *>(x) + i), xv);
+        Elem<T>::unpack(*yp, yv);
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) yv[e] = fmaf(ca, xv[e], cb * yv[e]);
+        *yp = Elem<T>::pack(yv);
+    }
+    for (long long i = n_vec16 * EPV + tid; i < n; i += nthreads)
+        Elem<T>::store1(y + i, fmaf(ca, as_float(x[i]), cb * as_float(y[i])));
+}
+
 // ---- dropout (the paper's networks use batch normalisation and dropout between all layers, Sec. 4.2) ------
 // Counter-based: element i is kept when the top 24 bits of SplitMix64's (i+1)-th output for `seed` reach
 // p * 2^24; nothing is stored, the backward pass draws the same mask again from the seed.
@@ -445,6 +464,25 @@ sar_status sar_dropout(int64_t n_elems, sar_dtype t, const void *x, float p, uin
         SAR_LAUNCH("dropout", st, (dropout_kernel<float><<<(unsigned)blocks, 256, 0, st>>>(n_elems, static_cast<const float *>(x), static_cast<float *>(y), threshold, scale, seed, n_vec16)));
     else
         SAR_LAUNCH("dropout", st, (dropout_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, st>>>(n_elems, static_cast<const __nv_bfloat16 *>(x), static_cast<__nv_bfloat16 *>(y), threshold, scale, seed, n_vec16)));
+    return sar_after_launch();
+}
+
+sar_status sar_axpby(int64_t n_elems, sar_dtype t, float a, const void *x, float b, void *y, void *stream) {
+    if (n_elems < 0 || (n_elems > 0 && (!x || !y))) return SAR_ERR_INVALID_ARG;
+    if (t != SAR_F32 && t != SAR_BF16) return SAR_ERR_INVALID_ARG;
+    if (x == y) return SAR_ERR_INVALID_ARG;
+    SAR_TRY(check_elem_align({x, y}, sar_elem_size(t)));
+    if (n_elems == 0) return SAR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool vec = sar_aligned(x, 16) && sar_aligned(y, 16);
+    const long long n_vec16 = vec ? n_elems / (t == SAR_F32 ? 4 : 8) : 0;
+    const long long work = n_vec16 > 0 ? n_vec16 : n_elems;
+    long long blocks = (work + 255) / 256;
+    if (blocks > 148 * 64) blocks = 148 * 64;
+    if (t == SAR_F32)
+        SAR_LAUNCH("axpby", st, (axpby_kernel<float><<<(unsigned)blocks, 256, 0, st>>>(n_elems, a, static_cast<const float *>(x), b, static_cast<float *>(y), n_vec16)));
+    else
+        SAR_LAUNCH("axpby", st, (axpby_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, st>>>(n_elems, a, static_cast<const __nv_bfloat16 *>(x), b, static_cast<__nv_bfloat16 *>(y), n_vec16)));
     return sar_after_launch();
 }
 

@@ -6,7 +6,7 @@ import torch
 
 import oracle
 import workloads
-from helpers import allclose_report
+from helpers import allclose_report, small_problem
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -75,3 +75,47 @@ def test_weighted_sum_rejects_the_mean_flag_and_accepts_no_scales():
     # without scales it is the plain sum, bit for bit
     B.sar_spmm_agg_scaled(g.whole, x, 16, B.SAR_FIRST | B.SAR_LAST, None, None, out, ws)
     assert torch.equal(out, api.spmm_sum(g.whole, x))
+
+
+@pytest.mark.parametrize("n,dtype", [(1, "f32"), (1000, "f32"), (4099, "bf16"), (1 << 20, "bf16"), ((1 << 20) + 3, "f32")])
+def test_axpby(n, dtype):
+    from paper_2111_06483_b200 import binding as B
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    rng = np.random.default_rng(n)
+    x = torch.from_numpy(rng.standard_normal(n).astype(np.float32)).to(tdt).to(DEV)
+    y = torch.from_numpy(rng.standard_normal(n).astype(np.float32)).to(tdt).to(DEV)
+    want = 0.25 * x.double().cpu().numpy() - 1.5 * y.double().cpu().numpy()
+    B.sar_axpby(0.25, x, -1.5, y)
+    tol = dict(rtol=1e-6, atol=1e-6) if dtype == "f32" else dict(rtol=2.0 ** -8, atol=2.0 ** -8)
+    allclose_report(y.double().cpu().numpy(), want, what="a x + b y", **tol)
+    # an unaligned view takes the element-wise path
+    if n > 8:
+        xs, ys = x[1:], y[1:]
+        want = 2.0 * xs.double().cpu().numpy() + 0.5 * ys.double().cpu().numpy()
+        B.sar_axpby(2.0, xs, 0.5, ys)
+        allclose_report(ys.double().cpu().numpy(), want, what="a x + b y, unaligned", **tol)
+    with pytest.raises(B.SarError):
+        B.sar_axpby(1.0, y, 1.0, y)
+
+
+@pytest.mark.parametrize("dtype,k", [("f32", 1), ("f32", 3), ("bf16", 1), ("bf16", 4)])
+def test_iterated_propagation(dtype, k):
+    from paper_2111_06483_b200 import api
+    n, e, F, alpha, iters = 3000, 20000, 24, 0.8, 6
+    tdt = torch.float32 if dtype == "f32" else torch.bfloat16
+    p = small_problem(n, e, 1, 4, 77)
+    src = np.concatenate([p["src"], p["dst"]]).astype(np.int32)   # undirected: every edge in both directions
+    dst = np.concatenate([p["dst"], p["src"]]).astype(np.int32)
+    indptr, indices = oracle.csr_from_coo(n, n, src, dst)
+    g = api.Graph.from_coo(n, torch.from_numpy(src).to(DEV), torch.from_numpy(dst).to(DEV), k=k, build_parts=k > 1)
+    s_src, s_dst = api.sym_norm_scales(g)
+    deg = np.diff(indptr).astype(np.float64)
+    want_scale = np.where(deg > 0, 1.0 / np.sqrt(np.maximum(deg, 1)), 0.0)
+    allclose_report(s_dst.cpu().numpy().astype(np.float64), want_scale, 1e-6, 0.0, "in-degree^-1/2")
+    allclose_report(s_src.cpu().numpy().astype(np.float64), want_scale, 1e-6, 0.0, "out-degree^-1/2")
+    x0 = torch.from_numpy(np.random.default_rng(4).standard_normal((n, F)).astype(np.float32)).to(tdt)
+    got = api.propagate(g, x0.to(DEV), alpha, iters, s_src, s_dst)
+    want = oracle.propagate(indptr, indices, x0.float().numpy(), alpha, iters,
+                            s_src.cpu().numpy(), s_dst.cpu().numpy())
+    tol = dict(rtol=1e-5, atol=1e-5) if dtype == "f32" else dict(rtol=2e-2, atol=2e-2)  # bf16: two roundings per step
+    allclose_report(got.float().cpu().numpy(), want, what=f"{iters} propagation steps", **tol)

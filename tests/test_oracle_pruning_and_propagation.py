@@ -98,3 +98,29 @@ def test_scaled_sum_is_the_sparse_matrix_product():
     s = np.where(deg > 0, 1.0 / np.sqrt(np.maximum(deg, 1)), 0.0)
     v = np.sqrt(deg)[:, None]
     assert np.allclose(oracle.spmm_scaled(ptr, idx, v, s, s), v, rtol=1e-12, atol=1e-12)
+
+
+def _undirected(n, e, seed):
+    p = small_problem(n, e, 1, 4, seed)
+    src = np.concatenate([p["src"], p["dst"]]).astype(np.int32)
+    dst = np.concatenate([p["dst"], p["src"]]).astype(np.int32)
+    indptr, indices = oracle.csr_from_coo(n, n, src, dst)
+    A = count_matrix(n, n, src, dst)
+    deg = A.sum(axis=1)
+    inv_sqrt = np.where(deg > 0, 1.0 / np.sqrt(np.maximum(deg, 1)), 0.0)
+    return indptr, indices, A, inv_sqrt
+
+
+def test_iterated_propagation_steps_and_fixed_point():
+    n, alpha = 45, 0.8
+    indptr, indices, A, s = _undirected(n, 120, 13)
+    S = s[:, None] * A * s[None, :]
+    x0 = np.random.default_rng(3).standard_normal((n, 3))
+    assert np.array_equal(oracle.propagate(indptr, indices, x0, alpha, 0, s, s), x0)
+    one = oracle.propagate(indptr, indices, x0, alpha, 1, s, s)
+    assert np.allclose(one, (1 - alpha) * x0 + alpha * S @ x0, rtol=1e-13, atol=1e-13)
+    two = oracle.propagate(indptr, indices, x0, alpha, 2, s, s)
+    assert np.allclose(two, (1 - alpha) * x0 + alpha * S @ one, rtol=1e-13, atol=1e-13)
+    # the eigenvalues of the symmetric normalisation lie in [-1, 1]: the iteration converges to (1-a)(I - aS)^-1 x0
+    limit = np.linalg.solve(np.eye(n) - alpha * S, (1 - alpha) * x0)
+    assert np.allclose(oracle.propagate(indptr, indices, x0, alpha, 300, s, s), limit, rtol=1e-10, atol=1e-10)
