@@ -177,7 +177,7 @@ class ShardedGatLayer:
                 got = returning.wait()
                 dfeat_acc += got[0].to(wide)
                 der_acc += got[1]
-                returning = None
+                returning = got = None  # the receive buffer is released before the next one is posted
             if s == 0:
                 dfeat_acc, der_acc = dfeat_q.to(wide, copy=True), der_q.clone()
             else:
