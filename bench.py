@@ -49,6 +49,9 @@ def parse_args():
     ap.add_argument("--ids", default="permuted", choices=["permuted", "degree_sorted"],
                     help="node numbering of the power-law graph: seeded random permutation (the workload) or "
                          "degree rank = id (locality ablation)")
+    ap.add_argument("--spmm", action="store_true",
+                    help="time the sum aggregation (sar_spmm_agg forward + its backward on the transposed graph) "
+                         "on the workload's graph instead of the attention stack; its own metric, not the headline")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample", type=float, default=0.05, help="fraction of the workload the oracle is timed on")
@@ -481,6 +484,70 @@ def run_ours(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def run_spmm(args, local_rank):
+    """--spmm: one step = out = A x (CSR) and dx = A^T gout (the same call on the transposed partition), Eq. 2's
+    aggregation with F columns per node.  One GPU; prints its own JSON line (metric spmm_fwd_bwd_edges_per_sec)."""
+    import torch
+    import workloads
+    from paper_2111_06483_b200 import api, binding as B
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    dev = torch.device(f"cuda:{local_rank}")
+    torch.cuda.set_device(dev)
+    cfg = workloads.CONFIGS[args.workload]
+    if args.scale != 1.0:
+        cfg = cfg.scaled(args.scale)
+    dtype = args.dtype or cfg.dtypes[-1]
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    b = 2 if dtype == "bf16" else 4
+    n, F = cfg.n, cfg.spmm_feat or cfg.heads * cfg.feat
+    threshold = args.threshold if args.threshold is not None else api.DEFAULT_THRESHOLD
+    src, dst = workloads.make_graph(cfg, device=dev, permute=args.ids == "permuted")
+    e = src.numel()
+    g = api.Graph.from_coo(n, src, dst, k=1, threshold=threshold)
+    del src, dst
+    x = workloads.normal_tensor((n, F), cfg.seed, 20, device=dev, dtype=tdt)
+    gout = workloads.normal_tensor((n, F), cfg.seed, 21, device=dev, dtype=tdt)
+    out, dx = torch.empty_like(x), torch.empty_like(x)
+    fwd, bwd = g.whole, g.whole.transposed()
+    ws = torch.empty(max(B.sar_spmm_workspace_bytes(fwd, F, B._dtype(x)), B.sar_spmm_workspace_bytes(bwd, F, B._dtype(x))),
+                     dtype=torch.uint8, device=dev)
+
+    def step():
+        B.sar_spmm_agg(fwd, x, F, B.SAR_FIRST | B.SAR_LAST, None, out, ws)
+        B.sar_spmm_agg(bwd, gout, F, B.SAR_FIRST | B.SAR_LAST, None, dx, ws)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with B.LaunchTimer() as lt:
+        e0.record()
+        for _ in range(args.steps):
+            step()
+        e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms_per_step = e0.elapsed_time(e1) / args.steps
+    kernels = lt.summary()
+    peak, peak_src = load_peaks()
+    alg = idx_bytes(n, e) + 2 * n * F * b  # per direction: indices, every input row once, every output row once
+    achieved = 2 * alg / (ms_per_step * 1e-3) / 1e9
+    line = {
+        "metric": "spmm_fwd_bwd_edges_per_sec", "value": e / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": cfg.name, "n": n, "e": e, "columns": F, "storage_dtype": dtype, "ids": args.ids,
+                   "l2": "inputs_exceed_l2" if n * F * b > 126e6 else "inputs_fit_l2", "long_row_threshold": threshold},
+        "roofline": {"bound": "hbm", "kernel": "spmm (forward + transposed)", "achieved": achieved, "peak": peak,
+                     "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
+                     "algorithmic_bytes_per_step": 2 * alg, "gathered_bytes_per_step": 2 * e * F * b},
+        "kernels": kernels, "gpu_launches": sum(v["launches"] for v in kernels.values()), "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     args = parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -488,6 +555,10 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.spmm:
+        if rank == 0:
+            run_spmm(args, local_rank)
         return
     run_ours(args, rank, world, local_rank)
 
