@@ -14,7 +14,11 @@
  *   exp(old_max - new_max) whenever the max moves, and divided at the end.
  *   Backward (Algorithm 2 with the rematerialisation of Sec. 3.3): the attention is rebuilt from
  *   (el, er, m, d) per partition to produce dFeat, dEl and dEr.
- *   Sum aggregation (Eq. 2, "case 1" of Sec. 3.2).
+ *   Sum aggregation (Eq. 2, "case 1" of Sec. 3.2), plain, mean or weighted per edge end.
+ *   Around the aggregation: graph preparation and message-flow pruning (Appendix B), the dense
+ *   projection of a layer and the score projections with their backward passes (Eq. 1, Eq. 3), ReLU,
+ *   dropout and batch normalisation over the nodes (Sec. 3.4, Sec. 4.2), the helpers of the relational
+ *   layer (Appendix A), and a whole-stack entry point on HOST buffers.
  *
  * Conventions
  *   - Every function returns a sar_status; nothing throws, aborts or prints.
@@ -74,7 +78,8 @@ typedef enum { SAR_F32 = 0, SAR_BF16 = 1 } sar_dtype;
 #define SAR_MAX_PARTS 64
 #define SAR_MAX_ROW_BYTES 4096 /* H*F*sizeof(element) handled by the fast kernels             */
 
-/* Optional split of long rows into segments, built once per graph by sar_plan_build.  Rows
+/* Optional split of long rows into segments, built once per graph by sar_plan_count +
+ * sar_plan_fill.  Rows
  * with more than `threshold` edges are cut into segments of at most `threshold` edges that
  * are processed in parallel and merged by a second launch (no atomics).  All arrays DEVICE. */
 typedef struct {

@@ -439,6 +439,10 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
             __syncwarp();
         } else if constexpr (MODE != kSum) {
             const bool vec4 = GEO ? true : a.hvec != 0;  // heads handled four at a time with 16-byte accesses
+            // A segment launch of the four-head geometry stages one row: every position would hit the same four
+            // shared-memory words, so each lane keeps its own maxima and the warp reduces them once per chunk.
+            constexpr bool kLaneMax = kFwdMode && STATIC == 2 && GEO == 1;
+            unsigned kmax[4] = {kKeyNegInf, kKeyNegInf, kKeyNegInf, kKeyNegInf};
             int i = 0;
             for (int q0 = lane; q0 < npos; q0 += 64) {
                 int col[2], rbase[2];
@@ -478,7 +482,8 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                                         op[j] = SAR_NEG_INF;  // padding: weight exp(-inf - max) = 0
                                         if (col[u] >= 0) {
                                             op[j] = leaky(s4[j], a.slope, gr);
-                                            atomicMax(&skey[rb + j], fkey(op[j]));
+                                            if constexpr (kLaneMax) kmax[j] = max(kmax[j], fkey(op[j]));
+                                            else atomicMax(&skey[rb + j], fkey(op[j]));
                                         }
                                     }
                                 } else {
@@ -575,6 +580,13 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                             }
                         }
                     }
+                }
+            }
+            if constexpr (kLaneMax) {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const unsigned k = __reduce_max_sync(0xffffffffu, kmax[j]);
+                    if (lane == 0 && k > skey[j]) skey[j] = k;
                 }
             }
             __syncwarp();
