@@ -49,6 +49,9 @@ def parse_args():
     ap.add_argument("--ids", default="permuted", choices=["permuted", "degree_sorted"],
                     help="node numbering of the power-law graph: seeded random permutation (the workload) or "
                          "degree rank = id (locality ablation)")
+    ap.add_argument("--bn-dropout", action="store_true",
+                    help="with --glue on a bf16 workload: batch normalisation over the nodes and dropout (p = 0.5) "
+                         "between the layers, as in the paper's networks (Sec. 4.2), forward and backward")
     ap.add_argument("--spmm", action="store_true",
                     help="time the sum aggregation (sar_spmm_agg forward + its backward on the transposed graph) "
                          "on the workload's graph instead of the attention stack; its own metric, not the headline")
@@ -310,7 +313,49 @@ def run_ours(args, rank, world, local_rank):
         lws = torch.empty(B.sar_linear_workspace_bytes(n, D, D), dtype=torch.uint8, device=dev)
         flat = lambda x: x.view(n, D)
 
-        def step():
+        bnd = args.bn_dropout
+        if bnd:
+            # layer l's aggregation output stays in feats[l+1] (batch normalisation needs it again in the backward
+            # pass); hs[l+1] = dropout(ReLU(BN(feats[l+1]))) is the next layer's input
+            hs = [feats[0]] + [torch.empty((n, H, F), dtype=tdt, device=dev) for _ in range(L - 1)]
+            bn_mean = [torch.empty(D, dtype=torch.float32, device=dev) for _ in range(L)]
+            bn_m2 = [torch.empty(D, dtype=torch.float32, device=dev) for _ in range(L)]
+            bn_rstd = [torch.empty(D, dtype=torch.float32, device=dev) for _ in range(L)]
+            bn_s0, bn_s1 = torch.empty(D, dtype=torch.float32, device=dev), torch.empty(D, dtype=torch.float32, device=dev)
+            bws = torch.empty(B.sar_bn_workspace_bytes(D), dtype=torch.uint8, device=dev)
+            p_drop, seeds = 0.5, [1000 + l for l in range(L)]
+            gx_bn = torch.empty((n, H, F), dtype=tdt, device=dev)  # gradient w.r.t. a layer's aggregation output
+
+            def step():
+                for l in range(L):
+                    B.sar_linear(flat(hs[l]), Ws[l], flat(zs[l]), lws)
+                    B.sar_gat_project(zs[l], a_ls[l], a_rs[l], els[l], ers[l], 0)
+                    B.sar_gat_fwd_fused(g.whole, g.bounds, z_q[l], els[l], er_q[l], H, F, cfg.slope, ms[l], ds[l],
+                                        feats[l + 1], ws)
+                    if l + 1 < L:
+                        x = flat(feats[l + 1])
+                        B.sar_bn_stats(x, bn_mean[l], bn_m2[l], bws)
+                        torch.rsqrt(bn_m2[l] / n + 1e-5, out=bn_rstd[l])  # C floats: the statistics' last step
+                        B.sar_bn_apply(x, bn_mean[l], bn_rstd[l], None, None, flat(hs[l + 1]))
+                        B.sar_relu(hs[l + 1])
+                        B.sar_dropout(hs[l + 1], p_drop, seeds[l], hs[l + 1])
+                gin = gout
+                for l in reversed(range(L)):
+                    B.sar_gat_bwd_fused(g.whole, g.bounds, z_q[l], els[l], er_q[l], ms[l], ds[l], gin, H, F, cfg.slope,
+                                        gbuf_q[0], dels[l], der_q[l], ws)
+                    B.sar_gat_project_bwd(zs[l], a_ls[l], a_rs[l], dels[l], ders[l], gbuf[0], da_l, da_r, pws, 0)
+                    B.sar_linear_bwd_weight(flat(hs[l]), flat(gbuf[0]), dW, lws)
+                    B.sar_linear_bwd_input(flat(gbuf[0]), Ws[l], flat(gbuf[1]), lws)
+                    if l > 0:
+                        gh = gbuf[1]                                    # gradient w.r.t. hs[l]
+                        B.sar_dropout(gh, p_drop, seeds[l - 1], gh)     # the same mask, drawn again from the seed
+                        B.sar_relu_bwd(hs[l], gh)                       # hs[l] > 0 exactly where the ReLU passed and the mask kept
+                        x = flat(feats[l])
+                        B.sar_bn_bwd_stats(x, bn_mean[l - 1], bn_rstd[l - 1], flat(gh), bn_s0, bn_s1, bws)
+                        B.sar_bn_bwd_apply(x, bn_mean[l - 1], bn_rstd[l - 1], None, flat(gh), bn_s0, bn_s1, 1.0 / n, flat(gx_bn))
+                        gin = gx_bn
+
+        def step_plain():
             for l in range(L):
                 if l > 0:
                     B.sar_relu(feats[l])
@@ -331,6 +376,9 @@ def run_ours(args, rank, world, local_rank):
                 if l > 0:
                     B.sar_relu_bwd(feats[l], gbuf[1])
                 gin = gbuf[1]
+
+        if not bnd:
+            step = step_plain
     else:
         def step():
             for l in range(L):
@@ -467,7 +515,7 @@ def run_ours(args, rank, world, local_rank):
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {
                 "workload": cfg.name, "n": n, "e": e, "heads": H, "feat_per_head": F, "layers": L, "partitions": K,
-                "storage_dtype": dtype, "layer_glue": bool(args.glue), "ids": args.ids, "schedule": "fused row-stationary (sar_gat_fwd_fused / sar_gat_bwd_fused)",
+                "storage_dtype": dtype, "layer_glue": bool(args.glue), "bn_dropout": bool(args.glue and args.bn_dropout), "ids": args.ids, "schedule": "fused row-stationary (sar_gat_fwd_fused / sar_gat_bwd_fused)",
                 "l2": "inputs_exceed_l2", "long_row_threshold": threshold, "parallelism": f"replicas x{world}",
                 "edges_x_heads_x_feat_per_sec": value * H * F,
             },
