@@ -335,7 +335,7 @@ def run_ours(args, rank, world, local_rank):
                     if l + 1 < L:
                         x = flat(feats[l + 1])
                         B.sar_bn_stats(x, bn_mean[l], bn_m2[l], bws)
-                        torch.rsqrt(bn_m2[l] / n + 1e-5, out=bn_rstd[l])  # C floats: the statistics' last step
+                        B.sar_bn_rstd(bn_m2[l], n, 1e-5, bn_rstd[l])
                         B.sar_bn_apply(x, bn_mean[l], bn_rstd[l], None, None, flat(hs[l + 1]))
                         B.sar_relu(hs[l + 1])
                         B.sar_dropout(hs[l + 1], p_drop, seeds[l], hs[l + 1])

@@ -393,6 +393,7 @@ SAR_API sar_status sar_rgcn_basis_bwd(int32_t R, int32_t B, int64_t size, const 
  *                     (two passes, no cancellation).  Workers combine (n, mean, m2) triples by the pairwise
  *                     rule mean = sum n_r mean_r / N, m2 = sum [m2_r + n_r (mean_r - mean)^2]; the variance
  *                     is m2 / N and rstd = 1 / sqrt(variance + eps).
+ *   sar_bn_rstd       rstd[c] = 1 / sqrt(m2[c] / count + eps) from the (global) m2 and row count.
  *   sar_bn_apply      the normalisation with given (global) mean and rstd.
  *   sar_bn_bwd_stats  sum_gy[c] = sum_i gy[i,c] (= d beta) and sum_gy_xhat[c] = sum_i gy[i,c] * xhat[i,c]
  *                     (= d gamma) over the local rows, xhat = (x - mean) * rstd; workers add these up.
@@ -405,6 +406,7 @@ SAR_API sar_status sar_rgcn_basis_bwd(int32_t R, int32_t B, int64_t size, const 
 SAR_API size_t sar_bn_workspace_bytes(int32_t C);
 SAR_API sar_status sar_bn_stats(int64_t n, int32_t C, sar_dtype t, const void *x, float *mean, float *m2,
                                 void *workspace, size_t workspace_bytes, void *stream);
+SAR_API sar_status sar_bn_rstd(int32_t C, const float *m2, int64_t count, float eps, float *rstd, void *stream);
 SAR_API sar_status sar_bn_apply(int64_t n, int32_t C, sar_dtype t, const void *x, const float *mean,
                                 const float *rstd, const float *gamma, const float *beta, void *y, void *stream);
 SAR_API sar_status sar_bn_bwd_stats(int64_t n, int32_t C, sar_dtype t, const void *x, const float *mean,

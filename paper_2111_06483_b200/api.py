@@ -295,7 +295,8 @@ def bn_forward(x: torch.Tensor, eps: float = 1e-5, gamma: Optional[torch.Tensor]
     m2 = torch.empty(C, dtype=torch.float32, device=dev)
     B.sar_bn_stats(x, mean, m2, ws)
     n_all, mean, m2 = combine_moments(n, mean, m2, group)
-    rstd = torch.rsqrt(m2 / max(n_all, 1) + eps)
+    rstd = torch.empty_like(m2)
+    B.sar_bn_rstd(m2, max(n_all, 1), eps, rstd)
     y = torch.empty_like(x)
     B.sar_bn_apply(x, mean, rstd, gamma, beta, y)
     return y, (mean, rstd, n_all)

@@ -32,7 +32,7 @@ EXPORTS = [
     "sar_mfg_frontier", "sar_csr_filter_rows_indptr", "sar_csr_filter_rows_indices", "sar_spmm_agg_scaled",
     "sar_gat_stack_host_wait", "sar_bn_workspace_bytes", "sar_bn_stats", "sar_bn_apply", "sar_bn_bwd_stats",
     "sar_bn_bwd_apply", "sar_dropout", "sar_linear_workspace_bytes", "sar_linear", "sar_linear_bwd_input",
-    "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd", "sar_axpby",
+    "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd", "sar_axpby", "sar_bn_rstd",
 ]
 
 
@@ -430,6 +430,11 @@ def sar_bn_stats(x: torch.Tensor, mean: torch.Tensor, m2: torch.Tensor, workspac
     w, wb = _ws(workspace)
     _check("sar_bn_stats", lib().sar_bn_stats(c_int64(n), c_int32(C), ctypes.c_int(_dtype(x)), _ptr(x), _ptr(mean),
                                               _ptr(m2), w, wb, _stream()))
+
+
+def sar_bn_rstd(m2: torch.Tensor, count: int, eps: float, rstd: torch.Tensor) -> None:
+    _check("sar_bn_rstd", lib().sar_bn_rstd(c_int32(m2.numel()), _ptr(m2), c_int64(count), c_float(eps), _ptr(rstd),
+                                            _stream()))
 
 
 def sar_bn_apply(x: torch.Tensor, mean: torch.Tensor, rstd: torch.Tensor, gamma: Optional[torch.Tensor],

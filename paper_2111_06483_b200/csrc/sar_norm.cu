@@ -250,6 +250,14 @@ static sar_status norm_apply(const Shape &s, const NormArgs &a, cudaStream_t st,
 
 using namespace sar;
 
+namespace sar {
+// rstd[c] = 1 / sqrt(m2[c] / count + eps): the last step of the statistics, on C floats
+__global__ void norm_rstd_kernel(int C, const float *__restrict__ m2, double inv_count, float eps, float *__restrict__ rstd) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c < C) rstd[c] = (float)(1.0 / sqrt((double)m2[c] * inv_count + (double)eps));
+}
+}  // namespace sar
+
 extern "C" {
 
 size_t sar_bn_workspace_bytes(int32_t C) {
@@ -279,6 +287,13 @@ sar_status sar_bn_stats(int64_t n, int32_t C, sar_dtype t, const void *x, float 
     SAR_TRY(norm_sums<kSumX>(s, a, 1.0 / (double)n, mean, nullptr, workspace, workspace_bytes, st, "bn_mean"));
     a.mean = mean;
     return norm_sums<kSumDev2>(s, a, 1.0, m2, nullptr, workspace, workspace_bytes, st, "bn_m2");
+}
+
+sar_status sar_bn_rstd(int32_t C, const float *m2, int64_t count, float eps, float *rstd, void *stream) {
+    if (C < 1 || count < 1 || !m2 || !rstd || !(eps >= 0.f)) return SAR_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SAR_LAUNCH("bn_rstd", st, (sar::norm_rstd_kernel<<<(unsigned)((C + 127) / 128), 128, 0, st>>>(C, m2, 1.0 / (double)count, eps, rstd)));
+    return sar_after_launch();
 }
 
 sar_status sar_bn_apply(int64_t n, int32_t C, sar_dtype t, const void *x, const float *mean, const float *rstd,
