@@ -328,6 +328,13 @@ SAR_API sar_status sar_relu_bwd(int64_t n_elems, sar_dtype t, const void *y, voi
  * step of an iterated propagation X <- (1-alpha) X0 + alpha S X (Sec. 4.2: label-propagation post-processing), whose
  * product S X is sar_spmm_agg_scaled. */
 SAR_API sar_status sar_axpby(int64_t n_elems, sar_dtype t, float a, const void *x, float b, void *y, void *stream);
+/* The sum of the error contributions a worker receives for its own rows (Algorithm 2: every other worker returns the
+ * error of this worker's features with respect to its part of the output).
+ *   sar_accumulate  acc[i] += x[i], or acc[i] = x[i] with flags = SAR_FIRST; x of type t, acc float32 (the sum of K
+ *                   terms is formed in float32 whatever the storage type), n_elems each, DEVICE memory.
+ *   sar_round_to    y[i] = acc[i] rounded to type t. */
+SAR_API sar_status sar_accumulate(int64_t n_elems, sar_dtype t, const void *x, float *acc, uint32_t flags, void *stream);
+SAR_API sar_status sar_round_to(int64_t n_elems, sar_dtype t, const float *acc, void *y, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * The dense projection of a layer, z = h W (Eq. 1 / Eq. 3 apply a weight matrix to every node's features

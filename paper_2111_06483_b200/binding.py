@@ -32,7 +32,7 @@ EXPORTS = [
     "sar_mfg_frontier", "sar_csr_filter_rows_indptr", "sar_csr_filter_rows_indices", "sar_spmm_agg_scaled",
     "sar_gat_stack_host_wait", "sar_bn_workspace_bytes", "sar_bn_stats", "sar_bn_apply", "sar_bn_bwd_stats",
     "sar_bn_bwd_apply", "sar_dropout", "sar_linear_workspace_bytes", "sar_linear", "sar_linear_bwd_input",
-    "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd", "sar_axpby", "sar_bn_rstd",
+    "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd", "sar_axpby", "sar_bn_rstd", "sar_accumulate", "sar_round_to",
 ]
 
 
@@ -589,6 +589,19 @@ def sar_axpby(a: float, x: torch.Tensor, b: float, y: torch.Tensor) -> None:
     assert x.numel() == y.numel() and x.dtype == y.dtype
     _check("sar_axpby", lib().sar_axpby(c_int64(x.numel()), ctypes.c_int(_dtype(x)), c_float(a), _ptr(x), c_float(b),
                                         _ptr(y), _stream()))
+
+
+def sar_accumulate(x: torch.Tensor, acc: torch.Tensor, first: bool = False) -> None:
+    """acc (float32) += x, or acc = x with first=True."""
+    assert x.numel() == acc.numel() and acc.dtype == torch.float32
+    _check("sar_accumulate", lib().sar_accumulate(c_int64(x.numel()), ctypes.c_int(_dtype(x)), _ptr(x), _ptr(acc),
+                                                  c_uint32(SAR_FIRST if first else 0), _stream()))
+
+
+def sar_round_to(acc: torch.Tensor, y: torch.Tensor) -> None:
+    assert y.numel() == acc.numel() and acc.dtype == torch.float32
+    _check("sar_round_to", lib().sar_round_to(c_int64(acc.numel()), ctypes.c_int(_dtype(y)), _ptr(acc), _ptr(y),
+                                              _stream()))
 
 
 def sar_relu_bwd(y: torch.Tensor, g: torch.Tensor) -> None:

@@ -286,6 +286,21 @@ __global__ void axpby_kernel(long long n, float ca, const T *x, float cb, T *y, 
         Elem<T>::store1(y + i, fmaf(ca, as_float(x[i]), cb * as_float(y[i])));
 }
 
+// acc[i] (+)= x[i] with x of the storage type and acc float32 (sums of the errors the other workers return,
+// Algorithm 2), and the rounding of such a sum back to the storage type
+template <typename T, bool ADD>
+__global__ void widen_kernel(long long n, const T *__restrict__ x, float *__restrict__ acc) {
+    const long long nthreads = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += nthreads)
+        acc[i] = ADD ? acc[i] + as_float(x[i]) : as_float(x[i]);
+}
+template <typename T>
+__global__ void narrow_kernel(long long n, const float *__restrict__ acc, T *__restrict__ y) {
+    const long long nthreads = (long long)gridDim.x * blockDim.x;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += nthreads) Elem<T>::store1(y + i, acc[i]);
+}
+
+
 // ---- dropout (the paper's networks use batch normalisation and dropout between all layers, Sec. 4.2) ------
 // Counter-based: element i is kept when the top 24 bits of SplitMix64's (i+1)-th output for `seed` reach
 // p * 2^24; nothing is stored, the backward pass draws the same mask again from the seed.
@@ -483,6 +498,42 @@ sar_status sar_axpby(int64_t n_elems, sar_dtype t, float a, const void *x, float
         SAR_LAUNCH("axpby", st, (axpby_kernel<float><<<(unsigned)blocks, 256, 0, st>>>(n_elems, a, static_cast<const float *>(x), b, static_cast<float *>(y), n_vec16)));
     else
         SAR_LAUNCH("axpby", st, (axpby_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, st>>>(n_elems, a, static_cast<const __nv_bfloat16 *>(x), b, static_cast<__nv_bfloat16 *>(y), n_vec16)));
+    return sar_after_launch();
+}
+
+sar_status sar_accumulate(int64_t n_elems, sar_dtype t, const void *x, float *acc, uint32_t flags, void *stream) {
+    if (n_elems < 0 || (n_elems > 0 && (!x || !acc)) || (flags & ~(uint32_t)SAR_FIRST)) return SAR_ERR_INVALID_ARG;
+    if (t != SAR_F32 && t != SAR_BF16) return SAR_ERR_INVALID_ARG;
+    SAR_TRY(check_elem_align({x}, sar_elem_size(t)));
+    SAR_TRY(check_elem_align({acc}, 4));
+    if (n_elems == 0) return SAR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    long long blocks = (n_elems + 255) / 256;
+    if (blocks > 148 * 64) blocks = 148 * 64;
+    const bool first = flags & SAR_FIRST;
+    if (t == SAR_F32) {
+        if (first) SAR_LAUNCH("accumulate", st, (widen_kernel<float, false><<<(unsigned)blocks, 256, 0, st>>>(n_elems, static_cast<const float *>(x), acc)));
+        else SAR_LAUNCH("accumulate", st, (widen_kernel<float, true><<<(unsigned)blocks, 256, 0, st>>>(n_elems, static_cast<const float *>(x), acc)));
+    } else {
+        if (first) SAR_LAUNCH("accumulate", st, (widen_kernel<__nv_bfloat16, false><<<(unsigned)blocks, 256, 0, st>>>(n_elems, static_cast<const __nv_bfloat16 *>(x), acc)));
+        else SAR_LAUNCH("accumulate", st, (widen_kernel<__nv_bfloat16, true><<<(unsigned)blocks, 256, 0, st>>>(n_elems, static_cast<const __nv_bfloat16 *>(x), acc)));
+    }
+    return sar_after_launch();
+}
+
+sar_status sar_round_to(int64_t n_elems, sar_dtype t, const float *acc, void *y, void *stream) {
+    if (n_elems < 0 || (n_elems > 0 && (!acc || !y))) return SAR_ERR_INVALID_ARG;
+    if (t != SAR_F32 && t != SAR_BF16) return SAR_ERR_INVALID_ARG;
+    SAR_TRY(check_elem_align({y}, sar_elem_size(t)));
+    SAR_TRY(check_elem_align({acc}, 4));
+    if (n_elems == 0) return SAR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    long long blocks = (n_elems + 255) / 256;
+    if (blocks > 148 * 64) blocks = 148 * 64;
+    if (t == SAR_F32)
+        SAR_LAUNCH("round_to", st, (narrow_kernel<float><<<(unsigned)blocks, 256, 0, st>>>(n_elems, acc, static_cast<float *>(y))));
+    else
+        SAR_LAUNCH("round_to", st, (narrow_kernel<__nv_bfloat16><<<(unsigned)blocks, 256, 0, st>>>(n_elems, acc, static_cast<__nv_bfloat16 *>(y))));
     return sar_after_launch();
 }
 

@@ -122,6 +122,22 @@ class CudaGatBackend:
     def bwd_end(self):
         return self.del_
 
+    # the sums of the error contributions other workers return (Algorithm 2), formed in float32
+    def sum_begin(self, x: torch.Tensor) -> torch.Tensor:
+        acc = torch.empty(x.shape, dtype=torch.float32, device=x.device)
+        B.sar_accumulate(x, acc, first=True)
+        return acc
+
+    def sum_add(self, acc: torch.Tensor, x: torch.Tensor) -> None:
+        B.sar_accumulate(x, acc)
+
+    def sum_end(self, acc: torch.Tensor, like: torch.Tensor) -> torch.Tensor:
+        if like.dtype == torch.float32:
+            return acc
+        y = torch.empty(acc.shape, dtype=like.dtype, device=acc.device)
+        B.sar_round_to(acc, y)
+        return y
+
 
 # ----------------------------------------------------------------------------------------------
 # the schedule
@@ -167,19 +183,18 @@ class ShardedGatLayer:
         be.bwd_begin(gout)
         pending = self._fetch(1, feat, er) if K > 1 else None
         cur = (feat, er)
-        dfeat_acc = der_acc = None
-        wide = torch.float32 if feat.dtype in (torch.bfloat16, torch.float16) else feat.dtype  # sums of K terms
+        dfeat_acc = der_acc = None  # sums of K terms, kept by the backend in a wide type
         returning = None
         for s in range(K):
             q = (p + s) % K
             dfeat_q, der_q = be.bwd_step(q, cur[0], cur[1], s == 0, s == K - 1)
             if returning is not None:  # the error exchanged during the previous step, added in step order
                 got = returning.wait()
-                dfeat_acc += got[0].to(wide)
-                der_acc += got[1]
+                be.sum_add(dfeat_acc, got[0])
+                be.sum_add(der_acc, got[1])
                 returning = got = None  # the receive buffer is released before the next one is posted
             if s == 0:
-                dfeat_acc, der_acc = dfeat_q.to(wide, copy=True), der_q.clone()
+                dfeat_acc, der_acc = be.sum_begin(dfeat_q), be.sum_begin(der_q)
             else:
                 # our error for partition q goes to its owner; worker (p-s) mod K holds the error for our sources
                 returning = self.comm.start(q, [dfeat_q, der_q], (p - s) % K, [feat, er])
@@ -188,6 +203,6 @@ class ShardedGatLayer:
                 pending = self._fetch(s + 2, feat, er) if s + 2 < K else None
         if returning is not None:
             got = returning.wait()
-            dfeat_acc += got[0].to(wide)
-            der_acc += got[1]
-        return dfeat_acc.to(feat.dtype), be.bwd_end(), der_acc
+            be.sum_add(dfeat_acc, got[0])
+            be.sum_add(der_acc, got[1])
+        return be.sum_end(dfeat_acc, feat), be.bwd_end(), be.sum_end(der_acc, er)

@@ -67,6 +67,15 @@ class TorchRefBackend:
     def bwd_end(self):
         return self.del_
 
+    def sum_begin(self, x):
+        return x.double().clone()
+
+    def sum_add(self, acc, x):
+        acc += x.double()
+
+    def sum_end(self, acc, like):
+        return acc.to(like.dtype)
+
 
 class ThreadComm:
     """Emulated workers as threads of one process: mail[(a, b)] carries the messages from a to b in order."""

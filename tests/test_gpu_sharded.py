@@ -66,3 +66,23 @@ def test_sharded_layer_on_the_gpu_equals_the_whole_graph(K, dt):
         allclose_report(cat(5), b.der, 1e-4, 1e-5 * rms(b.der), "der")
     allclose_report(cat(1), f.m, 1e-5, 1e-6, "m")   # float32 scores against the oracle's float64 ones
     allclose_report(cat(2), f.d, 1e-5, 1e-6, "d")
+
+
+@pytest.mark.parametrize("n,dtype", [(1, torch.float32), (1000, torch.bfloat16), (100003, torch.bfloat16), (4096, torch.float32)])
+def test_error_sums_in_float32(n, dtype):
+    """acc = x0; acc += x1; acc += x2 in float32, then one rounding to the storage type: the sum of the errors
+    returned by the other workers (Algorithm 2)."""
+    from paper_2111_06483_b200 import binding as B
+    rng = np.random.default_rng(n)
+    xs = [torch.from_numpy(rng.standard_normal(n).astype(np.float32)).to(dtype).cuda() for _ in range(3)]
+    acc = torch.full((n,), float("nan"), dtype=torch.float32, device="cuda")
+    B.sar_accumulate(xs[0], acc, first=True)
+    B.sar_accumulate(xs[1], acc)
+    B.sar_accumulate(xs[2], acc)
+    want = (xs[0].float() + xs[1].float()) + xs[2].float()  # the same float32 additions in the same order
+    assert torch.equal(acc, want)
+    y = torch.empty(n, dtype=dtype, device="cuda")
+    B.sar_round_to(acc, y)
+    assert torch.equal(y, want.to(dtype))  # round to nearest even
+    with pytest.raises(AssertionError):  # the sum is float32 whatever the storage type
+        B.sar_accumulate(xs[0], acc.double())
