@@ -324,6 +324,7 @@ def run_ours(args, rank, world, local_rank):
             bn_s0, bn_s1 = torch.empty(D, dtype=torch.float32, device=dev), torch.empty(D, dtype=torch.float32, device=dev)
             bws = torch.empty(B.sar_bn_workspace_bytes(D), dtype=torch.uint8, device=dev)
             p_drop, seeds = 0.5, [1000 + l for l in range(L)]
+            act = B.SAR_GLUE_RELU | B.SAR_GLUE_DROPOUT  # y = dropout(relu(bn(x))) in one pass over the node array
             gx_bn = torch.empty((n, H, F), dtype=tdt, device=dev)  # gradient w.r.t. a layer's aggregation output
 
             def step():
@@ -336,9 +337,7 @@ def run_ours(args, rank, world, local_rank):
                         x = flat(feats[l + 1])
                         B.sar_bn_stats(x, bn_mean[l], bn_m2[l], bws)
                         B.sar_bn_rstd(bn_m2[l], n, 1e-5, bn_rstd[l])
-                        B.sar_bn_apply(x, bn_mean[l], bn_rstd[l], None, None, flat(hs[l + 1]))
-                        B.sar_relu(hs[l + 1])
-                        B.sar_dropout(hs[l + 1], p_drop, seeds[l], hs[l + 1])
+                        B.sar_bn_apply_act(x, bn_mean[l], bn_rstd[l], None, None, act, p_drop, seeds[l], flat(hs[l + 1]))
                 gin = gout
                 for l in reversed(range(L)):
                     B.sar_gat_bwd_fused(g.whole, g.bounds, z_q[l], els[l], er_q[l], ms[l], ds[l], gin, H, F, cfg.slope,
@@ -347,12 +346,12 @@ def run_ours(args, rank, world, local_rank):
                     B.sar_linear_bwd_weight(flat(hs[l]), flat(gbuf[0]), dW, lws)
                     B.sar_linear_bwd_input(flat(gbuf[0]), Ws[l], flat(gbuf[1]), lws)
                     if l > 0:
-                        gh = gbuf[1]                                    # gradient w.r.t. hs[l]
-                        B.sar_dropout(gh, p_drop, seeds[l - 1], gh)     # the same mask, drawn again from the seed
-                        B.sar_relu_bwd(hs[l], gh)                       # hs[l] > 0 exactly where the ReLU passed and the mask kept
-                        x = flat(feats[l])
-                        B.sar_bn_bwd_stats(x, bn_mean[l - 1], bn_rstd[l - 1], flat(gh), bn_s0, bn_s1, bws)
-                        B.sar_bn_bwd_apply(x, bn_mean[l - 1], bn_rstd[l - 1], None, flat(gh), bn_s0, bn_s1, 1.0 / n, flat(gx_bn))
+                        gh = flat(gbuf[1])      # gradient w.r.t. hs[l]; the two calls take it back through the dropout
+                        x = flat(feats[l])      # and the ReLU (hs[l] > 0 where both let it pass) on the fly
+                        B.sar_bn_bwd_stats_act(x, bn_mean[l - 1], bn_rstd[l - 1], gh, flat(hs[l]), act, p_drop, seeds[l - 1],
+                                               bn_s0, bn_s1, bws)
+                        B.sar_bn_bwd_apply_act(x, bn_mean[l - 1], bn_rstd[l - 1], None, gh, flat(hs[l]), act, p_drop,
+                                               seeds[l - 1], bn_s0, bn_s1, 1.0 / n, flat(gx_bn))
                         gin = gx_bn
 
         def step_plain():

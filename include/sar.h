@@ -309,6 +309,7 @@ SAR_API sar_status sar_spmm_agg_scaled(const sar_part *g, const void *feat_q, in
  * ------------------------------------------------------------------------------------------- */
 SAR_API size_t sar_gat_project_workspace_bytes(int32_t H, int32_t F);
 #define SAR_GLUE_RELU 1u
+#define SAR_GLUE_DROPOUT 2u /* only for the sar_bn_*_act calls */
 SAR_API sar_status sar_gat_project(int64_t n, int32_t H, int32_t F, sar_dtype t, void *z, const float *a_l,
                                    const float *a_r, float *el, float *er, uint32_t flags, void *stream);
 SAR_API sar_status sar_gat_project_bwd(int64_t n, int32_t H, int32_t F, sar_dtype t, const void *z, const float *a_l,
@@ -422,6 +423,27 @@ SAR_API sar_status sar_bn_bwd_stats(int64_t n, int32_t C, sar_dtype t, const voi
 SAR_API sar_status sar_bn_bwd_apply(int64_t n, int32_t C, sar_dtype t, const void *x, const float *mean,
                                     const float *rstd, const float *gamma, const void *gy, const float *sum_gy,
                                     const float *sum_gy_xhat, float inv_count, void *gx, void *stream);
+
+/* The same three calls with the chain that follows the normalisation in the paper's networks (Sec. 4.2: batch
+ * normalisation and dropout between all layers) folded in, so that the node array is read and written once instead
+ * of three times: y = dropout(relu(bn(x))), with flags = SAR_GLUE_RELU and / or SAR_GLUE_DROPOUT choosing the links
+ * (0: plain sar_bn_apply).  The dropout is sar_dropout's: element i (flat index into [n, C]) is kept and scaled by
+ * 1/(1-p) when the top 24 bits of SplitMix64's (i+1)-th output for `seed` reach p * 2^24.
+ * Backward: gy is the gradient with respect to y; both calls first take it back through the dropout (same seed)
+ * and the ReLU and then proceed as sar_bn_bwd_stats / sar_bn_bwd_apply.  `post` is y as the forward call left it
+ * (needed when SAR_GLUE_RELU is set: the ReLU passed where y > 0; with both flags y > 0 also tells which elements
+ * the mask kept, so no random number is drawn).  gx may be gy.  Other flag bits: SAR_ERR_INVALID_ARG. */
+SAR_API sar_status sar_bn_apply_act(int64_t n, int32_t C, sar_dtype t, const void *x, const float *mean,
+                                    const float *rstd, const float *gamma, const float *beta, uint32_t flags, float p,
+                                    uint64_t seed, void *y, void *stream);
+SAR_API sar_status sar_bn_bwd_stats_act(int64_t n, int32_t C, sar_dtype t, const void *x, const float *mean,
+                                        const float *rstd, const void *gy, const void *post, uint32_t flags, float p,
+                                        uint64_t seed, float *sum_gy, float *sum_gy_xhat, void *workspace,
+                                        size_t workspace_bytes, void *stream);
+SAR_API sar_status sar_bn_bwd_apply_act(int64_t n, int32_t C, sar_dtype t, const void *x, const float *mean,
+                                        const float *rstd, const float *gamma, const void *gy, const void *post,
+                                        uint32_t flags, float p, uint64_t seed, const float *sum_gy,
+                                        const float *sum_gy_xhat, float inv_count, void *gx, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Backward pass without any caller-provided scratch.  (The paper has no counterpart: this is a

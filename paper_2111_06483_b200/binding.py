@@ -32,7 +32,8 @@ EXPORTS = [
     "sar_mfg_frontier", "sar_csr_filter_rows_indptr", "sar_csr_filter_rows_indices", "sar_spmm_agg_scaled",
     "sar_gat_stack_host_wait", "sar_bn_workspace_bytes", "sar_bn_stats", "sar_bn_apply", "sar_bn_bwd_stats",
     "sar_bn_bwd_apply", "sar_dropout", "sar_linear_workspace_bytes", "sar_linear", "sar_linear_bwd_input",
-    "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd", "sar_axpby", "sar_bn_rstd", "sar_accumulate", "sar_round_to",
+    "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd", "sar_axpby", "sar_bn_rstd", "sar_accumulate", "sar_round_to", "sar_bn_apply_act",
+    "sar_bn_bwd_stats_act", "sar_bn_bwd_apply_act",
 ]
 
 
@@ -462,6 +463,35 @@ def sar_bn_bwd_apply(x: torch.Tensor, mean: torch.Tensor, rstd: torch.Tensor, ga
                                                       _ptr(sum_gy_xhat), c_float(inv_count), _ptr(gx), _stream()))
 
 
+def sar_bn_apply_act(x: torch.Tensor, mean: torch.Tensor, rstd: torch.Tensor, gamma: Optional[torch.Tensor],
+                     beta: Optional[torch.Tensor], flags: int, p: float, seed: int, y: torch.Tensor) -> None:
+    n, C = x.shape
+    _check("sar_bn_apply_act", lib().sar_bn_apply_act(c_int64(n), c_int32(C), ctypes.c_int(_dtype(x)), _ptr(x), _ptr(mean),
+                                                      _ptr(rstd), _ptr(gamma), _ptr(beta), c_uint32(flags), c_float(p),
+                                                      ctypes.c_uint64(seed & 0xFFFFFFFFFFFFFFFF), _ptr(y), _stream()))
+
+
+def sar_bn_bwd_stats_act(x: torch.Tensor, mean: torch.Tensor, rstd: torch.Tensor, gy: torch.Tensor,
+                         post: Optional[torch.Tensor], flags: int, p: float, seed: int, sum_gy: torch.Tensor,
+                         sum_gy_xhat: torch.Tensor, workspace: torch.Tensor) -> None:
+    n, C = x.shape
+    w, wb = _ws(workspace)
+    _check("sar_bn_bwd_stats_act", lib().sar_bn_bwd_stats_act(
+        c_int64(n), c_int32(C), ctypes.c_int(_dtype(x)), _ptr(x), _ptr(mean), _ptr(rstd), _ptr(gy), _ptr(post),
+        c_uint32(flags), c_float(p), ctypes.c_uint64(seed & 0xFFFFFFFFFFFFFFFF), _ptr(sum_gy), _ptr(sum_gy_xhat), w, wb,
+        _stream()))
+
+
+def sar_bn_bwd_apply_act(x: torch.Tensor, mean: torch.Tensor, rstd: torch.Tensor, gamma: Optional[torch.Tensor],
+                         gy: torch.Tensor, post: Optional[torch.Tensor], flags: int, p: float, seed: int,
+                         sum_gy: torch.Tensor, sum_gy_xhat: torch.Tensor, inv_count: float, gx: torch.Tensor) -> None:
+    n, C = x.shape
+    _check("sar_bn_bwd_apply_act", lib().sar_bn_bwd_apply_act(
+        c_int64(n), c_int32(C), ctypes.c_int(_dtype(x)), _ptr(x), _ptr(mean), _ptr(rstd), _ptr(gamma), _ptr(gy),
+        _ptr(post), c_uint32(flags), c_float(p), ctypes.c_uint64(seed & 0xFFFFFFFFFFFFFFFF), _ptr(sum_gy),
+        _ptr(sum_gy_xhat), c_float(inv_count), _ptr(gx), _stream()))
+
+
 def sar_gat_stack_host_wait() -> None:
     _check("sar_gat_stack_host_wait", lib().sar_gat_stack_host_wait(_stream()))
 
@@ -495,6 +525,7 @@ def sar_gat_project_workspace_bytes(H: int, F: int) -> int:
 
 
 SAR_GLUE_RELU = 1
+SAR_GLUE_DROPOUT = 2
 
 
 def sar_gat_project(z: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, el: torch.Tensor, er: torch.Tensor,

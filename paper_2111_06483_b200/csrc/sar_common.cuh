@@ -42,6 +42,15 @@ static inline size_t sar_elem_size(sar_dtype t) { return t == SAR_BF16 ? 2 : 4; 
 
 #define SAR_NEG_INF (-INFINITY)
 
+// SplitMix64's (i+1)-th output for `seed`: the counter-based generator of the dropout mask (element i is kept
+// when the top 24 bits reach p * 2^24); nothing is stored, the mask is drawn again wherever it is needed.
+__host__ __device__ inline unsigned long long splitmix64_at(unsigned long long seed, unsigned long long i) {
+    unsigned long long z = seed + (i + 1ull) * 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
 // launch observer (sar_set_launch_hook)
 namespace sar {
 extern sar_launch_hook_fn g_launch_hook;

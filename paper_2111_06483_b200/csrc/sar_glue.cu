@@ -304,12 +304,6 @@ __global__ void narrow_kernel(long long n, const float *__restrict__ acc, T *__r
 // ---- dropout (the paper's networks use batch normalisation and dropout between all layers, Sec. 4.2) ------
 // Counter-based: element i is kept when the top 24 bits of SplitMix64's (i+1)-th output for `seed` reach
 // p * 2^24; nothing is stored, the backward pass draws the same mask again from the seed.
-__device__ __forceinline__ unsigned long long splitmix64_at(unsigned long long seed, unsigned long long i) {
-    unsigned long long z = seed + (i + 1ull) * 0x9E3779B97F4A7C15ull;
-    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
-    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
-    return z ^ (z >> 31);
-}
 
 template <typename T>
 __global__ void dropout_kernel(long long n, const T *x, T *y, unsigned threshold, float scale, unsigned long long seed,

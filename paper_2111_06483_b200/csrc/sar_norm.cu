@@ -21,7 +21,35 @@ struct NormArgs {
     float inv_count;
     float *partial;              // [blocks][2][C]
     RowGeom g;
+    // optional chain after the normalisation, y = dropout(relu(bn(x))) (the paper's networks, Sec. 4.2), and its
+    // mirror in front of the backward pass: the incoming gradient is masked by the dropout and the ReLU first
+    unsigned act;                // bit 0 (SAR_GLUE_RELU), bit 1 (SAR_GLUE_DROPOUT)
+    unsigned threshold;          // floor(p * 2^24)
+    float scale;                 // 1 / (1 - p)
+    unsigned long long seed;
+    const void *post;            // backward: y as the forward chain left it
 };
+
+// forward chain on one element of flat index idx
+// ACT (template argument of the kernels): 0 = no chain, 3 = ReLU and dropout (the networks' case, decided at compile
+// time so that the backward kernels carry no generator code), 1 = whatever NormArgs::act says.
+template <int ACT>
+__device__ __forceinline__ float act_fwd(const NormArgs &a, float o, long long idx) {
+    const unsigned act = ACT == 3 ? 3u : a.act;
+    if (act & 1u) o = o > 0.f ? o : 0.f;
+    if (act & 2u) o = (unsigned)(splitmix64_at(a.seed, (unsigned long long)idx) >> 40) >= a.threshold ? o * a.scale : 0.f;
+    return o;
+}
+// the gradient that reaches the normalisation's output: through the dropout (kept and scaled, or 0) and the ReLU.
+// With both, y > 0 exactly where the ReLU passed and the mask kept, so the stored y decides alone.
+template <int ACT>
+__device__ __forceinline__ float act_bwd(const NormArgs &a, float g, float post, long long idx) {
+    if constexpr (ACT == 3) return post > 0.f ? g * a.scale : 0.f;
+    if ((a.act & 3u) == 3u) return post > 0.f ? g * a.scale : 0.f;
+    if (a.act & 2u) g = (unsigned)(splitmix64_at(a.seed, (unsigned long long)idx) >> 40) >= a.threshold ? g * a.scale : 0.f;
+    if (a.act & 1u) g = post > 0.f ? g : 0.f;
+    return g;
+}
 
 enum NormSum { kSumX = 0, kSumDev2 = 1, kSumGrad = 2 };
 
@@ -42,7 +70,7 @@ __device__ __forceinline__ void load_cols(const float *__restrict__ p, float fil
 
 // Column sums over the block's rows: WHAT = kSumX: sum x; kSumDev2: sum (x - mean)^2; kSumGrad: sum gy and
 // sum gy * xhat with xhat = (x - mean) * rstd.  Per-block partials, no atomics.
-template <typename T, int G, int V, int WHAT>
+template <typename T, int G, int V, int WHAT, int ACT = 0>
 __global__ void __launch_bounds__(kThreads) norm_sums_kernel(const NormArgs a) {
     constexpr int EPV = Elem<T>::EPV;
     constexpr int RPW = 32 / G;
@@ -62,7 +90,22 @@ __global__ void __launch_bounds__(kThreads) norm_sums_kernel(const NormArgs a) {
     for (long long row = (long long)blockIdx.x * GPB + group; row < a.n; row += stride) {
         float xv[V][EPV], gv[V][EPV];
         load_row_vec<T, G, V>(a.x, row, a.g.n_vec, id.gl, vg.vok, xv);
-        if constexpr (WHAT == kSumGrad) load_row_vec<T, G, V>(a.gy, row, a.g.n_vec, id.gl, vg.vok, gv);
+        if constexpr (WHAT == kSumGrad) {
+            load_row_vec<T, G, V>(a.gy, row, a.g.n_vec, id.gl, vg.vok, gv);
+            if constexpr (ACT != 0) {
+                float pv[V][EPV];
+#pragma unroll
+                for (int v = 0; v < V; ++v)
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) pv[v][e] = 0.f;
+                if (ACT == 3 || (a.act & 1u)) load_row_vec<T, G, V>(a.post, row, a.g.n_vec, id.gl, vg.vok, pv);
+#pragma unroll
+                for (int v = 0; v < V; ++v)
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e)
+                        gv[v][e] = vg.vok[v] ? act_bwd<ACT>(a, gv[v][e], pv[v][e], row * a.C + (v * G + id.gl) * EPV + e) : 0.f;
+            }
+        }
 #pragma unroll
         for (int v = 0; v < V; ++v)
 #pragma unroll
@@ -113,7 +156,7 @@ __global__ void norm_reduce_kernel(int blocks, int C, const float *__restrict__ 
 
 // y = (x - mean) * rstd * gamma + beta             (BWD = false)
 // gx = gamma * rstd * (gy - s0/N - xhat * s1/N)    (BWD = true; inv_count = 1/N)
-template <typename T, int G, int V, bool BWD>
+template <typename T, int G, int V, bool BWD, int ACT = 0>
 __global__ void __launch_bounds__(kThreads) norm_apply_kernel(const NormArgs a) {
     constexpr int EPV = Elem<T>::EPV;
     constexpr int RPW = 32 / G;
@@ -131,16 +174,33 @@ __global__ void __launch_bounds__(kThreads) norm_apply_kernel(const NormArgs a) 
         float xv[V][EPV], gv[V][EPV], ov[V][EPV];
         // plain loads: the output may be the same array as x or gy
         load_row_vec<T, G, V, false>(a.x, row, a.g.n_vec, id.gl, vg.vok, xv);
-        if constexpr (BWD) load_row_vec<T, G, V, false>(a.gy, row, a.g.n_vec, id.gl, vg.vok, gv);
+        if constexpr (BWD) {
+            load_row_vec<T, G, V, false>(a.gy, row, a.g.n_vec, id.gl, vg.vok, gv);
+            if constexpr (ACT != 0) {
+                float pv[V][EPV];
+#pragma unroll
+                for (int v = 0; v < V; ++v)
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e) pv[v][e] = 0.f;
+                if (ACT == 3 || (a.act & 1u)) load_row_vec<T, G, V, false>(a.post, row, a.g.n_vec, id.gl, vg.vok, pv);
+#pragma unroll
+                for (int v = 0; v < V; ++v)
+#pragma unroll
+                    for (int e = 0; e < EPV; ++e)
+                        gv[v][e] = vg.vok[v] ? act_bwd<ACT>(a, gv[v][e], pv[v][e], row * a.C + (v * G + id.gl) * EPV + e) : 0.f;
+            }
+        }
 #pragma unroll
         for (int v = 0; v < V; ++v)
 #pragma unroll
             for (int e = 0; e < EPV; ++e) {
                 const float xh = (xv[v][e] - mu[v][e]) * rs[v][e];
-                if constexpr (BWD)
+                if constexpr (BWD) {
                     ov[v][e] = ga[v][e] * rs[v][e] * (gv[v][e] - m0[v][e] * a.inv_count - xh * (m1[v][e] * a.inv_count));
-                else
+                } else {
                     ov[v][e] = fmaf(xh, ga[v][e], be[v][e]);
+                    if constexpr (ACT != 0) ov[v][e] = act_fwd<ACT>(a, ov[v][e], row * a.C + (v * G + id.gl) * EPV + e);
+                }
             }
         store_row_vec<T, G, V>(a.y, row, a.g.n_vec, id.gl, vg.vok, ov);
     }
@@ -163,7 +223,8 @@ __global__ void norm_sums_generic(const NormArgs a, int slices) {
         } else if (WHAT == kSumDev2) {
             s0 = fmaf(xv - mu, xv - mu, s0);
         } else {
-            const float g = nrm_as_float(gy[i * a.C + c]);
+            float g = nrm_as_float(gy[i * a.C + c]);
+            if (a.act) g = act_bwd<1>(a, g, (a.act & 1u) ? nrm_as_float(reinterpret_cast<const T *>(a.post)[i * a.C + c]) : 0.f, i * a.C + c);
             s0 += g;
             s1 = fmaf(g, (xv - mu) * rs, s1);
         }
@@ -180,10 +241,14 @@ __global__ void norm_apply_generic(const NormArgs a) {
         const float xh = (nrm_as_float(reinterpret_cast<const T *>(a.x)[i]) - a.mean[c]) * a.rstd[c];
         const float ga = a.gamma ? a.gamma[c] : 1.f;
         float o;
-        if (BWD)
-            o = ga * a.rstd[c] * (nrm_as_float(reinterpret_cast<const T *>(a.gy)[i]) - a.s0[c] * a.inv_count - xh * (a.s1[c] * a.inv_count));
-        else
+        if (BWD) {
+            float g = nrm_as_float(reinterpret_cast<const T *>(a.gy)[i]);
+            if (a.act) g = act_bwd<1>(a, g, (a.act & 1u) ? nrm_as_float(reinterpret_cast<const T *>(a.post)[i]) : 0.f, i);
+            o = ga * a.rstd[c] * (g - a.s0[c] * a.inv_count - xh * (a.s1[c] * a.inv_count));
+        } else {
             o = fmaf(xh, ga, a.beta ? a.beta[c] : 0.f);
+            if (a.act) o = act_fwd<1>(a, o, i);
+        }
         Elem<T>::store1(reinterpret_cast<T *>(a.y) + i, o);
     }
 }
@@ -216,7 +281,9 @@ static sar_status norm_sums(const Shape &s, NormArgs a, double scale, float *out
         using T = typename C::type;
         constexpr int EPV = Elem<T>::EPV;
         const size_t smem = (size_t)kWarpsPerBlock * (32 / C::g) * 2 * (C::g * C::v * EPV) * 4;
-        auto kern = norm_sums_kernel<T, C::g, C::v, WHAT>;
+        auto kern = (WHAT != kSumGrad || a.act == 0) ? norm_sums_kernel<T, C::g, C::v, WHAT, 0>
+                    : (a.act == 3 ? norm_sums_kernel<T, C::g, C::v, WHAT, (WHAT == kSumGrad ? 3 : 0)>
+                                  : norm_sums_kernel<T, C::g, C::v, WHAT, (WHAT == kSumGrad ? 1 : 0)>);
         SAR_TRY(ensure_smem(kern, smem));
         SAR_LAUNCH(name, st, kern<<<kNormBlocks, kThreads, smem, st>>>(a));
         SAR_TRY(sar_after_launch());
@@ -241,7 +308,9 @@ static sar_status norm_apply(const Shape &s, const NormArgs &a, cudaStream_t st,
         using T = typename C::type;
         unsigned blocks = blocks_for(a.n, C::g);
         if (blocks > (unsigned)kNormBlocks * 4) blocks = kNormBlocks * 4;
-        SAR_LAUNCH(name, st, (norm_apply_kernel<T, C::g, C::v, BWD><<<blocks, kThreads, 0, st>>>(a)));
+        auto kern = a.act == 0 ? norm_apply_kernel<T, C::g, C::v, BWD, 0>
+                               : (a.act == 3 ? norm_apply_kernel<T, C::g, C::v, BWD, 3> : norm_apply_kernel<T, C::g, C::v, BWD, 1>);
+        SAR_LAUNCH(name, st, (kern<<<blocks, kThreads, 0, st>>>(a)));
         return sar_after_launch();
     });
 }
@@ -255,6 +324,24 @@ namespace sar {
 __global__ void norm_rstd_kernel(int C, const float *__restrict__ m2, double inv_count, float eps, float *__restrict__ rstd) {
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
     if (c < C) rstd[c] = (float)(1.0 / sqrt((double)m2[c] * inv_count + (double)eps));
+}
+}  // namespace sar
+
+namespace sar {
+static sar_status norm_set_act(NormArgs &a, uint32_t flags, float p, uint64_t seed, const void *post, bool backward) {
+    if (flags & ~(uint32_t)(SAR_GLUE_RELU | SAR_GLUE_DROPOUT)) return SAR_ERR_INVALID_ARG;
+    a.act = flags;
+    a.threshold = 0;
+    a.scale = 1.f;
+    a.seed = seed;
+    a.post = post;
+    if (flags & SAR_GLUE_DROPOUT) {
+        if (!(p >= 0.f && p < 1.f)) return SAR_ERR_INVALID_ARG;
+        a.threshold = (unsigned)((double)p * 16777216.0);  // floor(p * 2^24), as sar_dropout
+        a.scale = 1.f / (1.f - p);
+    }
+    if (backward && (flags & SAR_GLUE_RELU) && a.n > 0 && !post) return SAR_ERR_INVALID_ARG;
+    return SAR_OK;
 }
 }  // namespace sar
 
@@ -365,6 +452,82 @@ sar_status sar_bn_bwd_apply(int64_t n, int32_t C, sar_dtype t, const void *x, co
     a.inv_count = inv_count;
     a.g = s.geom;
     return norm_apply<true>(s, a, static_cast<cudaStream_t>(stream), "bn_bwd_apply");
+}
+
+sar_status sar_bn_apply_act(int64_t n, int32_t C, sar_dtype t, const void *x, const float *mean, const float *rstd,
+                            const float *gamma, const float *beta, uint32_t flags, float p, uint64_t seed, void *y,
+                            void *stream) {
+    if (!mean || !rstd || (n > 0 && (!x || !y))) return SAR_ERR_INVALID_ARG;
+    Shape s;
+    SAR_TRY(norm_shape(n, C, t, {x, y}, &s));
+    SAR_TRY(check_elem_align({mean, rstd, gamma, beta}, 4));
+    SAR_TRY(check_elem_align({x, y}, sar_elem_size(t)));
+    NormArgs a{};
+    a.n = n;
+    a.C = C;
+    a.x = x;
+    a.y = y;
+    a.mean = mean;
+    a.rstd = rstd;
+    a.gamma = gamma;
+    a.beta = beta;
+    a.g = s.geom;
+    SAR_TRY(norm_set_act(a, flags, p, seed, nullptr, false));
+    if (n == 0) return SAR_OK;
+    return norm_apply<false>(s, a, static_cast<cudaStream_t>(stream), "bn_apply_act");
+}
+
+sar_status sar_bn_bwd_stats_act(int64_t n, int32_t C, sar_dtype t, const void *x, const float *mean, const float *rstd,
+                                const void *gy, const void *post, uint32_t flags, float p, uint64_t seed, float *sum_gy,
+                                float *sum_gy_xhat, void *workspace, size_t workspace_bytes, void *stream) {
+    if (!mean || !rstd || !sum_gy || !sum_gy_xhat || (n > 0 && (!x || !gy))) return SAR_ERR_INVALID_ARG;
+    Shape s;
+    SAR_TRY(norm_shape(n, C, t, {x, gy, post}, &s));
+    SAR_TRY(check_elem_align({mean, rstd, sum_gy, sum_gy_xhat}, 4));
+    SAR_TRY(check_elem_align({x, gy, post}, sar_elem_size(t)));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    NormArgs a{};
+    a.n = n;
+    a.C = C;
+    a.x = x;
+    a.gy = gy;
+    a.mean = mean;
+    a.rstd = rstd;
+    a.g = s.geom;
+    SAR_TRY(norm_set_act(a, flags, p, seed, post, true));
+    if (n == 0) {
+        SAR_CUDA_TRY(cudaMemsetAsync(sum_gy, 0, (size_t)C * 4, st));
+        SAR_CUDA_TRY(cudaMemsetAsync(sum_gy_xhat, 0, (size_t)C * 4, st));
+        return SAR_OK;
+    }
+    return norm_sums<kSumGrad>(s, a, 1.0, sum_gy, sum_gy_xhat, workspace, workspace_bytes, st, "bn_bwd_sums_act");
+}
+
+sar_status sar_bn_bwd_apply_act(int64_t n, int32_t C, sar_dtype t, const void *x, const float *mean, const float *rstd,
+                                const float *gamma, const void *gy, const void *post, uint32_t flags, float p,
+                                uint64_t seed, const float *sum_gy, const float *sum_gy_xhat, float inv_count, void *gx,
+                                void *stream) {
+    if (!mean || !rstd || !sum_gy || !sum_gy_xhat || (n > 0 && (!x || !gy || !gx))) return SAR_ERR_INVALID_ARG;
+    Shape s;
+    SAR_TRY(norm_shape(n, C, t, {x, gy, gx, post}, &s));
+    SAR_TRY(check_elem_align({mean, rstd, gamma, sum_gy, sum_gy_xhat}, 4));
+    SAR_TRY(check_elem_align({x, gy, gx, post}, sar_elem_size(t)));
+    NormArgs a{};
+    a.n = n;
+    a.C = C;
+    a.x = x;
+    a.gy = gy;
+    a.y = gx;
+    a.mean = mean;
+    a.rstd = rstd;
+    a.gamma = gamma;
+    a.s0 = sum_gy;
+    a.s1 = sum_gy_xhat;
+    a.inv_count = inv_count;
+    a.g = s.geom;
+    SAR_TRY(norm_set_act(a, flags, p, seed, post, true));
+    if (n == 0) return SAR_OK;
+    return norm_apply<true>(s, a, static_cast<cudaStream_t>(stream), "bn_bwd_apply_act");
 }
 
 }  // extern "C"
