@@ -269,16 +269,22 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
     constexpr int NP = EPV / 2;
     f32x2 pacc0[V][NP], pacc1[V][NP];  // packed float32 pairs
     float sv[V], mrun[V];
-    float rv[V][EPV];  // row-stationary vector (bwd)
+    // Row-stationary vector of the backward passes (gout of the row / feat of the source), needed only when the
+    // row is finalised.  It is kept as loaded (packed) and requested one row ahead, so that nothing waits for it.
+    uint4 rvq[V], rvq_next[V];
 #pragma unroll
     for (int v = 0; v < V; ++v) {
         sv[v] = 0.f;
         mrun[v] = SAR_NEG_INF;
 #pragma unroll
         for (int k = 0; k < NP; ++k) pacc0[v][k] = pacc1[v][k] = zero2();
-#pragma unroll
-        for (int e = 0; e < EPV; ++e) rv[v][e] = 0.f;
+        rvq[v] = rvq_next[v] = make_uint4(0u, 0u, 0u, 0u);
     }
+    auto request_rowvec = [&](long long row_, uint4 (&dst)[V]) {
+        const uint4 *rp = reinterpret_cast<const uint4 *>(a.rowvec) + row_ * n_vec + gl;
+#pragma unroll
+        for (int v = 0; v < V; ++v) dst[v] = vok[v] ? __ldg(rp + v * G) : make_uint4(0u, 0u, 0u, 0u);
+    };
 
     const int deg_l = (lane < nrows && !excluded) ? (int)((ee - eb) > 0x3fffffff ? 0x3fffffff : (ee - eb)) : 0;
     const unsigned excl_all = __ballot_sync(0xffffffffu, excluded);
@@ -408,6 +414,12 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
         }
         __syncwarp();
 
+        if constexpr (kDst || kSrc) {
+            if (mode_ == 0) {  // the first row that starts in this chunk (a continued row brought its vector along)
+                const int first = cont ? 1 : 0;
+                if (first < nr) request_rowvec(row0 + r + first, rvq_next);
+            }
+        }
         // ---- start the gather ring now: the first S slots need only the column ids ----------------
         auto issue = [&](int s_, unsigned dst_s) {
             const int col = lds_s32(sj_s + s_ * (EPW * 4));  // -1 past the row's / chunk's end: zero fill
@@ -647,13 +659,19 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
             const long long row = row0 + r + ri;
             const bool row_starts = !(cont && ri == 0);
             const bool row_ends = !(unfinished && ri == nr - 1);
+            if constexpr (kDst || kSrc) {
+                if (mode_ == 0 && row_starts) {
+#pragma unroll
+                    for (int v = 0; v < V; ++v) rvq[v] = rvq_next[v];
+                    if (ri + 1 < nr) request_rowvec(row + 1, rvq_next);
+                }
+            }
             if (s_end == s && !(write_empty && row_starts)) continue;  // no edges here, nothing to write
             if (row_starts) {
                 if constexpr (kFwdMode) {
 #pragma unroll
                     for (int v = 0; v < V; ++v) mrun[v] = sc2[ri * Hp + hv[v]];
                 }
-                if constexpr (kDst || kSrc) load_row_vec<T, G, V>(a.rowvec, row, n_vec, gl, vok, rv);
             }
             for (; s < s_end; ++s) {
                 cp_async_wait<S - 1>();  // this lane's copies of slot s have landed
@@ -788,9 +806,10 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                             if (lead[v]) rec[2 * rowf + hv[v]] = sv[v];
                     }
                 } else {
-                    float pA[V], pB[V];
+                    float pA[V], pB[V], rv[V][EPV];
 #pragma unroll
                     for (int v = 0; v < V; ++v) {
+                        Elem<T>::unpack(rvq[v], rv[v]);
                         pA[v] = pB[v] = 0.f;
 #pragma unroll
                         for (int e = 0; e < EPV; ++e) {
@@ -836,9 +855,10 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                             if (lead[v]) rec[2 * rowf + hv[v]] = sv[v];
                     }
                 } else {
-                    float pC[V];
+                    float pC[V], rv[V][EPV];
 #pragma unroll
                     for (int v = 0; v < V; ++v) {
+                        Elem<T>::unpack(rvq[v], rv[v]);
                         pC[v] = 0.f;
 #pragma unroll
                         for (int e = 0; e < EPV; ++e) pC[v] = fmaf(rv[v][e], acc1[v][e], pC[v]);
