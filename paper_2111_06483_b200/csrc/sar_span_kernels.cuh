@@ -420,6 +420,25 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                 if (first < nr) request_rowvec(row0 + r + first, rvq_next);
             }
         }
+        // ---- the score terms er[col, :] of every position travel asynchronously too (forward and destination-major
+        // passes with heads in groups of four): one 16-byte copy per position and head group straight into the
+        // position's weight record, all in flight together and with the ring's first slots, instead of register
+        // loads whose latency every sweep of the score phase would wait for.  Each lane copies the positions it
+        // will score itself (q = lane mod 32).
+        constexpr bool kErAsyncMode = kFwdMode || kDst;
+        const bool er_async = kErAsyncMode && (GEO ? true : a.hvec != 0);
+        if constexpr (kErAsyncMode) {
+            if (er_async) {
+                const unsigned sw_s = (unsigned)__cvta_generic_to_shared(sw);
+                for (int q = lane; q < npos; q += 32) {
+                    const int col = sj[q];
+                    const float *src = a.er + (long long)(col < 0 ? 0 : col) * H;
+                    for (int h = 0; h < H; h += 4)
+                        cp_async16_s(sw_s + (unsigned)(((q << lgHp) + h) * 4), src + h, col >= 0 ? 16 : 0);
+                }
+                cp_async_commit();
+            }
+        }
         // ---- start the gather ring now: the first S slots need only the column ids ----------------
         auto issue = [&](int s_, unsigned dst_s) {
             const int col = lds_s32(sj_s + s_ * (EPW * 4));  // -1 past the row's / chunk's end: zero fill
@@ -430,6 +449,12 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
         };
 #pragma unroll
         for (int s_ = 0; s_ < S; ++s_) issue(s_, stage_s + s_ * (V * 512));
+        if constexpr (kErAsyncMode) {
+            if (er_async) {
+                cp_async_wait<S>();  // the score terms have landed (the ring's S groups may still be in flight)
+                __syncwarp();
+            }
+        }
 
         // ---- stage C: weight records, two positions per lane and sweep, all their heads -----------
         if constexpr (MODE == kSumW) {
@@ -476,7 +501,8 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
 #pragma unroll
                             for (int u = 0; u < 2; ++u) {
                                 e4[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                                if (col[u] >= 0) e4[u] = __ldg(reinterpret_cast<const float4 *>(a.er + (long long)col[u] * H + h));
+                                if (col[u] >= 0)  // staged in the position's own record (overwritten by its weights below)
+                                    e4[u] = *reinterpret_cast<const float4 *>(reinterpret_cast<const float *>(sw) + ((q0 + 32 * u) << lgHp) + h);
                             }
 #pragma unroll
                             for (int u = 0; u < 2; ++u) {
