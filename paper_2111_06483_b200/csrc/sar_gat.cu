@@ -93,7 +93,7 @@ static sar_status check_part(const sar_part *g, bool need_csc) {
 
 
 // ---- span kernels ---------------------------------------------------------------------------------
-constexpr int kCapFwd = 256, kCapDst = 256, kCapSrc = 128, kCapSum = 256;
+constexpr int kCapFwd = 256, kCapDst = 256, kCapSrc = 192, kCapSum = 256;
 constexpr int kCapSeg = 128;  // capacity of the segment launches (segments hold at most the plan threshold)
 constexpr int kMinBlocksFwd = 24, kMinBlocksBwd = 20;  // resident blocks per SM the register budget is cut for
 
