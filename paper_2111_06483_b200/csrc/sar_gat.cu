@@ -99,7 +99,7 @@ constexpr int kMinBlocksFwd = 24, kMinBlocksBwd = 20;  // resident blocks per SM
 
 static int rows_per_span(long long n_rows, long long nnz, int cap) {
     const double avg = n_rows > 0 ? (double)nnz / (double)n_rows : 0.0;
-    int R = avg > 0.5 ? (int)(0.75 * cap / avg + 0.5) : kMaxSpanRows;  // about 3/4 cap edges per span
+    int R = avg > 0.5 ? (int)(1.0 * cap / avg + 0.5) : kMaxSpanRows;  // about cap edges per span (the long rows counted in avg are skipped)
     if (R < 1) R = 1;
     if (R > kMaxSpanRows) R = kMaxSpanRows;
     return R;
