@@ -4,11 +4,26 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
 One STEP is one pass of the whole hot path over one batch of synthetic node tensors: for each of
-the workload's layers the fused forward over the K source partitions, then for each layer the
-rematerialising backward (destination-major and source-major passes).  The graph (CSR, CSC,
-long-row plan) is prepared once by the library before the timed region and its time is reported
-as `prep_ms`; a graph is fixed across the training steps the paper times (its partitioning is an
-offline step).
+the workload's layers the forward over the K source partitions, then for each layer the
+rematerialising backward (destination-major and source-major passes).  Two SCHEDULES of the K
+partitions are timed on the same inputs:
+
+  fused       one row-stationary walk per pass over the un-split graph: sources ascend within a row, so
+              a row meets the partitions in order and the running state never leaves the registers.  The
+              kernels see ONE partition (the K bounds only describe where the partitions lie);
+  sequential  Algorithm 1 / Algorithm 2 call by call: K calls of sar_gat_fwd with the running numerator,
+              max and normaliser in device memory, then sar_gat_bwd_prepare and K calls of sar_gat_bwd.
+
+`value` comes from the schedule named in `config.schedule` (--schedule, default fused); both are
+reported under `schedules`.  The graph (CSR, CSC, per-partition sub-graphs, long-row plans) is
+prepared once by the library before the timed region and its time is reported as `prep_ms`; a graph
+is fixed across the training steps the paper times (its partitioning is an offline step).
+
+The default run (workload large, one GPU) also times, briefly, the other named workloads
+(`workloads`), the sum aggregation on the headline graph with the same row width as a measured
+ceiling for any gather kernel on this input (`gather_ceiling`), a deliberately plain variant that
+stores the attention coefficients (`storing_baseline`), the end-to-end path through host buffers
+(`e2e`) and the CPU oracle (`cpu_baseline`).
 
 Prints ONE JSON line (rank 0).  `value` = edges x layers processed per second by all ranks (each
 rank runs an independent replica: the path does not shard, so scaling is "weak" with no
@@ -17,8 +32,8 @@ collective on the data path).
 from __future__ import annotations
 
 import argparse
+import gc
 import json
-import math
 import os
 import subprocess
 import sys
@@ -31,6 +46,7 @@ if ROOT not in sys.path:
 
 METRIC = "gat_fwd_bwd_edges_per_sec"
 UNIT = "edges/s"
+TARGET_FRAC = 0.60  # of the HBM roofline, on the largest single-GPU graph
 
 
 def parse_args():
@@ -41,8 +57,11 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", help="tiny | seqpart | medium | dense | large")
     ap.add_argument("--dtype", default=None, help="f32 | bf16 (default: the workload's last listed dtype)")
-    ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (debugging only)")
+    ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (debugging and profiling)")
     ap.add_argument("--threshold", type=int, default=None, help="long-row split threshold")
+    ap.add_argument("--schedule", default="fused", choices=["fused", "sequential"],
+                    help="which schedule of the K partitions `value` is taken from (both are timed)")
+    ap.add_argument("--only-schedule", action="store_true", help="time only the schedule named by --schedule")
     ap.add_argument("--glue", action="store_true",
                     help="also run the rest of the layer each step: dense projection z = h W (bf16 workloads), score "
                          "projections, ReLU, and their backward passes (default: aggregation kernels only)")
@@ -57,6 +76,8 @@ def parse_args():
                          "on the workload's graph instead of the attention stack; its own metric, not the headline")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true",
+                    help="skip the other workloads, the gather ceiling and the storing baseline")
     ap.add_argument("--cpu-sample", type=float, default=0.05, help="fraction of the workload the oracle is timed on")
     return ap.parse_args()
 
@@ -97,14 +118,27 @@ def bytes_layer_fwd_bwd(n, e, H, F, b):
     return 3 * idx_bytes(n, e) + 4 * n * H * F * b + 10 * n * H * 4
 
 
+def bytes_spmm(n, e, F, b):
+    # one direction of the sum aggregation: indices, every input row once, every output row once
+    return idx_bytes(n, e) + 2 * n * F * b
+
+
+def state_bytes_sequential(n, H, F, K, L):
+    """Bytes of running state (float32 numerator, max, normaliser) the call-by-call forward writes and
+    reads back between partitions, per step: every partition but the last writes it, every one but the
+    first reads it (Algorithm 1 keeps it in the worker's memory)."""
+    per = n * H * F * 4 + 2 * n * H * 4
+    return L * 2 * max(K - 1, 0) * per
+
+
 KERNEL_BYTES = {"gat_fwd": bytes_fwd, "gat_bwd_dst": bytes_bwd_dst, "gat_bwd_src": bytes_bwd_src}
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one pass (rows + segments + merge launches),
-# from the one-pass ncu capture at full size whose launch list is summarised under profiles/.
-NCU_TRAFFIC_BYTES = {
-    ("large", "bf16", "gat_fwd"): 81.89e9,
-    ("large", "bf16", "gat_bwd_dst"): 84.07e9,
-    ("large", "bf16", "gat_bwd_src"): 89.08e9,
+# DRAM traffic of one pass (rows + segments + merge launches), dram__bytes_read.sum + dram__bytes_write.sum.
+# Measured with ncu on the workload scaled to 10 % (feature arrays of 512 MB, a few GB on the device, one
+# launch of each kernel) and scaled to a full launch by the edge count; see profiles/.  None: not captured
+# for the kernels of this tree.
+NCU_TRAFFIC = {
+    # (workload, storage dtype, pass): (bytes per full-size pass, source)
 }
 
 
@@ -119,17 +153,34 @@ def max_over_ranks(value: float, dist=None, device="cpu") -> float:
 
 
 def group_passes(kernels: dict) -> dict:
-    """Launch names -> passes: 'gat_fwd', 'gat_fwd_seg', 'gat_fwd_merge' together are one pass over the edges."""
+    """Launch names -> passes: 'gat_fwd', 'gat_fwd_seg', 'gat_fwd_merge' together are one pass over the edges.
+    `ms` adds the launches' average durations (one launch of each per pass: the fused schedule); `total_ms`
+    adds everything the pass's launches took inside the timed region (any schedule)."""
     passes = {}
     for name, v in kernels.items():
         base = name
         for suffix in ("_seg", "_merge"):
             if name.endswith(suffix):
                 base = name[:-len(suffix)]
-        p_ = passes.setdefault(base, {"ms": 0.0, "launches": []})
+        p_ = passes.setdefault(base, {"ms": 0.0, "total_ms": 0.0, "launches": []})
         p_["ms"] += v["avg_ms"]
+        p_["total_ms"] += v.get("total_ms", v["avg_ms"] * v.get("launches", 1))
         p_["launches"].append(name)
     return passes
+
+
+def pass_table(kernels, passes_per_run, n, e, H, F, b, peak):
+    """Per pass over the E edges: milliseconds (all its launches, averaged over the passes of the timed
+    region), edges/s and the fraction of the compulsory-byte roofline."""
+    out = {}
+    for name, p_ in group_passes(kernels).items():
+        if name not in KERNEL_BYTES or passes_per_run <= 0:
+            continue
+        ms = p_["total_ms"] / passes_per_run
+        alg = KERNEL_BYTES[name](n, e, H, F, b)
+        out[name] = {"ms": ms, "edges_per_sec": e / (ms * 1e-3), "algorithmic_bytes": alg,
+                     "frac_of_roofline": alg / (ms * 1e-3) / 1e9 / peak, "launches": sorted(p_["launches"])}
+    return out
 
 
 # --------------------------------------------------------------------------------------------------
@@ -191,6 +242,13 @@ class ClockSampler:
         return out
 
 
+def gpu_index_of(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+    if vis.replace(",", "").isdigit():
+        return int(vis.split(",")[local_rank])
+    return local_rank
+
+
 # --------------------------------------------------------------------------------------------------
 # the CPU oracle as a timed baseline (reference arm and cpu_baseline leg)
 # --------------------------------------------------------------------------------------------------
@@ -243,67 +301,253 @@ def run_reference(args, rank):
     print(json.dumps(line), flush=True)
 
 
+def cpu_baseline_leg(cfg_name, dtype, fraction, slope):
+    """The oracle as it stands on the host cores: all cores on a `fraction` sample of the workload, and
+    one thread on a sample an eighth of that (so that both end within seconds)."""
+    import oracle
+    import workloads
+    cfg = workloads.CONFIGS[cfg_name]
+    small, s_src, s_dst, h = oracle_sample(cfg, dtype, min(1.0, fraction))
+    cores = oracle.num_threads()
+    secs = oracle_step(small, s_src, s_dst, h, slope)
+    out = {"value": small.e / secs, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": f"{small.name}: n={small.n} e={small.e} H={small.heads} F={small.feat}, one layer fwd+bwd, "
+                     f"{secs:.1f} s"}
+    tiny, t_src, t_dst, th = oracle_sample(cfg, dtype, min(1.0, fraction / 8))
+    oracle.set_num_threads(1)
+    try:
+        secs1 = oracle_step(tiny, t_src, t_dst, th, slope)
+    finally:
+        oracle.set_num_threads(cores)
+    out["single_thread"] = {"value": tiny.e / secs1, "unit": UNIT, "cores": 1,
+                            "sample": f"{tiny.name}: n={tiny.n} e={tiny.e}, one layer fwd+bwd, {secs1:.1f} s"}
+    return out
+
+
 # --------------------------------------------------------------------------------------------------
-# our arm
+# the aggregation stack on the device
 # --------------------------------------------------------------------------------------------------
 
-def run_ours(args, rank, world, local_rank):
+class AggStack:
+    """L chained aggregation layers of one workload: the graph and every node tensor on the device.
+
+    feat^{l+1} = out^l with seeded el^l, er^l; the backward pass feeds dfeat^{l+1} as gout of layer l."""
+
+    def __init__(self, cfg, dtype, dev, ids="permuted", threshold=None, parts=True):
+        import torch
+        import workloads
+        from paper_2111_06483_b200 import api, binding as B
+        self.B, self.api, self.torch = B, api, torch
+        self.cfg, self.dtype, self.dev = cfg, dtype, dev
+        self.tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+        self.b = 2 if dtype == "bf16" else 4
+        n, H, F, L, K = cfg.n, cfg.heads, cfg.feat, cfg.layers, cfg.k
+        self.n, self.H, self.F, self.L, self.K = n, H, F, L, K
+        self.threshold = threshold if threshold is not None else api.DEFAULT_THRESHOLD
+        src, dst = workloads.make_graph(cfg, device=dev, permute=ids == "permuted")
+        self.e = src.numel()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        self.g = api.Graph.from_coo(n, src, dst, k=K, threshold=self.threshold, build_parts=parts and K > 1)
+        torch.cuda.synchronize()
+        self.prep_ms = 1e3 * (time.perf_counter() - t0)
+        del src, dst
+        tdt = self.tdt
+        self.feats = [workloads.normal_tensor((n, H, F), cfg.seed, 10, device=dev, dtype=tdt)]
+        self.feats += [torch.empty((n, H, F), dtype=tdt, device=dev) for _ in range(L)]
+        self.els = [workloads.normal_tensor((n, H), cfg.seed, 16 * l + 12, device=dev) for l in range(L)]
+        self.ers = [workloads.normal_tensor((n, H), cfg.seed, 16 * l + 13, device=dev) for l in range(L)]
+        self.gout = workloads.normal_tensor((n, H, F), cfg.seed, 11, device=dev, dtype=tdt)
+        self.gbuf = [torch.empty((n, H, F), dtype=tdt, device=dev) for _ in range(2)]
+        f32 = lambda: torch.empty((n, H), dtype=torch.float32, device=dev)
+        self.ms, self.ds = [f32() for _ in range(L)], [f32() for _ in range(L)]
+        self.dels, self.ders = [f32() for _ in range(L)], [f32() for _ in range(L)]
+        g = self.g
+        nbytes = B.sar_gat_workspace_bytes(g.whole, H, F, B._dtype(self.feats[0]))
+        for p in g.parts:
+            nbytes = max(nbytes, B.sar_gat_workspace_bytes(p, H, F, B._dtype(self.feats[0])))
+        self.ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=dev)
+        self.acc = None
+        cut = lambda t: [t[g.bounds[q]:] for q in range(K)]
+        self.feat_q = [cut(f) for f in self.feats]
+        self.er_q = [cut(x) for x in self.ers]
+        self.der_q = [cut(x) for x in self.ders]
+        self.gbuf_q = [cut(x) for x in self.gbuf]
+
+    def can_run_sequential(self):
+        return self.K == 1 or bool(self.g.parts)
+
+    def step_fused(self):
+        B, g, c = self.B, self.g, self.cfg
+        H, F, L = self.H, self.F, self.L
+        for l in range(L):
+            B.sar_gat_fwd_fused(g.whole, g.bounds, self.feat_q[l], self.els[l], self.er_q[l], H, F, c.slope, self.ms[l],
+                                self.ds[l], self.feats[l + 1], self.ws)
+        gin = self.gout
+        for i, l in enumerate(reversed(range(L))):
+            B.sar_gat_bwd_fused(g.whole, g.bounds, self.feat_q[l], self.els[l], self.er_q[l], self.ms[l], self.ds[l], gin,
+                                H, F, c.slope, self.gbuf_q[i % 2], self.dels[l], self.der_q[l], self.ws)
+            gin = self.gbuf[i % 2]
+
+    def step_sequential(self):
+        """Algorithm 1 and Algorithm 2 call by call: the running state (numerator, max, normaliser) lives in
+        device memory between the K forward calls; the backward pass rebuilds each partition's attention."""
+        B, g, c, torch = self.B, self.g, self.cfg, self.torch
+        H, F, L, K, n = self.H, self.F, self.L, self.K, self.n
+        parts = g.parts if K > 1 else [g.whole]
+        if K > 1 and self.acc is None:
+            self.acc = torch.empty((n, H, F), dtype=torch.float32, device=self.dev)
+        for l in range(L):
+            for q, part in enumerate(parts):
+                flags = (B.SAR_FIRST if q == 0 else 0) | (B.SAR_LAST if q == K - 1 else 0)
+                s0, s1 = g.bounds[q], g.bounds[q + 1]
+                B.sar_gat_fwd(part, self.feats[l][s0:s1], self.els[l], self.ers[l][s0:s1], H, F, c.slope, flags, self.acc,
+                              self.ms[l], self.ds[l], self.feats[l + 1], self.ws)
+        gin = self.gout
+        for i, l in enumerate(reversed(range(L))):
+            if K > 1:
+                B.sar_gat_bwd_prepare(n, H, F, self.feats[l + 1], False, gin, self.els[l], self.ms[l], self.ds[l], None,
+                                      self.ws)
+            for q, part in enumerate(parts):
+                flags = (B.SAR_FIRST if q == 0 else 0) | (B.SAR_LAST if q == K - 1 else 0)
+                s0, s1 = g.bounds[q], g.bounds[q + 1]
+                B.sar_gat_bwd(part, self.feats[l][s0:s1], self.els[l], self.ers[l][s0:s1], self.ms[l], self.ds[l], gin, H,
+                              F, c.slope, flags, self.gbuf[i % 2][s0:s1], self.dels[l], self.ders[l][s0:s1], self.ws)
+            gin = self.gbuf[i % 2]
+
+    def step(self, schedule):
+        return self.step_fused if schedule == "fused" else self.step_sequential
+
+
+def measure(step, steps, warmup, dist=None, dev=None, clocks_gpu=None):
+    """`warmup` untimed steps, then exactly `steps` steps between a barrier + synchronize on both sides,
+    timed with CUDA events on the launching stream; per-kernel times from the library's launch observer."""
+    import torch
+    from paper_2111_06483_b200 import binding as B
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(clocks_gpu) if clocks_gpu is not None else None
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with B.LaunchTimer() as lt:
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
+    torch.cuda.synchronize()
+    if dist:
+        dist.barrier()
+    elapsed_ms = max_over_ranks(e0.elapsed_time(e1), dist, dev)
+    clocks = sampler.stop() if sampler else None
+    kernels = lt.summary()
+    return {"ms_per_step": elapsed_ms / steps, "kernels": kernels, "clocks": clocks,
+            "launches": sum(v["launches"] for v in kernels.values())}
+
+
+def schedule_entry(st: AggStack, schedule, r, steps, peak):
+    n, e, H, F, b, L, K = st.n, st.e, st.H, st.F, st.b, st.L, st.K
+    entry = {
+        "ms_per_step": r["ms_per_step"], "steps": steps, "edges_per_sec": L * e / (r["ms_per_step"] * 1e-3),
+        "partitions_seen_by_the_kernels": 1 if schedule == "fused" else K,
+        "launches_per_step": r["launches"] // max(steps, 1),
+        "passes": pass_table(r["kernels"], steps * L, n, e, H, F, b, peak),
+        "step_frac_of_roofline": L * bytes_layer_fwd_bwd(n, e, H, F, b) / (r["ms_per_step"] * 1e-3) / 1e9 / peak,
+    }
+    if schedule == "sequential":
+        entry["state_bytes_per_step"] = state_bytes_sequential(n, H, F, K, L)
+        entry["calls"] = f"{K} x sar_gat_fwd, sar_gat_bwd_prepare + {K} x sar_gat_bwd per layer"
+    else:
+        entry["calls"] = "sar_gat_fwd_fused, sar_gat_bwd_fused per layer (one walk over the un-split graph)"
+    if r.get("clocks"):
+        entry["clocks"] = r["clocks"]
+    return entry
+
+
+# --------------------------------------------------------------------------------------------------
+# legs of the default run
+# --------------------------------------------------------------------------------------------------
+
+def time_spmm(g, x, gout, steps, warmup, peak, n, e, b):
+    """Sum aggregation forward (CSR) + its backward (the same call on the transposed graph)."""
+    import torch
+    from paper_2111_06483_b200 import binding as B
+    F = x.shape[1]
+    out, dx = torch.empty_like(x), torch.empty_like(x)
+    fwd, bwd = g.whole, g.whole.transposed()
+    ws = torch.empty(max(B.sar_spmm_workspace_bytes(fwd, F, B._dtype(x)), B.sar_spmm_workspace_bytes(bwd, F, B._dtype(x)), 256),
+                     dtype=torch.uint8, device=x.device)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    f_ms = b_ms = 0.0
+    for it in range(warmup + steps):
+        ev[0].record()
+        B.sar_spmm_agg(fwd, x, F, B.SAR_FIRST | B.SAR_LAST, None, out, ws)
+        ev[1].record()
+        B.sar_spmm_agg(bwd, gout, F, B.SAR_FIRST | B.SAR_LAST, None, dx, ws)
+        ev[2].record()
+        torch.cuda.synchronize()
+        if it >= warmup:
+            f_ms += ev[0].elapsed_time(ev[1]) / steps
+            b_ms += ev[1].elapsed_time(ev[2]) / steps
+    alg = bytes_spmm(n, e, F, b)
+    return {"columns": F, "csr_ms": f_ms, "csc_ms": b_ms, "ms_per_step": f_ms + b_ms,
+            "edges_per_sec": e / ((f_ms + b_ms) * 1e-3), "algorithmic_bytes_per_direction": alg,
+            "frac_of_roofline": 2 * alg / ((f_ms + b_ms) * 1e-3) / 1e9 / peak,
+            "gathered_bytes_per_direction": e * F * b}
+
+
+def extra_workloads(dev, peak, args):
+    """The other named workloads, a few steps each (configs 2-4 and the sum aggregation of config 3)."""
     import torch
     import workloads
-    from paper_2111_06483_b200 import api, binding as B
+    from paper_2111_06483_b200 import api
+    out = {}
+    plan = [("seqpart", "f32", ("fused", "sequential")), ("medium", "f32", ("fused",)),
+            ("medium", "bf16", ("fused", "sequential")), ("dense", "bf16", ("fused", "sequential"))]
+    steps, warmup = 5, 3
+    for name, dtype, schedules in plan:
+        cfg = workloads.CONFIGS[name]
+        need = (6 * cfg.n * cfg.heads * cfg.feat * (2 if dtype == "bf16" else 4) + 4 * cfg.n * cfg.heads * cfg.feat
+                + 40 * cfg.e) * 1.3
+        if torch.cuda.get_device_properties(dev).total_memory < need:
+            out[f"{name}_{dtype}"] = {"skipped": "not enough device memory"}
+            continue
+        st = AggStack(cfg, dtype, dev, ids=args.ids, parts="sequential" in schedules)
+        entry = {"n": st.n, "e": st.e, "heads": st.H, "feat_per_head": st.F, "layers": st.L, "partitions": st.K,
+                 "storage_dtype": dtype, "prep_ms": st.prep_ms, "schedules": {}}
+        for sch in schedules:
+            r = measure(st.step(sch), steps, warmup, clocks_gpu=None)
+            entry["schedules"][sch] = schedule_entry(st, sch, r, steps, peak)
+        out[f"{name}_{dtype}"] = entry
+        if name == "medium" and cfg.spmm_feat:
+            x = workloads.normal_tensor((st.n, cfg.spmm_feat), cfg.seed, 20, device=dev, dtype=st.tdt)
+            go = workloads.normal_tensor((st.n, cfg.spmm_feat), cfg.seed, 21, device=dev, dtype=st.tdt)
+            out[f"spmm_{name}_{dtype}"] = time_spmm(st.g, x, go, steps, warmup, peak, st.n, st.e, st.b)
+            del x, go
+        del st
+        gc.collect()
+        torch.cuda.empty_cache()
+    return out
 
-    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
-    dev = torch.device(f"cuda:{local_rank}")
-    torch.cuda.set_device(dev)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=dev)
 
-    cfg = workloads.CONFIGS[args.workload]
-    if args.scale != 1.0:
-        cfg = cfg.scaled(args.scale)
-    dtype = args.dtype or cfg.dtypes[-1]
-    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
-    b = 2 if dtype == "bf16" else 4
-    n, H, F, L, K = cfg.n, cfg.heads, cfg.feat, cfg.layers, cfg.k
-    threshold = args.threshold if args.threshold is not None else api.DEFAULT_THRESHOLD
+def make_glue_step(args, st: AggStack):
+    """--glue: the rest of the layer around the aggregation (fused schedule only)."""
+    import torch
+    import workloads
+    B, g, cfg, dev = st.B, st.g, st.cfg, st.dev
+    n, H, F, L, tdt = st.n, st.H, st.F, st.L, st.tdt
+    feats, els, ers, ms, ds, dels, ders = st.feats, st.els, st.ers, st.ms, st.ds, st.dels, st.ders
+    gout, gbuf, ws = st.gout, st.gbuf, st.ws
+    feat_q, er_q, der_q, gbuf_q = st.feat_q, st.er_q, st.der_q, st.gbuf_q
+    cut = lambda t: [t[g.bounds[q]:] for q in range(st.K)]
+    a_ls = [workloads.normal_tensor((H, F), cfg.seed, 16 * l + 14, device=dev) / F ** 0.5 for l in range(L)]
+    a_rs = [workloads.normal_tensor((H, F), cfg.seed, 16 * l + 15, device=dev) / F ** 0.5 for l in range(L)]
+    da_l, da_r = torch.empty((H, F), device=dev), torch.empty((H, F), device=dev)
+    pws = torch.empty(B.sar_gat_project_workspace_bytes(H, F), dtype=torch.uint8, device=dev)
 
-    # ---- inputs (seeded, generated on the device; same recipe as the parity tests) --------------
-    src, dst = workloads.make_graph(cfg, device=dev, permute=args.ids == "permuted")
-    e = src.numel()
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    g = api.Graph.from_coo(n, src, dst, k=K, threshold=threshold)
-    torch.cuda.synchronize()
-    prep_ms = 1e3 * (time.perf_counter() - t0)
-    del src, dst
-    feats = [workloads.normal_tensor((n, H, F), cfg.seed, 10, device=dev, dtype=tdt)]
-    feats += [torch.empty((n, H, F), dtype=tdt, device=dev) for _ in range(L)]
-    els = [workloads.normal_tensor((n, H), cfg.seed, 16 * l + 12, device=dev) for l in range(L)]
-    ers = [workloads.normal_tensor((n, H), cfg.seed, 16 * l + 13, device=dev) for l in range(L)]
-    gout = workloads.normal_tensor((n, H, F), cfg.seed, 11, device=dev, dtype=tdt)
-    gbuf = [torch.empty((n, H, F), dtype=tdt, device=dev) for _ in range(2)]
-    ms = [torch.empty((n, H), dtype=torch.float32, device=dev) for _ in range(L)]
-    ds = [torch.empty((n, H), dtype=torch.float32, device=dev) for _ in range(L)]
-    dels = [torch.empty((n, H), dtype=torch.float32, device=dev) for _ in range(L)]
-    ders = [torch.empty((n, H), dtype=torch.float32, device=dev) for _ in range(L)]
-    ws = api.gat_workspace(g.whole, H, F, tdt)
-    cut = lambda t: [t[g.bounds[q]:] for q in range(K)]
-    feat_q = [cut(f) for f in feats]
-    er_q = [cut(x) for x in ers]
-    der_q = [cut(x) for x in ders]
-    gbuf_q = [cut(x) for x in gbuf]
-
-    glue = args.glue
-    if glue:
-        a_ls = [workloads.normal_tensor((H, F), cfg.seed, 16 * l + 14, device=dev) / F ** 0.5 for l in range(L)]
-        a_rs = [workloads.normal_tensor((H, F), cfg.seed, 16 * l + 15, device=dev) / F ** 0.5 for l in range(L)]
-        da_l, da_r = torch.empty((H, F), device=dev), torch.empty((H, F), device=dev)
-        pws = torch.empty(B.sar_gat_project_workspace_bytes(H, F), dtype=torch.uint8, device=dev)
-
-    if glue and tdt == torch.bfloat16 and (H * F) % 8 == 0:
+    if tdt == torch.bfloat16 and (H * F) % 8 == 0:
         # the whole layer: dense projection z = h W on the tensor cores, scores, aggregation, ReLU
         D = H * F
         Ws = [(workloads.normal_tensor((D, D), cfg.seed, 16 * l + 9, device=dev) / D ** 0.5).to(tdt) for l in range(L)]
@@ -313,8 +557,7 @@ def run_ours(args, rank, world, local_rank):
         lws = torch.empty(B.sar_linear_workspace_bytes(n, D, D), dtype=torch.uint8, device=dev)
         flat = lambda x: x.view(n, D)
 
-        bnd = args.bn_dropout
-        if bnd:
+        if args.bn_dropout:
             # layer l's aggregation output stays in feats[l+1] (batch normalisation needs it again in the backward
             # pass); hs[l+1] = dropout(ReLU(BN(feats[l+1]))) is the next layer's input
             hs = [feats[0]] + [torch.empty((n, H, F), dtype=tdt, device=dev) for _ in range(L - 1)]
@@ -353,6 +596,7 @@ def run_ours(args, rank, world, local_rank):
                         B.sar_bn_bwd_apply_act(x, bn_mean[l - 1], bn_rstd[l - 1], None, gh, flat(hs[l]), act, p_drop,
                                                seeds[l - 1], bn_s0, bn_s1, 1.0 / n, flat(gx_bn))
                         gin = gx_bn
+            return step
 
         def step_plain():
             for l in range(L):
@@ -375,137 +619,169 @@ def run_ours(args, rank, world, local_rank):
                 if l > 0:
                     B.sar_relu_bwd(feats[l], gbuf[1])
                 gin = gbuf[1]
+        return step_plain
 
-        if not bnd:
-            step = step_plain
-    else:
-        def step():
-            for l in range(L):
-                if glue:  # the ReLU closing layer l-1 runs inside layer l's projection
-                    B.sar_gat_project(feats[l], a_ls[l], a_rs[l], els[l], ers[l], B.SAR_GLUE_RELU if l > 0 else 0)
-                B.sar_gat_fwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], H, F, cfg.slope, ms[l], ds[l],
-                                    feats[l + 1], ws)
-            if glue:
-                B.sar_relu(feats[L])
-            gin = gout
-            if glue:
-                B.sar_relu_bwd(feats[L], gin)  # masks gout in place on the first pass; the same mask every step
-            for i, l in enumerate(reversed(range(L))):
-                B.sar_gat_bwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], ms[l], ds[l], gin, H, F, cfg.slope,
-                                    gbuf_q[i % 2], dels[l], der_q[l], ws)
-                gin = gbuf[i % 2]
-                if glue:
-                    B.sar_gat_project_bwd(feats[l], a_ls[l], a_rs[l], dels[l], ders[l], gin, da_l, da_r, pws,
-                                          B.SAR_GLUE_RELU if l > 0 else 0)
+    def step():
+        for l in range(L):  # the ReLU closing layer l-1 runs inside layer l's projection
+            B.sar_gat_project(feats[l], a_ls[l], a_rs[l], els[l], ers[l], B.SAR_GLUE_RELU if l > 0 else 0)
+            B.sar_gat_fwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], H, F, cfg.slope, ms[l], ds[l],
+                                feats[l + 1], ws)
+        B.sar_relu(feats[L])
+        gin = gout
+        B.sar_relu_bwd(feats[L], gin)  # masks gout in place on the first pass; the same mask every step
+        for i, l in enumerate(reversed(range(L))):
+            B.sar_gat_bwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], ms[l], ds[l], gin, H, F, cfg.slope,
+                                gbuf_q[i % 2], dels[l], der_q[l], ws)
+            gin = gbuf[i % 2]
+            B.sar_gat_project_bwd(feats[l], a_ls[l], a_rs[l], dels[l], ders[l], gin, da_l, da_r, pws,
+                                  B.SAR_GLUE_RELU if l > 0 else 0)
+    return step
+
+
+def time_e2e(st: AggStack, args, dist, world):
+    """The same metric through sar_gat_stack_host with pinned HOST buffers: every step copies all its inputs in
+    and all its results out inside the timed region."""
+    import torch
+    import workloads
+    B, g, cfg, dev = st.B, st.g, st.cfg, st.dev
+    n, H, F, L, tdt, b = st.n, st.H, st.F, st.L, st.tdt, st.b
+    pin = lambda shape, dt: torch.empty(shape, dtype=dt).pin_memory()
+    h_feat0 = pin((n, H, F), tdt)
+    h_gout = pin((n, H, F), tdt)
+    h_out, h_dfeat = pin((n, H, F), tdt), pin((n, H, F), tdt)
+    h_el = [pin((n, H), torch.float32) for _ in range(L)]
+    h_er = [pin((n, H), torch.float32) for _ in range(L)]
+    h_del = [pin((n, H), torch.float32) for _ in range(L)]
+    h_der = [pin((n, H), torch.float32) for _ in range(L)]
+    h_feat0.copy_(workloads.normal_tensor((n, H, F), cfg.seed, 10, device=dev, dtype=tdt))
+    h_gout.copy_(workloads.normal_tensor((n, H, F), cfg.seed, 11, device=dev, dtype=tdt))
+    for l in range(L):
+        h_el[l].copy_(st.els[l])
+        h_er[l].copy_(st.ers[l])
+    # two working sets: the pipelined mode overlaps the copies of step t+1 with the kernels of step t
+    one = (B.sar_gat_stack_arena_bytes(g.whole, L, H, F, B._dtype(h_feat0)) + 255) // 256 * 256
+    arena = torch.empty(2 * one, dtype=torch.uint8, device=dev)
+
+    def host_step():
+        B.sar_gat_stack_host(g.whole, g.bounds, H, F, cfg.slope, h_feat0, h_el, h_er, h_gout, h_out, h_dfeat,
+                             h_del, h_der, arena, pipelined=True)
+
+    for _ in range(3):
+        host_step()
+    B.sar_gat_stack_host_wait()
+    torch.cuda.synchronize()
+    n_e2e = max(1, min(args.steps, 10))
+    if dist:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(n_e2e):
+        host_step()
+    B.sar_gat_stack_host_wait()
+    torch.cuda.synchronize()
+    dt = time.perf_counter() - t0
+    dt = max_over_ranks(dt, dist, dev)
+    h2d = 2 * n * H * F * b + 2 * L * n * H * 4
+    d2h = 2 * n * H * F * b + 2 * L * n * H * 4
+    return {"value": world * L * st.e * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "ms_per_step": 1e3 * dt / n_e2e, "steps": n_e2e, "warmup": 3,
+            "entry_point": "sar_gat_stack_host, pipelined (every step copies all its inputs in and all its results out)"}
+
+
+# --------------------------------------------------------------------------------------------------
+# our arm
+# --------------------------------------------------------------------------------------------------
+
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import workloads
+
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU path)"
+    dev = torch.device(f"cuda:{local_rank}")
+    torch.cuda.set_device(dev)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=dev)
+
+    cfg = workloads.CONFIGS[args.workload]
+    if args.scale != 1.0:
+        cfg = cfg.scaled(args.scale)
+    dtype = args.dtype or cfg.dtypes[-1]
+    peak, peak_src = load_peaks()
+    glue = args.glue
+    schedules = [args.schedule] if (args.only_schedule or glue) else ["fused", "sequential"]
+    if glue:
+        schedules = ["fused"]
+    st = AggStack(cfg, dtype, dev, ids=args.ids, threshold=args.threshold, parts="sequential" in schedules)
+    n, e, H, F, b, L, K = st.n, st.e, st.H, st.F, st.b, st.L, st.K
+    main_sched = "fused" if glue else args.schedule
+    gpu_index = gpu_index_of(local_rank)
+    prep_ms, threshold = st.prep_ms, st.threshold
 
     torch.cuda.reset_peak_memory_stats()
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
+    results = {}
+    for sch in schedules:
+        step = make_glue_step(args, st) if glue else st.step(sch)
+        is_main = sch == main_sched
+        steps = args.steps if is_main else max(1, min(args.steps, 3))
+        results[sch] = measure(step, steps, args.warmup, dist, dev, clocks_gpu=gpu_index if (is_main and rank == 0) else None)
+        results[sch]["steps"] = steps
     peak_mem = torch.cuda.max_memory_allocated()
-
-    # ---- timed region ----------------------------------------------------------------------------
-    gpu_index = int(os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",")[local_rank]) \
-        if os.environ.get("CUDA_VISIBLE_DEVICES", "").replace(",", "").isdigit() else local_rank
-    sampler = ClockSampler(gpu_index) if rank == 0 else None
-    if dist:
-        dist.barrier()
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with B.LaunchTimer() as lt:
-        e0.record()
-        for _ in range(args.steps):
-            step()
-        e1.record()
-    torch.cuda.synchronize()
-    if dist:
-        dist.barrier()
-    elapsed_ms = e0.elapsed_time(e1)
-    clocks = sampler.stop() if sampler else {}
-    elapsed_ms = max_over_ranks(elapsed_ms, dist, dev)
-    kernels = lt.summary()
-    launches = sum(v["launches"] for v in kernels.values())
-    ms_per_step = elapsed_ms / args.steps
+    main = results[main_sched]
+    ms_per_step = main["ms_per_step"]
     value = world * L * e / (ms_per_step * 1e-3)
+    kernels = main["kernels"]
+    sched_out = {sch: schedule_entry(st, sch, r, r["steps"], peak) for sch, r in results.items()}
 
     # ---- roofline of the dominant pass ---------------------------------------------------------------
-    # A pass over the E edges is up to three launches of the library (rows, long-row segments, merge);
-    # its algorithmic bytes are divided by the sum of their average CUDA-event durations.
-    peak, peak_src = load_peaks()
-    passes = group_passes(kernels)
-    dom = max(passes, key=lambda k_: passes[k_]["ms"])
+    # A pass over the E edges is the launches of the library that together visit every edge once (rows,
+    # long-row segments, merge; K times as many in the sequential schedule); its algorithmic bytes are
+    # divided by the CUDA-event time those launches took per pass.
+    passes = sched_out[main_sched]["passes"]
     roofline = None
-    if dom in KERNEL_BYTES:
-        alg = KERNEL_BYTES[dom](n, e, H, F, b)
+    if passes:
+        dom = max(passes, key=lambda k_: passes[k_]["ms"])
+        alg = passes[dom]["algorithmic_bytes"]
         achieved = alg / (passes[dom]["ms"] * 1e-3) / 1e9
+        traffic = NCU_TRAFFIC.get((args.workload, dtype, dom)) if (args.scale == 1.0 and main_sched == "fused") else None
         roofline = {"bound": "hbm", "kernel": dom, "launches": passes[dom]["launches"], "achieved": achieved,
                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                    "traffic": NCU_TRAFFIC_BYTES.get((args.workload, dtype, dom)) if args.scale == 1.0 else None,
-                    "algorithmic_bytes_per_launch": alg, "avg_launch_ms": passes[dom]["ms"]}
-    pass_ms = {k_: v["ms"] for k_, v in passes.items() if k_ in KERNEL_BYTES}
-    per_pass = {k_: {"ms": ms_, "edges_per_sec": e / (ms_ * 1e-3),
-                     "frac_of_roofline": KERNEL_BYTES[k_](n, e, H, F, b) / (ms_ * 1e-3) / 1e9 / peak}
-                for k_, ms_ in pass_ms.items()}
+                    "traffic": traffic[0] if traffic else None, "traffic_source": traffic[1] if traffic else None,
+                    "algorithmic_bytes_per_launch": alg, "avg_launch_ms": passes[dom]["ms"],
+                    "target_frac": TARGET_FRAC, "target_met": bool(achieved / peak >= TARGET_FRAC)}
     step_bytes = L * bytes_layer_fwd_bwd(n, e, H, F, b)
     step_frac = step_bytes / (ms_per_step * 1e-3) / 1e9 / peak
 
-    # ---- end to end through the host-buffer entry point ---------------------------------------------
+    extras = (not args.no_extras) and world == 1 and not glue and args.scale == 1.0 and args.workload == "large"
+    ceiling = None
+    if extras:
+        # what ANY gather kernel can reach on this graph with this row width: the sum aggregation (no scores, no
+        # softmax, one accumulator), CSR and CSC direction
+        x = st.feats[0].view(n, H * F)
+        ceiling = time_spmm(st.g, x, st.gout.view(n, H * F), 5, 3, peak, n, e, b)
+        for name, p_ in passes.items():
+            ref = ceiling["csc_ms"] if name == "gat_bwd_src" else ceiling["csr_ms"]
+            p_["frac_of_gather_ceiling"] = ref / p_["ms"]
+
     e2e = None
-    if not args.no_e2e:
-        del feats, gbuf, feat_q, gbuf_q, gout
+    if not args.no_e2e and not glue:
+        st.feats, st.gbuf, st.feat_q, st.gbuf_q, st.gout, st.acc = None, None, None, None, None, None
+        gc.collect()
         torch.cuda.empty_cache()
-        pin = lambda shape, dt: torch.empty(shape, dtype=dt).pin_memory()
-        h_feat0 = pin((n, H, F), tdt)
-        h_gout = pin((n, H, F), tdt)
-        h_out, h_dfeat = pin((n, H, F), tdt), pin((n, H, F), tdt)
-        h_el = [pin((n, H), torch.float32) for _ in range(L)]
-        h_er = [pin((n, H), torch.float32) for _ in range(L)]
-        h_del = [pin((n, H), torch.float32) for _ in range(L)]
-        h_der = [pin((n, H), torch.float32) for _ in range(L)]
-        h_feat0.copy_(workloads.normal_tensor((n, H, F), cfg.seed, 10, device=dev, dtype=tdt))
-        h_gout.copy_(workloads.normal_tensor((n, H, F), cfg.seed, 11, device=dev, dtype=tdt))
-        for l in range(L):
-            h_el[l].copy_(els[l])
-            h_er[l].copy_(ers[l])
-        # two working sets: the pipelined mode overlaps the copies of step t+1 with the kernels of step t
-        one = (B.sar_gat_stack_arena_bytes(g.whole, L, H, F, B._dtype(h_feat0)) + 255) // 256 * 256
-        arena = torch.empty(2 * one, dtype=torch.uint8, device=dev)
+        e2e = time_e2e(st, args, dist, world)
 
-        def host_step():
-            B.sar_gat_stack_host(g.whole, g.bounds, H, F, cfg.slope, h_feat0, h_el, h_er, h_gout, h_out, h_dfeat,
-                                 h_del, h_der, arena, pipelined=True)
+    others = None
+    if extras:
+        del st
+        gc.collect()
+        torch.cuda.empty_cache()
+        others = extra_workloads(dev, peak, args)
 
-        host_step()
-        host_step()
-        B.sar_gat_stack_host_wait()
-        torch.cuda.synchronize()
-        n_e2e = max(1, min(args.steps, 10))
-        if dist:
-            dist.barrier()
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        for _ in range(n_e2e):
-            host_step()
-        B.sar_gat_stack_host_wait()
-        torch.cuda.synchronize()
-        dt = time.perf_counter() - t0
-        dt = max_over_ranks(dt, dist, dev)
-        h2d = 2 * n * H * F * b + 2 * L * n * H * 4
-        d2h = 2 * n * H * F * b + 2 * L * n * H * 4
-        e2e = {"value": world * L * e * n_e2e / dt, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-               "ms_per_step": 1e3 * dt / n_e2e, "steps": n_e2e,
-               "entry_point": "sar_gat_stack_host, pipelined (every step copies all its inputs in and all its results out)"}
-
-    # ---- the oracle on the host cores, bounded sample ------------------------------------------------
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        import oracle
-        small, s_src, s_dst, h = oracle_sample(workloads.CONFIGS[args.workload], dtype,
-                                               min(1.0, args.cpu_sample * args.scale))
-        secs = oracle_step(small, s_src, s_dst, h, cfg.slope)
-        cpu = {"value": small.e / secs, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-               "sample": f"{small.name}: n={small.n} e={small.e} H={small.heads} F={small.feat}, one layer fwd+bwd, "
-                         f"{secs:.1f} s"}
+        cpu = cpu_baseline_leg(args.workload, dtype, args.cpu_sample * args.scale, cfg.slope)
 
     if rank == 0:
         line = {
@@ -513,18 +789,24 @@ def run_ours(args, rank, world, local_rank):
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {
-                "workload": cfg.name, "n": n, "e": e, "heads": H, "feat_per_head": F, "layers": L, "partitions": K,
-                "storage_dtype": dtype, "layer_glue": bool(args.glue), "bn_dropout": bool(args.glue and args.bn_dropout), "ids": args.ids, "schedule": "fused row-stationary (sar_gat_fwd_fused / sar_gat_bwd_fused)",
-                "l2": "inputs_exceed_l2", "long_row_threshold": threshold, "parallelism": f"replicas x{world}",
+                "workload": cfg.name, "n": n, "e": e, "heads": H, "feat_per_head": F, "layers": L,
+                "schedule": main_sched, "partitions": sched_out[main_sched]["partitions_seen_by_the_kernels"],
+                "partitions_configured": K, "storage_dtype": dtype, "layer_glue": bool(glue),
+                "bn_dropout": bool(glue and args.bn_dropout), "ids": args.ids,
+                "l2": "inputs_exceed_l2" if n * H * F * b > 126e6 else "inputs_fit_l2",
+                "long_row_threshold": threshold, "parallelism": f"replicas x{world}",
                 "edges_x_heads_x_feat_per_sec": value * H * F,
             },
             "roofline": roofline,
             "step_roofline": {"compulsory_bytes_per_step": step_bytes, "frac_of_peak": step_frac, "peak": peak,
                               "peak_source": peak_src},
-            "passes": per_pass, "kernels": kernels, "gpu_launches": launches, "prep_ms": prep_ms,
-            "peak_mem_bytes": peak_mem, "attention_bytes_if_stored": L * e * H * 4,
+            "schedules": sched_out, "passes": passes, "kernels": kernels, "gpu_launches": main["launches"],
+            "prep_ms": prep_ms,
+            "peak_mem_bytes": peak_mem,
+            "attention_bytes_if_stored": {"value": L * e * H * 4, "kind": "computed: 4 bytes x E x H x layers"},
             "stats_bytes_kept": L * 2 * n * H * 4,
-            "clocks": clocks, "e2e": e2e, "cpu_baseline": cpu,
+            "gather_ceiling": ceiling, "workloads": others,
+            "clocks": main["clocks"] or {}, "e2e": e2e, "cpu_baseline": cpu,
         }
         print(json.dumps(line), flush=True)
     if dist:
@@ -564,22 +846,10 @@ def run_spmm(args, local_rank):
         B.sar_spmm_agg(fwd, x, F, B.SAR_FIRST | B.SAR_LAST, None, out, ws)
         B.sar_spmm_agg(bwd, gout, F, B.SAR_FIRST | B.SAR_LAST, None, dx, ws)
 
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
-    sampler = ClockSampler(local_rank)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    with B.LaunchTimer() as lt:
-        e0.record()
-        for _ in range(args.steps):
-            step()
-        e1.record()
-    torch.cuda.synchronize()
-    clocks = sampler.stop()
-    ms_per_step = e0.elapsed_time(e1) / args.steps
-    kernels = lt.summary()
+    r = measure(step, args.steps, args.warmup, clocks_gpu=gpu_index_of(local_rank))
+    ms_per_step = r["ms_per_step"]
     peak, peak_src = load_peaks()
-    alg = idx_bytes(n, e) + 2 * n * F * b  # per direction: indices, every input row once, every output row once
+    alg = bytes_spmm(n, e, F, b)  # per direction
     achieved = 2 * alg / (ms_per_step * 1e-3) / 1e9
     line = {
         "metric": "spmm_fwd_bwd_edges_per_sec", "value": e / (ms_per_step * 1e-3), "unit": UNIT, "n_gpus": 1,
@@ -590,7 +860,7 @@ def run_spmm(args, local_rank):
         "roofline": {"bound": "hbm", "kernel": "spmm (forward + transposed)", "achieved": achieved, "peak": peak,
                      "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src, "traffic": None,
                      "algorithmic_bytes_per_step": 2 * alg, "gathered_bytes_per_step": 2 * e * F * b},
-        "kernels": kernels, "gpu_launches": sum(v["launches"] for v in kernels.values()), "clocks": clocks,
+        "kernels": r["kernels"], "gpu_launches": r["launches"], "clocks": r["clocks"],
     }
     print(json.dumps(line), flush=True)
 

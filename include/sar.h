@@ -73,6 +73,7 @@ typedef enum { SAR_F32 = 0, SAR_BF16 = 1 } sar_dtype;
 #define SAR_FIRST 1u /* first partition: ignore incoming running state / overwrite outputs   */
 #define SAR_LAST 2u  /* last partition: normalise and write the final result                 */
 #define SAR_MEAN 4u  /* sar_spmm_agg with SAR_LAST: divide by `deg_total`                    */
+#define SAR_KEEP_NUMERATOR 8u /* sar_gat_fwd with SAR_LAST: also leave the complete numerator in acc */
 
 #define SAR_MAX_HEADS 16
 #define SAR_MAX_PARTS 64
@@ -155,6 +156,14 @@ SAR_API sar_status sar_csr_split_indices(int64_t n_dst, const int64_t *indptr, c
                                  const int64_t *bounds, const int64_t *indptr_all, const int64_t *nnz_off,
                                  int32_t *indices_all, void *stream);
 
+/* The CSC (edges grouped by source) of partition q: because the sources bounds[q] <= j < bounds[q+1] are
+ * consecutive rows of the whole graph's CSC, the partition's destination ids are the slice
+ * t_indices[t_indptr[s0] .. t_indptr[s1]) of the whole array as it stands, and its offsets are
+ * t_indptr[s0..s1] counted from t_indptr[s0].  This call writes those s1 - s0 + 1 offsets to t_indptr_q
+ * (DEVICE arrays; s0 = bounds[q], s1 = bounds[q+1]). */
+SAR_API sar_status sar_csc_slice_indptr(int64_t s0, int64_t s1, const int64_t *t_indptr, int64_t *t_indptr_q,
+                                        void *stream);
+
 /* Message-flow pruning (Appendix B: with few labelled nodes, a layer only has to update the nodes that can
  * still influence a labelled node's output).  Both masks are DEVICE arrays of n bytes (0 / non-zero).
  *
@@ -206,6 +215,9 @@ SAR_API size_t sar_gat_workspace_bytes(const sar_part *g, int32_t H, int32_t F, 
  *   With SAR_LAST, out [n_dst,H,F] (type t) = acc/d is written (0 where d == 0) and m, d hold the
  *   final statistics the backward pass needs.  With SAR_FIRST|SAR_LAST (one partition holding all
  *   sources) acc may be NULL: the numerator never leaves the registers.
+ *   SAR_KEEP_NUMERATOR together with SAR_LAST also writes the complete float32 numerator to acc (which
+ *   must then be given), for sar_gat_bwd_prepare's acc_is_numerator mode: the row dot of the
+ *   per-partition backward pass is then formed from float32 values instead of a rounded bf16 out.
  *   Destinations without edges in this partition are skipped unless a flag forces a write. */
 SAR_API sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, const float *er_q, int32_t H,
                        int32_t F, sar_dtype t, float slope, uint32_t flags, float *acc, float *m, float *d,
@@ -234,9 +246,8 @@ SAR_API sar_status sar_gat_fwd_fused(const sar_part *g, int32_t k, const int64_t
  * {el, m, 1/d, D} (16 bytes per (i,h), written to the start of `workspace`) that lets each
  * partition's backward step run independently of the others.  `out` may be given as the COMPLETE float32
  * numerator with acc_is_numerator != 0 (then out = acc/d is formed on the fly), which avoids the
- * rounding of a bf16 `out`; note that the forward call with SAR_LAST does not update `acc`, so the
- * complete numerator exists only for a caller that runs all partitions without SAR_LAST and
- * normalises itself.  D may be NULL. */
+ * rounding of a bf16 `out`; the forward call of the last partition leaves the complete numerator in
+ * `acc` when it is given SAR_KEEP_NUMERATOR.  D may be NULL. */
 SAR_API sar_status sar_gat_bwd_prepare(int64_t n_dst, int32_t H, int32_t F, sar_dtype t, const void *out_or_acc,
                                int32_t acc_is_numerator, const void *gout, const float *el, const float *m,
                                const float *d, float *D, void *workspace, size_t workspace_bytes,
@@ -462,7 +473,9 @@ SAR_API sar_status sar_bn_bwd_apply_act(int64_t n, int32_t C, sar_dtype t, const
  *     (destination, head) plus the long-row partials); larger problems return SAR_ERR_WORKSPACE and launch
  *     nothing.  Every GPU that loads the library carries the array until the process exits.
  *   - The first call on each device looks up the array's device address (with that device current) and
- *     remembers it; make that first call before any stream capture begins.
+ *     remembers it for the life of the process; make that first call before any stream capture begins.
+ *     The remembered address belongs to the device's context at that time: after a cudaDeviceReset of
+ *     that device it is stale, and this entry point must not be called on that device again.
  *   - All calls on a device share the one array, which keeps whatever the previous call left in it.  The
  *     pass writes every byte of it that it later reads, so nothing needs clearing between calls; but two
  *     calls whose kernels overlap on the GPU (different streams, no dependency) race on it: keep calls to

@@ -128,8 +128,9 @@ def split_parts(whole: B.Part, bounds: List[int], threshold: int, ws: Optional[t
         s0, s1 = bounds[q], bounds[q + 1]
         ip = indptr_all[q]
         idx = indices_all[nnz_off[q]:nnz_off[q + 1]]
-        # CSC of partition q: the sources s0..s1 of the whole CSC, offsets rebased to 0
-        t_ip = (whole.t_indptr[s0:s1 + 1] - whole.t_indptr[s0]).contiguous()
+        # CSC of partition q: the sources s0..s1 of the whole CSC, offsets counted from the slice's first edge
+        t_ip = torch.empty(s1 - s0 + 1, dtype=torch.int64, device=dev)
+        B.sar_csc_slice_indptr(s0, s1, whole.t_indptr, t_ip)
         e0 = int(whole.t_indptr[s0])
         t_idx = whole.t_indices[e0:e0 + nnz_q[q]]
         split = build_plan(n, ip, threshold) if threshold else None
@@ -146,9 +147,11 @@ def gat_workspace(part: B.Part, H: int, F: int, dtype: torch.dtype) -> torch.Ten
 
 
 def gat_forward(g: Graph, feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor, slope: float,
-                workspace: Optional[torch.Tensor] = None, mode: str = "fused"):
+                workspace: Optional[torch.Tensor] = None, mode: str = "fused", keep_numerator: bool = False):
     """Forward over the K partitions.  mode "fused": one row-stationary launch (sar_gat_fwd_fused);
-    mode "stateful": K calls of sar_gat_fwd with the running state in global memory (Algorithm 1)."""
+    mode "stateful": K calls of sar_gat_fwd with the running state in global memory (Algorithm 1).
+    keep_numerator (stateful mode): returns (out, m, d, acc) with the complete float32 numerator in acc,
+    which gat_backward can take in place of `out` for the row dot."""
     n, H, F = feat.shape
     dev = feat.device
     m = torch.empty((g.n, H), dtype=torch.float32, device=dev)
@@ -161,20 +164,22 @@ def gat_forward(g: Graph, feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor
         B.sar_gat_fwd_fused(g.whole, g.bounds, feat_q, el, er_q, H, F, slope, m, d, out, ws)
         return out, m, d
     assert g.parts, "stateful mode needs Graph.from_coo(..., build_parts=True)"
-    acc = torch.empty((g.n, H, F), dtype=torch.float32, device=dev) if g.k > 1 else None
+    acc = torch.empty((g.n, H, F), dtype=torch.float32, device=dev) if (g.k > 1 or keep_numerator) else None
     for q, part in enumerate(g.parts):
         flags = (B.SAR_FIRST if q == 0 else 0) | (B.SAR_LAST if q == g.k - 1 else 0)
+        if keep_numerator and q == g.k - 1:
+            flags |= B.SAR_KEEP_NUMERATOR
         ws = gat_workspace(part, H, F, feat.dtype)
         s0, s1 = g.bounds[q], g.bounds[q + 1]
         B.sar_gat_fwd(part, feat[s0:s1], el, er[s0:s1], H, F, slope, flags, acc, m, d, out, ws)
-    return out, m, d
+    return (out, m, d, acc) if keep_numerator else (out, m, d)
 
 
 def gat_backward(g: Graph, feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor, m: torch.Tensor,
                  d: torch.Tensor, gout: torch.Tensor, slope: float, out: Optional[torch.Tensor] = None,
-                 workspace: Optional[torch.Tensor] = None, mode: str = "fused"):
-    """Backward over the K partitions; returns (dfeat, del, der).  "stateful" needs `out` (for the
-    row dot) and runs sar_gat_bwd_prepare followed by K calls of sar_gat_bwd."""
+                 workspace: Optional[torch.Tensor] = None, mode: str = "fused", acc: Optional[torch.Tensor] = None):
+    """Backward over the K partitions; returns (dfeat, del, der).  "stateful" needs `out` or the complete
+    float32 numerator `acc` (for the row dot) and runs sar_gat_bwd_prepare followed by K calls of sar_gat_bwd."""
     n, H, F = feat.shape
     dev = feat.device
     dfeat = torch.empty_like(feat)
@@ -186,10 +191,13 @@ def gat_backward(g: Graph, feat: torch.Tensor, el: torch.Tensor, er: torch.Tenso
         B.sar_gat_bwd_fused(g.whole, g.bounds, sl(feat), el, sl(er), m, d, gout, H, F, slope, sl(dfeat), del_,
                             sl(der), ws)
         return dfeat, del_, der
-    assert g.parts and out is not None
+    assert g.parts and (out is not None or acc is not None)
     nbytes = max(B.sar_gat_workspace_bytes(p, H, F, B._dtype(feat)) for p in g.parts)
     ws = _workspace(nbytes, dev)
-    B.sar_gat_bwd_prepare(g.n, H, F, out, False, gout, el, m, d, None, ws)
+    if acc is not None:
+        B.sar_gat_bwd_prepare(g.n, H, F, acc, True, gout, el, m, d, None, ws)
+    else:
+        B.sar_gat_bwd_prepare(g.n, H, F, out, False, gout, el, m, d, None, ws)
     for q, part in enumerate(g.parts):
         flags = (B.SAR_FIRST if q == 0 else 0) | (B.SAR_LAST if q == g.k - 1 else 0)
         s0, s1 = g.bounds[q], g.bounds[q + 1]

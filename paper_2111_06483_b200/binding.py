@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_PKG, "libsar.so")
 
 SAR_OK = 0
 SAR_F32, SAR_BF16 = 0, 1
-SAR_FIRST, SAR_LAST, SAR_MEAN = 1, 2, 4
+SAR_FIRST, SAR_LAST, SAR_MEAN, SAR_KEEP_NUMERATOR = 1, 2, 4, 8
 SAR_MAX_PARTS = 64
 
 EXPORTS = [
@@ -33,7 +33,7 @@ EXPORTS = [
     "sar_gat_stack_host_wait", "sar_bn_workspace_bytes", "sar_bn_stats", "sar_bn_apply", "sar_bn_bwd_stats",
     "sar_bn_bwd_apply", "sar_dropout", "sar_linear_workspace_bytes", "sar_linear", "sar_linear_bwd_input",
     "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd", "sar_axpby", "sar_bn_rstd", "sar_accumulate", "sar_round_to", "sar_bn_apply_act",
-    "sar_bn_bwd_stats_act", "sar_bn_bwd_apply_act",
+    "sar_bn_bwd_stats_act", "sar_bn_bwd_apply_act", "sar_csc_slice_indptr",
 ]
 
 
@@ -249,6 +249,12 @@ def sar_csr_split_indices(n_dst: int, indptr: torch.Tensor, indices: torch.Tenso
     _check("sar_csr_split_indices", lib().sar_csr_split_indices(c_int64(n_dst), _ptr(indptr), _ptr(indices),
                                                                 c_int32(k), _host_i64(bounds), _ptr(indptr_all),
                                                                 _host_i64(nnz_off), _ptr(indices_all), _stream()))
+
+
+def sar_csc_slice_indptr(s0: int, s1: int, t_indptr: torch.Tensor, t_indptr_q: torch.Tensor) -> None:
+    assert t_indptr.dtype == torch.int64 and t_indptr_q.dtype == torch.int64 and t_indptr_q.numel() == s1 - s0 + 1
+    _check("sar_csc_slice_indptr", lib().sar_csc_slice_indptr(c_int64(s0), c_int64(s1), _ptr(t_indptr),
+                                                              _ptr(t_indptr_q), _stream()))
 
 
 def sar_mfg_frontier(n: int, indptr: torch.Tensor, indices: torch.Tensor, need_out: torch.Tensor,

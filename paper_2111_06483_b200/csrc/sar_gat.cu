@@ -123,7 +123,7 @@ static sar_status launch_span(SpanArgs a, long long nnz, const char *name, const
     const long long spans = (a.n_rows + a.R - 1) / a.R;
     if (spans > 0) {
         const unsigned blocks = (unsigned)((spans + kSpanWarps - 1) / kSpanWarps);
-        if ((a.flags & SAR_FIRST) && (a.flags & SAR_LAST)) {  // the epilogue's flag tests decided at compile time
+        if ((a.flags & SAR_FIRST) && (a.flags & SAR_LAST) && !(a.flags & SAR_KEEP_NUMERATOR)) {  // the epilogue's flag tests decided at compile time
             if (geo) {
                 auto whole = span_kernel<T, G, V, S, MODE, CAP, MINB, 1, kGeo>;
                 SAR_TRY(ensure_smem(whole, smem));
@@ -211,12 +211,13 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
                        int32_t F, sar_dtype t, float slope, uint32_t flags, float *acc, float *m, float *d,
                        void *out, void *workspace, size_t workspace_bytes, void *stream) {
     SAR_TRY(check_part(g, false));
-    if (flags & ~(SAR_FIRST | SAR_LAST)) return SAR_ERR_INVALID_ARG;
+    if (flags & ~(SAR_FIRST | SAR_LAST | SAR_KEEP_NUMERATOR)) return SAR_ERR_INVALID_ARG;
     const bool first = flags & SAR_FIRST, last = flags & SAR_LAST;
+    if ((flags & SAR_KEEP_NUMERATOR) && !last) return SAR_ERR_INVALID_ARG;
     if (!el || !m || !d) return SAR_ERR_INVALID_ARG;
     if (g->n_src > 0 && (!feat_q || !er_q)) return SAR_ERR_INVALID_ARG;
     if (last && !out) return SAR_ERR_INVALID_ARG;
-    if (!(first && last) && !acc) return SAR_ERR_INVALID_ARG;
+    if ((!(first && last) || (flags & SAR_KEEP_NUMERATOR)) && !acc) return SAR_ERR_INVALID_ARG;
     SAR_TRY(check_elem_align({el, er_q, m, d, acc}, 4));
     SAR_TRY(check_elem_align({feat_q, out}, sar_elem_size(t)));
     Shape s;

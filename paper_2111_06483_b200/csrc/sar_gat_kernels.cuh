@@ -88,6 +88,7 @@ __global__ void __launch_bounds__(kThreads) gat_fwd_merge_kernel(const FwdArgs a
             }
     }
     if (last) {
+        if (a.flags & SAR_KEEP_NUMERATOR) store_acc_row<G, V, EPV>(a.acc + row * rowf, id.gl, vg.vok, acc);
 #pragma unroll
         for (int v = 0; v < V; ++v) {
             const float inv = dv[v] > 0.f ? 1.f / dv[v] : 0.f;

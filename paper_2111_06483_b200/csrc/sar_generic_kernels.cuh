@@ -69,8 +69,7 @@ __global__ void gat_fwd_generic(const GenericArgs a) {
         }
         if (last)
             Elem<T>::store1(reinterpret_cast<T *>(a.out) + o, dsum > 0.f ? acc / dsum : 0.f);
-        else
-            a.acc[o] = acc;
+        if (!last || (a.flags & SAR_KEEP_NUMERATOR)) a.acc[o] = acc;
     }
     a.m[idx] = Mn;
     a.d[idx] = dsum;

@@ -83,6 +83,12 @@ __global__ void split_fill_kernel(long long n_dst, const int64_t *__restrict__ i
     }
 }
 
+// out[i] = in[i] - in[0]: the offsets of a run of consecutive rows, counted from the run's first edge
+__global__ void rebase_kernel(long long count, const int64_t *__restrict__ in, int64_t *__restrict__ out) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < count) out[i] = in[i] - in[0];
+}
+
 struct IsLongRow {
     const int64_t *indptr;
     int threshold;
@@ -339,6 +345,14 @@ sar_status sar_csr_split_indices(int64_t n_dst, const int64_t *indptr, const int
     if (!indices || !indices_all) return SAR_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     split_fill_kernel<<<nblk(n_dst), 256, 0, st>>>(n_dst, indptr, indices, b, off, indptr_all, indices_all);
+    return sar_after_launch();
+}
+
+sar_status sar_csc_slice_indptr(int64_t s0, int64_t s1, const int64_t *t_indptr, int64_t *t_indptr_q, void *stream) {
+    if (s0 < 0 || s1 < s0 || !t_indptr || !t_indptr_q) return SAR_ERR_INVALID_ARG;
+    if (!sar_aligned(t_indptr, 8) || !sar_aligned(t_indptr_q, 8)) return SAR_ERR_ALIGNMENT;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rebase_kernel<<<nblk(s1 - s0 + 1), 256, 0, st>>>(s1 - s0 + 1, t_indptr + s0, t_indptr_q);
     return sar_after_launch();
 }
 

@@ -803,6 +803,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                     }
                     if (writer) {
                         if (last_part) {
+                            if (flags_ & SAR_KEEP_NUMERATOR) store_acc_row<G, V, EPV>(a.acc_state + row * rowf, gl, vok, acc0);
 #pragma unroll
                             for (int v = 0; v < V; ++v) {
                                 const float inv = sv[v] > 0.f ? __fdividef(1.f, sv[v]) : 0.f;

@@ -59,7 +59,12 @@ def dense_gat_torch(C, feat, el, er, slope):
     return torch.einsum("ijh,jhf->ihf", P, feat)
 
 
+TOLERANCE_USE = []   # (what, worst error, share of the tolerance used) of every check since the last drain
+
+
 def allclose_report(got, want, rtol, atol, what=""):
+    """|got - want| <= atol + rtol * |want| element by element; records the largest error seen and the
+    share of its tolerance that it used (drained into the test's properties by conftest.py)."""
     got = np.asarray(got, dtype=np.float64)
     want = np.asarray(want, dtype=np.float64)
     assert got.shape == want.shape, (what, got.shape, want.shape)
@@ -68,6 +73,11 @@ def allclose_report(got, want, rtol, atol, what=""):
         err = np.where(both_inf, 0.0, np.abs(got - want))
     tol = atol + rtol * np.where(both_inf, 0.0, np.abs(want))
     bad = ~(err <= tol)
+    if got.size:
+        with np.errstate(invalid="ignore", divide="ignore"):
+            use = np.where(tol > 0, err / tol, np.where(err > 0, np.inf, 0.0))
+        use = np.where(np.isnan(use), np.inf, use)
+        TOLERANCE_USE.append((what, float(np.nanmax(np.where(np.isnan(err), np.inf, err))), float(use.max())))
     if bad.any():
         k = np.argmax(np.where(bad, err - tol, -np.inf))
         idx = np.unravel_index(k, got.shape)

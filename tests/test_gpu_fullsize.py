@@ -1,5 +1,6 @@
-"""GPU parity at the full sizes of the named workloads, in the launch configuration bench.py times
-(fused calls over the K partitions of the un-split graph, long-row plan with the default threshold).
+"""GPU parity at the full sizes of the named workloads, in the launch configurations bench.py times
+(the fused calls over the un-split graph and the call-by-call sequence over the K partitions, long-row
+plans with the default threshold).
 
 The oracle cannot run 300 M edges in test time, so outputs are SAMPLED: a sub-problem that contains
 every edge the sampled outputs depend on is cut out with torch indexing, handed to the oracle, and
@@ -43,40 +44,50 @@ def _tol(dtype, want, grad=False):
     return dict(rtol=1e-4, atol=1e-5 * scale) if grad else dict(rtol=1e-5, atol=1e-6)
 
 
+def _run_schedule(g, t, cfg, dtype, mode):
+    """Forward + backward of one layer in one schedule of the K partitions; returns the six outputs."""
+    feat, gout, el, er = t["feat"], t["gout"], t["el"], t["er"]
+    if mode == "fused":
+        out, m, d = api.gat_forward(g, feat, el, er, cfg.slope)
+        dfeat, del_, der = api.gat_backward(g, feat, el, er, m, d, gout, cfg.slope)
+    else:
+        # K calls of sar_gat_fwd with the running state in device memory (Algorithm 1), then
+        # sar_gat_bwd_prepare and K calls of sar_gat_bwd (Algorithm 2).  With bf16 storage the row dot is
+        # formed from the float32 numerator the last forward call leaves behind.
+        keep = dtype == "bf16" and g.k > 1
+        fw = api.gat_forward(g, feat, el, er, cfg.slope, mode="stateful", keep_numerator=keep)
+        out, m, d = fw[:3]
+        dfeat, del_, der = api.gat_backward(g, feat, el, er, m, d, gout, cfg.slope, out=out, mode="stateful",
+                                            acc=fw[3] if keep else None)
+        del fw
+    torch.cuda.synchronize()
+    return out, m, d, dfeat, del_, der
+
+
 @pytest.mark.parametrize("name,dtype", [("seqpart", "f32"), ("medium", "f32"), ("medium", "bf16"), ("dense", "bf16"),
                                         ("large", "bf16")])
 def test_sampled_rows_at_full_size(name, dtype):
+    """Every named workload at its full size, in BOTH schedules of its K partitions: the fused row-stationary
+    calls bench.py times by default, and the call-by-call sequence of Algorithm 1 / Algorithm 2 with K
+    partitions (seqpart K = 8, medium K = 4, dense K = 8, large K = 16), each against the oracle on sampled
+    rows; the running max must end bit-identical in the two schedules."""
     cfg = workloads.CONFIGS[name]
     n, H, F = cfg.n, cfg.heads, cfg.feat
-    need = (4 * n * H * F * (2 if dtype == "bf16" else 4) + 24 * cfg.e) * 1.5
+    need = (5 * n * H * F * (2 if dtype == "bf16" else 4) + 4 * n * H * F + 40 * cfg.e) * 1.5
     if torch.cuda.get_device_properties(0).total_memory < need:
         pytest.skip("not enough device memory for this workload")
     src, dst = workloads.make_graph(cfg, device=DEV)
-    g = api.Graph.from_coo(n, src, dst, k=cfg.k)
+    g = api.Graph.from_coo(n, src, dst, k=cfg.k, build_parts=True)
     del src, dst
+    assert g.k == cfg.k and len(g.parts) == cfg.k
     t = workloads.make_node_inputs(n, H, F, cfg.seed, dtype=dtype, device=DEV)
     feat, gout, el, er = t["feat"], t["gout"], t["el"], t["er"]
-    out, m, d = api.gat_forward(g, feat, el, er, cfg.slope)
-    dfeat, del_, der = api.gat_backward(g, feat, el, er, m, d, gout, cfg.slope)
-    torch.cuda.synchronize()
     W = g.whole
     in_deg = W.indptr[1:] - W.indptr[:-1]
     out_deg = W.t_indptr[1:] - W.t_indptr[:-1]
-
-    # ---- invariants over the whole arrays ----------------------------------------------------------
-    assert torch.isfinite(out.float()).all() and torch.isfinite(dfeat.float()).all()
     empty = in_deg == 0
-    assert (d[empty] == 0).all() and torch.isneginf(m[empty]).all() and (out[empty] == 0).all()
-    assert (d[~empty] >= 1.0 - 1e-5).all()                      # the max term contributes exp(0) = 1
-    s_del, s_der = del_.double().sum(0), der.double().sum(0)      # two groupings of the same per-edge terms
-    scale = float(del_.double().abs().sum(0).max())
-    assert float((s_del - s_der).abs().max()) <= (2e-2 if dtype == "bf16" else 1e-4) * max(scale, 1.0) ** 0.5 * 50
-    want_sum = gout[~empty].double().sum(0)                       # every edge hands alpha*gout to its source
-    got_sum = dfeat.double().sum(0)
-    tol = (2e-2 if dtype == "bf16" else 1e-4) * float(gout.double().abs().sum(0).max()) ** 0.5 * 50
-    assert float((got_sum - want_sum).abs().max()) <= tol
 
-    # ---- sampled destinations: out, m, d, del --------------------------------------------------------
+    # ---- the oracle on two sampled sub-problems ------------------------------------------------------
     gen = torch.Generator(device="cpu").manual_seed(cfg.seed + 100)
     rows = torch.randperm(n, generator=gen)[:3000].to(DEV)
     hubs = torch.topk(in_deg, 3).indices                          # the longest rows go through the segment path
@@ -84,17 +95,12 @@ def test_sampled_rows_at_full_size(name, dtype):
     sub_indptr, cols = _rows_subgraph(W.indptr, W.indices, rows)
     ucols, inv = torch.unique(cols, return_inverse=True)
     f_sub = feat[ucols].float().cpu().numpy()
-    fwd = oracle.gat_fwd(sub_indptr.cpu().numpy(), inv.cpu().numpy().astype(np.int32), f_sub,
-                         el[rows].cpu().numpy(), er[ucols].cpu().numpy(), cfg.slope)
-    allclose_report(out[rows].float().cpu().numpy(), fwd.out, what="out", **_tol(dtype, fwd.out))
-    allclose_report(m[rows].cpu().numpy(), fwd.m, 1e-6, 1e-6, "m")
-    allclose_report(d[rows].cpu().numpy(), fwd.d, 1e-5, 1e-6, "d")
-    bwd = oracle.gat_bwd(sub_indptr.cpu().numpy(), inv.cpu().numpy().astype(np.int32), f_sub,
-                         el[rows].cpu().numpy(), er[ucols].cpu().numpy(), fwd.alpha,
-                         gout[rows].float().cpu().numpy(), cfg.slope)
-    allclose_report(del_[rows].cpu().numpy(), bwd.del_, what="del", **_tol(dtype, bwd.del_, grad=True))
-
-    # ---- sampled sources: dfeat, der (two-hop sub-problem) -------------------------------------------
+    fwd1 = oracle.gat_fwd(sub_indptr.cpu().numpy(), inv.cpu().numpy().astype(np.int32), f_sub,
+                          el[rows].cpu().numpy(), er[ucols].cpu().numpy(), cfg.slope)
+    bwd1 = oracle.gat_bwd(sub_indptr.cpu().numpy(), inv.cpu().numpy().astype(np.int32), f_sub,
+                          el[rows].cpu().numpy(), er[ucols].cpu().numpy(), fwd1.alpha,
+                          gout[rows].float().cpu().numpy(), cfg.slope)
+    # sampled sources with all their out-edges, plus every in-edge of the destinations those reach
     avg_deg = cfg.e / n
     srcs = torch.randperm(n, generator=gen)[:max(3, int(2000 / avg_deg))].to(DEV)
     if avg_deg < 50:                                             # and a couple of busy sources
@@ -108,17 +114,44 @@ def test_sampled_rows_at_full_size(name, dtype):
     ucols, inv = torch.unique(cols, return_inverse=True)
     f_sub = feat[ucols].float().cpu().numpy()
     ip, ix = sub_indptr.cpu().numpy(), inv.cpu().numpy().astype(np.int32)
-    fwd = oracle.gat_fwd(ip, ix, f_sub, el[drows].cpu().numpy(), er[ucols].cpu().numpy(), cfg.slope)
-    bwd = oracle.gat_bwd(ip, ix, f_sub, el[drows].cpu().numpy(), er[ucols].cpu().numpy(), fwd.alpha,
-                         gout[drows].float().cpu().numpy(), cfg.slope)
+    fwd2 = oracle.gat_fwd(ip, ix, f_sub, el[drows].cpu().numpy(), er[ucols].cpu().numpy(), cfg.slope)
+    bwd2 = oracle.gat_bwd(ip, ix, f_sub, el[drows].cpu().numpy(), er[ucols].cpu().numpy(), fwd2.alpha,
+                          gout[drows].float().cpu().numpy(), cfg.slope)
     where = torch.searchsorted(ucols, srcs)                      # sampled sources inside the sub-problem
     has_out = out_deg[srcs] > 0
     where_np, srcs_ok = where[has_out].cpu().numpy(), srcs[has_out]
-    allclose_report(dfeat[srcs_ok].float().cpu().numpy(), bwd.dfeat[where_np], what="dfeat",
-                    **_tol(dtype, bwd.dfeat[where_np], grad=True))
-    allclose_report(der[srcs_ok].cpu().numpy(), bwd.der[where_np], what="der", **_tol(dtype, bwd.der[where_np], grad=True))
     no_out = srcs[~has_out]
-    assert (dfeat[no_out] == 0).all() and (der[no_out] == 0).all()
+    del f_sub, fwd2, cols, inv, ucols
+
+    m_by_mode = {}
+    for mode in ("fused", "stateful"):
+        out, m, d, dfeat, del_, der = _run_schedule(g, t, cfg, dtype, mode)
+        m_by_mode[mode] = m
+        # ---- invariants over the whole arrays --------------------------------------------------------
+        assert torch.isfinite(out.float()).all() and torch.isfinite(dfeat.float()).all()
+        assert (d[empty] == 0).all() and torch.isneginf(m[empty]).all() and (out[empty] == 0).all()
+        assert (d[~empty] >= 1.0 - 1e-5).all()                      # the max term contributes exp(0) = 1
+        s_del, s_der = del_.double().sum(0), der.double().sum(0)      # two groupings of the same per-edge terms
+        scale = float(del_.double().abs().sum(0).max())
+        assert float((s_del - s_der).abs().max()) <= (2e-2 if dtype == "bf16" else 1e-4) * max(scale, 1.0) ** 0.5 * 50
+        want_sum = gout[~empty].double().sum(0)                       # every edge hands alpha*gout to its source
+        got_sum = dfeat.double().sum(0)
+        tol = (2e-2 if dtype == "bf16" else 1e-4) * float(gout.double().abs().sum(0).max()) ** 0.5 * 50
+        assert float((got_sum - want_sum).abs().max()) <= tol
+        # ---- sampled destinations: out, m, d, del ----------------------------------------------------
+        allclose_report(out[rows].float().cpu().numpy(), fwd1.out, what=f"out[{mode}]", **_tol(dtype, fwd1.out))
+        allclose_report(m[rows].cpu().numpy(), fwd1.m, 1e-6, 1e-6, f"m[{mode}]")
+        allclose_report(d[rows].cpu().numpy(), fwd1.d, 1e-5, 1e-6, f"d[{mode}]")
+        allclose_report(del_[rows].cpu().numpy(), bwd1.del_, what=f"del[{mode}]", **_tol(dtype, bwd1.del_, grad=True))
+        # ---- sampled sources: dfeat, der -------------------------------------------------------------
+        allclose_report(dfeat[srcs_ok].float().cpu().numpy(), bwd2.dfeat[where_np], what=f"dfeat[{mode}]",
+                        **_tol(dtype, bwd2.dfeat[where_np], grad=True))
+        allclose_report(der[srcs_ok].cpu().numpy(), bwd2.der[where_np], what=f"der[{mode}]",
+                        **_tol(dtype, bwd2.der[where_np], grad=True))
+        assert (dfeat[no_out] == 0).all() and (der[no_out] == 0).all()
+        del out, d, dfeat, del_, der
+        torch.cuda.empty_cache()
+    assert torch.equal(m_by_mode["fused"], m_by_mode["stateful"])   # the running max is exact in any schedule
 
 
 def test_stack_host_entry_point_matches_device_calls():

@@ -73,13 +73,14 @@ class Problem:
         h = self.host
         return oracle.gat_bwd(self.indptr, self.indices, h["feat"], h["el"], h["er"], fwd.alpha, h["gout"], slope)
 
-    def gpu_fwd(self, mode="fused", slope=0.2):
+    def gpu_fwd(self, mode="fused", slope=0.2, keep_numerator=False):
         d = self.dev
-        return api.gat_forward(self.graph, d["feat"], d["el"], d["er"], slope, mode=mode)
+        return api.gat_forward(self.graph, d["feat"], d["el"], d["er"], slope, mode=mode, keep_numerator=keep_numerator)
 
-    def gpu_bwd(self, m, dd, out=None, mode="fused", slope=0.2):
+    def gpu_bwd(self, m, dd, out=None, mode="fused", slope=0.2, acc=None):
         d = self.dev
-        return api.gat_backward(self.graph, d["feat"], d["el"], d["er"], m, dd, d["gout"], slope, out=out, mode=mode)
+        return api.gat_backward(self.graph, d["feat"], d["el"], d["er"], m, dd, d["gout"], slope, out=out, mode=mode,
+                                acc=acc)
 
 
 def uniform_problem(n, e, H, F, seed, loops=False, **kw):
@@ -181,19 +182,19 @@ def _full_check(p, dtype="f32", modes=("fused",), slope=0.2, grad_floor=1.0):
     b = p.oracle_bwd(f, slope)
     results = {}
     for mode in modes:
-        out, m, d = p.gpu_fwd(mode, slope)
+        # Call by call the row dot D = <gout, out> comes from sar_gat_bwd_prepare.  With bf16 storage it is
+        # formed from the complete float32 numerator the last forward call leaves behind
+        # (SAR_KEEP_NUMERATOR), so that the rounding of `out` never enters and the ordinary tolerances hold.
+        keep = mode == "stateful" and dtype == "bf16" and p.k > 1
+        fw = p.gpu_fwd(mode, slope, keep_numerator=keep)
+        out, m, d = fw[:3]
         check_out(out, f.out, dtype, f"out[{mode}]")
         allclose_report(m.cpu().numpy(), f.m, 1e-6, 1e-6, f"m[{mode}]")
         allclose_report(d.cpu().numpy(), f.d, 1e-5, 1e-6, f"d[{mode}]")
-        dfeat, del_, der = p.gpu_bwd(m, d, out=out, mode=mode, slope=slope)
+        dfeat, del_, der = p.gpu_bwd(m, d, out=out, mode=mode, slope=slope, acc=fw[3] if keep else None)
         check_grad(dfeat, b.dfeat, dtype, f"dfeat[{mode}]")
-        if mode == "stateful" and dtype == "bf16" and p.k > 1:
-            # the row dot is taken from the bf16-rounded `out` here: a looser floor applies
-            allclose_report(del_.cpu().numpy(), b.del_, 2e-2, 0.1 * rms(b.del_), f"del[{mode}]")
-            allclose_report(der.cpu().numpy(), b.der, 2e-2, 0.1 * rms(b.der), f"der[{mode}]")
-        else:
-            check_grad(del_, b.del_, dtype, f"del[{mode}]", grad_floor)
-            check_grad(der, b.der, dtype, f"der[{mode}]", grad_floor)
+        check_grad(del_, b.del_, dtype, f"del[{mode}]", grad_floor)
+        check_grad(der, b.der, dtype, f"der[{mode}]", grad_floor)
         results[mode] = (out, m, d, dfeat, del_, der)
     return f, b, results
 

@@ -6,12 +6,17 @@ acceptable, a fixed memory budget).  For them the library keeps a fixed scratch 
 This test calls that entry point through the C-ABI twice in a row, on two different problems, and
 checks each result against the ordinary entry point (same kernels, caller-provided workspace): the
 second call finds the first call's leftovers in the shared array and must not be disturbed by them.
+The two entry points run the same kernels in the same order, so besides the tolerance check the
+results must agree bit for bit; the first problem is also compared with the CPU oracle.
 It sits in a file of its own, collected last, so that a failure here cannot hide other tests.
 """
+import numpy as np
 import pytest
 import torch
 
+import oracle
 import workloads
+from helpers import allclose_report
 
 pytestmark = pytest.mark.gpu
 
@@ -28,8 +33,9 @@ def _problem(n, e, H, F, seed, dtype, hub):
     else:
         src, dst = workloads.uniform_edges(n, e, seed, self_loops=True)
     g = api.Graph.from_coo(n, src.to(DEV), dst.to(DEV), threshold=32)
-    t = {k: v.to(DEV) for k, v in workloads.make_node_inputs(n, H, F, seed, dtype=dtype).items()}
-    return g, t, H, F
+    host = workloads.make_node_inputs(n, H, F, seed, dtype=dtype)
+    t = {k: v.to(DEV) for k, v in host.items()}
+    return g, t, H, F, (src, dst, host)
 
 
 def _both_ways(g, t, H, F, slope=0.2):
@@ -60,8 +66,20 @@ def test_two_calls_in_a_row_match_the_ordinary_entry_point():
     second = _problem(2000, 20000, 4, 16, 12, "f32", hub=False)     # smaller: the array still holds call 1's data
     assert first[0].whole.split is not None
     for prob, dtype in ((first, "bf16"), (second, "f32")):
-        want, got = _both_ways(*prob)
+        want, got = _both_ways(*prob[:4])
         _close(got, want, dtype)
+        for a, b, name in zip(got, want, ("dfeat", "del", "der")):
+            assert torch.equal(a, b), f"{name}: same kernels, same order, yet not bit-identical"
+    # the first problem against the oracle as well (bf16 storage: rtol 2e-2, floor 2e-2 x RMS)
+    g, t, H, F, (src, dst, host) = first
+    _, got = _both_ways(g, t, H, F)
+    h = {k: v.float().numpy() for k, v in host.items()}
+    indptr, indices = oracle.csr_from_coo(g.n, g.n, src.numpy(), dst.numpy())
+    f = oracle.gat_fwd(indptr, indices, h["feat"], h["el"], h["er"], 0.2)
+    b = oracle.gat_bwd(indptr, indices, h["feat"], h["el"], h["er"], f.alpha, h["gout"], 0.2)
+    for a, w, name in zip(got, (b.dfeat, b.del_, b.der), ("dfeat", "del", "der")):
+        floor = 2e-2 * max(float(np.sqrt(np.mean(w * w))), 1.0)
+        allclose_report(a.float().cpu().numpy(), w, 2e-2, floor, f"noalloc {name} vs oracle")
 
 
 def test_problems_beyond_the_fixed_scratch_are_refused():
