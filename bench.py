@@ -59,6 +59,7 @@ def parse_args():
     ap.add_argument("--dtype", default=None, help="f32 | bf16 (default: the workload's last listed dtype)")
     ap.add_argument("--scale", type=float, default=1.0, help="shrink the workload (debugging and profiling)")
     ap.add_argument("--threshold", type=int, default=None, help="long-row split threshold")
+    ap.add_argument("--t-threshold", type=int, default=None, help="long-row split threshold of the CSC (default: the same)")
     ap.add_argument("--schedule", default="fused", choices=["fused", "sequential"],
                     help="which schedule of the K partitions `value` is taken from (both are timed)")
     ap.add_argument("--only-schedule", action="store_true", help="time only the schedule named by --schedule")
@@ -333,7 +334,7 @@ class AggStack:
 
     feat^{l+1} = out^l with seeded el^l, er^l; the backward pass feeds dfeat^{l+1} as gout of layer l."""
 
-    def __init__(self, cfg, dtype, dev, ids="permuted", threshold=None, parts=True):
+    def __init__(self, cfg, dtype, dev, ids="permuted", threshold=None, parts=True, t_threshold=None):
         import torch
         import workloads
         from paper_2111_06483_b200 import api, binding as B
@@ -348,7 +349,8 @@ class AggStack:
         self.e = src.numel()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        self.g = api.Graph.from_coo(n, src, dst, k=K, threshold=self.threshold, build_parts=parts and K > 1)
+        self.g = api.Graph.from_coo(n, src, dst, k=K, threshold=self.threshold, build_parts=parts and K > 1,
+                                    t_threshold=t_threshold)
         torch.cuda.synchronize()
         self.prep_ms = 1e3 * (time.perf_counter() - t0)
         del src, dst
@@ -714,7 +716,8 @@ def run_ours(args, rank, world, local_rank):
     schedules = [args.schedule] if (args.only_schedule or glue) else ["fused", "sequential"]
     if glue:
         schedules = ["fused"]
-    st = AggStack(cfg, dtype, dev, ids=args.ids, threshold=args.threshold, parts="sequential" in schedules)
+    st = AggStack(cfg, dtype, dev, ids=args.ids, threshold=args.threshold, parts="sequential" in schedules,
+                  t_threshold=args.t_threshold)
     n, e, H, F, b, L, K = st.n, st.e, st.H, st.F, st.b, st.L, st.K
     main_sched = "fused" if glue else args.schedule
     gpu_index = gpu_index_of(local_rank)

@@ -12,7 +12,8 @@ import torch
 
 from . import binding as B
 
-DEFAULT_THRESHOLD = 384  # rows with more edges are cut into segments of this many edges
+DEFAULT_THRESHOLD = 256    # rows of the CSR with more edges are cut into segments of this many edges
+DEFAULT_T_THRESHOLD = 384  # the same for the CSC (the source-major backward pass measured best with longer segments)
 
 
 def _workspace(nbytes: int, device) -> torch.Tensor:
@@ -20,12 +21,14 @@ def _workspace(nbytes: int, device) -> torch.Tensor:
 
 
 def build_plan(n_rows: int, indptr: torch.Tensor, threshold: int) -> Optional[B.Split]:
-    """Long-row plan of one CSR (None when no row is longer than `threshold`)."""
+    """Long-row plan of one CSR.  A plan without long rows (n_long = 0) still tells the library that no row
+    is longer than `threshold`."""
     dev = indptr.device
     counts = torch.zeros(2, dtype=torch.int64, device=dev)
     n_long, n_seg = B.sar_plan_count(n_rows, indptr, threshold, counts)
     if n_long == 0:
-        return None
+        return B.Split(threshold, 0, 0, torch.empty(0, dtype=torch.int32, device=dev),
+                       torch.zeros(1, dtype=torch.int64, device=dev))
     long_row = torch.empty(n_long, dtype=torch.int32, device=dev)
     long_seg = torch.empty(n_long + 1, dtype=torch.int64, device=dev)
     ws = _workspace(B.sar_graph_workspace_bytes(0, n_rows), dev)
@@ -45,7 +48,7 @@ class Graph:
 
     @staticmethod
     def from_coo(n: int, src: torch.Tensor, dst: torch.Tensor, k: int = 1, threshold: int = DEFAULT_THRESHOLD,
-                 build_parts: bool = False) -> "Graph":
+                 build_parts: bool = False, t_threshold: Optional[int] = None) -> "Graph":
         """src[t] -> dst[t] int32 CUDA tensors.  Builds CSR by destination, its transpose, the long-row
         plans and (build_parts) the K per-partition sub-graphs with local source ids."""
         dev = src.device
@@ -57,8 +60,10 @@ class Graph:
         t_indptr = torch.empty(n + 1, dtype=torch.int64, device=dev)
         t_indices = torch.empty(nnz, dtype=torch.int32, device=dev)
         B.sar_csr_from_coo(n, n, src, dst, t_indptr, t_indices, ws)
+        if t_threshold is None:   # the CSC's plan has its own threshold
+            t_threshold = DEFAULT_T_THRESHOLD if threshold == DEFAULT_THRESHOLD else threshold
         split = build_plan(n, indptr, threshold) if threshold else None
-        t_split = build_plan(n, t_indptr, threshold) if threshold else None
+        t_split = build_plan(n, t_indptr, t_threshold) if t_threshold else None
         whole = B.Part(n, n, indptr, indices, t_indptr, t_indices, split, t_split)
         g = Graph(n=n, nnz=nnz, whole=whole, k=k, bounds=B.sar_partition_bounds(n, k))
         if build_parts:

@@ -18,12 +18,16 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(CSRC, "build")
 LIB = os.path.join(PKG, "libsar.so")
-SOURCES = ["sar_gat.cu", "sar_graph.cu", "sar_host.cu", "sar_noalloc.cu", "sar_glue.cu", "sar_norm.cu", "sar_linear.cu", "sar_rgcn.cu"]
+SOURCES = ["sar_gat.cu", "sar_lean_fwd_f32.cu", "sar_lean_fwd_bf16.cu", "sar_lean_bwd_dst_f32.cu", "sar_lean_bwd_dst_bf16.cu",
+           "sar_graph.cu", "sar_host.cu", "sar_noalloc.cu",
+           "sar_glue.cu", "sar_norm.cu", "sar_linear.cu", "sar_rgcn.cu"]
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "--expt-relaxed-constexpr",
     "-DSAR_BUILT_FOR_SM=100", "-I", os.path.join(ROOT, "include"), "-I", CSRC,
 ]
+# extra flags for the lean-kernel translation units only (tuning experiments), e.g. SAR_LEAN_NVCC_EXTRA="-DSAR_LEAN_EXPERIMENT"
+LEAN_EXTRA = os.environ.get("SAR_LEAN_NVCC_EXTRA", "").split()
 
 
 def _nvcc() -> str:
@@ -43,49 +47,71 @@ def _cutlass_includes() -> list:
             base = os.path.join(root, sub) if root else ""
             if base and os.path.exists(os.path.join(base, "include", "cute", "arch", "mma_sm100_umma.hpp")):
                 return ["-I", os.path.join(base, "include"), "-I", os.path.join(base, "tools", "util", "include")]
-    raise RuntimeError("no CUTLASS header tree with sm100 support found (set CUTLASS_PATH)")
+    raise RuntimeError("sar_linear.cu needs a CUTLASS / CuTe header tree with sm100 support (cute/arch/mma_sm100_umma.hpp): "
+                       "none found in this Python environment's flashinfer or tilelang packages; set CUTLASS_PATH to the "
+                       "root of a CUTLASS checkout (the directory that holds include/ and tools/util/include/)")
 
 
-def _fingerprint() -> str:
+def _deps(path: str, seen=None) -> list:
+    """The file and every header of this library it includes, directly or not (quoted includes only)."""
+    import re
+    seen = seen if seen is not None else []
+    if path in seen or not os.path.exists(path):
+        return seen
+    seen.append(path)
+    for inc in re.findall(r'^\s*#\s*include\s+"([^"]+)"', open(path).read(), flags=re.M):
+        for base in (os.path.dirname(path), CSRC, os.path.join(ROOT, "include")):
+            cand = os.path.join(base, inc)
+            if os.path.exists(cand):
+                _deps(cand, seen)
+                break
+    return seen
+
+
+def _fingerprint(src: str) -> str:
+    """Hash of one source file, the headers it reaches and the compiler flags."""
     h = hashlib.sha256()
-    for name in sorted(os.listdir(CSRC)):
-        path = os.path.join(CSRC, name)
-        if os.path.isfile(path):
-            h.update(name.encode())
-            h.update(open(path, "rb").read())
-    h.update(open(os.path.join(ROOT, "include", "sar.h"), "rb").read())
-    h.update(" ".join(NVCC_FLAGS).encode())
+    for path in sorted(_deps(os.path.join(CSRC, src))):
+        h.update(os.path.basename(path).encode())
+        h.update(open(path, "rb").read())
+    h.update(" ".join(NVCC_FLAGS + (LEAN_EXTRA if src.startswith("sar_lean_") else [])).encode())
     return h.hexdigest()
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
+    """Compiles the sources whose contents (or headers, or flags) changed since their object was built, in
+    parallel, and links libsar.so when any object is new."""
     os.makedirs(OBJ, exist_ok=True)
-    stamp = os.path.join(OBJ, "fingerprint.txt")
-    fp = _fingerprint()
-    if not force and os.path.exists(LIB) and os.path.exists(stamp) and open(stamp).read() == fp:
-        return LIB
     nvcc = _nvcc()
     extra = ["-Xptxas", "-v"] if verbose else []
 
     def compile_one(src):
         obj = os.path.join(OBJ, src.replace(".cu", ".o"))
+        stamp = obj + ".fingerprint"
+        fp = _fingerprint(src)
+        if not force and os.path.exists(obj) and os.path.exists(stamp) and open(stamp).read() == fp:
+            return obj, False
         inc = _cutlass_includes() if src == "sar_linear.cu" else []
-        cmd = [nvcc, *NVCC_FLAGS, *inc, *extra, "-c", os.path.join(CSRC, src), "-o", obj]
+        lean = LEAN_EXTRA if src.startswith("sar_lean_") else []
+        cmd = [nvcc, *NVCC_FLAGS, *lean, *inc, *extra, "-c", os.path.join(CSRC, src), "-o", obj]
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             raise RuntimeError(f"nvcc failed on {src}:\n{r.stdout}\n{r.stderr}")
         if verbose:
             sys.stderr.write(r.stderr)
-        return obj
+        open(stamp, "w").write(fp)
+        return obj, True
 
-    with ThreadPoolExecutor(len(SOURCES)) as ex:
-        objs = list(ex.map(compile_one, SOURCES))
+    with ThreadPoolExecutor(min(len(SOURCES), os.cpu_count() or 4)) as ex:
+        results = list(ex.map(compile_one, SOURCES))
+    objs = [o for o, _ in results]
+    if not force and os.path.exists(LIB) and not any(new for _, new in results):
+        return LIB
     tmp = LIB + f".tmp{os.getpid()}"
     r = subprocess.run([nvcc, "-shared", "-o", tmp, *objs, "-Xcompiler", "-fPIC"], capture_output=True, text=True)
     if r.returncode != 0:
         raise RuntimeError(f"link failed:\n{r.stdout}\n{r.stderr}")
     os.replace(tmp, LIB)
-    open(stamp, "w").write(fp)
     return LIB
 
 

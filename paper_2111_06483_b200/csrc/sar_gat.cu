@@ -2,6 +2,7 @@
 // kernel selection and launches.  Declarations and contracts are in include/sar.h.
 #include "sar_gat_kernels.cuh"
 #include "sar_span_kernels.cuh"
+#include "sar_lean.cuh"
 #include "sar_dispatch.cuh"
 #include "sar_generic_kernels.cuh"
 
@@ -289,10 +290,29 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
     a.g = s.geom;
     a.sp = ma.sp;
     a.hvec = (H % 4 == 0) && sar_aligned(er_q, 16);
+    const bool lean = lean_applies(s, flags, slope, g->split, g->n_src) && sar_aligned(er_q, 16);
+    LeanArgs la{};
+    if (lean) {
+        la.n_rows = g->n_dst;
+        la.indptr = g->indptr;
+        la.indices = g->indices;
+        la.gather = feat_q;
+        la.el = el;
+        la.er = er_q;
+        la.m_out = m;
+        la.d_out = d;
+        la.out = out;
+        la.slope = slope;
+        la.sp = ma.sp;
+        la.sp.threshold = g->split->threshold;
+    }
     return dispatch(s, [&](auto cfg) -> sar_status {
         using C = decltype(cfg);
         using T = typename C::type;
-        SAR_TRY((launch_span<T, C::g, C::v, UFwd<C::v>::u, kFwd, kCapFwd, kMinBlocksFwd>(a, g->nnz, "gat_fwd", "gat_fwd_seg", st)));
+        if (lean)
+            SAR_TRY(s.t == SAR_F32 ? lean_fwd_f32(s, la, g->nnz, st) : lean_fwd_bf16(s, la, g->nnz, st));
+        else
+            SAR_TRY((launch_span<T, C::g, C::v, UFwd<C::v>::u, kFwd, kCapFwd, kMinBlocksFwd>(a, g->nnz, "gat_fwd", "gat_fwd_seg", st)));
         if (ma.sp.threshold > 0) {
             SAR_LAUNCH("gat_fwd_merge", st, gat_fwd_merge_kernel<T, C::g, C::v><<<blocks_for(ma.sp.n_long, C::g), kThreads, 0, st>>>(ma));
             SAR_TRY(sar_after_launch());
@@ -516,6 +536,25 @@ sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, c
     s1.sp = sa.sp;
     s1.hvec = (H % 4 == 0);
 
+    const bool lean_dst = whole && lean_applies(s, flags, slope, g->split, g->n_src) && sar_aligned(er_q, 16);
+    LeanArgs ld{};
+    if (lean_dst) {
+        ld.n_rows = g->n_dst;
+        ld.indptr = g->indptr;
+        ld.indices = g->indices;
+        ld.gather = feat_q;
+        ld.rowvec = gout;
+        ld.el = el;
+        ld.er = er_q;
+        ld.m = m;
+        ld.d = d;
+        ld.rec_out = rec;
+        ld.del = del;
+        ld.slope = slope;
+        ld.sp = da.sp;
+        ld.sp.threshold = g->split->threshold;
+    }
+
     return dispatch(s, [&](auto cfg) -> sar_status {
         using C = decltype(cfg);
         using T = typename C::type;
@@ -523,7 +562,10 @@ sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, c
         const size_t msmem = (size_t)kWarpsPerBlock * warp_smem_floats(s.geom.Hp, C::v, 4) * 4;
         if (g->n_dst > 0) {
             if (whole) {
-                SAR_TRY((launch_span<T, C::g, C::v, U, kBwdDst, kCapDst, kMinBlocksBwd>(d1, g->nnz, "gat_bwd_dst", "gat_bwd_dst_seg", st)));
+                if (lean_dst)
+                    SAR_TRY(s.t == SAR_F32 ? lean_bwd_dst_f32(s, ld, g->nnz, st) : lean_bwd_dst_bf16(s, ld, g->nnz, st));
+                else
+                    SAR_TRY((launch_span<T, C::g, C::v, U, kBwdDst, kCapDst, kMinBlocksBwd>(d1, g->nnz, "gat_bwd_dst", "gat_bwd_dst_seg", st)));
                 if (da.sp.threshold > 0) {
                     auto merge = gat_bwd_dst_merge_kernel<T, C::g, C::v, false>;
                     SAR_TRY(ensure_smem(merge, msmem));

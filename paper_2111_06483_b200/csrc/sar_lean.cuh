@@ -1,0 +1,51 @@
+// Host-side interface of the lean span kernels (internal): arguments, applicability test and the launchers,
+// which are compiled in translation units of their own (sar_lean_*.cu), one per pass and storage type.
+// They cover the forward pass and the destination-major backward pass.
+#pragma once
+
+#include "sar_rowkernels.cuh"
+
+namespace sar {
+
+struct LeanArgs {
+    long long n_rows;
+    const int64_t *indptr;
+    const int32_t *indices;
+    const void *gather;      // rows fetched per edge: feat
+    const void *rowvec;      // row-stationary vector of the backward pass: gout
+    const float *el, *er;    // el[row], er[col]
+    const float *m, *d;      // bwd-dst: final statistics of the row
+    float4 *rec_out;         // bwd-dst: record {el, m, 1/d, D} written per (row, head)
+    float *m_out, *d_out;    // forward
+    void *out;               // forward: out
+    float *del;              // bwd-dst
+    float slope;
+    SplitArgs sp;
+    int R;                   // rows per span (<= kMaxSpanRows)
+};
+
+constexpr int kLeanCap = 256;   // edges a chunk stages; rows and segments must not exceed it
+
+// Do the lean kernels cover this call?  Whole graph in one call, slope >= 0, heads in groups of four, rows of
+// exactly G*V vectors with V <= 2, the vectors of a head a power of two within one lane group, and a long-row
+// plan whose threshold fits a chunk (so that no row of the rows launch and no segment exceeds it), and a gathered
+// array of n_gathered rows whose 16-byte vectors can be counted in 32 bits (the staged row offsets are 32-bit).
+static inline bool lean_applies(const Shape &s, unsigned flags, float slope, const sar_split *sp, long long n_gathered) {
+    if (!s.fast || (flags & (SAR_FIRST | SAR_LAST | SAR_KEEP_NUMERATOR)) != (SAR_FIRST | SAR_LAST)) return false;
+    if (!(slope >= 0.f) || !sp || sp->threshold < 1 || sp->threshold > kLeanCap) return false;
+    const int H = s.geom.H, nv = s.geom.n_vec;
+    if (H % 4 != 0 || nv != s.G * s.V || s.V > 2 || nv % H != 0) return false;
+    const int vph = nv / H;
+    if (vph > s.G || (vph & (vph - 1)) != 0) return false;
+    if ((unsigned long long)nv * (unsigned long long)(n_gathered > 0 ? n_gathered : 0) > 0xffffffffull) return false;
+    return (s.G == 16 && s.V == 1 && H == 4) || (s.G == 32 && s.V == 1 && (H == 4 || H == 8)) ||
+           (s.G == 32 && s.V == 2 && H == 4);
+}
+
+// Rows launch + segment launch of one pass.
+sar_status lean_fwd_f32(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
+sar_status lean_fwd_bf16(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
+sar_status lean_bwd_dst_f32(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
+sar_status lean_bwd_dst_bf16(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
+
+}  // namespace sar

@@ -157,7 +157,7 @@ def test_graph_preparation_is_bit_exact(n, e, k):
         assert np.array_equal(s.long_seg.cpu().numpy(), np.concatenate([[0], np.cumsum(segs)]))
         assert s.n_seg == segs.sum()
     else:
-        assert g.whole.split is None
+        assert g.whole.split.n_long == 0 and g.whole.split.n_seg == 0
 
 
 def test_validate_part_flags_a_broken_graph():
