@@ -500,6 +500,48 @@ def time_spmm(g, x, gout, steps, warmup, peak, n, e, b):
             "gathered_bytes_per_direction": e * F * b}
 
 
+def storing_leg(st: AggStack, steps=2, warmup=1):
+    """The non-rematerialising baseline on the same stack: every layer's forward pass writes its attention
+    coefficients alpha[E,H] (kept until that layer's backward pass reads them).  Reports its step time and the
+    device memory both variants hold at their peak, measured by the allocator during one step each."""
+    import torch
+    B, g, cfg = st.B, st.g, st.cfg
+    n, H, F, L, e = st.n, st.H, st.F, st.L, st.e
+    torch.cuda.synchronize()
+    torch.cuda.reset_peak_memory_stats()
+    st.step_fused()
+    torch.cuda.synchronize()
+    remat_peak = torch.cuda.max_memory_allocated()
+    held = torch.cuda.memory_allocated()
+    need = L * e * H * 4 + B.sar_gat_storing_workspace_bytes(g.whole, H)
+    free = torch.cuda.mem_get_info()[0]
+    if need > 0.9 * free:
+        return {"skipped": f"needs {need} more bytes, {free} free", "remat_peak_mem_bytes": remat_peak}
+    torch.cuda.reset_peak_memory_stats()
+    alphas = [torch.empty((e, H), dtype=torch.float32, device=st.dev) for _ in range(L)]
+    ws = torch.empty(B.sar_gat_storing_workspace_bytes(g.whole, H), dtype=torch.uint8, device=st.dev)
+
+    def step():
+        for l in range(L):
+            B.sar_gat_fwd_storing(g.whole, st.feats[l], st.els[l], st.ers[l], H, F, cfg.slope, alphas[l], st.feats[l + 1])
+        gin = st.gout
+        for i, l in enumerate(reversed(range(L))):
+            B.sar_gat_bwd_storing(g.whole, st.feats[l], st.els[l], st.ers[l], alphas[l], gin, H, F, cfg.slope,
+                                  st.gbuf[i % 2], st.dels[l], st.ders[l], ws)
+            gin = st.gbuf[i % 2]
+
+    r = measure(step, steps, warmup)
+    storing_peak = torch.cuda.max_memory_allocated()
+    del alphas, ws
+    return {"ms_per_step": r["ms_per_step"], "steps": steps, "warmup": warmup,
+            "kernels": {k: v["avg_ms"] for k, v in r["kernels"].items()},
+            "peak_mem_bytes": storing_peak, "remat_peak_mem_bytes": remat_peak,
+            "extra_bytes_over_remat": storing_peak - remat_peak,
+            "attention_bytes_kept": L * e * H * 4, "stats_bytes_kept_by_remat": L * 2 * n * H * 4,
+            "held_before_bytes": held,
+            "kind": "plain two-step kernels, one warp per row, not tuned (sar_gat_fwd_storing / sar_gat_bwd_storing)"}
+
+
 def extra_workloads(dev, peak, args):
     """The other named workloads, a few steps each (configs 2-4 and the sum aggregation of config 3)."""
     import torch
@@ -522,6 +564,9 @@ def extra_workloads(dev, peak, args):
         for sch in schedules:
             r = measure(st.step(sch), steps, warmup, clocks_gpu=None)
             entry["schedules"][sch] = schedule_entry(st, sch, r, steps, peak)
+        if name == "dense":
+            entry["storing_baseline"] = storing_leg(st)
+            entry["storing_baseline"]["remat_ms_per_step"] = entry["schedules"]["fused"]["ms_per_step"]
         out[f"{name}_{dtype}"] = entry
         if name == "medium" and cfg.spmm_feat:
             x = workloads.normal_tensor((st.n, cfg.spmm_feat), cfg.seed, 20, device=dev, dtype=st.tdt)
@@ -768,6 +813,11 @@ def run_ours(args, rank, world, local_rank):
             ref = ceiling["csc_ms"] if name == "gat_bwd_src" else ceiling["csr_ms"]
             p_["frac_of_gather_ceiling"] = ref / p_["ms"]
 
+    storing = None
+    if extras:
+        storing = storing_leg(st)
+        storing["remat_ms_per_step"] = sched_out["fused"]["ms_per_step"] if "fused" in sched_out else None
+
     e2e = None
     if not args.no_e2e and not glue:
         st.feats, st.gbuf, st.feat_q, st.gbuf_q, st.gout, st.acc = None, None, None, None, None, None
@@ -777,6 +827,7 @@ def run_ours(args, rank, world, local_rank):
 
     others = None
     if extras:
+        step = None   # the bound method keeps the stack alive
         del st
         gc.collect()
         torch.cuda.empty_cache()
@@ -808,7 +859,7 @@ def run_ours(args, rank, world, local_rank):
             "peak_mem_bytes": peak_mem,
             "attention_bytes_if_stored": {"value": L * e * H * 4, "kind": "computed: 4 bytes x E x H x layers"},
             "stats_bytes_kept": L * 2 * n * H * 4,
-            "gather_ceiling": ceiling, "workloads": others,
+            "gather_ceiling": ceiling, "storing_baseline": storing, "workloads": others,
             "clocks": main["clocks"] or {}, "e2e": e2e, "cpu_baseline": cpu,
         }
         print(json.dumps(line), flush=True)

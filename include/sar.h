@@ -275,6 +275,26 @@ SAR_API sar_status sar_gat_bwd_fused(const sar_part *g, int32_t k, const int64_t
                              size_t workspace_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * The non-rematerialising baseline (Sec. 4.1 compares the fused kernels with the usual two-step implementation
+ * that materialises the attention coefficients; Sec. 3.3 describes what fusing avoids).  A deliberately plain
+ * variant of the same layer for MEASUREMENT AND TESTS ONLY, so that the memory and time of keeping O(E*H)
+ * attention can be observed next to the rematerialising path: the forward call writes alpha [nnz,H] float32
+ * (CSR order: row t*H.. belongs to edge t of g->indices) and then forms out from it; the backward call reads
+ * alpha back, writes the per-edge score gradients to its scratch and reduces them to del, der and dfeat.
+ * `g` is one partition holding all sources, with its CSC; nnz < 2^31 for the backward call.  One warp per
+ * row, no tuning, no long-row handling.  Scratch of the backward call: sar_gat_storing_workspace_bytes
+ * (4 bytes per (edge, head) plus 4 bytes per edge), 16-byte aligned.  Errors as for sar_gat_fwd / sar_gat_bwd.
+ * ------------------------------------------------------------------------------------------- */
+SAR_API size_t sar_gat_storing_workspace_bytes(const sar_part *g, int32_t H);
+SAR_API sar_status sar_gat_fwd_storing(const sar_part *g, const void *feat, const float *el, const float *er,
+                                       int32_t H, int32_t F, sar_dtype t, float slope, float *alpha, void *out,
+                                       void *stream);
+SAR_API sar_status sar_gat_bwd_storing(const sar_part *g, const void *feat, const float *el, const float *er,
+                                       const float *alpha, const void *gout, int32_t H, int32_t F, sar_dtype t,
+                                       float slope, void *dfeat, float *del, float *der, void *workspace,
+                                       size_t workspace_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Sum aggregation (Eq. 2; Sec. 3.2 "case 1").  out[i,:] (+)= sum over this partition's in-edges of
  * feat_q[j,:]; feat_q [n_src,F], out [n_dst,F], both of type t, float32 accumulation within the
  * call.  SAR_FIRST overwrites out, otherwise the partition's sum is added to it.  SAR_MEAN with

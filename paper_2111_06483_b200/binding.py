@@ -34,6 +34,7 @@ EXPORTS = [
     "sar_bn_bwd_apply", "sar_dropout", "sar_linear_workspace_bytes", "sar_linear", "sar_linear_bwd_input",
     "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd", "sar_axpby", "sar_bn_rstd", "sar_accumulate", "sar_round_to", "sar_bn_apply_act",
     "sar_bn_bwd_stats_act", "sar_bn_bwd_apply_act", "sar_csc_slice_indptr",
+    "sar_gat_storing_workspace_bytes", "sar_gat_fwd_storing", "sar_gat_bwd_storing",
 ]
 
 
@@ -71,7 +72,7 @@ def lib() -> ctypes.CDLL:
         L.sar_built_for_sm.restype = c_int32
         for name in ("sar_graph_workspace_bytes", "sar_gat_workspace_bytes", "sar_spmm_workspace_bytes",
                      "sar_gat_stack_arena_bytes", "sar_gat_bwd_noalloc_limit", "sar_gat_project_workspace_bytes",
-                     "sar_bn_workspace_bytes", "sar_linear_workspace_bytes"):
+                     "sar_bn_workspace_bytes", "sar_linear_workspace_bytes", "sar_gat_storing_workspace_bytes"):
             getattr(L, name).restype = c_size_t
         _lib = L
     return _lib
@@ -363,6 +364,28 @@ def sar_gat_bwd_fused(part: Part, bounds: Sequence[int], feat_q: Sequence[torch.
                                                         ctypes.c_int(_dtype(gout)), c_float(slope),
                                                         _ptr_array(dfeat_q), _ptr(del_), _ptr_array(der_q), w, wb,
                                                         _stream()))
+
+
+def sar_gat_storing_workspace_bytes(part: Part, H: int) -> int:
+    return int(lib().sar_gat_storing_workspace_bytes(byref(part.c), c_int32(H)))
+
+
+def sar_gat_fwd_storing(part: Part, feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor, H: int, F: int,
+                        slope: float, alpha: torch.Tensor, out: torch.Tensor) -> None:
+    """The storing baseline's forward pass: writes alpha [nnz,H] and out (measurement and tests only)."""
+    _check("sar_gat_fwd_storing", lib().sar_gat_fwd_storing(byref(part.c), _ptr(feat), _ptr(el), _ptr(er), c_int32(H),
+                                                            c_int32(F), ctypes.c_int(_dtype(feat)), c_float(slope),
+                                                            _ptr(alpha), _ptr(out), _stream()))
+
+
+def sar_gat_bwd_storing(part: Part, feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor, alpha: torch.Tensor,
+                        gout: torch.Tensor, H: int, F: int, slope: float, dfeat: torch.Tensor, del_: torch.Tensor,
+                        der: torch.Tensor, workspace: torch.Tensor) -> None:
+    w, wb = _ws(workspace)
+    _check("sar_gat_bwd_storing", lib().sar_gat_bwd_storing(byref(part.c), _ptr(feat), _ptr(el), _ptr(er), _ptr(alpha),
+                                                            _ptr(gout), c_int32(H), c_int32(F),
+                                                            ctypes.c_int(_dtype(feat)), c_float(slope), _ptr(dfeat),
+                                                            _ptr(del_), _ptr(der), w, wb, _stream()))
 
 
 def sar_spmm_agg(part: Part, feat_q: torch.Tensor, F: int, flags: int, deg_total: Optional[torch.Tensor],

@@ -19,7 +19,7 @@ CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(CSRC, "build")
 LIB = os.path.join(PKG, "libsar.so")
 SOURCES = ["sar_gat.cu", "sar_lean_fwd_f32.cu", "sar_lean_fwd_bf16.cu", "sar_lean_bwd_dst_f32.cu", "sar_lean_bwd_dst_bf16.cu",
-           "sar_graph.cu", "sar_host.cu", "sar_noalloc.cu",
+           "sar_graph.cu", "sar_host.cu", "sar_noalloc.cu", "sar_storing.cu",
            "sar_glue.cu", "sar_norm.cu", "sar_linear.cu", "sar_rgcn.cu"]
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",

@@ -311,7 +311,7 @@ __global__ void __launch_bounds__(32, MINB) lean_kernel(const LeanArgs a) {
                     for (int v = 0; v < V; ++v) {
                         unsigned long long src;   // base + offset * 16 in one multiply-add
                         asm("mad.wide.u32 %0, %1, 16, %2;\n" : "=l"(src) : "r"(ov[t]), "l"(gbase_v[v]));
-                        cp_async16_full(dst + (unsigned)((kq + t) * EPW * ROWB + v * 512), reinterpret_cast<const void *>(src));
+                        cp_async16_full(dst + (unsigned)((kq + t) * EPW * ROWB + v * G * 16), reinterpret_cast<const void *>(src));
                     }
             }
         };
@@ -472,7 +472,7 @@ __global__ void __launch_bounds__(32, MINB) lean_kernel(const LeanArgs a) {
                         for (int v = 0; v < V; ++v) {
                             const float wk = (k % 4 == 0) ? w4[v].x : (k % 4 == 1) ? w4[v].y : (k % 4 == 2) ? w4[v].z : w4[v].w;
                             f32x2 x[NP];
-                            Pairs<T>::get(lds128(ring_a + (unsigned)(k * EPW * ROWB + v * 512)), x);
+                            Pairs<T>::get(lds128(ring_a + (unsigned)(k * EPW * ROWB + v * G * 16)), x);
                             if constexpr (kF) {
                                 sv[v] += wk;
                                 const f32x2 w2 = pack2(wk, wk);
