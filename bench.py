@@ -370,11 +370,6 @@ class AggStack:
             nbytes = max(nbytes, B.sar_gat_workspace_bytes(p, H, F, B._dtype(self.feats[0])))
         self.ws = torch.empty(max(nbytes, 256), dtype=torch.uint8, device=dev)
         self.acc = None
-        cut = lambda t: [t[g.bounds[q]:] for q in range(K)]
-        self.feat_q = [cut(f) for f in self.feats]
-        self.er_q = [cut(x) for x in self.ers]
-        self.der_q = [cut(x) for x in self.ders]
-        self.gbuf_q = [cut(x) for x in self.gbuf]
 
     def can_run_sequential(self):
         return self.K == 1 or bool(self.g.parts)
@@ -383,12 +378,12 @@ class AggStack:
         B, g, c = self.B, self.g, self.cfg
         H, F, L = self.H, self.F, self.L
         for l in range(L):
-            B.sar_gat_fwd_fused(g.whole, g.bounds, self.feat_q[l], self.els[l], self.er_q[l], H, F, c.slope, self.ms[l],
+            B.sar_gat_fwd_fused(g.whole, g.bounds, self.feats[l], self.els[l], self.ers[l], H, F, c.slope, self.ms[l],
                                 self.ds[l], self.feats[l + 1], self.ws)
         gin = self.gout
         for i, l in enumerate(reversed(range(L))):
-            B.sar_gat_bwd_fused(g.whole, g.bounds, self.feat_q[l], self.els[l], self.er_q[l], self.ms[l], self.ds[l], gin,
-                                H, F, c.slope, self.gbuf_q[i % 2], self.dels[l], self.der_q[l], self.ws)
+            B.sar_gat_bwd_fused(g.whole, g.bounds, self.feats[l], self.els[l], self.ers[l], self.ms[l], self.ds[l], gin,
+                                H, F, c.slope, self.gbuf[i % 2], self.dels[l], self.ders[l], self.ws)
             gin = self.gbuf[i % 2]
 
     def step_sequential(self):
@@ -587,8 +582,6 @@ def make_glue_step(args, st: AggStack):
     n, H, F, L, tdt = st.n, st.H, st.F, st.L, st.tdt
     feats, els, ers, ms, ds, dels, ders = st.feats, st.els, st.ers, st.ms, st.ds, st.dels, st.ders
     gout, gbuf, ws = st.gout, st.gbuf, st.ws
-    feat_q, er_q, der_q, gbuf_q = st.feat_q, st.er_q, st.der_q, st.gbuf_q
-    cut = lambda t: [t[g.bounds[q]:] for q in range(st.K)]
     a_ls = [workloads.normal_tensor((H, F), cfg.seed, 16 * l + 14, device=dev) / F ** 0.5 for l in range(L)]
     a_rs = [workloads.normal_tensor((H, F), cfg.seed, 16 * l + 15, device=dev) / F ** 0.5 for l in range(L)]
     da_l, da_r = torch.empty((H, F), device=dev), torch.empty((H, F), device=dev)
@@ -599,7 +592,6 @@ def make_glue_step(args, st: AggStack):
         D = H * F
         Ws = [(workloads.normal_tensor((D, D), cfg.seed, 16 * l + 9, device=dev) / D ** 0.5).to(tdt) for l in range(L)]
         zs = [torch.empty((n, H, F), dtype=tdt, device=dev) for _ in range(L)]
-        z_q = [cut(z) for z in zs]
         dW = torch.empty((D, D), dtype=torch.float32, device=dev)
         lws = torch.empty(B.sar_linear_workspace_bytes(n, D, D), dtype=torch.uint8, device=dev)
         flat = lambda x: x.view(n, D)
@@ -621,7 +613,7 @@ def make_glue_step(args, st: AggStack):
                 for l in range(L):
                     B.sar_linear(flat(hs[l]), Ws[l], flat(zs[l]), lws)
                     B.sar_gat_project(zs[l], a_ls[l], a_rs[l], els[l], ers[l], 0)
-                    B.sar_gat_fwd_fused(g.whole, g.bounds, z_q[l], els[l], er_q[l], H, F, cfg.slope, ms[l], ds[l],
+                    B.sar_gat_fwd_fused(g.whole, g.bounds, zs[l], els[l], ers[l], H, F, cfg.slope, ms[l], ds[l],
                                         feats[l + 1], ws)
                     if l + 1 < L:
                         x = flat(feats[l + 1])
@@ -630,8 +622,8 @@ def make_glue_step(args, st: AggStack):
                         B.sar_bn_apply_act(x, bn_mean[l], bn_rstd[l], None, None, act, p_drop, seeds[l], flat(hs[l + 1]))
                 gin = gout
                 for l in reversed(range(L)):
-                    B.sar_gat_bwd_fused(g.whole, g.bounds, z_q[l], els[l], er_q[l], ms[l], ds[l], gin, H, F, cfg.slope,
-                                        gbuf_q[0], dels[l], der_q[l], ws)
+                    B.sar_gat_bwd_fused(g.whole, g.bounds, zs[l], els[l], ers[l], ms[l], ds[l], gin, H, F, cfg.slope,
+                                        gbuf[0], dels[l], ders[l], ws)
                     B.sar_gat_project_bwd(zs[l], a_ls[l], a_rs[l], dels[l], ders[l], gbuf[0], da_l, da_r, pws, 0)
                     B.sar_linear_bwd_weight(flat(hs[l]), flat(gbuf[0]), dW, lws)
                     B.sar_linear_bwd_input(flat(gbuf[0]), Ws[l], flat(gbuf[1]), lws)
@@ -651,15 +643,15 @@ def make_glue_step(args, st: AggStack):
                     B.sar_relu(feats[l])
                 B.sar_linear(flat(feats[l]), Ws[l], flat(zs[l]), lws)
                 B.sar_gat_project(zs[l], a_ls[l], a_rs[l], els[l], ers[l], 0)
-                B.sar_gat_fwd_fused(g.whole, g.bounds, z_q[l], els[l], er_q[l], H, F, cfg.slope, ms[l], ds[l],
+                B.sar_gat_fwd_fused(g.whole, g.bounds, zs[l], els[l], ers[l], H, F, cfg.slope, ms[l], ds[l],
                                     feats[l + 1], ws)
             B.sar_relu(feats[L])
             gin = gout
             B.sar_relu_bwd(feats[L], gin)  # masks gout in place on the first pass; the same mask every step
             for l in reversed(range(L)):
                 # gbuf[0]: gradient w.r.t. z of this layer, gbuf[1]: w.r.t. the layer's input
-                B.sar_gat_bwd_fused(g.whole, g.bounds, z_q[l], els[l], er_q[l], ms[l], ds[l], gin, H, F, cfg.slope,
-                                    gbuf_q[0], dels[l], der_q[l], ws)
+                B.sar_gat_bwd_fused(g.whole, g.bounds, zs[l], els[l], ers[l], ms[l], ds[l], gin, H, F, cfg.slope,
+                                        gbuf[0], dels[l], ders[l], ws)
                 B.sar_gat_project_bwd(zs[l], a_ls[l], a_rs[l], dels[l], ders[l], gbuf[0], da_l, da_r, pws, 0)
                 B.sar_linear_bwd_weight(flat(feats[l]), flat(gbuf[0]), dW, lws)
                 B.sar_linear_bwd_input(flat(gbuf[0]), Ws[l], flat(gbuf[1]), lws)
@@ -671,14 +663,14 @@ def make_glue_step(args, st: AggStack):
     def step():
         for l in range(L):  # the ReLU closing layer l-1 runs inside layer l's projection
             B.sar_gat_project(feats[l], a_ls[l], a_rs[l], els[l], ers[l], B.SAR_GLUE_RELU if l > 0 else 0)
-            B.sar_gat_fwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], H, F, cfg.slope, ms[l], ds[l],
+            B.sar_gat_fwd_fused(g.whole, g.bounds, feats[l], els[l], ers[l], H, F, cfg.slope, ms[l], ds[l],
                                 feats[l + 1], ws)
         B.sar_relu(feats[L])
         gin = gout
         B.sar_relu_bwd(feats[L], gin)  # masks gout in place on the first pass; the same mask every step
         for i, l in enumerate(reversed(range(L))):
-            B.sar_gat_bwd_fused(g.whole, g.bounds, feat_q[l], els[l], er_q[l], ms[l], ds[l], gin, H, F, cfg.slope,
-                                gbuf_q[i % 2], dels[l], der_q[l], ws)
+            B.sar_gat_bwd_fused(g.whole, g.bounds, feats[l], els[l], ers[l], ms[l], ds[l], gin, H, F, cfg.slope,
+                                gbuf[i % 2], dels[l], ders[l], ws)
             gin = gbuf[i % 2]
             B.sar_gat_project_bwd(feats[l], a_ls[l], a_rs[l], dels[l], ders[l], gin, da_l, da_r, pws,
                                   B.SAR_GLUE_RELU if l > 0 else 0)
@@ -820,7 +812,7 @@ def run_ours(args, rank, world, local_rank):
 
     e2e = None
     if not args.no_e2e and not glue:
-        st.feats, st.gbuf, st.feat_q, st.gbuf_q, st.gout, st.acc = None, None, None, None, None, None
+        st.feats, st.gbuf, st.gout, st.acc = None, None, None, None
         gc.collect()
         torch.cuda.empty_cache()
         e2e = time_e2e(st, args, dist, world)

@@ -223,15 +223,17 @@ SAR_API sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const floa
                        int32_t F, sar_dtype t, float slope, uint32_t flags, float *acc, float *m, float *d,
                        void *out, void *workspace, size_t workspace_bytes, void *stream);
 
-/* The whole loop of Algorithm 1 in one launch, row-stationary: `g` is the UN-split graph (global
- * source ids, n_src = all sources); partition q owns the sources bounds[q] <= j < bounds[q+1]
- * (HOST bounds) whose rows live at feat_q[q] / er_q[q] (HOST arrays of k DEVICE pointers, e.g.
- * buffers fetched from k different owners).  Each destination walks its in-edges in ascending
- * source order, i.e. partition after partition, carrying (running max, normaliser, numerator) in
- * registers with the same correction rule, so nothing of size n_dst*H*F is re-read between
- * partitions.  Writes out, m, d as sar_gat_fwd does with SAR_LAST. */
-SAR_API sar_status sar_gat_fwd_fused(const sar_part *g, int32_t k, const int64_t *bounds, const void *const *feat_q,
-                             const float *el, const float *const *er_q, int32_t H, int32_t F, sar_dtype t,
+/* The whole loop of Algorithm 1 in one walk, row-stationary: `g` is the UN-split graph (global source ids,
+ * n_src = all sources) and partition q owns the sources bounds[q] <= j < bounds[q+1] (HOST array of k+1
+ * entries, bounds[0] = 0, bounds[k] = n_src, non-decreasing; k <= SAR_MAX_PARTS).  The partitions must be the
+ * slices of ONE array each: feat [n_src,H,F] and er [n_src,H] hold partition q's rows at rows bounds[q] ..
+ * bounds[q+1].  Each destination walks its in-edges in ascending source order, i.e. partition after partition,
+ * carrying (running max, normaliser, numerator) in registers, so nothing of size n_dst*H*F is written or re-read
+ * between partitions and the kernels see one partition; k and bounds only describe where the partitions lie
+ * (they are checked, and a caller whose partitions live in separately allocated buffers uses the call-by-call
+ * sar_gat_fwd instead).  Writes out, m, d as sar_gat_fwd does with SAR_FIRST | SAR_LAST. */
+SAR_API sar_status sar_gat_fwd_fused(const sar_part *g, int32_t k, const int64_t *bounds, const void *feat,
+                             const float *el, const float *er, int32_t H, int32_t F, sar_dtype t,
                              float slope, float *m, float *d, void *out, void *workspace,
                              size_t workspace_bytes, void *stream);
 
@@ -265,13 +267,12 @@ SAR_API sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const floa
                        float slope, uint32_t flags, void *dfeat_q, float *del, float *der_q, void *workspace,
                        size_t workspace_bytes, void *stream);
 
-/* The whole loop of Algorithm 2 on the un-split graph (see sar_gat_fwd_fused for the argument
- * conventions): dfeat_q[q], der_q[q] are HOST arrays of k DEVICE pointers to each partition's
- * gradient buffers. */
-SAR_API sar_status sar_gat_bwd_fused(const sar_part *g, int32_t k, const int64_t *bounds, const void *const *feat_q,
-                             const float *el, const float *const *er_q, const float *m, const float *d,
+/* The whole loop of Algorithm 2 on the un-split graph (see sar_gat_fwd_fused for the argument conventions):
+ * dfeat [n_src,H,F] and der [n_src,H] receive every partition's gradients at its rows. */
+SAR_API sar_status sar_gat_bwd_fused(const sar_part *g, int32_t k, const int64_t *bounds, const void *feat,
+                             const float *el, const float *er, const float *m, const float *d,
                              const void *gout, int32_t H, int32_t F, sar_dtype t, float slope,
-                             void *const *dfeat_q, float *del, float *const *der_q, void *workspace,
+                             void *dfeat, float *del, float *der, void *workspace,
                              size_t workspace_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------------------------
@@ -443,6 +444,17 @@ SAR_API sar_status sar_rgcn_basis_bwd(int32_t R, int32_t B, int64_t size, const 
  * n = 0 is allowed (statistics and sums are written as zeros).  Errors as for the other streaming calls.
  * ------------------------------------------------------------------------------------------- */
 SAR_API size_t sar_bn_workspace_bytes(int32_t C);
+/* The combination rule across R workers (Sec. 3.4, "Batch normalization"), on HOST arrays: what is communicated
+ * is a few floats per column, so the workers gather each other's triples with whatever transport they use and
+ * every worker evaluates the same rule in the same (rank) order, in float64.
+ *   sar_bn_combine_moments  n_r [R], mean_r [R,C], m2_r [R,C] (row r = worker r's local statistics from
+ *                           sar_bn_stats) -> *n_all = sum n_r, mean[c] = sum_r n_r mean_r / n_all,
+ *                           m2[c] = sum_r [ m2_r + n_r (mean_r - mean)^2 ]  (all rows of all workers).
+ *   sar_bn_combine_sums     sums_r [R,count] -> sums[i] = sum_r sums_r[r,i] (the backward statistics).
+ * No device work, no stream.  Errors: SAR_ERR_INVALID_ARG (R < 1, negative counts, NULL arrays). */
+SAR_API sar_status sar_bn_combine_moments(int32_t R, int32_t C, const int64_t *n_r, const float *mean_r,
+                                          const float *m2_r, int64_t *n_all, float *mean, float *m2);
+SAR_API sar_status sar_bn_combine_sums(int32_t R, int64_t count, const float *sums_r, float *sums);
 SAR_API sar_status sar_bn_stats(int64_t n, int32_t C, sar_dtype t, const void *x, float *mean, float *m2,
                                 void *workspace, size_t workspace_bytes, void *stream);
 SAR_API sar_status sar_bn_rstd(int32_t C, const float *m2, int64_t count, float eps, float *rstd, void *stream);

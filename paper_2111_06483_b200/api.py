@@ -153,7 +153,8 @@ def gat_workspace(part: B.Part, H: int, F: int, dtype: torch.dtype) -> torch.Ten
 
 def gat_forward(g: Graph, feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor, slope: float,
                 workspace: Optional[torch.Tensor] = None, mode: str = "fused", keep_numerator: bool = False):
-    """Forward over the K partitions.  mode "fused": one row-stationary launch (sar_gat_fwd_fused);
+    """Forward over the K partitions.  mode "fused": one row-stationary walk over the un-split graph, the
+    partitions being slices of the arrays (sar_gat_fwd_fused);
     mode "stateful": K calls of sar_gat_fwd with the running state in global memory (Algorithm 1).
     keep_numerator (stateful mode): returns (out, m, d, acc) with the complete float32 numerator in acc,
     which gat_backward can take in place of `out` for the row dot."""
@@ -164,9 +165,7 @@ def gat_forward(g: Graph, feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor
     out = torch.empty((g.n, H, F), dtype=feat.dtype, device=dev)
     if mode == "fused":
         ws = workspace if workspace is not None else gat_workspace(g.whole, H, F, feat.dtype)
-        feat_q = [feat[g.bounds[q]:] for q in range(g.k)]
-        er_q = [er[g.bounds[q]:] for q in range(g.k)]
-        B.sar_gat_fwd_fused(g.whole, g.bounds, feat_q, el, er_q, H, F, slope, m, d, out, ws)
+        B.sar_gat_fwd_fused(g.whole, g.bounds, feat, el, er, H, F, slope, m, d, out, ws)
         return out, m, d
     assert g.parts, "stateful mode needs Graph.from_coo(..., build_parts=True)"
     acc = torch.empty((g.n, H, F), dtype=torch.float32, device=dev) if (g.k > 1 or keep_numerator) else None
@@ -192,9 +191,7 @@ def gat_backward(g: Graph, feat: torch.Tensor, el: torch.Tensor, er: torch.Tenso
     der = torch.empty((g.n, H), dtype=torch.float32, device=dev)
     if mode == "fused":
         ws = workspace if workspace is not None else gat_workspace(g.whole, H, F, feat.dtype)
-        sl = lambda t: [t[g.bounds[q]:] for q in range(g.k)]
-        B.sar_gat_bwd_fused(g.whole, g.bounds, sl(feat), el, sl(er), m, d, gout, H, F, slope, sl(dfeat), del_,
-                            sl(der), ws)
+        B.sar_gat_bwd_fused(g.whole, g.bounds, feat, el, er, m, d, gout, H, F, slope, dfeat, del_, der, ws)
         return dfeat, del_, der
     assert g.parts and (out is not None or acc is not None)
     nbytes = max(B.sar_gat_workspace_bytes(p, H, F, B._dtype(feat)) for p in g.parts)
@@ -268,32 +265,36 @@ def spmm_scaled(part: B.Part, feat: torch.Tensor, src_scale: Optional[torch.Tens
 # batch normalisation over the node dimension (Sec. 3.4); with `group` the statistics are combined across
 # the workers of a torch.distributed process group (each holds some of the rows): a few floats per column.
 
+def _gather_rows(row: torch.Tensor, group) -> torch.Tensor:
+    """Every worker's copy of `row` (a flat tensor), stacked in rank order, on the HOST."""
+    import torch.distributed as dist
+    world = dist.get_world_size(group)
+    parts = [torch.empty_like(row) for _ in range(world)]
+    dist.all_gather(parts, row.contiguous(), group=group)
+    return torch.stack(parts).cpu()
+
+
 def combine_moments(n_local: int, mean: torch.Tensor, m2: torch.Tensor, group=None):
     """(n, mean, m2 = sum of squared deviations) of the local rows -> the same for all rows of all workers.
-    Pairwise rule: mean = sum n_r mean_r / N;  m2 = sum [m2_r + n_r (mean_r - mean)^2].  float64 on the way."""
+    torch.distributed only moves the triples; the rule of Sec. 3.4 is the library's sar_bn_combine_moments."""
     if group is None:
         return n_local, mean, m2
-    import torch.distributed as dist
-    acc = torch.cat([torch.tensor([float(n_local)], dtype=torch.float64, device=mean.device),
-                     mean.double() * n_local])
-    dist.all_reduce(acc, group=group)
-    n_all = int(round(float(acc[0])))
-    mean_all = acc[1:] / max(n_all, 1)
-    m2_part = m2.double() + n_local * (mean.double() - mean_all) ** 2
-    dist.all_reduce(m2_part, group=group)
-    return n_all, mean_all.float(), m2_part.float()
+    n_r = _gather_rows(torch.tensor([int(n_local)], dtype=torch.int64, device=mean.device), group)[:, 0].tolist()
+    rows = _gather_rows(torch.cat([mean.float(), m2.float()]), group)
+    C = mean.numel()
+    n_all, mean_all, m2_all = B.sar_bn_combine_moments(n_r, rows[:, :C], rows[:, C:])
+    return n_all, mean_all.to(mean.device), m2_all.to(mean.device)
 
 
 def combine_sums(tensors, group=None):
-    """Element-wise sums over the workers (the backward statistics)."""
+    """Element-wise sums over the workers (the backward statistics), by the library's sar_bn_combine_sums."""
     if group is None:
         return tensors
-    import torch.distributed as dist
-    flat = torch.cat([t.double().flatten() for t in tensors])
-    dist.all_reduce(flat, group=group)
+    rows = _gather_rows(torch.cat([t.float().flatten() for t in tensors]), group)
+    flat = B.sar_bn_combine_sums(rows)
     out, o = [], 0
     for t in tensors:
-        out.append(flat[o:o + t.numel()].reshape(t.shape).to(t.dtype))
+        out.append(flat[o:o + t.numel()].reshape(t.shape).to(device=t.device, dtype=t.dtype))
         o += t.numel()
     return out
 

@@ -34,7 +34,8 @@ EXPORTS = [
     "sar_bn_bwd_apply", "sar_dropout", "sar_linear_workspace_bytes", "sar_linear", "sar_linear_bwd_input",
     "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd", "sar_axpby", "sar_bn_rstd", "sar_accumulate", "sar_round_to", "sar_bn_apply_act",
     "sar_bn_bwd_stats_act", "sar_bn_bwd_apply_act", "sar_csc_slice_indptr",
-    "sar_gat_storing_workspace_bytes", "sar_gat_fwd_storing", "sar_gat_bwd_storing",
+    "sar_gat_storing_workspace_bytes", "sar_gat_fwd_storing", "sar_gat_bwd_storing", "sar_bn_combine_moments",
+    "sar_bn_combine_sums",
 ]
 
 
@@ -317,19 +318,15 @@ def sar_gat_fwd(part: Part, feat_q: torch.Tensor, el: torch.Tensor, er_q: torch.
                                             _ptr(m), _ptr(d), _ptr(out), w, wb, _stream()))
 
 
-def _ptr_array(ts: Sequence[torch.Tensor]):
-    return (c_void_p * len(ts))(*[t.data_ptr() for t in ts])
-
-
-def sar_gat_fwd_fused(part: Part, bounds: Sequence[int], feat_q: Sequence[torch.Tensor], el: torch.Tensor,
-                      er_q: Sequence[torch.Tensor], H: int, F: int, slope: float, m: torch.Tensor, d: torch.Tensor,
-                      out: torch.Tensor, workspace: Optional[torch.Tensor]) -> None:
+def sar_gat_fwd_fused(part: Part, bounds: Sequence[int], feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor,
+                      H: int, F: int, slope: float, m: torch.Tensor, d: torch.Tensor, out: torch.Tensor,
+                      workspace: Optional[torch.Tensor]) -> None:
     k = len(bounds) - 1
     w, wb = _ws(workspace)
-    _check("sar_gat_fwd_fused", lib().sar_gat_fwd_fused(byref(part.c), c_int32(k), _host_i64(bounds),
-                                                        _ptr_array(feat_q), _ptr(el), _ptr_array(er_q), c_int32(H),
-                                                        c_int32(F), ctypes.c_int(_dtype(feat_q[0])), c_float(slope),
-                                                        _ptr(m), _ptr(d), _ptr(out), w, wb, _stream()))
+    _check("sar_gat_fwd_fused", lib().sar_gat_fwd_fused(byref(part.c), c_int32(k), _host_i64(bounds), _ptr(feat),
+                                                        _ptr(el), _ptr(er), c_int32(H), c_int32(F),
+                                                        ctypes.c_int(_dtype(feat)), c_float(slope), _ptr(m), _ptr(d),
+                                                        _ptr(out), w, wb, _stream()))
 
 
 def sar_gat_bwd_prepare(n_dst: int, H: int, F: int, out_or_acc: torch.Tensor, acc_is_numerator: bool,
@@ -352,18 +349,15 @@ def sar_gat_bwd(part: Part, feat_q: torch.Tensor, el: torch.Tensor, er_q: torch.
                                             w, wb, _stream()))
 
 
-def sar_gat_bwd_fused(part: Part, bounds: Sequence[int], feat_q: Sequence[torch.Tensor], el: torch.Tensor,
-                      er_q: Sequence[torch.Tensor], m: torch.Tensor, d: torch.Tensor, gout: torch.Tensor, H: int,
-                      F: int, slope: float, dfeat_q: Sequence[torch.Tensor], del_: torch.Tensor,
-                      der_q: Sequence[torch.Tensor], workspace: torch.Tensor) -> None:
+def sar_gat_bwd_fused(part: Part, bounds: Sequence[int], feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor,
+                      m: torch.Tensor, d: torch.Tensor, gout: torch.Tensor, H: int, F: int, slope: float,
+                      dfeat: torch.Tensor, del_: torch.Tensor, der: torch.Tensor, workspace: torch.Tensor) -> None:
     k = len(bounds) - 1
     w, wb = _ws(workspace)
-    _check("sar_gat_bwd_fused", lib().sar_gat_bwd_fused(byref(part.c), c_int32(k), _host_i64(bounds),
-                                                        _ptr_array(feat_q), _ptr(el), _ptr_array(er_q), _ptr(m),
-                                                        _ptr(d), _ptr(gout), c_int32(H), c_int32(F),
-                                                        ctypes.c_int(_dtype(gout)), c_float(slope),
-                                                        _ptr_array(dfeat_q), _ptr(del_), _ptr_array(der_q), w, wb,
-                                                        _stream()))
+    _check("sar_gat_bwd_fused", lib().sar_gat_bwd_fused(byref(part.c), c_int32(k), _host_i64(bounds), _ptr(feat),
+                                                        _ptr(el), _ptr(er), _ptr(m), _ptr(d), _ptr(gout), c_int32(H),
+                                                        c_int32(F), ctypes.c_int(_dtype(gout)), c_float(slope),
+                                                        _ptr(dfeat), _ptr(del_), _ptr(der), w, wb, _stream()))
 
 
 def sar_gat_storing_workspace_bytes(part: Part, H: int) -> int:
@@ -453,6 +447,31 @@ def sar_gat_stack_host(part: Part, bounds: Sequence[int], H: int, F: int, slope:
 
 def sar_bn_workspace_bytes(C: int) -> int:
     return int(lib().sar_bn_workspace_bytes(c_int32(C)))
+
+
+def sar_bn_combine_moments(n_r: Sequence[int], mean_r: torch.Tensor, m2_r: torch.Tensor):
+    """HOST tensors mean_r, m2_r [R, C] float32 (row r: worker r's local statistics) -> (n_all, mean [C], m2 [C])."""
+    R, C = mean_r.shape
+    assert (not mean_r.is_cuda) and (not m2_r.is_cuda) and mean_r.dtype == torch.float32 and m2_r.dtype == torch.float32
+    mean_r, m2_r = mean_r.contiguous(), m2_r.contiguous()
+    mean, m2 = torch.empty(C, dtype=torch.float32), torch.empty(C, dtype=torch.float32)
+    n_all = c_int64(0)
+    _check("sar_bn_combine_moments", lib().sar_bn_combine_moments(c_int32(R), c_int32(C), _host_i64(n_r),
+                                                                  c_void_p(mean_r.data_ptr()), c_void_p(m2_r.data_ptr()),
+                                                                  byref(n_all), c_void_p(mean.data_ptr()),
+                                                                  c_void_p(m2.data_ptr())))
+    return int(n_all.value), mean, m2
+
+
+def sar_bn_combine_sums(sums_r: torch.Tensor) -> torch.Tensor:
+    """HOST tensor sums_r [R, count] float32 -> their sum over the workers [count], added in rank order."""
+    assert (not sums_r.is_cuda) and sums_r.dtype == torch.float32
+    sums_r = sums_r.contiguous()
+    R, count = sums_r.shape
+    out = torch.empty(count, dtype=torch.float32)
+    _check("sar_bn_combine_sums", lib().sar_bn_combine_sums(c_int32(R), c_int64(count), c_void_p(sums_r.data_ptr()),
+                                                            c_void_p(out.data_ptr())))
+    return out
 
 
 def sar_bn_stats(x: torch.Tensor, mean: torch.Tensor, m2: torch.Tensor, workspace: torch.Tensor) -> None:

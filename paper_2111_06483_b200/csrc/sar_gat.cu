@@ -321,14 +321,6 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
     });
 }
 
-// Are the k per-partition buffers one contiguous array cut at `bounds`?
-static bool contiguous(const void *const *ptrs, int32_t k, const int64_t *bounds, size_t row_bytes) {
-    for (int32_t q = 0; q < k; ++q)
-        if (static_cast<const char *>(ptrs[q]) != static_cast<const char *>(ptrs[0]) + (size_t)bounds[q] * row_bytes)
-            return false;
-    return true;
-}
-
 static sar_status check_fused(const sar_part *g, int32_t k, const int64_t *bounds) {
     if (!g || !bounds || k < 1) return SAR_ERR_INVALID_ARG;
     if (k > SAR_MAX_PARTS) return SAR_ERR_UNSUPPORTED;
@@ -338,21 +330,13 @@ static sar_status check_fused(const sar_part *g, int32_t k, const int64_t *bound
     return SAR_OK;
 }
 
-sar_status sar_gat_fwd_fused(const sar_part *g, int32_t k, const int64_t *bounds, const void *const *feat_q,
-                             const float *el, const float *const *er_q, int32_t H, int32_t F, sar_dtype t,
-                             float slope, float *m, float *d, void *out, void *workspace,
-                             size_t workspace_bytes, void *stream) {
+sar_status sar_gat_fwd_fused(const sar_part *g, int32_t k, const int64_t *bounds, const void *feat, const float *el,
+                             const float *er, int32_t H, int32_t F, sar_dtype t, float slope, float *m, float *d,
+                             void *out, void *workspace, size_t workspace_bytes, void *stream) {
     SAR_TRY(check_fused(g, k, bounds));
-    if (!feat_q || !er_q || H < 1 || F < 1) return SAR_ERR_INVALID_ARG;
-    for (int32_t q = 0; q < k; ++q)
-        if (!feat_q[q] || !er_q[q]) return SAR_ERR_INVALID_ARG;
     // Sources ascend within a row, so walking a row once IS the partition-after-partition visit.
-    // Buffers that form one array need no per-edge partition lookup.
-    if (!contiguous(feat_q, k, bounds, (size_t)H * F * sar_elem_size(t)) ||
-        !contiguous(reinterpret_cast<const void *const *>(er_q), k, bounds, (size_t)H * 4))
-        return SAR_ERR_UNSUPPORTED;
-    return sar_gat_fwd(g, feat_q[0], el, er_q[0], H, F, t, slope, SAR_FIRST | SAR_LAST, nullptr, m, d, out,
-                       workspace, workspace_bytes, stream);
+    return sar_gat_fwd(g, feat, el, er, H, F, t, slope, SAR_FIRST | SAR_LAST, nullptr, m, d, out, workspace,
+                       workspace_bytes, stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -595,22 +579,13 @@ sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, c
     });
 }
 
-sar_status sar_gat_bwd_fused(const sar_part *g, int32_t k, const int64_t *bounds, const void *const *feat_q,
-                             const float *el, const float *const *er_q, const float *m, const float *d,
-                             const void *gout, int32_t H, int32_t F, sar_dtype t, float slope,
-                             void *const *dfeat_q, float *del, float *const *der_q, void *workspace,
+sar_status sar_gat_bwd_fused(const sar_part *g, int32_t k, const int64_t *bounds, const void *feat, const float *el,
+                             const float *er, const float *m, const float *d, const void *gout, int32_t H, int32_t F,
+                             sar_dtype t, float slope, void *dfeat, float *del, float *der, void *workspace,
                              size_t workspace_bytes, void *stream) {
     SAR_TRY(check_fused(g, k, bounds));
-    if (!feat_q || !er_q || !dfeat_q || !der_q || H < 1 || F < 1) return SAR_ERR_INVALID_ARG;
-    for (int32_t q = 0; q < k; ++q)
-        if (!feat_q[q] || !er_q[q] || !dfeat_q[q] || !der_q[q]) return SAR_ERR_INVALID_ARG;
-    const size_t rb = (size_t)H * F * sar_elem_size(t);
-    if (!contiguous(feat_q, k, bounds, rb) || !contiguous(reinterpret_cast<const void *const *>(dfeat_q), k, bounds, rb) ||
-        !contiguous(reinterpret_cast<const void *const *>(er_q), k, bounds, (size_t)H * 4) ||
-        !contiguous(reinterpret_cast<const void *const *>(der_q), k, bounds, (size_t)H * 4))
-        return SAR_ERR_UNSUPPORTED;
-    return sar_gat_bwd(g, feat_q[0], el, er_q[0], m, d, gout, H, F, t, slope, SAR_FIRST | SAR_LAST, dfeat_q[0], del,
-                       der_q[0], workspace, workspace_bytes, stream);
+    return sar_gat_bwd(g, feat, el, er, m, d, gout, H, F, t, slope, SAR_FIRST | SAR_LAST, dfeat, del, der, workspace,
+                       workspace_bytes, stream);
 }
 
 // ---------------------------------------------------------------------------------------------

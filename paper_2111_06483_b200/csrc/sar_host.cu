@@ -163,22 +163,9 @@ sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bound
     SAR_CUDA_STEP(cudaMemcpyAsync(ga, io->gout, row_b, cudaMemcpyHostToDevice, up));
     SAR_CUDA_STEP(cudaEventRecord(e_gout, up));
 
-    // per-partition pointer lists (one array cut at `bounds`)
-    std::vector<const void *> fq(k);
-    std::vector<void *> dfq(k);
-    std::vector<const float *> erq(k);
-    std::vector<float *> derq(k);
-    const size_t rb = (size_t)H * F * sar_elem_size(io->t);
-    auto cut = [&](const void *base, size_t stride, int q) {
-        return static_cast<const char *>(base) + (size_t)bounds[q] * stride;
-    };
     for (int l = 0; l < L; ++l) {
-        for (int q = 0; q < k; ++q) {
-            fq[q] = cut(feat[l], rb, q);
-            erq[q] = reinterpret_cast<const float *>(cut(er[l], (size_t)H * 4, q));
-        }
         SAR_CUDA_STEP(cudaStreamWaitEvent(st, e_in[l], 0));
-        SAR_STEP(sar_gat_fwd_fused(g, k, bounds, fq.data(), el[l], erq.data(), H, F, io->t, io->slope, m[l], d[l],
+        SAR_STEP(sar_gat_fwd_fused(g, k, bounds, feat[l], el[l], er[l], H, F, io->t, io->slope, m[l], d[l],
                                    feat[l + 1], ws, ws_bytes, st));
     }
     if (io->out_last) {
@@ -191,14 +178,8 @@ sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bound
     SAR_CUDA_STEP(cudaStreamWaitEvent(st, e_gout, 0));
     void *gin = ga, *gout = gb;
     for (int l = L - 1; l >= 0; --l) {
-        for (int q = 0; q < k; ++q) {
-            fq[q] = cut(feat[l], rb, q);
-            erq[q] = reinterpret_cast<const float *>(cut(er[l], (size_t)H * 4, q));
-            dfq[q] = const_cast<char *>(cut(gout, rb, q));
-            derq[q] = reinterpret_cast<float *>(const_cast<char *>(cut(der[l], (size_t)H * 4, q)));
-        }
-        SAR_STEP(sar_gat_bwd_fused(g, k, bounds, fq.data(), el[l], erq.data(), m[l], d[l], gin, H, F, io->t, io->slope,
-                                   dfq.data(), del[l], derq.data(), ws, ws_bytes, st));
+        SAR_STEP(sar_gat_bwd_fused(g, k, bounds, feat[l], el[l], er[l], m[l], d[l], gin, H, F, io->t, io->slope, gout,
+                                   del[l], der[l], ws, ws_bytes, st));
         SAR_CUDA_STEP(cudaEventRecord(e_bwd[l], st));
         SAR_CUDA_STEP(cudaStreamWaitEvent(down, e_bwd[l], 0));
         if (io->del) SAR_CUDA_STEP(cudaMemcpyAsync(io->del[l], del[l], nh_b, cudaMemcpyDeviceToHost, down));

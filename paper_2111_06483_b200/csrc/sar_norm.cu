@@ -347,6 +347,40 @@ static sar_status norm_set_act(NormArgs &a, uint32_t flags, float p, uint64_t se
 
 extern "C" {
 
+sar_status sar_bn_combine_moments(int32_t R, int32_t C, const int64_t *n_r, const float *mean_r, const float *m2_r,
+                                  int64_t *n_all, float *mean, float *m2) {
+    if (R < 1 || C < 0 || !n_r || !n_all || (C > 0 && (!mean_r || !m2_r || !mean || !m2))) return SAR_ERR_INVALID_ARG;
+    long long N = 0;
+    for (int r = 0; r < R; ++r) {
+        if (n_r[r] < 0) return SAR_ERR_INVALID_ARG;
+        N += n_r[r];
+    }
+    *n_all = N;
+    for (int c = 0; c < C; ++c) {
+        double mu = 0.0;
+        for (int r = 0; r < R; ++r) mu += (double)n_r[r] * (double)mean_r[(size_t)r * C + c];
+        mu = N > 0 ? mu / (double)N : 0.0;
+        double q = 0.0;
+        for (int r = 0; r < R; ++r) {
+            const double dm = (double)mean_r[(size_t)r * C + c] - mu;
+            q += (double)m2_r[(size_t)r * C + c] + (double)n_r[r] * dm * dm;
+        }
+        mean[c] = (float)mu;
+        m2[c] = (float)q;
+    }
+    return SAR_OK;
+}
+
+sar_status sar_bn_combine_sums(int32_t R, int64_t count, const float *sums_r, float *sums) {
+    if (R < 1 || count < 0 || (count > 0 && (!sums_r || !sums))) return SAR_ERR_INVALID_ARG;
+    for (int64_t c = 0; c < count; ++c) {
+        double acc = 0.0;
+        for (int r = 0; r < R; ++r) acc += (double)sums_r[(size_t)r * count + c];   // rank order: the same on every worker
+        sums[c] = (float)acc;
+    }
+    return SAR_OK;
+}
+
 size_t sar_bn_workspace_bytes(int32_t C) {
     if (C < 1) return 0;
     return (size_t)kNormBlocks * 2 * C * 4 + 256;

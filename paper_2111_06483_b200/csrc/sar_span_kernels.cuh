@@ -268,6 +268,10 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
     // ---- per-row accumulators (persist across the chunks of a row longer than CAP) --------------
     constexpr int NP = EPV / 2;
     f32x2 pacc0[V][NP], pacc1[V][NP];  // packed float32 pairs
+    // Sum modes: the terms are added eight slots at a time into `pin` and `pin` into the row's accumulator, so that
+    // the longest chain of float32 additions behind one output is 8 + slots/8 instead of the row's edge count.
+    constexpr bool kTwoLevel = MODE == kSum || MODE == kSumW;
+    f32x2 pin[V][NP];
     float sv[V], mrun[V];
     // Row-stationary vector of the backward passes (gout of the row / feat of the source), needed only when the
     // row is finalised.  It is kept as loaded (packed) and requested one row ahead, so that nothing waits for it.
@@ -277,7 +281,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
         sv[v] = 0.f;
         mrun[v] = SAR_NEG_INF;
 #pragma unroll
-        for (int k = 0; k < NP; ++k) pacc0[v][k] = pacc1[v][k] = zero2();
+        for (int k = 0; k < NP; ++k) pacc0[v][k] = pacc1[v][k] = pin[v][k] = zero2();
         rvq[v] = rvq_next[v] = make_uint4(0u, 0u, 0u, 0u);
     }
     auto request_rowvec = [&](long long row_, uint4 (&dst)[V]) {
@@ -710,8 +714,13 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                     if constexpr (MODE == kSum) {
                         const f32x2 one = pack2(1.f, 1.f);
 #pragma unroll
-                        for (int k = 0; k < NP; ++k) pacc0[v][k] = fma2(x[k], one, pacc0[v][k]);
-                    } else if constexpr (kFwdMode || MODE == kSumW) {
+                        for (int k = 0; k < NP; ++k) pin[v][k] = fma2(x[k], one, pin[v][k]);
+                    } else if constexpr (MODE == kSumW) {
+                        const float w = lds_f32(w_s[v] + woff);
+                        const f32x2 w2 = pack2(w, w);
+#pragma unroll
+                        for (int k = 0; k < NP; ++k) pin[v][k] = fma2(w2, x[k], pin[v][k]);
+                    } else if constexpr (kFwdMode) {
                         const float w = lds_f32(w_s[v] + woff);
                         sv[v] += w;
                         const f32x2 w2 = pack2(w, w);
@@ -742,6 +751,18 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                     }
                 }
                 issue(s + S, src_s);  // refill the stage just consumed
+                if constexpr (kTwoLevel) {
+                    if ((s & 7) == 7 || s + 1 == s_end) {   // every eight slots and at the end of the row's slots
+                        const f32x2 one = pack2(1.f, 1.f);
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+#pragma unroll
+                            for (int k = 0; k < NP; ++k) {
+                                pacc0[v][k] = fma2(pin[v][k], one, pacc0[v][k]);
+                                pin[v][k] = zero2();
+                            }
+                    }
+                }
             }
             if (!row_ends) continue;
 

@@ -36,11 +36,14 @@ def _rows_subgraph(indptr, indices, rows):
     return sub_indptr, indices[pos].long()
 
 
-def _tol(dtype, want, grad=False):
+def _tol(dtype, want, grad=False, stored=True):
+    """The tolerances of test_gpu_parity.py: float32 outputs 1e-5 / 1e-6, float32 gradients 1e-4 with a floor of
+    1e-5 x max(RMS, 1); arrays stored in bf16 (out, dfeat) 2^-7 relative plus 2^-9 of the RMS; del and der are
+    float32 arrays in every variant."""
     x = np.asarray(want, dtype=np.float64)
     scale = max(float(np.sqrt(np.mean(x * x))) if x.size else 0.0, 1.0)
-    if dtype == "bf16":
-        return dict(rtol=2e-2, atol=2e-2 * scale)
+    if dtype == "bf16" and stored:
+        return dict(rtol=2.0 ** -7, atol=2.0 ** -9 * scale)
     return dict(rtol=1e-4, atol=1e-5 * scale) if grad else dict(rtol=1e-5, atol=1e-6)
 
 
@@ -142,12 +145,12 @@ def test_sampled_rows_at_full_size(name, dtype):
         allclose_report(out[rows].float().cpu().numpy(), fwd1.out, what=f"out[{mode}]", **_tol(dtype, fwd1.out))
         allclose_report(m[rows].cpu().numpy(), fwd1.m, 1e-6, 1e-6, f"m[{mode}]")
         allclose_report(d[rows].cpu().numpy(), fwd1.d, 1e-5, 1e-6, f"d[{mode}]")
-        allclose_report(del_[rows].cpu().numpy(), bwd1.del_, what=f"del[{mode}]", **_tol(dtype, bwd1.del_, grad=True))
+        allclose_report(del_[rows].cpu().numpy(), bwd1.del_, what=f"del[{mode}]", **_tol(dtype, bwd1.del_, grad=True, stored=False))
         # ---- sampled sources: dfeat, der -------------------------------------------------------------
         allclose_report(dfeat[srcs_ok].float().cpu().numpy(), bwd2.dfeat[where_np], what=f"dfeat[{mode}]",
                         **_tol(dtype, bwd2.dfeat[where_np], grad=True))
         allclose_report(der[srcs_ok].cpu().numpy(), bwd2.der[where_np], what=f"der[{mode}]",
-                        **_tol(dtype, bwd2.der[where_np], grad=True))
+                        **_tol(dtype, bwd2.der[where_np], grad=True, stored=False))
         assert (dfeat[no_out] == 0).all() and (der[no_out] == 0).all()
         del out, d, dfeat, del_, der
         torch.cuda.empty_cache()

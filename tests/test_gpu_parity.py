@@ -5,8 +5,10 @@ Tolerances (|got - want| <= atol + rtol*|want|, want = float64 oracle on the sam
   float32 outputs        rtol 1e-5, atol 1e-6
   float32 gradients      rtol 1e-4, atol 1e-5 * scale   (scale = max(RMS of the oracle's array, 1):
                          the sums cancel, so a floor proportional to the operand scale, which is
-                         O(1) for N(0,1) inputs, is needed)
-  bf16 storage variants  rtol 2e-2, atol 2e-2 * scale   (outputs are rounded to bf16 once)
+                         O(1) for N(0,1) inputs, is needed); del and der of the bf16 variants too
+  bf16 stored arrays     rtol 2^-7, atol 2^-9 * scale   (out, dfeat: rounded to bf16 once, 2^-9 relative;
+                         inside the benchmark spec's 2e-2 for the bf16 variants)
+Every check records the largest error it saw and the share of its tolerance that it used (pytest -rA).
 Integer outputs (CSR, CSC, partition split, plans) are compared bit for bit.
 """
 import numpy as np
@@ -32,18 +34,24 @@ def rms(x):
 
 
 def check_out(got, want, dtype, what):
+    """A stored output.  bf16 storage rounds once: half a bf16 ulp, 2^-9 relative; the check allows 2^-7
+    (the benchmark spec's bound for the bf16 variants is 2e-2) plus 2^-9 of the array's RMS for entries near zero."""
     got = got.float().cpu().numpy()
     if dtype == "bf16":
-        allclose_report(got, want, 2e-2, 2e-2 * rms(want), what)
+        allclose_report(got, want, 2.0 ** -7, 2.0 ** -9 * rms(want), what)
     else:
         allclose_report(got, want, 1e-5, 1e-6, what)
 
 
-def check_grad(got, want, dtype, what, floor=1.0):
+def check_grad(got, want, dtype, what, floor=1.0, stored=False):
+    """A gradient.  The sums cancel, so float32 rounding leaves about 2^-24 of the TERMS whatever the result:
+    a floor of 1e-5 x max(RMS, 1) besides the benchmark spec's 1e-4 relative.  del and der are float32 arrays computed
+    in float32 from inputs the oracle shares exactly, so they take this tolerance in the bf16 variants too;
+    dfeat is stored in the storage type (stored=True) and takes the rounding of a stored bf16 output on top."""
     got = got.float().cpu().numpy()
     scale = max(rms(want), floor)    # inputs are N(0,1): sums of O(1) terms that cancel
-    if dtype == "bf16":
-        allclose_report(got, want, 2e-2, 2e-2 * scale, what)
+    if dtype == "bf16" and stored:
+        allclose_report(got, want, 2.0 ** -7, 2.0 ** -9 * scale, what)
     else:
         allclose_report(got, want, 1e-4, 1e-5 * scale, what)
 
@@ -192,7 +200,7 @@ def _full_check(p, dtype="f32", modes=("fused",), slope=0.2, grad_floor=1.0):
         allclose_report(m.cpu().numpy(), f.m, 1e-6, 1e-6, f"m[{mode}]")
         allclose_report(d.cpu().numpy(), f.d, 1e-5, 1e-6, f"d[{mode}]")
         dfeat, del_, der = p.gpu_bwd(m, d, out=out, mode=mode, slope=slope, acc=fw[3] if keep else None)
-        check_grad(dfeat, b.dfeat, dtype, f"dfeat[{mode}]")
+        check_grad(dfeat, b.dfeat, dtype, f"dfeat[{mode}]", stored=True)
         check_grad(del_, b.del_, dtype, f"del[{mode}]", grad_floor)
         check_grad(der, b.der, dtype, f"der[{mode}]", grad_floor)
         results[mode] = (out, m, d, dfeat, del_, der)
@@ -335,11 +343,13 @@ def test_spmm_sum_forward_backward_mean_and_partitions(F, dtype, threshold):
     t_indptr, t_indices = oracle.csr_transpose(n, n, indptr, indices)
     want = oracle.spmm(indptr, indices, feat.float().numpy())
     got = api.spmm_sum(g.whole, feat.to(DEV))
-    # plain sums of N(0,1) rows cancel: sequential float32 accumulation of deg unit-scale terms
-    # leaves up to ~2^-24 * deg * |x| (typically eps*sqrt(deg)*|partial sum|), so the floor follows
-    # the longest row: 2^-23 * max degree
+    # Plain sums of N(0,1) rows cancel, so a relative bound alone is not enough.  The kernel adds a lane's terms
+    # eight slots at a time and then the groups of eight (and a long row's segments) one after the other: the longest
+    # chain of float32 additions behind an output is about 8 + deg/8, each leaving up to 2^-24 of a partial sum of
+    # O(sqrt(deg)) unit-scale terms.  Floor: 2^-23 * (8 + max degree / 8).
     max_deg = int(max(np.diff(indptr).max(), np.diff(t_indptr).max()))
-    tol = dict(rtol=2e-2, atol=2e-2 * rms(want)) if dtype == "bf16" else dict(rtol=1e-5, atol=2.0 ** -23 * max_deg)
+    tol = (dict(rtol=2.0 ** -7, atol=2.0 ** -9 * max(rms(want), 1.0)) if dtype == "bf16"
+           else dict(rtol=1e-5, atol=2.0 ** -23 * (8 + max_deg / 8)))
     allclose_report(got.float().cpu().numpy(), want, what="spmm", **tol)
     # backward = the same call on the transposed partition
     want_b = oracle.spmm(t_indptr, t_indices, gout.float().numpy())
@@ -357,8 +367,8 @@ def test_spmm_sum_forward_backward_mean_and_partitions(F, dtype, threshold):
         flags = (B.SAR_FIRST if q == 0 else 0) | (B.SAR_LAST if q == 3 else 0)
         ws = torch.empty(B.sar_spmm_workspace_bytes(part, F, B._dtype(fd)), dtype=torch.uint8, device=DEV)
         B.sar_spmm_agg(part, fd[g.bounds[q]:g.bounds[q + 1]], F, flags, None, out, ws)
-    # bf16 `out` is re-rounded after every partition: up to one bf16 ulp of the running sum per step
-    tol_k = dict(rtol=4e-2, atol=4 * 2.0 ** -8 * float(np.abs(want).max())) if dtype == "bf16" else tol
+    # bf16 `out` is re-rounded after every partition: up to half a bf16 ulp of the running sum per step (K = 4)
+    tol_k = dict(rtol=4 * 2.0 ** -8, atol=4 * 2.0 ** -9 * float(np.abs(want).max())) if dtype == "bf16" else tol
     allclose_report(out.float().cpu().numpy(), want, what="spmm K=4", **tol_k)
 
 
@@ -381,10 +391,9 @@ def test_argument_errors_return_status_codes():
     with pytest.raises(B.SarError) as ei:       # backward without workspace
         B.sar_gat_bwd(p.graph.whole, d["feat"], d["el"], d["er"], m, dd, d["gout"], 2, 8, 0.2, 3, out, m, dd, None)
     assert ei.value.code == -4
-    with pytest.raises(B.SarError) as ei:       # partition buffers that are not one array
-        B.sar_gat_fwd_fused(p.graph.whole, [0, 50, 100], [d["feat"], d["feat"]], d["el"], [d["er"], d["er"]], 2, 8, 0.2,
-                            m, dd, out, None)
-    assert ei.value.code == -2
+    with pytest.raises(B.SarError) as ei:       # partition bounds that do not cover the sources
+        B.sar_gat_fwd_fused(p.graph.whole, [0, 50, 99], d["feat"], d["el"], d["er"], 2, 8, 0.2, m, dd, out, None)
+    assert ei.value.code == -1
     fwd_only = B.Part(p.n, p.n, p.graph.whole.indptr, p.graph.whole.indices)
     ws = api.gat_workspace(p.graph.whole, 2, 8, torch.float32)
     with pytest.raises(B.SarError) as ei:       # backward needs the CSC

@@ -70,7 +70,7 @@ def test_two_calls_in_a_row_match_the_ordinary_entry_point():
         _close(got, want, dtype)
         for a, b, name in zip(got, want, ("dfeat", "del", "der")):
             assert torch.equal(a, b), f"{name}: same kernels, same order, yet not bit-identical"
-    # the first problem against the oracle as well (bf16 storage: rtol 2e-2, floor 2e-2 x RMS)
+    # the first problem against the oracle as well, with the parity tests' tolerances
     g, t, H, F, (src, dst, host) = first
     _, got = _both_ways(g, t, H, F)
     h = {k: v.float().numpy() for k, v in host.items()}
@@ -78,8 +78,11 @@ def test_two_calls_in_a_row_match_the_ordinary_entry_point():
     f = oracle.gat_fwd(indptr, indices, h["feat"], h["el"], h["er"], 0.2)
     b = oracle.gat_bwd(indptr, indices, h["feat"], h["el"], h["er"], f.alpha, h["gout"], 0.2)
     for a, w, name in zip(got, (b.dfeat, b.del_, b.der), ("dfeat", "del", "der")):
-        floor = 2e-2 * max(float(np.sqrt(np.mean(w * w))), 1.0)
-        allclose_report(a.float().cpu().numpy(), w, 2e-2, floor, f"noalloc {name} vs oracle")
+        scale = max(float(np.sqrt(np.mean(w * w))), 1.0)
+        if name == "dfeat":   # stored in bf16: one rounding
+            allclose_report(a.float().cpu().numpy(), w, 2.0 ** -7, 2.0 ** -9 * scale, f"noalloc {name} vs oracle")
+        else:                 # float32 arrays
+            allclose_report(a.float().cpu().numpy(), w, 1e-4, 1e-5 * scale, f"noalloc {name} vs oracle")
 
 
 def test_problems_beyond_the_fixed_scratch_are_refused():
