@@ -134,12 +134,16 @@ def state_bytes_sequential(n, H, F, K, L):
 
 KERNEL_BYTES = {"gat_fwd": bytes_fwd, "gat_bwd_dst": bytes_bwd_dst, "gat_bwd_src": bytes_bwd_src}
 
-# DRAM traffic of one pass (rows + segments + merge launches), dram__bytes_read.sum + dram__bytes_write.sum.
-# Measured with ncu on the workload scaled to 10 % (feature arrays of 512 MB, a few GB on the device, one
-# launch of each kernel) and scaled to a full launch by the edge count; see profiles/.  None: not captured
-# for the kernels of this tree.
+# DRAM traffic of one pass (rows + segments + merge launches), dram__bytes_read.sum + dram__bytes_write.sum from one-pass
+# ncu captures of the kernels of this tree at full size, nine forward and six backward launches at a time (commands and
+# per-launch figures: profiles/gat_kernels_large_launch_list_and_dram.md).  A constant of that capture, not of this run.
+NCU_TRAFFIC_SOURCE = ("ncu one-pass capture of these kernels at full size (profiles/gat_kernels_large_launch_list_and_dram.md), "
+                      "not measured in this run")
 NCU_TRAFFIC = {
-    # (workload, storage dtype, pass): (bytes per full-size pass, source)
+    # (workload, storage dtype, pass): bytes per full-size pass
+    ("large", "bf16", "gat_fwd"): 82.16e9,
+    ("large", "bf16", "gat_bwd_dst"): 84.33e9,
+    ("large", "bf16", "gat_bwd_src"): 89.16e9,
 }
 
 
@@ -785,10 +789,12 @@ def run_ours(args, rank, world, local_rank):
         dom = max(passes, key=lambda k_: passes[k_]["ms"])
         alg = passes[dom]["algorithmic_bytes"]
         achieved = alg / (passes[dom]["ms"] * 1e-3) / 1e9
-        traffic = NCU_TRAFFIC.get((args.workload, dtype, dom)) if (args.scale == 1.0 and main_sched == "fused") else None
+        default_plan = args.threshold is None and args.t_threshold is None and args.ids == "permuted"
+        traffic = (NCU_TRAFFIC.get((args.workload, dtype, dom))
+                   if (args.scale == 1.0 and main_sched == "fused" and default_plan) else None)
         roofline = {"bound": "hbm", "kernel": dom, "launches": passes[dom]["launches"], "achieved": achieved,
                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
-                    "traffic": traffic[0] if traffic else None, "traffic_source": traffic[1] if traffic else None,
+                    "traffic": traffic, "traffic_source": NCU_TRAFFIC_SOURCE if traffic else None,
                     "algorithmic_bytes_per_launch": alg, "avg_launch_ms": passes[dom]["ms"],
                     "target_frac": TARGET_FRAC, "target_met": bool(achieved / peak >= TARGET_FRAC)}
     step_bytes = L * bytes_layer_fwd_bwd(n, e, H, F, b)

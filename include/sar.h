@@ -298,7 +298,9 @@ SAR_API sar_status sar_gat_bwd_storing(const sar_part *g, const void *feat, cons
 /* ---------------------------------------------------------------------------------------------
  * Sum aggregation (Eq. 2; Sec. 3.2 "case 1").  out[i,:] (+)= sum over this partition's in-edges of
  * feat_q[j,:]; feat_q [n_src,F], out [n_dst,F], both of type t, float32 accumulation within the
- * call.  SAR_FIRST overwrites out, otherwise the partition's sum is added to it.  SAR_MEAN with
+ * call.  SAR_FIRST overwrites out, otherwise the partition's sum is added to it.  Between
+ * calls the running sum lives in `out` itself, i.e. in the storage type: with bf16 storage a sum over K partitions is
+ * rounded K times (half a bf16 ulp of the running sum each), a sum over one partition once.  SAR_MEAN with
  * SAR_LAST divides the result by deg_total[i] (int64 [n_dst] total in-degree over all partitions;
  * rows with degree 0 stay 0).  The backward pass of the sum is this same call on the transposed
  * partition applied to gout. */

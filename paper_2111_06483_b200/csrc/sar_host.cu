@@ -27,6 +27,9 @@ struct Copies {
     cudaEvent_t half_done[2] = {nullptr, nullptr};
     bool half_used[2] = {false, false};
     unsigned long long calls = 0;
+    // held for the whole of a call: the pipelined state above is read at its start and advanced at its end, so two
+    // host threads that call on the same device take turns
+    std::mutex call_mutex;
 };
 constexpr int kMaxDevices = 64;
 Copies g_copies[kMaxDevices];
@@ -81,6 +84,7 @@ sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bound
 
     Copies *cp = nullptr;
     SAR_TRY(copies_for_current_device(&cp));
+    std::lock_guard<std::mutex> call_lock(cp->call_mutex);
     const int half = pipelined ? (int)(cp->calls & 1ull) : 0;
     Arena a{static_cast<char *>(arena) + (size_t)half * one, 0, one};
     std::vector<void *> feat(L + 1);
@@ -139,7 +143,6 @@ sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bound
             SAR_CUDA_STEP(cudaStreamWaitEvent(up, cp->half_done[half], 0));
             SAR_CUDA_STEP(cudaStreamWaitEvent(st, cp->half_done[half], 0));
         }
-        ++cp->calls;
     } else {
         // a plain call after pipelined ones: let those finish first (they may be using this part of the arena)
         for (int i = 0; i < 2; ++i)
@@ -191,8 +194,11 @@ sar_status sar_gat_stack_host(const sar_part *g, int32_t k, const int64_t *bound
     // gin now holds dfeat of layer 0 (the last backward call has been waited for by `down` above)
     if (io->dfeat0) SAR_CUDA_STEP(cudaMemcpyAsync(io->dfeat0, gin, row_b, cudaMemcpyDeviceToHost, down));
     if (pipelined) {
+        // the half changes hands only once its completion event is in place: a call that failed earlier leaves the
+        // parity where it was, and the next call takes the same half again
         SAR_CUDA_STEP(cudaEventRecord(cp->half_done[half], down));
         cp->half_used[half] = true;
+        ++cp->calls;
     } else {
         SAR_CUDA_STEP(cudaEventRecord(e_done, down));
         SAR_CUDA_STEP(cudaStreamWaitEvent(st, e_done, 0));
