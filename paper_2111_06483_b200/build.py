@@ -18,7 +18,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(CSRC, "build")
 LIB = os.path.join(PKG, "libsar.so")
-SOURCES = ["sar_gat.cu", "sar_lean_fwd_f32.cu", "sar_lean_fwd_bf16.cu", "sar_lean_bwd_dst_f32.cu", "sar_lean_bwd_dst_bf16.cu",
+SOURCES = ["sar_gat.cu", "sar_lean_fwd_f32.cu", "sar_lean_fwd_bf16.cu", "sar_lean_bwd_dst_f32.cu", "sar_lean_bwd_dst_bf16.cu", "sar_lean_bwd_src_f32.cu", "sar_lean_bwd_src_bf16.cu",
            "sar_graph.cu", "sar_host.cu", "sar_noalloc.cu", "sar_storing.cu",
            "sar_glue.cu", "sar_norm.cu", "sar_linear.cu", "sar_rgcn.cu"]
 NVCC_FLAGS = [

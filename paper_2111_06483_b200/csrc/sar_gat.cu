@@ -521,7 +521,23 @@ sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, c
     s1.hvec = (H % 4 == 0);
 
     const bool lean_dst = whole && lean_applies(s, flags, slope, g->split, g->n_src) && sar_aligned(er_q, 16);
+    const bool lean_src = whole && lean_applies(s, flags, slope, g->t_split, g->n_dst);
     LeanArgs ld{};
+    LeanSrcArgs ls{};
+    if (lean_src) {
+        ls.n_rows = g->n_src;
+        ls.indptr = g->t_indptr;
+        ls.indices = g->t_indices;
+        ls.gather = gout;
+        ls.rowvec = feat_q;
+        ls.er = er_q;
+        ls.rec_in = rec;
+        ls.out = dfeat_q;
+        ls.der = der_q;
+        ls.slope = slope;
+        ls.sp = sa.sp;
+        ls.sp.threshold = g->t_split->threshold;
+    }
     if (lean_dst) {
         ld.n_rows = g->n_dst;
         ld.indptr = g->indptr;
@@ -567,7 +583,10 @@ sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, c
             }
         }
         if (g->n_src > 0) {
-            SAR_TRY((launch_span<T, C::g, C::v, U, kBwdSrc, kCapSrc, kMinBlocksBwd>(s1, g->nnz, "gat_bwd_src", "gat_bwd_src_seg", st)));
+            if (lean_src)
+                SAR_TRY(s.t == SAR_F32 ? lean_bwd_src_f32(s, ls, g->nnz, st) : lean_bwd_src_bf16(s, ls, g->nnz, st));
+            else
+                SAR_TRY((launch_span<T, C::g, C::v, U, kBwdSrc, kCapSrc, kMinBlocksBwd>(s1, g->nnz, "gat_bwd_src", "gat_bwd_src_seg", st)));
             if (sa.sp.threshold > 0) {
                 auto merge = gat_bwd_src_merge_kernel<T, C::g, C::v>;
                 SAR_TRY(ensure_smem(merge, msmem));

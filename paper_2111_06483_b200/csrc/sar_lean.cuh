@@ -1,6 +1,6 @@
 // Host-side interface of the lean span kernels (internal): arguments, applicability test and the launchers,
 // which are compiled in translation units of their own (sar_lean_*.cu), one per pass and storage type.
-// They cover the forward pass and the destination-major backward pass.
+// They cover the forward pass and both backward passes of a call that holds the whole graph.
 #pragma once
 
 #include "sar_rowkernels.cuh"
@@ -22,6 +22,21 @@ struct LeanArgs {
     float slope;
     SplitArgs sp;
     int R;                   // rows per span (<= kMaxSpanRows)
+};
+
+struct LeanSrcArgs {
+    long long n_rows;        // sources
+    const int64_t *indptr;   // CSC
+    const int32_t *indices;  // destinations
+    const void *gather;      // gout
+    const void *rowvec;      // feat
+    const float *er;         // [n_rows,H]
+    const float4 *rec_in;    // [n_dst,H] {el, m, 1/d, D}
+    void *out;               // dfeat
+    float *der;
+    float slope;
+    SplitArgs sp;
+    int R;
 };
 
 constexpr int kLeanCap = 256;   // edges a chunk stages; rows and segments must not exceed it
@@ -47,5 +62,7 @@ sar_status lean_fwd_f32(const Shape &s, const LeanArgs &a, long long nnz, cudaSt
 sar_status lean_fwd_bf16(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
 sar_status lean_bwd_dst_f32(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
 sar_status lean_bwd_dst_bf16(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
+sar_status lean_bwd_src_f32(const Shape &s, const LeanSrcArgs &a, long long nnz, cudaStream_t st);
+sar_status lean_bwd_src_bf16(const Shape &s, const LeanSrcArgs &a, long long nnz, cudaStream_t st);
 
 }  // namespace sar
