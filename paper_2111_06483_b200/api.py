@@ -13,7 +13,7 @@ import torch
 from . import binding as B
 
 DEFAULT_THRESHOLD = 256    # rows of the CSR with more edges are cut into segments of this many edges
-DEFAULT_T_THRESHOLD = 384  # the same for the CSC (the source-major backward pass measured best with longer segments)
+DEFAULT_T_THRESHOLD = 256  # the same for the CSC (its own knob: the two plans are independent)
 
 
 def _workspace(nbytes: int, device) -> torch.Tensor:

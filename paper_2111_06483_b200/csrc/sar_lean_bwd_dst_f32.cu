@@ -1,4 +1,4 @@
-// Lean span kernels, bwd dst pass, float32 storage (see sar_lean_kernels.cuh).
-#include "sar_lean_kernels.cuh"
+// Lean span kernel of the destination-major backward pass, float32 storage (see sar_lean_dst_kernels.cuh).
+#include "sar_lean_dst_kernels.cuh"
 
-SAR_LEAN_TU(bwd_dst_f32, float, sar::kBwdDst, "gat_bwd_dst", "gat_bwd_dst_seg")
+SAR_LEAN_DST_TU(f32, float)

@@ -53,7 +53,7 @@ __global__ void __launch_bounds__(32, MINB) lean_src_kernel(const LeanSrcArgs a)
     constexpr int ITEMS = P * H;                   // (position, head) pairs of a stage
     static_assert(H % 4 == 0 && NVEC % H == 0 && VPH <= G && (VPH & (VPH - 1)) == 0, "head geometry");
     static_assert((1 << LGNVEC) == NVEC, "row geometry");
-    static_assert(P <= 32 && 32 % P == 0 && SPS == 4, "stage geometry: four slots per stage");
+    static_assert(P <= 32 && 32 % P == 0 && (SPS == 4 || SPS == 8), "stage geometry: four or eight slots per stage");
     static_assert(ITEMS <= 64, "at most two (position, head) pairs per lane");
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const unsigned sbase = (unsigned)__cvta_generic_to_shared(smem_raw);
@@ -234,16 +234,19 @@ __global__ void __launch_bounds__(32, MINB) lean_src_kernel(const LeanSrcArgs a)
         auto issue_stage = [&](int j) {
             const unsigned dst = ring_l + (unsigned)((j % NS) * STAGE);
             const unsigned ob = offs_s + (unsigned)((j * P + half * SPS) * 4);
-            const uint4 o4 = lds128(ob);
-            const unsigned ov[4] = {o4.x, o4.y, o4.z, o4.w};
 #pragma unroll
-            for (int t = 0; t < 4; ++t)
+            for (int kq = 0; kq < SPS; kq += 4) {
+                const uint4 o4 = lds128(ob + kq * 4);
+                const unsigned ov[4] = {o4.x, o4.y, o4.z, o4.w};
 #pragma unroll
-                for (int v = 0; v < V; ++v) {
-                    unsigned long long src;
-                    asm("mad.wide.u32 %0, %1, 16, %2;\n" : "=l"(src) : "r"(ov[t]), "l"(gbase_v[v]));
-                    cp_async16_full(dst + (unsigned)(t * EPW * ROWB + v * G * 16), reinterpret_cast<const void *>(src));
-                }
+                for (int t = 0; t < 4; ++t)
+#pragma unroll
+                    for (int v = 0; v < V; ++v) {
+                        unsigned long long src;
+                        asm("mad.wide.u32 %0, %1, 16, %2;\n" : "=l"(src) : "r"(ov[t]), "l"(gbase_v[v]));
+                        cp_async16_full(dst + (unsigned)((kq + t) * EPW * ROWB + v * G * 16), reinterpret_cast<const void *>(src));
+                    }
+            }
 #pragma unroll
             for (int n = 0; n < NIT; ++n) {
                 const int it = lane + 32 * n;
@@ -316,16 +319,18 @@ __global__ void __launch_bounds__(32, MINB) lean_src_kernel(const LeanSrcArgs a)
                 }
                 float4 w4[V], u4[V];
 #pragma unroll
-                for (int v = 0; v < V; ++v) {
-                    w4[v] = lds_f4(w_s + (unsigned)(((half * H + hv[v]) * SPS) * 4));
-                    u4[v] = lds_f4(w_s + L::WB + (unsigned)(((half * H + hv[v]) * SPS) * 4));
-                }
-#pragma unroll
                 for (int k = 0; k < SPS; ++k) {
+                    if (k % 4 == 0) {
+#pragma unroll
+                        for (int v = 0; v < V; ++v) {
+                            w4[v] = lds_f4(w_s + (unsigned)(((half * H + hv[v]) * SPS + k) * 4));
+                            u4[v] = lds_f4(w_s + L::WB + (unsigned)(((half * H + hv[v]) * SPS + k) * 4));
+                        }
+                    }
 #pragma unroll
                     for (int v = 0; v < V; ++v) {
-                        const float wk = k == 0 ? w4[v].x : k == 1 ? w4[v].y : k == 2 ? w4[v].z : w4[v].w;
-                        const float uk = k == 0 ? u4[v].x : k == 1 ? u4[v].y : k == 2 ? u4[v].z : u4[v].w;
+                        const float wk = k % 4 == 0 ? w4[v].x : k % 4 == 1 ? w4[v].y : k % 4 == 2 ? w4[v].z : w4[v].w;
+                        const float uk = k % 4 == 0 ? u4[v].x : k % 4 == 1 ? u4[v].y : k % 4 == 2 ? u4[v].z : u4[v].w;
                         f32x2 x[NP];
                         Pairs<T>::get(lds128(ring_a + (unsigned)(k * EPW * ROWB + v * G * 16)), x);
                         const float al = fabsf(wk);
@@ -453,7 +458,7 @@ __global__ void __launch_bounds__(32, MINB) lean_src_kernel(const LeanSrcArgs a)
 template <typename T, int G, int V, int H>
 static sar_status launch_lean_src(LeanSrcArgs a, long long nnz, cudaStream_t st) {
     constexpr int NS = 2;
-    constexpr int P = 4 * (32 / G);            // four slots per stage
+    constexpr int P = (G == 32 && V == 1) ? 8 : 4 * (32 / G);   // stages of 2 KB (4 KB for rows of 512 bytes and more)
     using LR = LeanSrcLayout<G, V, H, false, kLeanCap, P, NS>;
     using LS = LeanSrcLayout<G, V, H, true, kLeanCap, P, NS>;
     a.R = lean_rows_per_span(a.n_rows, nnz, kLeanCap);
