@@ -5,7 +5,7 @@
 // Same plan as lean_src_kernel (sar_lean_src_kernels.cuh): stage-granular cp.async ring of the gathered feature rows,
 // the score terms er[col, :] of a stage's positions travelling with the stage (16 bytes per position and head group
 // into a small ring), the weights of a stage computed just before it is consumed, one (position, head) pair per lane.
-// Preconditions as for lean_kernel (checked by the host).
+// Preconditions as for lean_src_kernel, on the CSR (checked by the host).
 #pragma once
 
 #include "sar_lean_src_kernels.cuh"

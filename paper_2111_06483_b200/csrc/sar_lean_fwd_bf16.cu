@@ -1,4 +1,4 @@
-// Lean span kernels, fwd pass, bf16 storage (see sar_lean_kernels.cuh).
-#include "sar_lean_kernels.cuh"
+// Lean span kernel of the forward pass, bf16 storage (see sar_lean_fwd_kernels.cuh).
+#include "sar_lean_fwd_kernels.cuh"
 
-SAR_LEAN_TU(fwd_bf16, __nv_bfloat16, sar::kFwd, "gat_fwd", "gat_fwd_seg")
+SAR_LEAN_FWD_TU(bf16, __nv_bfloat16)

@@ -1,4 +1,4 @@
-// Lean span kernels, fwd pass, float32 storage (see sar_lean_kernels.cuh).
-#include "sar_lean_kernels.cuh"
+// Lean span kernel of the forward pass, float32 storage (see sar_lean_fwd_kernels.cuh).
+#include "sar_lean_fwd_kernels.cuh"
 
-SAR_LEAN_TU(fwd_f32, float, sar::kFwd, "gat_fwd", "gat_fwd_seg")
+SAR_LEAN_FWD_TU(f32, float)

@@ -2,18 +2,18 @@
 // der_j = <feat_j, sum_i alpha g' gout_i> - sum_i alpha g' D_i over the CSC, alpha rebuilt from the destination
 // records {el, m, 1/d, D} the destination-major pass left in the workspace.
 //
-// It shares the plan of lean_kernel (sar_lean_kernels.cuh: span of rows -> chunk -> stage-granular cp.async ring of
-// the gathered gout rows, uniform control flow, padding by repetition) but computes the weights of a stage JUST
-// BEFORE the stage is consumed: the 64-byte destination record of every position of a stage travels with the stage's
-// rows (one 16-byte cp.async per lane and stage into a small record ring), and when the stage has landed each lane
-// scores one (position, head) pair into a 256-byte weight block.  Nothing per chunk is staged except the row offsets,
-// so a warp needs 7.5 KB of shared memory instead of 13.5 KB, no record is ever loaded into a register ahead of its
-// use, and no lane waits for a gather inside a sweep.
-// Preconditions as for lean_kernel (checked by the host): SAR_FIRST|SAR_LAST, slope of any sign, a long-row plan of
-// the CSC with threshold <= CAP, fewer than 2^32 16-byte vectors in gout.
+// The plan is the one sar_lean_common.cuh describes (span of rows -> chunk -> stage-granular cp.async ring of the
+// gathered gout rows, uniform control flow, padding by repetition, weights of a stage computed JUST BEFORE the stage
+// is consumed): the 64-byte destination record of every position of a stage travels with the stage's rows (one
+// 16-byte cp.async per lane and stage into a small record ring), and when the stage has landed each lane scores one
+// (position, head) pair into a 256-byte weight block.  Nothing per chunk is staged except the row offsets, so a warp
+// needs 7.5 KB of shared memory, no record is ever loaded into a register ahead of its use, and no lane waits for a
+// gather inside a sweep.
+// Preconditions (checked by the host): SAR_FIRST|SAR_LAST, slope >= 0, a long-row plan of the CSC with threshold <= CAP,
+// fewer than 2^32 16-byte vectors in gout.
 #pragma once
 
-#include "sar_lean_kernels.cuh"
+#include "sar_lean_common.cuh"
 
 namespace sar {
 
