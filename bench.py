@@ -137,13 +137,15 @@ KERNEL_BYTES = {"gat_fwd": bytes_fwd, "gat_bwd_dst": bytes_bwd_dst, "gat_bwd_src
 # DRAM traffic of one pass (rows + segments + merge launches), dram__bytes_read.sum + dram__bytes_write.sum from one-pass
 # ncu captures of the kernels of this tree at full size, nine forward and six backward launches at a time (commands and
 # per-launch figures: profiles/gat_kernels_large_launch_list_and_dram.md).  A constant of that capture, not of this run.
+# `traffic_rate_frac` = that traffic / the pass's measured time / the peak: how close the pass runs to the copy
+# bandwidth for the bytes it really moves (the compulsory-byte fraction `frac` counts every row once).
 NCU_TRAFFIC_SOURCE = ("ncu one-pass capture of these kernels at full size (profiles/gat_kernels_large_launch_list_and_dram.md), "
                       "not measured in this run")
 NCU_TRAFFIC = {
     # (workload, storage dtype, pass): bytes per full-size pass
-    ("large", "bf16", "gat_fwd"): 82.16e9,
-    ("large", "bf16", "gat_bwd_dst"): 84.33e9,
-    ("large", "bf16", "gat_bwd_src"): 89.16e9,
+    ("large", "bf16", "gat_fwd"): 82.12e9,
+    ("large", "bf16", "gat_bwd_dst"): 84.30e9,
+    ("large", "bf16", "gat_bwd_src"): 89.40e9,
 }
 
 
@@ -795,6 +797,7 @@ def run_ours(args, rank, world, local_rank):
         roofline = {"bound": "hbm", "kernel": dom, "launches": passes[dom]["launches"], "achieved": achieved,
                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_source": peak_src,
                     "traffic": traffic, "traffic_source": NCU_TRAFFIC_SOURCE if traffic else None,
+                    "traffic_rate_frac": (traffic / (passes[dom]["ms"] * 1e-3) / 1e9 / peak) if traffic else None,
                     "algorithmic_bytes_per_launch": alg, "avg_launch_ms": passes[dom]["ms"],
                     "target_frac": TARGET_FRAC, "target_met": bool(achieved / peak >= TARGET_FRAC)}
     step_bytes = L * bytes_layer_fwd_bwd(n, e, H, F, b)

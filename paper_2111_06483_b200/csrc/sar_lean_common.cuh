@@ -61,6 +61,10 @@ __device__ __forceinline__ float4 lds_f4(unsigned addr) {
     asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
     return v;
 }
+// shared-memory max without a return value: nobody waits for it
+__device__ __forceinline__ void red_max_u32(unsigned addr, unsigned v) {
+    asm volatile("red.shared.max.u32 [%0], %1;\n" ::"r"(addr), "r"(v) : "memory");
+}
 // plain 16-byte asynchronous copy (every copy of the lean kernels is a whole, valid vector)
 __device__ __forceinline__ void cp_async16_full(unsigned smem_addr, const void *gsrc) {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"(smem_addr), "l"(gsrc) : "memory");
@@ -72,6 +76,10 @@ constexpr float kLog2e = 1.4426950408889634f;
 // One configuration: chunks of kLeanCap edges, ring of two stages of 2 KB (4 KB for rows of 512 bytes and more), measured
 // best on the large workload among stages of 2 / 4 KB, two to four stages, chunks of 128 / 192 / 256 edges.
 constexpr int kLeanMinBlocks = 8;
+// The rows launches of the two backward passes are compiled for 24 resident blocks per SM (72-78 registers instead of
+// 88, no spills): step of the large workload 153.1 -> 147.2 ms.  The same bound on the forward rows launch and on the
+// segment launches changes nothing (147.3 ms).
+constexpr int kLeanMinBlocksBwdRows = 24;
 
 static inline int lean_rows_per_span(long long n_rows, long long nnz, int cap) {
     const double avg = n_rows > 0 ? (double)nnz / (double)n_rows : 0.0;

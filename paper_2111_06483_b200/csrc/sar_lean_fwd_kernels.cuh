@@ -3,13 +3,16 @@
 //
 // Same plan as lean_dst_kernel (sar_lean_dst_kernels.cuh): stage-granular cp.async ring of the gathered feature rows,
 // the score terms er[col, :] of a stage's positions travelling with the stage, the weights of a stage computed just
-// before it is consumed, one (position, head) pair per lane.  The row max is not known before a row's last stage, so
-// the softmax runs online stage by stage (the running-max correction of Sec. 3.4 applied inside a row): a stage's
-// weights are taken against the max of the row's score terms seen so far, and when that max grows the accumulators
-// of the row that continues from the previous stage are scaled by exp(m_before - m_now) first.  Since
-// max_j LeakyReLU(el + er_j) = LeakyReLU(el + max_j er_j) for slope >= 0, the running max is kept over raw er: in a
-// register per lane for a segment (shuffles over the positions of a head), in shared memory per (row, head) for the
-// rows launch (one atomic max per pair).
+// before it is consumed, one (position, head) pair per lane.
+// Softmax shift: a row's weights are exp(e - c) with c the score of the row's FIRST edge (fetched while the chunk's
+// first stages are in flight), not the row max: the result does not depend on the shift, nothing has to be known about
+// later stages, no lane waits for a max, and a row's arithmetic does not depend on where the stage boundaries fall.
+// The exact max m (the statistic the backward pass rebuilds alpha from) is collected on the side over raw er - since
+// max_j LeakyReLU(el + er_j) = LeakyReLU(el + max_j er_j) for slope >= 0 - by fire-and-forget shared-memory
+// reductions (rows launch) or in a register per lane (segments), and d is brought to it at the end: d = d_c exp(c - m).
+// Should a score exceed its row's shift by more than kLeanMaxLead, the stage takes a slow path first: the shift of that
+// (row, head) moves up to the stage's max and the accumulators follow by exp(c_before - c_now) (the running-max
+// correction of Sec. 3.4 applied inside a row), so nothing can overflow.
 // Preconditions as for lean_dst_kernel (checked by the host).
 #pragma once
 
@@ -31,11 +34,10 @@ struct LeanFwdLayout {
     static constexpr int ring = 0;
     static constexpr int rec = ring + NS * STAGE;
     static constexpr int w = rec + NS * RECB;
-    static constexpr int scale = w + WB;                          // exp(m_before - m_now) per head of the continuing row
-    static constexpr int offs = scale + ((H * 4 + 15) / 16) * 16;
+    static constexpr int offs = w + WB;
     static constexpr int prow = offs + POSMAX * 4;
-    static constexpr int rc = prow + POSMAX;                      // el; key of the running max of er
-    static constexpr int sout = rc + 2 * RCN;                     // d
+    static constexpr int rc = prow + POSMAX;                      // el; key of the max of er; shift c; scratch of the slow path
+    static constexpr int sout = rc + 4 * RCN;                     // d against the shift
     static constexpr int srb = sout + RCN;
     static constexpr int sso = srb + ((MAXR + 1) * 4 + 15) / 16 * 16;
     static constexpr int endm = sso + ((MAXR + 1) * 4 + 15) / 16 * 16;
@@ -60,8 +62,9 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
     const unsigned sbase = (unsigned)__cvta_generic_to_shared(smem_raw);
     const unsigned ring_s = sbase + L::ring, rec_s = sbase + L::rec, w_s = sbase + L::w, offs_s = sbase + L::offs;
     const unsigned prow_s = sbase + L::prow, rc_s = sbase + L::rc, sout_s = sbase + L::sout, endm_s = sbase + L::endm;
-    const unsigned scale_s = sbase + L::scale;
+    const unsigned key_s = rc_s + L::RCN, cref_s = rc_s + 2 * L::RCN, ftab_s = rc_s + 3 * L::RCN;
     int *srb = reinterpret_cast<int *>(smem_raw + L::srb);
+    constexpr float kLeanMaxLead = 60.f;   // a score may exceed its row's shift by this much before the shift moves
     int *sso = reinterpret_cast<int *>(smem_raw + L::sso);
     unsigned *skey = reinterpret_cast<unsigned *>(smem_raw + L::rc + L::RCN);
 
@@ -219,11 +222,6 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
                     }
                 }
             }
-            for (int x = lane; x < nr * H; x += 32) {
-                sts_f32(rc_s + 4 * x, __ldg(a.el + (row0 + r) * H + x));
-                skey[x] = kKeyNegInf;
-                sts_f32(sout_s + 4 * x, 0.f);
-            }
         }
         __syncwarp();
 
@@ -257,6 +255,24 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
             cp_async_commit();
         }
 
+        // per (row, head): el, the shift c = score of the row's first edge, the key of the max (the loads fly with the
+        // first stages)
+        for (int x = lane; x < nr * H; x += 32) {
+            const int i = x / H;
+            const float el_ = __ldg(a.el + (row0 + r) * H + x);
+            float c_ = SAR_NEG_INF;
+            if ((nemask >> i) & 1u) {
+                const unsigned col = lds_u32(offs_s + 4 * (unsigned)perm(sso[i] * EPW)) >> LGNVEC;
+                float gr;
+                c_ = leaky(el_ + __ldg(a.er + (size_t)col * H + (x % H)), a.slope, gr);
+            }
+            sts_f32(rc_s + 4 * x, el_);
+            skey[x] = kKeyNegInf;
+            sts_f32(cref_s + 4 * x, c_);
+            sts_f32(sout_s + 4 * x, 0.f);
+        }
+        __syncwarp();
+
         // rows without edges: their vector outputs are zeros (the scalars leave with the others at the chunk's end)
         if constexpr (!SEG) {
             unsigned em = ~nemask & ((1u << nr) - 1u);
@@ -272,16 +288,15 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
         {
             int s = 0;
             int ri = SEG ? 0 : (__ffs(nemask) - 1);
-            bool open = false;                      // the row being accumulated began in an earlier stage (uniform)
             float mrun = SAR_NEG_INF;               // segment: max of er[., lane % H] over the stages so far
             float el_seg = 0.f;
             if constexpr (SEG) el_seg = lds_f32(rc_s + 4 * (unsigned)hl);
             for (int j = 0; j < nstages; ++j) {
                 cp_async_wait<NS - 1>();
                 __syncwarp();   // the score terms of this stage were copied by other lanes; the previous weights are consumed
-                // -- weights of this stage: one (position, head) pair per lane, against the running max --
-                float erv[NIT];
-                unsigned prv[NIT];
+                // -- weights of this stage: one (position, head) pair per lane, against the shift of the pair's row --
+                float erv[NIT], w0[NIT];
+                unsigned prv[NIT], rx[NIT];
 #pragma unroll
                 for (int n = 0; n < NIT; ++n) {
                     const int it = lane + 32 * n;
@@ -291,69 +306,73 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
                         prv[n] = lds_u8(prow_s + (unsigned)(j * P + it / H));
                         erv[n] = lds_f32(rec_s + (unsigned)((j % NS) * L::RECB + it * 4));
                     }
+                    rx[n] = (unsigned)((((SEG ? 0u : (prv[n] & 0x7fu)) * H) + hl) * 4);
                 }
+                // the exact max, on the side
                 if constexpr (SEG) {
                     float vmax = SAR_NEG_INF;
 #pragma unroll
                     for (int n = 0; n < NIT; ++n) vmax = fmaxf(vmax, (prv[n] & 0x80u) ? SAR_NEG_INF : erv[n]);
 #pragma unroll
                     for (int off = H; off < 32; off <<= 1) vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, off));
-                    const float mnew = fmaxf(mrun, vmax);
-                    float gr;
-                    const float mm = leaky(el_seg + mnew, a.slope, gr);
-                    if (open && lane < H) sts_f32(scale_s + 4 * lane, ex2_approx((leaky(el_seg + mrun, a.slope, gr) - mm) * kLog2e));
-                    mrun = mnew;
-                    const float nm = -mm * kLog2e;
-#pragma unroll
-                    for (int n = 0; n < NIT; ++n) {
-                        const int it = lane + 32 * n;
-                        if (ITEMS % 32 == 0 || it < ITEMS) {
-                            const int p = it / H;
-                            float w0 = ex2_approx(fmaf(leaky(el_seg + erv[n], a.slope, gr), kLog2e, nm));
-                            if (prv[n] & 0x80u) w0 = 0.f;
-                            sts_f32(w_s + (unsigned)((((p % EPW) * H + hl) * SPS + p / EPW) * 4), w0);
-                        }
-                    }
+                    mrun = fmaxf(mrun, vmax);
                 } else {
-                    unsigned oldk = kKeyNegInf;
-                    if (open && lane < H) oldk = skey[ri * H + lane];
-                    __syncwarp();
 #pragma unroll
                     for (int n = 0; n < NIT; ++n)
-                        if (!(prv[n] & 0x80u)) atomicMax(&skey[(prv[n] & 0x7fu) * H + hl], fkey(erv[n]));
-                    __syncwarp();
-                    float gr;
+                        if (!(prv[n] & 0x80u)) red_max_u32(key_s + rx[n], fkey(erv[n]));
+                }
+                for (;;) {
+                    bool over = false;
 #pragma unroll
                     for (int n = 0; n < NIT; ++n) {
-                        const int it = lane + 32 * n;
-                        if (ITEMS % 32 == 0 || it < ITEMS) {
-                            const int p = it / H;
-                            const unsigned rx = (unsigned)(((prv[n] & 0x7fu) * H + hl) * 4);
-                            const float el_ = lds_f32(rc_s + rx);
-                            const float mm = leaky(el_ + fkey_inv(skey[(prv[n] & 0x7fu) * H + hl]), a.slope, gr);
-                            float w0 = ex2_approx(fmaf(leaky(el_ + erv[n], a.slope, gr), kLog2e, -mm * kLog2e));
-                            if (prv[n] & 0x80u) w0 = 0.f;
-                            sts_f32(w_s + (unsigned)((((p % EPW) * H + hl) * SPS + p / EPW) * 4), w0);
+                        float gr;
+                        const float dx = leaky(lds_f32(rc_s + rx[n]) + erv[n], a.slope, gr) - lds_f32(cref_s + rx[n]);
+                        const bool pad = (prv[n] & 0x80u) != 0u;
+                        over = over || (!pad && dx > kLeanMaxLead);
+                        w0[n] = pad ? 0.f : ex2_approx(dx * kLog2e);
+                    }
+                    if (!__any_sync(0xffffffffu, over)) break;
+                    // slow path: the shift of every (row, head) some score of this stage leads by more than kLeanMaxLead
+                    // moves up to the stage's largest score of that pair; the accumulators of the row in progress follow
+                    for (int x = lane; x < L::MAXR * H; x += 32) sts_u32(ftab_s + 4 * x, fkey(lds_f32(cref_s + 4 * x)));
+                    __syncwarp();
+#pragma unroll
+                    for (int n = 0; n < NIT; ++n) {
+                        if (!(prv[n] & 0x80u)) {
+                            float gr;
+                            red_max_u32(ftab_s + rx[n], fkey(leaky(lds_f32(rc_s + rx[n]) + erv[n], a.slope, gr)));
                         }
                     }
-                    if (open && lane < H) {
-                        const float el_ = lds_f32(rc_s + (unsigned)((ri * H + lane) * 4));
-                        const float mb = leaky(el_ + fkey_inv(oldk), a.slope, gr);
-                        const float mn = leaky(el_ + fkey_inv(skey[ri * H + lane]), a.slope, gr);
-                        sts_f32(scale_s + 4 * lane, ex2_approx((mb - mn) * kLog2e));
+                    __syncwarp();
+                    for (int x = lane; x < L::MAXR * H; x += 32) {
+                        const float cn = fkey_inv(lds_u32(ftab_s + 4 * x)), co = lds_f32(cref_s + 4 * x);
+                        const bool moved = cn - co > kLeanMaxLead;
+                        sts_f32(ftab_s + 4 * x, moved ? ex2_approx((co - cn) * kLog2e) : 1.f);
+                        if (moved) sts_f32(cref_s + 4 * x, cn);
+                    }
+                    __syncwarp();
+                    {
+                        const int rcur = ri < L::MAXR ? ri : 0;
+#pragma unroll
+                        for (int v = 0; v < V; ++v) {
+                            const float sc = lds_f32(ftab_s + (unsigned)((rcur * H + hv[v]) * 4));
+                            sv[v] *= sc;
+                            const f32x2 s2 = pack2(sc, sc);
+#pragma unroll
+                            for (int t = 0; t < NP; ++t) pacc0[v][t] = fma2(pacc0[v][t], s2, zero2());
+                        }
+                    }
+                    __syncwarp();
+                }
+#pragma unroll
+                for (int n = 0; n < NIT; ++n) {
+                    const int it = lane + 32 * n;
+                    if (ITEMS % 32 == 0 || it < ITEMS) {
+                        const int p = it / H;
+                        sts_f32(w_s + (unsigned)((((p % EPW) * H + hl) * SPS + p / EPW) * 4), w0[n]);
                     }
                 }
                 __syncwarp();
-                if (open) {
-#pragma unroll
-                    for (int v = 0; v < V; ++v) {
-                        const float sc = lds_f32(scale_s + 4 * (unsigned)hv[v]);
-                        sv[v] *= sc;
-                        const f32x2 s2 = pack2(sc, sc);
-#pragma unroll
-                        for (int t = 0; t < NP; ++t) pacc0[v][t] = fma2(pacc0[v][t], s2, zero2());
-                    }
-                }
                 const unsigned ring_a = ring_l + (unsigned)((j % NS) * STAGE);
                 const int cnt = nslots - s;
                 unsigned ends;
@@ -367,7 +386,6 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
                     }
                     ends = __ballot_sync(0xffffffffu, bit != 0);
                 }
-                open = (ends & (1u << (SPS - 1))) == 0u;
                 float4 w4[V];
 #pragma unroll
                 for (int k = 0; k < SPS; ++k) {
@@ -389,12 +407,28 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
                         // ---- the row is complete -------------------------------------------------------------
                         const long long row = row0 + r + ri;
                         if constexpr (SEG) {
-                            // partial accumulators of the segment, float32, with its own max, for the merge launch
+                            // partial accumulators of the segment, float32, against its own max, for the merge launch
+                            constexpr long long rowf = (long long)NVEC * EPV;
+                            float *rec = a.sp.part + seg * a.sp.pstride;
+                            if (lane < H) {
+                                float gr;
+                                const float mm = leaky(el_seg + mrun, a.slope, gr);
+                                rec[rowf + lane] = mm;
+                                sts_f32(ftab_s + 4 * lane, ex2_approx((lds_f32(cref_s + 4 * lane) - mm) * kLog2e));
+                            }
+                            __syncwarp();
                             float acc0[V][EPV];
 #pragma unroll
-                            for (int v = 0; v < V; ++v)
+                            for (int v = 0; v < V; ++v) {
+                                const float sc = lds_f32(ftab_s + 4 * (unsigned)hv[v]);
+                                sv[v] *= sc;
 #pragma unroll
-                                for (int t = 0; t < NP; ++t) unpack2(pacc0[v][t], acc0[v][2 * t], acc0[v][2 * t + 1]);
+                                for (int t = 0; t < NP; ++t) {
+                                    unpack2(pacc0[v][t], acc0[v][2 * t], acc0[v][2 * t + 1]);
+                                    acc0[v][2 * t] *= sc;
+                                    acc0[v][2 * t + 1] *= sc;
+                                }
+                            }
 #pragma unroll
                             for (int off = G; off < 32; off <<= 1)
 #pragma unroll
@@ -403,8 +437,6 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
 #pragma unroll
                                     for (int e = 0; e < EPV; ++e) acc0[v][e] += __shfl_xor_sync(0xffffffffu, acc0[v][e], off);
                                 }
-                            constexpr long long rowf = (long long)NVEC * EPV;
-                            float *rec = a.sp.part + seg * a.sp.pstride;
                             if (half == 0) {
                                 bool vok[V];
 #pragma unroll
@@ -413,10 +445,6 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
 #pragma unroll
                                 for (int v = 0; v < V; ++v)
                                     if ((gl % VPH) == 0) rec[rowf + H + hv[v]] = sv[v];
-                            }
-                            if (lane < H) {
-                                float gr;
-                                rec[rowf + lane] = leaky(el_seg + mrun, a.slope, gr);
                             }
                         } else {
 #pragma unroll
@@ -481,7 +509,7 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
                     mm = leaky(lds_f32(rc_s + 4 * x) + fkey_inv(k), a.slope, gr);
                 }
                 a.m_out[o] = mm;
-                a.d_out[o] = lds_f32(sout_s + 4 * x);
+                a.d_out[o] = k != kKeyNegInf ? lds_f32(sout_s + 4 * x) * ex2_approx((lds_f32(cref_s + 4 * x) - mm) * kLog2e) : 0.f;
             }
             __syncwarp();
         }

@@ -464,7 +464,7 @@ static sar_status launch_lean_src(LeanSrcArgs a, long long nnz, cudaStream_t st)
     a.R = lean_rows_per_span(a.n_rows, nnz, kLeanCap);
     const long long spans = (a.n_rows + a.R - 1) / a.R;
     if (spans > 0) {
-        auto kern = lean_src_kernel<T, G, V, H, false, kLeanCap, P, NS, kLeanMinBlocks>;
+        auto kern = lean_src_kernel<T, G, V, H, false, kLeanCap, P, NS, kLeanMinBlocksBwdRows>;
         SAR_TRY(ensure_smem(kern, LR::total));
         SAR_LAUNCH("gat_bwd_src", st, kern<<<(unsigned)spans, 32, LR::total, st>>>(a));
         SAR_TRY(sar_after_launch());

@@ -285,6 +285,34 @@ def test_large_logits_stay_finite_and_match():
         allclose_report(m.cpu().numpy(), f.m, 1e-6, 1e-6, "m")
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_scores_far_above_a_rows_first_score(dtype):
+    """The whole-graph forward pass shifts a row's softmax by the score of its first edge and moves the shift when a
+    later score leads it by more than 60: score terms of magnitude ~50 make that happen in short rows, in rows that span
+    several stages and in the segments of hub rows; out, m, d and the gradients must still match the oracle."""
+    n, src, dst = hub_graph(n=4000, e=60000, d_max=900.0, seed=21)
+    p = Problem(n, src, dst, 4, 32, 77, scale=25.0, dtype=dtype)
+    f = p.oracle_fwd()
+    b = p.oracle_bwd(f)
+    out, m, d = p.gpu_fwd("fused")[:3]
+    assert torch.isfinite(out).all() and torch.isfinite(d).all()
+    # scores of magnitude ~1e2 carry float32 rounding of ~1e-5 in the exponent, whatever the kernel
+    if dtype == "f32":
+        allclose_report(out.float().cpu().numpy(), f.out, 1e-4, 2e-5, "out[far]")
+    else:
+        check_out(out, f.out, dtype, "out[far]")
+    allclose_report(m.cpu().numpy(), f.m, 1e-6, 1e-6, "m[far]")
+    allclose_report(d.cpu().numpy(), f.d, 1e-4, 1e-6, "d[far]")
+    dfeat, del_, der = p.gpu_bwd(m, d, out=out, mode="fused")
+    if dtype == "f32":
+        allclose_report(dfeat.float().cpu().numpy(), b.dfeat, 1e-4, 1e-4 * max(rms(b.dfeat), 1.0), "dfeat[far]")
+    else:
+        check_grad(dfeat, b.dfeat, dtype, "dfeat[far]", stored=True)
+    # sums of O(1) terms that cancel, each carrying the exponent's rounding
+    allclose_report(del_.cpu().numpy(), b.del_, 1e-4, 5e-4 * max(rms(b.del_), 1.0), "del[far]")
+    allclose_report(der.cpu().numpy(), b.der, 1e-4, 5e-4 * max(rms(b.der), 1.0), "der[far]")
+
+
 def test_degenerate_graphs():
     # no edges at all
     n = 37
