@@ -143,9 +143,9 @@ NCU_TRAFFIC_SOURCE = ("ncu one-pass capture of these kernels at full size (profi
                       "not measured in this run")
 NCU_TRAFFIC = {
     # (workload, storage dtype, pass): bytes per full-size pass
-    ("large", "bf16", "gat_fwd"): 82.12e9,
-    ("large", "bf16", "gat_bwd_dst"): 84.30e9,
-    ("large", "bf16", "gat_bwd_src"): 89.40e9,
+    ("large", "bf16", "gat_fwd"): 82.36e9,
+    ("large", "bf16", "gat_bwd_dst"): 84.37e9,
+    ("large", "bf16", "gat_bwd_src"): 89.50e9,
 }
 
 
