@@ -65,27 +65,45 @@ __global__ void __launch_bounds__(kThreads) gat_fwd_merge_kernel(const FwdArgs a
             }
         load_acc_row<G, V, EPV>(a.acc + row * rowf, id.gl, vg.vok, acc);
     }
-    for (long long s = s0; s < s1; ++s) {
-        const float *rec = a.sp.part + s * a.sp.pstride;
+    // a hub row has hundreds of segments: the records of U segments are requested together, then folded in order
+    constexpr int U = MergeBatch<V>::U;
+    for (long long s = s0; s < s1; s += U) {
+        float4 buf[U][V][EPV / 4];
+        float Ms[U][V], ds[U][V];
 #pragma unroll
-        for (int v = 0; v < V; ++v)
-            if (vg.vok[v]) {
-                const float Ms = rec[rowf + vg.hv[v]], ds = rec[rowf + H + vg.hv[v]];
-                const float Mn = fmaxf(Mv[v], Ms);
-                const float c_old = (Mn == SAR_NEG_INF) ? 1.f : fast_exp(Mv[v] - Mn);
-                const float c_new = (Mn == SAR_NEG_INF) ? 1.f : fast_exp(Ms - Mn);
-                const float4 *p = reinterpret_cast<const float4 *>(rec + (size_t)(v * G + id.gl) * EPV);
+        for (int u = 0; u < U; ++u) {
+            if (s + u < s1) {
+                const float *rec = a.sp.part + (s + u) * a.sp.pstride;
+                load_acc_vecs<G, V, EPV>(rec, id.gl, vg.vok, buf[u]);
 #pragma unroll
-                for (int q = 0; q < EPV / 4; ++q) {
-                    const float4 x = p[q];
-                    acc[v][4 * q] = acc[v][4 * q] * c_old + x.x * c_new;
-                    acc[v][4 * q + 1] = acc[v][4 * q + 1] * c_old + x.y * c_new;
-                    acc[v][4 * q + 2] = acc[v][4 * q + 2] * c_old + x.z * c_new;
-                    acc[v][4 * q + 3] = acc[v][4 * q + 3] * c_old + x.w * c_new;
+                for (int v = 0; v < V; ++v) {
+                    Ms[u][v] = vg.vok[v] ? rec[rowf + vg.hv[v]] : SAR_NEG_INF;
+                    ds[u][v] = vg.vok[v] ? rec[rowf + H + vg.hv[v]] : 0.f;
                 }
-                dv[v] = dv[v] * c_old + ds * c_new;
-                Mv[v] = Mn;
             }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (s + u < s1) {
+#pragma unroll
+                for (int v = 0; v < V; ++v)
+                    if (vg.vok[v]) {
+                        const float Mn = fmaxf(Mv[v], Ms[u][v]);
+                        const float c_old = (Mn == SAR_NEG_INF) ? 1.f : fast_exp(Mv[v] - Mn);
+                        const float c_new = (Mn == SAR_NEG_INF) ? 1.f : fast_exp(Ms[u][v] - Mn);
+#pragma unroll
+                        for (int q = 0; q < EPV / 4; ++q) {
+                            const float4 x = buf[u][v][q];
+                            acc[v][4 * q] = acc[v][4 * q] * c_old + x.x * c_new;
+                            acc[v][4 * q + 1] = acc[v][4 * q + 1] * c_old + x.y * c_new;
+                            acc[v][4 * q + 2] = acc[v][4 * q + 2] * c_old + x.z * c_new;
+                            acc[v][4 * q + 3] = acc[v][4 * q + 3] * c_old + x.w * c_new;
+                        }
+                        dv[v] = dv[v] * c_old + ds[u][v] * c_new;
+                        Mv[v] = Mn;
+                    }
+            }
+        }
     }
     if (last) {
         if (a.flags & SAR_KEEP_NUMERATOR) store_acc_row<G, V, EPV>(a.acc + row * rowf, id.gl, vg.vok, acc);
@@ -192,13 +210,32 @@ __global__ void __launch_bounds__(kThreads) gat_bwd_dst_merge_kernel(const BwdDs
     long long row = -1;
     if (active) {
         row = a.sp.long_row[lr];
-        for (long long s = a.sp.long_seg[lr]; s < a.sp.long_seg[lr + 1]; ++s) {
-            const float *recp = a.sp.part + s * a.sp.pstride;
-            add_acc_row<G, V, EPV>(recp, id.gl, vg.vok, accB, 1.f, 1.f);
-            if constexpr (!GIVEN_D) add_acc_row<G, V, EPV>(recp + rowf, id.gl, vg.vok, accA, 1.f, 1.f);
+        // the records of U segments are requested together, then added in order
+        constexpr int U = MergeBatch<V>::U;
+        const long long s1 = a.sp.long_seg[lr + 1];
+        for (long long s = a.sp.long_seg[lr]; s < s1; s += U) {
+            float4 bufB[U][V][EPV / 4], bufA[U][V][EPV / 4];
+            float Ss[U][V];
 #pragma unroll
-            for (int v = 0; v < V; ++v)
-                if (vg.vok[v]) S[v] += recp[2 * rowf + vg.hv[v]];
+            for (int u = 0; u < U; ++u) {
+                if (s + u < s1) {
+                    const float *recp = a.sp.part + (s + u) * a.sp.pstride;
+                    load_acc_vecs<G, V, EPV>(recp, id.gl, vg.vok, bufB[u]);
+                    if constexpr (!GIVEN_D) load_acc_vecs<G, V, EPV>(recp + rowf, id.gl, vg.vok, bufA[u]);
+#pragma unroll
+                    for (int v = 0; v < V; ++v) Ss[u][v] = vg.vok[v] ? recp[2 * rowf + vg.hv[v]] : 0.f;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (s + u < s1) {
+                    add_acc_vecs<V, EPV>(bufB[u], vg.vok, accB, 1.f, 1.f);
+                    if constexpr (!GIVEN_D) add_acc_vecs<V, EPV>(bufA[u], vg.vok, accA, 1.f, 1.f);
+#pragma unroll
+                    for (int v = 0; v < V; ++v)
+                        if (vg.vok[v]) S[v] += Ss[u][v];
+                }
+            }
         }
         load_row_vec<T, G, V>(a.gout, row, a.g.n_vec, id.gl, vg.vok, gv);
     }
@@ -275,13 +312,32 @@ __global__ void __launch_bounds__(kThreads) gat_bwd_src_merge_kernel(const BwdSr
     long long row = -1;
     if (lr < a.sp.n_long) {
         row = a.sp.long_row[lr];
-        for (long long s = a.sp.long_seg[lr]; s < a.sp.long_seg[lr + 1]; ++s) {
-            const float *recp = a.sp.part + s * a.sp.pstride;
-            add_acc_row<G, V, EPV>(recp, id.gl, vg.vok, accD, 1.f, 1.f);
-            add_acc_row<G, V, EPV>(recp + rowf, id.gl, vg.vok, accC, 1.f, 1.f);
+        // the records of U segments are requested together, then added in order
+        constexpr int U = MergeBatch<V>::U;
+        const long long s1 = a.sp.long_seg[lr + 1];
+        for (long long s = a.sp.long_seg[lr]; s < s1; s += U) {
+            float4 bufD[U][V][EPV / 4], bufC[U][V][EPV / 4];
+            float Ss[U][V];
 #pragma unroll
-            for (int v = 0; v < V; ++v)
-                if (vg.vok[v]) S[v] += recp[2 * rowf + vg.hv[v]];
+            for (int u = 0; u < U; ++u) {
+                if (s + u < s1) {
+                    const float *recp = a.sp.part + (s + u) * a.sp.pstride;
+                    load_acc_vecs<G, V, EPV>(recp, id.gl, vg.vok, bufD[u]);
+                    load_acc_vecs<G, V, EPV>(recp + rowf, id.gl, vg.vok, bufC[u]);
+#pragma unroll
+                    for (int v = 0; v < V; ++v) Ss[u][v] = vg.vok[v] ? recp[2 * rowf + vg.hv[v]] : 0.f;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (s + u < s1) {
+                    add_acc_vecs<V, EPV>(bufD[u], vg.vok, accD, 1.f, 1.f);
+                    add_acc_vecs<V, EPV>(bufC[u], vg.vok, accC, 1.f, 1.f);
+#pragma unroll
+                    for (int v = 0; v < V; ++v)
+                        if (vg.vok[v]) S[v] += Ss[u][v];
+                }
+            }
         }
     }
     bwd_src_epilogue<T, G, V>(a, id, vg, scratch, row, accD, accC, S);
@@ -401,8 +457,17 @@ __global__ void __launch_bounds__(kThreads) spmm_merge_kernel(const SumArgs a) {
     for (int v = 0; v < V; ++v)
 #pragma unroll
         for (int e = 0; e < EPV; ++e) acc[v][e] = 0.f;
-    for (long long s = a.sp.long_seg[lr]; s < a.sp.long_seg[lr + 1]; ++s)
-        add_acc_row<G, V, EPV>(a.sp.part + s * a.sp.pstride, id.gl, vg.vok, acc, 1.f, 1.f);
+    constexpr int U = MergeBatch<V>::U;
+    const long long s1 = a.sp.long_seg[lr + 1];
+    for (long long s = a.sp.long_seg[lr]; s < s1; s += U) {
+        float4 buf[U][V][EPV / 4];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (s + u < s1) load_acc_vecs<G, V, EPV>(a.sp.part + (s + u) * a.sp.pstride, id.gl, vg.vok, buf[u]);
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (s + u < s1) add_acc_vecs<V, EPV>(buf[u], vg.vok, acc, 1.f, 1.f);
+    }
     sum_epilogue<T, G, V>(a, id.gl, vg, a.sp.long_row[lr], acc);
 }
 

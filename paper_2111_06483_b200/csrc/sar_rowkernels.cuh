@@ -116,6 +116,41 @@ __device__ __forceinline__ void add_acc_row(const float *__restrict__ rowp, int 
         }
 }
 
+// The same in two steps, so that a merge loop can have the loads of several records in flight before it folds
+// them in order: load the lane's vectors of one float32 record row ...
+template <int G, int V, int EPV>
+__device__ __forceinline__ void load_acc_vecs(const float *__restrict__ rowp, int gl, const bool (&vok)[V],
+                                              float4 (&buf)[V][EPV / 4]) {
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        const float4 *p = reinterpret_cast<const float4 *>(rowp + (size_t)(v * G + gl) * EPV);
+#pragma unroll
+        for (int q = 0; q < EPV / 4; ++q) buf[v][q] = vok[v] ? p[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+}
+// ... and fold them (the arithmetic of add_acc_row, term by term)
+template <int V, int EPV>
+__device__ __forceinline__ void add_acc_vecs(const float4 (&buf)[V][EPV / 4], const bool (&vok)[V], float (&acc)[V][EPV],
+                                             float scale_old, float scale_new) {
+#pragma unroll
+    for (int v = 0; v < V; ++v)
+        if (vok[v]) {
+#pragma unroll
+            for (int q = 0; q < EPV / 4; ++q) {
+                const float4 x = buf[v][q];
+                acc[v][4 * q] = acc[v][4 * q] * scale_old + x.x * scale_new;
+                acc[v][4 * q + 1] = acc[v][4 * q + 1] * scale_old + x.y * scale_new;
+                acc[v][4 * q + 2] = acc[v][4 * q + 2] * scale_old + x.z * scale_new;
+                acc[v][4 * q + 3] = acc[v][4 * q + 3] * scale_old + x.w * scale_new;
+            }
+        }
+}
+// records a merge loop keeps in flight
+template <int V>
+struct MergeBatch {
+    static constexpr int U = V == 1 ? 4 : 2;
+};
+
 // One row vector of storage type T -> float registers.
 // READONLY = false for arrays the same launch also writes (plain, coherent loads).
 template <typename T, int G, int V, bool READONLY = true>
