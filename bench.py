@@ -833,6 +833,18 @@ def run_ours(args, rank, world, local_rank):
         gc.collect()
         torch.cuda.empty_cache()
         others = extra_workloads(dev, peak, args)
+        if args.ids == "permuted":
+            # locality ablation: the same recipe with node id = degree rank (hubs next to each other, rows of similar
+            # length in a span) instead of the seeded permutation; fused schedule, five steps
+            st2 = AggStack(cfg, dtype, dev, ids="degree_sorted", parts=False)
+            r2 = measure(st2.step("fused"), 5, 3, clocks_gpu=None)
+            others["large_ids_in_degree_order"] = {"ms_per_step": r2["ms_per_step"], "steps": 5,
+                                                   "edges_per_sec": L * e / (r2["ms_per_step"] * 1e-3),
+                                                   "passes_ms": {k: v["ms"] for k, v in pass_table(r2["kernels"], 5 * L, n, e, H, F, b, peak).items()},
+                                                   "note": "ablation, not the workload's recipe: ids are a seeded permutation there"}
+            del st2
+            gc.collect()
+            torch.cuda.empty_cache()
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
