@@ -285,13 +285,13 @@ def test_large_logits_stay_finite_and_match():
         allclose_report(m.cpu().numpy(), f.m, 1e-6, 1e-6, "m")
 
 
-@pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_scores_far_above_a_rows_first_score(dtype):
+@pytest.mark.parametrize("H,F,dtype", [(4, 32, "f32"), (4, 32, "bf16"), (8, 32, "bf16"), (4, 64, "f32")])
+def test_scores_far_above_a_rows_first_score(H, F, dtype):
     """The whole-graph forward pass shifts a row's softmax by the score of its first edge and moves the shift when a
     later score leads it by more than 60: score terms of magnitude ~50 make that happen in short rows, in rows that span
     several stages and in the segments of hub rows; out, m, d and the gradients must still match the oracle."""
     n, src, dst = hub_graph(n=4000, e=60000, d_max=900.0, seed=21)
-    p = Problem(n, src, dst, 4, 32, 77, scale=25.0, dtype=dtype)
+    p = Problem(n, src, dst, H, F, 77, scale=25.0, dtype=dtype)
     f = p.oracle_fwd()
     b = p.oracle_bwd(f)
     out, m, d = p.gpu_fwd("fused")[:3]
