@@ -340,7 +340,7 @@ class AggStack:
 
     feat^{l+1} = out^l with seeded el^l, er^l; the backward pass feeds dfeat^{l+1} as gout of layer l."""
 
-    def __init__(self, cfg, dtype, dev, ids="permuted", threshold=None, parts=True, t_threshold=None):
+    def __init__(self, cfg, dtype, dev, ids="permuted", threshold=None, parts=True, t_threshold=None, reorder=None):
         import torch
         import workloads
         from paper_2111_06483_b200 import api, binding as B
@@ -356,7 +356,7 @@ class AggStack:
         torch.cuda.synchronize()
         t0 = time.perf_counter()
         self.g = api.Graph.from_coo(n, src, dst, k=K, threshold=self.threshold, build_parts=parts and K > 1,
-                                    t_threshold=t_threshold)
+                                    t_threshold=t_threshold, reorder=reorder)
         torch.cuda.synchronize()
         self.prep_ms = 1e3 * (time.perf_counter() - t0)
         del src, dst
@@ -366,6 +366,11 @@ class AggStack:
         self.els = [workloads.normal_tensor((n, H), cfg.seed, 16 * l + 12, device=dev) for l in range(L)]
         self.ers = [workloads.normal_tensor((n, H), cfg.seed, 16 * l + 13, device=dev) for l in range(L)]
         self.gout = workloads.normal_tensor((n, H, F), cfg.seed, 11, device=dev, dtype=tdt)
+        if reorder:   # the node arrays enter the graph's numbering once, before the timed region
+            self.feats[0] = self.g.to_internal(self.feats[0])
+            self.els = [self.g.to_internal(x) for x in self.els]
+            self.ers = [self.g.to_internal(x) for x in self.ers]
+            self.gout = self.g.to_internal(self.gout)
         self.gbuf = [torch.empty((n, H, F), dtype=tdt, device=dev) for _ in range(2)]
         f32 = lambda: torch.empty((n, H), dtype=torch.float32, device=dev)
         self.ms, self.ds = [f32() for _ in range(L)], [f32() for _ in range(L)]
@@ -834,14 +839,16 @@ def run_ours(args, rank, world, local_rank):
         torch.cuda.empty_cache()
         others = extra_workloads(dev, peak, args)
         if args.ids == "permuted":
-            # locality ablation: the same recipe with node id = degree rank (hubs next to each other, rows of similar
-            # length in a span) instead of the seeded permutation; fused schedule, five steps
-            st2 = AggStack(cfg, dtype, dev, ids="degree_sorted", parts=False)
+            # the same workload (ids a seeded permutation) with the library's renumbering by degree in graph preparation
+            # (sar_degree_order: hubs next to each other, rows of similar length in a span); the node arrays are
+            # carried into the new numbering once, outside the timed region; fused schedule, five steps
+            st2 = AggStack(cfg, dtype, dev, ids="permuted", parts=False, reorder="degree")
             r2 = measure(st2.step("fused"), 5, 3, clocks_gpu=None)
-            others["large_ids_in_degree_order"] = {"ms_per_step": r2["ms_per_step"], "steps": 5,
+            others["large_renumbered_by_degree"] = {"ms_per_step": r2["ms_per_step"], "steps": 5, "prep_ms": st2.prep_ms,
                                                    "edges_per_sec": L * e / (r2["ms_per_step"] * 1e-3),
                                                    "passes_ms": {k: v["ms"] for k, v in pass_table(r2["kernels"], 5 * L, n, e, H, F, b, peak).items()},
-                                                   "note": "ablation, not the workload's recipe: ids are a seeded permutation there"}
+                                                   "note": "graph preparation with reorder='degree' (sar_degree_order, sar_relabel, sar_permute_rows); "
+                                                           "`value` above is measured without it"}
             del st2
             gc.collect()
             torch.cuda.empty_cache()

@@ -164,6 +164,27 @@ SAR_API sar_status sar_csr_split_indices(int64_t n_dst, const int64_t *indptr, c
 SAR_API sar_status sar_csc_slice_indptr(int64_t s0, int64_t s1, const int64_t *t_indptr, int64_t *t_indptr_q,
                                         void *stream);
 
+/* Node order for locality (no counterpart in the paper's algorithms; the paper prepares its graphs offline with a
+ * graph partitioner, Sec. 4.2, so that a worker's rows mostly gather their own features - this is what a single GPU
+ * can do in that step for an input whose node ids carry no locality).  Nodes are numbered by total degree (edges
+ * as a source + edges as a destination), descending, ties by ascending id: frequently gathered rows become
+ * neighbours, and the rows a span of the kernels owns have similar lengths.  Integer work, results unique.
+ *
+ * sar_degree_order: src, dst are the DEVICE edge list (e entries each, ids in [0, n)); writes order[n] (new id ->
+ *   old id) and rank[n] (old id -> new id), DEVICE arrays.  workspace: DEVICE, 256-byte aligned, at least
+ *   sar_degree_order_workspace_bytes(n) bytes, else SAR_ERR_WORKSPACE.
+ * sar_relabel: out[t] = rank[ids[t]] for t < e (out may equal ids).  The relabelled edge list then goes through
+ *   sar_csr_from_coo as usual.
+ * sar_permute_rows: out row i = in row index[i], n rows of row_bytes bytes, DEVICE arrays, in != out.  With
+ *   index = order it carries a node array into the new numbering, with index = rank it carries one back.
+ * All three enqueue on `stream` and return without synchronising; nothing is allocated. */
+SAR_API size_t sar_degree_order_workspace_bytes(int64_t n);
+SAR_API sar_status sar_degree_order(int64_t n, int64_t e, const int32_t *src, const int32_t *dst, int32_t *order,
+                                    int32_t *rank, void *workspace, size_t workspace_bytes, void *stream);
+SAR_API sar_status sar_relabel(int64_t e, const int32_t *ids, const int32_t *rank, int32_t *out, void *stream);
+SAR_API sar_status sar_permute_rows(int64_t n, int64_t row_bytes, const int32_t *index, const void *in, void *out,
+                                    void *stream);
+
 /* Message-flow pruning (Appendix B: with few labelled nodes, a layer only has to update the nodes that can
  * still influence a labelled node's output).  Both masks are DEVICE arrays of n bytes (0 / non-zero).
  *

@@ -344,6 +344,21 @@ def csr_filter_rows(indptr, indices, keep):
     return out_ptr, out_idx
 
 
+def degree_order(n: int, src, dst):
+    """Node order by total degree (edges as a source + edges as a destination), descending, ties by ascending id:
+    order[new] = old, rank[old] = new.  Graph preparation for locality; the paper's counterpart is its offline
+    partitioning (Sec. 4.2), not one of its algorithms."""
+    src, dst = _i32(src), _i32(dst)
+    deg = np.zeros(n, dtype=np.int64)
+    for t in range(src.shape[0]):
+        deg[src[t]] += 1
+        deg[dst[t]] += 1
+    order = np.array(sorted(range(n), key=lambda i: (-deg[i], i)), dtype=np.int32)
+    rank = np.empty(n, dtype=np.int32)
+    rank[order] = np.arange(n, dtype=np.int32)
+    return order, rank
+
+
 def spmm_scaled(indptr, indices, feat, src_scale=None, dst_scale=None):
     """out[i,:] = dst_scale[i] * sum over the in-edges (j -> i) of src_scale[j] * feat[j,:], float64
     (the propagation X <- diag(dst_scale) A diag(src_scale) X; a missing scale is all ones)."""

@@ -45,14 +45,47 @@ class Graph:
     k: int = 1
     bounds: List[int] = field(default_factory=list)
     parts: List[B.Part] = field(default_factory=list)
+    order: Optional[torch.Tensor] = None    # reorder="degree": the graph's node i is the caller's node order[i]
+    rank: Optional[torch.Tensor] = None     # ... and the caller's node j is the graph's node rank[j]
+
+    def to_internal(self, x: torch.Tensor) -> torch.Tensor:
+        """A node array [n, ...] in the caller's numbering -> the graph's numbering (a copy; x itself when the graph
+        keeps the caller's numbering)."""
+        if self.order is None:
+            return x
+        out = torch.empty_like(x)
+        B.sar_permute_rows(self.order, x.contiguous(), out)
+        return out
+
+    def to_external(self, x: torch.Tensor) -> torch.Tensor:
+        """The inverse of to_internal."""
+        if self.rank is None:
+            return x
+        out = torch.empty_like(x)
+        B.sar_permute_rows(self.rank, x.contiguous(), out)
+        return out
 
     @staticmethod
     def from_coo(n: int, src: torch.Tensor, dst: torch.Tensor, k: int = 1, threshold: int = DEFAULT_THRESHOLD,
-                 build_parts: bool = False, t_threshold: Optional[int] = None) -> "Graph":
+                 build_parts: bool = False, t_threshold: Optional[int] = None,
+                 reorder: Optional[str] = None) -> "Graph":
         """src[t] -> dst[t] int32 CUDA tensors.  Builds CSR by destination, its transpose, the long-row
-        plans and (build_parts) the K per-partition sub-graphs with local source ids."""
+        plans and (build_parts) the K per-partition sub-graphs with local source ids.
+        reorder="degree": the nodes are renumbered by total degree first (sar_degree_order); every node array then
+        enters through to_internal and leaves through to_external."""
         dev = src.device
         nnz = src.numel()
+        order = rank = None
+        if reorder == "degree":
+            order = torch.empty(n, dtype=torch.int32, device=dev)
+            rank = torch.empty(n, dtype=torch.int32, device=dev)
+            B.sar_degree_order(n, src, dst, order, rank, _workspace(B.sar_degree_order_workspace_bytes(n), dev))
+            src2, dst2 = torch.empty_like(src), torch.empty_like(dst)
+            B.sar_relabel(src, rank, src2)
+            B.sar_relabel(dst, rank, dst2)
+            src, dst = src2, dst2
+        elif reorder is not None:
+            raise ValueError(f"unknown reorder {reorder!r}")
         ws = _workspace(B.sar_graph_workspace_bytes(nnz, n), dev)
         indptr = torch.empty(n + 1, dtype=torch.int64, device=dev)
         indices = torch.empty(nnz, dtype=torch.int32, device=dev)
@@ -65,7 +98,7 @@ class Graph:
         split = build_plan(n, indptr, threshold) if threshold else None
         t_split = build_plan(n, t_indptr, t_threshold) if t_threshold else None
         whole = B.Part(n, n, indptr, indices, t_indptr, t_indices, split, t_split)
-        g = Graph(n=n, nnz=nnz, whole=whole, k=k, bounds=B.sar_partition_bounds(n, k))
+        g = Graph(n=n, nnz=nnz, whole=whole, k=k, bounds=B.sar_partition_bounds(n, k), order=order, rank=rank)
         if build_parts:
             g.parts = split_parts(whole, g.bounds, threshold, ws)
         return g

@@ -35,7 +35,7 @@ EXPORTS = [
     "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd", "sar_axpby", "sar_bn_rstd", "sar_accumulate", "sar_round_to", "sar_bn_apply_act",
     "sar_bn_bwd_stats_act", "sar_bn_bwd_apply_act", "sar_csc_slice_indptr",
     "sar_gat_storing_workspace_bytes", "sar_gat_fwd_storing", "sar_gat_bwd_storing", "sar_bn_combine_moments",
-    "sar_bn_combine_sums",
+    "sar_bn_combine_sums", "sar_degree_order_workspace_bytes", "sar_degree_order", "sar_relabel", "sar_permute_rows",
 ]
 
 
@@ -73,7 +73,8 @@ def lib() -> ctypes.CDLL:
         L.sar_built_for_sm.restype = c_int32
         for name in ("sar_graph_workspace_bytes", "sar_gat_workspace_bytes", "sar_spmm_workspace_bytes",
                      "sar_gat_stack_arena_bytes", "sar_gat_bwd_noalloc_limit", "sar_gat_project_workspace_bytes",
-                     "sar_bn_workspace_bytes", "sar_linear_workspace_bytes", "sar_gat_storing_workspace_bytes"):
+                     "sar_bn_workspace_bytes", "sar_linear_workspace_bytes", "sar_gat_storing_workspace_bytes",
+                     "sar_degree_order_workspace_bytes"):
             getattr(L, name).restype = c_size_t
         _lib = L
     return _lib
@@ -257,6 +258,35 @@ def sar_csc_slice_indptr(s0: int, s1: int, t_indptr: torch.Tensor, t_indptr_q: t
     assert t_indptr.dtype == torch.int64 and t_indptr_q.dtype == torch.int64 and t_indptr_q.numel() == s1 - s0 + 1
     _check("sar_csc_slice_indptr", lib().sar_csc_slice_indptr(c_int64(s0), c_int64(s1), _ptr(t_indptr),
                                                               _ptr(t_indptr_q), _stream()))
+
+
+def sar_degree_order_workspace_bytes(n: int) -> int:
+    return int(lib().sar_degree_order_workspace_bytes(c_int64(n)))
+
+
+def sar_degree_order(n: int, src: torch.Tensor, dst: torch.Tensor, order: torch.Tensor, rank: torch.Tensor,
+                     workspace: torch.Tensor) -> None:
+    assert src.dtype == torch.int32 and dst.dtype == torch.int32 and src.numel() == dst.numel()
+    assert order.dtype == torch.int32 and rank.dtype == torch.int32 and order.numel() == n and rank.numel() == n
+    wp, wb = _ws(workspace)
+    _check("sar_degree_order", lib().sar_degree_order(c_int64(n), c_int64(src.numel()), _ptr(src), _ptr(dst), _ptr(order),
+                                                      _ptr(rank), wp, wb, _stream()))
+
+
+def sar_relabel(ids: torch.Tensor, rank: torch.Tensor, out: torch.Tensor) -> None:
+    assert ids.dtype == torch.int32 and rank.dtype == torch.int32 and out.dtype == torch.int32
+    assert out.numel() == ids.numel()
+    _check("sar_relabel", lib().sar_relabel(c_int64(ids.numel()), _ptr(ids), _ptr(rank), _ptr(out), _stream()))
+
+
+def sar_permute_rows(index: torch.Tensor, x: torch.Tensor, out: torch.Tensor) -> None:
+    """out row i = x row index[i]; x, out contiguous with the same shape, first dimension = index.numel()."""
+    assert index.dtype == torch.int32 and x.is_contiguous() and out.is_contiguous()
+    assert x.shape == out.shape and x.dtype == out.dtype and x.shape[0] == index.numel()
+    n = index.numel()
+    row_bytes = (x.numel() // n) * x.element_size() if n else 1
+    _check("sar_permute_rows", lib().sar_permute_rows(c_int64(n), c_int64(row_bytes), _ptr(index), _ptr(x), _ptr(out),
+                                                      _stream()))
 
 
 def sar_mfg_frontier(n: int, indptr: torch.Tensor, indices: torch.Tensor, need_out: torch.Tensor,

@@ -173,6 +173,47 @@ __global__ void filter_fill_kernel(long long n, const int64_t *__restrict__ indp
     for (long long t = lane; t < cnt; t += 32) indices_out[w + t] = indices[beg + t];
 }
 
+// ---- node order by degree ---------------------------------------------------------------------------------------
+// degree of a node = edges it is the source of + edges it is the destination of (integer atomics: order-independent)
+__global__ void degree_count_kernel(long long e, const int32_t *__restrict__ src, const int32_t *__restrict__ dst,
+                                    unsigned *__restrict__ deg) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= e) return;
+    atomicAdd(deg + src[t], 1u);
+    atomicAdd(deg + dst[t], 1u);
+}
+
+// key of node i: (2^32 - 1 - degree) in the high word, i in the low word: ascending keys = descending degree, ties by id
+__global__ void order_keys_kernel(long long n, const unsigned *__restrict__ deg, unsigned long long *__restrict__ keys) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) keys[i] = ((unsigned long long)(0xffffffffu - deg[i]) << 32) | (unsigned)i;
+}
+
+__global__ void order_from_keys_kernel(long long n, const unsigned long long *__restrict__ keys,
+                                       int32_t *__restrict__ order, int32_t *__restrict__ rank) {
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int32_t old = (int32_t)(unsigned)(keys[i] & 0xffffffffull);
+    order[i] = old;
+    rank[old] = (int32_t)i;
+}
+
+__global__ void relabel_kernel(long long e, const int32_t *__restrict__ ids, const int32_t *__restrict__ rank,
+                               int32_t *__restrict__ out) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t < e) out[t] = rank[ids[t]];
+}
+
+// out row i = in row index[i]; W = the widest word that divides the row
+template <typename W>
+__global__ void permute_rows_kernel(long long n, long long words, const int32_t *__restrict__ index,
+                                    const W *__restrict__ in, W *__restrict__ out) {
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= n * words) return;
+    const long long i = t / words, w = t - i * words;
+    out[t] = in[(long long)index[i] * words + w];
+}
+
 static inline unsigned nblk(long long n) { return (unsigned)((n + 255) / 256); }
 
 static size_t sort_temp_bytes(long long nnz) {
@@ -461,6 +502,63 @@ sar_status sar_plan_fill(int64_t n_rows, const int64_t *indptr, int32_t threshol
     if (need > temp_bytes) return SAR_ERR_WORKSPACE;
     SAR_CUDA_TRY(cub::DeviceScan::ExclusiveSum(temp, need, long_seg, long_seg, n_long + 1, st));
     return SAR_OK;
+}
+
+size_t sar_degree_order_workspace_bytes(int64_t n) {
+    if (n < 0) return 0;
+    return 2 * sar_round_up((size_t)n * 8, 256) + sar_round_up(sort_temp_bytes(n), 256) + sar_round_up((size_t)n * 4, 256) + 512;
+}
+
+sar_status sar_degree_order(int64_t n, int64_t e, const int32_t *src, const int32_t *dst, int32_t *order, int32_t *rank,
+                            void *workspace, size_t workspace_bytes, void *stream) {
+    if (n < 0 || e < 0 || (n > 0 && (!order || !rank)) || (e > 0 && (!src || !dst))) return SAR_ERR_INVALID_ARG;
+    if (n > INT32_MAX) return SAR_ERR_UNSUPPORTED;
+    if (!sar_aligned(src, 4) || !sar_aligned(dst, 4) || !sar_aligned(order, 4) || !sar_aligned(rank, 4)) return SAR_ERR_ALIGNMENT;
+    if (n == 0) return SAR_OK;
+    const size_t kb = sar_round_up((size_t)n * 8, 256), db = sar_round_up((size_t)n * 4, 256);
+    if (!workspace || !sar_aligned(workspace, 256) || workspace_bytes < 2 * kb + db) return SAR_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // layout: keys | sorted keys | CUB scratch ... | degrees (last)
+    unsigned *deg = reinterpret_cast<unsigned *>(static_cast<char *>(workspace) + workspace_bytes - db - (workspace_bytes - db) % 256);
+    if (reinterpret_cast<char *>(deg) < static_cast<char *>(workspace) + 2 * kb) return SAR_ERR_WORKSPACE;
+    const size_t sort_bytes = (size_t)(reinterpret_cast<char *>(deg) - static_cast<char *>(workspace));
+    SAR_CUDA_TRY(cudaMemsetAsync(deg, 0, (size_t)n * 4, st));
+    if (e > 0) {
+        degree_count_kernel<<<nblk(e), 256, 0, st>>>(e, src, dst, deg);
+        SAR_TRY(sar_after_launch());
+    }
+    unsigned long long *keys = static_cast<unsigned long long *>(workspace);
+    order_keys_kernel<<<nblk(n), 256, 0, st>>>(n, deg, keys);
+    SAR_TRY(sar_after_launch());
+    unsigned long long *sorted = keys;
+    SAR_TRY(sort_keys(n, 64, workspace, sort_bytes, st, &sorted));
+    order_from_keys_kernel<<<nblk(n), 256, 0, st>>>(n, sorted, order, rank);
+    return sar_after_launch();
+}
+
+sar_status sar_relabel(int64_t e, const int32_t *ids, const int32_t *rank, int32_t *out, void *stream) {
+    if (e < 0 || (e > 0 && (!ids || !rank || !out))) return SAR_ERR_INVALID_ARG;
+    if (!sar_aligned(ids, 4) || !sar_aligned(rank, 4) || !sar_aligned(out, 4)) return SAR_ERR_ALIGNMENT;
+    if (e == 0) return SAR_OK;
+    relabel_kernel<<<nblk(e), 256, 0, static_cast<cudaStream_t>(stream)>>>(e, ids, rank, out);
+    return sar_after_launch();
+}
+
+sar_status sar_permute_rows(int64_t n, int64_t row_bytes, const int32_t *index, const void *in, void *out, void *stream) {
+    if (n < 0 || row_bytes < 1 || (n > 0 && (!index || !in || !out))) return SAR_ERR_INVALID_ARG;
+    if (in == out) return SAR_ERR_INVALID_ARG;
+    if (n == 0) return SAR_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (row_bytes % 16 == 0 && sar_aligned(in, 16) && sar_aligned(out, 16)) {
+        const long long w = row_bytes / 16;
+        permute_rows_kernel<uint4><<<nblk(n * w), 256, 0, st>>>(n, w, index, static_cast<const uint4 *>(in), static_cast<uint4 *>(out));
+    } else if (row_bytes % 4 == 0 && sar_aligned(in, 4) && sar_aligned(out, 4)) {
+        const long long w = row_bytes / 4;
+        permute_rows_kernel<uint32_t><<<nblk(n * w), 256, 0, st>>>(n, w, index, static_cast<const uint32_t *>(in), static_cast<uint32_t *>(out));
+    } else {
+        permute_rows_kernel<uint8_t><<<nblk(n * row_bytes), 256, 0, st>>>(n, row_bytes, index, static_cast<const uint8_t *>(in), static_cast<uint8_t *>(out));
+    }
+    return sar_after_launch();
 }
 
 }  // extern "C"
