@@ -99,6 +99,8 @@ class CudaGatBackend:
 
     def fwd_step(self, q: int, feat_q: torch.Tensor, er_q: torch.Tensor, first: bool, last: bool):
         flags = (B.SAR_FIRST if first else 0) | (B.SAR_LAST if last else 0)
+        if last and self.k > 1:   # the complete float32 numerator stays in acc: the row dot of the backward pass
+            flags |= B.SAR_KEEP_NUMERATOR   # is formed from it, not from the rounded out
         B.sar_gat_fwd(self.parts[q], feat_q, self.el, er_q, self.H, self.F, self.slope, flags, self.acc, self.m, self.d,
                       self.out, self.ws)
 
@@ -108,8 +110,8 @@ class CudaGatBackend:
     def bwd_begin(self, gout: torch.Tensor):
         self.gout = gout
         self.del_ = torch.empty((self.rows, self.H), dtype=torch.float32, device=self.dev)
-        if self.k > 1:  # the row dot D = <gout, out> every partition's step needs
-            B.sar_gat_bwd_prepare(self.rows, self.H, self.F, self.out, False, gout, self.el, self.m, self.d, None, self.ws)
+        if self.k > 1:  # the row dot D = <gout, numerator> / d every partition's step needs
+            B.sar_gat_bwd_prepare(self.rows, self.H, self.F, self.acc, True, gout, self.el, self.m, self.d, None, self.ws)
 
     def bwd_step(self, q: int, feat_q: torch.Tensor, er_q: torch.Tensor, first: bool, last: bool):
         flags = (B.SAR_FIRST if first else 0) | (B.SAR_LAST if last else 0)

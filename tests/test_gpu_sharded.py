@@ -57,8 +57,10 @@ def test_sharded_layer_on_the_gpu_equals_the_whole_graph(K, dt):
         allclose_report(cat(0), f.out, 2e-2, 2e-2 * rms(f.out), "out")
         # K bf16 contributions per source are rounded before they travel: a few bf16 ulps of the largest term
         allclose_report(cat(3), b.dfeat, 4e-2, 4e-2 * rms(b.dfeat), "dfeat")
-        allclose_report(cat(4), b.del_, 2e-2, 0.1 * rms(b.del_), "del")   # D = <gout, out> from a bf16 out
-        allclose_report(cat(5), b.der, 2e-2, 0.1 * rms(b.der), "der")
+        # float32 arrays computed in float32 from inputs the oracle shares exactly (the row dot comes from the float32
+        # numerator the last forward step leaves behind, not from the rounded out)
+        allclose_report(cat(4), b.del_, 1e-4, 1e-5 * rms(b.del_), "del")
+        allclose_report(cat(5), b.der, 1e-4, 1e-5 * rms(b.der), "der")
     else:
         allclose_report(cat(0), f.out, 1e-5, 1e-6, "out")
         allclose_report(cat(3), b.dfeat, 1e-4, 1e-5 * rms(b.dfeat), "dfeat")
