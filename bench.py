@@ -465,7 +465,16 @@ def schedule_entry(st: AggStack, schedule, r, steps, peak):
         "step_frac_of_roofline": L * bytes_layer_fwd_bwd(n, e, H, F, b) / (r["ms_per_step"] * 1e-3) / 1e9 / peak,
     }
     if schedule == "sequential":
-        entry["state_bytes_per_step"] = state_bytes_sequential(n, H, F, K, L)
+        # what the forward calls really move: the first call writes every row's state, a middle call reads and writes
+        # the rows that have edges in its partition (the kernel skips the others), the last call reads every row's
+        entry["state_bytes_upper_bound"] = state_bytes_sequential(n, H, F, K, L)
+        if st.g.parts and K > 1:
+            touched = [int(((p_.indptr[1:] - p_.indptr[:-1]) > 0).sum().item()) for p_ in st.g.parts[1:-1]]
+            per = H * F * 4 + 2 * H * 4
+            entry["state_bytes_per_step"] = L * per * (2 * n + 2 * sum(touched))
+            entry["rows_with_edges_per_middle_partition"] = sum(touched) / max(len(touched), 1) / n
+        else:
+            entry["state_bytes_per_step"] = entry["state_bytes_upper_bound"]
         entry["calls"] = f"{K} x sar_gat_fwd, sar_gat_bwd_prepare + {K} x sar_gat_bwd per layer"
     else:
         entry["calls"] = "sar_gat_fwd_fused, sar_gat_bwd_fused per layer (one walk over the un-split graph)"
