@@ -313,6 +313,17 @@ def test_scores_far_above_a_rows_first_score(H, F, dtype):
     allclose_report(der.cpu().numpy(), b.der, 1e-4, 5e-4 * max(rms(b.der), 1.0), "der[far]")
 
 
+@pytest.mark.parametrize("slope", [0.0, 0.01, 1.0, -0.5])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_other_slopes(slope, dtype):
+    """Slope 0 (ReLU scores: every non-positive score is 0), 1 (the activation is the identity and `el` drops out of the
+    softmax), a small positive one, and a negative one (not monotone: the whole-graph calls then take the general kernel,
+    whose row max is a max over the scores themselves)."""
+    n, src, dst = hub_graph(n=3000, e=40000, d_max=700.0, seed=33)
+    p = Problem(n, src, dst, 4, 32, 5, dtype=dtype)
+    _full_check(p, dtype, slope=slope)
+
+
 def test_degenerate_graphs():
     # no edges at all
     n = 37
