@@ -631,8 +631,7 @@ def make_glue_step(args, st: AggStack):
 
             def step():
                 for l in range(L):
-                    B.sar_linear(flat(hs[l]), Ws[l], flat(zs[l]), lws)
-                    B.sar_gat_project(zs[l], a_ls[l], a_rs[l], els[l], ers[l], 0)
+                    B.sar_linear_project(flat(hs[l]), Ws[l], a_ls[l], a_rs[l], flat(zs[l]), els[l], ers[l], lws)
                     B.sar_gat_fwd_fused(g.whole, g.bounds, zs[l], els[l], ers[l], H, F, cfg.slope, ms[l], ds[l],
                                         feats[l + 1], ws)
                     if l + 1 < L:
@@ -661,8 +660,7 @@ def make_glue_step(args, st: AggStack):
             for l in range(L):
                 if l > 0:
                     B.sar_relu(feats[l])
-                B.sar_linear(flat(feats[l]), Ws[l], flat(zs[l]), lws)
-                B.sar_gat_project(zs[l], a_ls[l], a_rs[l], els[l], ers[l], 0)
+                B.sar_linear_project(flat(feats[l]), Ws[l], a_ls[l], a_rs[l], flat(zs[l]), els[l], ers[l], lws)
                 B.sar_gat_fwd_fused(g.whole, g.bounds, zs[l], els[l], ers[l], H, F, cfg.slope, ms[l], ds[l],
                                     feats[l + 1], ws)
             B.sar_relu(feats[L])

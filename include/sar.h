@@ -400,6 +400,14 @@ SAR_API sar_status sar_round_to(int64_t n_elems, sar_dtype t, const float *acc, 
  *   sar_linear             z[n, d_out]  = h[n, d_in] W[d_in, d_out]          (bf16 out)
  *   sar_linear_accumulate  z[n, d_out] += h[n, d_in] W[d_in, d_out]          (z read and written, bf16: the sum
  *                          over relations of Appendix A's layer, one call per relation)
+ *   sar_linear_project     z = h W as sar_linear with d_out = H F, and in the same kernel the two halves of Eq. 3's
+ *                          a^T (z_i || z_j): el[i,h] = <z[i,h,:], a_l[h,:]>, er[i,h] = <z[i,h,:], a_r[h,:]> taken of
+ *                          the bf16-rounded z while the accumulator tile leaves tensor memory (what sar_linear
+ *                          followed by sar_gat_project computes, without reading z back).  a_l, a_r [H,F] and el, er
+ *                          [n,H] float32.  F must be a multiple of 8 that divides 128 (a head may not straddle the
+ *                          128-column tiles), else SAR_ERR_UNSUPPORTED.  flag (DEVICE int, may be NULL) is set to 1
+ *                          if the epilogue's thread layout does not give every row to one thread (el, er are then
+ *                          not written for the rows concerned); the library's tests check that it stays 0.
  *   sar_linear_bwd_input   dh[n, d_in]  = dz[n, d_out] W^T                   (bf16 out)
  *   sar_linear_bwd_weight  dw[d_in, d_out] = h^T dz                          (float32 out; the n-long
  *                          contraction is cut across the SMs and the partial tiles are reduced in the scratch)
@@ -408,6 +416,9 @@ SAR_API sar_status sar_round_to(int64_t n_elems, sar_dtype t, const float *acc, 
  * all of these calls.  n = 0 is allowed (dw is then written as zeros).
  * ------------------------------------------------------------------------------------------- */
 SAR_API size_t sar_linear_workspace_bytes(int64_t n, int32_t d_in, int32_t d_out);
+SAR_API sar_status sar_linear_project(int64_t n, int32_t d_in, int32_t H, int32_t F, sar_dtype t, const void *h,
+                                      const void *w, const float *a_l, const float *a_r, void *z, float *el, float *er,
+                                      int32_t *flag, void *workspace, size_t workspace_bytes, void *stream);
 SAR_API sar_status sar_linear(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *h, const void *w,
                               void *z, void *workspace, size_t workspace_bytes, void *stream);
 SAR_API sar_status sar_linear_accumulate(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *h,

@@ -35,7 +35,7 @@ EXPORTS = [
     "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd", "sar_axpby", "sar_bn_rstd", "sar_accumulate", "sar_round_to", "sar_bn_apply_act",
     "sar_bn_bwd_stats_act", "sar_bn_bwd_apply_act", "sar_csc_slice_indptr",
     "sar_gat_storing_workspace_bytes", "sar_gat_fwd_storing", "sar_gat_bwd_storing", "sar_bn_combine_moments",
-    "sar_bn_combine_sums", "sar_degree_order_workspace_bytes", "sar_degree_order", "sar_relabel", "sar_permute_rows",
+    "sar_bn_combine_sums", "sar_degree_order_workspace_bytes", "sar_degree_order", "sar_relabel", "sar_permute_rows", "sar_linear_project",
 ]
 
 
@@ -639,6 +639,21 @@ def sar_linear(h: torch.Tensor, w: torch.Tensor, z: torch.Tensor, workspace: tor
     ws, wb = _ws(workspace)
     _check("sar_linear", lib().sar_linear(c_int64(n), c_int32(d_in), c_int32(d_out), ctypes.c_int(_dtype(h)), _ptr(h),
                                           _ptr(w), _ptr(z), ws, wb, _stream()))
+
+
+def sar_linear_project(h: torch.Tensor, w: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, z: torch.Tensor,
+                       el: torch.Tensor, er: torch.Tensor, workspace: torch.Tensor,
+                       flag: Optional[torch.Tensor] = None) -> None:
+    """z[n,H,F] = h W and el, er [n,H] = <z, a_l>, <z, a_r> in one kernel."""
+    n, d_in = h.shape
+    H, F = a_l.shape
+    assert w.shape == (d_in, H * F) and z.numel() == n * H * F and el.shape == (n, H) and er.shape == (n, H)
+    assert a_l.dtype == torch.float32 and a_r.dtype == torch.float32 and el.dtype == torch.float32
+    assert flag is None or flag.dtype == torch.int32
+    ws, wb = _ws(workspace)
+    _check("sar_linear_project", lib().sar_linear_project(c_int64(n), c_int32(d_in), c_int32(H), c_int32(F),
+                                                          ctypes.c_int(_dtype(h)), _ptr(h), _ptr(w), _ptr(a_l), _ptr(a_r),
+                                                          _ptr(z), _ptr(el), _ptr(er), _ptr(flag), ws, wb, _stream()))
 
 
 def sar_linear_accumulate(h: torch.Tensor, w: torch.Tensor, z: torch.Tensor, workspace: torch.Tensor) -> None:

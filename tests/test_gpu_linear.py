@@ -38,6 +38,35 @@ def test_projection_forward_and_backward(d_in, d_out, n):
     allclose_report(_np(dw), want_dw, 1e-4, 1e-5 * max(1.0, float(np.sqrt(n))), "dw")
 
 
+@pytest.mark.parametrize("d_in,H,F", [(128, 4, 32), (64, 8, 32), (128, 2, 64), (40, 4, 16), (64, 1, 128), (128, 16, 8)])
+@pytest.mark.parametrize("n", [1, 100, 4097, 300001])
+def test_projection_with_scores_in_the_epilogue(d_in, H, F, n):
+    """sar_linear_project = sar_linear followed by sar_gat_project, in one kernel: z bit for bit, el / er up to the
+    order of the F float32 additions; both against the oracle's projection of the bf16-rounded z as well."""
+    from paper_2111_06483_b200 import binding as B
+    d_out = H * F
+    h = _normal((n, d_in), 93, 1).to(torch.bfloat16).cuda()
+    w = (_normal((d_in, d_out), 93, 2) / d_in ** 0.5).to(torch.bfloat16).cuda()
+    a_l = (_normal((H, F), 93, 4) / F ** 0.5).cuda()
+    a_r = (_normal((H, F), 93, 5) / F ** 0.5).cuda()
+    ws = torch.empty(B.sar_linear_workspace_bytes(n, d_in, d_out), dtype=torch.uint8, device="cuda")
+    z0 = torch.empty((n, d_out), dtype=torch.bfloat16, device="cuda")
+    B.sar_linear(h, w, z0, ws)
+    el0, er0 = torch.empty((n, H), device="cuda"), torch.empty((n, H), device="cuda")
+    B.sar_gat_project(z0.view(n, H, F), a_l, a_r, el0, er0)
+    z = torch.full((n, d_out), float("nan"), dtype=torch.bfloat16, device="cuda")
+    el = torch.full((n, H), float("nan"), device="cuda")
+    er = torch.full((n, H), float("nan"), device="cuda")
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    B.sar_linear_project(h, w, a_l, a_r, z, el, er, ws, flag)
+    assert int(flag.item()) == 0          # every row's elements sit in one thread of the epilogue
+    assert torch.equal(z, z0)
+    want_el, want_er = oracle.project(_np(z0).reshape(n, H, F), _np(a_l), _np(a_r))
+    for got, ref, want, what in ((el, el0, want_el, "el"), (er, er0, want_er, "er")):
+        allclose_report(_np(got), want, 1e-5, 1e-6 * F ** 0.5, what + " vs oracle")
+        allclose_report(_np(got), _np(ref), 1e-5, 1e-6 * F ** 0.5, what + " vs the two-call path")
+
+
 def test_projection_rejects_what_it_cannot_do():
     from paper_2111_06483_b200 import binding as B
     h = torch.zeros((16, 12), dtype=torch.bfloat16, device="cuda")
