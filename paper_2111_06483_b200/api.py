@@ -378,10 +378,13 @@ def full_layer_forward(g: Graph, h: torch.Tensor, W: torch.Tensor, a_l: torch.Te
         B.sar_relu(h)
     z = torch.empty((n, H, F), dtype=h.dtype, device=h.device)
     ws = _workspace(B.sar_linear_workspace_bytes(n, h.shape[1], H * F), h.device)
-    B.sar_linear(h, W, z.view(n, H * F), ws)
     el = torch.empty((n, H), dtype=torch.float32, device=h.device)
     er = torch.empty_like(el)
-    B.sar_gat_project(z, a_l, a_r, el, er, 0)
+    if F % 8 == 0 and 128 % F == 0:   # the scores leave the projection's epilogue
+        B.sar_linear_project(h, W, a_l, a_r, z.view(n, H * F), el, er, ws)
+    else:
+        B.sar_linear(h, W, z.view(n, H * F), ws)
+        B.sar_gat_project(z, a_l, a_r, el, er, 0)
     out, m, d = gat_forward(g, z, el, er, slope)
     return out, (z, el, er, m, d)
 
