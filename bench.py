@@ -657,13 +657,11 @@ def make_glue_step(args, st: AggStack):
             return step
 
         def step_plain():
-            for l in range(L):
-                if l > 0:
-                    B.sar_relu(feats[l])
+            relu_flags = B.SAR_FIRST | B.SAR_LAST | B.SAR_RELU_OUT
+            for l in range(L):   # the ReLU that closes a layer is applied where its aggregate is finalised
                 B.sar_linear_project(flat(feats[l]), Ws[l], a_ls[l], a_rs[l], flat(zs[l]), els[l], ers[l], lws)
-                B.sar_gat_fwd_fused(g.whole, g.bounds, zs[l], els[l], ers[l], H, F, cfg.slope, ms[l], ds[l],
-                                    feats[l + 1], ws)
-            B.sar_relu(feats[L])
+                B.sar_gat_fwd(g.whole, zs[l], els[l], ers[l], H, F, cfg.slope, relu_flags, None, ms[l], ds[l],
+                              feats[l + 1], ws)
             gin = gout
             B.sar_relu_bwd(feats[L], gin)  # masks gout in place on the first pass; the same mask every step
             for l in reversed(range(L)):

@@ -74,6 +74,7 @@ typedef enum { SAR_F32 = 0, SAR_BF16 = 1 } sar_dtype;
 #define SAR_LAST 2u  /* last partition: normalise and write the final result                 */
 #define SAR_MEAN 4u  /* sar_spmm_agg with SAR_LAST: divide by `deg_total`                    */
 #define SAR_KEEP_NUMERATOR 8u /* sar_gat_fwd with SAR_LAST: also leave the complete numerator in acc */
+#define SAR_RELU_OUT 16u      /* sar_gat_fwd with SAR_LAST: out = max(acc/d, 0), the f_node of Algorithm 1 as a ReLU */
 
 #define SAR_MAX_HEADS 16
 #define SAR_MAX_PARTS 64
@@ -239,6 +240,9 @@ SAR_API size_t sar_gat_workspace_bytes(const sar_part *g, int32_t H, int32_t F, 
  *   SAR_KEEP_NUMERATOR together with SAR_LAST also writes the complete float32 numerator to acc (which
  *   must then be given), for sar_gat_bwd_prepare's acc_is_numerator mode: the row dot of the
  *   per-partition backward pass is then formed from float32 values instead of a rounded bf16 out.
+ *   SAR_RELU_OUT together with SAR_LAST writes out = max(acc/d, 0) (NaN -> 0): the ReLU that closes the layer
+ *   (Algorithm 1 applies f_node to the finished aggregate) without a pass of its own; m, d and a kept
+ *   numerator are those of the aggregate before the ReLU.
  *   Destinations without edges in this partition are skipped unless a flag forces a write. */
 SAR_API sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, const float *er_q, int32_t H,
                        int32_t F, sar_dtype t, float slope, uint32_t flags, float *acc, float *m, float *d,

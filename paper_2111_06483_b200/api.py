@@ -185,12 +185,14 @@ def gat_workspace(part: B.Part, H: int, F: int, dtype: torch.dtype) -> torch.Ten
 
 
 def gat_forward(g: Graph, feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor, slope: float,
-                workspace: Optional[torch.Tensor] = None, mode: str = "fused", keep_numerator: bool = False):
+                workspace: Optional[torch.Tensor] = None, mode: str = "fused", keep_numerator: bool = False,
+                relu_out: bool = False):
     """Forward over the K partitions.  mode "fused": one row-stationary walk over the un-split graph, the
     partitions being slices of the arrays (sar_gat_fwd_fused);
     mode "stateful": K calls of sar_gat_fwd with the running state in global memory (Algorithm 1).
     keep_numerator (stateful mode): returns (out, m, d, acc) with the complete float32 numerator in acc,
-    which gat_backward can take in place of `out` for the row dot."""
+    which gat_backward can take in place of `out` for the row dot.
+    relu_out: out = max(out, 0), the ReLU that closes the layer, applied where the aggregate is finalised."""
     n, H, F = feat.shape
     dev = feat.device
     m = torch.empty((g.n, H), dtype=torch.float32, device=dev)
@@ -198,7 +200,10 @@ def gat_forward(g: Graph, feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor
     out = torch.empty((g.n, H, F), dtype=feat.dtype, device=dev)
     if mode == "fused":
         ws = workspace if workspace is not None else gat_workspace(g.whole, H, F, feat.dtype)
-        B.sar_gat_fwd_fused(g.whole, g.bounds, feat, el, er, H, F, slope, m, d, out, ws)
+        if relu_out:   # the un-split graph as one partition holding all sources
+            B.sar_gat_fwd(g.whole, feat, el, er, H, F, slope, B.SAR_FIRST | B.SAR_LAST | B.SAR_RELU_OUT, None, m, d, out, ws)
+        else:
+            B.sar_gat_fwd_fused(g.whole, g.bounds, feat, el, er, H, F, slope, m, d, out, ws)
         return out, m, d
     assert g.parts, "stateful mode needs Graph.from_coo(..., build_parts=True)"
     acc = torch.empty((g.n, H, F), dtype=torch.float32, device=dev) if (g.k > 1 or keep_numerator) else None
@@ -206,6 +211,8 @@ def gat_forward(g: Graph, feat: torch.Tensor, el: torch.Tensor, er: torch.Tensor
         flags = (B.SAR_FIRST if q == 0 else 0) | (B.SAR_LAST if q == g.k - 1 else 0)
         if keep_numerator and q == g.k - 1:
             flags |= B.SAR_KEEP_NUMERATOR
+        if relu_out and q == g.k - 1:
+            flags |= B.SAR_RELU_OUT
         ws = gat_workspace(part, H, F, feat.dtype)
         s0, s1 = g.bounds[q], g.bounds[q + 1]
         B.sar_gat_fwd(part, feat[s0:s1], el, er[s0:s1], H, F, slope, flags, acc, m, d, out, ws)

@@ -19,7 +19,7 @@ LIB_PATH = os.path.join(_PKG, "libsar.so")
 
 SAR_OK = 0
 SAR_F32, SAR_BF16 = 0, 1
-SAR_FIRST, SAR_LAST, SAR_MEAN, SAR_KEEP_NUMERATOR = 1, 2, 4, 8
+SAR_FIRST, SAR_LAST, SAR_MEAN, SAR_KEEP_NUMERATOR, SAR_RELU_OUT = 1, 2, 4, 8, 16
 SAR_MAX_PARTS = 64
 
 EXPORTS = [

@@ -124,7 +124,7 @@ static sar_status launch_span(SpanArgs a, long long nnz, const char *name, const
     const long long spans = (a.n_rows + a.R - 1) / a.R;
     if (spans > 0) {
         const unsigned blocks = (unsigned)((spans + kSpanWarps - 1) / kSpanWarps);
-        if ((a.flags & SAR_FIRST) && (a.flags & SAR_LAST) && !(a.flags & SAR_KEEP_NUMERATOR)) {  // the epilogue's flag tests decided at compile time
+        if ((a.flags & SAR_FIRST) && (a.flags & SAR_LAST) && !(a.flags & (SAR_KEEP_NUMERATOR | SAR_RELU_OUT))) {  // the epilogue's flag tests decided at compile time
             if (geo) {
                 auto whole = span_kernel<T, G, V, S, MODE, CAP, MINB, 1, kGeo>;
                 SAR_TRY(ensure_smem(whole, smem));
@@ -212,9 +212,9 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
                        int32_t F, sar_dtype t, float slope, uint32_t flags, float *acc, float *m, float *d,
                        void *out, void *workspace, size_t workspace_bytes, void *stream) {
     SAR_TRY(check_part(g, false));
-    if (flags & ~(SAR_FIRST | SAR_LAST | SAR_KEEP_NUMERATOR)) return SAR_ERR_INVALID_ARG;
+    if (flags & ~(SAR_FIRST | SAR_LAST | SAR_KEEP_NUMERATOR | SAR_RELU_OUT)) return SAR_ERR_INVALID_ARG;
     const bool first = flags & SAR_FIRST, last = flags & SAR_LAST;
-    if ((flags & SAR_KEEP_NUMERATOR) && !last) return SAR_ERR_INVALID_ARG;
+    if ((flags & (SAR_KEEP_NUMERATOR | SAR_RELU_OUT)) && !last) return SAR_ERR_INVALID_ARG;
     if (!el || !m || !d) return SAR_ERR_INVALID_ARG;
     if (g->n_src > 0 && (!feat_q || !er_q)) return SAR_ERR_INVALID_ARG;
     if (last && !out) return SAR_ERR_INVALID_ARG;
@@ -302,6 +302,7 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
         la.m_out = m;
         la.d_out = d;
         la.out = out;
+        la.relu = (flags & SAR_RELU_OUT) ? 1 : 0;
         la.slope = slope;
         la.sp = ma.sp;
         la.sp.threshold = g->split->threshold;

@@ -112,6 +112,10 @@ __global__ void __launch_bounds__(kThreads) gat_fwd_merge_kernel(const FwdArgs a
             const float inv = dv[v] > 0.f ? 1.f / dv[v] : 0.f;
 #pragma unroll
             for (int e = 0; e < EPV; ++e) acc[v][e] *= inv;
+            if (a.flags & SAR_RELU_OUT) {
+#pragma unroll
+                for (int e = 0; e < EPV; ++e) acc[v][e] = fmaxf(acc[v][e], 0.f);
+            }
         }
         store_row_vec<T, G, V>(a.out, row, a.g.n_vec, id.gl, vg.vok, acc);
     } else {

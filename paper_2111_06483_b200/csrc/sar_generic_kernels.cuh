@@ -67,8 +67,10 @@ __global__ void gat_fwd_generic(const GenericArgs a) {
             const float w = expf(leaky(el_i + a.er[j * a.H + h], a.slope, gr) - Mn);
             acc = fmaf(w, Elem<T>::load1(feat + j * HF + (long long)h * a.F + f), acc);
         }
-        if (last)
-            Elem<T>::store1(reinterpret_cast<T *>(a.out) + o, dsum > 0.f ? acc / dsum : 0.f);
+        if (last) {
+            const float y = dsum > 0.f ? acc / dsum : 0.f;
+            Elem<T>::store1(reinterpret_cast<T *>(a.out) + o, (a.flags & SAR_RELU_OUT) ? fmaxf(y, 0.f) : y);
+        }
         if (!last || (a.flags & SAR_KEEP_NUMERATOR)) a.acc[o] = acc;
     }
     a.m[idx] = Mn;

@@ -22,6 +22,7 @@ struct LeanArgs {
     float slope;
     SplitArgs sp;
     int R;                   // rows per span (<= kMaxSpanRows)
+    int relu;                // forward: out = max(out, 0)
 };
 
 struct LeanSrcArgs {

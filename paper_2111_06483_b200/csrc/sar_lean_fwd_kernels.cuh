@@ -471,6 +471,10 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
                                         const f32x2 y = fma2(pacc0[v][t], i2, zero2());
                                         unpack2(y, acc0[2 * t], acc0[2 * t + 1]);
                                     }
+                                    if (a.relu) {
+#pragma unroll
+                                        for (int e = 0; e < EPV; ++e) acc0[e] = fmaxf(acc0[e], 0.f);
+                                    }
                                     rp[v * G] = Elem<T>::pack(acc0);
                                     if ((gl % VPH) == 0) sts_f32(sout_s + (unsigned)((ri * H + hv[v]) * 4), sv[v]);
                                 }

@@ -830,6 +830,10 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                                 const float inv = sv[v] > 0.f ? __fdividef(1.f, sv[v]) : 0.f;
 #pragma unroll
                                 for (int e = 0; e < EPV; ++e) acc0[v][e] *= inv;
+                                if (flags_ & SAR_RELU_OUT) {
+#pragma unroll
+                                    for (int e = 0; e < EPV; ++e) acc0[v][e] = fmaxf(acc0[v][e], 0.f);
+                                }
                             }
                             store_row_vec<T, G, V>(a.out, row, n_vec, gl, vok, acc0);
                         } else {

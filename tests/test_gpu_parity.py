@@ -324,6 +324,23 @@ def test_other_slopes(slope, dtype):
     _full_check(p, dtype, slope=slope)
 
 
+@pytest.mark.parametrize("H,F,dtype", [(4, 32, "bf16"), (4, 32, "f32"), (8, 32, "bf16"), (3, 5, "f32"), (2, 7, "bf16")])
+@pytest.mark.parametrize("mode", ["fused", "stateful"])
+def test_relu_in_the_output_epilogue(H, F, dtype, mode):
+    """SAR_RELU_OUT: out = max(aggregate, 0) wherever the aggregate is finalised (the rows launch, the merge of long
+    rows, the call-by-call path, the scalar kernels); m and d stay those of the aggregate.  Equal to sar_relu applied to
+    the plain output bit for bit (the ReLU of a rounded value is the rounded ReLU)."""
+    n, src, dst = hub_graph(n=3000, e=40000, d_max=700.0, seed=41)
+    p = Problem(n, src, dst, H, F, 6, dtype=dtype, k=3, build_parts=True)
+    f = p.oracle_fwd()
+    d = p.dev
+    plain = api.gat_forward(p.graph, d["feat"], d["el"], d["er"], 0.2, mode=mode)
+    fused = api.gat_forward(p.graph, d["feat"], d["el"], d["er"], 0.2, mode=mode, relu_out=True)
+    assert torch.equal(fused[0], torch.clamp_min(plain[0], 0))
+    assert torch.equal(fused[1], plain[1]) and torch.equal(fused[2], plain[2])
+    check_out(fused[0], np.maximum(f.out, 0.0), dtype, f"relu(out)[{mode}]")
+
+
 def test_degenerate_graphs():
     # no edges at all
     n = 37
