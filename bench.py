@@ -670,9 +670,10 @@ def make_glue_step(args, st: AggStack):
                                         gbuf[0], dels[l], ders[l], ws)
                 B.sar_gat_project_bwd(zs[l], a_ls[l], a_rs[l], dels[l], ders[l], gbuf[0], da_l, da_r, pws, 0)
                 B.sar_linear_bwd_weight(flat(feats[l]), flat(gbuf[0]), dW, lws)
-                B.sar_linear_bwd_input(flat(gbuf[0]), Ws[l], flat(gbuf[1]), lws)
-                if l > 0:
-                    B.sar_relu_bwd(feats[l], gbuf[1])
+                if l > 0:   # the backward of the ReLU that produced this layer's input, in the GEMM's epilogue
+                    B.sar_linear_bwd_input_relu(flat(gbuf[0]), Ws[l], flat(feats[l]), flat(gbuf[1]), lws)
+                else:
+                    B.sar_linear_bwd_input(flat(gbuf[0]), Ws[l], flat(gbuf[1]), lws)
                 gin = gbuf[1]
         return step_plain
 

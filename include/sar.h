@@ -413,6 +413,10 @@ SAR_API sar_status sar_round_to(int64_t n_elems, sar_dtype t, const float *acc, 
  *                          if the epilogue's thread layout does not give every row to one thread (el, er are then
  *                          not written for the rows concerned); the library's tests check that it stays 0.
  *   sar_linear_bwd_input   dh[n, d_in]  = dz[n, d_out] W^T                   (bf16 out)
+ *   sar_linear_bwd_input_relu  the same followed by the backward of the ReLU that produced the layer's input h:
+ *                          dh[i, c] = 0 where y[i, c] <= 0, y [n, d_in] (bf16) being that ReLU's output (= h); the
+ *                          mask is applied in the GEMM's epilogue (what sar_relu_bwd(y, dh) would do in a pass of
+ *                          its own)
  *   sar_linear_bwd_weight  dw[d_in, d_out] = h^T dz                          (float32 out; the n-long
  *                          contraction is cut across the SMs and the partial tiles are reduced in the scratch)
  * All arrays row-major DEVICE memory, 16-byte aligned; t must be SAR_BF16 and d_in, d_out multiples of 8
@@ -420,6 +424,9 @@ SAR_API sar_status sar_round_to(int64_t n_elems, sar_dtype t, const float *acc, 
  * all of these calls.  n = 0 is allowed (dw is then written as zeros).
  * ------------------------------------------------------------------------------------------- */
 SAR_API size_t sar_linear_workspace_bytes(int64_t n, int32_t d_in, int32_t d_out);
+SAR_API sar_status sar_linear_bwd_input_relu(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *dz,
+                                             const void *w, const void *y, void *dh, void *workspace,
+                                             size_t workspace_bytes, void *stream);
 SAR_API sar_status sar_linear_project(int64_t n, int32_t d_in, int32_t H, int32_t F, sar_dtype t, const void *h,
                                       const void *w, const float *a_l, const float *a_r, void *z, float *el, float *er,
                                       int32_t *flag, void *workspace, size_t workspace_bytes, void *stream);

@@ -35,7 +35,7 @@ EXPORTS = [
     "sar_linear_bwd_weight", "sar_linear_accumulate", "sar_degree_scale", "sar_rgcn_basis", "sar_rgcn_basis_bwd", "sar_axpby", "sar_bn_rstd", "sar_accumulate", "sar_round_to", "sar_bn_apply_act",
     "sar_bn_bwd_stats_act", "sar_bn_bwd_apply_act", "sar_csc_slice_indptr",
     "sar_gat_storing_workspace_bytes", "sar_gat_fwd_storing", "sar_gat_bwd_storing", "sar_bn_combine_moments",
-    "sar_bn_combine_sums", "sar_degree_order_workspace_bytes", "sar_degree_order", "sar_relabel", "sar_permute_rows", "sar_linear_project",
+    "sar_bn_combine_sums", "sar_degree_order_workspace_bytes", "sar_degree_order", "sar_relabel", "sar_permute_rows", "sar_linear_project", "sar_linear_bwd_input_relu",
 ]
 
 
@@ -639,6 +639,18 @@ def sar_linear(h: torch.Tensor, w: torch.Tensor, z: torch.Tensor, workspace: tor
     ws, wb = _ws(workspace)
     _check("sar_linear", lib().sar_linear(c_int64(n), c_int32(d_in), c_int32(d_out), ctypes.c_int(_dtype(h)), _ptr(h),
                                           _ptr(w), _ptr(z), ws, wb, _stream()))
+
+
+def sar_linear_bwd_input_relu(dz: torch.Tensor, w: torch.Tensor, y: torch.Tensor, dh: torch.Tensor,
+                              workspace: torch.Tensor) -> None:
+    """dh = (dz W^T) where y > 0, else 0 (y: the output of the ReLU that produced the layer's input)."""
+    n, d_out = dz.shape
+    d_in = w.shape[0]
+    assert y.shape == (n, d_in) and dh.shape == (n, d_in) and y.dtype == dz.dtype
+    ws, wb = _ws(workspace)
+    _check("sar_linear_bwd_input_relu", lib().sar_linear_bwd_input_relu(c_int64(n), c_int32(d_in), c_int32(d_out),
+                                                                        ctypes.c_int(_dtype(dz)), _ptr(dz), _ptr(w), _ptr(y),
+                                                                        _ptr(dh), ws, wb, _stream()))
 
 
 def sar_linear_project(h: torch.Tensor, w: torch.Tensor, a_l: torch.Tensor, a_r: torch.Tensor, z: torch.Tensor,

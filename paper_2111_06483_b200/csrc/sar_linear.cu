@@ -7,7 +7,9 @@
 
 #include "cutlass/cutlass.h"
 #include "cutlass/epilogue/collective/collective_builder.hpp"
+#include "cutlass/epilogue/fusion/operations.hpp"
 #include "cutlass/epilogue/fusion/sm90_visitor_load_tma_warpspecialized.hpp"
+#include "cutlass/epilogue/thread/activation.h"
 #include "cutlass/epilogue/fusion/sm90_visitor_tma_warpspecialized.hpp"
 #include "cutlass/gemm/collective/collective_builder.hpp"
 #include "cutlass/gemm/device/gemm_universal_adapter.h"
@@ -161,7 +163,25 @@ using ProjectRow = cutlass::epilogue::fusion::Sm90RowBroadcast<0, ProjectTile, f
 using ProjectFusion =
     cutlass::epilogue::fusion::Sm90EVT<ProjectVisitor, cutlass::epilogue::fusion::Sm90AccFetch, ProjectRow, ProjectRow>;
 
-template <class LayoutA, class LayoutB, class ElementOut, class Scheduler, class Fusion = void>
+// D = (A B) where y != 0, else 0: the backward of a ReLU whose output y (>= 0) is the auxiliary tile (a CUTLASS fusion
+// operation: the mask is applied while the accumulators leave tensor memory)
+template <class T>
+struct ReluMask {
+    CUTLASS_HOST_DEVICE T operator()(T g, T y) const { return y > T(0) ? g : T(0); }
+};
+template <class T, int N>
+struct ReluMask<cutlass::Array<T, N>> {
+    CUTLASS_HOST_DEVICE cutlass::Array<T, N> operator()(cutlass::Array<T, N> const &g, cutlass::Array<T, N> const &y) const {
+        cutlass::Array<T, N> r;
+        CUTLASS_PRAGMA_UNROLL
+        for (int i = 0; i < N; ++i) r[i] = y[i] > T(0) ? g[i] : T(0);
+        return r;
+    }
+};
+using MaskFusion = cutlass::epilogue::fusion::LinCombDeEltAct<cutlass::layout::RowMajor, ReluMask, cutlass::bfloat16_t, float,
+                                                              cutlass::bfloat16_t>;
+
+template <class LayoutA, class LayoutB, class ElementOut, class Scheduler, class Fusion = void, bool kEvt = !cute::is_void_v<Fusion>>
 struct LinearGemm {
     using ElementA = cutlass::bfloat16_t;
     using ElementB = cutlass::bfloat16_t;
@@ -173,7 +193,7 @@ struct LinearGemm {
     using ClusterShape = Shape<_1, _1, _1>;
     static constexpr bool kFused = !cute::is_void_v<Fusion>;
     using DefaultFusion = cutlass::epilogue::fusion::LinearCombination<ElementOut, ElementAcc, ElementOut, ElementAcc>;
-    using ElementCin = cute::conditional_t<kFused, void, ElementOut>;   // the fused epilogue reads no source tile
+    using ElementCin = cute::conditional_t<kEvt, void, ElementOut>;   // the visitor epilogue reads no source tile
     using Epilogue = typename cutlass::epilogue::collective::CollectiveBuilder<
         cutlass::arch::Sm100, cutlass::arch::OpClassTensorOp, TileShape, ClusterShape,
         cutlass::epilogue::collective::EpilogueTileAuto, ElementAcc, ElementAcc, ElementCin, LayoutC, AlignC, ElementOut,
@@ -209,6 +229,32 @@ struct LinearGemm {
                                 const ProjectVisitor::Arguments &pv, void *workspace, size_t workspace_bytes_, cudaStream_t st,
                                 const char *name) {
         auto args = arguments_fused(M, N, K, a, b, d, a_l, a_r, pv);
+        Gemm gemm;
+        if (gemm.can_implement(args) != cutlass::Status::kSuccess) return SAR_ERR_UNSUPPORTED;
+        const size_t need = Gemm::get_workspace_size(args);
+        if (need > 0 && (!workspace || workspace_bytes_ < need || !sar_aligned(workspace, 16))) return SAR_ERR_WORKSPACE;
+        if (gemm.initialize(args, workspace, st) != cutlass::Status::kSuccess) return SAR_ERR_CUDA;
+        cutlass::Status rc;
+        SAR_LAUNCH(name, st, rc = gemm.run(st));
+        if (rc != cutlass::Status::kSuccess) return SAR_ERR_CUDA;
+        return sar_after_launch();
+    }
+
+    // D = mask(A B, y): y [M, N] in the output type, row-major
+    static sar_status run_masked(int M, int N, int K, const void *a, const void *b, void *d, const void *y, void *workspace,
+                                 size_t workspace_bytes_, cudaStream_t st, const char *name) {
+        typename Gemm::Arguments args{
+            cutlass::gemm::GemmUniversalMode::kGemm,
+            {M, N, K, 1},
+            {static_cast<const ElementA *>(a), cutlass::make_cute_packed_stride(StrideA{}, cute::make_shape(M, K, 1)),
+             static_cast<const ElementB *>(b), cutlass::make_cute_packed_stride(StrideB{}, cute::make_shape(N, K, 1))},
+            {{},
+             static_cast<const ElementOut *>(d), cutlass::make_cute_packed_stride(StrideC{}, cute::make_shape(M, N, 1)),
+             static_cast<ElementOut *>(d), cutlass::make_cute_packed_stride(StrideD{}, cute::make_shape(M, N, 1))}};
+        args.epilogue.thread.alpha = 1.f;
+        args.epilogue.thread.beta = 0.f;
+        args.epilogue.thread.aux_ptr = static_cast<const ElementOut *>(y);
+        args.epilogue.thread.dAux = cutlass::make_cute_packed_stride(StrideC{}, cute::make_shape(M, N, 1));
         Gemm gemm;
         if (gemm.can_implement(args) != cutlass::Status::kSuccess) return SAR_ERR_UNSUPPORTED;
         const size_t need = Gemm::get_workspace_size(args);
@@ -259,6 +305,8 @@ using GemmForward = LinearGemm<RowMajor, RowMajor, cutlass::bfloat16_t, void>;
 using GemmForwardProject = LinearGemm<RowMajor, RowMajor, cutlass::bfloat16_t, void, ProjectFusion>;
 // dh[n, d_in] = dz[n, d_out] W^T:           A = dz, B[k, n] = W[n, k]: K contiguous
 using GemmBwdInput = LinearGemm<RowMajor, ColMajor, cutlass::bfloat16_t, void>;
+// the same followed by the backward of the ReLU that produced the layer's input
+using GemmBwdInputMasked = LinearGemm<RowMajor, ColMajor, cutlass::bfloat16_t, void, MaskFusion, false>;
 // dW[d_in, d_out] = h^T dz, K = n (millions): A[m, k] = h[k, m] (M contiguous), B = dz (N contiguous); the
 // K range is cut across the SMs by the stream-K scheduler (one 128x128 output tile would otherwise keep one SM busy)
 using GemmBwdWeight = LinearGemm<ColMajor, RowMajor, float, cutlass::gemm::StreamKScheduler>;
@@ -336,6 +384,14 @@ sar_status sar_linear_bwd_input(int64_t n, int32_t d_in, int32_t d_out, sar_dtyp
     SAR_TRY(linear_check(n, d_in, d_out, t, {dz, w, dh}));
     return GemmBwdInput::run((int)n, d_in, d_out, dz, w, dh, workspace, workspace_bytes, static_cast<cudaStream_t>(stream),
                              "linear_bwd_input");
+}
+
+sar_status sar_linear_bwd_input_relu(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *dz, const void *w,
+                                     const void *y, void *dh, void *workspace, size_t workspace_bytes, void *stream) {
+    if (n == 0 && d_in > 0 && d_out > 0) return t == SAR_BF16 ? SAR_OK : SAR_ERR_UNSUPPORTED;
+    SAR_TRY(linear_check(n, d_in, d_out, t, {dz, w, y, dh}));
+    return GemmBwdInputMasked::run_masked((int)n, d_in, d_out, dz, w, dh, y, workspace, workspace_bytes,
+                                          static_cast<cudaStream_t>(stream), "linear_bwd_input_relu");
 }
 
 sar_status sar_linear_bwd_weight(int64_t n, int32_t d_in, int32_t d_out, sar_dtype t, const void *h, const void *dz,

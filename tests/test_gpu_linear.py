@@ -67,6 +67,25 @@ def test_projection_with_scores_in_the_epilogue(d_in, H, F, n):
         allclose_report(_np(got), _np(ref), 1e-5, 1e-6 * F ** 0.5, what + " vs the two-call path")
 
 
+@pytest.mark.parametrize("d_in,d_out", [(128, 128), (64, 256), (8, 8), (40, 72)])
+@pytest.mark.parametrize("n", [1, 4097, 300001])
+def test_input_gradient_with_the_relu_mask_in_the_epilogue(d_in, d_out, n):
+    """sar_linear_bwd_input_relu = sar_linear_bwd_input followed by sar_relu_bwd, in one kernel, bit for bit."""
+    from paper_2111_06483_b200 import binding as B
+    dz = _normal((n, d_out), 95, 1).to(torch.bfloat16).cuda()
+    w = (_normal((d_in, d_out), 95, 2) / d_in ** 0.5).to(torch.bfloat16).cuda()
+    y = torch.clamp_min(_normal((n, d_in), 95, 3), 0).to(torch.bfloat16).cuda()   # a ReLU's output: about half zeros
+    ws = torch.empty(B.sar_linear_workspace_bytes(n, d_in, d_out), dtype=torch.uint8, device="cuda")
+    ref = torch.empty((n, d_in), dtype=torch.bfloat16, device="cuda")
+    B.sar_linear_bwd_input(dz, w, ref, ws)
+    B.sar_relu_bwd(y, ref)
+    got = torch.full((n, d_in), float("nan"), dtype=torch.bfloat16, device="cuda")
+    B.sar_linear_bwd_input_relu(dz, w, y, got, ws)
+    assert torch.equal(got, ref)
+    want_dh, _ = oracle.linear_bwd(np.zeros((n, d_in)), _np(w), _np(dz))
+    allclose_report(_np(got), np.where(_np(y) > 0, want_dh, 0.0), 2.0 ** -8, 2.0 ** -8 * 0.5, "masked dh")
+
+
 def test_projection_rejects_what_it_cannot_do():
     from paper_2111_06483_b200 import binding as B
     h = torch.zeros((16, 12), dtype=torch.bfloat16, device="cuda")
