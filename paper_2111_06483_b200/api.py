@@ -411,9 +411,10 @@ def full_layer_backward(g: Graph, h: torch.Tensor, W: torch.Tensor, a_l: torch.T
     dW = torch.empty((d_in, H * F), dtype=torch.float32, device=h.device)
     B.sar_linear_bwd_weight(h, dz.view(n, H * F), dW, ws)
     dh = torch.empty_like(h)
-    B.sar_linear_bwd_input(dz.view(n, H * F), W, dh, ws)
-    if relu_input:
-        B.sar_relu_bwd(h, dh)
+    if relu_input:   # the mask of the input's ReLU is applied in the GEMM's epilogue
+        B.sar_linear_bwd_input_relu(dz.view(n, H * F), W, h, dh, ws)
+    else:
+        B.sar_linear_bwd_input(dz.view(n, H * F), W, dh, ws)
     return dh, dW, da_l, da_r
 
 
