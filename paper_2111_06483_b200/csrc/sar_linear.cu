@@ -2,7 +2,7 @@
 // pass: the one dense contraction around the aggregation, run on the 5th-generation tensor cores
 // (tcgen05 MMA with accumulators in tensor memory, operands staged by TMA) through CUTLASS's sm100
 // collective templates instantiated here; bf16 operands, float32 accumulation.  Contracts are in
-// include/sar.h.  Cluster shape 1x1x1: no multicast loads.
+// include/sar.h.  Cluster shape 1x1x1: every CTA loads its own operand tiles.
 #include "sar_common.cuh"
 
 #include "cutlass/cutlass.h"
