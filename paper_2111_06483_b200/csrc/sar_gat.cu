@@ -97,6 +97,7 @@ static sar_status check_part(const sar_part *g, bool need_csc) {
 constexpr int kCapFwd = 256, kCapDst = 256, kCapSrc = 192, kCapSum = 256;
 constexpr int kCapSeg = 128;  // capacity of the segment launches (segments hold at most the plan threshold)
 constexpr int kMinBlocksFwd = 24, kMinBlocksBwd = 20;  // resident blocks per SM the register budget is cut for
+constexpr size_t kStageBytes = 16 * 1024;              // shared memory a partition step may spend on the rows' own data
 
 static int rows_per_span(long long n_rows, long long nnz, int cap) {
     const double avg = n_rows > 0 ? (double)nnz / (double)n_rows : 0.0;
@@ -121,21 +122,36 @@ static sar_status launch_span(SpanArgs a, long long nnz, const char *name, const
     constexpr int kGeo = (kIsSum || G * V >= 4) ? 1 : 0;
     const bool geo = kGeo && a.g.n_vec == G * V && (kIsSum ? a.g.H == 1 : (a.g.H == 4 && a.g.Hp == 4 && a.hvec));
     a.R = rows_per_span(a.n_rows, nnz, CAP);
+    const bool whole = (a.flags & SAR_FIRST) && (a.flags & SAR_LAST);
+    // A partition step of the destination-major pass stages the rows' output-gradient rows per chunk when that fits
+    // kStageBytes of shared memory, with fewer rows per span if need be.
+    size_t stage_bytes = 0;
+    a.stage_rows = 0;
+    if (!whole && (MODE == kBwdDst || MODE == kBwdDstGivenD)) {
+        const size_t rsb = (size_t)a.g.n_vec * 16;
+        if (rsb <= kStageBytes) {
+            if ((size_t)a.R * rsb > kStageBytes) a.R = (int)(kStageBytes / rsb);
+            a.stage_rows = a.R;
+            stage_bytes = (size_t)a.R * rsb;
+        }
+    }
     const long long spans = (a.n_rows + a.R - 1) / a.R;
     if (spans > 0) {
         const unsigned blocks = (unsigned)((spans + kSpanWarps - 1) / kSpanWarps);
-        if ((a.flags & SAR_FIRST) && (a.flags & SAR_LAST) && !(a.flags & (SAR_KEEP_NUMERATOR | SAR_RELU_OUT))) {  // the epilogue's flag tests decided at compile time
+        if (whole && !(a.flags & (SAR_KEEP_NUMERATOR | SAR_RELU_OUT))) {  // the epilogue's flag tests decided at compile time
             if (geo) {
-                auto whole = span_kernel<T, G, V, S, MODE, CAP, MINB, 1, kGeo>;
-                SAR_TRY(ensure_smem(whole, smem));
-                SAR_LAUNCH(name, st, whole<<<blocks, kSpanThreads, smem, st>>>(a));
+                auto wk = span_kernel<T, G, V, S, MODE, CAP, MINB, 1, kGeo>;
+                SAR_TRY(ensure_smem(wk, smem));
+                SAR_LAUNCH(name, st, wk<<<blocks, kSpanThreads, smem, st>>>(a));
             } else {
-                auto whole = span_kernel<T, G, V, S, MODE, CAP, MINB, 1>;
-                SAR_TRY(ensure_smem(whole, smem));
-                SAR_LAUNCH(name, st, whole<<<blocks, kSpanThreads, smem, st>>>(a));
+                auto wk = span_kernel<T, G, V, S, MODE, CAP, MINB, 1>;
+                SAR_TRY(ensure_smem(wk, smem));
+                SAR_LAUNCH(name, st, wk<<<blocks, kSpanThreads, smem, st>>>(a));
             }
         } else {
-            SAR_LAUNCH(name, st, kern<<<blocks, kSpanThreads, smem, st>>>(a));
+            const size_t smem_st = (size_t)kSpanWarps * span_layout<MODE>(a.g.Hp, V, CAP, S, 32 / G, stage_bytes).total;
+            SAR_TRY(ensure_smem(kern, smem_st));
+            SAR_LAUNCH(name, st, kern<<<blocks, kSpanThreads, smem_st, st>>>(a));
         }
         SAR_TRY(sar_after_launch());
     }

@@ -54,6 +54,7 @@ struct SpanArgs {
     int mode;                // 0: spans of R rows; 1: one long-row segment per warp
     int R;                   // rows per span (<= kMaxSpanRows)
     int hvec;                // heads are scored four at a time (H % 4 == 0 and er is 16-byte aligned)
+    int stage_rows;          // mode 0: rows whose own data is staged in shared memory per chunk (R, or 0: none)
 };
 
 // order-preserving float -> unsigned key (for shared-memory atomicMax)
@@ -133,11 +134,12 @@ struct Pairs<__nv_bfloat16> {
 
 // Shared-memory layout of one warp (byte offsets).
 struct SpanSmem {
-    size_t stage, sj, w, rowc, srb, sso, mrun, fac, scratch, total;
+    size_t stage, sj, w, rowc, srb, sso, mrun, fac, scratch, rowst, total;
 };
+constexpr int kSpanPlanes = 5;            // planes of per-(row, head) constants
 __host__ __device__ inline size_t span_align16(size_t x) { return (x + 15) & ~(size_t)15; }
 template <int MODE>
-__host__ __device__ inline SpanSmem span_layout(int Hp, int V, int cap, int stages, int epw) {
+__host__ __device__ inline SpanSmem span_layout(int Hp, int V, int cap, int stages, int epw, size_t row_stage_bytes = 0) {
     const size_t wbytes = MODE == kSum ? 0 : sizeof(typename WeightOf<MODE>::type);
     const size_t pos = (size_t)cap + (size_t)kMaxSpanRows * (epw - 1) + (size_t)stages * epw;  // padded positions
     SpanSmem L;
@@ -145,13 +147,15 @@ __host__ __device__ inline SpanSmem span_layout(int Hp, int V, int cap, int stag
     L.stage = o;   o += (size_t)stages * V * 512;                // ring of gathered slots
     L.sj = o;      o += span_align16(pos * 4);                   // column id per padded position (-1: padding)
     L.w = o;       o += span_align16(pos * Hp * wbytes);         // weight record per (position, head)
-    L.rowc = o;    o += span_align16((size_t)kMaxSpanRows * Hp * 4) * 3;  // three planes of per-(row, head) constants
+    L.rowc = o;    o += span_align16((size_t)kMaxSpanRows * Hp * 4) * kSpanPlanes;  // planes of per-(row, head) constants
     L.srb = o;     o += (size_t)(kMaxSpanRows + 1) * 4;          // local first edge of each row
     L.sso = o;     o += (size_t)(kMaxSpanRows + 1) * 4;          // first slot of each row
     L.mrun = o;    o += (size_t)Hp * 4;                          // running max of a continued row
     L.fac = o;     o += (size_t)Hp * 4;                          // its rescale factors
     o = span_align16(o);
     L.scratch = o; o += (size_t)(64 * V + 32) * 4;               // epilogue scratch
+    o = span_align16(o);
+    L.rowst = o;   o += row_stage_bytes;                         // the staged rows' own data (partition steps)
     L.total = span_align16(o);
     return L;
 }
@@ -184,7 +188,16 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
     const long long rowf = (long long)n_vec * EPV;
 
     // ---- shared memory carve-up (per warp) ----------------------------------------------------
-    const SpanSmem L = span_layout<MODE>(Hp, V, CAP, S, EPW);
+    // A partition step of the destination-major pass (a launch over the rows that is not the whole graph) stages the
+    // rows' own data - the output-gradient row, D, del so far - for a chunk at a time, with the chunk's first gathers
+    // in flight, instead of loading it around each row's end: the rows of a partition are short (most of a row's edges
+    // lie in other partitions), so a load per completed row, waited for on the spot, is a large part of such a launch.
+    // (Measured on the large workload, 16 partitions: 129 -> 108 ms per layer.  The same for the forward pass's running
+    // numerator, 512 bytes per row, costs more in resident warps than it saves: 98 -> 127 ms.)
+    constexpr bool kStageMode = MODE == kBwdDst || MODE == kBwdDstGivenD;
+    const bool staged = kStageMode && STATIC == 0 && a.mode == 0 && a.stage_rows != 0;
+    const unsigned rsb = (unsigned)n_vec * 16u;   // bytes of a staged row
+    const SpanSmem L = span_layout<MODE>(Hp, V, CAP, S, EPW, staged ? (size_t)a.stage_rows * rsb : 0);
     unsigned char *wb = smem_raw + (size_t)warp * L.total;
     uint4 *stage = reinterpret_cast<uint4 *>(wb + L.stage);  // [S][V][32]
     int *sj = reinterpret_cast<int *>(wb + L.sj);
@@ -193,6 +206,9 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
     float *sc0 = reinterpret_cast<float *>(wb + L.rowc);  // el of the row (CSR passes) / er of the row (CSC pass)
     float *sc1 = sc0 + plane;                             // forward: max key; bwd-dst: m
     float *sc2 = sc1 + plane;                             // forward: reference max; bwd-dst: 1/d
+    float *sc3 = sc2 + plane;                             // bwd-dst, staged rows: D given
+    float *sc4 = sc3 + plane;                             // bwd-dst, staged rows: del so far
+    const unsigned rowst_s = (unsigned)__cvta_generic_to_shared(wb + L.rowst);
     int *srb = reinterpret_cast<int *>(wb + L.srb);
     int *sso = reinterpret_cast<int *>(wb + L.sso);
     float *smrun = reinterpret_cast<float *>(wb + L.mrun);
@@ -353,40 +369,67 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
         const int nslots = sso[nr];
         const int npos = nslots * EPW;
 
+        // ---- the own data of the chunk's rows that will be finalised (a partition step, see `staged`): the copies join
+        // the commit group of the score terms below --------------------------------------------------------------------
+        const bool staged_now = staged && !piece;
+        if constexpr (kStageMode) {
+            if (staged_now) {
+                const int i = lane - r;
+                unsigned todo = __ballot_sync(0xffffffffu, i >= 0 && i < nr && (deg_l > 0 || write_empty)) >> r;
+                const unsigned char *base = reinterpret_cast<const unsigned char *>(a.rowvec);
+                while (todo) {
+                    const int i2 = __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    const unsigned char *src = base + (size_t)(row0 + r + i2) * rsb;
+                    for (unsigned x = (unsigned)lane * 16u; x < rsb; x += 512u) cp_async16_s(rowst_s + (unsigned)i2 * rsb + x, src + x, 16);
+                }
+            }
+        }
+
         // Every stage below first ISSUES all of its global loads into registers and only then
         // consumes them: a warp executes in order, so a load followed by its use inside a loop body
         // would expose one full memory latency per sweep.
         // ---- stage B: per-(row, head) constants and column ids (slot-major) -----------------------
-        auto load_consts = [&](int x, float &c0, float &c1, float &c2) {
-            c0 = 0.f;
-            c1 = __uint_as_float(kKeyNegInf);
-            c2 = 0.f;
+        auto load_consts = [&](int x, float (&c)[5]) {
+            c[0] = 0.f;
+            c[1] = __uint_as_float(kKeyNegInf);
+            c[2] = c[3] = c[4] = 0.f;
             const int i = x >> lgHp, h = x & (Hp - 1);
             if (x < nr * Hp && h < H) {
                 const long long o = (row0 + r + i) * H + h;
                 if constexpr (kFwdMode) {
-                    c0 = __ldg(a.el + o);
+                    c[0] = __ldg(a.el + o);
                 } else if constexpr (kDst) {
-                    c0 = __ldg(a.el + o);
-                    c1 = __ldg(a.m + o);
-                    c2 = __ldg(a.d + o);
+                    c[0] = __ldg(a.el + o);
+                    c[1] = __ldg(a.m + o);
+                    c[2] = __ldg(a.d + o);
+                    if (staged_now) {
+                        if constexpr (MODE == kBwdDstGivenD) c[3] = __ldg(&a.rec_in[o].w);
+                        if (!(flags_ & SAR_FIRST)) c[4] = a.del[o];   // plain load: this launch rewrites it
+                    }
                 } else {
-                    c0 = __ldg(a.er + o);
+                    c[0] = __ldg(a.er + o);
                 }
             }
         };
-        auto store_consts = [&](int x, float c0, float c1, float c2) {
+        auto store_consts = [&](int x, float (&c)[5]) {
             if (x < nr * Hp) {
-                if constexpr (kDst) c2 = c2 > 0.f ? __fdividef(1.f, c2) : 0.f;  // 1/d
-                sc0[x] = c0;
-                sc1[x] = c1;
-                sc2[x] = c2;
+                if constexpr (kDst) c[2] = c[2] > 0.f ? __fdividef(1.f, c[2]) : 0.f;  // 1/d
+                sc0[x] = c[0];
+                sc1[x] = c[1];
+                sc2[x] = c[2];
+                if constexpr (kDst) {
+                    if (staged_now) {
+                        sc3[x] = c[3];
+                        sc4[x] = c[4];
+                    }
+                }
             }
         };
-        float ca[2][3];
+        float ca[2][5];
         if constexpr (MODE != kSum && MODE != kSumW) {
-            load_consts(lane, ca[0][0], ca[0][1], ca[0][2]);
-            load_consts(lane + 32, ca[1][0], ca[1][1], ca[1][2]);
+            load_consts(lane, ca[0]);
+            load_consts(lane + 32, ca[1]);
         }
         {   // two positions per lane and sweep: both loads are issued before either is stored
             int i = 0;
@@ -408,18 +451,18 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
             for (int q = npos + lane; q < npos + S * EPW; q += 32) sj[q] = -1;  // the ring's run-out
         }
         if constexpr (MODE != kSum && MODE != kSumW) {
-            store_consts(lane, ca[0][0], ca[0][1], ca[0][2]);
-            store_consts(lane + 32, ca[1][0], ca[1][1], ca[1][2]);
+            store_consts(lane, ca[0]);
+            store_consts(lane + 32, ca[1]);
             for (int x = lane + 64; x < nr * Hp; x += 32) {  // many heads x many rows: the rest, plainly
-                float c0, c1, c2;
-                load_consts(x, c0, c1, c2);
-                store_consts(x, c0, c1, c2);
+                float c[5];
+                load_consts(x, c);
+                store_consts(x, c);
             }
         }
         __syncwarp();
 
         if constexpr (kDst || kSrc) {
-            if (mode_ == 0) {  // the first row that starts in this chunk (a continued row brought its vector along)
+            if (mode_ == 0 && !staged_now) {  // the first row that starts in this chunk (a continued row brought its vector along)
                 const int first = cont ? 1 : 0;
                 if (first < nr) request_rowvec(row0 + r + first, rvq_next);
             }
@@ -431,6 +474,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
         // will score itself (q = lane mod 32).
         constexpr bool kErAsyncMode = kFwdMode || kDst;
         const bool er_async = kErAsyncMode && (GEO ? true : a.hvec != 0);
+        const bool pre_group = er_async || staged_now;   // a commit group ahead of the ring's
         if constexpr (kErAsyncMode) {
             if (er_async) {
                 const unsigned sw_s = (unsigned)__cvta_generic_to_shared(sw);
@@ -440,9 +484,9 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                     for (int h = 0; h < H; h += 4)
                         cp_async16_s(sw_s + (unsigned)(((q << lgHp) + h) * 4), src + h, col >= 0 ? 16 : 0);
                 }
-                cp_async_commit();
             }
         }
+        if (pre_group) cp_async_commit();
         // ---- start the gather ring now: the first S slots need only the column ids ----------------
         auto issue = [&](int s_, unsigned dst_s) {
             const int col = lds_s32(sj_s + s_ * (EPW * 4));  // -1 past the row's / chunk's end: zero fill
@@ -453,11 +497,9 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
         };
 #pragma unroll
         for (int s_ = 0; s_ < S; ++s_) issue(s_, stage_s + s_ * (V * 512));
-        if constexpr (kErAsyncMode) {
-            if (er_async) {
-                cp_async_wait<S>();  // the score terms have landed (the ring's S groups may still be in flight)
-                __syncwarp();
-            }
+        if (pre_group) {
+            cp_async_wait<S>();  // the score terms and the staged rows have landed (the ring's S groups may still be in flight)
+            __syncwarp();
         }
 
         // ---- stage C: weight records, two positions per lane and sweep, all their heads -----------
@@ -690,7 +732,7 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
             const bool row_starts = !(cont && ri == 0);
             const bool row_ends = !(unfinished && ri == nr - 1);
             if constexpr (kDst || kSrc) {
-                if (mode_ == 0 && row_starts) {
+                if (mode_ == 0 && row_starts && !staged_now) {
 #pragma unroll
                     for (int v = 0; v < V; ++v) rvq[v] = rvq_next[v];
                     if (ri + 1 < nr) request_rowvec(row + 1, rvq_next);
@@ -859,6 +901,11 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                     }
                 } else {
                     float pA[V], pB[V], rv[V][EPV];
+                    if (staged_now) {
+#pragma unroll
+                        for (int v = 0; v < V; ++v)
+                            rvq[v] = vok[v] ? lds128(rowst_s + (unsigned)ri * rsb + (unsigned)((v * G + gl) * 16)) : make_uint4(0u, 0u, 0u, 0u);
+                    }
 #pragma unroll
                     for (int v = 0; v < V; ++v) {
                         Elem<T>::unpack(rvq[v], rv[v]);
@@ -887,10 +934,10 @@ __global__ void __launch_bounds__(kSpanThreads, MINB) span_kernel(const SpanArgs
                             DA += scratch[32 * V + lane * vph + k];
                         }
                         const float Sh = scratch[64 * V + lane];
-                        const float D = MODE == kBwdDstGivenD ? a.rec_in[row * H + lane].w : DA;
+                        const float D = MODE == kBwdDstGivenD ? (staged_now ? sc3[ri * Hp + lane] : a.rec_in[row * H + lane].w) : DA;
                         const float val = DB - D * Sh;
                         float *p = a.del + row * H + lane;
-                        *p = (flags_ & SAR_FIRST) ? val : *p + val;
+                        *p = (flags_ & SAR_FIRST) ? val : (staged_now ? sc4[ri * Hp + lane] : *p) + val;
                         if constexpr (MODE == kBwdDst)
                             a.rec_out[row * H + lane] = make_float4(sc0[ri * Hp + lane], sc1[ri * Hp + lane], sc2[ri * Hp + lane], D);
                     }
