@@ -307,8 +307,10 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
     a.sp = ma.sp;
     a.hvec = (H % 4 == 0) && sar_aligned(er_q, 16);
     const bool lean = lean_applies(s, flags, slope, g->split, g->n_src) && sar_aligned(er_q, 16);
+    // a partition step that neither opens nor closes the state
+    const bool lean_part = !first && !last && lean_shape_applies(s, slope, g->split, g->n_src) && sar_aligned(er_q, 16);
     LeanArgs la{};
-    if (lean) {
+    if (lean || lean_part) {
         la.n_rows = g->n_dst;
         la.indptr = g->indptr;
         la.indices = g->indices;
@@ -317,6 +319,7 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
         la.er = er_q;
         la.m_out = m;
         la.d_out = d;
+        la.acc_state = acc;
         la.out = out;
         la.relu = (flags & SAR_RELU_OUT) ? 1 : 0;
         la.slope = slope;
@@ -328,6 +331,8 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
         using T = typename C::type;
         if (lean)
             SAR_TRY(s.t == SAR_F32 ? lean_fwd_f32(s, la, g->nnz, st) : lean_fwd_bf16(s, la, g->nnz, st));
+        else if (lean_part)
+            SAR_TRY(s.t == SAR_F32 ? lean_fwd_part_f32(s, la, g->nnz, st) : lean_fwd_part_bf16(s, la, g->nnz, st));
         else
             SAR_TRY((launch_span<T, C::g, C::v, UFwd<C::v>::u, kFwd, kCapFwd, kMinBlocksFwd>(a, g->nnz, "gat_fwd", "gat_fwd_seg", st)));
         if (ma.sp.threshold > 0) {
@@ -537,8 +542,10 @@ sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, c
     s1.sp = sa.sp;
     s1.hvec = (H % 4 == 0);
 
-    const bool lean_dst = whole && lean_applies(s, flags, slope, g->split, g->n_src) && sar_aligned(er_q, 16);
-    const bool lean_src = whole && lean_applies(s, flags, slope, g->t_split, g->n_dst);
+    const bool lean_dst_shape = lean_shape_applies(s, slope, g->split, g->n_src) && sar_aligned(er_q, 16);
+    const bool lean_dst = whole && lean_dst_shape;
+    const bool lean_dst_part = !whole && lean_dst_shape;   // a partition step: D given, del collects
+    const bool lean_src = lean_shape_applies(s, slope, g->t_split, g->n_dst);   // whole graph or partition step alike
     LeanArgs ld{};
     LeanSrcArgs ls{};
     if (lean_src) {
@@ -555,7 +562,7 @@ sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, c
         ls.sp = sa.sp;
         ls.sp.threshold = g->t_split->threshold;
     }
-    if (lean_dst) {
+    if (lean_dst || lean_dst_part) {
         ld.n_rows = g->n_dst;
         ld.indptr = g->indptr;
         ld.indices = g->indices;
@@ -566,6 +573,8 @@ sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, c
         ld.m = m;
         ld.d = d;
         ld.rec_out = rec;
+        ld.rec_in = rec;
+        ld.first = (flags & SAR_FIRST) ? 1 : 0;
         ld.del = del;
         ld.slope = slope;
         ld.sp = da.sp;
@@ -590,7 +599,10 @@ sar_status sar_gat_bwd(const sar_part *g, const void *feat_q, const float *el, c
                     SAR_TRY(sar_after_launch());
                 }
             } else {
-                SAR_TRY((launch_span<T, C::g, C::v, U, kBwdDstGivenD, kCapDst, kMinBlocksBwd>(d1, g->nnz, "gat_bwd_dst", "gat_bwd_dst_seg", st)));
+                if (lean_dst_part)
+                    SAR_TRY(s.t == SAR_F32 ? lean_bwd_dst_part_f32(s, ld, g->nnz, st) : lean_bwd_dst_part_bf16(s, ld, g->nnz, st));
+                else
+                    SAR_TRY((launch_span<T, C::g, C::v, U, kBwdDstGivenD, kCapDst, kMinBlocksBwd>(d1, g->nnz, "gat_bwd_dst", "gat_bwd_dst_seg", st)));
                 if (da.sp.threshold > 0) {
                     auto merge = gat_bwd_dst_merge_kernel<T, C::g, C::v, true>;
                     SAR_TRY(ensure_smem(merge, msmem));

@@ -16,7 +16,10 @@ struct LeanArgs {
     const float *el, *er;    // el[row], er[col]
     const float *m, *d;      // bwd-dst: final statistics of the row
     float4 *rec_out;         // bwd-dst: record {el, m, 1/d, D} written per (row, head)
-    float *m_out, *d_out;    // forward
+    const float4 *rec_in;    // bwd-dst, partition step: the record written beforehand (D is read from it)
+    int first;               // bwd-dst, partition step: del starts here (else it adds to what is there)
+    float *m_out, *d_out;    // forward (a partition step reads the state there and writes it back)
+    float *acc_state;        // forward, partition step: running numerator [n_rows, H*F], float32
     void *out;               // forward: out
     float *del;              // bwd-dst
     float slope;
@@ -42,12 +45,12 @@ struct LeanSrcArgs {
 
 constexpr int kLeanCap = 256;   // edges a chunk stages; rows and segments must not exceed it
 
-// Do the lean kernels cover this call?  Whole graph in one call, slope >= 0, heads in groups of four, rows of
+// Do the lean kernels cover this shape?  Slope >= 0, heads in groups of four, rows of
 // exactly G*V vectors with V <= 2, the vectors of a head a power of two within one lane group, and a long-row
 // plan whose threshold fits a chunk (so that no row of the rows launch and no segment exceeds it), and a gathered
 // array of n_gathered rows whose 16-byte vectors can be counted in 32 bits (the staged row offsets are 32-bit).
-static inline bool lean_applies(const Shape &s, unsigned flags, float slope, const sar_split *sp, long long n_gathered) {
-    if (!s.fast || (flags & (SAR_FIRST | SAR_LAST | SAR_KEEP_NUMERATOR)) != (SAR_FIRST | SAR_LAST)) return false;
+static inline bool lean_shape_applies(const Shape &s, float slope, const sar_split *sp, long long n_gathered) {
+    if (!s.fast) return false;
     if (!(slope >= 0.f) || !sp || sp->threshold < 1 || sp->threshold > kLeanCap) return false;
     const int H = s.geom.H, nv = s.geom.n_vec;
     if (H % 4 != 0 || nv != s.G * s.V || s.V > 2 || nv % H != 0) return false;
@@ -57,12 +60,22 @@ static inline bool lean_applies(const Shape &s, unsigned flags, float slope, con
     return (s.G == 16 && s.V == 1 && H == 4) || (s.G == 32 && s.V == 1 && (H == 4 || H == 8)) ||
            (s.G == 32 && s.V == 2 && H == 4);
 }
+// ... and is the call one that holds the whole graph (the forward pass and the destination-major pass of a partition
+// step have variants of their own; the source-major pass is the same for both, a source lies in one partition)?
+static inline bool lean_applies(const Shape &s, unsigned flags, float slope, const sar_split *sp, long long n_gathered) {
+    if ((flags & (SAR_FIRST | SAR_LAST | SAR_KEEP_NUMERATOR)) != (SAR_FIRST | SAR_LAST)) return false;
+    return lean_shape_applies(s, slope, sp, n_gathered);
+}
 
 // Rows launch + segment launch of one pass.
 sar_status lean_fwd_f32(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
 sar_status lean_fwd_bf16(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
+sar_status lean_fwd_part_f32(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
+sar_status lean_fwd_part_bf16(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
 sar_status lean_bwd_dst_f32(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
 sar_status lean_bwd_dst_bf16(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
+sar_status lean_bwd_dst_part_f32(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
+sar_status lean_bwd_dst_part_bf16(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st);
 sar_status lean_bwd_src_f32(const Shape &s, const LeanSrcArgs &a, long long nnz, cudaStream_t st);
 sar_status lean_bwd_src_bf16(const Shape &s, const LeanSrcArgs &a, long long nnz, cudaStream_t st);
 

@@ -81,11 +81,14 @@ constexpr int kLeanMinBlocks = 8;
 // segment launches changes nothing (147.3 ms).
 constexpr int kLeanMinBlocksBwdRows = 24;
 
-static inline int lean_rows_per_span(long long n_rows, long long nnz, int cap) {
+// Resident blocks per SM the rows launch of a partition step is compiled for.
+constexpr int kLeanMinBlocksPart = 16;
+
+static inline int lean_rows_per_span(long long n_rows, long long nnz, int cap, int max_rows = kMaxSpanRows) {
     const double avg = n_rows > 0 ? (double)nnz / (double)n_rows : 0.0;
-    int R = avg > 0.5 ? (int)(1.0 * cap / avg + 0.5) : kMaxSpanRows;
+    int R = avg > 0.5 ? (int)(1.0 * cap / avg + 0.5) : max_rows;
     if (R < 1) R = 1;
-    if (R > kMaxSpanRows) R = kMaxSpanRows;
+    if (R > max_rows) R = max_rows;
     return R;
 }
 

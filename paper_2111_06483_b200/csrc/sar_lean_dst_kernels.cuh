@@ -6,6 +6,13 @@
 // the score terms er[col, :] of a stage's positions travelling with the stage (16 bytes per position and head group
 // into a small ring), the weights of a stage computed just before it is consumed, one (position, head) pair per lane.
 // Preconditions as for lean_src_kernel, on the CSR (checked by the host).
+//
+// PART = true is the same pass as one PARTITION STEP of Algorithm 2: the call holds the edges from one source partition,
+// D_i is given (it needs the whole row and was computed beforehand) and del_i collects <gout_i, B> - D_i S partition by
+// partition (rec_in, first).  Most of a row's edges lie in other partitions, so the rows are short and most have no
+// edge at all; the variant is laid out for that: spans of up to kLeanPartRows rows, rows without edges cost nothing
+// (no record, no write unless `first`), and the output-gradient rows of the chunk's rows that do have edges are copied
+// into shared memory with the chunk's first stage instead of being loaded row after row.
 #pragma once
 
 #include "sar_lean_src_kernels.cuh"
@@ -13,12 +20,15 @@
 namespace sar {
 
 
-template <int G, int V, int H, bool SEG, int CAP, int P, int NS>
+constexpr int kLeanPartRows = 31;    // rows per span of a partition step (one lane per row, one more for the end)
+constexpr int kLeanPartStaged = 16;  // rows with edges per chunk of a partition step (their own data is staged)
+
+template <int G, int V, int H, bool SEG, int CAP, int P, int NS, bool PART = false>
 struct LeanDstLayout {
     static constexpr int EPW = 32 / G;
     static constexpr int ROWB = G * V * 16;
     static constexpr int STAGE = P * ROWB;
-    static constexpr int MAXR = SEG ? 1 : kMaxSpanRows;
+    static constexpr int MAXR = SEG ? 1 : (PART ? kLeanPartRows : kMaxSpanRows);
     static constexpr int POSMAX = ((CAP + MAXR * (EPW - 1) + 31) / 32) * 32;
     static constexpr int RCN = ((MAXR * H * 4 + 15) / 16) * 16;
     static constexpr int MASKW = POSMAX / EPW / 32 + 1;
@@ -34,12 +44,14 @@ struct LeanDstLayout {
     static constexpr int srb = sout + 2 * RCN;
     static constexpr int sso = srb + ((MAXR + 1) * 4 + 15) / 16 * 16;
     static constexpr int endm = sso + ((MAXR + 1) * 4 + 15) / 16 * 16;
-    static constexpr int total = endm + ((MASKW * 4 + 15) / 16) * 16;
+    static constexpr int rowst = endm + ((MASKW * 4 + 15) / 16) * 16;   // partition step: gout of the rows with edges
+    static constexpr int total = rowst + ((PART && !SEG) ? kLeanPartStaged * ROWB : 0);
 };
 
-template <typename T, int G, int V, int H, bool SEG, int CAP, int P, int NS, int MINB>
+template <typename T, int G, int V, int H, bool SEG, int CAP, int P, int NS, int MINB, bool PART = false>
 __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
-    using L = LeanDstLayout<G, V, H, SEG, CAP, P, NS>;
+    static_assert(!(PART && SEG), "the segments of a partition step run the whole-graph segment kernel");
+    using L = LeanDstLayout<G, V, H, SEG, CAP, P, NS, PART>;
     constexpr int EPV = Elem<T>::EPV, NP = EPV / 2;
     constexpr int EPW = L::EPW, ROWB = L::ROWB, STAGE = L::STAGE;
     constexpr int NVEC = G * V, VPH = NVEC / H;
@@ -55,6 +67,7 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
     const unsigned sbase = (unsigned)__cvta_generic_to_shared(smem_raw);
     const unsigned ring_s = sbase + L::ring, rec_s = sbase + L::rec, w_s = sbase + L::w, offs_s = sbase + L::offs;
     const unsigned prow_s = sbase + L::prow, rc_s = sbase + L::rc, sout_s = sbase + L::sout, endm_s = sbase + L::endm;
+    const unsigned rowst_s = sbase + L::rowst;
     int *srb = reinterpret_cast<int *>(smem_raw + L::srb);
     int *sso = reinterpret_cast<int *>(smem_raw + L::sso);
 
@@ -149,7 +162,12 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
             }
             const unsigned later = excl_all & ~((1u << r) - 1u);
             const int stop = later ? __ffs(later) - 1 : nrows;
-            const unsigned fits = __ballot_sync(0xffffffffu, lane >= r && lane < stop && pre <= CAP);
+            bool ok = lane >= r && lane < stop && pre <= CAP;
+            if constexpr (PART) {   // and no more rows with edges than there is room for their staged data
+                const unsigned ne_all = __ballot_sync(0xffffffffu, deg_l > 0);
+                ok = ok && __popc(ne_all & ~((1u << r) - 1u) & ((2u << lane) - 1u)) <= kLeanPartStaged;
+            }
+            const unsigned fits = __ballot_sync(0xffffffffu, ok);
             r2 = r + __popc(fits);
             ne = __shfl_sync(0xffffffffu, pre, r2 - 1);
         }
@@ -218,15 +236,47 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
                     }
                 }
             }
-            for (int x = lane; x < nr * H; x += 32) {
-                const long long o = (row0 + r) * H + x;
-                const float mm = __ldg(a.m + o), dd = __ldg(a.d + o);
-                sts_f32(rc_s + 4 * x, __ldg(a.el + o));
-                sts_f32(rc_s + L::RCN + 4 * x, mm);
-                sts_f32(rc_s + 2 * L::RCN + 4 * x, dd > 0.f ? __fdividef(1.f, dd) : 0.f);
-                sts_f32(rc_s + 3 * L::RCN + 4 * x, -mm * kLog2e);
-                sts_f32(sout_s + 4 * x, 0.f);
-                sts_f32(sout_s + L::RCN + 4 * x, 0.f);
+            if constexpr (PART) {
+                // the constants of the rows with edges only, every load issued before the first store: el, m, d, the D
+                // given and del so far
+                constexpr int NX = (L::MAXR * H + 31) / 32;
+                float cv[NX][5];
+#pragma unroll
+                for (int n = 0; n < NX; ++n) {
+                    const int x = lane + 32 * n;
+                    cv[n][0] = cv[n][1] = cv[n][2] = cv[n][3] = cv[n][4] = 0.f;
+                    if (x < nr * H && ((nemask >> (x / H)) & 1u)) {
+                        const long long o = (row0 + r) * H + x;
+                        cv[n][0] = __ldg(a.el + o);
+                        cv[n][1] = __ldg(a.m + o);
+                        cv[n][2] = __ldg(a.d + o);
+                        cv[n][3] = __ldg(&a.rec_in[o].w);
+                        if (!a.first) cv[n][4] = a.del[o];   // plain load: this launch rewrites it
+                    }
+                }
+#pragma unroll
+                for (int n = 0; n < NX; ++n) {
+                    const int x = lane + 32 * n;
+                    if (x < nr * H) {
+                        sts_f32(rc_s + 4 * x, cv[n][0]);
+                        sts_f32(rc_s + L::RCN + 4 * x, cv[n][1]);
+                        sts_f32(rc_s + 2 * L::RCN + 4 * x, cv[n][2] > 0.f ? __fdividef(1.f, cv[n][2]) : 0.f);
+                        sts_f32(rc_s + 3 * L::RCN + 4 * x, -cv[n][1] * kLog2e);
+                        sts_f32(sout_s + 4 * x, cv[n][4]);
+                        sts_f32(sout_s + L::RCN + 4 * x, cv[n][3]);
+                    }
+                }
+            } else {
+                for (int x = lane; x < nr * H; x += 32) {
+                    const long long o = (row0 + r) * H + x;
+                    const float mm = __ldg(a.m + o), dd = __ldg(a.d + o);
+                    sts_f32(rc_s + 4 * x, __ldg(a.el + o));
+                    sts_f32(rc_s + L::RCN + 4 * x, mm);
+                    sts_f32(rc_s + 2 * L::RCN + 4 * x, dd > 0.f ? __fdividef(1.f, dd) : 0.f);
+                    sts_f32(rc_s + 3 * L::RCN + 4 * x, -mm * kLog2e);
+                    sts_f32(sout_s + 4 * x, 0.f);
+                    sts_f32(sout_s + L::RCN + 4 * x, 0.f);
+                }
             }
         }
         __syncwarp();
@@ -255,13 +305,24 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
                 cp_async16_full(rec_s + (unsigned)((j % NS) * L::RECB + lane * 16), a.er + (size_t)col * H + hq * 4);
             }
         };
+        if constexpr (PART) {   // the output-gradient rows of the rows with edges, in their order, with the first stage
+            unsigned todo = nemask;
+            unsigned dst = rowst_s + (unsigned)lane * 16u;
+            while (todo) {
+                const int i2 = __ffs(todo) - 1;
+                todo &= todo - 1;
+                const uint4 *src = reinterpret_cast<const uint4 *>(a.rowvec) + (row0 + r + i2) * NVEC;
+                for (int x = lane; x < NVEC; x += 32) cp_async16_full(dst + (unsigned)(x - lane) * 16u, src + x);
+                dst += ROWB;
+            }
+        }
 #pragma unroll
         for (int j = 0; j < NS; ++j) {
             if (j < nstages) issue_stage(j);
             cp_async_commit();
         }
 
-        if constexpr (!SEG) {
+        if constexpr (!SEG && !PART) {
             if (nslots > 0) request_rowvec(row0 + r + (__ffs(nemask) - 1), rvq_next);
         }
 
@@ -269,6 +330,7 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
         {
             int s = 0;
             int ri = SEG ? 0 : (__ffs(nemask) - 1);
+            unsigned staged_row = rowst_s + (unsigned)(gl * 16);   // partition step: gout of the row in progress
             for (int j = 0; j < nstages; ++j) {
                 cp_async_wait<NS - 1>();
                 __syncwarp();   // the records of this stage were copied by other lanes; the previous weights are consumed
@@ -323,14 +385,18 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
                         const f32x2 a2 = pack2(al, al), g2 = pack2(wg, wg);
 #pragma unroll
                         for (int t = 0; t < NP; ++t) {
-                            pacc0[v][t] = fma2(a2, x[t], pacc0[v][t]);
+                            if constexpr (!PART) pacc0[v][t] = fma2(a2, x[t], pacc0[v][t]);   // A is for D, given to a partition step
                             pacc1[v][t] = fma2(g2, x[t], pacc1[v][t]);
                         }
                     }
                     if (ends & (1u << k)) {
                         // ---- the row is complete -------------------------------------------------------------
                         const long long row = row0 + r + ri;
-                        if constexpr (!SEG) {
+                        if constexpr (PART) {
+#pragma unroll
+                            for (int v = 0; v < V; ++v) rvq[v] = lds128(staged_row + (unsigned)(v * G * 16));
+                            staged_row += ROWB;
+                        } else if constexpr (!SEG) {
 #pragma unroll
                             for (int v = 0; v < V; ++v) rvq[v] = rvq_next[v];
                             const unsigned rest = nemask & ~((2u << ri) - 1u);
@@ -379,7 +445,7 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
                                 f32x2 qa = zero2(), qb = zero2();
 #pragma unroll
                                 for (int t = 0; t < NP; ++t) {
-                                    qa = fma2(rv[t], pacc0[v][t], qa);
+                                    if constexpr (!PART) qa = fma2(rv[t], pacc0[v][t], qa);
                                     qb = fma2(rv[t], pacc1[v][t], qb);
                                 }
                                 pA[v] = qa.x + qa.y;
@@ -390,7 +456,7 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
                                 if (off < VPH || off >= G) {
 #pragma unroll
                                     for (int v = 0; v < V; ++v) {
-                                        pA[v] += __shfl_xor_sync(0xffffffffu, pA[v], off);
+                                        if constexpr (!PART) pA[v] += __shfl_xor_sync(0xffffffffu, pA[v], off);
                                         pB[v] += __shfl_xor_sync(0xffffffffu, pB[v], off);
                                         if (off >= G) sv[v] += __shfl_xor_sync(0xffffffffu, sv[v], off);
                                     }
@@ -399,8 +465,13 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
                             if ((gl % VPH) == 0 && half == 0) {
 #pragma unroll
                                 for (int v = 0; v < V; ++v) {
-                                    sts_f32(sout_s + (unsigned)((ri * H + hv[v]) * 4), pB[v] - pA[v] * sv[v]);   // del
-                                    sts_f32(sout_s + L::RCN + (unsigned)((ri * H + hv[v]) * 4), pA[v]);         // D
+                                    const unsigned so = sout_s + (unsigned)((ri * H + hv[v]) * 4);
+                                    if constexpr (PART) {   // del so far + this partition's share, with the D given
+                                        sts_f32(so, lds_f32(so) + (pB[v] - lds_f32(so + L::RCN) * sv[v]));
+                                    } else {
+                                        sts_f32(so, pB[v] - pA[v] * sv[v]);   // del
+                                        sts_f32(so + L::RCN, pA[v]);           // D
+                                    }
                                 }
                             }
                         }
@@ -430,9 +501,13 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
             __syncwarp();
             for (int x = lane; x < nr * H; x += 32) {
                 const long long o = (row0 + r) * H + x;
-                a.del[o] = lds_f32(sout_s + 4 * x);
-                a.rec_out[o] = make_float4(lds_f32(rc_s + 4 * x), lds_f32(rc_s + L::RCN + 4 * x),
-                                           lds_f32(rc_s + 2 * L::RCN + 4 * x), lds_f32(sout_s + L::RCN + 4 * x));
+                if constexpr (PART) {
+                    if (a.first || ((nemask >> (x / H)) & 1u)) a.del[o] = lds_f32(sout_s + 4 * x);
+                } else {
+                    a.del[o] = lds_f32(sout_s + 4 * x);
+                    a.rec_out[o] = make_float4(lds_f32(rc_s + 4 * x), lds_f32(rc_s + L::RCN + 4 * x),
+                                               lds_f32(rc_s + 2 * L::RCN + 4 * x), lds_f32(sout_s + L::RCN + 4 * x));
+                }
             }
             __syncwarp();
         }
@@ -464,6 +539,31 @@ static sar_status launch_lean_dst(LeanArgs a, long long nnz, cudaStream_t st) {
     return SAR_OK;
 }
 
+// A partition step: the rows launch is the PART variant, the segments of the long rows run the whole-graph segment
+// kernel (same partial records; the merge launch is the caller's and takes D as given).
+template <typename T, int G, int V, int H>
+static sar_status launch_lean_dst_part(LeanArgs a, long long nnz, cudaStream_t st) {
+    constexpr int NS = 2;
+    constexpr int P = (G == 32 && V == 1) ? 8 : 4 * (32 / G);
+    using LR = LeanDstLayout<G, V, H, false, kLeanCap, P, NS, true>;
+    using LS = LeanDstLayout<G, V, H, true, kLeanCap, P, NS>;
+    a.R = lean_rows_per_span(a.n_rows, nnz, kLeanCap, kLeanPartRows);
+    const long long spans = (a.n_rows + a.R - 1) / a.R;
+    if (spans > 0) {
+        auto kern = lean_dst_kernel<T, G, V, H, false, kLeanCap, P, NS, kLeanMinBlocksPart, true>;
+        SAR_TRY(ensure_smem(kern, LR::total));
+        SAR_LAUNCH("gat_bwd_dst", st, kern<<<(unsigned)spans, 32, LR::total, st>>>(a));
+        SAR_TRY(sar_after_launch());
+    }
+    if (a.sp.n_seg > 0) {
+        auto kern = lean_dst_kernel<T, G, V, H, true, kLeanCap, P, NS, kLeanMinBlocks>;
+        SAR_TRY(ensure_smem(kern, LS::total));
+        SAR_LAUNCH("gat_bwd_dst_seg", st, kern<<<(unsigned)a.sp.n_seg, 32, LS::total, st>>>(a));
+        SAR_TRY(sar_after_launch());
+    }
+    return SAR_OK;
+}
+
 template <typename T>
 static sar_status dispatch_lean_dst(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st) {
     if (s.G == 16 && s.V == 1 && s.geom.H == 4) return launch_lean_dst<T, 16, 1, 4>(a, nnz, st);
@@ -473,11 +573,23 @@ static sar_status dispatch_lean_dst(const Shape &s, const LeanArgs &a, long long
     return SAR_ERR_UNSUPPORTED;
 }
 
+template <typename T>
+static sar_status dispatch_lean_dst_part(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st) {
+    if (s.G == 16 && s.V == 1 && s.geom.H == 4) return launch_lean_dst_part<T, 16, 1, 4>(a, nnz, st);
+    if (s.G == 32 && s.V == 1 && s.geom.H == 4) return launch_lean_dst_part<T, 32, 1, 4>(a, nnz, st);
+    if (s.G == 32 && s.V == 1 && s.geom.H == 8) return launch_lean_dst_part<T, 32, 1, 8>(a, nnz, st);
+    if (s.G == 32 && s.V == 2 && s.geom.H == 4) return launch_lean_dst_part<T, 32, 2, 4>(a, nnz, st);
+    return SAR_ERR_UNSUPPORTED;
+}
+
 }  // namespace sar
 
-#define SAR_LEAN_DST_TU(SUFFIX, TYPE)                                                                     \
-    namespace sar {                                                                                       \
-    sar_status lean_bwd_dst_##SUFFIX(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st) { \
-        return dispatch_lean_dst<TYPE>(s, a, nnz, st);                                                    \
-    }                                                                                                     \
+#define SAR_LEAN_DST_TU(SUFFIX, TYPE)                                                                          \
+    namespace sar {                                                                                            \
+    sar_status lean_bwd_dst_##SUFFIX(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st) {      \
+        return dispatch_lean_dst<TYPE>(s, a, nnz, st);                                                         \
+    }                                                                                                          \
+    sar_status lean_bwd_dst_part_##SUFFIX(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st) { \
+        return dispatch_lean_dst_part<TYPE>(s, a, nnz, st);                                                    \
+    }                                                                                                          \
     }

@@ -14,18 +14,27 @@
 // (row, head) moves up to the stage's max and the accumulators follow by exp(c_before - c_now) (the running-max
 // correction of Sec. 3.4 applied inside a row), so nothing can overflow.
 // Preconditions as for lean_dst_kernel (checked by the host).
+//
+// PART = true is one PARTITION STEP of Algorithm 1 that is neither the first nor the last: the call holds the edges
+// from one source partition, and a row's sums are folded into the state the earlier partitions left - the running
+// max m, the denominator d and the float32 numerator, all against m - with the running-max correction of Sec. 3.4:
+// m' = max(m, m_k), numerator' = numerator exp(m - m') + numerator_k exp(c - m'), d likewise (c the shift the
+// partition's sums were taken against).  Laid out like the partition step of lean_dst_kernel: spans of up to
+// kLeanPartRows rows, rows without edges cost nothing and keep their state untouched, the state rows of the chunk's
+// rows that have edges are copied into shared memory with the chunk's first stage.
 #pragma once
 
 #include "sar_lean_dst_kernels.cuh"
 
 namespace sar {
 
-template <int G, int V, int H, bool SEG, int CAP, int P, int NS>
+template <int G, int V, int H, bool SEG, int CAP, int P, int NS, bool PART = false, int EPV = 4>
 struct LeanFwdLayout {
     static constexpr int EPW = 32 / G;
     static constexpr int ROWB = G * V * 16;
+    static constexpr int SROWB = G * V * EPV * 4;                 // a row of the float32 numerator
     static constexpr int STAGE = P * ROWB;
-    static constexpr int MAXR = SEG ? 1 : kMaxSpanRows;
+    static constexpr int MAXR = SEG ? 1 : (PART ? kLeanPartRows : kMaxSpanRows);
     static constexpr int POSMAX = ((CAP + MAXR * (EPW - 1) + 31) / 32) * 32;
     static constexpr int RCN = ((MAXR * H * 4 + 15) / 16) * 16;
     static constexpr int MASKW = POSMAX / EPW / 32 + 1;
@@ -41,12 +50,15 @@ struct LeanFwdLayout {
     static constexpr int srb = sout + RCN;
     static constexpr int sso = srb + ((MAXR + 1) * 4 + 15) / 16 * 16;
     static constexpr int endm = sso + ((MAXR + 1) * 4 + 15) / 16 * 16;
-    static constexpr int total = endm + ((MASKW * 4 + 15) / 16) * 16;
+    static constexpr int stm = endm + ((MASKW * 4 + 15) / 16) * 16;  // partition step: m and d of the state, in and out
+    static constexpr int rowst = stm + ((PART && !SEG) ? 2 * RCN : 0); // partition step: numerator rows of the rows with edges
+    static constexpr int total = rowst + ((PART && !SEG) ? kLeanPartStaged * SROWB : 0);
 };
 
-template <typename T, int G, int V, int H, bool SEG, int CAP, int P, int NS, int MINB>
+template <typename T, int G, int V, int H, bool SEG, int CAP, int P, int NS, int MINB, bool PART = false>
 __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
-    using L = LeanFwdLayout<G, V, H, SEG, CAP, P, NS>;
+    static_assert(!(PART && SEG), "the segments of a partition step run the whole-graph segment kernel");
+    using L = LeanFwdLayout<G, V, H, SEG, CAP, P, NS, PART, Elem<T>::EPV>;
     constexpr int EPV = Elem<T>::EPV, NP = EPV / 2;
     constexpr int EPW = L::EPW, ROWB = L::ROWB, STAGE = L::STAGE;
     constexpr int NVEC = G * V, VPH = NVEC / H;
@@ -63,6 +75,7 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
     const unsigned ring_s = sbase + L::ring, rec_s = sbase + L::rec, w_s = sbase + L::w, offs_s = sbase + L::offs;
     const unsigned prow_s = sbase + L::prow, rc_s = sbase + L::rc, sout_s = sbase + L::sout, endm_s = sbase + L::endm;
     const unsigned key_s = rc_s + L::RCN, cref_s = rc_s + 2 * L::RCN, ftab_s = rc_s + 3 * L::RCN;
+    const unsigned stm_s = sbase + L::stm, std_s = stm_s + L::RCN, rowst_s = sbase + L::rowst;
     int *srb = reinterpret_cast<int *>(smem_raw + L::srb);
     constexpr float kLeanMaxLead = 60.f;   // a score may exceed its row's shift by this much before the shift moves
     int *sso = reinterpret_cast<int *>(smem_raw + L::sso);
@@ -153,7 +166,12 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
             }
             const unsigned later = excl_all & ~((1u << r) - 1u);
             const int stop = later ? __ffs(later) - 1 : nrows;
-            const unsigned fits = __ballot_sync(0xffffffffu, lane >= r && lane < stop && pre <= CAP);
+            bool ok = lane >= r && lane < stop && pre <= CAP;
+            if constexpr (PART) {   // and no more rows with edges than there is room for their staged state
+                const unsigned ne_all = __ballot_sync(0xffffffffu, deg_l > 0);
+                ok = ok && __popc(ne_all & ~((1u << r) - 1u) & ((2u << lane) - 1u)) <= kLeanPartStaged;
+            }
+            const unsigned fits = __ballot_sync(0xffffffffu, ok);
             r2 = r + __popc(fits);
             ne = __shfl_sync(0xffffffffu, pre, r2 - 1);
         }
@@ -249,6 +267,17 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
                 cp_async16_full(rec_s + (unsigned)((j % NS) * L::RECB + lane * 16), a.er + (size_t)col * H + hq * 4);
             }
         };
+        if constexpr (PART) {   // the numerator rows of the rows with edges, in their order, with the first stage
+            unsigned todo = nemask;
+            unsigned dst = rowst_s + (unsigned)lane * 16u;
+            while (todo) {
+                const int i2 = __ffs(todo) - 1;
+                todo &= todo - 1;
+                const uint4 *src = reinterpret_cast<const uint4 *>(a.acc_state) + (row0 + r + i2) * (L::SROWB / 16);
+                for (int x = lane; x < L::SROWB / 16; x += 32) cp_async16_full(dst + (unsigned)(x - lane) * 16u, src + x);
+                dst += L::SROWB;
+            }
+        }
 #pragma unroll
         for (int j = 0; j < NS; ++j) {
             if (j < nstages) issue_stage(j);
@@ -257,6 +286,39 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
 
         // per (row, head): el, the shift c = score of the row's first edge, the key of the max (the loads fly with the
         // first stages)
+        if constexpr (PART) {
+            // rows with edges only, every load issued before the first store; and the state's m and d
+            constexpr int NX = (L::MAXR * H + 31) / 32;
+            float cv[NX][4];
+#pragma unroll
+            for (int n = 0; n < NX; ++n) {
+                const int x = lane + 32 * n;
+                cv[n][0] = 0.f;
+                cv[n][1] = cv[n][2] = SAR_NEG_INF;
+                cv[n][3] = 0.f;
+                if (x < nr * H && ((nemask >> (x / H)) & 1u)) {
+                    const long long o = (row0 + r) * H + x;
+                    const unsigned col = lds_u32(offs_s + 4 * (unsigned)perm(sso[x / H] * EPW)) >> LGNVEC;
+                    cv[n][0] = __ldg(a.el + o);
+                    cv[n][1] = __ldg(a.er + (size_t)col * H + (x % H));
+                    cv[n][2] = a.m_out[o];   // plain loads: this launch rewrites the state
+                    cv[n][3] = a.d_out[o];
+                }
+            }
+#pragma unroll
+            for (int n = 0; n < NX; ++n) {
+                const int x = lane + 32 * n;
+                if (x < nr * H) {
+                    float gr;
+                    sts_f32(rc_s + 4 * x, cv[n][0]);
+                    skey[x] = kKeyNegInf;
+                    sts_f32(cref_s + 4 * x, ((nemask >> (x / H)) & 1u) ? leaky(cv[n][0] + cv[n][1], a.slope, gr) : SAR_NEG_INF);
+                    sts_f32(sout_s + 4 * x, 0.f);
+                    sts_f32(stm_s + 4 * x, cv[n][2]);
+                    sts_f32(std_s + 4 * x, cv[n][3]);
+                }
+            }
+        } else
         for (int x = lane; x < nr * H; x += 32) {
             const int i = x / H;
             const float el_ = __ldg(a.el + (row0 + r) * H + x);
@@ -273,8 +335,9 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
         }
         __syncwarp();
 
-        // rows without edges: their vector outputs are zeros (the scalars leave with the others at the chunk's end)
-        if constexpr (!SEG) {
+        // rows without edges: their vector outputs are zeros (the scalars leave with the others at the chunk's end);
+        // in a partition step they keep their state
+        if constexpr (!SEG && !PART) {
             unsigned em = ~nemask & ((1u << nr) - 1u);
             while (em) {
                 const int i = __ffs(em) - 1;
@@ -288,6 +351,7 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
         {
             int s = 0;
             int ri = SEG ? 0 : (__ffs(nemask) - 1);
+            unsigned staged_row = rowst_s + (unsigned)(gl * EPV * 4);   // partition step: numerator of the row in progress
             float mrun = SAR_NEG_INF;               // segment: max of er[., lane % H] over the stages so far
             float el_seg = 0.f;
             if constexpr (SEG) el_seg = lds_f32(rc_s + 4 * (unsigned)hl);
@@ -459,6 +523,45 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
                                         pacc0[v][t] = fma2(o, pack2(1.f, 1.f), pacc0[v][t]);
                                     }
                                 }
+                            if constexpr (PART) {
+                                // fold into the state: m' = max(m, m_k); what was there scales by exp(m - m'), this
+                                // partition's sums (taken against the shift c) by exp(c - m')
+                                float mn[V], dn[V];
+                                float *sp_ = a.acc_state + row * (long long)(NVEC * EPV);
+#pragma unroll
+                                for (int v = 0; v < V; ++v) {
+                                    const unsigned rx = (unsigned)((ri * H + hv[v]) * 4);
+                                    float gr;
+                                    const float mk = leaky(lds_f32(rc_s + rx) + fkey_inv(lds_u32(key_s + rx)), a.slope, gr);
+                                    const float mo = lds_f32(stm_s + rx);
+                                    mn[v] = fmaxf(mo, mk);
+                                    const float fo = ex2_approx((mo - mn[v]) * kLog2e);
+                                    const float fn = ex2_approx((lds_f32(cref_s + rx) - mn[v]) * kLog2e);
+                                    dn[v] = lds_f32(std_s + rx) * fo + sv[v] * fn;
+                                    if (half == 0) {
+                                        const f32x2 fo2 = pack2(fo, fo), fn2 = pack2(fn, fn);
+                                        const unsigned so = staged_row + (unsigned)(v * G * EPV * 4);
+#pragma unroll
+                                        for (int q = 0; q < EPV / 4; ++q) {
+                                            const float4 old = lds_f4(so + 16 * q);
+                                            const f32x2 lo = fma2(pack2(old.x, old.y), fo2, fma2(pacc0[v][2 * q], fn2, zero2()));
+                                            const f32x2 hi = fma2(pack2(old.z, old.w), fo2, fma2(pacc0[v][2 * q + 1], fn2, zero2()));
+                                            reinterpret_cast<float4 *>(sp_ + (v * G + gl) * EPV)[q] = make_float4(lo.x, lo.y, hi.x, hi.y);
+                                        }
+                                    }
+                                }
+                                __syncwarp();   // every lane has read the state's m and d of this row
+                                if (half == 0) {
+#pragma unroll
+                                    for (int v = 0; v < V; ++v)
+                                        if ((gl % VPH) == 0) {
+                                            const unsigned rx = (unsigned)((ri * H + hv[v]) * 4);
+                                            sts_f32(std_s + rx, dn[v]);
+                                            sts_f32(stm_s + rx, mn[v]);
+                                        }
+                                }
+                                staged_row += L::SROWB;
+                            } else
                             if (half == 0) {
                                 uint4 *rp = reinterpret_cast<uint4 *>(a.out) + row * NVEC + gl;
 #pragma unroll
@@ -504,6 +607,15 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
         // ---- the chunk's row statistics, coalesced: m = LeakyReLU(el + max er), exactly the max of the row's scores ----
         if constexpr (!SEG) {
             __syncwarp();
+            if constexpr (PART) {
+                for (int x = lane; x < nr * H; x += 32) {
+                    if ((nemask >> (x / H)) & 1u) {
+                        const long long o = (row0 + r) * H + x;
+                        a.m_out[o] = lds_f32(stm_s + 4 * x);
+                        a.d_out[o] = lds_f32(std_s + 4 * x);
+                    }
+                }
+            } else
             for (int x = lane; x < nr * H; x += 32) {
                 const long long o = (row0 + r) * H + x;
                 const unsigned k = skey[x];
@@ -545,6 +657,40 @@ static sar_status launch_lean_fwd(LeanArgs a, long long nnz, cudaStream_t st) {
     return SAR_OK;
 }
 
+// A partition step that is neither the first nor the last: the rows launch is the PART variant, the segments of the long
+// rows run the whole-graph segment kernel (same partial records; the merge launch is the caller's and folds the state).
+template <typename T, int G, int V, int H>
+static sar_status launch_lean_fwd_part(LeanArgs a, long long nnz, cudaStream_t st) {
+    constexpr int NS = 2;
+    constexpr int P = (G == 32 && V == 1) ? 8 : 4 * (32 / G);
+    using LR = LeanFwdLayout<G, V, H, false, kLeanCap, P, NS, true, Elem<T>::EPV>;
+    using LS = LeanFwdLayout<G, V, H, true, kLeanCap, P, NS>;
+    a.R = lean_rows_per_span(a.n_rows, nnz, kLeanCap, kLeanPartRows);
+    const long long spans = (a.n_rows + a.R - 1) / a.R;
+    if (spans > 0) {
+        auto kern = lean_fwd_kernel<T, G, V, H, false, kLeanCap, P, NS, kLeanMinBlocksPart, true>;
+        SAR_TRY(ensure_smem(kern, LR::total));
+        SAR_LAUNCH("gat_fwd", st, kern<<<(unsigned)spans, 32, LR::total, st>>>(a));
+        SAR_TRY(sar_after_launch());
+    }
+    if (a.sp.n_seg > 0) {
+        auto kern = lean_fwd_kernel<T, G, V, H, true, kLeanCap, P, NS, kLeanMinBlocks>;
+        SAR_TRY(ensure_smem(kern, LS::total));
+        SAR_LAUNCH("gat_fwd_seg", st, kern<<<(unsigned)a.sp.n_seg, 32, LS::total, st>>>(a));
+        SAR_TRY(sar_after_launch());
+    }
+    return SAR_OK;
+}
+
+template <typename T>
+static sar_status dispatch_lean_fwd_part(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st) {
+    if (s.G == 16 && s.V == 1 && s.geom.H == 4) return launch_lean_fwd_part<T, 16, 1, 4>(a, nnz, st);
+    if (s.G == 32 && s.V == 1 && s.geom.H == 4) return launch_lean_fwd_part<T, 32, 1, 4>(a, nnz, st);
+    if (s.G == 32 && s.V == 1 && s.geom.H == 8) return launch_lean_fwd_part<T, 32, 1, 8>(a, nnz, st);
+    if (s.G == 32 && s.V == 2 && s.geom.H == 4) return launch_lean_fwd_part<T, 32, 2, 4>(a, nnz, st);
+    return SAR_ERR_UNSUPPORTED;
+}
+
 template <typename T>
 static sar_status dispatch_lean_fwd(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st) {
     if (s.G == 16 && s.V == 1 && s.geom.H == 4) return launch_lean_fwd<T, 16, 1, 4>(a, nnz, st);
@@ -556,9 +702,12 @@ static sar_status dispatch_lean_fwd(const Shape &s, const LeanArgs &a, long long
 
 }  // namespace sar
 
-#define SAR_LEAN_FWD_TU(SUFFIX, TYPE)                                                                  \
-    namespace sar {                                                                                    \
-    sar_status lean_fwd_##SUFFIX(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st) {  \
-        return dispatch_lean_fwd<TYPE>(s, a, nnz, st);                                                 \
-    }                                                                                                  \
+#define SAR_LEAN_FWD_TU(SUFFIX, TYPE)                                                                      \
+    namespace sar {                                                                                        \
+    sar_status lean_fwd_##SUFFIX(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st) {      \
+        return dispatch_lean_fwd<TYPE>(s, a, nnz, st);                                                     \
+    }                                                                                                      \
+    sar_status lean_fwd_part_##SUFFIX(const Shape &s, const LeanArgs &a, long long nnz, cudaStream_t st) { \
+        return dispatch_lean_fwd_part<TYPE>(s, a, nnz, st);                                                \
+    }                                                                                                      \
     }

@@ -313,6 +313,41 @@ def test_scores_far_above_a_rows_first_score(H, F, dtype):
     allclose_report(der.cpu().numpy(), b.der, 1e-4, 5e-4 * max(rms(b.der), 1.0), "der[far]")
 
 
+@pytest.mark.parametrize("H,F,dtype", [(4, 32, "bf16"), (4, 32, "f32"), (8, 32, "bf16"), (4, 64, "f32"), (4, 128, "bf16")])
+@pytest.mark.parametrize("K", [4, 16])
+def test_partition_steps_with_short_and_empty_rows(H, F, dtype, K):
+    """Call by call over K source partitions on the shapes that have kernels of their own for a partition step (the
+    forward steps between the first and the last, every destination-major step, every source-major step).  With K = 4
+    nearly every row has edges in every partition, so that a span of 31 rows holds more rows with edges than a chunk
+    stages and has to be cut; with K = 16 about half of the (row, partition) pairs are empty and must leave the state
+    as it is.  Hub rows go through the segment launches and the merge.  Forward and backward against the oracle."""
+    n, src, dst = hub_graph(n=5000, e=60000, d_max=800.0, seed=41)
+    p = Problem(n, src, dst, H, F, 91 + K, dtype=dtype, k=K, threshold=48, build_parts=True)
+    per_part = np.stack([np.diff(q.indptr.cpu().numpy()) for q in p.graph.parts])
+    assert (per_part == 0).any() and per_part.max() > 48
+    if K == 4:
+        assert ((per_part > 0).reshape(K, -1)[:, :n - n % 31].reshape(K, -1, 31).sum(-1) > 16).any()
+    _full_check(p, dtype=dtype, modes=("stateful",))
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_partition_steps_with_scores_far_above_the_first(dtype):
+    """The forward partition step takes a row's sums against the score of the row's first edge in that partition and
+    folds them into the state with exp(shift - new max): score terms of magnitude ~50 move the shift inside a step and
+    make the state's max jump from one partition to the next."""
+    n, src, dst = hub_graph(n=4000, e=60000, d_max=900.0, seed=21)
+    p = Problem(n, src, dst, 4, 32, 78, scale=25.0, dtype=dtype, k=8, threshold=48, build_parts=True)
+    f = p.oracle_fwd()
+    out, m, d = p.gpu_fwd("stateful")[:3]
+    assert torch.isfinite(out).all() and torch.isfinite(d).all()
+    if dtype == "f32":
+        allclose_report(out.float().cpu().numpy(), f.out, 1e-4, 2e-5, "out[far, steps]")
+    else:
+        check_out(out, f.out, dtype, "out[far, steps]")
+    allclose_report(m.cpu().numpy(), f.m, 1e-6, 1e-6, "m[far, steps]")
+    allclose_report(d.cpu().numpy(), f.d, 1e-4, 1e-6, "d[far, steps]")
+
+
 @pytest.mark.parametrize("slope", [0.0, 0.01, 1.0, -0.5])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_other_slopes(slope, dtype):
