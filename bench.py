@@ -160,13 +160,14 @@ def max_over_ranks(value: float, dist=None, device="cpu") -> float:
 
 
 def group_passes(kernels: dict) -> dict:
-    """Launch names -> passes: 'gat_fwd', 'gat_fwd_seg', 'gat_fwd_merge' together are one pass over the edges.
+    """Launch names -> passes: 'gat_fwd', 'gat_fwd_seg', 'gat_fwd_merge' (and, call by call, the 'gat_fwd_finalize' that
+    divides after the last partition) together are one pass over the edges.
     `ms` adds the launches' average durations (one launch of each per pass: the fused schedule); `total_ms`
     adds everything the pass's launches took inside the timed region (any schedule)."""
     passes = {}
     for name, v in kernels.items():
         base = name
-        for suffix in ("_seg", "_merge"):
+        for suffix in ("_seg", "_merge", "_finalize"):
             if name.endswith(suffix):
                 base = name[:-len(suffix)]
         p_ = passes.setdefault(base, {"ms": 0.0, "total_ms": 0.0, "launches": []})

@@ -307,8 +307,9 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
     a.sp = ma.sp;
     a.hvec = (H % 4 == 0) && sar_aligned(er_q, 16);
     const bool lean = lean_applies(s, flags, slope, g->split, g->n_src) && sar_aligned(er_q, 16);
-    // a partition step that neither opens nor closes the state
-    const bool lean_part = !first && !last && lean_shape_applies(s, slope, g->split, g->n_src) && sar_aligned(er_q, 16);
+    // A partition step that does not open the state.  The last one folds like the others and leaves the division to a
+    // launch of its own over all rows (most rows have no edge in a given partition, and every row has to be divided).
+    const bool lean_part = !first && lean_shape_applies(s, slope, g->split, g->n_src) && sar_aligned(er_q, 16);
     LeanArgs la{};
     if (lean || lean_part) {
         la.n_rows = g->n_dst;
@@ -335,8 +336,16 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
             SAR_TRY(s.t == SAR_F32 ? lean_fwd_part_f32(s, la, g->nnz, st) : lean_fwd_part_bf16(s, la, g->nnz, st));
         else
             SAR_TRY((launch_span<T, C::g, C::v, UFwd<C::v>::u, kFwd, kCapFwd, kMinBlocksFwd>(a, g->nnz, "gat_fwd", "gat_fwd_seg", st)));
+        const bool divide_after = lean_part && last;
         if (ma.sp.threshold > 0) {
-            SAR_LAUNCH("gat_fwd_merge", st, gat_fwd_merge_kernel<T, C::g, C::v><<<blocks_for(ma.sp.n_long, C::g), kThreads, 0, st>>>(ma));
+            FwdArgs mm = ma;
+            if (divide_after) mm.flags = 0;   // the long rows' state is folded like the others'
+            SAR_LAUNCH("gat_fwd_merge", st, gat_fwd_merge_kernel<T, C::g, C::v><<<blocks_for(mm.sp.n_long, C::g), kThreads, 0, st>>>(mm));
+            SAR_TRY(sar_after_launch());
+        }
+        if (divide_after) {
+            const long long nv = g->n_dst * (long long)s.geom.n_vec;
+            SAR_LAUNCH("gat_fwd_finalize", st, gat_fwd_finalize_kernel<T><<<(unsigned)((nv + 255) / 256), 256, 0, st>>>(ma));
             SAR_TRY(sar_after_launch());
         }
         return SAR_OK;

@@ -32,6 +32,34 @@ struct FwdArgs {
     int mode;           // 0: one group per row; 1: one group per long-row segment
 };
 
+// The end of Algorithm 1 on its own: out = numerator / d for every row (0 where d = 0), one thread per 16-byte vector
+// of `out`.  Follows a last partition step that left the complete state behind.
+template <typename T>
+__global__ void __launch_bounds__(256) gat_fwd_finalize_kernel(const FwdArgs a) {
+    constexpr int EPV = Elem<T>::EPV;
+    const long long vi = (long long)blockIdx.x * 256 + threadIdx.x;
+    if (vi >= a.n_dst * a.g.n_vec) return;
+    const long long row = vi / a.g.n_vec;
+    const int v = (int)(vi - row * a.g.n_vec);
+    const float dd = a.d[row * a.g.H + v / a.g.vph];
+    const float inv = dd > 0.f ? __fdividef(1.f, dd) : 0.f;
+    const float4 *src = reinterpret_cast<const float4 *>(a.acc) + vi * (EPV / 4);
+    float x[EPV];
+#pragma unroll
+    for (int q = 0; q < EPV / 4; ++q) {
+        const float4 t = src[q];
+        x[4 * q] = t.x * inv;
+        x[4 * q + 1] = t.y * inv;
+        x[4 * q + 2] = t.z * inv;
+        x[4 * q + 3] = t.w * inv;
+    }
+    if (a.flags & SAR_RELU_OUT) {
+#pragma unroll
+        for (int e = 0; e < EPV; ++e) x[e] = fmaxf(x[e], 0.f);
+    }
+    reinterpret_cast<uint4 *>(a.out)[vi] = Elem<T>::pack(x);
+}
+
 // Merge of the forward partials of the long rows: one group per long row folds its segments in
 // order with the same running-max rule, starting from the incoming state unless SAR_FIRST.
 template <typename T, int G, int V>
