@@ -21,7 +21,12 @@ namespace sar {
 
 
 constexpr int kLeanPartRows = 31;    // rows per span of a partition step (one lane per row, one more for the end)
-constexpr int kLeanPartStaged = 16;  // rows with edges per chunk of a partition step (their own data is staged)
+// Rows with edges per chunk of a partition step (their own data is staged): of the destination-major step (rows of the
+// storage type) and of the forward step (float32 numerator rows).  Measured on the large workload with 16 partitions,
+// per step: forward 4 / 8 / 16 rows 3.22 / 3.10 / 3.30 ms, destination-major with the source-major pass 8 / 16 / 31 rows
+// 3.57 / 3.47 / 4.04 ms (more staged rows cut fewer chunks short but leave fewer warps resident).
+constexpr int kLeanPartStaged = 16;
+constexpr int kLeanPartStagedFwd = 8;
 
 template <int G, int V, int H, bool SEG, int CAP, int P, int NS, bool PART = false>
 struct LeanDstLayout {

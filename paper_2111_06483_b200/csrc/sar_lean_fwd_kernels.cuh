@@ -52,7 +52,7 @@ struct LeanFwdLayout {
     static constexpr int endm = sso + ((MAXR + 1) * 4 + 15) / 16 * 16;
     static constexpr int stm = endm + ((MASKW * 4 + 15) / 16) * 16;  // partition step: m and d of the state, in and out
     static constexpr int rowst = stm + ((PART && !SEG) ? 2 * RCN : 0); // partition step: numerator rows of the rows with edges
-    static constexpr int total = rowst + ((PART && !SEG) ? kLeanPartStaged * SROWB : 0);
+    static constexpr int total = rowst + ((PART && !SEG) ? kLeanPartStagedFwd * SROWB : 0);
 };
 
 template <typename T, int G, int V, int H, bool SEG, int CAP, int P, int NS, int MINB, bool PART = false>
@@ -169,7 +169,7 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
             bool ok = lane >= r && lane < stop && pre <= CAP;
             if constexpr (PART) {   // and no more rows with edges than there is room for their staged state
                 const unsigned ne_all = __ballot_sync(0xffffffffu, deg_l > 0);
-                ok = ok && __popc(ne_all & ~((1u << r) - 1u) & ((2u << lane) - 1u)) <= kLeanPartStaged;
+                ok = ok && __popc(ne_all & ~((1u << r) - 1u) & ((2u << lane) - 1u)) <= kLeanPartStagedFwd;
             }
             const unsigned fits = __ballot_sync(0xffffffffu, ok);
             r2 = r + __popc(fits);
