@@ -233,7 +233,9 @@ SAR_API size_t sar_gat_workspace_bytes(const sar_part *g, int32_t H, int32_t F, 
 /* One step of Algorithm 1's loop: fold partition q into the running state.
  *   feat_q [n_src,H,F] (storage type t), el [n_dst,H], er_q [n_src,H].
  *   acc [n_dst,H,F] float32 running numerator, m [n_dst,H] running max, d [n_dst,H] running
- *   normaliser: read unless SAR_FIRST, written unless SAR_LAST (m, d are always written).
+ *   normaliser: read unless SAR_FIRST, written unless SAR_LAST (m, d are always written; after a call with
+ *   SAR_LAST and without SAR_KEEP_NUMERATOR the contents of acc are unspecified: the call may or may not have
+ *   completed the numerator there before dividing).
  *   With SAR_LAST, out [n_dst,H,F] (type t) = acc/d is written (0 where d == 0) and m, d hold the
  *   final statistics the backward pass needs.  With SAR_FIRST|SAR_LAST (one partition holding all
  *   sources) acc may be NULL: the numerator never leaves the registers.
