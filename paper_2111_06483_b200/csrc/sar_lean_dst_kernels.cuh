@@ -11,8 +11,9 @@
 // D_i is given (it needs the whole row and was computed beforehand) and del_i collects <gout_i, B> - D_i S partition by
 // partition (rec_in, first).  Most of a row's edges lie in other partitions, so the rows are short and most have no
 // edge at all; the variant is laid out for that: spans of up to kLeanPartRows rows, rows without edges cost nothing
-// (no record, no write unless `first`), and the output-gradient rows of the chunk's rows that do have edges are copied
-// into shared memory with the chunk's first stage instead of being loaded row after row.
+// (no record, no write unless `first`), the position -> row map is found by bisection, and the output-gradient rows of
+// the chunk's first kLeanPartStaged rows that do have edges are copied into shared memory with the chunk's first stage
+// instead of being loaded row after row (the rows beyond that load theirs when they complete).
 #pragma once
 
 #include "sar_lean_src_kernels.cuh"
@@ -21,11 +22,12 @@ namespace sar {
 
 
 constexpr int kLeanPartRows = 31;    // rows per span of a partition step (one lane per row, one more for the end)
-// Rows with edges per chunk of a partition step (their own data is staged): of the destination-major step (rows of the
-// storage type) and of the forward step (float32 numerator rows).  Measured on the large workload with 16 partitions,
-// per step: forward 4 / 8 / 16 rows 3.22 / 3.10 / 3.30 ms, destination-major with the source-major pass 8 / 16 / 31 rows
-// 3.57 / 3.47 / 4.04 ms (more staged rows cut fewer chunks short but leave fewer warps resident).
-constexpr int kLeanPartStaged = 16;
+// Rows with edges of a chunk of a partition step whose own data is staged (the chunk's first ones; the others load it
+// when they complete): of the destination-major step (rows of the storage type) and of the forward step (float32
+// numerator rows).  Measured on the large workload with 16 partitions, per step: forward 4 / 8 / 12 rows 3.07 / 2.98 /
+// 3.05 ms, destination-major with the source-major pass 8 / 12 / 16 rows 3.30 / 3.24 / 3.30 ms (more staged rows leave
+// fewer loads to wait for but fewer warps resident).
+constexpr int kLeanPartStaged = 12;
 constexpr int kLeanPartStagedFwd = 8;
 
 template <int G, int V, int H, bool SEG, int CAP, int P, int NS, bool PART = false>
@@ -167,12 +169,7 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
             }
             const unsigned later = excl_all & ~((1u << r) - 1u);
             const int stop = later ? __ffs(later) - 1 : nrows;
-            bool ok = lane >= r && lane < stop && pre <= CAP;
-            if constexpr (PART) {   // and no more rows with edges than there is room for their staged data
-                const unsigned ne_all = __ballot_sync(0xffffffffu, deg_l > 0);
-                ok = ok && __popc(ne_all & ~((1u << r) - 1u) & ((2u << lane) - 1u)) <= kLeanPartStaged;
-            }
-            const unsigned fits = __ballot_sync(0xffffffffu, ok);
+            const unsigned fits = __ballot_sync(0xffffffffu, lane >= r && lane < stop && pre <= CAP);
             r2 = r + __popc(fits);
             ne = __shfl_sync(0xffffffffu, pre, r2 - 1);
         }
@@ -220,7 +217,15 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
                 for (int u = 0; u < 2; ++u) {
                     const int q = q0 + 32 * u + lane;
                     if (q < npos) {
-                        if constexpr (!SEG) {
+                        if constexpr (PART) {   // many short rows: the position's row by bisection over the rows' first slots
+                            const int slot = q / EPW;
+                            int lo = 0, hi = nr;
+                            while (hi - lo > 1) {
+                                const int mid = (lo + hi) >> 1;
+                                if (sso[mid] <= slot) lo = mid; else hi = mid;
+                            }
+                            i = lo;
+                        } else if constexpr (!SEG) {
                             while (q >= sso[i + 1] * EPW) ++i;
                         }
                         const int t = srb[i] + (q - sso[i] * EPW);
@@ -310,10 +315,10 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
                 cp_async16_full(rec_s + (unsigned)((j % NS) * L::RECB + lane * 16), a.er + (size_t)col * H + hq * 4);
             }
         };
-        if constexpr (PART) {   // the output-gradient rows of the rows with edges, in their order, with the first stage
+        if constexpr (PART) {   // the output-gradient rows of the first rows with edges, in their order, with the first stage
             unsigned todo = nemask;
             unsigned dst = rowst_s + (unsigned)lane * 16u;
-            while (todo) {
+            for (int ci = 0; todo && ci < kLeanPartStaged; ++ci) {
                 const int i2 = __ffs(todo) - 1;
                 todo &= todo - 1;
                 const uint4 *src = reinterpret_cast<const uint4 *>(a.rowvec) + (row0 + r + i2) * NVEC;
@@ -336,6 +341,7 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
             int s = 0;
             int ri = SEG ? 0 : (__ffs(nemask) - 1);
             unsigned staged_row = rowst_s + (unsigned)(gl * 16);   // partition step: gout of the row in progress
+            int staged_left = kLeanPartStaged;                     // ... and how many more rows found room
             for (int j = 0; j < nstages; ++j) {
                 cp_async_wait<NS - 1>();
                 __syncwarp();   // the records of this stage were copied by other lanes; the previous weights are consumed
@@ -398,9 +404,14 @@ __global__ void __launch_bounds__(32, MINB) lean_dst_kernel(const LeanArgs a) {
                         // ---- the row is complete -------------------------------------------------------------
                         const long long row = row0 + r + ri;
                         if constexpr (PART) {
+                            if (staged_left > 0) {
 #pragma unroll
-                            for (int v = 0; v < V; ++v) rvq[v] = lds128(staged_row + (unsigned)(v * G * 16));
-                            staged_row += ROWB;
+                                for (int v = 0; v < V; ++v) rvq[v] = lds128(staged_row + (unsigned)(v * G * 16));
+                                staged_row += ROWB;
+                                --staged_left;
+                            } else {   // more rows with edges in this chunk than there was room for
+                                request_rowvec(row, rvq);
+                            }
                         } else if constexpr (!SEG) {
 #pragma unroll
                             for (int v = 0; v < V; ++v) rvq[v] = rvq_next[v];

@@ -20,8 +20,9 @@
 // max m, the denominator d and the float32 numerator, all against m - with the running-max correction of Sec. 3.4:
 // m' = max(m, m_k), numerator' = numerator exp(m - m') + numerator_k exp(c - m'), d likewise (c the shift the
 // partition's sums were taken against).  Laid out like the partition step of lean_dst_kernel: spans of up to
-// kLeanPartRows rows, rows without edges cost nothing and keep their state untouched, the state rows of the chunk's
-// rows that have edges are copied into shared memory with the chunk's first stage.
+// kLeanPartRows rows, rows without edges cost nothing and keep their state untouched, the numerator rows of the chunk's
+// first kLeanPartStagedFwd rows that have edges are copied into shared memory with the chunk's first stage (the rows
+// beyond that load theirs when they complete).
 #pragma once
 
 #include "sar_lean_dst_kernels.cuh"
@@ -166,12 +167,7 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
             }
             const unsigned later = excl_all & ~((1u << r) - 1u);
             const int stop = later ? __ffs(later) - 1 : nrows;
-            bool ok = lane >= r && lane < stop && pre <= CAP;
-            if constexpr (PART) {   // and no more rows with edges than there is room for their staged state
-                const unsigned ne_all = __ballot_sync(0xffffffffu, deg_l > 0);
-                ok = ok && __popc(ne_all & ~((1u << r) - 1u) & ((2u << lane) - 1u)) <= kLeanPartStagedFwd;
-            }
-            const unsigned fits = __ballot_sync(0xffffffffu, ok);
+            const unsigned fits = __ballot_sync(0xffffffffu, lane >= r && lane < stop && pre <= CAP);
             r2 = r + __popc(fits);
             ne = __shfl_sync(0xffffffffu, pre, r2 - 1);
         }
@@ -219,7 +215,15 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
                 for (int u = 0; u < 2; ++u) {
                     const int q = q0 + 32 * u + lane;
                     if (q < npos) {
-                        if constexpr (!SEG) {
+                        if constexpr (PART) {   // many short rows: the position's row by bisection over the rows' first slots
+                            const int slot = q / EPW;
+                            int lo = 0, hi = nr;
+                            while (hi - lo > 1) {
+                                const int mid = (lo + hi) >> 1;
+                                if (sso[mid] <= slot) lo = mid; else hi = mid;
+                            }
+                            i = lo;
+                        } else if constexpr (!SEG) {
                             while (q >= sso[i + 1] * EPW) ++i;
                         }
                         const int t = srb[i] + (q - sso[i] * EPW);
@@ -267,10 +271,10 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
                 cp_async16_full(rec_s + (unsigned)((j % NS) * L::RECB + lane * 16), a.er + (size_t)col * H + hq * 4);
             }
         };
-        if constexpr (PART) {   // the numerator rows of the rows with edges, in their order, with the first stage
+        if constexpr (PART) {   // the numerator rows of the first rows with edges, in their order, with the first stage
             unsigned todo = nemask;
             unsigned dst = rowst_s + (unsigned)lane * 16u;
-            while (todo) {
+            for (int ci = 0; todo && ci < kLeanPartStagedFwd; ++ci) {
                 const int i2 = __ffs(todo) - 1;
                 todo &= todo - 1;
                 const uint4 *src = reinterpret_cast<const uint4 *>(a.acc_state) + (row0 + r + i2) * (L::SROWB / 16);
@@ -352,6 +356,7 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
             int s = 0;
             int ri = SEG ? 0 : (__ffs(nemask) - 1);
             unsigned staged_row = rowst_s + (unsigned)(gl * EPV * 4);   // partition step: numerator of the row in progress
+            int staged_left = kLeanPartStagedFwd;                       // ... and how many more rows found room
             float mrun = SAR_NEG_INF;               // segment: max of er[., lane % H] over the stages so far
             float el_seg = 0.f;
             if constexpr (SEG) el_seg = lds_f32(rc_s + 4 * (unsigned)hl);
@@ -543,7 +548,9 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
                                         const unsigned so = staged_row + (unsigned)(v * G * EPV * 4);
 #pragma unroll
                                         for (int q = 0; q < EPV / 4; ++q) {
-                                            const float4 old = lds_f4(so + 16 * q);
+                                            // (more rows with edges in this chunk than there was room for: from memory)
+                                            const float4 old = staged_left > 0 ? lds_f4(so + 16 * q)
+                                                                               : reinterpret_cast<const float4 *>(sp_ + (v * G + gl) * EPV)[q];
                                             const f32x2 lo = fma2(pack2(old.x, old.y), fo2, fma2(pacc0[v][2 * q], fn2, zero2()));
                                             const f32x2 hi = fma2(pack2(old.z, old.w), fo2, fma2(pacc0[v][2 * q + 1], fn2, zero2()));
                                             reinterpret_cast<float4 *>(sp_ + (v * G + gl) * EPV)[q] = make_float4(lo.x, lo.y, hi.x, hi.y);
@@ -561,6 +568,7 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
                                         }
                                 }
                                 staged_row += L::SROWB;
+                                --staged_left;
                             } else
                             if (half == 0) {
                                 uint4 *rp = reinterpret_cast<uint4 *>(a.out) + row * NVEC + gl;
