@@ -307,9 +307,10 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
     a.sp = ma.sp;
     a.hvec = (H % 4 == 0) && sar_aligned(er_q, 16);
     const bool lean = lean_applies(s, flags, slope, g->split, g->n_src) && sar_aligned(er_q, 16);
-    // A partition step that does not open the state.  The last one folds like the others and leaves the division to a
+    // A partition step of a call-by-call pass.  The last one folds like the others and leaves the division to a
     // launch of its own over all rows (most rows have no edge in a given partition, and every row has to be divided).
-    const bool lean_part = !first && lean_shape_applies(s, slope, g->split, g->n_src) && sar_aligned(er_q, 16);
+    const bool lean_part = !(first && last) && lean_shape_applies(s, slope, g->split, g->n_src) && sar_aligned(er_q, 16) &&
+                           (!first || g->nnz < (long long)kLeanPartFirstMaxDegree * g->n_dst);
     LeanArgs la{};
     if (lean || lean_part) {
         la.n_rows = g->n_dst;
@@ -321,6 +322,7 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
         la.m_out = m;
         la.d_out = d;
         la.acc_state = acc;
+        la.first = first ? 1 : 0;
         la.out = out;
         la.relu = (flags & SAR_RELU_OUT) ? 1 : 0;
         la.slope = slope;

@@ -15,14 +15,18 @@
 // correction of Sec. 3.4 applied inside a row), so nothing can overflow.
 // Preconditions as for lean_dst_kernel (checked by the host).
 //
-// PART = true is one PARTITION STEP of Algorithm 1 that is neither the first nor the last: the call holds the edges
+// PART = true is one PARTITION STEP of Algorithm 1 that leaves the state behind (the last step does so too; the division
+// that ends the algorithm is then a launch of its own): the call holds the edges
 // from one source partition, and a row's sums are folded into the state the earlier partitions left - the running
 // max m, the denominator d and the float32 numerator, all against m - with the running-max correction of Sec. 3.4:
 // m' = max(m, m_k), numerator' = numerator exp(m - m') + numerator_k exp(c - m'), d likewise (c the shift the
 // partition's sums were taken against).  Laid out like the partition step of lean_dst_kernel: spans of up to
 // kLeanPartRows rows, rows without edges cost nothing and keep their state untouched, the numerator rows of the chunk's
 // first kLeanPartStagedFwd rows that have edges are copied into shared memory with the chunk's first stage (the rows
-// beyond that load theirs when they complete).
+// beyond that load theirs when they complete).  In the first step (`first`) there is no state to read, a row with edges
+// leaves its sums against its own max, and a row without edges gets the empty state (m = -inf, d = 0, numerator 0):
+// FIRST = true, which the host picks for a sparse first partition (fewer than kLeanPartFirstMaxDegree edges per row;
+// rows of a denser one are better served by span_kernel's whole-chunk score phase).
 #pragma once
 
 #include "sar_lean_dst_kernels.cuh"
@@ -56,9 +60,10 @@ struct LeanFwdLayout {
     static constexpr int total = rowst + ((PART && !SEG) ? kLeanPartStagedFwd * SROWB : 0);
 };
 
-template <typename T, int G, int V, int H, bool SEG, int CAP, int P, int NS, int MINB, bool PART = false>
+template <typename T, int G, int V, int H, bool SEG, int CAP, int P, int NS, int MINB, bool PART = false, bool FIRST = false>
 __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
     static_assert(!(PART && SEG), "the segments of a partition step run the whole-graph segment kernel");
+    static_assert(PART || !FIRST, "FIRST is the first partition step");
     using L = LeanFwdLayout<G, V, H, SEG, CAP, P, NS, PART, Elem<T>::EPV>;
     constexpr int EPV = Elem<T>::EPV, NP = EPV / 2;
     constexpr int EPW = L::EPW, ROWB = L::ROWB, STAGE = L::STAGE;
@@ -272,7 +277,7 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
             }
         };
         if constexpr (PART) {   // the numerator rows of the first rows with edges, in their order, with the first stage
-            unsigned todo = nemask;
+            unsigned todo = FIRST ? 0u : nemask;
             unsigned dst = rowst_s + (unsigned)lane * 16u;
             for (int ci = 0; todo && ci < kLeanPartStagedFwd; ++ci) {
                 const int i2 = __ffs(todo) - 1;
@@ -305,8 +310,10 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
                     const unsigned col = lds_u32(offs_s + 4 * (unsigned)perm(sso[x / H] * EPW)) >> LGNVEC;
                     cv[n][0] = __ldg(a.el + o);
                     cv[n][1] = __ldg(a.er + (size_t)col * H + (x % H));
-                    cv[n][2] = a.m_out[o];   // plain loads: this launch rewrites the state
-                    cv[n][3] = a.d_out[o];
+                    if constexpr (!FIRST) {
+                        cv[n][2] = a.m_out[o];   // plain loads: this launch rewrites the state
+                        cv[n][3] = a.d_out[o];
+                    }
                 }
             }
 #pragma unroll
@@ -340,7 +347,18 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
         __syncwarp();
 
         // rows without edges: their vector outputs are zeros (the scalars leave with the others at the chunk's end);
-        // in a partition step they keep their state
+        // in a partition step they keep their state, or get the empty one in the first step
+        if constexpr (PART) {
+            if constexpr (FIRST) {
+                unsigned em = ~nemask & ((1u << nr) - 1u);
+                while (em) {
+                    const int i = __ffs(em) - 1;
+                    em &= em - 1;
+                    uint4 *rp = reinterpret_cast<uint4 *>(a.acc_state) + (row0 + r + i) * (L::SROWB / 16);
+                    for (int x = lane; x < L::SROWB / 16; x += 32) rp[x] = make_uint4(0u, 0u, 0u, 0u);
+                }
+            }
+        }
         if constexpr (!SEG && !PART) {
             unsigned em = ~nemask & ((1u << nr) - 1u);
             while (em) {
@@ -549,8 +567,9 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
 #pragma unroll
                                         for (int q = 0; q < EPV / 4; ++q) {
                                             // (more rows with edges in this chunk than there was room for: from memory)
-                                            const float4 old = staged_left > 0 ? lds_f4(so + 16 * q)
-                                                                               : reinterpret_cast<const float4 *>(sp_ + (v * G + gl) * EPV)[q];
+                                            const float4 old = FIRST ? make_float4(0.f, 0.f, 0.f, 0.f)
+                                                               : staged_left > 0 ? lds_f4(so + 16 * q)
+                                                                                 : reinterpret_cast<const float4 *>(sp_ + (v * G + gl) * EPV)[q];
                                             const f32x2 lo = fma2(pack2(old.x, old.y), fo2, fma2(pacc0[v][2 * q], fn2, zero2()));
                                             const f32x2 hi = fma2(pack2(old.z, old.w), fo2, fma2(pacc0[v][2 * q + 1], fn2, zero2()));
                                             reinterpret_cast<float4 *>(sp_ + (v * G + gl) * EPV)[q] = make_float4(lo.x, lo.y, hi.x, hi.y);
@@ -617,7 +636,7 @@ __global__ void __launch_bounds__(32, MINB) lean_fwd_kernel(const LeanArgs a) {
             __syncwarp();
             if constexpr (PART) {
                 for (int x = lane; x < nr * H; x += 32) {
-                    if ((nemask >> (x / H)) & 1u) {
+                    if (FIRST || ((nemask >> (x / H)) & 1u)) {
                         const long long o = (row0 + r) * H + x;
                         a.m_out[o] = lds_f32(stm_s + 4 * x);
                         a.d_out[o] = lds_f32(std_s + 4 * x);
@@ -665,7 +684,7 @@ static sar_status launch_lean_fwd(LeanArgs a, long long nnz, cudaStream_t st) {
     return SAR_OK;
 }
 
-// A partition step that is neither the first nor the last: the rows launch is the PART variant, the segments of the long
+// A partition step of a call-by-call forward pass: the rows launch is the PART variant, the segments of the long
 // rows run the whole-graph segment kernel (same partial records; the merge launch is the caller's and folds the state).
 template <typename T, int G, int V, int H>
 static sar_status launch_lean_fwd_part(LeanArgs a, long long nnz, cudaStream_t st) {
@@ -676,8 +695,10 @@ static sar_status launch_lean_fwd_part(LeanArgs a, long long nnz, cudaStream_t s
     a.R = lean_rows_per_span(a.n_rows, nnz, kLeanCap, kLeanPartRows);
     const long long spans = (a.n_rows + a.R - 1) / a.R;
     if (spans > 0) {
-        auto kern = lean_fwd_kernel<T, G, V, H, false, kLeanCap, P, NS, kLeanMinBlocksPart, true>;
-        SAR_TRY(ensure_smem(kern, LR::total));
+        auto kern = a.first ? lean_fwd_kernel<T, G, V, H, false, kLeanCap, P, NS, kLeanMinBlocksPart, true, true>
+                            : lean_fwd_kernel<T, G, V, H, false, kLeanCap, P, NS, kLeanMinBlocksPart, true, false>;
+        SAR_TRY(ensure_smem(lean_fwd_kernel<T, G, V, H, false, kLeanCap, P, NS, kLeanMinBlocksPart, true, true>, LR::total));
+        SAR_TRY(ensure_smem(lean_fwd_kernel<T, G, V, H, false, kLeanCap, P, NS, kLeanMinBlocksPart, true, false>, LR::total));
         SAR_LAUNCH("gat_fwd", st, kern<<<(unsigned)spans, 32, LR::total, st>>>(a));
         SAR_TRY(sar_after_launch());
     }
