@@ -330,6 +330,25 @@ def test_partition_steps_with_short_and_empty_rows(H, F, dtype, K):
     _full_check(p, dtype=dtype, modes=("stateful",))
 
 
+@pytest.mark.parametrize("empty", ["first", "last", "middle"])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_partition_steps_over_partitions_without_edges(empty, dtype):
+    """Eight partitions of which some hold no edge at all (all sources lie in one part of the id range): the first step
+    then opens the empty state for every row, a middle step leaves every row as it is, the last step only divides.
+    Shape with partition-step kernels of its own; forward and backward against the oracle."""
+    n, e = 4000, 30000
+    src, dst = workloads.uniform_edges(n, e, 17, False)
+    lo, hi = {"first": (n // 2, n), "last": (0, n // 2), "middle": (0, n)}[empty]
+    src = (lo + src.long() % (hi - lo)).to(torch.int32)
+    if empty == "middle":   # sources in the first and the last quarter only
+        src = torch.where(src < n // 2, src // 2, n - 1 - (n - 1 - src) // 2).to(torch.int32)
+    p = Problem(n, src, dst, 4, 32, 19, dtype=dtype, k=8, threshold=48, build_parts=True)
+    nnz = [int(q.nnz) for q in p.graph.parts]
+    assert {"first": nnz[0] == 0 and nnz[-1] > 0, "last": nnz[-1] == 0 and nnz[0] > 0,
+            "middle": nnz[3] == 0 and nnz[4] == 0 and nnz[0] > 0 and nnz[-1] > 0}[empty], nnz
+    _full_check(p, dtype=dtype, modes=("stateful",))
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_partition_steps_with_scores_far_above_the_first(dtype):
     """The forward partition step takes a row's sums against the score of the row's first edge in that partition and
