@@ -310,7 +310,8 @@ sar_status sar_gat_fwd(const sar_part *g, const void *feat_q, const float *el, c
     // A partition step of a call-by-call pass.  The last one folds like the others and leaves the division to a
     // launch of its own over all rows (most rows have no edge in a given partition, and every row has to be divided).
     const bool lean_part = !(first && last) && lean_shape_applies(s, slope, g->split, g->n_src) && sar_aligned(er_q, 16) &&
-                           (!first || g->nnz < (long long)kLeanPartFirstMaxDegree * g->n_dst);
+                           (g->nnz < (long long)kLeanPartMaxDegree * g->n_dst ||
+                            (g->nnz >= (long long)kLeanPartMinDenseDegree * g->n_dst && !first));
     LeanArgs la{};
     if (lean || lean_part) {
         la.n_rows = g->n_dst;

@@ -44,9 +44,15 @@ struct LeanSrcArgs {
 };
 
 constexpr int kLeanCap = 256;   // edges a chunk stages; rows and segments must not exceed it
-// The first forward partition step takes the lean partition-step kernel when the partition holds fewer edges per row than
-// this (large workload, 0.94 edges per row: 5.8 -> 3.2 ms; medium workload, 6.3 edges per row: slower by a tenth).
-constexpr int kLeanPartFirstMaxDegree = 2;
+// A forward partition step takes the lean partition-step kernel when the partition holds fewer than kLeanPartMaxDegree
+// edges per row (mostly empty rows: what the kernel is laid out for) or at least kLeanPartMinDenseDegree (a span then
+// holds few rows, all or most of them with their numerator staged).  In between - short rows, nearly all with edges,
+// 31 of them per span but room for the numerators of 8 - span_kernel is faster.  Per step, partition-step kernel
+// against span_kernel: large workload (0.94 edges per row and partition) 3.0 against 6.1 ms, first step 3.1 against
+// 5.8 ms, last step 5.1 against 11.1 ms; dense workload (25 edges) 2.38 against 2.64 ms; medium workload (6.3 edges)
+// 2.05 against 1.93 ms, last step 2.59 against 2.01 ms.
+constexpr int kLeanPartMaxDegree = 2;
+constexpr int kLeanPartMinDenseDegree = 16;
 
 // Do the lean kernels cover this shape?  Slope >= 0, heads in groups of four, rows of
 // exactly G*V vectors with V <= 2, the vectors of a head a power of two within one lane group, and a long-row

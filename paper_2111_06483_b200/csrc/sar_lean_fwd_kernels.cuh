@@ -25,8 +25,7 @@
 // first kLeanPartStagedFwd rows that have edges are copied into shared memory with the chunk's first stage (the rows
 // beyond that load theirs when they complete).  In the first step (`first`) there is no state to read, a row with edges
 // leaves its sums against its own max, and a row without edges gets the empty state (m = -inf, d = 0, numerator 0):
-// FIRST = true, which the host picks for a sparse first partition (fewer than kLeanPartFirstMaxDegree edges per row;
-// rows of a denser one are better served by span_kernel's whole-chunk score phase).
+// FIRST = true.  Which partitions get these variants: kLeanPartMaxDegree, kLeanPartMinDenseDegree (sar_lean.cuh).
 #pragma once
 
 #include "sar_lean_dst_kernels.cuh"
