@@ -319,8 +319,10 @@ def test_partition_steps_with_short_and_empty_rows(H, F, dtype, K):
     """Call by call over K source partitions on the shapes that have kernels of their own for a partition step (the
     forward steps between the first and the last, every destination-major step, every source-major step).  With K = 4
     nearly every row has edges in every partition, so that a span of 31 rows holds more rows with edges than a chunk
-    stages and has to be cut; with K = 16 about half of the (row, partition) pairs are empty and must leave the state
-    as it is.  Hub rows go through the segment launches and the merge.  Forward and backward against the oracle."""
+    stages (the later ones load their own data when they complete; three edges per row and partition is also the density
+    at which the forward steps stay with the general kernel); with K = 16 about half of the (row, partition) pairs are
+    empty and must leave the state as it is, and the first and the last forward step take the partition-step kernel
+    too.  Hub rows go through the segment launches and the merge.  Forward and backward against the oracle."""
     n, src, dst = hub_graph(n=5000, e=60000, d_max=800.0, seed=41)
     p = Problem(n, src, dst, H, F, 91 + K, dtype=dtype, k=K, threshold=48, build_parts=True)
     per_part = np.stack([np.diff(q.indptr.cpu().numpy()) for q in p.graph.parts])
