@@ -351,6 +351,24 @@ def test_partition_steps_over_partitions_without_edges(empty, dtype):
     _full_check(p, dtype=dtype, modes=("stateful",))
 
 
+@pytest.mark.parametrize("edges_per_partition", [(80000, 3000, 20000, 70000), (3000, 20000, 2500, 18000)])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_partition_steps_of_mixed_density(edges_per_partition, dtype):
+    """Four partitions of 1000 sources with very different numbers of edges into the 4000 rows: the forward steps of a
+    partition with fewer than 2 or at least 16 edges per row take the partition-step kernel, the others the general
+    one, and the state must pass from one to the other unchanged in meaning (first / middle / last step of either
+    kind).  Forward and backward against the oracle."""
+    n = 4000
+    srcs, dsts = [], []
+    for q, e in enumerate(edges_per_partition):
+        s, d = workloads.uniform_edges(n, e, 23 + q, False)
+        srcs.append((1000 * q + s.long() % 1000).to(torch.int32))
+        dsts.append(d)
+    p = Problem(n, torch.cat(srcs), torch.cat(dsts), 4, 32, 29, dtype=dtype, k=4, threshold=48, build_parts=True)
+    assert [int(q.nnz) for q in p.graph.parts] == list(edges_per_partition)
+    _full_check(p, dtype=dtype, modes=("stateful",))
+
+
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_partition_steps_with_scores_far_above_the_first(dtype):
     """The forward partition step takes a row's sums against the score of the row's first edge in that partition and
