@@ -421,7 +421,11 @@ sar_status sar_gat_bwd_prepare(int64_t n_dst, int32_t H, int32_t F, sar_dtype t,
         using C = decltype(cfg);
         using T = typename C::type;
         const size_t smem = (size_t)kWarpsPerBlock * 32 * C::v * 4;
-        SAR_LAUNCH("gat_bwd_prepare", st, gat_bwd_prepare_kernel<T, C::g, C::v><<<blocks_for(n_dst, C::g), kThreads, smem, st>>>(a));
+        const unsigned blocks = blocks_for((n_dst + PrepRows<C::v>::n - 1) / PrepRows<C::v>::n, C::g);
+        if (acc_is_numerator)
+            SAR_LAUNCH("gat_bwd_prepare", st, gat_bwd_prepare_kernel<T, C::g, C::v, true><<<blocks, kThreads, smem, st>>>(a));
+        else
+            SAR_LAUNCH("gat_bwd_prepare", st, gat_bwd_prepare_kernel<T, C::g, C::v, false><<<blocks, kThreads, smem, st>>>(a));
         return sar_after_launch();
     });
 }

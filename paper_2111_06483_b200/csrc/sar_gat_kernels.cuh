@@ -389,43 +389,62 @@ struct PrepArgs {
     RowGeom g;
 };
 
-template <typename T, int G, int V>
+// A lane group takes PrepRows<V>::n consecutive rows and asks for all of their data before it reduces the first (one
+// row per group leaves too little in flight for a pass that only streams two arrays).  The loads carry no branch: a
+// row past the end reads the last row again and is dropped when it comes to writing.
+template <int V>
+struct PrepRows {
+    static constexpr int n = V == 1 ? 4 : (V == 2 ? 2 : 1);
+};
+
+template <typename T, int G, int V, bool NUMERATOR>
 __global__ void __launch_bounds__(kThreads) gat_bwd_prepare_kernel(const PrepArgs a) {
     constexpr int EPV = Elem<T>::EPV;
     constexpr int RPW = 32 / G;
+    constexpr int RPG = PrepRows<V>::n;
     extern __shared__ __align__(16) float smem[];
     const LaneId<G> id;
     float *scratch = smem + (size_t)id.warp * (32 * V) + id.gid * (G * V);
-    const long long row = ((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid;
-    const bool active = row < a.n_dst;
+    const long long row0 = (((long long)blockIdx.x * kWarpsPerBlock + id.warp) * RPW + id.gid) * RPG;
     const VecGeom<G, V> vg(a.g, id.gl);
     const int H = a.g.H;
-    float gv[V][EPV], ov[V][EPV], p[V];
+    const int hl = id.gl < H ? id.gl : 0;
+    float gv[RPG][V][EPV], ov[RPG][V][EPV], dd[RPG], el_[RPG], m_[RPG];
 #pragma unroll
-    for (int v = 0; v < V; ++v)
+    for (int j = 0; j < RPG; ++j) {
+        const long long row = row0 + j < a.n_dst ? row0 + j : a.n_dst - 1;
+        load_row_vec<T, G, V>(a.gout, row, a.g.n_vec, id.gl, vg.vok, gv[j]);
+        if constexpr (NUMERATOR) {
 #pragma unroll
-        for (int e = 0; e < EPV; ++e) gv[v][e] = ov[v][e] = 0.f;
-    if (active) {
-        load_row_vec<T, G, V>(a.gout, row, a.g.n_vec, id.gl, vg.vok, gv);
-        if (a.acc_is_numerator)
+            for (int v = 0; v < V; ++v)
+#pragma unroll
+                for (int e = 0; e < EPV; ++e) ov[j][v][e] = 0.f;
             load_acc_row<G, V, EPV>(reinterpret_cast<const float *>(a.out) + row * (long long)(a.g.n_vec * EPV), id.gl,
-                                    vg.vok, ov);
-        else
-            load_row_vec<T, G, V>(a.out, row, a.g.n_vec, id.gl, vg.vok, ov);
+                                    vg.vok, ov[j]);
+        } else {
+            load_row_vec<T, G, V>(a.out, row, a.g.n_vec, id.gl, vg.vok, ov[j]);
+        }
+        dd[j] = a.d[row * H + hl];
+        el_[j] = a.el[row * H + hl];
+        m_[j] = a.m[row * H + hl];
     }
 #pragma unroll
-    for (int v = 0; v < V; ++v) {
-        p[v] = 0.f;
+    for (int j = 0; j < RPG; ++j) {
+        const long long row = row0 + j;
+        float p[V];
 #pragma unroll
-        for (int e = 0; e < EPV; ++e) p[v] = fmaf(gv[v][e], ov[v][e], p[v]);
-    }
-    float D = head_sum<G, V>(scratch, p, vg.vok, id.gl, a.g);
-    if (active && id.gl < H) {
-        const float dd = a.d[row * H + id.gl];
-        const float inv = dd > 0.f ? 1.f / dd : 0.f;
-        if (a.acc_is_numerator) D *= inv;
-        if (a.D) a.D[row * H + id.gl] = D;
-        a.rec[row * H + id.gl] = make_float4(a.el[row * H + id.gl], a.m[row * H + id.gl], inv, D);
+        for (int v = 0; v < V; ++v) {
+            p[v] = 0.f;
+#pragma unroll
+            for (int e = 0; e < EPV; ++e) p[v] = fmaf(gv[j][v][e], ov[j][v][e], p[v]);
+        }
+        float D = head_sum<G, V>(scratch, p, vg.vok, id.gl, a.g);
+        if (row < a.n_dst && id.gl < H) {
+            const float inv = dd[j] > 0.f ? 1.f / dd[j] : 0.f;
+            if (NUMERATOR) D *= inv;
+            if (a.D) a.D[row * H + id.gl] = D;
+            a.rec[row * H + id.gl] = make_float4(el_[j], m_[j], inv, D);
+        }
     }
 }
 
