@@ -351,6 +351,15 @@ def test_partition_steps_over_partitions_without_edges(empty, dtype):
     _full_check(p, dtype=dtype, modes=("stateful",))
 
 
+@pytest.mark.parametrize("n,e,K", [(3, 7, 2), (31, 40, 3), (32, 45, 4), (63, 70, 5), (1000, 900, 3)])
+def test_partition_steps_on_tiny_graphs(n, e, K):
+    """Graphs of one or two spans of the partition-step kernels (31 rows each), with a ragged last span, fewer edges than
+    rows, more partitions than a row has edges."""
+    src, dst = workloads.uniform_edges(n, e, 3 + n, True)
+    p = Problem(n, src, dst, 4, 32, 7 + n, k=K, threshold=48, build_parts=True)
+    _full_check(p, modes=("stateful", "fused"))
+
+
 @pytest.mark.parametrize("edges_per_partition", [(80000, 3000, 20000, 70000), (3000, 20000, 2500, 18000)])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_partition_steps_of_mixed_density(edges_per_partition, dtype):
